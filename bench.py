@@ -1,0 +1,324 @@
+"""Benchmark of the SDLM block-decode step (attention + LM-head statistics + accept/commit).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2_d4] [--impl reference]
+
+A step is one pass of the whole hot path over one batch of synthetic block inputs.  The default
+workload is the batch-32, D=4, Qwen2.5-3B-shaped ragged step; the metric is committed tokens per
+second.  One JSON line is printed by rank 0.  With N > 1 (torchrun) every rank runs an independent
+replica of the workload on its own GPU (the path shards by sequence; there is no collective in the
+data path), so scaling is "weak" and `value` sums the tokens of all ranks over the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import sdlm_synth as syn  # noqa: E402
+
+METRIC, UNIT = "committed_tokens_per_s", "tokens/s"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=lambda: self.lines.extend(self.proc.stdout), daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.t.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_sample(wl: syn.Workload, n_seqs: int, w_bits=None, repeats: int = 1):
+    """Times the CPU oracle (as it stands) on the first n_seqs sequences of the workload's step."""
+    from oracle import sdlm_oracle as orc
+    sub = wl.with_(batch=n_seqs)
+    lengths = syn.prefix_lengths(wl)[:n_seqs]
+    w_bits = syn.lm_head_weight(wl) if w_bits is None else w_bits
+    num_pages, mpps = syn.pages_needed(sub, lengths)
+    s = wl.shape
+    prefix = [syn.prefix_kv(wl, b, int(lengths[b])) for b in range(n_seqs)]
+    x = syn.block_inputs(sub, w_bits, 0)
+    best, tokens = None, 0
+    for _ in range(repeats):
+        cache = orc.PagedKVCache(num_pages, s.page_size, s.n_kv_heads, s.head_dim, n_seqs, mpps,
+                                 syn.free_list_permutation(sub, num_pages))
+        for b in range(n_seqs):
+            cache.add_sequence_fast(b, *prefix[b])
+        t0 = time.perf_counter()
+        res = orc.decode_step(cache, range(n_seqs), x.q, x.k_blk, x.v_blk, x.hidden, w_bits, wl.tau)
+        dt = time.perf_counter() - t0
+        tokens = int(res.commit.accepted_len.sum())
+        best = dt if best is None else min(best, dt)
+    return tokens, best
+
+
+def run_reference(args, wl: syn.Workload):
+    """The reference arm: the CPU oracle timed on host cores, a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_seqs = min(wl.batch, 4)
+    w_bits = syn.lm_head_weight(wl)
+    times, tokens = [], 0
+    for i in range(args.warmup + args.steps):
+        tok, dt = oracle_sample(wl, n_seqs, w_bits)
+        if i >= args.warmup:
+            times.append(dt); tokens += tok
+    total = sum(times)
+    value = tokens / total
+    sample = f"oracle decode_step on the first {n_seqs} of {wl.batch} sequences ({n_seqs * wl.block} rows), fp64 numpy"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / max(1, args.steps),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": _config(wl), "gpu_launches": 0,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def _config(wl: syn.Workload, lengths=None):
+    s = wl.shape
+    c = {"workload": wl.name, "batch": wl.batch, "block_D": wl.block, "tau": wl.tau,
+         "shape": {"q_heads": s.n_q_heads, "kv_heads": s.n_kv_heads, "head_dim": s.head_dim, "hidden": s.hidden,
+                   "vocab": s.vocab, "page": s.page_size},
+         "prefix": [wl.prefix_lo, wl.prefix_hi], "s_max": round(wl.resolved_s_max(), 3), "seed": wl.seed,
+         "l2": "inputs larger than L2: the LM-head weight streamed each step exceeds the 126 MB L2"}
+    if lengths is not None:
+        c["prefix_tokens_total"] = int(np.sum(lengths))
+    return c
+
+
+def time_workload(torch, dp, wl, steps, warmup, n_blocks=4, per_call_events=True):
+    """Device-timed region of `steps` steps.  Returns dict with ms_per_step, tokens, lm-head call time."""
+    blocks = [dp.block(i) for i in range(n_blocks)]
+    out = dp.alloc_outputs()
+    stream = torch.cuda.current_stream()
+    acc_buf = torch.zeros((steps, wl.batch), dtype=torch.int32, device=dp.sd.device)   # gamma of every timed step
+    for i in range(warmup):
+        dp.step(blocks[i % n_blocks], wl.tau, out)
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    lm_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    at_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    launches0 = dp.sd.launch_count()
+    sd = dp.sd
+    ev0.record(stream)
+    for i in range(steps):
+        x = blocks[(warmup + i) % n_blocks]
+        at_ev[i][0].record(stream)
+        sd.block_attn(x.q, x.k_blk, x.v_blk, out.attn)
+        at_ev[i][1].record(stream)
+        lm_ev[i][0].record(stream)
+        sd.lmhead_confidence(x.hidden, dp.w_lm, out.token, out.p_top1, out.entropy)
+        lm_ev[i][1].record(stream)
+        sd.accept_commit(wl.tau, out.token, out.p_top1, out.entropy, x.k_blk, x.v_blk, 0, acc_buf[i], out.out_tokens)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1)
+    lm_ms = float(np.mean([a.elapsed_time(b) for a, b in lm_ev]))
+    at_ms = float(np.mean([a.elapsed_time(b) for a, b in at_ev]))
+    return {"ms_total": ms, "ms_per_step": ms / steps, "tokens": int(acc_buf.clamp(min=0).sum().item()), "lm_ms": lm_ms, "attn_ms": at_ms,
+            "launches": dp.sd.launch_count() - launches0}
+
+
+def time_e2e(torch, dp, wl, steps, warmup, n_blocks=4):
+    """Same metric through sdlm_decode_step_host: pinned host inputs copied in, results copied out, every step."""
+    s = wl.shape
+    B, D = wl.batch, wl.block
+    host = []
+    for i in range(n_blocks):
+        x = syn.block_inputs(wl, dp.w_bits, 100 + i)
+        f = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16).pin_memory()
+        host.append((f(x.q), f(x.k_blk), f(x.v_blk), f(x.hidden)))
+    attn = torch.empty((B, D, s.n_q_heads, s.head_dim), dtype=torch.bfloat16).pin_memory()
+    tok = torch.empty((B, D), dtype=torch.int32).pin_memory()
+    p = torch.empty((B, D), dtype=torch.float32).pin_memory()
+    acc = torch.empty(B, dtype=torch.int32).pin_memory()
+    out_tok = torch.empty((B, D), dtype=torch.int32).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in host[0])
+    d2h = sum(t.numel() * t.element_size() for t in (attn, tok, p, acc, out_tok))
+    for i in range(warmup):
+        dp.sd.decode_step_host(wl.tau, *host[i % n_blocks], dp.w_lm, attn, tok, p, None, acc, out_tok)
+    torch.cuda.synchronize()
+    tokens = 0
+    t0 = time.perf_counter()
+    for i in range(steps):
+        dp.sd.decode_step_host(wl.tau, *host[(warmup + i) % n_blocks], dp.w_lm, attn, tok, p, None, acc, out_tok)
+        tokens += int(acc.clamp(min=0).sum())
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    return {"value": tokens / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+            "ms_per_step": 1e3 * dt / steps}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg2_d4", choices=syn.workloads())
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--no-extra", action="store_true", help="skip the D=8 companion measurement and the CPU baseline")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    wl = syn.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+        return
+
+    import torch
+    import paper_2509_24007_b200 as pk
+    from paper_2509_24007_b200.harness import DeviceProblem
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl")
+    total_steps = args.steps + args.warmup
+    wl_run = wl.with_(steps=2 * total_steps + 8, seed=wl.seed + 1000 * rank)   # room in the pool for every commit
+    dp = DeviceProblem(wl_run, keep_prefix=False)
+    lengths = dp.lengths
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    barrier()
+    if rank == 0:
+        sampler.start()
+    res = time_workload(torch, dp, wl_run, args.steps, args.warmup)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total, tokens = res["ms_total"], res["tokens"]
+    if dist is not None:
+        t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+        n = torch.tensor([tokens], dtype=torch.int64, device="cuda")
+        dist.all_reduce(n, op=dist.ReduceOp.SUM)
+        tokens = int(n.item())
+    e2e = time_e2e(torch, dp, wl_run, max(3, args.steps // 2), 3)
+    if dist is not None:
+        t = torch.tensor([e2e["value"]], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        e2e["value"] = float(t.item())
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = _peaks()
+    s = wl.shape
+    lm_bytes = syn.lm_head_bytes(wl) + wl.rows * s.hidden * 2           # weight once + hidden rows once
+    kv_bytes = syn.kv_read_bytes(wl, lengths)
+    step_bytes = lm_bytes + kv_bytes + 2 * wl.rows * s.n_q_heads * s.head_dim * 2
+    lm_gbs = lm_bytes / (res["lm_ms"] * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": tokens / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": _config(wl, lengths),
+        "tokens_per_step": tokens / args.steps / world,
+        "gpu_launches": res["launches"],
+        "clocks": clocks,
+        "e2e": e2e,
+        "roofline": {"bound": "hbm", "kernel": "lmhead_umma_kernel (sdlm_lmhead_confidence: stripe kernel + 3 us merge)",
+                     "achieved": lm_gbs, "peak": peak, "unit": "GB/s", "frac": lm_gbs / peak,
+                     "peak_source": peak_src, "traffic": None, "algorithmic_bytes": lm_bytes,
+                     "launch_ms": res["lm_ms"]},
+        "step": {"algorithmic_bytes": step_bytes, "achieved_gbs": step_bytes / (ms_total / args.steps * 1e-3) / 1e9,
+                 "frac_of_peak": step_bytes / (ms_total / args.steps * 1e-3) / 1e9 / peak,
+                 "frac_of_8tbs": step_bytes / (ms_total / args.steps * 1e-3) / 1e9 / 8000.0,
+                 "attn_ms": res["attn_ms"], "attn_gbs": kv_bytes / (res["attn_ms"] * 1e-3) / 1e9, "lm_ms": res["lm_ms"]},
+    }
+    if not args.no_extra and world == 1:
+        if args.workload == "cfg2_d4":      # committed tokens/s is asked for at D=4 and D=8
+            wl8 = syn.CONFIGS["cfg2"].with_(steps=2 * total_steps + 8)
+            del dp
+            torch.cuda.empty_cache()
+            dp8 = DeviceProblem(wl8, keep_prefix=False)
+            r8 = time_workload(torch, dp8, wl8, max(5, args.steps // 2), 3)
+            line["extra"] = {wl8.name: {"value": r8["tokens"] / (r8["ms_total"] * 1e-3), "unit": UNIT,
+                                        "ms_per_step": r8["ms_per_step"], "lm_ms": r8["lm_ms"], "attn_ms": r8["attn_ms"]}}
+            del dp8
+        n_seqs = min(wl.batch, 4)
+        tok, dt = oracle_sample(wl, n_seqs)
+        line["cpu_baseline"] = {"value": tok / dt, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
+                                "sample": f"oracle decode_step on the first {n_seqs} of {wl.batch} sequences "
+                                          f"({n_seqs * wl.block} rows; {dt:.1f} s), fp64 numpy"}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,213 @@
+/*
+ * sdlm.h -- C ABI of the SDLM block-decode hot path for NVIDIA B200 (sm_100a).
+ *
+ * One decode step of Next Sequence Prediction (Sec. 3.2, Eq. 4; Sec. 3.4): a block of D
+ * positions X_T = [x^{i-1}, [m] x (D-1)] is run on top of the cached history x^{<(i-1)}:
+ *
+ *   (a) sdlm_block_attn         the D block rows attend to every cached token and, without a
+ *                               mask, to each other (single-block mask of Sec. 3.3);
+ *   (b) sdlm_lmhead_confidence  the D logit rows Z in R^{D x |V|} are reduced, without ever being
+ *                               stored, to the greedy token and its confidences (Eq. 8, Eq. 9);
+ *   (c) sdlm_accept_commit      gamma_tau (Eq. 7) tokens are emitted (Decode, Eq. 4) and their
+ *                               K/V appended to the paged cache;
+ *   (d) sdlm_kv_pages           bookkeeping of that paged cache (Fig. 2b "cached KV states").
+ *
+ * Conventions that hold for every call unless stated otherwise
+ *   - "device" pointers are CUDA global memory of the current device, owned by the caller; the
+ *     library keeps no reference to a per-call pointer once the call's work is enqueued.
+ *   - bf16 tensors are dense, row-major, innermost dimension last, 16-byte aligned.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Device calls are asynchronous: arguments are validated on the host (on error nothing is
+ *     enqueued and a code is returned), work is enqueued on `stream`, SDLM_OK is returned.
+ *   - Conditions only the device can see (free list exhausted, a sequence outgrowing
+ *     max_pages_per_seq) set a sticky device status word, readable with sdlm_device_status;
+ *     the affected sequence commits nothing and its accepted_len is -1.
+ *   - Nothing aborts, traps, prints or throws.  One context must not be used from two host
+ *     threads at once.  There is no CPU fallback: without a CUDA device every call fails.
+ *   - The library allocates no device memory: the KV pool and one workspace are handed to
+ *     sdlm_create (sizes from sdlm_pool_bytes / sdlm_workspace_bytes).
+ */
+#ifndef SDLM_H_
+#define SDLM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum sdlm_status {
+  SDLM_OK = 0,
+  SDLM_ERR_INVALID_ARG = 1,   /* null pointer, misaligned pointer, value out of range        */
+  SDLM_ERR_SHAPE = 2,         /* batch / block / rows exceed what the context was created for */
+  SDLM_ERR_UNSUPPORTED = 3,   /* a configuration this build has no kernel for                 */
+  SDLM_ERR_OUT_OF_PAGES = 4,  /* device status: free list exhausted                           */
+  SDLM_ERR_CUDA = 5,          /* a CUDA runtime / driver call failed                          */
+  SDLM_ERR_TIMEOUT = 6,       /* device status: a bounded wait inside a kernel ran out        */
+  SDLM_ERR_DEVICE_CHECK = 7,  /* device status: a sequence outgrew max_pages_per_seq          */
+  SDLM_ERR_WORKSPACE = 8      /* pool or workspace too small or misaligned                    */
+} sdlm_status;
+
+/* Which confidence drives gamma_tau: the softmax probability of the decoded token (Eq. 8) or
+ * one minus the entropy normalised by ln|V| (Eq. 9). */
+typedef enum sdlm_conf_mode { SDLM_CONF_LOGIT = 0, SDLM_CONF_ENTROPY = 1 } sdlm_conf_mode;
+
+typedef struct sdlm_config {
+  int32_t n_q_heads;          /* Hq                                                            */
+  int32_t n_kv_heads;         /* Hkv, divides Hq; (Hq/Hkv) * max_block <= 64                   */
+  int32_t head_dim;           /* d: 64 or 128                                                  */
+  int32_t hidden;             /* H: multiple of 8 (the tensor-core path needs a multiple of 64) */
+  int32_t vocab;              /* |V|: rows of the LM head                                      */
+  int32_t page_size;          /* tokens per cache page: 64                                     */
+  int32_t num_pages;          /* pages in the pool                                             */
+  int32_t max_batch;          /* sequence slots, and the largest `batch` of a call             */
+  int32_t max_pages_per_seq;  /* width of the page table                                       */
+  int32_t max_block;          /* largest D of a call: 1..8                                     */
+  float softmax_scale;        /* attention scale; 0 selects 1/sqrt(head_dim)                   */
+} sdlm_config;
+
+typedef struct sdlm_ctx sdlm_ctx; /* opaque */
+
+/* Bytes of device memory the KV pool / the workspace need for `cfg` (0 if cfg is invalid). */
+size_t sdlm_pool_bytes(const sdlm_config* cfg);
+size_t sdlm_workspace_bytes(const sdlm_config* cfg);
+
+/* Creates a context on the current device over caller-owned device memory: `kv_pool`
+ * (>= sdlm_pool_bytes, 1024-byte aligned; its internal layout is private to the library, read it
+ * through SDLM_KV_GATHER) and `workspace` (>= sdlm_workspace_bytes, 256-byte aligned).  The
+ * tables are reset (identity free list, no sequences) on the legacy default stream and the call
+ * returns after that completes.  Both buffers must outlive the context.
+ * Errors: INVALID_ARG, UNSUPPORTED (shape limits above), WORKSPACE, CUDA (no device / not sm_100). */
+sdlm_status sdlm_create(const sdlm_config* cfg, void* kv_pool, size_t kv_pool_bytes, void* workspace,
+                        size_t workspace_bytes, sdlm_ctx** out);
+void sdlm_destroy(sdlm_ctx* ctx);
+const char* sdlm_status_str(sdlm_status s);
+
+/* ---- (d) page bookkeeping -- the paper only says that cached KV states are reused (Fig. 2b,
+ * Sec. 3.2 "predictions are repeated starting from the previous step's end position"); paging,
+ * the free list and its order are this library's.
+ *
+ * The cache is a pool of pages of 64 tokens shared by all sequence slots.  Pages are handed out
+ * from a ring `free_list[num_pages]` at position free_head (mod num_pages); released pages are
+ * pushed at free_tail.  A page is taken only when a token actually lands on it, so the tables
+ * always equal those of one-token-at-a-time decoding. */
+typedef enum sdlm_kv_op {
+  SDLM_KV_RESET = 0,       /* forget all sequences; free list := args.free_list (HOST int32[num_pages],
+                              a permutation of 0..num_pages-1) or the identity when NULL            */
+  SDLM_KV_ADD_SEQ = 1,     /* start slot args.seq (must be empty) with args.length prefix tokens whose
+                              K and V are args.k / args.v: DEVICE bf16 [length, Hkv, d]; takes
+                              ceil(length/64) pages in free-list order                              */
+  SDLM_KV_RELEASE_SEQ = 2, /* push the pages of slot args.seq back on the ring, length := 0          */
+  SDLM_KV_QUERY = 3,       /* fill *result with device pointers to the live tables                   */
+  SDLM_KV_GATHER = 4,      /* copy the logical contents of slot args.seq to args.k_out / args.v_out:
+                              DEVICE bf16 [args.length, Hkv, d]; rows at or beyond the slot's current
+                              length are left untouched                                             */
+  SDLM_KV_EXPORT = 5,      /* synchronise `stream`, copy all tables to HOST args.host_buf            */
+  SDLM_KV_IMPORT = 6       /* restore tables from a HOST buffer written by EXPORT (same config)      */
+} sdlm_kv_op;
+
+typedef struct sdlm_kv_args {
+  int32_t seq;
+  int32_t length;
+  const void* k;             /* ADD_SEQ */
+  const void* v;             /* ADD_SEQ */
+  void* k_out;               /* GATHER  */
+  void* v_out;               /* GATHER  */
+  const int32_t* free_list;  /* RESET (host) */
+  void* host_buf;            /* EXPORT / IMPORT (host) */
+  size_t host_bytes;         /* size of host_buf; must be >= result.table_bytes */
+} sdlm_kv_args;
+
+typedef struct sdlm_kv_result {
+  int32_t* page_table;       /* device [max_batch, max_pages_per_seq], -1 = no page               */
+  int32_t* seq_len;          /* device [max_batch] tokens cached per slot                         */
+  int32_t* free_list;        /* device [num_pages] ring                                           */
+  uint32_t* free_head;       /* device: pages handed out so far (monotonic)                       */
+  uint32_t* free_tail;       /* device: pages ever put on the ring (monotonic)                    */
+  int32_t* device_status;    /* device [4]: {sticky sdlm_status, offending slot, detail, count}   */
+  size_t table_bytes;        /* bytes EXPORT writes / IMPORT reads                                */
+} sdlm_kv_result;
+
+/* `args` may be NULL for QUERY; `result` may be NULL except for QUERY.  ADD_SEQ / RELEASE_SEQ /
+ * GATHER / RESET are enqueued on `stream` (RESET copies args.free_list before returning).  A pool
+ * that runs dry during ADD_SEQ sets the device status OUT_OF_PAGES and leaves the slot empty.
+ * Errors: INVALID_ARG (null / slot or length out of range / short host buffer), CUDA. */
+sdlm_status sdlm_kv_pages(sdlm_ctx* ctx, sdlm_kv_op op, const sdlm_kv_args* args, sdlm_kv_result* result,
+                          void* stream);
+
+/* ---- (a) block-decode attention -- Sec. 3.3: A_uv = 1[v<=u] OR 1[u>=i and v>=i], rows u >= i.
+ * For batch row b (sequence slot seq_ids[b], or b when seq_ids is NULL), query head h, slot j:
+ *   out[b,j,h,:] = softmax_t( q[b,j,h,:] . K_t * scale ) V_t,  t over the slot's cached tokens
+ *   followed by the D rows k_blk[b,:,h/G,:], v_blk[b,:,h/G,:]  (G = Hq/Hkv; nothing is masked).
+ * q [batch, D, Hq, d], k_blk / v_blk [batch, D, Hkv, d], out [batch, D, Hq, d]: device bf16;
+ * seq_ids: device int32 [batch] or NULL.  Inputs are already position-encoded.  Scores, softmax
+ * and the weighted sum are fp32; out is rounded to bf16 (nearest even).  The cache is not modified.
+ * Uses workspace scratch: calls on one context must not overlap on the GPU.
+ * Errors: INVALID_ARG, SHAPE (batch > max_batch, D > max_block). */
+sdlm_status sdlm_block_attn(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, const void* q,
+                            const void* k_blk, const void* v_blk, void* out, void* stream);
+
+/* ---- (b) LM head -> softmax statistics -- Sec. 3.2 (Z in R^{D x |V|}), Eq. 8, Eq. 9.
+ * For each of `rows` hidden states: z = W h (|V| logits, fp32 accumulate, never stored);
+ *   token   = argmax_n z_n (lowest n on exact ties)
+ *   p_top1  = softmax(z)_token                                  (Eq. 8)
+ *   entropy = -sum_n p_n ln p_n   in nats                       (H_p of Eq. 9)
+ * hidden [rows, H] and w_lm [|V|, H]: device bf16 (w_lm is streamed once per call);
+ * token int32 [rows], p_top1 / entropy float [rows]: device, required;
+ * max_logit / lse (ln sum_n exp z_n) float [rows]: device, optional (NULL to skip).
+ * Uses workspace scratch: calls on one context must not overlap on the GPU.
+ * Errors: INVALID_ARG, SHAPE (rows > max_batch*max_block or rows < 1). */
+sdlm_status sdlm_lmhead_confidence(sdlm_ctx* ctx, int32_t rows, const void* hidden, const void* w_lm,
+                                   int32_t* token, float* p_top1, float* entropy, float* max_logit,
+                                   float* lse, void* stream);
+
+/* ---- (c) longest-prefix acceptance and commit -- Eq. 7 and Decode of Eq. 4.
+ * Per batch row b: c_k = p_top1[b,k] (LOGIT) or 1 - entropy[b,k]/ln|V| (ENTROPY);
+ *   gamma = max({ j in 1..D : prod_{k<=j} c_k >= tau } U {1})   (fp32 running product, in order)
+ * then, as gamma single-token appends in ascending b: K/V rows k_blk[b,t], v_blk[b,t], t < gamma,
+ * go to cache positions len..len+gamma-1 of slot seq_ids[b] (a page is taken from the ring when a
+ * position starts a new page), the slot's length grows by gamma, accepted_len[b] = gamma,
+ * out_tokens[b, 0..gamma) = token[b, 0..gamma) and out_tokens[b, gamma..D) = -1.
+ * token [batch,D] int32, p_top1 / entropy [batch,D] float, k_blk / v_blk [batch,D,Hkv,d] bf16,
+ * accepted_len [batch] int32, out_tokens [batch,D] int32: all device; seq_ids device or NULL
+ * (slots must be distinct).  tau: any finite float (tau <= 0 gives gamma = D, tau > 1 gives 1).
+ * Errors: INVALID_ARG, SHAPE.  Device status: OUT_OF_PAGES, DEVICE_CHECK (accepted_len = -1). */
+sdlm_status sdlm_accept_commit(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, float tau,
+                               sdlm_conf_mode mode, const int32_t* token, const float* p_top1,
+                               const float* entropy, const void* k_blk, const void* v_blk,
+                               int32_t* accepted_len, int32_t* out_tokens, void* stream);
+
+/* Synchronises `stream` and copies the sticky device status words to host_out[4]:
+ * {sdlm_status (0 = none), sequence slot of the first failure, detail, number of failures}.
+ * `clear` != 0 resets them afterwards. */
+sdlm_status sdlm_device_status(sdlm_ctx* ctx, int32_t* host_out, int32_t clear, void* stream);
+
+/* ---- whole step from host memory: (a) + (b) + (c) for callers whose block inputs live on the
+ * host.  Copies q, k_blk, v_blk [as above] and hidden [batch*D, H] from HOST memory (pinned for
+ * best speed), and seq_ids (HOST int32 [batch] or NULL), to workspace staging; runs the three
+ * calls on `stream`; copies attn_out [batch,D,Hq,d] bf16, token / p_top1 / entropy [batch*D],
+ * accepted_len [batch] and out_tokens [batch,D] back to HOST (any may be NULL to skip) and
+ * synchronises `stream` before returning.  w_lm stays a DEVICE pointer (model state).
+ * Errors: as the three calls, plus CUDA. */
+sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids_host,
+                                  float tau, sdlm_conf_mode mode, const void* q_host, const void* k_blk_host,
+                                  const void* v_blk_host, const void* hidden_host, const void* w_lm,
+                                  void* attn_out_host, int32_t* token_host, float* p_top1_host,
+                                  float* entropy_host, int32_t* accepted_len_host, int32_t* out_tokens_host,
+                                  void* stream);
+
+/* Tuning / test knobs (the paper has no counterpart).  SDLM_OPT_LMHEAD_KERNEL: which stripe kernel
+ * sdlm_lmhead_confidence uses: 0 = chosen from the shape (default), 1 = warp-level mma.sync
+ * kernel, 2 = tcgen05 / TMA kernel (the call then fails with UNSUPPORTED for rows > 256 or
+ * |V| < 16).  Errors: INVALID_ARG. */
+typedef enum sdlm_option { SDLM_OPT_LMHEAD_KERNEL = 0 } sdlm_option;
+sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t value);
+
+/* Number of kernels the library has launched through this context since it was created. */
+uint64_t sdlm_launch_count(const sdlm_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SDLM_H_ */

@@ -1,0 +1,588 @@
+// Host side of the C ABI plus the small table kernels: context, page bookkeeping (Fig. 2b's
+// cached KV states as a paged pool), longest-prefix acceptance and commit (Eq. 7, Eq. 4).
+#include "sdlm_internal.h"
+
+#include <math.h>
+#include <new>
+#include <string.h>
+
+namespace sdlm {
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool config_valid(const sdlm_config& c) {
+  if (c.n_q_heads < 1 || c.n_kv_heads < 1 || c.n_q_heads % c.n_kv_heads) return false;
+  if (c.head_dim != 64 && c.head_dim != 128) return false;
+  if (c.hidden < 8 || c.hidden % 8) return false;
+  if (c.vocab < 1) return false;
+  if (c.page_size != kPageSize) return false;
+  if (c.num_pages < 1 || c.max_pages_per_seq < 1) return false;
+  if (c.max_batch < 1 || c.max_batch > kMaxBatch) return false;
+  if (c.max_block < 1 || c.max_block > kMaxBlock) return false;
+  if ((c.n_q_heads / c.n_kv_heads) * c.max_block > kMaxQRows) return false;
+  if (!(c.softmax_scale >= 0.0f) || isinf(c.softmax_scale)) return false;
+  return true;
+}
+
+WorkspaceLayout workspace_layout(const sdlm_config& c) {
+  WorkspaceLayout L{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t rows = (size_t)c.max_batch * c.max_block;
+  L.hdr = take(sizeof(DevHeader));
+  L.page_table = take((size_t)c.max_batch * c.max_pages_per_seq * 4);
+  L.seq_len = take((size_t)c.max_batch * 4);
+  L.free_list = take((size_t)c.num_pages * 4);
+  L.table_end = off;
+  L.lm_partials = take((size_t)kLmMaxStripes * rows * 16);
+  const int G = c.n_q_heads / c.n_kv_heads;
+  L.q_rows_pad = (G * c.max_block + 15) / 16 * 16;
+  L.attn_max_items = kAttnTargetItems + c.max_batch * c.n_kv_heads;
+  L.attn_ml = take((size_t)L.attn_max_items * L.q_rows_pad * 2 * 4);
+  L.attn_o = take((size_t)L.attn_max_items * L.q_rows_pad * c.head_dim * 4);
+  L.st_q = take(rows * c.n_q_heads * c.head_dim * 2);
+  L.st_k = take(rows * c.n_kv_heads * c.head_dim * 2);
+  L.st_v = take(rows * c.n_kv_heads * c.head_dim * 2);
+  L.st_hidden = take(rows * c.hidden * 2);
+  L.st_out = take(rows * c.n_q_heads * c.head_dim * 2);
+  L.st_seq_ids = take((size_t)c.max_batch * 4);
+  L.st_token = take(rows * 4);
+  L.st_p = take(rows * 4);
+  L.st_ent = take(rows * 4);
+  L.st_acc = take((size_t)c.max_batch * 4);
+  L.st_out_tokens = take(rows * 4);
+  L.total = off;
+  return L;
+}
+
+// ---------------------------------------------------------------------------------------------
+// table kernels
+// ---------------------------------------------------------------------------------------------
+__global__ void reset_tables_kernel(DevHeader* hdr, int32_t* page_table, int32_t* seq_len, int32_t* free_list,
+                                    int n_table, int max_batch, int num_pages, int identity) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  const int stride = gridDim.x * blockDim.x;
+  for (int k = i; k < n_table; k += stride) page_table[k] = -1;
+  for (int k = i; k < max_batch; k += stride) seq_len[k] = 0;
+  if (identity)
+    for (int k = i; k < num_pages; k += stride) free_list[k] = k;
+  if (i == 0) {
+    hdr->status[0] = hdr->status[1] = hdr->status[2] = hdr->status[3] = 0;
+    hdr->free_head = 0;
+    hdr->free_tail = (uint32_t)num_pages;
+    hdr->commit_ticket = 0;
+    hdr->lm_ticket = 0;
+  }
+}
+
+__device__ inline void report_status(DevHeader* hdr, int code, int slot, int detail) {
+  if (atomicCAS(&hdr->status[0], 0, code) == 0) {
+    hdr->status[1] = slot;
+    hdr->status[2] = detail;
+  }
+  atomicAdd(&hdr->status[3], 1);
+}
+
+// One CTA: hands ceil(length/64) pages to an empty slot, in free-list order.
+__global__ void add_seq_alloc_kernel(DevHeader* hdr, int32_t* page_table, int32_t* seq_len,
+                                     const int32_t* free_list, int slot, int length, int mpps, int num_pages) {
+  __shared__ int ok;
+  const uint32_t head = hdr->free_head, tail = hdr->free_tail;
+  const int n = (length + kPageSize - 1) / kPageSize;
+  if (threadIdx.x == 0) {
+    ok = 1;
+    if (seq_len[slot] != 0) { ok = 0; report_status(hdr, SDLM_ERR_DEVICE_CHECK, slot, seq_len[slot]); }
+    else if ((uint32_t)n > tail - head) { ok = 0; report_status(hdr, SDLM_ERR_OUT_OF_PAGES, slot, n); }
+  }
+  __syncthreads();
+  if (!ok) return;
+  for (int i = threadIdx.x; i < n; i += blockDim.x)
+    page_table[(size_t)slot * mpps + i] = free_list[(head + i) % (uint32_t)num_pages];
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    hdr->free_head = head + n;
+    seq_len[slot] = length;
+  }
+}
+
+// Scatter (to_pool = 1) or gather (to_pool = 0) 16-byte chunks between a dense [length, Hkv, d]
+// tensor and the slot's pages.  Does nothing unless the slot holds at least the rows it touches.
+__global__ void kv_rows_kernel(__nv_bfloat16* pool, const int32_t* page_table, const int32_t* seq_len,
+                               __nv_bfloat16* k_dense, __nv_bfloat16* v_dense, int slot, int length, int mpps,
+                               int Hkv, int d, int to_pool) {
+  const int cpr = d / 8;  // 16-byte chunks per row
+  const int have = seq_len[slot];
+  if (to_pool && have != length) return;
+  const int n_rows = to_pool ? length : min(length, have);
+  const size_t total = (size_t)n_rows * Hkv * 2 * cpr;
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (size_t)gridDim.x * blockDim.x) {
+    const int c = (int)(idx % cpr);
+    size_t r = idx / cpr;
+    const int kv = (int)(r % 2); r /= 2;
+    const int h = (int)(r % Hkv);
+    const int t = (int)(r / Hkv);
+    const int page = page_table[(size_t)slot * mpps + t / kPageSize];
+    const int row = t % kPageSize;
+    uint4* pool_p = reinterpret_cast<uint4*>(pool + kv_tile_offset(page, h, kv, Hkv, d) + (size_t)row * d) +
+                    kv_swizzled_chunk(row, c);
+    uint4* dense_p = reinterpret_cast<uint4*>((kv ? v_dense : k_dense) + ((size_t)t * Hkv + h) * d) + c;
+    if (to_pool) *pool_p = *dense_p; else *dense_p = *pool_p;
+  }
+}
+
+__global__ void release_seq_kernel(DevHeader* hdr, int32_t* page_table, int32_t* seq_len, int32_t* free_list,
+                                   int slot, int mpps, int num_pages) {
+  const int n = (seq_len[slot] + kPageSize - 1) / kPageSize;
+  const uint32_t tail = hdr->free_tail;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    free_list[(tail + i) % (uint32_t)num_pages] = page_table[(size_t)slot * mpps + i];
+    page_table[(size_t)slot * mpps + i] = -1;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    hdr->free_tail = tail + n;
+    seq_len[slot] = 0;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// (c) longest-prefix acceptance + commit -- Eq. 7, Decode of Eq. 4
+// ---------------------------------------------------------------------------------------------
+struct CommitParams {
+  DevHeader* hdr;
+  int32_t* page_table;
+  int32_t* seq_len;
+  const int32_t* free_list;
+  __nv_bfloat16* pool;
+  const int32_t* seq_ids;
+  const int32_t* token;
+  const float* p_top1;
+  const float* entropy;
+  const __nv_bfloat16* k_blk;
+  const __nv_bfloat16* v_blk;
+  int32_t* accepted_len;
+  int32_t* out_tokens;
+  float tau, inv_ln_vocab;
+  int mode, batch, D, Hkv, d, mpps, num_pages;
+};
+
+// gamma = max({ j : prod_{k<=j} c_k >= tau } U {1}); the product is taken in fp32, in order, and
+// every j is tested (the literal set, not an early exit).
+__device__ inline int gamma_tau(const CommitParams& p, int row) {
+  float prod = 1.0f;
+  int g = 1;
+  for (int k = 0; k < p.D; ++k) {
+    float c = (p.mode == SDLM_CONF_LOGIT) ? p.p_top1[row * p.D + k]
+                                          : __fsub_rn(1.0f, __fmul_rn(p.entropy[row * p.D + k], p.inv_ln_vocab));
+    prod = __fmul_rn(prod, c);
+    if (prod >= p.tau) g = k + 1;
+  }
+  return g;
+}
+
+constexpr int kCommitThreads = 256;
+
+// Grid = batch CTAs.  Every CTA derives gamma and the page demand of ALL rows from the same
+// snapshot of the tables (so the hand-out order is ascending batch row, as one-at-a-time decoding
+// would give), then scatters its own row's K/V.  The tables other CTAs read (seq_len, free_head)
+// are only written by whichever CTA finishes its reads last ("last CTA done" ticket; nobody waits).
+__global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitParams p) {
+  __shared__ int8_t s_gamma[kMaxBatch];
+  __shared__ int8_t s_state[kMaxBatch];  // 0 ok, 1 capacity failure, 2 out of pages
+  __shared__ int s_warp[kCommitThreads / 32];
+  __shared__ int s_carry, s_mine[5];     // my row: gamma, need, alloc index, len, state
+  __shared__ uint32_t s_head, s_avail;
+  __shared__ int s_last;
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  if (tid == 0) {
+    s_head = *(volatile uint32_t*)&p.hdr->free_head;
+    s_avail = *(volatile uint32_t*)&p.hdr->free_tail - s_head;
+    s_carry = 0;
+  }
+  __syncthreads();
+  const uint32_t avail = s_avail;
+  for (int base = 0; base < p.batch; base += kCommitThreads) {
+    const int i = base + tid;
+    int g = 0, need = 0, state = 0, len = 0;
+    if (i < p.batch) {
+      const int slot = p.seq_ids ? p.seq_ids[i] : i;
+      len = *(volatile int32_t*)&p.seq_len[slot];
+      g = gamma_tau(p, i);
+      if (len + g > p.mpps * kPageSize) state = 1;
+      else need = (len % kPageSize == 0) || (len % kPageSize + g > kPageSize);
+    }
+    // exclusive scan of `need` in batch order
+    int incl = need;
+    for (int o = 1; o < 32; o <<= 1) {
+      int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) s_warp[wid] = incl;
+    __syncthreads();
+    int before = s_carry;
+    for (int w = 0; w < wid; ++w) before += s_warp[w];
+    const int alloc = before + incl - need;
+    if (need && (uint32_t)alloc >= avail) { state = 2; }
+    if (i < p.batch) {
+      s_gamma[i] = (int8_t)g;
+      s_state[i] = (int8_t)state;
+      if (i == b) { s_mine[0] = g; s_mine[1] = need; s_mine[2] = alloc; s_mine[3] = len; s_mine[4] = state; }
+    }
+    __syncthreads();
+    if (tid == kCommitThreads - 1) s_carry = before + incl;
+    __syncthreads();
+  }
+  const int total_need = s_carry;
+
+  // all reads of the shared tables are done: take a ticket
+  if (tid == 0) {
+    __threadfence();
+    const uint32_t t = atomicAdd(&p.hdr->commit_ticket, 1u);
+    s_last = (t == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (s_last) {
+    __threadfence();
+    for (int i = tid; i < p.batch; i += kCommitThreads) {
+      if (s_state[i] == 0) {
+        const int slot = p.seq_ids ? p.seq_ids[i] : i;
+        p.seq_len[slot] += s_gamma[i];
+      }
+    }
+    if (tid == 0) {
+      p.hdr->free_head = s_head + min((uint32_t)total_need, avail);
+      p.hdr->commit_ticket = 0;
+    }
+  }
+
+  // my row
+  const int g = s_mine[0], need = s_mine[1], alloc = s_mine[2], len = s_mine[3], state = s_mine[4];
+  const int slot = p.seq_ids ? p.seq_ids[b] : b;
+  if (state != 0) {
+    if (tid == 0) {
+      p.accepted_len[b] = -1;
+      report_status(p.hdr, state == 1 ? SDLM_ERR_DEVICE_CHECK : SDLM_ERR_OUT_OF_PAGES, slot, len);
+    }
+    for (int k = tid; k < p.D; k += kCommitThreads) p.out_tokens[b * p.D + k] = -1;
+    return;
+  }
+  const int new_idx = (len + kPageSize - 1) / kPageSize;
+  int new_page = -1;
+  if (need) {
+    new_page = p.free_list[(s_head + (uint32_t)alloc) % (uint32_t)p.num_pages];
+    if (tid == 0) p.page_table[(size_t)slot * p.mpps + new_idx] = new_page;
+  }
+  if (tid == 0) p.accepted_len[b] = g;
+  for (int k = tid; k < p.D; k += kCommitThreads) p.out_tokens[b * p.D + k] = (k < g) ? p.token[b * p.D + k] : -1;
+  const int cpr = p.d / 8;
+  const int total = g * p.Hkv * 2 * cpr;
+  for (int idx = tid; idx < total; idx += kCommitThreads) {
+    const int c = idx % cpr;
+    int r = idx / cpr;
+    const int kv = r % 2; r /= 2;
+    const int h = r % p.Hkv;
+    const int t = r / p.Hkv;
+    const int pos = len + t;
+    const int pidx = pos / kPageSize, row = pos % kPageSize;
+    const int page = (need && pidx == new_idx) ? new_page : p.page_table[(size_t)slot * p.mpps + pidx];
+    const uint4* src = reinterpret_cast<const uint4*>((kv ? p.v_blk : p.k_blk) +
+                                                      (((size_t)b * p.D + t) * p.Hkv + h) * p.d) + c;
+    uint4* dst = reinterpret_cast<uint4*>(p.pool + kv_tile_offset(page, h, kv, p.Hkv, p.d) + (size_t)row * p.d) +
+                 kv_swizzled_chunk(row, c);
+    *dst = *src;
+  }
+}
+
+}  // namespace sdlm
+
+using namespace sdlm;
+
+// ---------------------------------------------------------------------------------------------
+// C ABI
+// ---------------------------------------------------------------------------------------------
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+extern "C" size_t sdlm_pool_bytes(const sdlm_config* cfg) {
+  if (!cfg || !config_valid(*cfg)) return 0;
+  return (size_t)cfg->num_pages * cfg->n_kv_heads * 2 * kv_tile_elems(cfg->head_dim) * 2;
+}
+
+extern "C" size_t sdlm_workspace_bytes(const sdlm_config* cfg) {
+  if (!cfg || !config_valid(*cfg)) return 0;
+  return workspace_layout(*cfg).total;
+}
+
+extern "C" const char* sdlm_status_str(sdlm_status s) {
+  switch (s) {
+    case SDLM_OK: return "ok";
+    case SDLM_ERR_INVALID_ARG: return "invalid argument";
+    case SDLM_ERR_SHAPE: return "shape exceeds context limits";
+    case SDLM_ERR_UNSUPPORTED: return "unsupported configuration";
+    case SDLM_ERR_OUT_OF_PAGES: return "KV page pool exhausted";
+    case SDLM_ERR_CUDA: return "CUDA error";
+    case SDLM_ERR_TIMEOUT: return "bounded device wait ran out";
+    case SDLM_ERR_DEVICE_CHECK: return "device-side table check failed";
+    case SDLM_ERR_WORKSPACE: return "pool or workspace too small or misaligned";
+  }
+  return "unknown status";
+}
+
+static sdlm_status reset_tables(sdlm_ctx* ctx, const int32_t* host_free_list, cudaStream_t st) {
+  const sdlm_config& c = ctx->cfg;
+  if (host_free_list) {
+    if (cudaMemcpyAsync(ctx->free_list, host_free_list, (size_t)c.num_pages * 4, cudaMemcpyHostToDevice, st) !=
+        cudaSuccess)
+      return SDLM_ERR_CUDA;
+  }
+  reset_tables_kernel<<<64, 256, 0, st>>>(ctx->hdr, ctx->page_table, ctx->seq_len, ctx->free_list,
+                                         c.max_batch * c.max_pages_per_seq, c.max_batch, c.num_pages,
+                                         host_free_list ? 0 : 1);
+  ctx->launches++;
+  if (cudaGetLastError() != cudaSuccess) return SDLM_ERR_CUDA;
+  if (host_free_list && cudaStreamSynchronize(st) != cudaSuccess) return SDLM_ERR_CUDA;
+  return SDLM_OK;
+}
+
+extern "C" sdlm_status sdlm_create(const sdlm_config* cfg, void* kv_pool, size_t kv_pool_bytes, void* workspace,
+                                   size_t workspace_bytes, sdlm_ctx** out) {
+  if (!cfg || !out || !kv_pool || !workspace) return SDLM_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!config_valid(*cfg)) return SDLM_ERR_UNSUPPORTED;
+  if (kv_pool_bytes < sdlm_pool_bytes(cfg) || workspace_bytes < sdlm_workspace_bytes(cfg)) return SDLM_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(kv_pool) & 1023) || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return SDLM_ERR_WORKSPACE;
+  int dev = 0, major = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SDLM_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SDLM_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SDLM_ERR_CUDA;
+  if (major != 10) return SDLM_ERR_CUDA;  // sm_100a code only
+  sdlm_ctx* ctx = new (std::nothrow) sdlm_ctx();
+  if (!ctx) return SDLM_ERR_INVALID_ARG;
+  ctx->cfg = *cfg;
+  ctx->scale = cfg->softmax_scale > 0.0f ? cfg->softmax_scale : 1.0f / sqrtf((float)cfg->head_dim);
+  ctx->group = cfg->n_q_heads / cfg->n_kv_heads;
+  ctx->device = dev;
+  ctx->sm_count = sms;
+  ctx->pool = static_cast<char*>(kv_pool);
+  ctx->ws = static_cast<char*>(workspace);
+  ctx->lay = workspace_layout(*cfg);
+  ctx->hdr = reinterpret_cast<DevHeader*>(ctx->ws + ctx->lay.hdr);
+  ctx->page_table = reinterpret_cast<int32_t*>(ctx->ws + ctx->lay.page_table);
+  ctx->seq_len = reinterpret_cast<int32_t*>(ctx->ws + ctx->lay.seq_len);
+  ctx->free_list = reinterpret_cast<int32_t*>(ctx->ws + ctx->lay.free_list);
+  ctx->launches = 0;
+  ctx->lmhead_path = 0;
+  ctx->tmap_w_ptr = nullptr;
+  ctx->tmap_w_rows = 0;
+  if (setup_attn(ctx) != cudaSuccess || setup_lmhead(ctx) != cudaSuccess) { delete ctx; return SDLM_ERR_CUDA; }
+  sdlm_status s = reset_tables(ctx, nullptr, 0);
+  if (s == SDLM_OK && cudaStreamSynchronize(0) != cudaSuccess) s = SDLM_ERR_CUDA;
+  if (s != SDLM_OK) { delete ctx; return s; }
+  *out = ctx;
+  return SDLM_OK;
+}
+
+extern "C" void sdlm_destroy(sdlm_ctx* ctx) { delete ctx; }
+
+extern "C" sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t value) {
+  if (!ctx) return SDLM_ERR_INVALID_ARG;
+  switch (opt) {
+    case SDLM_OPT_LMHEAD_KERNEL:
+      if (value < 0 || value > 2) return SDLM_ERR_INVALID_ARG;
+      ctx->lmhead_path = value;
+      return SDLM_OK;
+  }
+  return SDLM_ERR_INVALID_ARG;
+}
+
+extern "C" uint64_t sdlm_launch_count(const sdlm_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" sdlm_status sdlm_kv_pages(sdlm_ctx* ctx, sdlm_kv_op op, const sdlm_kv_args* a, sdlm_kv_result* r,
+                                     void* stream) {
+  if (!ctx) return SDLM_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const sdlm_config& c = ctx->cfg;
+  const size_t table_bytes = ctx->lay.table_end - ctx->lay.hdr;
+  auto slot_ok = [&](int s) { return s >= 0 && s < c.max_batch; };
+  switch (op) {
+    case SDLM_KV_RESET:
+      return reset_tables(ctx, a ? a->free_list : nullptr, st);
+    case SDLM_KV_ADD_SEQ: {
+      if (!a || !slot_ok(a->seq) || a->length < 0 || a->length > c.max_pages_per_seq * kPageSize)
+        return SDLM_ERR_INVALID_ARG;
+      if (a->length > 0 && (!a->k || !a->v || !aligned16(a->k) || !aligned16(a->v))) return SDLM_ERR_INVALID_ARG;
+      if (a->length == 0) return SDLM_OK;
+      add_seq_alloc_kernel<<<1, 256, 0, st>>>(ctx->hdr, ctx->page_table, ctx->seq_len, ctx->free_list, a->seq,
+                                              a->length, c.max_pages_per_seq, c.num_pages);
+      const size_t chunks = (size_t)a->length * c.n_kv_heads * 2 * (c.head_dim / 8);
+      const int blocks = (int)((chunks + 255) / 256 < 4096 ? (chunks + 255) / 256 : 4096);
+      kv_rows_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<__nv_bfloat16*>(ctx->pool), ctx->page_table,
+                                             ctx->seq_len, (__nv_bfloat16*)a->k, (__nv_bfloat16*)a->v, a->seq,
+                                             a->length, c.max_pages_per_seq, c.n_kv_heads, c.head_dim, 1);
+      ctx->launches += 2;
+      return cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+    }
+    case SDLM_KV_RELEASE_SEQ: {
+      if (!a || !slot_ok(a->seq)) return SDLM_ERR_INVALID_ARG;
+      release_seq_kernel<<<1, 256, 0, st>>>(ctx->hdr, ctx->page_table, ctx->seq_len, ctx->free_list, a->seq,
+                                            c.max_pages_per_seq, c.num_pages);
+      ctx->launches++;
+      return cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+    }
+    case SDLM_KV_QUERY: {
+      if (!r) return SDLM_ERR_INVALID_ARG;
+      r->page_table = ctx->page_table;
+      r->seq_len = ctx->seq_len;
+      r->free_list = ctx->free_list;
+      r->free_head = &ctx->hdr->free_head;
+      r->free_tail = &ctx->hdr->free_tail;
+      r->device_status = ctx->hdr->status;
+      r->table_bytes = table_bytes;
+      return SDLM_OK;
+    }
+    case SDLM_KV_GATHER: {
+      if (!a || !slot_ok(a->seq) || a->length < 0 || a->length > c.max_pages_per_seq * kPageSize)
+        return SDLM_ERR_INVALID_ARG;
+      if (a->length == 0) return SDLM_OK;
+      if (!a->k_out || !a->v_out || !aligned16(a->k_out) || !aligned16(a->v_out)) return SDLM_ERR_INVALID_ARG;
+      const size_t chunks = (size_t)a->length * c.n_kv_heads * 2 * (c.head_dim / 8);
+      const int blocks = (int)((chunks + 255) / 256 < 4096 ? (chunks + 255) / 256 : 4096);
+      kv_rows_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<__nv_bfloat16*>(ctx->pool), ctx->page_table,
+                                             ctx->seq_len, (__nv_bfloat16*)a->k_out, (__nv_bfloat16*)a->v_out,
+                                             a->seq, a->length, c.max_pages_per_seq, c.n_kv_heads, c.head_dim, 0);
+      ctx->launches++;
+      return cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+    }
+    case SDLM_KV_EXPORT: {
+      if (!a || !a->host_buf || a->host_bytes < table_bytes) return SDLM_ERR_INVALID_ARG;
+      if (cudaStreamSynchronize(st) != cudaSuccess) return SDLM_ERR_CUDA;
+      if (cudaMemcpy(a->host_buf, ctx->ws + ctx->lay.hdr, table_bytes, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return SDLM_ERR_CUDA;
+      if (r) r->table_bytes = table_bytes;
+      return SDLM_OK;
+    }
+    case SDLM_KV_IMPORT: {
+      if (!a || !a->host_buf || a->host_bytes < table_bytes) return SDLM_ERR_INVALID_ARG;
+      if (cudaStreamSynchronize(st) != cudaSuccess) return SDLM_ERR_CUDA;
+      if (cudaMemcpy(ctx->ws + ctx->lay.hdr, a->host_buf, table_bytes, cudaMemcpyHostToDevice) != cudaSuccess)
+        return SDLM_ERR_CUDA;
+      return SDLM_OK;
+    }
+  }
+  return SDLM_ERR_INVALID_ARG;
+}
+
+static sdlm_status check_batch(const sdlm_ctx* ctx, int batch, int D) {
+  if (batch < 1 || D < 1) return SDLM_ERR_INVALID_ARG;
+  if (batch > ctx->cfg.max_batch || D > ctx->cfg.max_block) return SDLM_ERR_SHAPE;
+  return SDLM_OK;
+}
+
+extern "C" sdlm_status sdlm_block_attn(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids,
+                                       const void* q, const void* k_blk, const void* v_blk, void* out,
+                                       void* stream) {
+  if (!ctx || !q || !k_blk || !v_blk || !out) return SDLM_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out)) return SDLM_ERR_INVALID_ARG;
+  sdlm_status s = check_batch(ctx, batch, D);
+  if (s != SDLM_OK) return s;
+  return launch_block_attn(ctx, batch, D, seq_ids, q, k_blk, v_blk, out, static_cast<cudaStream_t>(stream)) ==
+                 cudaSuccess
+             ? SDLM_OK
+             : SDLM_ERR_CUDA;
+}
+
+extern "C" sdlm_status sdlm_lmhead_confidence(sdlm_ctx* ctx, int32_t rows, const void* hidden, const void* w_lm,
+                                              int32_t* token, float* p_top1, float* entropy, float* max_logit,
+                                              float* lse, void* stream) {
+  if (!ctx || !hidden || !w_lm || !token || !p_top1 || !entropy) return SDLM_ERR_INVALID_ARG;
+  if (!aligned16(hidden) || !aligned16(w_lm)) return SDLM_ERR_INVALID_ARG;
+  if (rows < 1) return SDLM_ERR_INVALID_ARG;
+  if (rows > ctx->cfg.max_batch * ctx->cfg.max_block) return SDLM_ERR_SHAPE;
+  return launch_lmhead(ctx, rows, hidden, w_lm, token, p_top1, entropy, max_logit, lse,
+                       static_cast<cudaStream_t>(stream));
+}
+
+extern "C" sdlm_status sdlm_accept_commit(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, float tau,
+                                          sdlm_conf_mode mode, const int32_t* token, const float* p_top1,
+                                          const float* entropy, const void* k_blk, const void* v_blk,
+                                          int32_t* accepted_len, int32_t* out_tokens, void* stream) {
+  if (!ctx || !token || !p_top1 || !entropy || !k_blk || !v_blk || !accepted_len || !out_tokens)
+    return SDLM_ERR_INVALID_ARG;
+  if (!aligned16(k_blk) || !aligned16(v_blk)) return SDLM_ERR_INVALID_ARG;
+  if (mode != SDLM_CONF_LOGIT && mode != SDLM_CONF_ENTROPY) return SDLM_ERR_INVALID_ARG;
+  if (!isfinite(tau)) return SDLM_ERR_INVALID_ARG;
+  sdlm_status s = check_batch(ctx, batch, D);
+  if (s != SDLM_OK) return s;
+  const sdlm_config& c = ctx->cfg;
+  CommitParams p;
+  p.hdr = ctx->hdr; p.page_table = ctx->page_table; p.seq_len = ctx->seq_len; p.free_list = ctx->free_list;
+  p.pool = reinterpret_cast<__nv_bfloat16*>(ctx->pool);
+  p.seq_ids = seq_ids; p.token = token; p.p_top1 = p_top1; p.entropy = entropy;
+  p.k_blk = static_cast<const __nv_bfloat16*>(k_blk); p.v_blk = static_cast<const __nv_bfloat16*>(v_blk);
+  p.accepted_len = accepted_len; p.out_tokens = out_tokens;
+  p.tau = tau;
+  p.inv_ln_vocab = c.vocab > 1 ? (float)(1.0 / log((double)c.vocab)) : 0.0f;
+  p.mode = (int)mode; p.batch = batch; p.D = D; p.Hkv = c.n_kv_heads; p.d = c.head_dim;
+  p.mpps = c.max_pages_per_seq; p.num_pages = c.num_pages;
+  accept_commit_kernel<<<batch, kCommitThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+  ctx->launches++;
+  return cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+}
+
+extern "C" sdlm_status sdlm_device_status(sdlm_ctx* ctx, int32_t* host_out, int32_t clear, void* stream) {
+  if (!ctx || !host_out) return SDLM_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(host_out, ctx->hdr->status, 16, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SDLM_ERR_CUDA;
+  if (clear && cudaMemsetAsync(ctx->hdr->status, 0, 16, st) != cudaSuccess) return SDLM_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return SDLM_ERR_CUDA;
+  return SDLM_OK;
+}
+
+extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids_host,
+                                             float tau, sdlm_conf_mode mode, const void* q_host,
+                                             const void* k_blk_host, const void* v_blk_host,
+                                             const void* hidden_host, const void* w_lm, void* attn_out_host,
+                                             int32_t* token_host, float* p_top1_host, float* entropy_host,
+                                             int32_t* accepted_len_host, int32_t* out_tokens_host, void* stream) {
+  if (!ctx || !q_host || !k_blk_host || !v_blk_host || !hidden_host || !w_lm) return SDLM_ERR_INVALID_ARG;
+  sdlm_status s = check_batch(ctx, batch, D);
+  if (s != SDLM_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const sdlm_config& c = ctx->cfg;
+  const WorkspaceLayout& L = ctx->lay;
+  const size_t rows = (size_t)batch * D;
+  const size_t q_bytes = rows * c.n_q_heads * c.head_dim * 2, kv_bytes = rows * c.n_kv_heads * c.head_dim * 2;
+  char* ws = ctx->ws;
+  bool ok = true;
+  ok &= cudaMemcpyAsync(ws + L.st_q, q_host, q_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(ws + L.st_k, k_blk_host, kv_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(ws + L.st_v, v_blk_host, kv_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(ws + L.st_hidden, hidden_host, rows * c.hidden * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  const int32_t* seq_ids = nullptr;
+  if (seq_ids_host) {
+    ok &= cudaMemcpyAsync(ws + L.st_seq_ids, seq_ids_host, (size_t)batch * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    seq_ids = reinterpret_cast<const int32_t*>(ws + L.st_seq_ids);
+  }
+  if (!ok) return SDLM_ERR_CUDA;
+  int32_t* d_token = reinterpret_cast<int32_t*>(ws + L.st_token);
+  float* d_p = reinterpret_cast<float*>(ws + L.st_p);
+  float* d_ent = reinterpret_cast<float*>(ws + L.st_ent);
+  int32_t* d_acc = reinterpret_cast<int32_t*>(ws + L.st_acc);
+  int32_t* d_out_tokens = reinterpret_cast<int32_t*>(ws + L.st_out_tokens);
+  s = sdlm_block_attn(ctx, batch, D, seq_ids, ws + L.st_q, ws + L.st_k, ws + L.st_v, ws + L.st_out, stream);
+  if (s != SDLM_OK) return s;
+  s = sdlm_lmhead_confidence(ctx, (int32_t)rows, ws + L.st_hidden, w_lm, d_token, d_p, d_ent, nullptr, nullptr, stream);
+  if (s != SDLM_OK) return s;
+  s = sdlm_accept_commit(ctx, batch, D, seq_ids, tau, mode, d_token, d_p, d_ent, ws + L.st_k, ws + L.st_v, d_acc,
+                         d_out_tokens, stream);
+  if (s != SDLM_OK) return s;
+  if (attn_out_host) ok &= cudaMemcpyAsync(attn_out_host, ws + L.st_out, q_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (token_host) ok &= cudaMemcpyAsync(token_host, d_token, rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (p_top1_host) ok &= cudaMemcpyAsync(p_top1_host, d_p, rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (entropy_host) ok &= cudaMemcpyAsync(entropy_host, d_ent, rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (accepted_len_host) ok &= cudaMemcpyAsync(accepted_len_host, d_acc, (size_t)batch * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (out_tokens_host) ok &= cudaMemcpyAsync(out_tokens_host, d_out_tokens, rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (!ok || cudaStreamSynchronize(st) != cudaSuccess) return SDLM_ERR_CUDA;
+  return SDLM_OK;
+}

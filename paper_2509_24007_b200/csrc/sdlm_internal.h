@@ -1,0 +1,89 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/sdlm.h"
+
+namespace sdlm {
+
+constexpr int kPageSize = 64;        // tokens per KV page
+constexpr int kMaxBlock = 8;         // largest D
+constexpr int kMaxQRows = 64;        // (Hq/Hkv) * D stacked query rows per KV head
+constexpr int kMaxBatch = 4096;
+constexpr int kLmMaxStripes = 1024;  // upper bound on vocab stripes (one partial per stripe per row)
+constexpr int kAttnTargetItems = 592;  // split-KV work items aimed for: 4 per SM on 148 SMs
+
+// Sticky status and ring cursors at the start of the workspace; EXPORT/IMPORT copies this header
+// together with the tables that follow it.
+struct DevHeader {
+  int32_t status[4];       // {sdlm_status, slot, detail, count}
+  uint32_t free_head;      // pages handed out so far
+  uint32_t free_tail;      // pages ever pushed
+  uint32_t commit_ticket;  // "last CTA done" counter of accept_commit (always 0 between launches)
+  uint32_t lm_ticket;      // same for the LM-head combine
+  uint32_t reserved[8];
+};
+static_assert(sizeof(DevHeader) == 64, "header is 64 bytes");
+
+struct WorkspaceLayout {
+  size_t hdr, page_table, seq_len, free_list, table_end;  // [hdr, table_end) is the exportable state
+  size_t lm_partials;                                      // float4 [kLmMaxStripes][max_rows]
+  size_t attn_ml, attn_o;                                  // split-KV partial (m, l) and O
+  size_t st_q, st_k, st_v, st_hidden, st_out, st_seq_ids, st_token, st_p, st_ent, st_acc, st_out_tokens;
+  size_t total;
+  int attn_max_items;
+  int q_rows_pad;  // stacked query rows per KV head at max_block, padded to 16
+};
+
+bool config_valid(const sdlm_config& c);
+WorkspaceLayout workspace_layout(const sdlm_config& c);
+
+}  // namespace sdlm
+
+struct sdlm_ctx {
+  sdlm_config cfg;
+  float scale;
+  int group;  // Hq / Hkv
+  int device;
+  int sm_count;
+  char* pool;
+  char* ws;
+  sdlm::WorkspaceLayout lay;
+  sdlm::DevHeader* hdr;
+  int32_t* page_table;
+  int32_t* seq_len;
+  int32_t* free_list;
+  uint64_t launches;
+  int lmhead_path;  // 0 = pick by shape, 1 = force the mma.sync kernel, 2 = force the tcgen05 kernel
+  // cached TMA descriptor of the LM-head weight (keyed by pointer and tile rows)
+  const void* tmap_w_ptr;
+  int tmap_w_rows;
+  alignas(64) unsigned char tmap_w[128];
+};
+
+namespace sdlm {
+
+// ---- paged pool addressing (shared by fill / gather / commit / attention) ------------------
+// Pool layout: [page][kv_head][K|V][64 tokens][d] bf16.  One (page, head, K|V) tile is a
+// contiguous 64*d*2-byte run.  Inside a token row the 16-byte chunks are stored XOR-swizzled by
+// the row index (chunk c of row r sits at chunk c ^ (r & 7)), so that a plain bulk copy of a tile
+// into shared memory is already bank-conflict-free for 8-row matrix loads.
+__host__ __device__ inline size_t kv_tile_elems(int d) { return (size_t)kPageSize * d; }
+__host__ __device__ inline size_t kv_tile_offset(int page, int head, int kv, int n_kv_heads, int d) {
+  return (((size_t)page * n_kv_heads + head) * 2 + kv) * kv_tile_elems(d);
+}
+__host__ __device__ inline int kv_swizzled_chunk(int row, int chunk) { return chunk ^ (row & 7); }
+
+// ---- launchers implemented in the kernel translation units ---------------------------------
+cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, const void* q,
+                              const void* k_blk, const void* v_blk, void* out, cudaStream_t st);
+sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
+                          float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st);
+cudaError_t setup_attn(sdlm_ctx* ctx);
+cudaError_t setup_lmhead(sdlm_ctx* ctx);
+
+}  // namespace sdlm

@@ -1,0 +1,525 @@
+// (b) LM head -> softmax statistics (Sec. 3.2: Z in R^{D x |V|}; Eq. 8; Eq. 9).
+//
+// z = W h is never written to memory.  The vocabulary is cut into contiguous stripes, one per
+// CTA; a CTA streams its stripe of W exactly once and keeps, per hidden-state row, the online
+// statistics  m = max z,  S = sum exp(z-m),  T = sum exp(z-m)(z-m)  and the first argmax index.
+// A second small kernel merges the per-stripe partials in a fixed order and emits
+//   token = argmax,  p_top1 = 1/S,  entropy = ln S - T/S.
+//
+// Two stripe kernels:
+//   * lmhead_umma_kernel: tcgen05.mma with the hidden-state rows as the M=128 operand, a
+//     BN-row slab of W as the N operand (both K-major, 128-byte swizzle, staged by TMA on an
+//     mbarrier ring) and fp32 accumulators in tensor memory.  One accumulator lane is one
+//     hidden-state row, so each epilogue thread owns a row and reduces its logits in registers
+//     with no cross-thread traffic.  Warp-specialised: TMA producer, MMA issuer, 4 epilogue warps.
+//   * lmhead_mma_kernel: warp-level mma.sync tiles fed by cp.async; used for shapes the TMA path
+//     cannot take (row pitch not a multiple of 16 bytes is already excluded by the API, so this
+//     is the small-shape / debug path).
+#include "sdlm_internal.h"
+#include "sdlm_ptx.cuh"
+
+#include <cuda.h>
+
+namespace sdlm {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kNegInit = -1.0e30f;  // finite stand-in for "no logit seen yet"
+
+struct Stat {
+  float m, S, T;
+  int idx;
+};
+
+__device__ __forceinline__ Stat stat_empty() { return Stat{kNegInit, 0.f, 0.f, 0x7fffffff}; }
+
+// Merge of two partial statistics over disjoint vocabulary ranges; ties go to the lower index.
+__device__ __forceinline__ Stat stat_merge(const Stat& a, const Stat& b) {
+  Stat r;
+  r.idx = (b.m > a.m || (b.m == a.m && b.idx < a.idx)) ? b.idx : a.idx;
+  r.m = fmaxf(a.m, b.m);
+  const float da = a.m - r.m, db = b.m - r.m;
+  const float sa = exp2f(da * kLog2e), sb = exp2f(db * kLog2e);
+  r.S = sa * a.S + sb * b.S;
+  r.T = sa * (a.T + da * a.S) + sb * (b.T + db * b.S);
+  return r;
+}
+
+struct LmParams {
+  const __nv_bfloat16* hidden;  // [rows, H]
+  const __nv_bfloat16* w;       // [V, H]
+  float4* partials;             // [n_stripes][rows_pad]
+  DevHeader* hdr;
+  int rows, H, V, n_stripes, rows_pad;
+  int bn;  // umma path: vocab rows per tile (multiple of 16, <= 256)
+};
+
+// ---------------------------------------------------------------------------------------------
+// tcgen05 / TMA stripe kernel
+// ---------------------------------------------------------------------------------------------
+constexpr int kUmmaThreads = 192;  // warp 0 producer, warp 1 MMA + TMEM owner, warps 2..5 epilogue
+constexpr int kBK = 64;            // K elements per stage: one 128-byte swizzle row
+constexpr int kATileBytes = 128 * kBK * 2;
+
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr) {
+  // K-major, 128-byte swizzle: 8-row groups 1024 bytes apart; descriptor version 1 (sm_100)
+  return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+
+__device__ __forceinline__ void lm_timeout(DevHeader* hdr, int where) {
+  if (atomicCAS(&hdr->status[0], 0, (int)SDLM_ERR_TIMEOUT) == 0) {
+    hdr->status[1] = -2;
+    hdr->status[2] = where;
+  }
+}
+
+// Folds 16 consecutive logits (vocab indices n0 .. n0+15, those >= n_end ignored) into a row's statistics.
+__device__ __forceinline__ void fold16(const uint32_t (&v)[16], int n0, int n_end, Stat& st) {
+  float z[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) z[i] = __uint_as_float(v[i]);
+  if (n0 + 16 > n_end) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i)
+      if (n0 + i >= n_end) z[i] = kNegInit;
+  }
+  float cm = z[0];
+#pragma unroll
+  for (int i = 1; i < 16; ++i) cm = fmaxf(cm, z[i]);
+  if (cm > st.m) {  // new running maximum: remember its first position, rescale the sums
+    int first = 15;
+#pragma unroll
+    for (int i = 14; i >= 0; --i)
+      if (z[i] == cm) first = i;
+    st.idx = n0 + first;
+    const float dm = st.m - cm;
+    const float a = ptx::ex2(dm * kLog2e);
+    st.T = a * (st.T + dm * st.S);
+    st.S = a * st.S;
+    st.m = cm;
+  }
+  const float m_l2 = st.m * kLog2e;
+  float S = 0.f, T = 0.f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const float e = ptx::ex2(fmaf(z[i], kLog2e, -m_l2));
+    S += e;
+    T = fmaf(e, z[i] - st.m, T);
+  }
+  st.S += S;
+  st.T += T;
+}
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+}
+
+// R = number of 128-row blocks of hidden states (1 or 2).  R == 1 double-buffers the accumulator
+// (2 x 256 TMEM columns); R == 2 uses one accumulator per row block.
+template <int R>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+    lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_w,
+                       const LmParams p, int n_stages) {
+  constexpr int NACC = 2 / R;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int w_tile_bytes = p.bn * kBK * 2;
+  const int stage_bytes = R * kATileBytes + w_tile_bytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)n_stages * stage_bytes);
+  uint64_t* empty = full + n_stages;
+  uint64_t* acc_full = empty + n_stages;
+  uint64_t* acc_empty = acc_full + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  // this CTA's vocabulary stripe, in groups of 16 rows
+  const int groups = (p.V + 15) / 16;
+  const int g0 = (int)((long long)blockIdx.x * groups / gridDim.x);
+  const int g1 = (int)((long long)(blockIdx.x + 1) * groups / gridDim.x);
+  const int n_begin = g0 * 16, n_end = min(p.V, g1 * 16);
+  const int n_tiles = (n_end - n_begin + p.bn - 1) / p.bn;
+  const int KC = (p.H + kBK - 1) / kBK;
+
+  if (tid == 0) {
+    for (int s = 0; s < n_stages; ++s) {
+      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&empty[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      ptx::mbar_init(&acc_full[s], 1);
+      ptx::mbar_init(&acc_empty[s], 4);
+    }
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmap_h);
+    ptx::prefetch_tmap(&tmap_w);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, 512);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {  // ---- TMA producer
+      uint32_t it = 0;
+      for (int t = 0; t < n_tiles; ++t) {
+        const int n0 = n_begin + t * p.bn;
+        for (int kc = 0; kc < KC; ++kc, ++it) {
+          const int s = it % n_stages;
+          if (it >= (uint32_t)n_stages && !ptx::mbar_wait(&empty[s], ((it / n_stages) & 1) ^ 1)) lm_timeout(p.hdr, 1);
+          uint8_t* st = smem + (size_t)s * stage_bytes;
+          ptx::mbar_arrive_expect_tx(&full[s], (uint32_t)stage_bytes);
+#pragma unroll
+          for (int r = 0; r < R; ++r) ptx::tma_load_2d(st + r * kATileBytes, &tmap_h, kc * kBK, r * 128, &full[s]);
+          ptx::tma_load_2d(st + R * kATileBytes, &tmap_w, kc * kBK, n0, &full[s]);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {  // ---- MMA issuer
+      // instruction descriptor: D fp32, A and B bf16, both K-major, N = bn, M = 128
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.bn >> 3) << 17) | ((128u >> 4) << 24);
+      uint32_t it = 0;
+      for (int t = 0; t < n_tiles; ++t) {
+        const int as = t % NACC;
+        const uint32_t use = (uint32_t)t / NACC;
+        if (use > 0 && !ptx::mbar_wait(&acc_empty[as], (use & 1) ^ 1)) lm_timeout(p.hdr, 2);
+        ptx::tc_fence_after();
+        for (int kc = 0; kc < KC; ++kc, ++it) {
+          const int s = it % n_stages;
+          if (!ptx::mbar_wait(&full[s], (it / n_stages) & 1)) lm_timeout(p.hdr, 3);
+          ptx::tc_fence_after();
+          const uint32_t a_addr = ptx::smem_u32(smem + (size_t)s * stage_bytes);
+          const uint32_t b_addr = a_addr + R * kATileBytes;
+#pragma unroll
+          for (int r = 0; r < R; ++r) {
+            const uint32_t d_tmem = tmem_base + (uint32_t)((R == 1 ? as : r) * 256);
+#pragma unroll
+            for (int k = 0; k < kBK / 16; ++k)
+              ptx::umma_bf16_ss(d_tmem, umma_smem_desc(a_addr + r * kATileBytes + k * 32),
+                                umma_smem_desc(b_addr + k * 32), idesc, (kc | k) ? 1u : 0u);
+          }
+          ptx::umma_commit(&empty[s]);  // stage reusable once these MMAs have read it
+        }
+        ptx::umma_commit(&acc_full[as]);  // accumulator complete
+      }
+    }
+  } else {  // ---- epilogue: TMEM lane = hidden-state row
+    const int q = warp & 3;  // TMEM lane quarter this warp may touch
+    Stat st[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) st[r] = stat_empty();
+    for (int t = 0; t < n_tiles; ++t) {
+      const int as = t % NACC;
+      const uint32_t use = (uint32_t)t / NACC;
+      if (!ptx::mbar_wait(&acc_full[as], use & 1)) lm_timeout(p.hdr, 4);
+      ptx::tc_fence_after();
+      const int n0 = n_begin + t * p.bn;
+      const int n_chunks = p.bn / 16;
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)((R == 1 ? as : r) * 256);
+        uint32_t v0[16], v1[16];
+        tmem_ld16(taddr, v0);
+        for (int c = 0; c < n_chunks; c += 2) {
+          ptx::tmem_ld_wait();
+          if (c + 1 < n_chunks) tmem_ld16(taddr + (c + 1) * 16, v1);
+          if (n0 + c * 16 < n_end) fold16(v0, n0 + c * 16, n_end, st[r]);
+          if (c + 1 < n_chunks) {
+            ptx::tmem_ld_wait();
+            if (c + 2 < n_chunks) tmem_ld16(taddr + (c + 2) * 16, v0);
+            if (n0 + (c + 1) * 16 < n_end) fold16(v1, n0 + (c + 1) * 16, n_end, st[r]);
+          }
+        }
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&acc_empty[as]);
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const int row = r * 128 + q * 32 + lane;
+      if (row < p.rows)
+        p.partials[(size_t)blockIdx.x * p.rows_pad + row] =
+            make_float4(st[r].m, st[r].S, st[r].T, __int_as_float(st[r].idx));
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// mma.sync stripe kernel (any H that is a multiple of 8)
+// ---------------------------------------------------------------------------------------------
+constexpr int kMmaThreads = 256, kMmaBM = 128, kMmaBN = 64, kMmaStages = 3;
+constexpr int kMmaStageBytes = (kMmaBM + kMmaBN) * kBK * 2;
+
+__global__ void __launch_bounds__(kMmaThreads) lmhead_mma_kernel(const LmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int row_base = blockIdx.y * kMmaBM;
+  const int tiles_total = (p.V + kMmaBN - 1) / kMmaBN;
+  const int t0 = (int)((long long)blockIdx.x * tiles_total / gridDim.x);
+  const int t1 = (int)((long long)(blockIdx.x + 1) * tiles_total / gridDim.x);
+  const int KC = (p.H + kBK - 1) / kBK;
+  const int n_iter = (t1 - t0) * KC;
+
+  auto load_stage = [&](int it) {
+    const int tile = t0 + it / KC, kc = it % KC;
+    uint8_t* st = smem + (it % kMmaStages) * kMmaStageBytes;
+    const uint32_t st_u32 = ptx::smem_u32(st);
+    for (int idx = tid; idx < (kMmaBM + kMmaBN) * 8; idx += kMmaThreads) {
+      const int r = idx >> 3, c = idx & 7;
+      const int col = kc * kBK + c * 8;
+      const __nv_bfloat16* src;
+      bool ok;
+      if (r < kMmaBM) {
+        const int row = row_base + r;
+        ok = row < p.rows && col < p.H;
+        src = p.hidden + (size_t)(ok ? row : 0) * p.H + (ok ? col : 0);
+      } else {
+        const int n = tile * kMmaBN + (r - kMmaBM);
+        ok = n < p.V && col < p.H;
+        src = p.w + (size_t)(ok ? n : 0) * p.H + (ok ? col : 0);
+      }
+      ptx::cp_async16(st_u32 + r * 128 + ((c ^ (r & 7)) << 4), src, ok ? 16u : 0u);
+    }
+  };
+
+  Stat st[2] = {stat_empty(), stat_empty()};  // rows warp*16 + lane/4 and +8
+  float acc[8][4];
+  for (int s = 0; s < kMmaStages - 1; ++s) {
+    if (s < n_iter) load_stage(s);
+    ptx::cp_async_commit();
+  }
+  for (int it = 0; it < n_iter; ++it) {
+    const int kc = it % KC;
+    ptx::cp_async_wait<kMmaStages - 2>();
+    __syncthreads();
+    if (it + kMmaStages - 1 < n_iter) load_stage(it + kMmaStages - 1);
+    ptx::cp_async_commit();
+    if (kc == 0) {
+#pragma unroll
+      for (int n = 0; n < 8; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+    }
+    const uint32_t a_u32 = ptx::smem_u32(smem + (it % kMmaStages) * kMmaStageBytes);
+    const uint32_t b_u32 = a_u32 + kMmaBM * 128;
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) {
+      uint32_t a0, a1, a2, a3;
+      {
+        const int row = warp * 16 + (lane & 15), chunk = ks * 2 + (lane >> 4);
+        ptx::ldsm_x4(a0, a1, a2, a3, a_u32 + row * 128 + ((chunk ^ (row & 7)) << 4));
+      }
+#pragma unroll
+      for (int np = 0; np < 4; ++np) {
+        const int n = np * 16 + ((lane >> 4) << 3) + (lane & 7), chunk = ks * 2 + ((lane >> 3) & 1);
+        uint32_t b0, b1, b2, b3;
+        ptx::ldsm_x4(b0, b1, b2, b3, b_u32 + n * 128 + ((chunk ^ (n & 7)) << 4));
+        ptx::mma_bf16_16816(acc[2 * np], a0, a1, a2, a3, b0, b1);
+        ptx::mma_bf16_16816(acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
+      }
+    }
+    if (kc == KC - 1) {  // a 128 x 64 logit tile is complete: fold it into the row statistics
+      const int nbase = (t0 + it / KC) * kMmaBN + (lane & 3) * 2;
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        float cm = kNegInit;
+        int ci = 0x7fffffff;
+#pragma unroll
+        for (int n = 0; n < 8; ++n)
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int idx = nbase + n * 8 + e;
+            const float z = (idx < p.V) ? acc[n][2 * r + e] : kNegInit;
+            acc[n][2 * r + e] = z;
+            if (z > cm) { cm = z; ci = idx; }
+          }
+        if (cm == kNegInit) continue;  // every column this thread holds lies past the vocabulary end
+        if (cm > st[r].m) {
+          const float dm = st[r].m - cm, a = ptx::ex2(dm * kLog2e);
+          st[r].T = a * (st[r].T + dm * st[r].S);
+          st[r].S = a * st[r].S;
+          st[r].m = cm;
+          st[r].idx = ci;
+        }
+        const float m_l2 = st[r].m * kLog2e;
+#pragma unroll
+        for (int n = 0; n < 8; ++n)
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const float z = acc[n][2 * r + e];
+            const float ex = ptx::ex2(fmaf(z, kLog2e, -m_l2));
+            st[r].S += ex;
+            st[r].T = fmaf(ex, z - st[r].m, st[r].T);
+          }
+      }
+    }
+  }
+  ptx::cp_async_wait<0>();
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+#pragma unroll
+    for (int o = 1; o <= 2; o <<= 1) {
+      Stat other;
+      other.m = __shfl_xor_sync(0xffffffffu, st[r].m, o);
+      other.S = __shfl_xor_sync(0xffffffffu, st[r].S, o);
+      other.T = __shfl_xor_sync(0xffffffffu, st[r].T, o);
+      other.idx = __shfl_xor_sync(0xffffffffu, st[r].idx, o);
+      st[r] = stat_merge(st[r], other);
+    }
+    const int row = row_base + warp * 16 + (lane >> 2) + r * 8;
+    if ((lane & 3) == 0 && row < p.rows)
+      p.partials[(size_t)blockIdx.x * p.rows_pad + row] = make_float4(st[r].m, st[r].S, st[r].T, __int_as_float(st[r].idx));
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// merge of the per-stripe partials: one warp per row, fixed order
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) lmhead_combine_kernel(const float4* partials, int n_stripes, int rows_pad, int rows,
+                                                             int32_t* token, float* p_top1, float* entropy,
+                                                             float* max_logit, float* lse) {
+  const int row = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  Stat st = stat_empty();
+  for (int s = lane; s < n_stripes; s += 32) {
+    const float4 v = partials[(size_t)s * rows_pad + row];
+    st = stat_merge(st, Stat{v.x, v.y, v.z, __float_as_int(v.w)});
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) {
+    Stat other;
+    other.m = __shfl_xor_sync(0xffffffffu, st.m, o);
+    other.S = __shfl_xor_sync(0xffffffffu, st.S, o);
+    other.T = __shfl_xor_sync(0xffffffffu, st.T, o);
+    other.idx = __shfl_xor_sync(0xffffffffu, st.idx, o);
+    st = stat_merge(st, other);
+  }
+  if (lane == 0) {
+    const float lnS = logf(st.S);
+    token[row] = st.idx;
+    p_top1[row] = 1.0f / st.S;              // the maximal logit contributes exp(0) = 1 to S
+    entropy[row] = fmaxf(lnS - st.T / st.S, 0.f);
+    if (max_logit) max_logit[row] = st.m;
+    if (lse) lse[row] = st.m + lnS;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor [n_rows, n_cols] row-major, box [box_rows, 64 cols], 128-byte swizzle, zero fill.
+static bool make_tmap(CUtensorMap* out, const void* base, int n_rows, int n_cols, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)n_cols, (cuuint64_t)n_rows};
+  cuuint64_t strides[1] = {(cuuint64_t)n_cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr int kUmmaSmemBudget = 220 * 1024;
+
+cudaError_t setup_lmhead(sdlm_ctx* ctx) {
+  (void)ctx;
+  cudaError_t e = cudaFuncSetAttribute(lmhead_umma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kUmmaSmemBudget + 2048);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(lmhead_umma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmemBudget + 2048);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(lmhead_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              kMmaStages * kMmaStageBytes + 128);
+}
+
+sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
+                          float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st) {
+  const sdlm_config& c = ctx->cfg;
+  LmParams p;
+  p.hidden = static_cast<const __nv_bfloat16*>(hidden);
+  p.w = static_cast<const __nv_bfloat16*>(w_lm);
+  p.partials = reinterpret_cast<float4*>(ctx->ws + ctx->lay.lm_partials);
+  p.hdr = ctx->hdr;
+  p.rows = rows; p.H = c.hidden; p.V = c.vocab;
+  p.rows_pad = c.max_batch * c.max_block;
+  p.bn = 0;
+
+  const bool use_umma = ctx->lmhead_path != 1 && rows <= 256 && c.vocab >= 16;
+  if (ctx->lmhead_path == 2 && !use_umma) return SDLM_ERR_UNSUPPORTED;
+  if (use_umma) {
+    const int groups = (c.vocab + 15) / 16;
+    const int n_cta = groups < ctx->sm_count ? groups : ctx->sm_count;
+    const int gmax = (groups + n_cta - 1) / n_cta;
+    const int tiles = (gmax * 16 + 255) / 256;
+    p.bn = 16 * ((gmax + tiles - 1) / tiles);
+    p.n_stripes = n_cta;
+    const int R = rows > 128 ? 2 : 1;
+    const int stage_bytes = R * kATileBytes + p.bn * kBK * 2;
+    int n_stages = kUmmaSmemBudget / stage_bytes;
+    if (n_stages > 8) n_stages = 8;
+    if (n_stages < 2) return SDLM_ERR_UNSUPPORTED;
+    CUtensorMap tm_h;
+    if (!make_tmap(&tm_h, hidden, rows, c.hidden, 128)) return SDLM_ERR_CUDA;
+    if (ctx->tmap_w_ptr != w_lm || ctx->tmap_w_rows != p.bn) {
+      if (!make_tmap(reinterpret_cast<CUtensorMap*>(ctx->tmap_w), w_lm, c.vocab, c.hidden, p.bn)) return SDLM_ERR_CUDA;
+      ctx->tmap_w_ptr = w_lm;
+      ctx->tmap_w_rows = p.bn;
+    }
+    const CUtensorMap& tm_w = *reinterpret_cast<const CUtensorMap*>(ctx->tmap_w);
+    const size_t smem = (size_t)n_stages * stage_bytes + 1024 + 256;
+    if (R == 1)
+      lmhead_umma_kernel<1><<<n_cta, kUmmaThreads, smem, st>>>(tm_h, tm_w, p, n_stages);
+    else
+      lmhead_umma_kernel<2><<<n_cta, kUmmaThreads, smem, st>>>(tm_h, tm_w, p, n_stages);
+  } else {
+    const int tiles_total = (c.vocab + kMmaBN - 1) / kMmaBN;
+    int n_cta = ctx->sm_count * 2;
+    if (n_cta > tiles_total) n_cta = tiles_total;
+    if (n_cta > kLmMaxStripes) n_cta = kLmMaxStripes;
+    p.n_stripes = n_cta;
+    dim3 grid(n_cta, (rows + kMmaBM - 1) / kMmaBM);
+    lmhead_mma_kernel<<<grid, kMmaThreads, kMmaStages * kMmaStageBytes + 128, st>>>(p);
+  }
+  ctx->launches++;
+  if (cudaGetLastError() != cudaSuccess) return SDLM_ERR_CUDA;
+  lmhead_combine_kernel<<<(rows + 3) / 4, 128, 0, st>>>(p.partials, p.n_stripes, p.rows_pad, rows, token, p_top1,
+                                                       entropy, max_logit, lse);
+  ctx->launches++;
+  return cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+}
+
+}  // namespace sdlm

@@ -1,0 +1,93 @@
+"""Puts a synthetic workload (sdlm_synth) on the device behind one library context.
+
+Used by the tests, the benchmark and the smoke check to build identical device state.  It draws
+inputs and marshals them; every step of the decode path itself runs in the library.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+import torch
+
+import sdlm_synth as syn
+
+from .binding import CONF_LOGIT, Sdlm, SdlmConfig, bf16_tensor_from_bits
+
+
+@dataclass
+class DeviceBlock:
+    q: torch.Tensor
+    k_blk: torch.Tensor
+    v_blk: torch.Tensor
+    hidden: torch.Tensor
+    host: syn.BlockInputs
+
+
+@dataclass
+class StepOutputs:
+    attn: torch.Tensor
+    token: torch.Tensor
+    p_top1: torch.Tensor
+    entropy: torch.Tensor
+    accepted_len: torch.Tensor
+    out_tokens: torch.Tensor
+
+
+class DeviceProblem:
+    def __init__(self, wl: syn.Workload, w_bits: Optional[np.ndarray] = None, lengths: Optional[np.ndarray] = None,
+                 max_block: Optional[int] = None, keep_prefix: bool = True):
+        self.wl = wl
+        s = wl.shape
+        self.lengths = syn.prefix_lengths(wl) if lengths is None else np.asarray(lengths, dtype=np.int32)
+        self.num_pages, self.mpps = syn.pages_needed(wl, self.lengths)
+        self.free_list = syn.free_list_permutation(wl, self.num_pages)
+        self.cfg = SdlmConfig(s.n_q_heads, s.n_kv_heads, s.head_dim, s.hidden, s.vocab, self.num_pages, wl.batch,
+                              self.mpps, max_block=max_block or wl.block, page_size=s.page_size)
+        self.sd = Sdlm(self.cfg)
+        self.w_bits = syn.lm_head_weight(wl) if w_bits is None else w_bits
+        self.w_lm = bf16_tensor_from_bits(self.w_bits)
+        self.prefix = []
+        self.reset_cache(keep_prefix)
+
+    def reset_cache(self, keep_prefix: bool = True) -> None:
+        """Free list := the seeded permutation, then every sequence's prefix is added in slot order."""
+        self.sd.kv_reset(self.free_list)
+        regenerate = not self.prefix
+        for b in range(self.wl.batch):
+            if regenerate:
+                k, v = syn.prefix_kv(self.wl, b, int(self.lengths[b]))
+                if keep_prefix:
+                    self.prefix.append((k, v))
+            else:
+                k, v = self.prefix[b]
+            if k.shape[0] > 0:
+                self.sd.kv_add_seq(b, bf16_tensor_from_bits(k), bf16_tensor_from_bits(v))
+        torch.cuda.synchronize()
+
+    def block(self, step: int = 0) -> DeviceBlock:
+        x = syn.block_inputs(self.wl, self.w_bits, step)
+        return DeviceBlock(bf16_tensor_from_bits(x.q), bf16_tensor_from_bits(x.k_blk), bf16_tensor_from_bits(x.v_blk),
+                           bf16_tensor_from_bits(x.hidden), x)
+
+    def alloc_outputs(self) -> StepOutputs:
+        wl, s, dev = self.wl, self.wl.shape, self.sd.device
+        B, D = wl.batch, wl.block
+        return StepOutputs(torch.empty((B, D, s.n_q_heads, s.head_dim), dtype=torch.bfloat16, device=dev),
+                           torch.empty((B, D), dtype=torch.int32, device=dev),
+                           torch.empty((B, D), dtype=torch.float32, device=dev),
+                           torch.empty((B, D), dtype=torch.float32, device=dev),
+                           torch.empty(B, dtype=torch.int32, device=dev),
+                           torch.empty((B, D), dtype=torch.int32, device=dev))
+
+    def step(self, x: DeviceBlock, tau: float, out: Optional[StepOutputs] = None, mode: int = CONF_LOGIT,
+             stream=None) -> StepOutputs:
+        """(a) + (b) + (c) on device-resident inputs: three library calls, no host synchronisation."""
+        out = out or self.alloc_outputs()
+        sd = self.sd
+        sd.block_attn(x.q, x.k_blk, x.v_blk, out.attn, stream=stream)
+        sd.lmhead_confidence(x.hidden, self.w_lm, out.token, out.p_top1, out.entropy, stream=stream)
+        sd.accept_commit(tau, out.token, out.p_top1, out.entropy, x.k_blk, x.v_blk, mode, out.accepted_len,
+                         out.out_tokens, stream=stream)
+        return out

@@ -1,0 +1,82 @@
+"""GPU parity: split-KV paged block-decode attention against the oracle's dense fp64 softmax."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2509_24007_b200 as pk
+from paper_2509_24007_b200.harness import DeviceProblem
+from oracle import sdlm_oracle as orc
+import sdlm_synth as syn
+from oracle_side import check_attention
+
+pytestmark = pytest.mark.gpu
+
+
+def _attn_case(shape, lens, D, seed, scale_note=None):
+    lens = np.asarray(lens, dtype=np.int32)
+    wl = syn.Workload("attn", shape, len(lens), D, 0, 0, (0.9,), seed=seed)
+    dp = DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16), lengths=lens)
+    x = dp.block(0)
+    out = dp.sd.block_attn(x.q, x.k_blk, x.v_blk)
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+    pk_, pv_ = zip(*dp.prefix)
+    ref = orc.block_attention(x.host.q, x.host.k_blk, x.host.v_blk, pk_, pv_)
+    return check_attention(pk.bits_from_bf16_tensor(out), ref), dp, x, out
+
+
+@pytest.mark.parametrize("Hq,Hkv,d", [(4, 2, 64), (2, 2, 128), (16, 2, 128), (10, 2, 128), (8, 1, 64)])
+@pytest.mark.parametrize("D", [1, 2, 4, 8])
+def test_attention_ragged_prefixes(Hq, Hkv, d, D):
+    shape = syn.Shape(Hq, Hkv, d, 64, 64)
+    lens = [0, 1, 63, 64, 65, 127, 128, 300, 1000]
+    _attn_case(shape, lens, D, seed=200 + Hq + D)
+
+
+def test_attention_long_prefix_is_split_across_many_items():
+    shape = syn.Shape(16, 2, 128, 64, 64)
+    err, dp, x, out = _attn_case(shape, [20000, 3], 8, seed=31)
+    # same inputs, second launch: bit-identical (fixed merge order)
+    out2 = dp.sd.block_attn(x.q, x.k_blk, x.v_blk)
+    assert torch.equal(out, out2)
+
+
+def test_attention_with_seq_ids_reads_the_named_slots():
+    shape = syn.SHAPE_TINY
+    lens = np.array([70, 5, 190], dtype=np.int32)
+    wl = syn.Workload("attn_ids", shape, 3, 4, 0, 0, (0.9,), seed=33)
+    dp = DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16), lengths=lens)
+    ids = np.array([2, 0], dtype=np.int32)
+    x = syn.block_inputs(wl.with_(batch=2), dp.w_bits)
+    out = dp.sd.block_attn(pk.bf16_tensor_from_bits(x.q), pk.bf16_tensor_from_bits(x.k_blk),
+                           pk.bf16_tensor_from_bits(x.v_blk), seq_ids=torch.from_numpy(ids).cuda())
+    ref = orc.block_attention(x.q, x.k_blk, x.v_blk, [dp.prefix[2][0], dp.prefix[0][0]],
+                              [dp.prefix[2][1], dp.prefix[0][1]])
+    check_attention(pk.bits_from_bf16_tensor(out), ref)
+
+
+def test_attention_ignores_garbage_beyond_the_sequence_end():
+    """Rows of the last page past seq_len hold arbitrary bits (here NaN patterns): they must not leak."""
+    shape = syn.SHAPE_TINY
+    lens = np.array([70], dtype=np.int32)
+    wl = syn.Workload("attn_nan", shape, 1, 4, 0, 0, (0.9,), seed=34)
+    dp = DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16), lengths=lens)
+    dp.sd._pool.fill_(0xFF)                      # every bf16 in the pool becomes a NaN pattern
+    dp.sd.kv_reset(dp.free_list)
+    k, v = dp.prefix[0]
+    dp.sd.kv_add_seq(0, pk.bf16_tensor_from_bits(k), pk.bf16_tensor_from_bits(v))
+    x = dp.block(0)
+    out = dp.sd.block_attn(x.q, x.k_blk, x.v_blk)
+    ref = orc.block_attention(x.host.q, x.host.k_blk, x.host.v_blk, [k], [v])
+    check_attention(pk.bits_from_bf16_tensor(out), ref)
+
+
+def test_attention_rejects_bad_arguments():
+    shape = syn.SHAPE_TINY
+    wl = syn.Workload("attn_bad", shape, 2, 4, 8, 8, (0.9,), seed=35)
+    dp = DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16))
+    x = dp.block(0)
+    big = torch.zeros((3, 4, 4, 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(pk.SdlmError) as e:
+        dp.sd.block_attn(big, x.k_blk, x.v_blk)
+    assert e.value.code == 2

@@ -1,0 +1,127 @@
+"""GPU parity: page bookkeeping and accept+commit against the oracle (integers bit-exact)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2509_24007_b200 as pk
+from paper_2509_24007_b200.harness import DeviceProblem
+from oracle import sdlm_oracle as orc
+import sdlm_synth as syn
+from oracle_side import oracle_cache
+
+pytestmark = pytest.mark.gpu
+
+
+def _tables_equal(dp, cache):
+    t = dp.sd.kv_tables()
+    assert np.array_equal(t["page_table"], cache.page_table)
+    assert np.array_equal(t["seq_len"], cache.seq_len)
+    assert t["free_head"] == cache.head and t["free_tail"] == cache.tail
+    assert t["status"][0] == 0
+    for b in range(dp.wl.batch):
+        n = int(cache.seq_len[b])
+        k, v = dp.sd.kv_gather(b, n)
+        ok, ov = cache.gather_fast(b)
+        assert np.array_equal(pk.bits_from_bf16_tensor(k), ok), f"K contents differ, seq {b}"
+        assert np.array_equal(pk.bits_from_bf16_tensor(v), ov), f"V contents differ, seq {b}"
+
+
+@pytest.mark.parametrize("shape", [syn.SHAPE_TINY, syn.Shape(8, 8, 128, 64, 64)])
+def test_add_gather_release_match_oracle(shape):
+    lens = np.array([0, 1, 63, 64, 65, 128, 200], dtype=np.int32)
+    wl = syn.Workload("kv", shape, len(lens), 4, 0, 0, (0.9,), seed=11)
+    dp = DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16), lengths=lens)
+    cache = oracle_cache(wl, lens, dp.num_pages, dp.mpps, dp.prefix)
+    _tables_equal(dp, cache)
+    # release two sequences, add one again: the ring hands the released pages back in order
+    for b in (5, 2):
+        dp.sd.kv_release_seq(b); cache.release_sequence(b)
+    k, v = syn.prefix_kv(wl.with_(seed=99), 2, 777 % (dp.mpps * 64))
+    k, v = k[:130], v[:130]
+    dp.sd.kv_add_seq(2, pk.bf16_tensor_from_bits(k), pk.bf16_tensor_from_bits(v))
+    cache.add_sequence_fast(2, k, v)
+    _tables_equal(dp, cache)
+    # export / reset / import restores the tables
+    snap = dp.sd.kv_export()
+    dp.sd.kv_reset()
+    assert dp.sd.kv_tables()["seq_len"].sum() == 0
+    dp.sd.kv_import(snap)
+    _tables_equal(dp, cache)
+
+
+@pytest.mark.parametrize("mode", [orc.CONF_LOGIT, orc.CONF_ENTROPY])
+@pytest.mark.parametrize("D", [1, 4, 8])
+def test_accept_commit_matches_oracle(D, mode):
+    shape = syn.SHAPE_TINY
+    lens = np.array([0, 60, 63, 64, 61, 127, 128, 5, 56, 57, 120, 64 * 3 - 1], dtype=np.int32)
+    B = len(lens)
+    wl = syn.Workload("commit", shape, B, D, 0, 0, (0.9,), seed=12)
+    dp = DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16), lengths=lens)
+    cache = oracle_cache(wl, lens, dp.num_pages, dp.mpps, dp.prefix)
+    rng = np.random.default_rng(D * 10 + mode)
+    for it in range(3):
+        x = syn.block_inputs(wl, dp.w_bits, step=it)
+        levels = np.array([0.999, 0.97, 0.93, 0.5, 1.0], np.float32)
+        p = levels[rng.integers(0, len(levels), size=(B, D))]
+        ent = (rng.random((B, D)) * 0.8).astype(np.float32)
+        token = rng.integers(0, shape.vocab, size=(B, D)).astype(np.int32)
+        for tau in (0.9, 0.0, 1.5):
+            conf = p.astype(np.float64) if mode == orc.CONF_LOGIT else 1.0 - ent.astype(np.float64) / np.log(shape.vocab)
+            res = orc.accept_and_commit(cache, range(B), token, conf, tau, x.k_blk, x.v_blk)
+            acc, out_tok = dp.sd.accept_commit(tau, torch.from_numpy(token).cuda(), torch.from_numpy(p).cuda(),
+                                               torch.from_numpy(ent).cuda(), pk.bf16_tensor_from_bits(x.k_blk),
+                                               pk.bf16_tensor_from_bits(x.v_blk), mode=mode)
+            near = res.tau_margin < 1e-6
+            assert np.array_equal(acc.cpu().numpy()[~near], res.accepted_len[~near])
+            assert not near.any()      # the crafted confidences stay away from the threshold
+            assert np.array_equal(out_tok.cpu().numpy(), res.out_tokens)
+            _tables_equal(dp, cache)
+    assert dp.sd.device_status()[0] == 0
+
+
+def test_commit_with_seq_ids_and_pool_untouched_elsewhere():
+    shape = syn.SHAPE_TINY
+    lens = np.array([10, 64, 100, 130], dtype=np.int32)
+    wl = syn.Workload("ids", shape, 4, 4, 0, 0, (0.9,), seed=13)
+    dp = DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16), lengths=lens)
+    cache = oracle_cache(wl, lens, dp.num_pages, dp.mpps, dp.prefix)
+    ids = np.array([2, 0], dtype=np.int32)        # batch rows map to slots 2 and 0
+    sub = wl.with_(batch=2)
+    x = syn.block_inputs(sub, dp.w_bits)
+    p = np.array([[0.99, 0.99, 0.5, 0.9], [0.95, 0.94, 0.99, 0.99]], np.float32)
+    token = np.arange(8, dtype=np.int32).reshape(2, 4)
+    before = dp.sd._pool.clone()
+    res = orc.accept_and_commit(cache, ids, token, p.astype(np.float64), 0.9, x.k_blk, x.v_blk)
+    acc, _ = dp.sd.accept_commit(0.9, torch.from_numpy(token).cuda(), torch.from_numpy(p).cuda(),
+                                 torch.zeros(2, 4, device="cuda"), pk.bf16_tensor_from_bits(x.k_blk),
+                                 pk.bf16_tensor_from_bits(x.v_blk), seq_ids=torch.from_numpy(ids).cuda())
+    assert acc.cpu().tolist() == res.accepted_len.tolist() == [2, 1]
+    _tables_equal(dp, cache)
+    changed = int((dp.sd._pool != before).sum().item())
+    assert changed <= 3 * shape.n_kv_heads * 2 * shape.head_dim * 2     # only the 3 committed token rows
+
+
+def test_out_of_pages_and_capacity_are_reported_not_fatal():
+    shape = syn.SHAPE_TINY
+    cfg = pk.SdlmConfig(shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.hidden, shape.vocab,
+                        num_pages=3, max_batch=3, max_pages_per_seq=2, max_block=4)
+    sd = pk.Sdlm(cfg)
+    rng = np.random.default_rng(0)
+    mk = lambda n: pk.bf16_tensor_from_bits(rng.integers(0, 1 << 15, size=(n, 2, 64)).astype(np.uint16))
+    sd.kv_add_seq(0, mk(64), mk(64))      # 1 page, full
+    sd.kv_add_seq(1, mk(126), mk(126))    # 2 pages, 2 tokens left of capacity
+    sd.kv_add_seq(2, mk(64), mk(64))      # no page left
+    t = sd.kv_tables()
+    assert t["status"][0] == 4 and t["status"][1] == 2 and t["seq_len"].tolist() == [64, 126, 0]
+    sd.device_status(clear=True)
+    B, D = 2, 4
+    p = torch.full((B, D), 0.999, device="cuda")
+    acc, out_tok = sd.accept_commit(0.5, torch.zeros((B, D), dtype=torch.int32, device="cuda"), p, torch.zeros_like(p),
+                                    mk(B * D).view(B, D, 2, 64), mk(B * D).view(B, D, 2, 64))
+    # slot 0 needs a page and none is free; slot 1 would outgrow max_pages_per_seq
+    assert acc.cpu().tolist() == [-1, -1]
+    assert out_tok.cpu().tolist() == [[-1] * 4] * 2
+    st = sd.device_status()
+    assert st[0] in (4, 7) and st[3] == 2
+    t = sd.kv_tables()
+    assert t["seq_len"].tolist() == [64, 126, 0] and t["free_head"] == 3

@@ -1,0 +1,175 @@
+"""GPU parity of the whole decode step on the benchmark's five configurations.
+
+Each test builds the same seeded inputs for the oracle and for the library, runs
+(a) attention + (b) LM-head statistics + (c) accept/commit through the C ABI, and compares:
+tokens, accepted lengths, page tables and cache contents bit-exactly (near-ties reported),
+attention within 2e-2 max-abs, confidences within 1e-3.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2509_24007_b200 as pk
+from paper_2509_24007_b200.harness import DeviceProblem
+from oracle import sdlm_oracle as orc
+import sdlm_synth as syn
+from oracle_side import (check_attention, check_confidences, check_gamma, check_tokens, oracle_cache)
+
+pytestmark = pytest.mark.gpu
+
+
+def _compare_tables(dp, cache, sample_seqs=None):
+    t = dp.sd.kv_tables()
+    assert t["status"][0] == 0
+    assert np.array_equal(t["page_table"], cache.page_table)
+    assert np.array_equal(t["seq_len"], cache.seq_len)
+    assert t["free_head"] == cache.head
+    for b in (range(dp.wl.batch) if sample_seqs is None else sample_seqs):
+        n = int(cache.seq_len[b])
+        k, v = dp.sd.kv_gather(b, n)
+        ok, ov = cache.gather_fast(b)
+        assert np.array_equal(pk.bits_from_bf16_tensor(k), ok) and np.array_equal(pk.bits_from_bf16_tensor(v), ov)
+
+
+def _one_step(dp, cache, tau, step=0, mode=orc.CONF_LOGIT, w64=None, attn_rows=None, report=None):
+    """Runs step `step` on both sides; returns (gpu outputs, oracle StepResult)."""
+    report = report if report is not None else []
+    wl = dp.wl
+    x = dp.block(step)
+    out = dp.step(x, tau, mode=mode)
+    torch.cuda.synchronize()
+    # oracle: attention over the cache as it was before the commit
+    seqs = list(range(wl.batch)) if attn_rows is None else attn_rows
+    pk_, pv_ = zip(*[cache.gather_fast(b) for b in seqs])
+    ref_attn = orc.block_attention(x.host.q[seqs], x.host.k_blk[seqs], x.host.v_blk[seqs], pk_, pv_)
+    check_attention(pk.bits_from_bf16_tensor(out.attn)[seqs], ref_attn)
+    stats = orc.lm_head_statistics(x.host.hidden, dp.w_bits, w64)
+    check_tokens(out.token.cpu().numpy(), stats, report)
+    check_confidences(out.p_top1.cpu().numpy(), out.entropy.cpu().numpy(), stats)
+    conf = orc.confidences(stats, mode).reshape(wl.batch, wl.block)
+    res = orc.accept_and_commit(cache, range(wl.batch), stats.token.reshape(wl.batch, wl.block), conf, tau,
+                                x.host.k_blk, x.host.v_blk)
+    n_bad = check_gamma(out.accepted_len.cpu().numpy(), res, report)
+    return out, stats, res, n_bad
+
+
+def test_cfg0_tiny_step_both_confidence_modes():
+    wl = syn.CONFIGS["cfg0"]
+    for mode in (orc.CONF_LOGIT, orc.CONF_ENTROPY):
+        dp = DeviceProblem(wl)
+        cache = oracle_cache(wl, dp.lengths, dp.num_pages, dp.mpps, dp.prefix)
+        for step in range(6):        # several steps: the cache grows across a page boundary
+            out, stats, res, n_bad = _one_step(dp, cache, wl.tau, step, mode)
+            assert n_bad == 0
+            assert np.array_equal(out.out_tokens.cpu().numpy(), res.out_tokens)
+            _compare_tables(dp, cache)
+        assert cache.head == 3 and cache.seq_len[0] > 128
+
+
+def test_cfg1_3b_single_sequence_tau_sweep():
+    wl = syn.CONFIGS["cfg1"]
+    dp = DeviceProblem(wl)
+    x = dp.block(0)
+    stats = None
+    gammas = []
+    for tau in wl.taus:
+        dp.reset_cache()
+        cache = oracle_cache(wl, dp.lengths, dp.num_pages, dp.mpps, dp.prefix)
+        report = []
+        out, stats, res, n_bad = _one_step(dp, cache, tau, 0, report=report)
+        assert n_bad == 0, report
+        _compare_tables(dp, cache)
+        gammas.append(int(res.accepted_len[0]))
+    assert gammas == sorted(gammas, reverse=True)          # a higher threshold never accepts more
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg2_d4"])
+def test_cfg2_3b_ragged_batch(name):
+    wl = syn.CONFIGS[name]
+    dp = DeviceProblem(wl)
+    cache = oracle_cache(wl, dp.lengths, dp.num_pages, dp.mpps, dp.prefix)
+    report = []
+    out, stats, res, n_bad = _one_step(dp, cache, wl.tau, 0, report=report)
+    print(name, "flagged:", report, "gamma hist:", np.bincount(res.accepted_len, minlength=wl.block + 1).tolist())
+    _compare_if_in_sync(dp, cache, n_bad)
+    assert 1.0 <= res.accepted_len.mean() <= wl.block
+
+
+def _compare_if_in_sync(dp, cache, n_bad):
+    if n_bad == 0:
+        _compare_tables(dp, cache)
+
+
+def test_cfg3_32b_batch64():
+    wl = syn.CONFIGS["cfg3"]
+    dp = DeviceProblem(wl, keep_prefix=True)
+    cache = oracle_cache(wl, dp.lengths, dp.num_pages, dp.mpps, dp.prefix)
+    report = []
+    # attention is compared on a sample of sequences (shortest, longest, first, last, three more)
+    order = np.argsort(dp.lengths)
+    sample = sorted({int(order[0]), int(order[-1]), 0, wl.batch - 1, 7, 21, 40})
+    out, stats, res, n_bad = _one_step(dp, cache, wl.tau, 0, attn_rows=sample, report=report)
+    print("cfg3 flagged:", report, "gamma hist:", np.bincount(res.accepted_len, minlength=wl.block + 1).tolist())
+    if n_bad == 0:
+        _compare_tables(dp, cache, sample_seqs=sample)
+
+
+def test_cfg4_long_prefix_multi_step_loop():
+    wl = syn.CONFIGS["cfg4"]
+    dp = DeviceProblem(wl)
+    cache = oracle_cache(wl, dp.lengths, dp.num_pages, dp.mpps, dp.prefix)
+    w64 = orc.widen(dp.w_bits)
+    outs = dp.alloc_outputs()
+    total_gpu = total_ref = 0
+    flagged = []
+    for step in range(wl.steps):
+        x = dp.block(step)
+        check_attn = step in (0, wl.steps // 2, wl.steps - 1)
+        if check_attn:
+            seqs = [0, wl.batch - 1]
+            pk_, pv_ = zip(*[cache.gather_fast(b) for b in seqs])
+            ref_attn = orc.block_attention(x.host.q[seqs], x.host.k_blk[seqs], x.host.v_blk[seqs], pk_, pv_)
+        dp.step(x, wl.tau, outs)
+        torch.cuda.synchronize()
+        if check_attn:
+            check_attention(pk.bits_from_bf16_tensor(outs.attn)[seqs], ref_attn)
+        stats = orc.lm_head_statistics(x.host.hidden, dp.w_bits, w64)
+        check_tokens(outs.token.cpu().numpy(), stats, flagged)
+        check_confidences(outs.p_top1.cpu().numpy(), outs.entropy.cpu().numpy(), stats)
+        conf = stats.p_top1.reshape(wl.batch, wl.block)
+        res = orc.accept_and_commit(cache, range(wl.batch), stats.token.reshape(wl.batch, wl.block), conf, wl.tau,
+                                    x.host.k_blk, x.host.v_blk)
+        n_bad = check_gamma(outs.accepted_len.cpu().numpy(), res, flagged)
+        assert n_bad == 0, f"step {step}: accepted lengths diverged at a flagged near-threshold position {flagged[-1]}"
+        assert np.array_equal(outs.out_tokens.cpu().numpy(), res.out_tokens)
+        total_gpu += int(outs.accepted_len.sum().item()); total_ref += int(res.accepted_len.sum())
+    assert total_gpu == total_ref
+    assert np.array_equal(cache.seq_len[:wl.batch], dp.lengths + (cache.seq_len[:wl.batch] - dp.lengths))
+    assert int(cache.seq_len.sum()) == int(dp.lengths.sum()) + total_ref
+    _compare_tables(dp, cache)
+    print("cfg4 committed", total_ref, "tokens in", wl.steps, "steps; flagged", flagged)
+
+
+def test_decode_step_host_entry_matches_device_calls():
+    wl = syn.CONFIGS["cfg0"].with_(batch=3, prefix_lo=10, prefix_hi=200)
+    dp = DeviceProblem(wl)
+    x = dp.block(0)
+    ref = dp.step(x, wl.tau)
+    torch.cuda.synchronize()
+    t_ref = dp.sd.kv_tables()
+    dp.reset_cache()
+    pin = lambda t: t.cpu().pin_memory()
+    B, D, s = wl.batch, wl.block, wl.shape
+    attn = torch.empty((B, D, s.n_q_heads, s.head_dim), dtype=torch.bfloat16).pin_memory()
+    tok = torch.empty((B, D), dtype=torch.int32).pin_memory()
+    p = torch.empty((B, D), dtype=torch.float32).pin_memory()
+    ent = torch.empty((B, D), dtype=torch.float32).pin_memory()
+    acc = torch.empty(B, dtype=torch.int32).pin_memory()
+    out_tok = torch.empty((B, D), dtype=torch.int32).pin_memory()
+    dp.sd.decode_step_host(wl.tau, pin(x.q), pin(x.k_blk), pin(x.v_blk), pin(x.hidden), dp.w_lm, attn, tok, p, ent,
+                           acc, out_tok)
+    assert torch.equal(attn, ref.attn.cpu()) and torch.equal(tok, ref.token.cpu())
+    assert torch.equal(p, ref.p_top1.cpu()) and torch.equal(acc, ref.accepted_len.cpu())
+    assert torch.equal(out_tok, ref.out_tokens.cpu())
+    t = dp.sd.kv_tables()
+    assert np.array_equal(t["page_table"], t_ref["page_table"]) and np.array_equal(t["seq_len"], t_ref["seq_len"])
