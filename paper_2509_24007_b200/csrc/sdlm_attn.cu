@@ -99,7 +99,8 @@ __global__ void __launch_bounds__(MT* WPM * 32, 2) block_attn_kernel(const AttnP
   uint8_t* stages = smem;
   uint8_t* q_s = smem + kAttnStages * STAGE_B;
   uint64_t* full = reinterpret_cast<uint64_t*>(q_s + ROWS * ROWB);
-  int* s_first = reinterpret_cast<int*>(full + kAttnStages);
+  volatile int* abort = reinterpret_cast<volatile int*>(full + kAttnStages);
+  int* s_first = const_cast<int*>(abort) + 2;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int mt = warp / WPM, kq = warp % WPM;
@@ -107,6 +108,7 @@ __global__ void __launch_bounds__(MT* WPM * 32, 2) block_attn_kernel(const AttnP
 
   if (tid == 0) {
     for (int s = 0; s < kAttnStages; ++s) ptx::mbar_init(&full[s], 1);
+    *abort = 0;
     ptx::fence_barrier_init();
   }
   const AttnSched sc = attn_schedule(p, s_first);  // contains a __syncthreads
@@ -242,7 +244,9 @@ __global__ void __launch_bounds__(MT* WPM * 32, 2) block_attn_kernel(const AttnP
       if (tid == 0 && t + kAttnStages - 1 < n_tiles) issue(t + kAttnStages - 1);
       const uint32_t c = tile_ctr + (uint32_t)t;
       const int stage = c % kAttnStages;
-      if (!ptx::mbar_wait(&full[stage], (c / kAttnStages) & 1)) attn_timeout(p);
+      // a wait that runs out is recorded and the tile is processed as it is (the result is then
+      // meaningless but every access stays inside shared memory); later waits return at once
+      if (!ptx::mbar_wait(&full[stage], (c / kAttnStages) & 1, abort) && (tid & 31) == 0) attn_timeout(p);
       uint8_t* sp = stages + stage * STAGE_B;
       int valid = kPageSize;
       if (pg0 + t == pages - 1) valid = len - (pages - 1) * kPageSize;
@@ -323,6 +327,14 @@ __global__ void __launch_bounds__(MT* WPM * 32, 2) block_attn_kernel(const AttnP
     }
     ptx::fence_proxy_async();
     __syncthreads();
+    const int dead = *abort;
+    __syncthreads();  // every thread has read the flag before anyone can set it in the next item
+    if (dead) {  // winding down: let this item's copies land, then stop taking items
+      if (tid == 0)
+        for (uint32_t c = tile_ctr > kAttnStages ? tile_ctr - kAttnStages : 0; c < tile_ctr; ++c)
+          ptx::mbar_wait_brief(&full[c % kAttnStages], (c / kAttnStages) & 1);
+      break;
+    }
   }
 }
 
@@ -357,7 +369,7 @@ __global__ void __launch_bounds__(256) block_attn_combine_kernel(const AttnParam
 // ---------------------------------------------------------------------------------------------
 template <int HD, int MT, int WPM>
 static size_t attn_smem_bytes(int batch) {
-  return 1024 + (size_t)kAttnStages * 2 * kPageSize * HD * 2 + (size_t)MT * 16 * HD * 2 + kAttnStages * 8 +
+  return 1024 + (size_t)kAttnStages * 2 * kPageSize * HD * 2 + (size_t)MT * 16 * HD * 2 + kAttnStages * 8 + 8 +
          (size_t)(batch + 1) * 4 + 16;
 }
 

@@ -135,7 +135,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
   uint64_t* empty = full + n_stages;
   uint64_t* acc_full = empty + n_stages;
   uint64_t* acc_empty = acc_full + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* drain = acc_empty + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+  volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -156,6 +158,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
       ptx::mbar_init(&acc_full[s], 1);
       ptx::mbar_init(&acc_empty[s], 4);
     }
+    ptx::mbar_init(drain, 1);
+    *abort = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmap_h);
     ptx::prefetch_tmap(&tmap_w);
@@ -172,11 +176,15 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
   if (warp == 0) {
     if (lane == 0) {  // ---- TMA producer
       uint32_t it = 0;
-      for (int t = 0; t < n_tiles; ++t) {
+      bool ok = true;
+      for (int t = 0; t < n_tiles && ok; ++t) {
         const int n0 = n_begin + t * p.bn;
         for (int kc = 0; kc < KC; ++kc, ++it) {
           const int s = it % n_stages;
-          if (it >= (uint32_t)n_stages && !ptx::mbar_wait(&empty[s], ((it / n_stages) & 1) ^ 1)) lm_timeout(p.hdr, 1);
+          if (it >= (uint32_t)n_stages && !ptx::mbar_wait(&empty[s], ((it / n_stages) & 1) ^ 1, abort)) {
+            ok = false;
+            break;
+          }
           uint8_t* st = smem + (size_t)s * stage_bytes;
           ptx::mbar_arrive_expect_tx(&full[s], (uint32_t)stage_bytes);
 #pragma unroll
@@ -184,20 +192,32 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
           ptx::tma_load_2d(st + R * kATileBytes, &tmap_w, kc * kBK, n0, &full[s]);
         }
       }
+      if (!ok || *abort) {  // winding down: let the copies already issued land before the CTA goes away
+        lm_timeout(p.hdr, 1);
+        const uint32_t first = it > (uint32_t)n_stages ? it - n_stages : 0;
+        for (uint32_t j = first; j < it; ++j) ptx::mbar_wait_brief(&full[j % n_stages], (j / n_stages) & 1);
+      }
     }
   } else if (warp == 1) {
     if (lane == 0) {  // ---- MMA issuer
       // instruction descriptor: D fp32, A and B bf16, both K-major, N = bn, M = 128
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.bn >> 3) << 17) | ((128u >> 4) << 24);
       uint32_t it = 0;
-      for (int t = 0; t < n_tiles; ++t) {
+      bool ok = true;
+      for (int t = 0; t < n_tiles && ok; ++t) {
         const int as = t % NACC;
         const uint32_t use = (uint32_t)t / NACC;
-        if (use > 0 && !ptx::mbar_wait(&acc_empty[as], (use & 1) ^ 1)) lm_timeout(p.hdr, 2);
+        if (use > 0 && !ptx::mbar_wait(&acc_empty[as], (use & 1) ^ 1, abort)) {
+          ok = false;
+          break;
+        }
         ptx::tc_fence_after();
         for (int kc = 0; kc < KC; ++kc, ++it) {
           const int s = it % n_stages;
-          if (!ptx::mbar_wait(&full[s], (it / n_stages) & 1)) lm_timeout(p.hdr, 3);
+          if (!ptx::mbar_wait(&full[s], (it / n_stages) & 1, abort)) {
+            ok = false;
+            break;
+          }
           ptx::tc_fence_after();
           const uint32_t a_addr = ptx::smem_u32(smem + (size_t)s * stage_bytes);
           const uint32_t b_addr = a_addr + R * kATileBytes;
@@ -211,7 +231,12 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
           }
           ptx::umma_commit(&empty[s]);  // stage reusable once these MMAs have read it
         }
-        ptx::umma_commit(&acc_full[as]);  // accumulator complete
+        if (ok) ptx::umma_commit(&acc_full[as]);  // accumulator complete
+      }
+      if (!ok) {  // winding down: the MMAs already issued must finish before TMEM and smem are released
+        lm_timeout(p.hdr, 2);
+        ptx::umma_commit(drain);
+        ptx::mbar_wait_brief(drain, 0);
       }
     }
   } else {  // ---- epilogue: TMEM lane = hidden-state row
@@ -222,7 +247,11 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
     for (int t = 0; t < n_tiles; ++t) {
       const int as = t % NACC;
       const uint32_t use = (uint32_t)t / NACC;
-      if (!ptx::mbar_wait(&acc_full[as], use & 1)) lm_timeout(p.hdr, 4);
+      // the whole warp takes the same branch: the tensor-memory loads below are warp-collective
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&acc_full[as], use & 1, abort))) {
+        if (lane == 0) lm_timeout(p.hdr, 3);
+        break;
+      }
       ptx::tc_fence_after();
       const int n0 = n_begin + t * p.bn;
       const int n_chunks = p.bn / 16;
@@ -500,7 +529,7 @@ sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const voi
       ctx->tmap_w_rows = p.bn;
     }
     const CUtensorMap& tm_w = *reinterpret_cast<const CUtensorMap*>(ctx->tmap_w);
-    const size_t smem = (size_t)n_stages * stage_bytes + 1024 + 256;
+    const size_t smem = (size_t)n_stages * stage_bytes + 1024 + 512;
     if (R == 1)
       lmhead_umma_kernel<1><<<n_cta, kUmmaThreads, smem, st>>>(tm_h, tm_w, p, n_stages);
     else

@@ -37,12 +37,36 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after ~0.3 s of polling and returns false (the caller records a timeout
-// status and carries on; every loop around it is bounded, so the kernel still ends).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  for (uint32_t i = 0; i < (1u << 22); ++i) {
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Polls until the phase with `parity` completes; gives up when `*abort` is already
+// set (another wait of this CTA ran out) or after about 0.2 s of wall time, in which case it sets
+// `*abort` and returns false.  Callers leave their loops on false, so a CTA whose pipeline stalls
+// ends within one such interval instead of spinning.
+constexpr uint64_t kWaitLimitNs = 200ull * 1000 * 1000;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_ns();
+  for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (i > 1024) __nanosleep(64);
+    if ((i & 63u) == 0) {
+      if (*abort) return false;
+      if (global_ns() - t0 > kWaitLimitNs) {
+        *abort = 1;
+        return false;
+      }
+      __nanosleep(32);
+    }
+  }
+}
+// Wait used only while winding down after a failed wait: a short, fixed number of polls.
+__device__ __forceinline__ bool mbar_wait_brief(uint64_t* bar, uint32_t parity) {
+  for (uint32_t i = 0; i < 4096; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    __nanosleep(256);
   }
   return false;
 }
