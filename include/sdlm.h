@@ -162,6 +162,28 @@ sdlm_status sdlm_lmhead_confidence(sdlm_ctx* ctx, int32_t rows, const void* hidd
                                    int32_t* token, float* p_top1, float* entropy, float* max_logit,
                                    float* lse, void* stream);
 
+/* ---- (b'), for callers that cannot allocate -- the paper has no counterpart.
+ * Same inputs, outputs, arithmetic and errors as sdlm_lmhead_confidence, but the per-stripe
+ * partial statistics (the only scratch this step needs) live in a fixed 768 KiB array that is part
+ * of the library image, not in the context's workspace.  It is meant for code that runs where
+ * device allocation is off limits -- a plugin inside a host application whose memory pool is
+ * already sealed, a step replayed under a no-allocation policy, a real-time loop -- and that
+ * therefore cannot grow a workspace for this call.  The call itself allocates nothing: no
+ * cudaMalloc / cudaFree, no allocating library routine.
+ *   - Limits: rows <= SDLM_STATIC_LMHEAD_MAX_ROWS (also <= max_batch*max_block of the context);
+ *     more gives SDLM_ERR_SHAPE and nothing is enqueued.  The array costs its 768 KiB on every
+ *     device that loads the library, until the process exits.
+ *   - The first call on a device looks up the array's device address (once per device, with the
+ *     context's device current; any other current device gives INVALID_ARG).  Make that first
+ *     call before starting a stream capture.
+ *   - One array per device is shared by every context and stream: calls that may overlap on the
+ *     GPU race on it and must be ordered by the caller.  It keeps the previous call's contents;
+ *     nothing in it has to start at zero, because each call overwrites every entry it later reads. */
+#define SDLM_STATIC_LMHEAD_MAX_ROWS 256
+sdlm_status sdlm_lmhead_confidence_static(sdlm_ctx* ctx, int32_t rows, const void* hidden, const void* w_lm,
+                                          int32_t* token, float* p_top1, float* entropy, float* max_logit,
+                                          float* lse, void* stream);
+
 /* ---- (c) longest-prefix acceptance and commit -- Eq. 7 and Decode of Eq. 4.
  * Per batch row b: c_k = p_top1[b,k] (LOGIT) or 1 - entropy[b,k]/ln|V| (ENTROPY);
  *   gamma = max({ j in 1..D : prod_{k<=j} c_k >= tau } U {1})   (fp32 running product, in order)

@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "UNSUPPORTED", 4: "OUT
                 6: "TIMEOUT", 7: "DEVICE_CHECK", 8: "WORKSPACE"}
 
 EXPORTED = ["sdlm_pool_bytes", "sdlm_workspace_bytes", "sdlm_create", "sdlm_destroy", "sdlm_status_str",
-            "sdlm_kv_pages", "sdlm_block_attn", "sdlm_lmhead_confidence", "sdlm_accept_commit",
+            "sdlm_kv_pages", "sdlm_block_attn", "sdlm_lmhead_confidence", "sdlm_lmhead_confidence_static", "sdlm_accept_commit",
             "sdlm_device_status", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count"]
 
 
@@ -102,6 +102,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdlm_block_attn.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.sdlm_lmhead_confidence.restype = C.c_int
     lib.sdlm_lmhead_confidence.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_lmhead_confidence_static.restype = C.c_int
+    lib.sdlm_lmhead_confidence_static.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_accept_commit.restype = C.c_int
     lib.sdlm_accept_commit.argtypes = [vp, i32, i32, vp, f32, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_device_status.restype = C.c_int
@@ -267,6 +269,17 @@ class Sdlm:
                                                                 _ptr(v_blk), _ptr(_dev(out, torch.bfloat16, "out")),
                                                                 _stream_ptr(stream)))
         return out
+
+    def lmhead_confidence_static(self, hidden: torch.Tensor, w_lm: torch.Tensor, token: torch.Tensor,
+                                 p_top1: torch.Tensor, entropy: torch.Tensor, max_logit: Optional[torch.Tensor] = None,
+                                 lse: Optional[torch.Tensor] = None, stream=None) -> None:
+        """sdlm_lmhead_confidence_static: the caller passes every output; nothing is allocated here."""
+        _dev(hidden, torch.bfloat16, "hidden"); _dev(w_lm, torch.bfloat16, "w_lm")
+        rows = hidden.numel() // self.cfg.hidden
+        self._check("sdlm_lmhead_confidence_static", self.lib.sdlm_lmhead_confidence_static(
+            self.ctx, rows, _ptr(hidden), _ptr(w_lm), _ptr(_dev(token, torch.int32, "token")),
+            _ptr(_dev(p_top1, torch.float32, "p_top1")), _ptr(_dev(entropy, torch.float32, "entropy")),
+            _ptr(max_logit), _ptr(lse), _stream_ptr(stream)))
 
     def lmhead_confidence(self, hidden: torch.Tensor, w_lm: torch.Tensor, token: Optional[torch.Tensor] = None,
                           p_top1: Optional[torch.Tensor] = None, entropy: Optional[torch.Tensor] = None,

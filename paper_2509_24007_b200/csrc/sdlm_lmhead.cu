@@ -20,6 +20,8 @@
 
 #include <cuda.h>
 
+#include <mutex>
+
 namespace sdlm {
 
 constexpr float kLog2e = 1.4426950408889634f;
@@ -495,23 +497,26 @@ cudaError_t setup_lmhead(sdlm_ctx* ctx) {
                               kMmaStages * kMmaStageBytes + 128);
 }
 
-sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
-                          float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st) {
+// `partials` holds one float4 per (stripe, row): [max_stripes][rows_pad].
+static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
+                                    float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st,
+                                    float4* partials, int rows_pad, int max_stripes) {
   const sdlm_config& c = ctx->cfg;
   LmParams p;
   p.hidden = static_cast<const __nv_bfloat16*>(hidden);
   p.w = static_cast<const __nv_bfloat16*>(w_lm);
-  p.partials = reinterpret_cast<float4*>(ctx->ws + ctx->lay.lm_partials);
+  p.partials = partials;
   p.hdr = ctx->hdr;
   p.rows = rows; p.H = c.hidden; p.V = c.vocab;
-  p.rows_pad = c.max_batch * c.max_block;
+  p.rows_pad = rows_pad;
   p.bn = 0;
 
   const bool use_umma = ctx->lmhead_path != 1 && rows <= 256 && c.vocab >= 16;
   if (ctx->lmhead_path == 2 && !use_umma) return SDLM_ERR_UNSUPPORTED;
   if (use_umma) {
     const int groups = (c.vocab + 15) / 16;
-    const int n_cta = groups < ctx->sm_count ? groups : ctx->sm_count;
+    int n_cta = groups < ctx->sm_count ? groups : ctx->sm_count;
+    if (n_cta > max_stripes) n_cta = max_stripes;
     const int gmax = (groups + n_cta - 1) / n_cta;
     const int tiles = (gmax * 16 + 255) / 256;
     p.bn = 16 * ((gmax + tiles - 1) / tiles);
@@ -538,7 +543,7 @@ sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const voi
     const int tiles_total = (c.vocab + kMmaBN - 1) / kMmaBN;
     int n_cta = ctx->sm_count * 2;
     if (n_cta > tiles_total) n_cta = tiles_total;
-    if (n_cta > kLmMaxStripes) n_cta = kLmMaxStripes;
+    if (n_cta > max_stripes) n_cta = max_stripes;
     p.n_stripes = n_cta;
     dim3 grid(n_cta, (rows + kMmaBM - 1) / kMmaBM);
     lmhead_mma_kernel<<<grid, kMmaThreads, kMmaStages * kMmaStageBytes + 128, st>>>(p);
@@ -551,4 +556,60 @@ sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const voi
   return cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
 }
 
+sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
+                          float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st) {
+  return launch_lmhead_on(ctx, rows, hidden, w_lm, token, p_top1, entropy, max_logit, lse, st,
+                          reinterpret_cast<float4*>(ctx->ws + ctx->lay.lm_partials),
+                          ctx->cfg.max_batch * ctx->cfg.max_block, kLmMaxStripes);
+}
+
 }  // namespace sdlm
+
+// ---------------------------------------------------------------------------------------------
+// sdlm_lmhead_confidence_static: the same computation with the per-stripe partial statistics kept
+// in a fixed array inside the library image instead of the caller's workspace.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticMaxRows = SDLM_STATIC_LMHEAD_MAX_ROWS;
+constexpr int kStaticMaxStripes = 192;
+constexpr int kStaticMaxDevices = 64;
+
+// 192 x 256 x 16 B = 768 KiB on every device that loads the library, until the process exits.
+static __device__ __align__(256) float4 g_static_partials[kStaticMaxStripes * kStaticMaxRows];
+
+std::mutex g_static_mutex;
+float4* g_static_ptr[kStaticMaxDevices] = {};
+
+// The array's name is only a host-side handle: the address kernels can use has to be asked for,
+// once per device, with that device current.
+sdlm_status static_partials_for_current_device(int device, float4** out) {
+  if (device < 0 || device >= kStaticMaxDevices) return SDLM_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_ptr[device]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_partials) != cudaSuccess || !ptr) return SDLM_ERR_CUDA;
+    g_static_ptr[device] = static_cast<float4*>(ptr);
+  }
+  *out = g_static_ptr[device];
+  return SDLM_OK;
+}
+
+}  // namespace
+
+extern "C" sdlm_status sdlm_lmhead_confidence_static(sdlm_ctx* ctx, int32_t rows, const void* hidden,
+                                                     const void* w_lm, int32_t* token, float* p_top1,
+                                                     float* entropy, float* max_logit, float* lse, void* stream) {
+  if (!ctx || !hidden || !w_lm || !token || !p_top1 || !entropy) return SDLM_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(hidden) & 15) || (reinterpret_cast<uintptr_t>(w_lm) & 15)) return SDLM_ERR_INVALID_ARG;
+  if (rows < 1) return SDLM_ERR_INVALID_ARG;
+  if (rows > kStaticMaxRows || rows > ctx->cfg.max_batch * ctx->cfg.max_block) return SDLM_ERR_SHAPE;
+  int device = -1;
+  if (cudaGetDevice(&device) != cudaSuccess) return SDLM_ERR_CUDA;
+  if (device != ctx->device) return SDLM_ERR_INVALID_ARG;
+  float4* partials = nullptr;
+  sdlm_status s = static_partials_for_current_device(device, &partials);
+  if (s != SDLM_OK) return s;
+  return sdlm::launch_lmhead_on(ctx, rows, hidden, w_lm, token, p_top1, entropy, max_logit, lse,
+                                static_cast<cudaStream_t>(stream), partials, kStaticMaxRows, kStaticMaxStripes);
+}
