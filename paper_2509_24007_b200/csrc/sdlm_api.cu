@@ -36,10 +36,11 @@ WorkspaceLayout workspace_layout(const sdlm_config& c) {
   L.table_end = off;
   L.lm_partials = take((size_t)kLmMaxStripes * rows * 16);
   const int G = c.n_q_heads / c.n_kv_heads;
-  L.q_rows_pad = (G * c.max_block + 15) / 16 * 16;
-  L.attn_max_items = kAttnTargetItems + c.max_batch * c.n_kv_heads;
+  L.q_rows_pad = G * c.max_block <= 32 ? 32 : 64;
+  L.attn_max_items = kAttnMaxCtas + c.max_batch * c.n_kv_heads;
   L.attn_ml = take((size_t)L.attn_max_items * L.q_rows_pad * 2 * 4);
   L.attn_o = take((size_t)L.attn_max_items * L.q_rows_pad * c.head_dim * 4);
+  L.attn_cnt = take((size_t)c.max_batch * c.n_kv_heads * 4);
   L.st_q = take(rows * c.n_q_heads * c.head_dim * 2);
   L.st_k = take(rows * c.n_kv_heads * c.head_dim * 2);
   L.st_v = take(rows * c.n_kv_heads * c.head_dim * 2);
@@ -105,29 +106,54 @@ __global__ void add_seq_alloc_kernel(DevHeader* hdr, int32_t* page_table, int32_
   }
 }
 
-// Scatter (to_pool = 1) or gather (to_pool = 0) 16-byte chunks between a dense [length, Hkv, d]
-// tensor and the slot's pages.  Does nothing unless the slot holds at least the rows it touches.
+// Scatter (to_pool = 1) or gather (to_pool = 0) between a dense [length, Hkv, d] tensor and the
+// slot's pages, 8 values at a time (a 16-byte chunk of a K row; eight separate V^T elements).
+// Scattering also clears the V^T columns between the sequence end and the end of its last page.
+// Does nothing unless the slot holds at least the rows it touches.
 __global__ void kv_rows_kernel(__nv_bfloat16* pool, const int32_t* page_table, const int32_t* seq_len,
                                __nv_bfloat16* k_dense, __nv_bfloat16* v_dense, int slot, int length, int mpps,
                                int Hkv, int d, int to_pool) {
   const int cpr = d / 8;  // 16-byte chunks per row
   const int have = seq_len[slot];
   if (to_pool && have != length) return;
-  const int n_rows = to_pool ? length : min(length, have);
-  const size_t total = (size_t)n_rows * Hkv * 2 * cpr;
+  const int n_valid = to_pool ? length : min(length, have);
+  const int n_rows = (n_valid + kPageSize - 1) / kPageSize * kPageSize;  // whole pages: key is the fastest index
+  const size_t total = (size_t)n_rows * Hkv * cpr;
   for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
        idx += (size_t)gridDim.x * blockDim.x) {
-    const int c = (int)(idx % cpr);
-    size_t r = idx / cpr;
-    const int kv = (int)(r % 2); r /= 2;
+    // consecutive threads take consecutive keys of one (head, chunk): V^T writes then share sectors
+    const int key = (int)(idx % kPageSize);
+    size_t r = idx / kPageSize;
+    const int c = (int)(r % cpr); r /= cpr;
     const int h = (int)(r % Hkv);
-    const int t = (int)(r / Hkv);
+    const int t = (int)(r / Hkv) * kPageSize + key;
     const int page = page_table[(size_t)slot * mpps + t / kPageSize];
-    const int row = t % kPageSize;
-    uint4* pool_p = reinterpret_cast<uint4*>(pool + kv_tile_offset(page, h, kv, Hkv, d) + (size_t)row * d) +
-                    kv_swizzled_chunk(row, c);
-    uint4* dense_p = reinterpret_cast<uint4*>((kv ? v_dense : k_dense) + ((size_t)t * Hkv + h) * d) + c;
-    if (to_pool) *pool_p = *dense_p; else *dense_p = *pool_p;
+    __nv_bfloat16* k_tile = pool + kv_tile_offset(page, h, 0, Hkv, d);
+    __nv_bfloat16* v_tile = pool + kv_tile_offset(page, h, 1, Hkv, d);
+    if (t >= n_valid) {  // padding rows of the last page: cleared when scattering, skipped when gathering
+      if (to_pool) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v_tile[vt_tile_elem(key, c * 8 + e)] = __float2bfloat16_rn(0.f);
+      }
+      continue;
+    }
+    uint4* k_pool = reinterpret_cast<uint4*>(k_tile + k_tile_elem(key, c * 8));
+    uint4* k_d = reinterpret_cast<uint4*>(k_dense + ((size_t)t * Hkv + h) * d) + c;
+    uint4* v_d = reinterpret_cast<uint4*>(v_dense + ((size_t)t * Hkv + h) * d) + c;
+    if (to_pool) {
+      *k_pool = *k_d;
+      const uint4 vv = *v_d;
+      const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(&vv);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v_tile[vt_tile_elem(key, c * 8 + e)] = ve[e];
+    } else {
+      *k_d = *k_pool;
+      uint4 vv;
+      __nv_bfloat16* ve = reinterpret_cast<__nv_bfloat16*>(&vv);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) ve[e] = v_tile[vt_tile_elem(key, c * 8 + e)];
+      *v_d = vv;
+    }
   }
 }
 
@@ -275,22 +301,31 @@ __global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitPar
   }
   if (tid == 0) p.accepted_len[b] = g;
   for (int k = tid; k < p.D; k += kCommitThreads) p.out_tokens[b * p.D + k] = (k < g) ? p.token[b * p.D + k] : -1;
+  if (need) {  // a page fresh from the ring may hold anything: clear its V^T tiles first
+    const int per_head = kPageSize * p.d / 8;
+    for (int idx = tid; idx < p.Hkv * per_head; idx += kCommitThreads)
+      reinterpret_cast<uint4*>(p.pool + kv_tile_offset(new_page, idx / per_head, 1, p.Hkv, p.d))[idx % per_head] =
+          make_uint4(0, 0, 0, 0);
+    __syncthreads();
+  }
   const int cpr = p.d / 8;
-  const int total = g * p.Hkv * 2 * cpr;
+  const int total = g * p.Hkv * cpr;
   for (int idx = tid; idx < total; idx += kCommitThreads) {
     const int c = idx % cpr;
     int r = idx / cpr;
-    const int kv = r % 2; r /= 2;
     const int h = r % p.Hkv;
     const int t = r / p.Hkv;
     const int pos = len + t;
-    const int pidx = pos / kPageSize, row = pos % kPageSize;
+    const int pidx = pos / kPageSize, key = pos % kPageSize;
     const int page = (need && pidx == new_idx) ? new_page : p.page_table[(size_t)slot * p.mpps + pidx];
-    const uint4* src = reinterpret_cast<const uint4*>((kv ? p.v_blk : p.k_blk) +
-                                                      (((size_t)b * p.D + t) * p.Hkv + h) * p.d) + c;
-    uint4* dst = reinterpret_cast<uint4*>(p.pool + kv_tile_offset(page, h, kv, p.Hkv, p.d) + (size_t)row * p.d) +
-                 kv_swizzled_chunk(row, c);
-    *dst = *src;
+    const size_t src = (((size_t)b * p.D + t) * p.Hkv + h) * p.d;
+    *reinterpret_cast<uint4*>(p.pool + kv_tile_offset(page, h, 0, p.Hkv, p.d) + k_tile_elem(key, c * 8)) =
+        *(reinterpret_cast<const uint4*>(p.k_blk + src) + c);
+    const uint4 vv = *(reinterpret_cast<const uint4*>(p.v_blk + src) + c);
+    const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(&vv);
+    __nv_bfloat16* v_tile = p.pool + kv_tile_offset(page, h, 1, p.Hkv, p.d);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v_tile[vt_tile_elem(key, c * 8 + e)] = ve[e];
   }
 }
 
@@ -335,6 +370,8 @@ static sdlm_status reset_tables(sdlm_ctx* ctx, const int32_t* host_free_list, cu
         cudaSuccess)
       return SDLM_ERR_CUDA;
   }
+  if (cudaMemsetAsync(ctx->ws + ctx->lay.attn_cnt, 0, (size_t)c.max_batch * c.n_kv_heads * 4, st) != cudaSuccess)
+    return SDLM_ERR_CUDA;
   reset_tables_kernel<<<64, 256, 0, st>>>(ctx->hdr, ctx->page_table, ctx->seq_len, ctx->free_list,
                                          c.max_batch * c.max_pages_per_seq, c.max_batch, c.num_pages,
                                          host_free_list ? 0 : 1);
@@ -415,7 +452,7 @@ extern "C" sdlm_status sdlm_kv_pages(sdlm_ctx* ctx, sdlm_kv_op op, const sdlm_kv
       if (a->length == 0) return SDLM_OK;
       add_seq_alloc_kernel<<<1, 256, 0, st>>>(ctx->hdr, ctx->page_table, ctx->seq_len, ctx->free_list, a->seq,
                                               a->length, c.max_pages_per_seq, c.num_pages);
-      const size_t chunks = (size_t)a->length * c.n_kv_heads * 2 * (c.head_dim / 8);
+      const size_t chunks = (size_t)(a->length + kPageSize) * c.n_kv_heads * (c.head_dim / 8);
       const int blocks = (int)((chunks + 255) / 256 < 4096 ? (chunks + 255) / 256 : 4096);
       kv_rows_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<__nv_bfloat16*>(ctx->pool), ctx->page_table,
                                              ctx->seq_len, (__nv_bfloat16*)a->k, (__nv_bfloat16*)a->v, a->seq,
@@ -446,7 +483,7 @@ extern "C" sdlm_status sdlm_kv_pages(sdlm_ctx* ctx, sdlm_kv_op op, const sdlm_kv
         return SDLM_ERR_INVALID_ARG;
       if (a->length == 0) return SDLM_OK;
       if (!a->k_out || !a->v_out || !aligned16(a->k_out) || !aligned16(a->v_out)) return SDLM_ERR_INVALID_ARG;
-      const size_t chunks = (size_t)a->length * c.n_kv_heads * 2 * (c.head_dim / 8);
+      const size_t chunks = (size_t)(a->length + kPageSize) * c.n_kv_heads * (c.head_dim / 8);
       const int blocks = (int)((chunks + 255) / 256 < 4096 ? (chunks + 255) / 256 : 4096);
       kv_rows_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<__nv_bfloat16*>(ctx->pool), ctx->page_table,
                                              ctx->seq_len, (__nv_bfloat16*)a->k_out, (__nv_bfloat16*)a->v_out,

@@ -1,20 +1,32 @@
 // (a) Block-decode attention (Sec. 3.3 single-block mask, rows u >= i): the D rows of a block
 // attend to every cached token of their sequence and, unmasked, to the D block tokens.
 //
-// Split-KV over a paged pool.  A work item is (batch row, KV head, range of cache pages); the
-// G*D query rows that share a KV head (G = Hq/Hkv) are stacked into 16-row tiles so that each
-// K/V byte fetched from HBM feeds G*D dot products on the tensor cores (mma.sync m16n8k16, bf16
-// in, fp32 accumulate).  K/V page tiles are contiguous 64*d*2-byte runs, pre-swizzled in the pool,
-// and are staged into shared memory with bulk (TMA-engine) copies on an mbarrier ring.  Softmax is
-// online in the log2 domain; partial (max, sum, O) per item are merged by a second kernel unless
-// one item covers the whole sequence.  The item list is derived on the device from seq_len, so
-// no host synchronisation is needed between steps.
+// One persistent CTA per SM.  The tiles of the whole batch -- one per cached page and KV head, plus
+// one per (sequence, KV head) for the D block tokens -- form one sequence that is cut into equal
+// contiguous ranges, one per CTA, so every SM streams the same number of bytes.  The part of a
+// (sequence, KV head) pair that falls into one CTA's range is an "item"; a pair cut by a range
+// boundary leaves partial (max, sum, O) results, which the last of its CTAs to finish merges
+// (arrival counter per pair; nobody waits).
+//
+// Inside a CTA the work is warp-specialised around the 5th-generation tensor cores:
+//   warp 0      issues one bulk copy per cached tile (K tile + V^T tile, contiguous in the pool and
+//               already in the tensor-core shared-memory layout) into an mbarrier ring;
+//   warp 1      one thread issues tcgen05.mma:  S = Q K^T  (M = 128, N = 64 keys, fp32 in tensor
+//               memory, double-buffered)  and  O += P V  (M = 128, N = d);
+//   warps 2..5  softmax: thread = one accumulator lane = one query row.  It reads its row of S,
+//               keeps the running max and sum, writes P as bf16 into the A-operand buffer;
+//   warp 6      stages the G*D stacked query rows and the block's own K/V rows (plain loads).
+// The G*D <= 32 (or <= 64) query rows that share a KV head are replicated 4 (or 2) times to fill the
+// 128 accumulator lanes; each replica's softmax warps exponentiate a different quarter (half) of a
+// tile's keys but write their piece of P into every replica, so all replicas accumulate the same
+// complete O and the only cross-warp exchange is the row sum at the end of an item.  Every replica
+// computes the row maximum over all 64 keys from identical S values, hence identical decisions.
+// The running maximum is only raised when it grew by more than 2^8 (P then stays <= 256, exact
+// arithmetic either way), which makes rescaling O in tensor memory rare.
 #include "sdlm_internal.h"
 #include "sdlm_ptx.cuh"
 
 namespace sdlm {
-
-constexpr int kAttnStages = 3;
 
 struct AttnParams {
   const __nv_bfloat16* pool;
@@ -25,402 +37,625 @@ struct AttnParams {
   const __nv_bfloat16* k_blk;
   const __nv_bfloat16* v_blk;
   __nv_bfloat16* out;
-  float* part_ml;  // [item][rows][2]  (running max in log2 units, sum)
-  float* part_o;   // [item][rows][d]
+  float* part_ml;  // [slot][row][2]  (reference max in log2 units, sum)
+  float* part_o;   // [slot][row][d]
+  int* pair_cnt;   // [batch * Hkv] arrivals of finished splits; zero between launches
   DevHeader* hdr;
   float scale_log2;  // softmax scale * log2(e)
-  int batch, D, Hq, Hkv, G, mpps, num_pages, target_items;
+  int batch, D, Hq, Hkv, G, mpps, num_pages, n_stages;
 };
 
-struct AttnSched {
-  int chunk;         // pages per item aimed for
-  int total_splits;  // sum over batch rows of their split count
-};
+constexpr int kAttnThreads = 224;
+constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
 __device__ __forceinline__ int attn_slot(const AttnParams& p, int i) { return p.seq_ids ? p.seq_ids[i] : i; }
 __device__ __forceinline__ int attn_len(const AttnParams& p, int i) {
-  int len = p.seq_len[attn_slot(p, i)];
+  const int len = p.seq_len[attn_slot(p, i)];
   return max(0, min(len, p.mpps * kPageSize));
 }
 
-// Fills s_first[0..batch] with the exclusive prefix sum of per-row split counts.  Every CTA of
-// both kernels computes the same list from the same seq_len values.
-__device__ AttnSched attn_schedule(const AttnParams& p, int* s_first) {
-  __shared__ int s_chunk;
-  if (threadIdx.x < 32) {
-    const int lane = threadIdx.x;
-    int tp = 0;
-    for (int i = lane; i < p.batch; i += 32) tp += (attn_len(p, i) + kPageSize - 1) / kPageSize;
-    for (int o = 16; o; o >>= 1) tp += __shfl_xor_sync(0xffffffffu, tp, o);
-    const int chunk = max(1, (tp * p.Hkv + p.target_items - 1) / p.target_items);
+__device__ __forceinline__ void attn_timeout(const AttnParams& p, int where) {
+  if (atomicCAS(&p.hdr->status[0], 0, (int)SDLM_ERR_TIMEOUT) == 0) {
+    p.hdr->status[1] = -1;
+    p.hdr->status[2] = where;
+  }
+}
+
+// One CTA's share of the tile sequence, walked identically by every role.
+struct Item {
+  int b, h, slot, len, pages;
+  int t0, t1;  // tiles [t0, t1) of the pair; tile index `pages` is the block's own tile
+  int pair, c_first, n_splits;
+};
+
+struct ItemWalk {
+  const int* s_first;  // [batch + 1] exclusive prefix sum of (pages + 1) per batch row
+  long long total;     // tiles in the whole launch
+  long long cur, hi;
+  int nc;
+};
+
+__device__ __forceinline__ int tile_owner(long long x, long long total, int nc) {
+  return (int)(((x + 1) * nc - 1) / total);  // the CTA c with floor(c*total/nc) <= x < floor((c+1)*total/nc)
+}
+
+__device__ __forceinline__ void walk_begin(ItemWalk& w, const int* s_first, int batch, int Hkv) {
+  w.s_first = s_first;
+  w.total = (long long)s_first[batch] * Hkv;
+  // never more ranges than tiles: every range is then non-empty and the CTAs that share a pair
+  // are consecutive
+  w.nc = (int)min((long long)gridDim.x, w.total);
+  if ((int)blockIdx.x >= w.nc) {
+    w.cur = w.hi = 0;
+    return;
+  }
+  w.cur = (long long)blockIdx.x * w.total / w.nc;
+  w.hi = (long long)(blockIdx.x + 1) * w.total / w.nc;
+}
+
+__device__ __forceinline__ bool walk_next(ItemWalk& w, const AttnParams& p, Item& it) {
+  if (w.cur >= w.hi) return false;
+  int lo = 0, hi = p.batch - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if ((long long)w.s_first[mid] * p.Hkv <= w.cur) lo = mid; else hi = mid - 1;
+  }
+  it.b = lo;
+  const int tiles_b = w.s_first[lo + 1] - w.s_first[lo];
+  const long long row_start = (long long)w.s_first[lo] * p.Hkv;
+  it.h = (int)((w.cur - row_start) / tiles_b);
+  const long long pair_start = row_start + (long long)it.h * tiles_b;
+  it.t0 = (int)(w.cur - pair_start);
+  const long long end = min(w.hi, pair_start + tiles_b);
+  it.t1 = (int)(end - pair_start);
+  it.pages = tiles_b - 1;
+  it.slot = attn_slot(p, lo);
+  it.len = attn_len(p, lo);
+  it.pair = lo * p.Hkv + it.h;
+  it.c_first = tile_owner(pair_start, w.total, w.nc);
+  it.n_splits = tile_owner(pair_start + tiles_b - 1, w.total, w.nc) - it.c_first + 1;
+  w.cur = end;
+  return true;
+}
+
+// Ring position of the n-th tile this CTA pushes through its stages.
+struct Ring {
+  int stage;
+  uint32_t phase;
+  __device__ __forceinline__ void advance(int n_stages) {
+    if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+  }
+};
+
+__device__ __forceinline__ uint64_t attn_smem_desc(uint32_t saddr) {
+  // K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart; descriptor version 1 (sm_100)
+  return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+
+template <bool FULL>
+__device__ __forceinline__ float row_max16(const uint32_t (&v)[16], int col0, int valid) {
+  float m = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) m = fmaxf(m, (FULL || col0 + i < valid) ? __uint_as_float(v[i]) : -INFINITY);
+  return m;
+}
+
+template <bool FULL>
+__device__ __forceinline__ float row_max64(uint32_t s_addr, int valid) {
+  uint32_t v0[16], v1[16];
+  ptx::tmem_ld16(s_addr, v0);
+  ptx::tmem_ld16(s_addr + 16, v1);
+  ptx::tmem_ld_wait();
+  float m = fmaxf(row_max16<FULL>(v0, 0, valid), row_max16<FULL>(v1, 16, valid));
+  ptx::tmem_ld16(s_addr + 32, v0);
+  ptx::tmem_ld16(s_addr + 48, v1);
+  ptx::tmem_ld_wait();
+  return fmaxf(m, fmaxf(row_max16<FULL>(v0, 32, valid), row_max16<FULL>(v1, 48, valid)));
+}
+
+__device__ __forceinline__ uint4 pack8_bf16(const float* x, float s) {
+  uint4 v;
+  v.x = ptx::pack_bf16(x[0] * s, x[1] * s);
+  v.y = ptx::pack_bf16(x[2] * s, x[3] * s);
+  v.z = ptx::pack_bf16(x[4] * s, x[5] * s);
+  v.w = ptx::pack_bf16(x[6] * s, x[7] * s);
+  return v;
+}
+
+template <int HD, int C>
+__global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const AttnParams p) {
+  constexpr int KH = HD / 64;               // 64-wide panels of a K tile / of Q
+  constexpr int K_TILE_B = kPageSize * HD * 2;
+  constexpr int TILE_B = 2 * K_TILE_B;      // K tile followed by V^T tile, as in the pool
+  constexpr int Q_PANEL_B = 128 * 128;      // 128 rows of 128 bytes
+  constexpr int P_BUF_B = 128 * 128;
+  constexpr int RP = 128 / C;               // rows of one replica
+  constexpr int KS = 64 / C;                // keys of a tile one replica exponentiates
+  constexpr int WPR = 4 / C;                // softmax warps per replica
+  constexpr int NCOL = HD / C;              // output columns one replica writes at the end of an item
+  constexpr uint32_t S_COL = 0, O_COL = 128, TMEM_COLS = 256;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* q_s = smem;
+  uint8_t* p_s = q_s + KH * Q_PANEL_B;
+  uint8_t* stages = p_s + 2 * P_BUF_B;
+  const int NS = p.n_stages;
+  uint64_t* full = reinterpret_cast<uint64_t*>(stages + (size_t)NS * TILE_B);
+  uint64_t* stage_free = full + NS;
+  uint64_t* s_full = stage_free + NS;   // [2]
+  uint64_t* s_free = s_full + 2;        // [2]
+  uint64_t* p_full = s_free + 2;        // [2]
+  uint64_t* p_free = p_full + 2;        // [2]
+  uint64_t* q_full = p_free + 2;
+  uint64_t* q_free = q_full + 1;
+  uint64_t* o_done = q_free + 1;
+  uint64_t* o_free = o_done + 1;
+  uint64_t* ep_bar = o_free + 1;
+  uint64_t* drain = ep_bar + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+  volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* s_last = abort + 1;
+  volatile int* blk_go = abort + 2;  // warp 0 -> warp 6: block-tile ring slots that are free so far
+  float* l_x = reinterpret_cast<float*>(const_cast<int*>(s_last) + 2);  // [2][4][32], by item parity
+  int* s_first = reinterpret_cast<int*>(l_x + 256);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int GD = p.G * p.D;
+
+  // exclusive prefix sum of (pages + 1) per batch row
+  if (warp == 0) {
     int carry = 0;
     for (int base = 0; base < p.batch; base += 32) {
       const int i = base + lane;
-      int sp = 0;
-      if (i < p.batch) sp = max(1, ((attn_len(p, i) + kPageSize - 1) / kPageSize + chunk - 1) / chunk);
-      int incl = sp;
+      const int n = (i < p.batch) ? (attn_len(p, i) + kPageSize - 1) / kPageSize + 1 : 0;
+      int incl = n;
       for (int o = 1; o < 32; o <<= 1) {
         const int v = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += v;
       }
-      if (i < p.batch) s_first[i] = carry + incl - sp;
+      if (i < p.batch) s_first[i] = carry + incl - n;
       carry += __shfl_sync(0xffffffffu, incl, 31);
     }
-    if (lane == 0) {
-      s_first[p.batch] = carry;
-      s_chunk = chunk;
-    }
+    if (lane == 0) s_first[p.batch] = carry;
   }
-  __syncthreads();
-  AttnSched s;
-  s.chunk = s_chunk;
-  s.total_splits = s_first[p.batch];
-  return s;
-}
-
-__device__ __forceinline__ void attn_timeout(const AttnParams& p) {
-  if (atomicCAS(&p.hdr->status[0], 0, (int)SDLM_ERR_TIMEOUT) == 0) p.hdr->status[1] = -1;
-}
-
-template <int HD, int MT, int WPM>
-__global__ void __launch_bounds__(MT* WPM * 32, 2) block_attn_kernel(const AttnParams p) {
-  constexpr int NW = MT * WPM, NTHREADS = NW * 32;
-  constexpr int KW = kPageSize / WPM;  // keys of a tile handled by one warp
-  constexpr int ROWB = HD * 2;         // bytes per token row
-  constexpr int CPR = HD / 8;          // 16-byte chunks per row
-  constexpr int TILE_B = kPageSize * ROWB;
-  constexpr int STAGE_B = 2 * TILE_B;  // K tile followed by V tile, as in the pool
-  constexpr int ROWS = MT * 16;
-  constexpr int MB_LD = HD + 2;        // merge buffer row: d accumulators, max, sum
-  static_assert(NW * 16 * MB_LD * 4 <= kAttnStages * STAGE_B, "merge buffer must fit in the stage ring");
-
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* stages = smem;
-  uint8_t* q_s = smem + kAttnStages * STAGE_B;
-  uint64_t* full = reinterpret_cast<uint64_t*>(q_s + ROWS * ROWB);
-  volatile int* abort = reinterpret_cast<volatile int*>(full + kAttnStages);
-  int* s_first = const_cast<int*>(abort) + 2;
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int mt = warp / WPM, kq = warp % WPM;
-  const int GD = p.G * p.D;
-
-  if (tid == 0) {
-    for (int s = 0; s < kAttnStages; ++s) ptx::mbar_init(&full[s], 1);
+  if (tid == 32) {
+    for (int s = 0; s < NS; ++s) {
+      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&stage_free[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      ptx::mbar_init(&s_full[s], 1);
+      ptx::mbar_init(&s_free[s], 4);
+      ptx::mbar_init(&p_full[s], 4);
+      ptx::mbar_init(&p_free[s], 1);
+    }
+    ptx::mbar_init(q_full, 1);
+    ptx::mbar_init(q_free, 1);
+    ptx::mbar_init(o_done, 1);
+    ptx::mbar_init(o_free, 4);
+    ptx::mbar_init(ep_bar, 4);
+    ptx::mbar_init(drain, 1);
     *abort = 0;
+    *blk_go = 0;
     ptx::fence_barrier_init();
   }
-  const AttnSched sc = attn_schedule(p, s_first);  // contains a __syncthreads
-  const int n_items = sc.total_splits * p.Hkv;
-  const uint32_t q_u32 = ptx::smem_u32(q_s);
-  uint32_t tile_ctr = 0;  // tiles this CTA has pushed through the ring so far
+  __syncthreads();
+  {
+    ItemWalk w0;
+    walk_begin(w0, s_first, p.batch, p.Hkv);
+    if (w0.cur >= w0.hi) return;  // nothing falls into this CTA's range (uniform for the CTA)
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
 
-  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-    const int pair = item / p.Hkv, h = item % p.Hkv;
-    int lo = 0, hi = p.batch - 1;
-    while (lo < hi) {
-      const int mid = (lo + hi + 1) >> 1;
-      if (s_first[mid] <= pair) lo = mid; else hi = mid - 1;
+  if (warp == 0) {
+    // ---------------------------------------------------------------- cached tiles: bulk copies
+    ItemWalk w;
+    walk_begin(w, s_first, p.batch, p.Hkv);
+    Item it;
+    Ring ring{0, 0};
+    uint32_t issued = 0;
+    bool ok = true;
+    while (ok && walk_next(w, p, it)) {
+      const int32_t* ptab = p.page_table + (size_t)it.slot * p.mpps;
+      const int n_cached = min(it.t1, it.pages) - it.t0;
+      for (int base = 0; base < n_cached && ok; base += 32) {
+        int my_page = 0;
+        if (base + lane < n_cached) my_page = ptab[it.t0 + base + lane];  // one latency per 32 tiles
+        const int n = min(32, n_cached - base);
+        for (int j = 0; j < n; ++j) {
+          int page = __shfl_sync(0xffffffffu, my_page, j);
+          if (lane == 0) {
+            if (issued >= (uint32_t)NS && !ptx::mbar_wait(&stage_free[ring.stage], ring.phase ^ 1u, abort)) ok = false;
+            if (ok) {
+              if (page < 0 || page >= p.num_pages) {  // never follow a bad table entry out of the pool
+                if (atomicCAS(&p.hdr->status[0], 0, (int)SDLM_ERR_DEVICE_CHECK) == 0) p.hdr->status[1] = it.slot;
+                page = 0;
+              }
+              const __nv_bfloat16* src = p.pool + kv_tile_offset(page, it.h, 0, p.Hkv, HD);
+              ptx::mbar_arrive_expect_tx(&full[ring.stage], TILE_B);
+              ptx::bulk_g2s(stages + (size_t)ring.stage * TILE_B, src, TILE_B, &full[ring.stage]);
+            }
+          }
+          ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+          if (!ok) break;
+          ring.advance(NS);
+          ++issued;
+        }
+      }
+      if (ok && it.t1 > it.pages) {
+        // The block's own tile is written by warp 6 once its ring slot is free.  This warp does the
+        // waiting, because it reaches the slot in ring order (a parity wait is only meaningful for a
+        // waiter that is at most one phase away from the barrier), and then passes the slot on through
+        // a counter.
+        if (lane == 0) {
+          if (issued >= (uint32_t)NS && !ptx::mbar_wait(&stage_free[ring.stage], ring.phase ^ 1u, abort)) ok = false;
+          if (ok) {
+            __threadfence_block();
+            *blk_go = *blk_go + 1;  // only this thread writes the counter
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+        ring.advance(NS);
+        ++issued;
+      }
     }
-    const int b = lo;
-    const int split = pair - s_first[b], n_splits = s_first[b + 1] - s_first[b];
-    const int slot = attn_slot(p, b);
-    const int len = attn_len(p, b);
-    const int pages = (len + kPageSize - 1) / kPageSize;
-    const int pg0 = (int)((long long)split * pages / n_splits);
-    const int pg1 = (int)((long long)(split + 1) * pages / n_splits);
-    const int n_tiles = pg1 - pg0;
-    const bool last = (split == n_splits - 1);
-    const int32_t* ptab = p.page_table + (size_t)slot * p.mpps;
-
-    auto issue = [&](int t) {  // thread 0 only
-      const uint32_t c = tile_ctr + (uint32_t)t;
-      const int stage = c % kAttnStages;
-      int page = ptab[pg0 + t];
-      if (page < 0 || page >= p.num_pages) {  // never follow a bad table entry out of the pool
-        if (atomicCAS(&p.hdr->status[0], 0, (int)SDLM_ERR_DEVICE_CHECK) == 0) p.hdr->status[1] = slot;
-        page = 0;
+    if (lane == 0 && (!ok || *abort)) {  // winding down: let the copies already issued land
+      attn_timeout(p, 1);
+      Ring r{0, 0};
+      for (uint32_t j = 0; j < issued; ++j) {
+        if (issued - j <= (uint32_t)NS) ptx::mbar_wait_brief(&full[r.stage], r.phase);
+        r.advance(NS);
       }
-      const __nv_bfloat16* src = p.pool + kv_tile_offset(page, h, 0, p.Hkv, HD);
-      ptx::mbar_arrive_expect_tx(&full[stage], STAGE_B);
-      ptx::bulk_g2s(stages + stage * STAGE_B, src, STAGE_B, &full[stage]);
-    };
-
-    if (tid == 0) {
-      ptx::fence_proxy_async();
-      for (int t = 0; t < kAttnStages - 1 && t < n_tiles; ++t) issue(t);
     }
-    // stacked query rows: row r = j*G + g  <->  q[b, j, h*G + g, :]
-    for (int idx = tid; idx < ROWS * CPR; idx += NTHREADS) {
-      const int r = idx / CPR, c = idx % CPR;
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (r < GD) {
-        const int j = r / p.G, g = r % p.G;
-        v = *(reinterpret_cast<const uint4*>(p.q + (((size_t)b * p.D + j) * p.Hq + h * p.G + g) * HD) + c);
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+      const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(HD >> 3) << 17) | ((128u >> 4) << 24);
+      const uint32_t q_addr = ptx::smem_u32(q_s), p_addr = ptx::smem_u32(p_s), st_addr = ptx::smem_u32(stages);
+      ItemWalk w;
+      walk_begin(w, s_first, p.batch, p.Hkv);
+      Item it;
+      Ring ring{0, 0}, pv_ring{0, 0};
+      uint32_t tc = 0, pv_tc = 0, item_idx = 0;
+      bool ok = true;
+      auto issue_pv = [&](bool first_of_item) {
+        const uint32_t pb = pv_tc & 1u;
+        if (!ptx::mbar_wait(&p_full[pb], (pv_tc >> 1) & 1u, abort)) { ok = false; return; }
+        if (first_of_item && item_idx > 0 && !ptx::mbar_wait(o_free, (item_idx - 1) & 1u, abort)) { ok = false; return; }
+        ptx::tc_fence_after();
+        const uint32_t a = p_addr + pb * P_BUF_B, bv = st_addr + (uint32_t)pv_ring.stage * TILE_B + K_TILE_B;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          ptx::umma_bf16_ss(tmem_base + O_COL, attn_smem_desc(a + k * 32), attn_smem_desc(bv + k * 32), idesc_pv,
+                            (first_of_item && k == 0) ? 0u : 1u);
+        ptx::umma_commit(&stage_free[pv_ring.stage]);
+        ptx::umma_commit(&p_free[pb]);
+        pv_ring.advance(NS);
+        ++pv_tc;
+      };
+      while (ok && walk_next(w, p, it)) {
+        if (!ptx::mbar_wait(q_full, item_idx & 1u, abort)) { ok = false; break; }
+        const int n = it.t1 - it.t0;
+        for (int t = 0; t < n && ok; ++t) {
+          const uint32_t sb = tc & 1u;
+          if (!ptx::mbar_wait(&full[ring.stage], ring.phase, abort)) { ok = false; break; }
+          if (tc >= 2 && !ptx::mbar_wait(&s_free[sb], ((tc >> 1) & 1u) ^ 1u, abort)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t bk = st_addr + (uint32_t)ring.stage * TILE_B;
+#pragma unroll
+          for (int kh = 0; kh < KH; ++kh)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              ptx::umma_bf16_ss(tmem_base + S_COL + sb * 64, attn_smem_desc(q_addr + kh * Q_PANEL_B + k * 32),
+                                attn_smem_desc(bk + kh * (K_TILE_B / KH) + k * 32), idesc_qk, (kh | k) ? 1u : 0u);
+          ptx::umma_commit(&s_full[sb]);
+          if (t == n - 1) ptx::umma_commit(q_free);  // every S of this item is computed: Q may be replaced
+          ring.advance(NS);
+          ++tc;
+          if (t > 0) issue_pv(t == 1);
+        }
+        if (ok) issue_pv(n == 1);
+        if (ok) ptx::umma_commit(o_done);
+        ++item_idx;
       }
-      *reinterpret_cast<uint4*>(q_s + r * ROWB + ((c ^ (r & 7)) << 4)) = v;
+      if (!ok) {  // winding down: the MMAs already issued must finish before TMEM and smem are released
+        attn_timeout(p, 2);
+        ptx::umma_commit(drain);
+        ptx::mbar_wait_brief(drain, 0);
+      }
     }
+  } else if (warp < 6) {
+    // ---------------------------------------------------------------- softmax: thread = query row
+    const int qd = warp & 3;                 // TMEM lane quarter of this warp
+    const int rep = qd / WPR;                // replica
+    const int row = (qd % WPR) * 32 + lane;  // stacked query row inside the replica
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(qd * 32) << 16);
+    ItemWalk w;
+    walk_begin(w, s_first, p.batch, p.Hkv);
+    Item it;
+    uint32_t tc = 0, item_idx = 0, ep_uses = 0;
+    bool ok = true;
+    while (ok && walk_next(w, p, it)) {
+      float m_ref = 0.f, l = 0.f;
+      const int n = it.t1 - it.t0;
+      for (int t = 0; t < n; ++t, ++tc) {
+        const uint32_t sb = tc & 1u;
+        const int tile = it.t0 + t;
+        const int valid = tile == it.pages ? p.D : (tile == it.pages - 1 ? it.len - tile * kPageSize : kPageSize);
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(&s_full[sb], (tc >> 1) & 1u, abort))) { ok = false; break; }
+        ptx::tc_fence_after();
+        const uint32_t s_addr = lane_addr + S_COL + sb * 64;
+        // row maximum over all keys of the tile (every replica sees the same values)
+        const float m_raw = valid == kPageSize ? row_max64<true>(s_addr, valid) : row_max64<false>(s_addr, valid);
+        // this replica's keys
+        uint32_t sv[KS];
+#pragma unroll
+        for (int c = 0; c < KS / 16; ++c)
+          ptx::tmem_ld16(s_addr + rep * KS + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&sv[c * 16]));
+        ptx::tmem_ld_wait();
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&s_free[sb]);
 
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-    float o[HD / 8][4];
+        const float m_tile = m_raw * p.scale_log2;
+        if (t == 0) {
+          m_ref = m_tile;
+        } else {
+          const bool need = m_tile > m_ref + kRescaleThreshold;
+          if (__any_sync(0xffffffffu, need)) {
+            // O holds sums relative to the old reference: bring them to the new one.  The previous
+            // P V must have finished writing O first.
+            const uint32_t prev = tc - 1;
+            if (!__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[prev & 1u], (prev >> 1) & 1u, abort))) { ok = false; break; }
+            ptx::tc_fence_after();
+            const float f = need ? ptx::ex2(m_ref - m_tile) : 1.0f;
+            if (need) { m_ref = m_tile; l *= f; }
 #pragma unroll
-    for (int n = 0; n < HD / 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
-
-    auto compute_tile = [&](const uint8_t* stage_ptr, int valid) {
-      if (kq * KW >= valid) return;  // none of this warp's keys exist
-      const uint32_t k_u32 = ptx::smem_u32(stage_ptr), v_u32 = k_u32 + TILE_B;
-      float s[KW / 8][4];
+            for (int c = 0; c < HD / 16; ++c) {
+              uint32_t o[16];
+              ptx::tmem_ld16(lane_addr + O_COL + c * 16, o);
+              ptx::tmem_ld_wait();
 #pragma unroll
-      for (int n = 0; n < KW / 8; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
-#pragma unroll
-      for (int ks = 0; ks < HD / 16; ++ks) {
-        uint32_t a0, a1, a2, a3;
-        {
-          const int row = mt * 16 + (lane & 15), chunk = ks * 2 + (lane >> 4);
-          ptx::ldsm_x4(a0, a1, a2, a3, q_u32 + row * ROWB + ((chunk ^ (row & 7)) << 4));
+              for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+              ptx::tmem_st16(lane_addr + O_COL + c * 16, o);
+            }
+            ptx::tmem_st_wait();
+          }
         }
+        // P = 2^(s*scale - m_ref) for this replica's keys, rounded to bf16
+        uint32_t pk[KS / 2];
+        float lsum = 0.f;
 #pragma unroll
-        for (int np = 0; np < KW / 16; ++np) {
-          const int key = kq * KW + np * 16 + ((lane >> 4) << 3) + (lane & 7), chunk = ks * 2 + ((lane >> 3) & 1);
-          uint32_t b0, b1, b2, b3;
-          ptx::ldsm_x4(b0, b1, b2, b3, k_u32 + key * ROWB + ((chunk ^ (key & 7)) << 4));
-          ptx::mma_bf16_16816(s[2 * np], a0, a1, a2, a3, b0, b1);
-          ptx::mma_bf16_16816(s[2 * np + 1], a0, a1, a2, a3, b2, b3);
+        for (int i = 0; i < KS; i += 2) {
+          const int key = rep * KS + i;
+          float e0 = ptx::ex2(fmaf(__uint_as_float(sv[i]), p.scale_log2, -m_ref));
+          float e1 = ptx::ex2(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -m_ref));
+          if (key >= valid) e0 = 0.f;
+          if (key + 1 >= valid) e1 = 0.f;
+          lsum += e0 + e1;
+          pk[i / 2] = ptx::pack_bf16(e0, e1);
         }
-      }
-      // online softmax, log2 domain; thread holds rows lane/4 (regs 0,1) and lane/4+8 (regs 2,3)
-      float rmax[2] = {-INFINITY, -INFINITY};
+        l += lsum;
+        if (tc >= 2 && !__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[sb], ((tc >> 1) & 1u) ^ 1u, abort))) { ok = false; break; }
+        uint8_t* pb = p_s + sb * P_BUF_B;
 #pragma unroll
-      for (int n = 0; n < KW / 8; ++n)
+        for (int r2 = 0; r2 < C; ++r2) {  // the same piece goes into every replica's rows
+          const int mr = r2 * RP + row;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int key = kq * KW + n * 8 + (lane & 3) * 2 + (e & 1);
-          const float v = (key < valid) ? s[n][e] * p.scale_log2 : -INFINITY;
-          s[n][e] = v;
-          rmax[e >> 1] = fmaxf(rmax[e >> 1], v);
+          for (int c = 0; c < KS / 8; ++c) {
+            const int chunk = rep * (KS / 8) + c;
+            *reinterpret_cast<uint4*>(pb + mr * 128 + ((chunk ^ (mr & 7)) << 4)) =
+                make_uint4(pk[c * 4], pk[c * 4 + 1], pk[c * 4 + 2], pk[c * 4 + 3]);
+          }
         }
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        rmax[r] = fmaxf(rmax[r], __shfl_xor_sync(0xffffffffu, rmax[r], 1));
-        rmax[r] = fmaxf(rmax[r], __shfl_xor_sync(0xffffffffu, rmax[r], 2));
-        const float m_new = fmaxf(m_run[r], rmax[r]);
-        const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-        const float alpha = ptx::ex2(m_run[r] - m_safe);
-        m_run[r] = m_new;
-        float psum = 0.f;
-#pragma unroll
-        for (int n = 0; n < KW / 8; ++n) {
-          const float p0 = ptx::ex2(s[n][2 * r] - m_safe), p1 = ptx::ex2(s[n][2 * r + 1] - m_safe);
-          s[n][2 * r] = p0;
-          s[n][2 * r + 1] = p1;
-          psum += p0 + p1;
-        }
-        l_run[r] = l_run[r] * alpha + psum;
-#pragma unroll
-        for (int n = 0; n < HD / 8; ++n) {
-          o[n][2 * r] *= alpha;
-          o[n][2 * r + 1] *= alpha;
-        }
-      }
-#pragma unroll
-      for (int kk = 0; kk < KW / 16; ++kk) {
-        const uint32_t a0 = ptx::pack_bf16(s[2 * kk][0], s[2 * kk][1]), a1 = ptx::pack_bf16(s[2 * kk][2], s[2 * kk][3]);
-        const uint32_t a2 = ptx::pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]),
-                       a3 = ptx::pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3]);
-#pragma unroll
-        for (int dp = 0; dp < HD / 16; ++dp) {
-          const int key = kq * KW + kk * 16 + (((lane >> 3) & 1) << 3) + (lane & 7), chunk = dp * 2 + (lane >> 4);
-          uint32_t b0, b1, b2, b3;
-          ptx::ldsm_x4_trans(b0, b1, b2, b3, v_u32 + key * ROWB + ((chunk ^ (key & 7)) << 4));
-          ptx::mma_bf16_16816(o[2 * dp], a0, a1, a2, a3, b0, b1);
-          ptx::mma_bf16_16816(o[2 * dp + 1], a0, a1, a2, a3, b2, b3);
-        }
-      }
-    };
-
-    for (int t = 0; t < n_tiles; ++t) {
-      __syncthreads();  // tile t-1 has been consumed by every warp: its stage may be refilled
-      if (tid == 0 && t + kAttnStages - 1 < n_tiles) issue(t + kAttnStages - 1);
-      const uint32_t c = tile_ctr + (uint32_t)t;
-      const int stage = c % kAttnStages;
-      // a wait that runs out is recorded and the tile is processed as it is (the result is then
-      // meaningless but every access stays inside shared memory); later waits return at once
-      if (!ptx::mbar_wait(&full[stage], (c / kAttnStages) & 1, abort) && (tid & 31) == 0) attn_timeout(p);
-      uint8_t* sp = stages + stage * STAGE_B;
-      int valid = kPageSize;
-      if (pg0 + t == pages - 1) valid = len - (pages - 1) * kPageSize;
-      if (valid < kPageSize) {  // rows past the sequence end hold arbitrary bits: clear V there
-        for (int idx = tid; idx < (kPageSize - valid) * CPR; idx += NTHREADS)
-          *reinterpret_cast<uint4*>(sp + TILE_B + (valid + idx / CPR) * ROWB + ((idx % CPR) << 4)) = make_uint4(0, 0, 0, 0);
         ptx::fence_proxy_async();
-        __syncthreads();
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&p_full[sb]);
       }
-      compute_tile(sp, valid);
-    }
-    tile_ctr += (uint32_t)n_tiles;
+      if (!ok) break;
 
-    if (last) {  // the block's own D keys, unmasked among themselves
-      __syncthreads();
-      uint8_t* sp = stages;
-      for (int idx = tid; idx < 2 * kPageSize * CPR; idx += NTHREADS) {
-        const int kv = idx / (kPageSize * CPR), r = (idx / CPR) % kPageSize, c = idx % CPR;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (r < p.D)
-          v = *(reinterpret_cast<const uint4*>((kv ? p.v_blk : p.k_blk) + (((size_t)b * p.D + r) * p.Hkv + h) * HD) + c);
-        *reinterpret_cast<uint4*>(sp + kv * TILE_B + r * ROWB + ((c ^ (r & 7)) << 4)) = v;
-      }
-      __syncthreads();
-      compute_tile(sp, p.D);
-    }
+      // ---- end of item: total row sum across replicas, then output or partial
+      float* lx = l_x + (item_idx & 1u) * 128;
+      lx[qd * 32 + lane] = l;
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ep_bar);
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(ep_bar, ep_uses & 1u, abort))) { ok = false; break; }
+      ++ep_uses;
+      float l_tot = 0.f;
+#pragma unroll
+      for (int r2 = 0; r2 < C; ++r2) l_tot += lx[(r2 * WPR + qd % WPR) * 32 + lane];
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(o_done, item_idx & 1u, abort))) { ok = false; break; }
+      ptx::tc_fence_after();
+      float o[NCOL];
+#pragma unroll
+      for (int c = 0; c < NCOL / 16; ++c)
+        ptx::tmem_ld16(lane_addr + O_COL + rep * NCOL + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&o[c * 16]));
+      ptx::tmem_ld_wait();
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(o_free);
+      ++item_idx;
 
-    // merge the warps that share query rows, then write the item's result
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
-      l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
-    }
-    __syncthreads();  // stage ring is idle from here: reuse it as the merge buffer
-    float* mb = reinterpret_cast<float*>(stages);
-    {
-      float* w = mb + warp * 16 * MB_LD;
-      const int r0 = lane >> 2, cq = (lane & 3) * 2;
-#pragma unroll
-      for (int n = 0; n < HD / 8; ++n) {
-        *reinterpret_cast<float2*>(w + r0 * MB_LD + n * 8 + cq) = make_float2(o[n][0], o[n][1]);
-        *reinterpret_cast<float2*>(w + (r0 + 8) * MB_LD + n * 8 + cq) = make_float2(o[n][2], o[n][3]);
-      }
-      if ((lane & 3) == 0) {
-        w[r0 * MB_LD + HD] = m_run[0];
-        w[r0 * MB_LD + HD + 1] = l_run[0];
-        w[(r0 + 8) * MB_LD + HD] = m_run[1];
-        w[(r0 + 8) * MB_LD + HD + 1] = l_run[1];
-      }
-    }
-    __syncthreads();
-    for (int idx = tid; idx < ROWS * HD; idx += NTHREADS) {
-      const int row = idx / HD, col = idx % HD;
-      const float* w = mb + ((row >> 4) * WPM * 16 + (row & 15)) * MB_LD;
-      float m = -INFINITY;
-#pragma unroll
-      for (int k = 0; k < WPM; ++k) m = fmaxf(m, w[k * 16 * MB_LD + HD]);
-      const float m_safe = (m == -INFINITY) ? 0.f : m;
-      float acc = 0.f, l = 0.f;
-#pragma unroll
-      for (int k = 0; k < WPM; ++k) {
-        const float a = ptx::ex2(w[k * 16 * MB_LD + HD] - m_safe);
-        acc += a * w[k * 16 * MB_LD + col];
-        l += a * w[k * 16 * MB_LD + HD + 1];
-      }
-      if (n_splits == 1) {
+      const int j = row / p.G, g = row % p.G;
+      __nv_bfloat16* out_row = p.out + (((size_t)it.b * p.D + j) * p.Hq + it.h * p.G + g) * HD + rep * NCOL;
+      if (it.n_splits == 1) {
         if (row < GD) {
-          const int j = row / p.G, g = row % p.G;
-          p.out[(((size_t)b * p.D + j) * p.Hq + h * p.G + g) * HD + col] = __float2bfloat16_rn(acc / l);
+          const float inv = 1.0f / l_tot;
+#pragma unroll
+          for (int c = 0; c < NCOL / 8; ++c) reinterpret_cast<uint4*>(out_row)[c] = pack8_bf16(&o[c * 8], inv);
         }
       } else {
-        p.part_o[((size_t)item * ROWS + row) * HD + col] = acc;
-        if (col == 0) {
-          p.part_ml[((size_t)item * ROWS + row) * 2] = m;
-          p.part_ml[((size_t)item * ROWS + row) * 2 + 1] = l;
+        const size_t slot_row = (size_t)(blockIdx.x + it.pair) * RP + row;
+        float* po = p.part_o + slot_row * HD + rep * NCOL;
+#pragma unroll
+        for (int c = 0; c < NCOL / 4; ++c)
+          reinterpret_cast<float4*>(po)[c] = make_float4(o[c * 4], o[c * 4 + 1], o[c * 4 + 2], o[c * 4 + 3]);
+        if (rep == 0) *reinterpret_cast<float2*>(p.part_ml + slot_row * 2) = make_float2(m_ref, l_tot);
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(ep_bar);
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(ep_bar, ep_uses & 1u, abort))) { ok = false; break; }
+        ++ep_uses;
+        if (warp == 2 && lane == 0) {  // every split of the pair counts once; the last one merges
+          const int arrived = atomicAdd(&p.pair_cnt[it.pair], 1);
+          const int last = arrived == it.n_splits - 1;
+          if (last) p.pair_cnt[it.pair] = 0;
+          *s_last = last;
+        }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(ep_bar);
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(ep_bar, ep_uses & 1u, abort))) { ok = false; break; }
+        ++ep_uses;
+        if (*s_last && row < GD) {
+          __threadfence();
+          float m = -INFINITY;
+          for (int s = 0; s < it.n_splits; ++s)
+            m = fmaxf(m, __ldcg(p.part_ml + ((size_t)(it.c_first + s + it.pair) * RP + row) * 2));
+          float acc[NCOL];
+#pragma unroll
+          for (int i = 0; i < NCOL; ++i) acc[i] = 0.f;
+          float lm = 0.f;
+          for (int s = 0; s < it.n_splits; ++s) {  // fixed order: run-to-run identical
+            const size_t sr = (size_t)(it.c_first + s + it.pair) * RP + row;
+            const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + sr * 2));
+            const float a = ptx::ex2(ml.x - m);
+            lm = fmaf(a, ml.y, lm);
+            const float4* src = reinterpret_cast<const float4*>(p.part_o + sr * HD + rep * NCOL);
+#pragma unroll
+            for (int c = 0; c < NCOL / 4; ++c) {
+              const float4 v = __ldcg(src + c);
+              acc[c * 4] = fmaf(a, v.x, acc[c * 4]);
+              acc[c * 4 + 1] = fmaf(a, v.y, acc[c * 4 + 1]);
+              acc[c * 4 + 2] = fmaf(a, v.z, acc[c * 4 + 2]);
+              acc[c * 4 + 3] = fmaf(a, v.w, acc[c * 4 + 3]);
+            }
+          }
+          const float inv = 1.0f / lm;
+#pragma unroll
+          for (int c = 0; c < NCOL / 8; ++c) reinterpret_cast<uint4*>(out_row)[c] = pack8_bf16(&acc[c * 8], inv);
         }
       }
     }
-    ptx::fence_proxy_async();
-    __syncthreads();
-    const int dead = *abort;
-    __syncthreads();  // every thread has read the flag before anyone can set it in the next item
-    if (dead) {  // winding down: let this item's copies land, then stop taking items
-      if (tid == 0)
-        for (uint32_t c = tile_ctr > kAttnStages ? tile_ctr - kAttnStages : 0; c < tile_ctr; ++c)
-          ptx::mbar_wait_brief(&full[c % kAttnStages], (c / kAttnStages) & 1);
-      break;
-    }
-  }
-}
+    if (!ok && lane == 0) attn_timeout(p, 3);
+  } else {
+    // ---------------------------------------------------------------- warp 6: Q rows and the block's own tile
+    ItemWalk w;
+    walk_begin(w, s_first, p.batch, p.Hkv);
+    Item it;
+    Ring ring{0, 0};
+    uint32_t blk_idx = 0, item_idx = 0;
+    bool ok = true;
+    while (ok && walk_next(w, p, it)) {
+      if (item_idx > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait(q_free, (item_idx - 1) & 1u, abort))) { ok = false; break; }
+      // stacked query rows: row r = j*G + g  <->  q[b, j, h*G + g, :]; rows beyond G*D are zero
+      for (int idx = lane; idx < RP * (HD / 8); idx += 32) {
+        const int r = idx / (HD / 8), c = idx % (HD / 8);
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (r < GD) {
+          const int j = r / p.G, g = r % p.G;
+          v = *(reinterpret_cast<const uint4*>(p.q + (((size_t)it.b * p.D + j) * p.Hq + it.h * p.G + g) * HD) + c);
+        }
+#pragma unroll
+        for (int r2 = 0; r2 < C; ++r2) {
+          const int mr = r2 * RP + r;
+          *reinterpret_cast<uint4*>(q_s + (c >> 3) * Q_PANEL_B + mr * 128 + (((c & 7) ^ (mr & 7)) << 4)) = v;
+        }
+      }
+      ptx::fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(q_full);
+      ++item_idx;
 
-// Merges the split partials of one (batch row, KV head): out = sum_s 2^(m_s-m) O_s / sum_s 2^(m_s-m) l_s.
-constexpr int kCombineRows = 8;
-__global__ void __launch_bounds__(256) block_attn_combine_kernel(const AttnParams p, int HD, int ROWS) {
-  extern __shared__ int s_first_c[];
-  attn_schedule(p, s_first_c);
-  const int b = blockIdx.z, h = blockIdx.y;
-  const int first = s_first_c[b], n_splits = s_first_c[b + 1] - first;
-  if (n_splits == 1) return;
-  const int GD = p.G * p.D;
-  const int row0 = blockIdx.x * kCombineRows;
-  for (int idx = threadIdx.x; idx < kCombineRows * HD; idx += blockDim.x) {
-    const int row = row0 + idx / HD, col = idx % HD;
-    if (row >= GD) break;
-    float m = -INFINITY;
-    for (int s = 0; s < n_splits; ++s) m = fmaxf(m, p.part_ml[((size_t)((first + s) * p.Hkv + h) * ROWS + row) * 2]);
-    const float m_safe = (m == -INFINITY) ? 0.f : m;
-    float acc = 0.f, l = 0.f;
-    for (int s = 0; s < n_splits; ++s) {
-      const size_t it = (size_t)((first + s) * p.Hkv + h) * ROWS + row;
-      const float a = ptx::ex2(p.part_ml[it * 2] - m_safe);
-      acc += a * p.part_o[it * HD + col];
-      l += a * p.part_ml[it * 2 + 1];
+      const int n_cached = min(it.t1, it.pages) - it.t0;
+      for (int t = 0; t < n_cached; ++t) ring.advance(NS);
+      if (it.t1 > it.pages) {  // this item ends with the block's own D keys
+        if (!__all_sync(0xffffffffu, ptx::counter_wait(blk_go, (int)blk_idx, abort))) {
+          ok = false;
+          break;
+        }
+        ++blk_idx;
+        uint8_t* k_t = stages + (size_t)ring.stage * TILE_B;
+        uint8_t* v_t = k_t + K_TILE_B;
+        for (int idx = lane; idx < K_TILE_B / 16; idx += 32) {  // keys beyond D: zeros in both tiles
+          reinterpret_cast<uint4*>(k_t)[idx] = make_uint4(0, 0, 0, 0);
+          reinterpret_cast<uint4*>(v_t)[idx] = make_uint4(0, 0, 0, 0);
+        }
+        __syncwarp();
+        for (int idx = lane; idx < p.D * (HD / 8); idx += 32) {
+          const int key = idx / (HD / 8), c = idx % (HD / 8);
+          const size_t src = (((size_t)it.b * p.D + key) * p.Hkv + it.h) * HD;
+          *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(k_t) + k_tile_elem(key, c * 8)) =
+              *(reinterpret_cast<const uint4*>(p.k_blk + src) + c);
+          const uint4 vv = *(reinterpret_cast<const uint4*>(p.v_blk + src) + c);
+          const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(&vv);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) reinterpret_cast<__nv_bfloat16*>(v_t)[vt_tile_elem(key, c * 8 + e)] = ve[e];
+        }
+        ptx::fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&full[ring.stage]);
+        ring.advance(NS);
+      }
     }
-    const int j = row / p.G, g = row % p.G;
-    p.out[(((size_t)b * p.D + j) * p.Hq + h * p.G + g) * HD + col] = __float2bfloat16_rn(acc / l);
+    if (!ok && lane == 0) attn_timeout(p, 4);
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, TMEM_COLS);
   }
 }
 
 // ---------------------------------------------------------------------------------------------
-template <int HD, int MT, int WPM>
-static size_t attn_smem_bytes(int batch) {
-  return 1024 + (size_t)kAttnStages * 2 * kPageSize * HD * 2 + (size_t)MT * 16 * HD * 2 + kAttnStages * 8 + 8 +
-         (size_t)(batch + 1) * 4 + 16;
+constexpr int kAttnSmemLimit = 232448;  // largest dynamic shared memory of one CTA on sm_100
+
+template <int HD>
+static int attn_fixed_smem(int batch) {
+  return 1024 + (HD / 64) * 128 * 128 + 2 * 128 * 128 + 14 * 8 + 16 + 1024 + (batch + 1) * 4 + 64;
 }
 
-template <int HD, int MT, int WPM>
-static cudaError_t attn_setup_one(int max_batch) {
-  return cudaFuncSetAttribute(block_attn_kernel<HD, MT, WPM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)attn_smem_bytes<HD, MT, WPM>(max_batch));
+template <int HD>
+static int attn_stage_count(int batch) {
+  const int tile_b = 2 * kPageSize * HD * 2;
+  int n = (kAttnSmemLimit - attn_fixed_smem<HD>(batch)) / (tile_b + 16);
+  return n > 8 ? 8 : n;
 }
 
-template <int HD, int MT, int WPM>
-static cudaError_t attn_launch_one(sdlm_ctx* ctx, const AttnParams& p, cudaStream_t st) {
-  const size_t smem = attn_smem_bytes<HD, MT, WPM>(p.batch);
-  int per_sm = 0;
-  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, block_attn_kernel<HD, MT, WPM>, MT * WPM * 32, smem);
-  if (e != cudaSuccess) return e;
-  if (per_sm < 1) return cudaErrorLaunchOutOfResources;
-  if (per_sm > 2) per_sm = 2;
-  block_attn_kernel<HD, MT, WPM><<<ctx->sm_count * per_sm, MT * WPM * 32, smem, st>>>(p);
-  ctx->launches++;
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-  dim3 grid((p.G * p.D + kCombineRows - 1) / kCombineRows, p.Hkv, p.batch);
-  block_attn_combine_kernel<<<grid, 256, (size_t)(p.batch + 1) * 4, st>>>(p, HD, MT * 16);
+template <int HD, int C>
+static cudaError_t attn_launch_one(sdlm_ctx* ctx, AttnParams& p, cudaStream_t st) {
+  p.n_stages = attn_stage_count<HD>(p.batch);
+  if (p.n_stages < 2) return cudaErrorLaunchOutOfResources;
+  const size_t smem = (size_t)attn_fixed_smem<HD>(p.batch) + (size_t)p.n_stages * (2 * kPageSize * HD * 2 + 16);
+  const int n_cta = ctx->sm_count < kAttnMaxCtas ? ctx->sm_count : kAttnMaxCtas;
+  block_attn_umma_kernel<HD, C><<<n_cta, kAttnThreads, smem, st>>>(p);
   ctx->launches++;
   return cudaGetLastError();
 }
 
-#define SDLM_ATTN_DISPATCH(FN, ...)                                       \
-  do {                                                                     \
-    if (hd == 128) {                                                       \
-      if (mt == 1) return FN<128, 1, 4>(__VA_ARGS__);                      \
-      if (mt == 2) return FN<128, 2, 2>(__VA_ARGS__);                      \
-      if (mt == 3) return FN<128, 3, 2>(__VA_ARGS__);                      \
-      return FN<128, 4, 2>(__VA_ARGS__);                                   \
-    } else {                                                               \
-      if (mt == 1) return FN<64, 1, 4>(__VA_ARGS__);                       \
-      if (mt == 2) return FN<64, 2, 2>(__VA_ARGS__);                       \
-      if (mt == 3) return FN<64, 3, 2>(__VA_ARGS__);                       \
-      return FN<64, 4, 2>(__VA_ARGS__);                                    \
-    }                                                                      \
-  } while (0)
-
-static cudaError_t attn_setup_mt(int hd, int mt, int max_batch) { SDLM_ATTN_DISPATCH(attn_setup_one, max_batch); }
-
 cudaError_t setup_attn(sdlm_ctx* ctx) {
-  const int max_mt = (ctx->group * ctx->cfg.max_block + 15) / 16;
-  for (int mt = 1; mt <= max_mt; ++mt) {
-    cudaError_t e = attn_setup_mt(ctx->cfg.head_dim, mt, ctx->cfg.max_batch);
-    if (e != cudaSuccess) return e;
+  cudaError_t e = cudaSuccess;
+  if (ctx->cfg.head_dim == 128) {
+    e = cudaFuncSetAttribute(block_attn_umma_kernel<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(block_attn_umma_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
+  } else {
+    e = cudaFuncSetAttribute(block_attn_umma_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(block_attn_umma_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
   }
-  return cudaSuccess;
+  return e;
 }
 
 cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, const void* q,
@@ -437,12 +672,14 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
   p.out = static_cast<__nv_bfloat16*>(out);
   p.part_ml = reinterpret_cast<float*>(ctx->ws + ctx->lay.attn_ml);
   p.part_o = reinterpret_cast<float*>(ctx->ws + ctx->lay.attn_o);
+  p.pair_cnt = reinterpret_cast<int*>(ctx->ws + ctx->lay.attn_cnt);
   p.hdr = ctx->hdr;
   p.scale_log2 = ctx->scale * 1.4426950408889634f;
   p.batch = batch; p.D = D; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.G = ctx->group;
-  p.mpps = c.max_pages_per_seq; p.num_pages = c.num_pages; p.target_items = kAttnTargetItems;
-  const int hd = c.head_dim, mt = (ctx->group * D + 15) / 16;
-  SDLM_ATTN_DISPATCH(attn_launch_one, ctx, p, st);
+  p.mpps = c.max_pages_per_seq; p.num_pages = c.num_pages; p.n_stages = 0;
+  const bool wide = ctx->group * D > 32;  // 2 replicas of up to 64 rows, else 4 replicas of up to 32
+  if (c.head_dim == 128) return wide ? attn_launch_one<128, 2>(ctx, p, st) : attn_launch_one<128, 4>(ctx, p, st);
+  return wide ? attn_launch_one<64, 2>(ctx, p, st) : attn_launch_one<64, 4>(ctx, p, st);
 }
 
 }  // namespace sdlm

@@ -15,7 +15,7 @@ constexpr int kMaxBlock = 8;         // largest D
 constexpr int kMaxQRows = 64;        // (Hq/Hkv) * D stacked query rows per KV head
 constexpr int kMaxBatch = 4096;
 constexpr int kLmMaxStripes = 1024;  // upper bound on vocab stripes (one partial per stripe per row)
-constexpr int kAttnTargetItems = 592;  // split-KV work items aimed for: 4 per SM on 148 SMs
+constexpr int kAttnMaxCtas = 160;    // upper bound on the attention grid (one CTA per SM)
 
 // Sticky status and ring cursors at the start of the workspace; EXPORT/IMPORT copies this header
 // together with the tables that follow it.
@@ -33,10 +33,11 @@ struct WorkspaceLayout {
   size_t hdr, page_table, seq_len, free_list, table_end;  // [hdr, table_end) is the exportable state
   size_t lm_partials;                                      // float4 [kLmMaxStripes][max_rows]
   size_t attn_ml, attn_o;                                  // split-KV partial (m, l) and O
+  size_t attn_cnt;                                         // per (batch row, KV head) arrival counters
   size_t st_q, st_k, st_v, st_hidden, st_out, st_seq_ids, st_token, st_p, st_ent, st_acc, st_out_tokens;
   size_t total;
   int attn_max_items;
-  int q_rows_pad;  // stacked query rows per KV head at max_block, padded to 16
+  int q_rows_pad;  // stacked query rows per KV head at max_block, padded to 32 or 64
 };
 
 bool config_valid(const sdlm_config& c);
@@ -68,15 +69,24 @@ struct sdlm_ctx {
 namespace sdlm {
 
 // ---- paged pool addressing (shared by fill / gather / commit / attention) ------------------
-// Pool layout: [page][kv_head][K|V][64 tokens][d] bf16.  One (page, head, K|V) tile is a
-// contiguous 64*d*2-byte run.  Inside a token row the 16-byte chunks are stored XOR-swizzled by
-// the row index (chunk c of row r sits at chunk c ^ (r & 7)), so that a plain bulk copy of a tile
-// into shared memory is already bank-conflict-free for 8-row matrix loads.
+// Pool layout: [page][kv_head][K tile | V^T tile], each tile 64*d bf16, so one (page, head) pair is
+// one contiguous run that a single bulk copy brings into shared memory.  Both tiles are stored in
+// the layout the tensor cores read directly (rows of 128 bytes, 16-byte chunks XOR-swizzled by the
+// row index within each group of 8 rows):
+//   K tile   : d/64 panels of [64 keys][64 dims]   -- element (key, col) of panel col/64
+//   V^T tile : [d dims][64 keys]                   -- element (col, key): V is stored transposed
+// Invariant kept by every writer: in a page that a page table refers to, the V^T columns of keys
+// at or beyond the sequence end hold zeros (a probability of exactly 0 times that value must be 0).
 __host__ __device__ inline size_t kv_tile_elems(int d) { return (size_t)kPageSize * d; }
 __host__ __device__ inline size_t kv_tile_offset(int page, int head, int kv, int n_kv_heads, int d) {
   return (((size_t)page * n_kv_heads + head) * 2 + kv) * kv_tile_elems(d);
 }
-__host__ __device__ inline int kv_swizzled_chunk(int row, int chunk) { return chunk ^ (row & 7); }
+__host__ __device__ inline int k_tile_elem(int key, int col) {
+  return (col >> 6) * (kPageSize * 64) + key * 64 + ((((col & 63) >> 3) ^ (key & 7)) << 3) + (col & 7);
+}
+__host__ __device__ inline int vt_tile_elem(int key, int col) {
+  return col * kPageSize + (((key >> 3) ^ (col & 7)) << 3) + (key & 7);
+}
 
 // ---- launchers implemented in the kernel translation units ---------------------------------
 cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, const void* q,
