@@ -11,11 +11,14 @@
 // Inside a CTA the work is warp-specialised around the 5th-generation tensor cores:
 //   warp 0      issues one bulk copy per cached tile (K tile + V^T tile, contiguous in the pool and
 //               already in the tensor-core shared-memory layout) into an mbarrier ring;
-//   warp 1      one thread issues tcgen05.mma:  S = Q K^T  (M = 128, N = 64 keys, fp32 in tensor
-//               memory, double-buffered)  and  O += P V  (M = 128, N = d);
+//   warp 1      one thread issues tcgen05.mma  S = Q K^T  (M = 128, N = 64 keys, fp32 in tensor
+//               memory, double-buffered);
+//   warp 7      one thread issues tcgen05.mma  O += P V  (M = 128, N = d), so that the next S never
+//               waits behind a P that is still being computed;
 //   warps 2..5  softmax: thread = one accumulator lane = one query row.  It reads its row of S,
 //               keeps the running max and sum, writes P as bf16 into the A-operand buffer;
-//   warp 6      stages the G*D stacked query rows and the block's own K/V rows (plain loads).
+//   warp 6      stages the G*D stacked query rows (fetched one item ahead into registers) and the
+//               block's own K/V rows (plain loads).
 // The G*D <= 32 (or <= 64) query rows that share a KV head are replicated 4 (or 2) times to fill the
 // 128 accumulator lanes; each replica's softmax warps exponentiate a different quarter (half) of a
 // tile's keys but write their piece of P into every replica, so all replicas accumulate the same
@@ -45,7 +48,7 @@ struct AttnParams {
   int batch, D, Hq, Hkv, G, mpps, num_pages, n_stages;
 };
 
-constexpr int kAttnThreads = 224;
+constexpr int kAttnThreads = 256;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
 __device__ __forceinline__ int attn_slot(const AttnParams& p, int i) { return p.seq_ids ? p.seq_ids[i] : i; }
@@ -134,24 +137,29 @@ __device__ __forceinline__ uint64_t attn_smem_desc(uint32_t saddr) {
 }
 
 template <bool FULL>
-__device__ __forceinline__ float row_max16(const uint32_t (&v)[16], int col0, int valid) {
-  float m = -INFINITY;
+__device__ __forceinline__ float row_max64(const uint32_t (&v)[64], int valid) {
+  float m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-  for (int i = 0; i < 16; ++i) m = fmaxf(m, (FULL || col0 + i < valid) ? __uint_as_float(v[i]) : -INFINITY);
-  return m;
+  for (int i = 0; i < 64; ++i) m[i & 3] = fmaxf(m[i & 3], (FULL || i < valid) ? __uint_as_float(v[i]) : -INFINITY);
+  return fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
 }
 
-template <bool FULL>
-__device__ __forceinline__ float row_max64(uint32_t s_addr, int valid) {
-  uint32_t v0[16], v1[16];
-  ptx::tmem_ld16(s_addr, v0);
-  ptx::tmem_ld16(s_addr + 16, v1);
-  ptx::tmem_ld_wait();
-  float m = fmaxf(row_max16<FULL>(v0, 0, valid), row_max16<FULL>(v1, 16, valid));
-  ptx::tmem_ld16(s_addr + 32, v0);
-  ptx::tmem_ld16(s_addr + 48, v1);
-  ptx::tmem_ld_wait();
-  return fmaxf(m, fmaxf(row_max16<FULL>(v0, 32, valid), row_max16<FULL>(v1, 48, valid)));
+// P = 2^(s*scale - m_ref) for keys OFF .. OFF+KS-1 of the tile, packed to bf16; returns their sum.
+template <int KS, int OFF>
+__device__ __forceinline__ float exp_part(const uint32_t (&v)[64], float scale_log2, float m_ref, int valid,
+                                          uint32_t (&pk)[KS / 2]) {
+  float sum[2] = {0.f, 0.f};
+#pragma unroll
+  for (int i = 0; i < KS; i += 2) {
+    float e0 = ptx::ex2(fmaf(__uint_as_float(v[OFF + i]), scale_log2, -m_ref));
+    float e1 = ptx::ex2(fmaf(__uint_as_float(v[OFF + i + 1]), scale_log2, -m_ref));
+    if (OFF + i >= valid) e0 = 0.f;
+    if (OFF + i + 1 >= valid) e1 = 0.f;
+    sum[0] += e0;
+    sum[1] += e1;
+    pk[i / 2] = ptx::pack_bf16(e0, e1);
+  }
+  return sum[0] + sum[1];
 }
 
 __device__ __forceinline__ uint4 pack8_bf16(const float* x, float s) {
@@ -193,8 +201,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
   uint64_t* o_done = q_free + 1;
   uint64_t* o_free = o_done + 1;
   uint64_t* ep_bar = o_free + 1;
-  uint64_t* drain = ep_bar + 1;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+  uint64_t* drain = ep_bar + 1;         // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 2);
   volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* s_last = abort + 1;
   volatile int* blk_go = abort + 2;  // warp 0 -> warp 6: block-tile ring slots that are free so far
@@ -236,7 +244,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
     ptx::mbar_init(o_done, 1);
     ptx::mbar_init(o_free, 4);
     ptx::mbar_init(ep_bar, 4);
-    ptx::mbar_init(drain, 1);
+    ptx::mbar_init(&drain[0], 1);
+    ptx::mbar_init(&drain[1], 1);
     *abort = 0;
     *blk_go = 0;
     ptx::fence_barrier_init();
@@ -316,37 +325,22 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
         r.advance(NS);
       }
     }
+    __syncwarp();
   } else if (warp == 1) {
-    // ---------------------------------------------------------------- MMA issuer
+    // ---------------------------------------------------------------- S = Q K^T issuer
     if (lane == 0) {
       const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
-      const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(HD >> 3) << 17) | ((128u >> 4) << 24);
-      const uint32_t q_addr = ptx::smem_u32(q_s), p_addr = ptx::smem_u32(p_s), st_addr = ptx::smem_u32(stages);
+      const uint32_t q_addr = ptx::smem_u32(q_s), st_addr = ptx::smem_u32(stages);
       ItemWalk w;
       walk_begin(w, s_first, p.batch, p.Hkv);
       Item it;
-      Ring ring{0, 0}, pv_ring{0, 0};
-      uint32_t tc = 0, pv_tc = 0, item_idx = 0;
+      Ring ring{0, 0};
+      uint32_t tc = 0, item_idx = 0;
       bool ok = true;
-      auto issue_pv = [&](bool first_of_item) {
-        const uint32_t pb = pv_tc & 1u;
-        if (!ptx::mbar_wait(&p_full[pb], (pv_tc >> 1) & 1u, abort)) { ok = false; return; }
-        if (first_of_item && item_idx > 0 && !ptx::mbar_wait(o_free, (item_idx - 1) & 1u, abort)) { ok = false; return; }
-        ptx::tc_fence_after();
-        const uint32_t a = p_addr + pb * P_BUF_B, bv = st_addr + (uint32_t)pv_ring.stage * TILE_B + K_TILE_B;
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          ptx::umma_bf16_ss(tmem_base + O_COL, attn_smem_desc(a + k * 32), attn_smem_desc(bv + k * 32), idesc_pv,
-                            (first_of_item && k == 0) ? 0u : 1u);
-        ptx::umma_commit(&stage_free[pv_ring.stage]);
-        ptx::umma_commit(&p_free[pb]);
-        pv_ring.advance(NS);
-        ++pv_tc;
-      };
       while (ok && walk_next(w, p, it)) {
         if (!ptx::mbar_wait(q_full, item_idx & 1u, abort)) { ok = false; break; }
         const int n = it.t1 - it.t0;
-        for (int t = 0; t < n && ok; ++t) {
+        for (int t = 0; t < n; ++t) {
           const uint32_t sb = tc & 1u;
           if (!ptx::mbar_wait(&full[ring.stage], ring.phase, abort)) { ok = false; break; }
           if (tc >= 2 && !ptx::mbar_wait(&s_free[sb], ((tc >> 1) & 1u) ^ 1u, abort)) { ok = false; break; }
@@ -362,18 +356,57 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
           if (t == n - 1) ptx::umma_commit(q_free);  // every S of this item is computed: Q may be replaced
           ring.advance(NS);
           ++tc;
-          if (t > 0) issue_pv(t == 1);
         }
-        if (ok) issue_pv(n == 1);
-        if (ok) ptx::umma_commit(o_done);
         ++item_idx;
       }
       if (!ok) {  // winding down: the MMAs already issued must finish before TMEM and smem are released
         attn_timeout(p, 2);
-        ptx::umma_commit(drain);
-        ptx::mbar_wait_brief(drain, 0);
+        ptx::umma_commit(&drain[0]);
+        ptx::mbar_wait_brief(&drain[0], 0);
       }
     }
+    __syncwarp();
+  } else if (warp == 7) {
+    // ---------------------------------------------------------------- O += P V issuer
+    if (lane == 0) {
+      const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(HD >> 3) << 17) | ((128u >> 4) << 24);
+      const uint32_t p_addr = ptx::smem_u32(p_s), st_addr = ptx::smem_u32(stages);
+      ItemWalk w;
+      walk_begin(w, s_first, p.batch, p.Hkv);
+      Item it;
+      Ring ring{0, 0};
+      uint32_t tc = 0, item_idx = 0;
+      bool ok = true;
+      while (ok && walk_next(w, p, it)) {
+        const int n = it.t1 - it.t0;
+        for (int t = 0; t < n; ++t) {
+          const uint32_t pb = tc & 1u;
+          if (!ptx::mbar_wait(&p_full[pb], (tc >> 1) & 1u, abort)) { ok = false; break; }
+          // the first P V of an item overwrites O: the previous item's O must have been read out
+          if (t == 0 && item_idx > 0 && !ptx::mbar_wait(o_free, (item_idx - 1) & 1u, abort)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t a = p_addr + pb * P_BUF_B, bv = st_addr + (uint32_t)ring.stage * TILE_B + K_TILE_B;
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            ptx::umma_bf16_ss(tmem_base + O_COL, attn_smem_desc(a + k * 32), attn_smem_desc(bv + k * 32), idesc_pv,
+                              (t == 0 && k == 0) ? 0u : 1u);
+          // P is only written after S of the same tile was read, so K of this stage is done as well
+          ptx::umma_commit(&stage_free[ring.stage]);
+          ptx::umma_commit(&p_free[pb]);
+          ring.advance(NS);
+          ++tc;
+        }
+        if (!ok) break;
+        ptx::umma_commit(o_done);
+        ++item_idx;
+      }
+      if (!ok) {
+        attn_timeout(p, 5);
+        ptx::umma_commit(&drain[1]);
+        ptx::mbar_wait_brief(&drain[1], 0);
+      }
+    }
+    __syncwarp();
   } else if (warp < 6) {
     // ---------------------------------------------------------------- softmax: thread = query row
     const int qd = warp & 3;                 // TMEM lane quarter of this warp
@@ -394,18 +427,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
         const int valid = tile == it.pages ? p.D : (tile == it.pages - 1 ? it.len - tile * kPageSize : kPageSize);
         if (!__all_sync(0xffffffffu, ptx::mbar_wait(&s_full[sb], (tc >> 1) & 1u, abort))) { ok = false; break; }
         ptx::tc_fence_after();
-        const uint32_t s_addr = lane_addr + S_COL + sb * 64;
-        // row maximum over all keys of the tile (every replica sees the same values)
-        const float m_raw = valid == kPageSize ? row_max64<true>(s_addr, valid) : row_max64<false>(s_addr, valid);
-        // this replica's keys
-        uint32_t sv[KS];
-#pragma unroll
-        for (int c = 0; c < KS / 16; ++c)
-          ptx::tmem_ld16(s_addr + rep * KS + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&sv[c * 16]));
+        // the whole row of S in one load; every replica sees the same values
+        uint32_t sv[64];
+        ptx::tmem_ld64(lane_addr + S_COL + sb * 64, sv);
         ptx::tmem_ld_wait();
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&s_free[sb]);
+        const float m_raw = valid == kPageSize ? row_max64<true>(sv, valid) : row_max64<false>(sv, valid);
 
         const float m_tile = m_raw * p.scale_log2;
         if (t == 0) {
@@ -434,17 +463,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
         }
         // P = 2^(s*scale - m_ref) for this replica's keys, rounded to bf16
         uint32_t pk[KS / 2];
-        float lsum = 0.f;
-#pragma unroll
-        for (int i = 0; i < KS; i += 2) {
-          const int key = rep * KS + i;
-          float e0 = ptx::ex2(fmaf(__uint_as_float(sv[i]), p.scale_log2, -m_ref));
-          float e1 = ptx::ex2(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -m_ref));
-          if (key >= valid) e0 = 0.f;
-          if (key + 1 >= valid) e1 = 0.f;
-          lsum += e0 + e1;
-          pk[i / 2] = ptx::pack_bf16(e0, e1);
-        }
+        float lsum;
+        if (rep == 0) lsum = exp_part<KS, 0>(sv, p.scale_log2, m_ref, valid, pk);
+        else if (rep == 1) lsum = exp_part<KS, KS>(sv, p.scale_log2, m_ref, valid, pk);
+        else if (rep == 2) lsum = exp_part<KS, (2 * KS) & 63>(sv, p.scale_log2, m_ref, valid, pk);
+        else lsum = exp_part<KS, (3 * KS) & 63>(sv, p.scale_log2, m_ref, valid, pk);
         l += lsum;
         if (tc >= 2 && !__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[sb], ((tc >> 1) & 1u) ^ 1u, abort))) { ok = false; break; }
         uint8_t* pb = p_s + sb * P_BUF_B;
@@ -520,12 +543,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
         if (*s_last && row < GD) {
           __threadfence();
           float m = -INFINITY;
+#pragma unroll 4
           for (int s = 0; s < it.n_splits; ++s)
             m = fmaxf(m, __ldcg(p.part_ml + ((size_t)(it.c_first + s + it.pair) * RP + row) * 2));
           float acc[NCOL];
 #pragma unroll
           for (int i = 0; i < NCOL; ++i) acc[i] = 0.f;
           float lm = 0.f;
+#pragma unroll 2
           for (int s = 0; s < it.n_splits; ++s) {  // fixed order: run-to-run identical
             const size_t sr = (size_t)(it.c_first + s + it.pair) * RP + row;
             const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + sr * 2));
@@ -550,26 +575,37 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
     if (!ok && lane == 0) attn_timeout(p, 3);
   } else {
     // ---------------------------------------------------------------- warp 6: Q rows and the block's own tile
+    constexpr int NQ = RP * (HD / 8) / 32;  // 16-byte chunks of the stacked query rows per lane
     ItemWalk w;
     walk_begin(w, s_first, p.batch, p.Hkv);
-    Item it;
+    Item it, nxt;
     Ring ring{0, 0};
     uint32_t blk_idx = 0, item_idx = 0;
     bool ok = true;
-    while (ok && walk_next(w, p, it)) {
-      if (item_idx > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait(q_free, (item_idx - 1) & 1u, abort))) { ok = false; break; }
-      // stacked query rows: row r = j*G + g  <->  q[b, j, h*G + g, :]; rows beyond G*D are zero
-      for (int idx = lane; idx < RP * (HD / 8); idx += 32) {
-        const int r = idx / (HD / 8), c = idx % (HD / 8);
-        uint4 v = make_uint4(0, 0, 0, 0);
+    uint4 qreg[NQ];
+    // stacked query rows: row r = j*G + g  <->  q[b, j, h*G + g, :]; rows beyond G*D are zero
+    auto fetch_q = [&](const Item& x) {
+#pragma unroll
+      for (int i = 0; i < NQ; ++i) {
+        const int idx = i * 32 + lane, r = idx / (HD / 8), c = idx % (HD / 8);
+        qreg[i] = make_uint4(0, 0, 0, 0);
         if (r < GD) {
           const int j = r / p.G, g = r % p.G;
-          v = *(reinterpret_cast<const uint4*>(p.q + (((size_t)it.b * p.D + j) * p.Hq + it.h * p.G + g) * HD) + c);
+          qreg[i] = __ldg(reinterpret_cast<const uint4*>(p.q + (((size_t)x.b * p.D + j) * p.Hq + x.h * p.G + g) * HD) + c);
         }
+      }
+    };
+    bool have = walk_next(w, p, it);
+    if (have) fetch_q(it);
+    while (ok && have) {
+      if (item_idx > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait(q_free, (item_idx - 1) & 1u, abort))) { ok = false; break; }
+#pragma unroll
+      for (int i = 0; i < NQ; ++i) {
+        const int idx = i * 32 + lane, r = idx / (HD / 8), c = idx % (HD / 8);
 #pragma unroll
         for (int r2 = 0; r2 < C; ++r2) {
           const int mr = r2 * RP + r;
-          *reinterpret_cast<uint4*>(q_s + (c >> 3) * Q_PANEL_B + mr * 128 + (((c & 7) ^ (mr & 7)) << 4)) = v;
+          *reinterpret_cast<uint4*>(q_s + (c >> 3) * Q_PANEL_B + mr * 128 + (((c & 7) ^ (mr & 7)) << 4)) = qreg[i];
         }
       }
       ptx::fence_proxy_async();
@@ -577,9 +613,25 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
       if (lane == 0) ptx::mbar_arrive(q_full);
       ++item_idx;
 
+      // the next item's query rows travel while this item is being processed
+      have = walk_next(w, p, nxt);
+      if (have) fetch_q(nxt);
+
       const int n_cached = min(it.t1, it.pages) - it.t0;
       for (int t = 0; t < n_cached; ++t) ring.advance(NS);
       if (it.t1 > it.pages) {  // this item ends with the block's own D keys
+        constexpr int NB = kMaxBlock * (HD / 8) / 32;  // chunks of the block's K (and V) rows per lane
+        uint4 kreg[NB], vreg[NB];
+#pragma unroll
+        for (int i = 0; i < NB; ++i) {
+          const int idx = i * 32 + lane, key = idx / (HD / 8), c = idx % (HD / 8);
+          kreg[i] = vreg[i] = make_uint4(0, 0, 0, 0);
+          if (key < p.D) {
+            const size_t src = (((size_t)it.b * p.D + key) * p.Hkv + it.h) * HD;
+            kreg[i] = __ldg(reinterpret_cast<const uint4*>(p.k_blk + src) + c);
+            vreg[i] = __ldg(reinterpret_cast<const uint4*>(p.v_blk + src) + c);
+          }
+        }
         if (!__all_sync(0xffffffffu, ptx::counter_wait(blk_go, (int)blk_idx, abort))) {
           ok = false;
           break;
@@ -587,26 +639,26 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
         ++blk_idx;
         uint8_t* k_t = stages + (size_t)ring.stage * TILE_B;
         uint8_t* v_t = k_t + K_TILE_B;
-        for (int idx = lane; idx < K_TILE_B / 16; idx += 32) {  // keys beyond D: zeros in both tiles
-          reinterpret_cast<uint4*>(k_t)[idx] = make_uint4(0, 0, 0, 0);
-          reinterpret_cast<uint4*>(v_t)[idx] = make_uint4(0, 0, 0, 0);
-        }
+        // V^T columns of keys beyond D must be zeros (0 * stale bits could be NaN); K rows beyond D
+        // only produce scores that are masked
+        for (int idx = lane; idx < K_TILE_B / 16; idx += 32) reinterpret_cast<uint4*>(v_t)[idx] = make_uint4(0, 0, 0, 0);
         __syncwarp();
-        for (int idx = lane; idx < p.D * (HD / 8); idx += 32) {
-          const int key = idx / (HD / 8), c = idx % (HD / 8);
-          const size_t src = (((size_t)it.b * p.D + key) * p.Hkv + it.h) * HD;
-          *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(k_t) + k_tile_elem(key, c * 8)) =
-              *(reinterpret_cast<const uint4*>(p.k_blk + src) + c);
-          const uint4 vv = *(reinterpret_cast<const uint4*>(p.v_blk + src) + c);
-          const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(&vv);
 #pragma unroll
-          for (int e = 0; e < 8; ++e) reinterpret_cast<__nv_bfloat16*>(v_t)[vt_tile_elem(key, c * 8 + e)] = ve[e];
+        for (int i = 0; i < NB; ++i) {
+          const int idx = i * 32 + lane, key = idx / (HD / 8), c = idx % (HD / 8);
+          if (key < p.D) {
+            *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(k_t) + k_tile_elem(key, c * 8)) = kreg[i];
+            const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(&vreg[i]);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) reinterpret_cast<__nv_bfloat16*>(v_t)[vt_tile_elem(key, c * 8 + e)] = ve[e];
+          }
         }
         ptx::fence_proxy_async();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&full[ring.stage]);
         ring.advance(NS);
       }
+      it = nxt;
     }
     if (!ok && lane == 0) attn_timeout(p, 4);
   }
@@ -623,7 +675,7 @@ constexpr int kAttnSmemLimit = 232448;  // largest dynamic shared memory of one 
 
 template <int HD>
 static int attn_fixed_smem(int batch) {
-  return 1024 + (HD / 64) * 128 * 128 + 2 * 128 * 128 + 14 * 8 + 16 + 1024 + (batch + 1) * 4 + 64;
+  return 1024 + (HD / 64) * 128 * 128 + 2 * 128 * 128 + 15 * 8 + 16 + 1024 + (batch + 1) * 4 + 64;
 }
 
 template <int HD>

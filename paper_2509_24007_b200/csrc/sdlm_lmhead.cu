@@ -200,6 +200,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
         for (uint32_t j = first; j < it; ++j) ptx::mbar_wait_brief(&full[j % n_stages], (j / n_stages) & 1);
       }
     }
+    __syncwarp();  // the warp arrives at the closing barrier as a whole
   } else if (warp == 1) {
     if (lane == 0) {  // ---- MMA issuer
       // instruction descriptor: D fp32, A and B bf16, both K-major, N = bn, M = 128
@@ -241,6 +242,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
         ptx::mbar_wait_brief(drain, 0);
       }
     }
+    __syncwarp();
   } else {  // ---- epilogue: TMEM lane = hidden-state row
     const int q = warp & 3;  // TMEM lane quarter this warp may touch
     Stat st[R];
