@@ -5,27 +5,27 @@
 // one per (sequence, KV head) for the D block tokens -- form one sequence that is cut into equal
 // contiguous ranges, one per CTA, so every SM streams the same number of bytes.  The part of a
 // (sequence, KV head) pair that falls into one CTA's range is an "item"; a pair cut by a range
-// boundary leaves partial (max, sum, O) results, which the last of its CTAs to finish merges
+// boundary leaves partial (reference, sum, O) results, which the last of its CTAs to finish merges
 // (arrival counter per pair; nobody waits).
 //
-// Inside a CTA the work is warp-specialised around the 5th-generation tensor cores:
-//   warp 0      issues one bulk copy per cached tile (K tile + V^T tile, contiguous in the pool and
-//               already in the tensor-core shared-memory layout) into an mbarrier ring;
-//   warp 1      one thread issues tcgen05.mma  S = Q K^T  (M = 128, N = 64 keys, fp32 in tensor
-//               memory, double-buffered);
-//   warp 7      one thread issues tcgen05.mma  O += P V  (M = 128, N = d), so that the next S never
-//               waits behind a P that is still being computed;
-//   warps 2..5  softmax: thread = one accumulator lane = one query row.  It reads its row of S,
-//               keeps the running max and sum, writes P as bf16 into the A-operand buffer;
-//   warp 6      stages the G*D stacked query rows (fetched one item ahead into registers) and the
-//               block's own K/V rows (plain loads).
-// The G*D <= 32 (or <= 64) query rows that share a KV head are replicated 4 (or 2) times to fill the
-// 128 accumulator lanes; each replica's softmax warps exponentiate a different quarter (half) of a
-// tile's keys but write their piece of P into every replica, so all replicas accumulate the same
-// complete O and the only cross-warp exchange is the row sum at the end of an item.  Every replica
-// computes the row maximum over all 64 keys from identical S values, hence identical decisions.
-// The running maximum is only raised when it grew by more than 2^8 (P then stays <= 256, exact
-// arithmetic either way), which makes rescaling O in tensor memory rare.
+// Inside a CTA the tiles of an item are taken two at a time (a "group" of up to 128 keys) and the
+// two contractions run on the 5th-generation tensor cores with the KEYS, not the few query rows,
+// on the 128 accumulator lanes:
+//     S^T = K Q^T      M = 128 keys,  N = the G*D stacked query rows (padded to 32 or 64), K = d
+//     O^T += V^T P^T   M = d,         N = query rows,                                     K = keys
+// so no lane computes padding and the operands re-read per instruction are small.  Roles:
+//   warp 0      bulk copies of cached tiles (K panels and V^T tile, stored in the pool in the
+//               tensor-core shared-memory layout) into a ring of two-tile buffers;
+//   warp 1      one thread issues the S^T instructions (S^T double-buffered in tensor memory);
+//   warp 7      one thread issues the O^T instructions;
+//   warps 2..5  softmax: thread = accumulator lane = one key; it holds that key's score for every
+//               query row, exponentiates against a per-row reference kept in shared memory, adds to
+//               its private row sums and writes its column of P^T (bf16) into the B-operand buffer;
+//   warp 6      stages the stacked query rows (fetched one item ahead) and the block's own K/V rows.
+// The reference of a row is not the running maximum: it is only moved (and O^T, sums rescaled)
+// when some score exceeds it by more than 2^32, which the softmax warps agree on once per group;
+// the first group of an item always sets it to that group's exact row maxima.  Probabilities are
+// therefore exact up to rounding, and rescaling O^T in tensor memory is rare.
 #include "sdlm_internal.h"
 #include "sdlm_ptx.cuh"
 
@@ -49,7 +49,7 @@ struct AttnParams {
 };
 
 constexpr int kAttnThreads = 256;
-constexpr float kRescaleThreshold = 8.0f;  // log2 units
+constexpr float kRebaseThreshold = 32.0f;  // log2 units a score may exceed its row reference by
 
 __device__ __forceinline__ int attn_slot(const AttnParams& p, int i) { return p.seq_ids ? p.seq_ids[i] : i; }
 __device__ __forceinline__ int attn_len(const AttnParams& p, int i) {
@@ -136,53 +136,34 @@ __device__ __forceinline__ uint64_t attn_smem_desc(uint32_t saddr) {
          ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
 
-template <bool FULL>
-__device__ __forceinline__ float row_max64(const uint32_t (&v)[64], int valid) {
-  float m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-  for (int i = 0; i < 64; ++i) m[i & 3] = fmaxf(m[i & 3], (FULL || i < valid) ? __uint_as_float(v[i]) : -INFINITY);
-  return fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
+
+constexpr int kIntMin = -2147483647 - 1;
+// Order-preserving map float -> int (for integer warp reductions of float maxima) and back.
+__device__ __forceinline__ int ordered_int(float f) {
+  const int i = __float_as_int(f);
+  return i >= 0 ? i : i ^ 0x7fffffff;
+}
+__device__ __forceinline__ float ordered_float(int i) { return __int_as_float(i >= 0 ? i : i ^ 0x7fffffff); }
+
+// Keys of tile `ti` of an item that exist (0 when the item has no such tile).
+__device__ __forceinline__ int tile_valid(const Item& it, int ti, int D) {
+  if (ti >= it.t1) return 0;
+  if (ti == it.pages) return D;
+  return ti == it.pages - 1 ? it.len - ti * kPageSize : kPageSize;
 }
 
-// P = 2^(s*scale - m_ref) for keys OFF .. OFF+KS-1 of the tile, packed to bf16; returns their sum.
-template <int KS, int OFF>
-__device__ __forceinline__ float exp_part(const uint32_t (&v)[64], float scale_log2, float m_ref, int valid,
-                                          uint32_t (&pk)[KS / 2]) {
-  float sum[2] = {0.f, 0.f};
-#pragma unroll
-  for (int i = 0; i < KS; i += 2) {
-    float e0 = ptx::ex2(fmaf(__uint_as_float(v[OFF + i]), scale_log2, -m_ref));
-    float e1 = ptx::ex2(fmaf(__uint_as_float(v[OFF + i + 1]), scale_log2, -m_ref));
-    if (OFF + i >= valid) e0 = 0.f;
-    if (OFF + i + 1 >= valid) e1 = 0.f;
-    sum[0] += e0;
-    sum[1] += e1;
-    pk[i / 2] = ptx::pack_bf16(e0, e1);
-  }
-  return sum[0] + sum[1];
-}
-
-__device__ __forceinline__ uint4 pack8_bf16(const float* x, float s) {
-  uint4 v;
-  v.x = ptx::pack_bf16(x[0] * s, x[1] * s);
-  v.y = ptx::pack_bf16(x[2] * s, x[3] * s);
-  v.z = ptx::pack_bf16(x[4] * s, x[5] * s);
-  v.w = ptx::pack_bf16(x[6] * s, x[7] * s);
-  return v;
-}
-
-template <int HD, int C>
+template <int HD, int NQ>
 __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const AttnParams p) {
-  constexpr int KH = HD / 64;               // 64-wide panels of a K tile / of Q
-  constexpr int K_TILE_B = kPageSize * HD * 2;
-  constexpr int TILE_B = 2 * K_TILE_B;      // K tile followed by V^T tile, as in the pool
-  constexpr int Q_PANEL_B = 128 * 128;      // 128 rows of 128 bytes
-  constexpr int P_BUF_B = 128 * 128;
-  constexpr int RP = 128 / C;               // rows of one replica
-  constexpr int KS = 64 / C;                // keys of a tile one replica exponentiates
-  constexpr int WPR = 4 / C;                // softmax warps per replica
-  constexpr int NCOL = HD / C;              // output columns one replica writes at the end of an item
-  constexpr uint32_t S_COL = 0, O_COL = 128, TMEM_COLS = 256;
+  constexpr int KH = HD / 64;                 // 64-wide panels of K and of Q
+  constexpr int K_PANEL_B = kPageSize * 128;  // one tile's panel: 64 keys x 128 bytes
+  constexpr int VT_B = HD * 128;              // one tile's V^T: d rows x 128 bytes
+  constexpr int TILE_B = KH * K_PANEL_B + VT_B;
+  constexpr int K_REGION_B = KH * 2 * K_PANEL_B;  // per panel: tile 0's rows, then tile 1's rows
+  constexpr int PAIR_B = K_REGION_B + 2 * VT_B;
+  constexpr int Q_PANEL_B = NQ * 128;
+  constexpr int P_PANEL_B = NQ * 128;             // P^T of one tile: NQ rows x 64 keys
+  constexpr int P_BUF_B = 2 * P_PANEL_B;
+  constexpr uint32_t O_COL = 128, TMEM_COLS = 256;  // S^T buffers at columns 0 and NQ
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -190,7 +171,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
   uint8_t* p_s = q_s + KH * Q_PANEL_B;
   uint8_t* stages = p_s + 2 * P_BUF_B;
   const int NS = p.n_stages;
-  uint64_t* full = reinterpret_cast<uint64_t*>(stages + (size_t)NS * TILE_B);
+  uint64_t* full = reinterpret_cast<uint64_t*>(stages + (size_t)NS * PAIR_B);
   uint64_t* stage_free = full + NS;
   uint64_t* s_full = stage_free + NS;   // [2]
   uint64_t* s_free = s_full + 2;        // [2]
@@ -202,12 +183,17 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
   uint64_t* o_free = o_done + 1;
   uint64_t* ep_bar = o_free + 1;
   uint64_t* drain = ep_bar + 1;         // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 2);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 3);  // one spare slot keeps the floats below 16-byte aligned
   volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* s_last = abort + 1;
-  volatile int* blk_go = abort + 2;  // warp 0 -> warp 6: block-tile ring slots that are free so far
-  float* l_x = reinterpret_cast<float*>(const_cast<int*>(s_last) + 2);  // [2][4][32], by item parity
-  int* s_first = reinterpret_cast<int*>(l_x + 256);
+  volatile int* blk_go = abort + 2;     // warp 0 -> warp 6: block-tile ring slots that are free so far
+  volatile int* flag = abort + 3;       // [3] "some score outgrew its reference", by group mod 3
+  float* mref = reinterpret_cast<float*>(const_cast<int*>(abort) + 7);  // [64] row references (log2 units); 16-byte aligned
+  float* mnew = mref + 64;              // [64]
+  float* fbuf = mnew + 64;              // [64] rescale factors of a reference move
+  int* mx = reinterpret_cast<int*>(fbuf + 64);                          // [4][64] per-warp row maxima
+  float* lsum = reinterpret_cast<float*>(mx + 256);                     // [2][4][64] per-warp row sums, by item parity
+  int* s_first = reinterpret_cast<int*>(lsum + 512);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int GD = p.G * p.D;
@@ -230,7 +216,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
   }
   if (tid == 32) {
     for (int s = 0; s < NS; ++s) {
-      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&full[s], 2);  // the copies' issuer, plus whoever completes the group (see warp 0)
       ptx::mbar_init(&stage_free[s], 1);
     }
     for (int s = 0; s < 2; ++s) {
@@ -248,6 +234,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
     ptx::mbar_init(&drain[1], 1);
     *abort = 0;
     *blk_go = 0;
+    flag[0] = flag[1] = flag[2] = 0;
     ptx::fence_barrier_init();
   }
   __syncthreads();
@@ -271,48 +258,49 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
     walk_begin(w, s_first, p.batch, p.Hkv);
     Item it;
     Ring ring{0, 0};
-    uint32_t issued = 0;
+    uint32_t issued = 0;  // groups so far
     bool ok = true;
     while (ok && walk_next(w, p, it)) {
       const int32_t* ptab = p.page_table + (size_t)it.slot * p.mpps;
-      const int n_cached = min(it.t1, it.pages) - it.t0;
-      for (int base = 0; base < n_cached && ok; base += 32) {
-        int my_page = 0;
-        if (base + lane < n_cached) my_page = ptab[it.t0 + base + lane];  // one latency per 32 tiles
-        const int n = min(32, n_cached - base);
-        for (int j = 0; j < n; ++j) {
-          int page = __shfl_sync(0xffffffffu, my_page, j);
-          if (lane == 0) {
-            if (issued >= (uint32_t)NS && !ptx::mbar_wait(&stage_free[ring.stage], ring.phase ^ 1u, abort)) ok = false;
-            if (ok) {
+      const int n = it.t1 - it.t0, n_cached = min(it.t1, it.pages) - it.t0;
+      int my_page = 0;
+      for (int g = 0; 2 * g < n && ok; ++g) {
+        if ((2 * g) % 32 == 0 && 2 * g + lane < n_cached) my_page = ptab[it.t0 + 2 * g + lane];  // one latency per 32 tiles
+        int page0 = __shfl_sync(0xffffffffu, my_page, (2 * g) & 31);
+        int page1 = __shfl_sync(0xffffffffu, my_page, (2 * g + 1) & 31);
+        if (lane == 0) {
+          if (issued >= (uint32_t)NS && !ptx::mbar_wait(&stage_free[ring.stage], ring.phase ^ 1u, abort)) ok = false;
+          if (ok) {
+            const int cached = max(0, min(2, n_cached - 2 * g));   // cached tiles of this group
+            const bool has_blk = n > n_cached && (n - 1) / 2 == g;  // the block's own tile is in it
+            uint8_t* st = stages + (size_t)ring.stage * PAIR_B;
+            if (cached > 0) ptx::mbar_arrive_expect_tx(&full[ring.stage], (uint32_t)(cached * TILE_B));
+            else ptx::mbar_arrive(&full[ring.stage]);
+            for (int j = 0; j < cached; ++j) {
+              int page = j ? page1 : page0;
               if (page < 0 || page >= p.num_pages) {  // never follow a bad table entry out of the pool
                 if (atomicCAS(&p.hdr->status[0], 0, (int)SDLM_ERR_DEVICE_CHECK) == 0) p.hdr->status[1] = it.slot;
                 page = 0;
               }
-              const __nv_bfloat16* src = p.pool + kv_tile_offset(page, it.h, 0, p.Hkv, HD);
-              ptx::mbar_arrive_expect_tx(&full[ring.stage], TILE_B);
-              ptx::bulk_g2s(stages + (size_t)ring.stage * TILE_B, src, TILE_B, &full[ring.stage]);
+              const uint8_t* src = reinterpret_cast<const uint8_t*>(p.pool + kv_tile_offset(page, it.h, 0, p.Hkv, HD));
+#pragma unroll
+              for (int kh = 0; kh < KH; ++kh)
+                ptx::bulk_g2s(st + kh * 2 * K_PANEL_B + j * K_PANEL_B, src + kh * K_PANEL_B, K_PANEL_B, &full[ring.stage]);
+              ptx::bulk_g2s(st + K_REGION_B + j * VT_B, src + KH * K_PANEL_B, VT_B, &full[ring.stage]);
             }
-          }
-          ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-          if (!ok) break;
-          ring.advance(NS);
-          ++issued;
-        }
-      }
-      if (ok && it.t1 > it.pages) {
-        // The block's own tile is written by warp 6 once its ring slot is free.  This warp does the
-        // waiting, because it reaches the slot in ring order (a parity wait is only meaningful for a
-        // waiter that is at most one phase away from the barrier), and then passes the slot on through
-        // a counter.
-        if (lane == 0) {
-          if (issued >= (uint32_t)NS && !ptx::mbar_wait(&stage_free[ring.stage], ring.phase ^ 1u, abort)) ok = false;
-          if (ok) {
-            __threadfence_block();
-            *blk_go = *blk_go + 1;  // only this thread writes the counter
+            if (has_blk) {
+              // The block's own tile is written by warp 6, which then gives the group's second
+              // arrival.  This warp does the waiting for the ring slot, because it reaches the slot
+              // in ring order, and passes it on through a counter.
+              __threadfence_block();
+              *blk_go = *blk_go + 1;  // only this thread writes the counter
+            } else {
+              ptx::mbar_arrive(&full[ring.stage]);
+            }
           }
         }
         ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+        if (!ok) break;
         ring.advance(NS);
         ++issued;
       }
@@ -327,35 +315,35 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ---------------------------------------------------------------- S = Q K^T issuer
+    // ---------------------------------------------------------------- S^T = K Q^T issuer
     if (lane == 0) {
-      const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NQ >> 3) << 17) | ((128u >> 4) << 24);
       const uint32_t q_addr = ptx::smem_u32(q_s), st_addr = ptx::smem_u32(stages);
       ItemWalk w;
       walk_begin(w, s_first, p.batch, p.Hkv);
       Item it;
       Ring ring{0, 0};
-      uint32_t tc = 0, item_idx = 0;
+      uint32_t gc = 0, item_idx = 0;
       bool ok = true;
       while (ok && walk_next(w, p, it)) {
         if (!ptx::mbar_wait(q_full, item_idx & 1u, abort)) { ok = false; break; }
-        const int n = it.t1 - it.t0;
-        for (int t = 0; t < n; ++t) {
-          const uint32_t sb = tc & 1u;
+        const int ng = (it.t1 - it.t0 + 1) / 2;
+        for (int g = 0; g < ng; ++g) {
+          const uint32_t sb = gc & 1u;
           if (!ptx::mbar_wait(&full[ring.stage], ring.phase, abort)) { ok = false; break; }
-          if (tc >= 2 && !ptx::mbar_wait(&s_free[sb], ((tc >> 1) & 1u) ^ 1u, abort)) { ok = false; break; }
+          if (gc >= 2 && !ptx::mbar_wait(&s_free[sb], ((gc >> 1) & 1u) ^ 1u, abort)) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint32_t bk = st_addr + (uint32_t)ring.stage * TILE_B;
+          const uint32_t bk = st_addr + (uint32_t)ring.stage * PAIR_B;
 #pragma unroll
           for (int kh = 0; kh < KH; ++kh)
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-              ptx::umma_bf16_ss(tmem_base + S_COL + sb * 64, attn_smem_desc(q_addr + kh * Q_PANEL_B + k * 32),
-                                attn_smem_desc(bk + kh * (K_TILE_B / KH) + k * 32), idesc_qk, (kh | k) ? 1u : 0u);
+              ptx::umma_bf16_ss(tmem_base + sb * NQ, attn_smem_desc(bk + kh * 2 * K_PANEL_B + k * 32),
+                                attn_smem_desc(q_addr + kh * Q_PANEL_B + k * 32), idesc, (kh | k) ? 1u : 0u);
           ptx::umma_commit(&s_full[sb]);
-          if (t == n - 1) ptx::umma_commit(q_free);  // every S of this item is computed: Q may be replaced
+          if (g == ng - 1) ptx::umma_commit(q_free);  // every S^T of this item is computed: Q may be replaced
           ring.advance(NS);
-          ++tc;
+          ++gc;
         }
         ++item_idx;
       }
@@ -367,34 +355,36 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
     }
     __syncwarp();
   } else if (warp == 7) {
-    // ---------------------------------------------------------------- O += P V issuer
+    // ---------------------------------------------------------------- O^T += V^T P^T issuer
     if (lane == 0) {
-      const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(HD >> 3) << 17) | ((128u >> 4) << 24);
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NQ >> 3) << 17) | ((128u >> 4) << 24);
       const uint32_t p_addr = ptx::smem_u32(p_s), st_addr = ptx::smem_u32(stages);
       ItemWalk w;
       walk_begin(w, s_first, p.batch, p.Hkv);
       Item it;
       Ring ring{0, 0};
-      uint32_t tc = 0, item_idx = 0;
+      uint32_t gc = 0, item_idx = 0;
       bool ok = true;
       while (ok && walk_next(w, p, it)) {
-        const int n = it.t1 - it.t0;
-        for (int t = 0; t < n; ++t) {
-          const uint32_t pb = tc & 1u;
-          if (!ptx::mbar_wait(&p_full[pb], (tc >> 1) & 1u, abort)) { ok = false; break; }
-          // the first P V of an item overwrites O: the previous item's O must have been read out
-          if (t == 0 && item_idx > 0 && !ptx::mbar_wait(o_free, (item_idx - 1) & 1u, abort)) { ok = false; break; }
+        const int n = it.t1 - it.t0, ng = (n + 1) / 2;
+        for (int g = 0; g < ng; ++g) {
+          const uint32_t pb = gc & 1u;
+          if (!ptx::mbar_wait(&p_full[pb], (gc >> 1) & 1u, abort)) { ok = false; break; }
+          // the first instruction of an item overwrites O^T: the previous item's must have been read out
+          if (g == 0 && item_idx > 0 && !ptx::mbar_wait(o_free, (item_idx - 1) & 1u, abort)) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint32_t a = p_addr + pb * P_BUF_B, bv = st_addr + (uint32_t)ring.stage * TILE_B + K_TILE_B;
+          const int tiles = min(2, n - 2 * g);
+          const uint32_t av = st_addr + (uint32_t)ring.stage * PAIR_B + K_REGION_B, bp = p_addr + pb * P_BUF_B;
+          for (int j = 0; j < tiles; ++j)
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            ptx::umma_bf16_ss(tmem_base + O_COL, attn_smem_desc(a + k * 32), attn_smem_desc(bv + k * 32), idesc_pv,
-                              (t == 0 && k == 0) ? 0u : 1u);
-          // P is only written after S of the same tile was read, so K of this stage is done as well
+            for (int k = 0; k < 4; ++k)
+              ptx::umma_bf16_ss(tmem_base + O_COL, attn_smem_desc(av + j * VT_B + k * 32),
+                                attn_smem_desc(bp + j * P_PANEL_B + k * 32), idesc, (g == 0 && j == 0 && k == 0) ? 0u : 1u);
+          // P^T is only written after S^T of the same group was read, so K of this stage is done as well
           ptx::umma_commit(&stage_free[ring.stage]);
           ptx::umma_commit(&p_free[pb]);
           ring.advance(NS);
-          ++tc;
+          ++gc;
         }
         if (!ok) break;
         ptx::umma_commit(o_done);
@@ -408,79 +398,121 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
     }
     __syncwarp();
   } else if (warp < 6) {
-    // ---------------------------------------------------------------- softmax: thread = query row
-    const int qd = warp & 3;                 // TMEM lane quarter of this warp
-    const int rep = qd / WPR;                // replica
-    const int row = (qd % WPR) * 32 + lane;  // stacked query row inside the replica
+    // ---------------------------------------------------------------- softmax: thread = key of the group
+    const int qd = warp & 3;             // TMEM lane quarter of this warp
+    const int kg = qd * 32 + lane;       // key within the group = accumulator lane; also the d index at the end
+    const int tj = kg >> 6, kt = kg & 63;  // tile of the group, key within that tile
     const uint32_t lane_addr = tmem_base + ((uint32_t)(qd * 32) << 16);
     ItemWalk w;
     walk_begin(w, s_first, p.batch, p.Hkv);
     Item it;
-    uint32_t tc = 0, item_idx = 0, ep_uses = 0;
+    uint32_t gc = 0, item_idx = 0, ep_uses = 0;
     bool ok = true;
+    // all four softmax warps meet; false when a wait ran out
+    auto meet = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ep_bar);
+      const bool r = __all_sync(0xffffffffu, ptx::mbar_wait(ep_bar, ep_uses & 1u, abort));
+      ++ep_uses;
+      return r;
+    };
     while (ok && walk_next(w, p, it)) {
-      float m_ref = 0.f, l = 0.f;
-      const int n = it.t1 - it.t0;
-      for (int t = 0; t < n; ++t, ++tc) {
-        const uint32_t sb = tc & 1u;
-        const int tile = it.t0 + t;
-        const int valid = tile == it.pages ? p.D : (tile == it.pages - 1 ? it.len - tile * kPageSize : kPageSize);
-        if (!__all_sync(0xffffffffu, ptx::mbar_wait(&s_full[sb], (tc >> 1) & 1u, abort))) { ok = false; break; }
+      float l[NQ];  // this key subset's share of every row sum
+#pragma unroll
+      for (int q = 0; q < NQ; ++q) l[q] = 0.f;
+      const int n = it.t1 - it.t0, ng = (n + 1) / 2;
+      for (int g = 0; g < ng; ++g, ++gc) {
+        const uint32_t sb = gc & 1u;
+        const bool mine = kt < tile_valid(it, it.t0 + 2 * g + tj, p.D);  // does my key exist?
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(&s_full[sb], (gc >> 1) & 1u, abort))) { ok = false; break; }
         ptx::tc_fence_after();
-        // the whole row of S in one load; every replica sees the same values
-        uint32_t sv[64];
-        ptx::tmem_ld64(lane_addr + S_COL + sb * 64, sv);
+        float x[NQ];  // my key's score for every row, then its exponent relative to the row reference
+#pragma unroll
+        for (int c = 0; c < NQ / 16; ++c)
+          ptx::tmem_ld16(lane_addr + sb * NQ + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&x[c * 16]));
         ptx::tmem_ld_wait();
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&s_free[sb]);
-        const float m_raw = valid == kPageSize ? row_max64<true>(sv, valid) : row_max64<false>(sv, valid);
 
-        const float m_tile = m_raw * p.scale_log2;
-        if (t == 0) {
-          m_ref = m_tile;
-        } else {
-          const bool need = m_tile > m_ref + kRescaleThreshold;
-          if (__any_sync(0xffffffffu, need)) {
-            // O holds sums relative to the old reference: bring them to the new one.  The previous
-            // P V must have finished writing O first.
-            const uint32_t prev = tc - 1;
+        const bool first = g == 0;
+        bool moved = first;  // the first group of an item always sets the references
+        const uint32_t fi = gc % 3u;
+        if (warp == 2 && lane == 0) flag[(fi + 1u) % 3u] = 0;  // last read two groups ago
+        float e[NQ];  // exponents of my key relative to the row references
+        if (!first) {
+          float xm = -INFINITY;
+#pragma unroll
+          for (int q4 = 0; q4 < NQ; q4 += 4) {
+            const float4 mr = *reinterpret_cast<const float4*>(mref + q4);
+            e[q4] = fmaf(x[q4], p.scale_log2, -mr.x);
+            e[q4 + 1] = fmaf(x[q4 + 1], p.scale_log2, -mr.y);
+            e[q4 + 2] = fmaf(x[q4 + 2], p.scale_log2, -mr.z);
+            e[q4 + 3] = fmaf(x[q4 + 3], p.scale_log2, -mr.w);
+            xm = fmaxf(fmaxf(xm, fmaxf(e[q4], e[q4 + 1])), fmaxf(e[q4 + 2], e[q4 + 3]));
+          }
+          const bool need = mine && xm > kRebaseThreshold;
+          if (__any_sync(0xffffffffu, need) && lane == 0) flag[fi] = 1;
+          if (!meet()) { ok = false; break; }
+          moved = flag[fi] != 0;
+        }
+        if (moved) {
+          // ---- move the row references to max(old reference, this group's row maxima)
+#pragma unroll
+          for (int q = 0; q < NQ; ++q) {
+            const int v = __reduce_max_sync(0xffffffffu, mine ? ordered_int(x[q] * p.scale_log2) : kIntMin);
+            if (lane == (q & 31)) mx[qd * 64 + q] = v;
+          }
+          if (!meet()) { ok = false; break; }
+#pragma unroll
+          for (int q = 0; q < NQ; ++q) {
+            const int gi = max(max(mx[q], mx[64 + q]), max(mx[128 + q], mx[192 + q]));
+            const float m_old = first ? -INFINITY : mref[q];
+            float m_new = gi == kIntMin ? m_old : fmaxf(m_old, ordered_float(gi));
+            if (m_new == -INFINITY) m_new = 0.f;  // no key at all (cannot happen: every group has one)
+            const float f = first ? 0.f : ptx::ex2(m_old - m_new);
+            l[q] *= f;
+            if (kg == q) { mnew[q] = m_new; fbuf[q] = f; }
+          }
+          if (!meet()) { ok = false; break; }  // everybody has read the old references
+          if (kg < NQ) mref[kg] = mnew[kg];
+          if (!first) {
+            // O^T holds sums relative to the old references; the previous O^T instruction must be done
+            const uint32_t prev = gc - 1;
             if (!__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[prev & 1u], (prev >> 1) & 1u, abort))) { ok = false; break; }
             ptx::tc_fence_after();
-            const float f = need ? ptx::ex2(m_ref - m_tile) : 1.0f;
-            if (need) { m_ref = m_tile; l *= f; }
 #pragma unroll
-            for (int c = 0; c < HD / 16; ++c) {
+            for (int c = 0; c < NQ / 16; ++c) {
               uint32_t o[16];
               ptx::tmem_ld16(lane_addr + O_COL + c * 16, o);
               ptx::tmem_ld_wait();
 #pragma unroll
-              for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+              for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * fbuf[c * 16 + i]);
               ptx::tmem_st16(lane_addr + O_COL + c * 16, o);
             }
             ptx::tmem_st_wait();
           }
-        }
-        // P = 2^(s*scale - m_ref) for this replica's keys, rounded to bf16
-        uint32_t pk[KS / 2];
-        float lsum;
-        if (rep == 0) lsum = exp_part<KS, 0>(sv, p.scale_log2, m_ref, valid, pk);
-        else if (rep == 1) lsum = exp_part<KS, KS>(sv, p.scale_log2, m_ref, valid, pk);
-        else if (rep == 2) lsum = exp_part<KS, (2 * KS) & 63>(sv, p.scale_log2, m_ref, valid, pk);
-        else lsum = exp_part<KS, (3 * KS) & 63>(sv, p.scale_log2, m_ref, valid, pk);
-        l += lsum;
-        if (tc >= 2 && !__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[sb], ((tc >> 1) & 1u) ^ 1u, abort))) { ok = false; break; }
-        uint8_t* pb = p_s + sb * P_BUF_B;
+          if (!meet()) { ok = false; break; }  // the new references are visible
 #pragma unroll
-        for (int r2 = 0; r2 < C; ++r2) {  // the same piece goes into every replica's rows
-          const int mr = r2 * RP + row;
-#pragma unroll
-          for (int c = 0; c < KS / 8; ++c) {
-            const int chunk = rep * (KS / 8) + c;
-            *reinterpret_cast<uint4*>(pb + mr * 128 + ((chunk ^ (mr & 7)) << 4)) =
-                make_uint4(pk[c * 4], pk[c * 4 + 1], pk[c * 4 + 2], pk[c * 4 + 3]);
+          for (int q4 = 0; q4 < NQ; q4 += 4) {
+            const float4 mr = *reinterpret_cast<const float4*>(mref + q4);
+            e[q4] = fmaf(x[q4], p.scale_log2, -mr.x);
+            e[q4 + 1] = fmaf(x[q4 + 1], p.scale_log2, -mr.y);
+            e[q4 + 2] = fmaf(x[q4 + 2], p.scale_log2, -mr.z);
+            e[q4 + 3] = fmaf(x[q4 + 3], p.scale_log2, -mr.w);
           }
         }
+        // P^T column of my key: 2^(s*scale - reference), rounded to bf16; absent keys give 0
+        if (gc >= 2 && !__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[sb], ((gc >> 1) & 1u) ^ 1u, abort))) { ok = false; break; }
+        uint8_t* pcol = p_s + sb * P_BUF_B + tj * P_PANEL_B + (kt & 7) * 2;
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+          e[q] = mine ? ptx::ex2(e[q]) : 0.f;
+          l[q] += e[q];
+        }
+#pragma unroll
+        for (int q = 0; q < NQ; ++q)
+          *reinterpret_cast<__nv_bfloat16*>(pcol + q * 128 + (((kt >> 3) ^ (q & 7)) << 4)) = __float2bfloat16_rn(e[q]);
         ptx::fence_proxy_async();
         ptx::tc_fence_before();
         __syncwarp();
@@ -488,105 +520,153 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
       }
       if (!ok) break;
 
-      // ---- end of item: total row sum across replicas, then output or partial
-      float* lx = l_x + (item_idx & 1u) * 128;
-      lx[qd * 32 + lane] = l;
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(ep_bar);
-      if (!__all_sync(0xffffffffu, ptx::mbar_wait(ep_bar, ep_uses & 1u, abort))) { ok = false; break; }
-      ++ep_uses;
-      float l_tot = 0.f;
+      // ---- end of item: row sums over all keys (lane q of each warp ends up with the warp's sum of row q)
+      float* ls = lsum + (item_idx & 1u) * 256;
 #pragma unroll
-      for (int r2 = 0; r2 < C; ++r2) l_tot += lx[(r2 * WPR + qd % WPR) * 32 + lane];
+      for (int half = 0; half < NQ / 32; ++half) {
+        float* v = &l[half * 32];
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+#pragma unroll
+          for (int i = 0; i < off; ++i) {
+            const bool up = (lane & off) != 0;
+            const float send = up ? v[i] : v[i + off], keep = up ? v[i + off] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+          }
+        }
+        ls[qd * 64 + half * 32 + lane] = v[0];
+      }
+      if (!meet()) { ok = false; break; }
       if (!__all_sync(0xffffffffu, ptx::mbar_wait(o_done, item_idx & 1u, abort))) { ok = false; break; }
       ptx::tc_fence_after();
-      float o[NCOL];
+      float o[NQ];  // O^T row d = kg: one value per query row
 #pragma unroll
-      for (int c = 0; c < NCOL / 16; ++c)
-        ptx::tmem_ld16(lane_addr + O_COL + rep * NCOL + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&o[c * 16]));
+      for (int c = 0; c < NQ / 16; ++c)
+        ptx::tmem_ld16(lane_addr + O_COL + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&o[c * 16]));
       ptx::tmem_ld_wait();
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(o_free);
       ++item_idx;
 
-      const int j = row / p.G, g = row % p.G;
-      __nv_bfloat16* out_row = p.out + (((size_t)it.b * p.D + j) * p.Hq + it.h * p.G + g) * HD + rep * NCOL;
+      const int d = kg;
+      // row q = j*G + g  <->  out[b, j, h*G + g, :]
+      __nv_bfloat16* out_base = p.out + ((size_t)it.b * p.D * p.Hq + it.h * p.G) * HD + d;
       if (it.n_splits == 1) {
-        if (row < GD) {
-          const float inv = 1.0f / l_tot;
+        if (d < HD) {
 #pragma unroll
-          for (int c = 0; c < NCOL / 8; ++c) reinterpret_cast<uint4*>(out_row)[c] = pack8_bf16(&o[c * 8], inv);
+          for (int q = 0; q < NQ; ++q) {
+            if (q < GD) {
+              const float lt = ls[q] + ls[64 + q] + ls[128 + q] + ls[192 + q];
+              out_base[((size_t)(q / p.G) * p.Hq + q % p.G) * HD] = __float2bfloat16_rn(o[q] / lt);
+            }
+          }
         }
       } else {
-        const size_t slot_row = (size_t)(blockIdx.x + it.pair) * RP + row;
-        float* po = p.part_o + slot_row * HD + rep * NCOL;
+        const size_t slot_row = (size_t)(blockIdx.x + it.pair) * NQ;
+        if (d < HD) {
 #pragma unroll
-        for (int c = 0; c < NCOL / 4; ++c)
-          reinterpret_cast<float4*>(po)[c] = make_float4(o[c * 4], o[c * 4 + 1], o[c * 4 + 2], o[c * 4 + 3]);
-        if (rep == 0) *reinterpret_cast<float2*>(p.part_ml + slot_row * 2) = make_float2(m_ref, l_tot);
+          for (int q = 0; q < NQ; ++q) p.part_o[(slot_row + q) * HD + d] = o[q];
+        }
+        if (kg < NQ)
+          *reinterpret_cast<float2*>(p.part_ml + (slot_row + kg) * 2) =
+              make_float2(mref[kg], ls[kg] + ls[64 + kg] + ls[128 + kg] + ls[192 + kg]);
         __threadfence();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(ep_bar);
-        if (!__all_sync(0xffffffffu, ptx::mbar_wait(ep_bar, ep_uses & 1u, abort))) { ok = false; break; }
-        ++ep_uses;
+        if (!meet()) { ok = false; break; }
         if (warp == 2 && lane == 0) {  // every split of the pair counts once; the last one merges
           const int arrived = atomicAdd(&p.pair_cnt[it.pair], 1);
           const int last = arrived == it.n_splits - 1;
           if (last) p.pair_cnt[it.pair] = 0;
           *s_last = last;
         }
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(ep_bar);
-        if (!__all_sync(0xffffffffu, ptx::mbar_wait(ep_bar, ep_uses & 1u, abort))) { ok = false; break; }
-        ++ep_uses;
-        if (*s_last && row < GD) {
+        if (!meet()) { ok = false; break; }
+        if (*s_last) {
+          // ---- merge the splits of this pair (fixed order: run-to-run identical).  Row q's weight of
+          // split s is 2^(m_s - m) / L with m = max_s m_s, L = sum_s 2^(m_s - m) l_s; the weights go
+          // through the (now idle) P^T buffers, then every thread sums four output columns.
           __threadfence();
-          float m = -INFINITY;
-#pragma unroll 4
-          for (int s = 0; s < it.n_splits; ++s)
-            m = fmaxf(m, __ldcg(p.part_ml + ((size_t)(it.c_first + s + it.pair) * RP + row) * 2));
-          float acc[NCOL];
+          constexpr int kCap = 128;  // splits whose weights fit into the P^T buffers at once
+          float* wbuf = reinterpret_cast<float*>(p_s);
+          const size_t first_row = (size_t)(it.c_first + it.pair) * NQ;
+          if (kg < GD) {
+            float m = -INFINITY;
+#pragma unroll 8
+            for (int s = 0; s < it.n_splits; ++s) m = fmaxf(m, __ldcg(p.part_ml + (first_row + (size_t)s * NQ + kg) * 2));
+            float L = 0.f;
+#pragma unroll 8
+            for (int s = 0; s < it.n_splits; ++s) {
+              const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (first_row + (size_t)s * NQ + kg) * 2));
+              L = fmaf(ptx::ex2(ml.x - m), ml.y, L);
+            }
+            mnew[kg] = m;
+            fbuf[kg] = 1.0f / L;
+          }
+          const int dq = tid & 31, qg = (tid >> 5) & 3;  // four columns 4*dq.. of the rows q = qg mod 4
+          float acc[NQ / 4][4];
 #pragma unroll
-          for (int i = 0; i < NCOL; ++i) acc[i] = 0.f;
-          float lm = 0.f;
+          for (int i = 0; i < NQ / 4; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
+          for (int c0 = 0; c0 < it.n_splits && ok; c0 += kCap) {
+            const int cn = min(kCap, it.n_splits - c0);
+            if (!meet()) { ok = false; break; }  // mnew / fbuf written; wbuf no longer read
+            if (kg < GD) {
+              const float m = mnew[kg], inv = fbuf[kg];
+#pragma unroll 8
+              for (int s = 0; s < cn; ++s)
+                wbuf[s * NQ + kg] = ptx::ex2(__ldcg(p.part_ml + (first_row + (size_t)(c0 + s) * NQ + kg) * 2) - m) * inv;
+            }
+            if (!meet()) { ok = false; break; }
+            if (4 * dq < HD) {
 #pragma unroll 2
-          for (int s = 0; s < it.n_splits; ++s) {  // fixed order: run-to-run identical
-            const size_t sr = (size_t)(it.c_first + s + it.pair) * RP + row;
-            const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + sr * 2));
-            const float a = ptx::ex2(ml.x - m);
-            lm = fmaf(a, ml.y, lm);
-            const float4* src = reinterpret_cast<const float4*>(p.part_o + sr * HD + rep * NCOL);
+              for (int s = 0; s < cn; ++s) {
+                const float* src = p.part_o + (first_row + (size_t)(c0 + s) * NQ) * HD + 4 * dq;
 #pragma unroll
-            for (int c = 0; c < NCOL / 4; ++c) {
-              const float4 v = __ldcg(src + c);
-              acc[c * 4] = fmaf(a, v.x, acc[c * 4]);
-              acc[c * 4 + 1] = fmaf(a, v.y, acc[c * 4 + 1]);
-              acc[c * 4 + 2] = fmaf(a, v.z, acc[c * 4 + 2]);
-              acc[c * 4 + 3] = fmaf(a, v.w, acc[c * 4 + 3]);
+                for (int i = 0; i < NQ / 4; ++i) {
+                  const int q = qg + 4 * i;
+                  if (q < GD) {
+                    const float wq = wbuf[s * NQ + q];
+                    const float4 v = __ldcg(reinterpret_cast<const float4*>(src + (size_t)q * HD));
+                    acc[i][0] = fmaf(wq, v.x, acc[i][0]);
+                    acc[i][1] = fmaf(wq, v.y, acc[i][1]);
+                    acc[i][2] = fmaf(wq, v.z, acc[i][2]);
+                    acc[i][3] = fmaf(wq, v.w, acc[i][3]);
+                  }
+                }
+              }
             }
           }
-          const float inv = 1.0f / lm;
+          if (!ok) break;
+          if (4 * dq < HD) {
+            __nv_bfloat16* ob = p.out + ((size_t)it.b * p.D * p.Hq + it.h * p.G) * HD + 4 * dq;
 #pragma unroll
-          for (int c = 0; c < NCOL / 8; ++c) reinterpret_cast<uint4*>(out_row)[c] = pack8_bf16(&acc[c * 8], inv);
+            for (int i = 0; i < NQ / 4; ++i) {
+              const int q = qg + 4 * i;
+              if (q < GD) {
+                uint2 v;
+                v.x = ptx::pack_bf16(acc[i][0], acc[i][1]);
+                v.y = ptx::pack_bf16(acc[i][2], acc[i][3]);
+                *reinterpret_cast<uint2*>(ob + ((size_t)(q / p.G) * p.Hq + q % p.G) * HD) = v;
+              }
+            }
+          }
+          if (!meet()) { ok = false; break; }  // the P^T buffers go back to the softmax
         }
       }
     }
     if (!ok && lane == 0) attn_timeout(p, 3);
   } else {
     // ---------------------------------------------------------------- warp 6: Q rows and the block's own tile
-    constexpr int NQ = RP * (HD / 8) / 32;  // 16-byte chunks of the stacked query rows per lane
+    constexpr int NQC = NQ * (HD / 8) / 32;  // 16-byte chunks of the stacked query rows per lane
     ItemWalk w;
     walk_begin(w, s_first, p.batch, p.Hkv);
     Item it, nxt;
     Ring ring{0, 0};
     uint32_t blk_idx = 0, item_idx = 0;
     bool ok = true;
-    uint4 qreg[NQ];
+    uint4 qreg[NQC];
     // stacked query rows: row r = j*G + g  <->  q[b, j, h*G + g, :]; rows beyond G*D are zero
     auto fetch_q = [&](const Item& x) {
 #pragma unroll
-      for (int i = 0; i < NQ; ++i) {
+      for (int i = 0; i < NQC; ++i) {
         const int idx = i * 32 + lane, r = idx / (HD / 8), c = idx % (HD / 8);
         qreg[i] = make_uint4(0, 0, 0, 0);
         if (r < GD) {
@@ -600,13 +680,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
     while (ok && have) {
       if (item_idx > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait(q_free, (item_idx - 1) & 1u, abort))) { ok = false; break; }
 #pragma unroll
-      for (int i = 0; i < NQ; ++i) {
+      for (int i = 0; i < NQC; ++i) {
         const int idx = i * 32 + lane, r = idx / (HD / 8), c = idx % (HD / 8);
-#pragma unroll
-        for (int r2 = 0; r2 < C; ++r2) {
-          const int mr = r2 * RP + r;
-          *reinterpret_cast<uint4*>(q_s + (c >> 3) * Q_PANEL_B + mr * 128 + (((c & 7) ^ (mr & 7)) << 4)) = qreg[i];
-        }
+        *reinterpret_cast<uint4*>(q_s + (c >> 3) * Q_PANEL_B + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = qreg[i];
       }
       ptx::fence_proxy_async();
       __syncwarp();
@@ -617,9 +693,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
       have = walk_next(w, p, nxt);
       if (have) fetch_q(nxt);
 
-      const int n_cached = min(it.t1, it.pages) - it.t0;
-      for (int t = 0; t < n_cached; ++t) ring.advance(NS);
-      if (it.t1 > it.pages) {  // this item ends with the block's own D keys
+      const int n = it.t1 - it.t0, ng = (n + 1) / 2;
+      for (int g = 0; g + 1 < ng; ++g) ring.advance(NS);
+      if (it.t1 > it.pages) {  // the item's last group holds the block's own D keys
         constexpr int NB = kMaxBlock * (HD / 8) / 32;  // chunks of the block's K (and V) rows per lane
         uint4 kreg[NB], vreg[NB];
 #pragma unroll
@@ -637,17 +713,18 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
           break;
         }
         ++blk_idx;
-        uint8_t* k_t = stages + (size_t)ring.stage * TILE_B;
-        uint8_t* v_t = k_t + K_TILE_B;
+        const int tj = (n - 1) & 1;  // the block's tile is the group's first or second
+        uint8_t* st = stages + (size_t)ring.stage * PAIR_B;
+        uint8_t* v_t = st + K_REGION_B + tj * VT_B;
         // V^T columns of keys beyond D must be zeros (0 * stale bits could be NaN); K rows beyond D
         // only produce scores that are masked
-        for (int idx = lane; idx < K_TILE_B / 16; idx += 32) reinterpret_cast<uint4*>(v_t)[idx] = make_uint4(0, 0, 0, 0);
+        for (int idx = lane; idx < VT_B / 16; idx += 32) reinterpret_cast<uint4*>(v_t)[idx] = make_uint4(0, 0, 0, 0);
         __syncwarp();
 #pragma unroll
         for (int i = 0; i < NB; ++i) {
           const int idx = i * 32 + lane, key = idx / (HD / 8), c = idx % (HD / 8);
           if (key < p.D) {
-            *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(k_t) + k_tile_elem(key, c * 8)) = kreg[i];
+            *reinterpret_cast<uint4*>(st + (c >> 3) * 2 * K_PANEL_B + tj * K_PANEL_B + key * 128 + (((c & 7) ^ (key & 7)) << 4)) = kreg[i];
             const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(&vreg[i]);
 #pragma unroll
             for (int e = 0; e < 8; ++e) reinterpret_cast<__nv_bfloat16*>(v_t)[vt_tile_elem(key, c * 8 + e)] = ve[e];
@@ -656,8 +733,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
         ptx::fence_proxy_async();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&full[ring.stage]);
-        ring.advance(NS);
       }
+      ring.advance(NS);
       it = nxt;
     }
     if (!ok && lane == 0) attn_timeout(p, 4);
@@ -673,25 +750,24 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
 // ---------------------------------------------------------------------------------------------
 constexpr int kAttnSmemLimit = 232448;  // largest dynamic shared memory of one CTA on sm_100
 
-template <int HD>
+template <int HD, int NQ>
 static int attn_fixed_smem(int batch) {
-  return 1024 + (HD / 64) * 128 * 128 + 2 * 128 * 128 + 15 * 8 + 16 + 1024 + (batch + 1) * 4 + 64;
+  // alignment slack, Q, two P^T buffers, 15 barriers, flags, row scratch, prefix sums; for d = 64 the
+  // M = 128 O^T instruction reads 64 rows past the last V^T tile, which must still be shared memory
+  return 1024 + (HD / 64) * NQ * 128 + 4 * NQ * 128 + 16 * 8 + 32 + 960 * 4 + (batch + 1) * 4 + 64 +
+         (HD == 64 ? 8192 : 0);
 }
 
-template <int HD>
-static int attn_stage_count(int batch) {
-  const int tile_b = 2 * kPageSize * HD * 2;
-  int n = (kAttnSmemLimit - attn_fixed_smem<HD>(batch)) / (tile_b + 16);
-  return n > 8 ? 8 : n;
-}
-
-template <int HD, int C>
+template <int HD, int NQ>
 static cudaError_t attn_launch_one(sdlm_ctx* ctx, AttnParams& p, cudaStream_t st) {
-  p.n_stages = attn_stage_count<HD>(p.batch);
-  if (p.n_stages < 2) return cudaErrorLaunchOutOfResources;
-  const size_t smem = (size_t)attn_fixed_smem<HD>(p.batch) + (size_t)p.n_stages * (2 * kPageSize * HD * 2 + 16);
+  const int pair_b = 2 * (2 * kPageSize * HD * 2);
+  int n = (kAttnSmemLimit - attn_fixed_smem<HD, NQ>(p.batch)) / (pair_b + 16);
+  if (n > 6) n = 6;
+  if (n < 2) return cudaErrorLaunchOutOfResources;
+  p.n_stages = n;
+  const size_t smem = (size_t)attn_fixed_smem<HD, NQ>(p.batch) + (size_t)n * (pair_b + 16);
   const int n_cta = ctx->sm_count < kAttnMaxCtas ? ctx->sm_count : kAttnMaxCtas;
-  block_attn_umma_kernel<HD, C><<<n_cta, kAttnThreads, smem, st>>>(p);
+  block_attn_umma_kernel<HD, NQ><<<n_cta, kAttnThreads, smem, st>>>(p);
   ctx->launches++;
   return cudaGetLastError();
 }
@@ -699,13 +775,13 @@ static cudaError_t attn_launch_one(sdlm_ctx* ctx, AttnParams& p, cudaStream_t st
 cudaError_t setup_attn(sdlm_ctx* ctx) {
   cudaError_t e = cudaSuccess;
   if (ctx->cfg.head_dim == 128) {
-    e = cudaFuncSetAttribute(block_attn_umma_kernel<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
+    e = cudaFuncSetAttribute(block_attn_umma_kernel<128, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(block_attn_umma_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
+      e = cudaFuncSetAttribute(block_attn_umma_kernel<128, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
   } else {
-    e = cudaFuncSetAttribute(block_attn_umma_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
+    e = cudaFuncSetAttribute(block_attn_umma_kernel<64, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(block_attn_umma_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
+      e = cudaFuncSetAttribute(block_attn_umma_kernel<64, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
   }
   return e;
 }
@@ -729,9 +805,9 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
   p.scale_log2 = ctx->scale * 1.4426950408889634f;
   p.batch = batch; p.D = D; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.G = ctx->group;
   p.mpps = c.max_pages_per_seq; p.num_pages = c.num_pages; p.n_stages = 0;
-  const bool wide = ctx->group * D > 32;  // 2 replicas of up to 64 rows, else 4 replicas of up to 32
-  if (c.head_dim == 128) return wide ? attn_launch_one<128, 2>(ctx, p, st) : attn_launch_one<128, 4>(ctx, p, st);
-  return wide ? attn_launch_one<64, 2>(ctx, p, st) : attn_launch_one<64, 4>(ctx, p, st);
+  const bool wide = ctx->group * D > 32;  // stacked query rows padded to 64, else to 32
+  if (c.head_dim == 128) return wide ? attn_launch_one<128, 64>(ctx, p, st) : attn_launch_one<128, 32>(ctx, p, st);
+  return wide ? attn_launch_one<64, 64>(ctx, p, st) : attn_launch_one<64, 32>(ctx, p, st);
 }
 
 }  // namespace sdlm

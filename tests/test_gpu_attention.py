@@ -71,6 +71,35 @@ def test_attention_ignores_garbage_beyond_the_sequence_end():
     check_attention(pk.bits_from_bf16_tensor(out), ref)
 
 
+@pytest.mark.parametrize("D", [4, 8])
+def test_attention_with_scores_that_keep_outgrowing_the_row_reference(D):
+    """Scores rise steadily along the sequence (by far more than 2^32 per 128 keys), and fall again
+    for a second sequence: the kernel has to move its softmax references many times, or never."""
+    shape = syn.Shape(16, 2, 128, 64, 64)
+    lens = np.array([700, 333], dtype=np.int32)
+    wl = syn.Workload("attn_rebase", shape, 2, D, 0, 0, (0.9,), seed=36)
+    dp = DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16), lengths=lens)
+    x = syn.block_inputs(wl, dp.w_bits)
+    q = syn.bf16_bits_to_f32(x.q) * 0.05
+    q[..., 0] = 8.0                                           # every query looks along coordinate 0
+    prefix = []
+    for b, n in enumerate(lens):
+        k, v = dp.prefix[b]
+        kf = syn.bf16_bits_to_f32(k) * 0.05
+        ramp = np.arange(n, dtype=np.float32) * 0.5
+        kf[:, :, 0] = (ramp if b == 0 else ramp[::-1])[:, None]
+        prefix.append((syn.f32_to_bf16_bits(kf), v))
+    dp.prefix = prefix
+    dp.reset_cache()
+    q_bits = syn.f32_to_bf16_bits(q)
+    out = dp.sd.block_attn(pk.bf16_tensor_from_bits(q_bits), pk.bf16_tensor_from_bits(x.k_blk),
+                           pk.bf16_tensor_from_bits(x.v_blk))
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+    ref = orc.block_attention(q_bits, x.k_blk, x.v_blk, [a for a, _ in prefix], [b for _, b in prefix])
+    check_attention(pk.bits_from_bf16_tensor(out), ref)
+
+
 def test_attention_rejects_bad_arguments():
     shape = syn.SHAPE_TINY
     wl = syn.Workload("attn_bad", shape, 2, 4, 8, 8, (0.9,), seed=35)
