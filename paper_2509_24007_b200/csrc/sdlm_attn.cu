@@ -73,27 +73,31 @@ struct Item {
 
 struct ItemWalk {
   const int* s_first;  // [batch + 1] exclusive prefix sum of (pages + 1) per batch row
-  long long total;     // tiles in the whole launch
-  long long cur, hi;
-  int nc;
+  const int* s_len;    // [batch] cached tokens per batch row
+  const int* s_slot;   // [batch] sequence slot per batch row
+  uint32_t total;      // tiles in the whole launch (the host keeps total * gridDim below 2^31)
+  uint32_t cur, hi;
+  uint32_t nc;
 };
 
-__device__ __forceinline__ int tile_owner(long long x, long long total, int nc) {
+__device__ __forceinline__ int tile_owner(uint32_t x, uint32_t total, uint32_t nc) {
   return (int)(((x + 1) * nc - 1) / total);  // the CTA c with floor(c*total/nc) <= x < floor((c+1)*total/nc)
 }
 
 __device__ __forceinline__ void walk_begin(ItemWalk& w, const int* s_first, int batch, int Hkv) {
   w.s_first = s_first;
-  w.total = (long long)s_first[batch] * Hkv;
+  w.s_len = s_first + batch + 1;
+  w.s_slot = w.s_len + batch;
+  w.total = (uint32_t)s_first[batch] * (uint32_t)Hkv;
   // never more ranges than tiles: every range is then non-empty and the CTAs that share a pair
   // are consecutive
-  w.nc = (int)min((long long)gridDim.x, w.total);
-  if ((int)blockIdx.x >= w.nc) {
+  w.nc = min(gridDim.x, w.total);
+  if (blockIdx.x >= w.nc) {
     w.cur = w.hi = 0;
     return;
   }
-  w.cur = (long long)blockIdx.x * w.total / w.nc;
-  w.hi = (long long)(blockIdx.x + 1) * w.total / w.nc;
+  w.cur = blockIdx.x * w.total / w.nc;
+  w.hi = (blockIdx.x + 1) * w.total / w.nc;
 }
 
 __device__ __forceinline__ bool walk_next(ItemWalk& w, const AttnParams& p, Item& it) {
@@ -101,19 +105,19 @@ __device__ __forceinline__ bool walk_next(ItemWalk& w, const AttnParams& p, Item
   int lo = 0, hi = p.batch - 1;
   while (lo < hi) {
     const int mid = (lo + hi + 1) >> 1;
-    if ((long long)w.s_first[mid] * p.Hkv <= w.cur) lo = mid; else hi = mid - 1;
+    if ((uint32_t)w.s_first[mid] * (uint32_t)p.Hkv <= w.cur) lo = mid; else hi = mid - 1;
   }
   it.b = lo;
-  const int tiles_b = w.s_first[lo + 1] - w.s_first[lo];
-  const long long row_start = (long long)w.s_first[lo] * p.Hkv;
+  const uint32_t tiles_b = (uint32_t)(w.s_first[lo + 1] - w.s_first[lo]);
+  const uint32_t row_start = (uint32_t)w.s_first[lo] * (uint32_t)p.Hkv;
   it.h = (int)((w.cur - row_start) / tiles_b);
-  const long long pair_start = row_start + (long long)it.h * tiles_b;
+  const uint32_t pair_start = row_start + (uint32_t)it.h * tiles_b;
   it.t0 = (int)(w.cur - pair_start);
-  const long long end = min(w.hi, pair_start + tiles_b);
+  const uint32_t end = min(w.hi, pair_start + tiles_b);
   it.t1 = (int)(end - pair_start);
-  it.pages = tiles_b - 1;
-  it.slot = attn_slot(p, lo);
-  it.len = attn_len(p, lo);
+  it.pages = (int)tiles_b - 1;
+  it.slot = w.s_slot[lo];
+  it.len = w.s_len[lo];
   it.pair = lo * p.Hkv + it.h;
   it.c_first = tile_owner(pair_start, w.total, w.nc);
   it.n_splits = tile_owner(pair_start + tiles_b - 1, w.total, w.nc) - it.c_first + 1;
@@ -193,7 +197,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
   float* fbuf = mnew + 64;              // [64] rescale factors of a reference move
   int* mx = reinterpret_cast<int*>(fbuf + 64);                          // [4][64] per-warp row maxima
   float* lsum = reinterpret_cast<float*>(mx + 256);                     // [2][4][64] per-warp row sums, by item parity
-  int* s_first = reinterpret_cast<int*>(lsum + 512);
+  int* row_off = reinterpret_cast<int*>(lsum + 512);  // [64] element offset of stacked row r inside a (b, KV head) slab
+  int* s_first = row_off + 64;                         // [batch + 1], then lengths [batch], then slots [batch]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int GD = p.G * p.D;
@@ -203,7 +208,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
     int carry = 0;
     for (int base = 0; base < p.batch; base += 32) {
       const int i = base + lane;
-      const int n = (i < p.batch) ? (attn_len(p, i) + kPageSize - 1) / kPageSize + 1 : 0;
+      int n = 0;
+      if (i < p.batch) {
+        const int len = attn_len(p, i);
+        s_first[p.batch + 1 + i] = len;
+        s_first[2 * p.batch + 1 + i] = attn_slot(p, i);
+        n = (len + kPageSize - 1) / kPageSize + 1;
+      }
       int incl = n;
       for (int o = 1; o < 32; o <<= 1) {
         const int v = __shfl_up_sync(0xffffffffu, incl, o);
@@ -214,6 +225,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
     }
     if (lane == 0) s_first[p.batch] = carry;
   }
+  // stacked row r = j*G + g is q[b, j, h*G + g, :] (and the same row of out)
+  if (tid >= 64 && tid < 128) row_off[tid - 64] = tid - 64 < GD ? (((tid - 64) / p.G) * p.Hq + (tid - 64) % p.G) * HD : -1;
   if (tid == 32) {
     for (int s = 0; s < NS; ++s) {
       ptx::mbar_init(&full[s], 2);  // the copies' issuer, plus whoever completes the group (see warp 0)
@@ -558,7 +571,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
           for (int q = 0; q < NQ; ++q) {
             if (q < GD) {
               const float lt = ls[q] + ls[64 + q] + ls[128 + q] + ls[192 + q];
-              out_base[((size_t)(q / p.G) * p.Hq + q % p.G) * HD] = __float2bfloat16_rn(o[q] / lt);
+              out_base[row_off[q]] = __float2bfloat16_rn(o[q] / lt);
             }
           }
         }
@@ -582,41 +595,36 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
         if (!meet()) { ok = false; break; }
         if (*s_last) {
           // ---- merge the splits of this pair (fixed order: run-to-run identical).  Row q's weight of
-          // split s is 2^(m_s - m) / L with m = max_s m_s, L = sum_s 2^(m_s - m) l_s; the weights go
-          // through the (now idle) P^T buffers, then every thread sums four output columns.
+          // split s is 2^(m_s - m) with m = max_s m_s; the weights go through the (now idle) P^T
+          // buffers, every thread sums four output columns, and the row sum L divides at the end.
           __threadfence();
           constexpr int kCap = 128;  // splits whose weights fit into the P^T buffers at once
           float* wbuf = reinterpret_cast<float*>(p_s);
           const size_t first_row = (size_t)(it.c_first + it.pair) * NQ;
+          float m = -INFINITY, L = 0.f;
           if (kg < GD) {
-            float m = -INFINITY;
 #pragma unroll 8
             for (int s = 0; s < it.n_splits; ++s) m = fmaxf(m, __ldcg(p.part_ml + (first_row + (size_t)s * NQ + kg) * 2));
-            float L = 0.f;
-#pragma unroll 8
-            for (int s = 0; s < it.n_splits; ++s) {
-              const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (first_row + (size_t)s * NQ + kg) * 2));
-              L = fmaf(ptx::ex2(ml.x - m), ml.y, L);
-            }
-            mnew[kg] = m;
-            fbuf[kg] = 1.0f / L;
           }
           const int dq = tid & 31, qg = (tid >> 5) & 3;  // four columns 4*dq.. of the rows q = qg mod 4
           float acc[NQ / 4][4];
 #pragma unroll
           for (int i = 0; i < NQ / 4; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
-          for (int c0 = 0; c0 < it.n_splits && ok; c0 += kCap) {
+          for (int c0 = 0; c0 < it.n_splits; c0 += kCap) {
             const int cn = min(kCap, it.n_splits - c0);
-            if (!meet()) { ok = false; break; }  // mnew / fbuf written; wbuf no longer read
+            if (c0 > 0 && !meet()) { ok = false; break; }  // the previous chunk's weights are no longer read
             if (kg < GD) {
-              const float m = mnew[kg], inv = fbuf[kg];
 #pragma unroll 8
-              for (int s = 0; s < cn; ++s)
-                wbuf[s * NQ + kg] = ptx::ex2(__ldcg(p.part_ml + (first_row + (size_t)(c0 + s) * NQ + kg) * 2) - m) * inv;
+              for (int s = 0; s < cn; ++s) {
+                const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (first_row + (size_t)(c0 + s) * NQ + kg) * 2));
+                const float a = ptx::ex2(ml.x - m);
+                L = fmaf(a, ml.y, L);
+                wbuf[s * NQ + kg] = a;
+              }
             }
             if (!meet()) { ok = false; break; }
             if (4 * dq < HD) {
-#pragma unroll 2
+#pragma unroll 4
               for (int s = 0; s < cn; ++s) {
                 const float* src = p.part_o + (first_row + (size_t)(c0 + s) * NQ) * HD + 4 * dq;
 #pragma unroll
@@ -635,20 +643,23 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
             }
           }
           if (!ok) break;
+          if (kg < GD) fbuf[kg] = 1.0f / L;
+          if (!meet()) { ok = false; break; }
           if (4 * dq < HD) {
             __nv_bfloat16* ob = p.out + ((size_t)it.b * p.D * p.Hq + it.h * p.G) * HD + 4 * dq;
 #pragma unroll
             for (int i = 0; i < NQ / 4; ++i) {
               const int q = qg + 4 * i;
               if (q < GD) {
+                const float inv = fbuf[q];
                 uint2 v;
-                v.x = ptx::pack_bf16(acc[i][0], acc[i][1]);
-                v.y = ptx::pack_bf16(acc[i][2], acc[i][3]);
-                *reinterpret_cast<uint2*>(ob + ((size_t)(q / p.G) * p.Hq + q % p.G) * HD) = v;
+                v.x = ptx::pack_bf16(acc[i][0] * inv, acc[i][1] * inv);
+                v.y = ptx::pack_bf16(acc[i][2] * inv, acc[i][3] * inv);
+                *reinterpret_cast<uint2*>(ob + row_off[q]) = v;
               }
             }
           }
-          if (!meet()) { ok = false; break; }  // the P^T buffers go back to the softmax
+          if (!meet()) { ok = false; break; }  // the P^T buffers and fbuf go back to the softmax
         }
       }
     }
@@ -669,10 +680,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
       for (int i = 0; i < NQC; ++i) {
         const int idx = i * 32 + lane, r = idx / (HD / 8), c = idx % (HD / 8);
         qreg[i] = make_uint4(0, 0, 0, 0);
-        if (r < GD) {
-          const int j = r / p.G, g = r % p.G;
-          qreg[i] = __ldg(reinterpret_cast<const uint4*>(p.q + (((size_t)x.b * p.D + j) * p.Hq + x.h * p.G + g) * HD) + c);
-        }
+        if (r < GD)
+          qreg[i] = __ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)x.b * p.D * p.Hq + x.h * p.G) * HD + row_off[r]) + c);
       }
     };
     bool have = walk_next(w, p, it);
@@ -754,7 +763,7 @@ template <int HD, int NQ>
 static int attn_fixed_smem(int batch) {
   // alignment slack, Q, two P^T buffers, 15 barriers, flags, row scratch, prefix sums; for d = 64 the
   // M = 128 O^T instruction reads 64 rows past the last V^T tile, which must still be shared memory
-  return 1024 + (HD / 64) * NQ * 128 + 4 * NQ * 128 + 16 * 8 + 32 + 960 * 4 + (batch + 1) * 4 + 64 +
+  return 1024 + (HD / 64) * NQ * 128 + 4 * NQ * 128 + 16 * 8 + 32 + 960 * 4 + 64 * 4 + (batch + 1) * 12 + 64 +
          (HD == 64 ? 8192 : 0);
 }
 
@@ -805,6 +814,8 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
   p.scale_log2 = ctx->scale * 1.4426950408889634f;
   p.batch = batch; p.D = D; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.G = ctx->group;
   p.mpps = c.max_pages_per_seq; p.num_pages = c.num_pages; p.n_stages = 0;
+  // the kernel's tile arithmetic is 32-bit: (tiles of the launch) x (CTAs) must stay below 2^31
+  if ((long long)batch * (c.max_pages_per_seq + 1) * c.n_kv_heads > 13000000ll) return cudaErrorInvalidConfiguration;
   const bool wide = ctx->group * D > 32;  // stacked query rows padded to 64, else to 32
   if (c.head_dim == 128) return wide ? attn_launch_one<128, 64>(ctx, p, st) : attn_launch_one<128, 32>(ctx, p, st);
   return wide ? attn_launch_one<64, 64>(ctx, p, st) : attn_launch_one<64, 32>(ctx, p, st);
