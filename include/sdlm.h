@@ -104,7 +104,11 @@ typedef enum sdlm_kv_op {
                               DEVICE bf16 [args.length, Hkv, d]; rows at or beyond the slot's current
                               length are left untouched                                             */
   SDLM_KV_EXPORT = 5,      /* synchronise `stream`, copy all tables to HOST args.host_buf            */
-  SDLM_KV_IMPORT = 6       /* restore tables from a HOST buffer written by EXPORT (same config)      */
+  SDLM_KV_IMPORT = 6,      /* restore tables from a HOST buffer written by EXPORT (same config)      */
+  SDLM_KV_SAVE = 7,        /* copy all tables to DEVICE args.dev_buf (>= table_bytes), enqueued on `stream`,
+                              no host synchronisation                                                */
+  SDLM_KV_RESTORE = 8      /* the reverse of SAVE: lengths, page tables and the free ring go back to the
+                              saved state (cache rows written since stay in the pool, unreferenced)   */
 } sdlm_kv_op;
 
 typedef struct sdlm_kv_args {
@@ -117,6 +121,8 @@ typedef struct sdlm_kv_args {
   const int32_t* free_list;  /* RESET (host) */
   void* host_buf;            /* EXPORT / IMPORT (host) */
   size_t host_bytes;         /* size of host_buf; must be >= result.table_bytes */
+  void* dev_buf;             /* SAVE / RESTORE (device), 16-byte aligned */
+  size_t dev_bytes;          /* size of dev_buf; must be >= result.table_bytes */
 } sdlm_kv_args;
 
 typedef struct sdlm_kv_result {
@@ -205,6 +211,17 @@ sdlm_status sdlm_accept_commit(sdlm_ctx* ctx, int32_t batch, int32_t D, const in
  * `clear` != 0 resets them afterwards. */
 sdlm_status sdlm_device_status(sdlm_ctx* ctx, int32_t* host_out, int32_t clear, void* stream);
 
+/* ---- whole step on device memory: (a) + (b) + (c) in one call, same arguments and results as the
+ * three calls made one after the other (Sec. 3.2: one forward pass, then Decode).  The library
+ * knows here that the LM head reads nothing attention writes, so with SDLM_OPT_STEP_OVERLAP it
+ * may overlap the two on the GPU; `hidden` and `w_lm` must not alias `attn_out`.  All pointers are DEVICE
+ * memory and required (seq_ids may be NULL).
+ * Errors: as the three calls. */
+sdlm_status sdlm_decode_step(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, float tau,
+                             sdlm_conf_mode mode, const void* q, const void* k_blk, const void* v_blk,
+                             const void* hidden, const void* w_lm, void* attn_out, int32_t* token, float* p_top1,
+                             float* entropy, int32_t* accepted_len, int32_t* out_tokens, void* stream);
+
 /* ---- whole step from host memory: (a) + (b) + (c) for callers whose block inputs live on the
  * host.  Copies q, k_blk, v_blk [as above] and hidden [batch*D, H] from HOST memory (pinned for
  * best speed), and seq_ids (HOST int32 [batch] or NULL), to workspace staging; runs the three
@@ -222,8 +239,10 @@ sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const
 /* Tuning / test knobs (the paper has no counterpart).  SDLM_OPT_LMHEAD_KERNEL: which stripe kernel
  * sdlm_lmhead_confidence uses: 0 = chosen from the shape (default), 1 = warp-level mma.sync
  * kernel, 2 = tcgen05 / TMA kernel (the call then fails with UNSUPPORTED for rows > 256 or
- * |V| < 16).  Errors: INVALID_ARG. */
-typedef enum sdlm_option { SDLM_OPT_LMHEAD_KERNEL = 0 } sdlm_option;
+ * |V| < 16).  SDLM_OPT_STEP_OVERLAP: 1 lets sdlm_decode_step / sdlm_decode_step_host start the
+ * LM-head kernel while attention's last thread blocks are still running (default 0: in order).
+ * Errors: INVALID_ARG. */
+typedef enum sdlm_option { SDLM_OPT_LMHEAD_KERNEL = 0, SDLM_OPT_STEP_OVERLAP = 1 } sdlm_option;
 sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t value);
 
 /* Number of kernels the library has launched through this context since it was created. */

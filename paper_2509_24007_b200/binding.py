@@ -19,15 +19,16 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsdlm.so")
 
 CONF_LOGIT, CONF_ENTROPY = 0, 1
-KV_RESET, KV_ADD_SEQ, KV_RELEASE_SEQ, KV_QUERY, KV_GATHER, KV_EXPORT, KV_IMPORT = range(7)
+KV_RESET, KV_ADD_SEQ, KV_RELEASE_SEQ, KV_QUERY, KV_GATHER, KV_EXPORT, KV_IMPORT, KV_SAVE, KV_RESTORE = range(9)
 OPT_LMHEAD_KERNEL = 0
+OPT_STEP_OVERLAP = 1
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "UNSUPPORTED", 4: "OUT_OF_PAGES", 5: "CUDA",
                 6: "TIMEOUT", 7: "DEVICE_CHECK", 8: "WORKSPACE"}
 
 EXPORTED = ["sdlm_pool_bytes", "sdlm_workspace_bytes", "sdlm_create", "sdlm_destroy", "sdlm_status_str",
             "sdlm_kv_pages", "sdlm_block_attn", "sdlm_lmhead_confidence", "sdlm_lmhead_confidence_static", "sdlm_accept_commit",
-            "sdlm_device_status", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count"]
+            "sdlm_device_status", "sdlm_decode_step", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count"]
 
 
 class SdlmError(RuntimeError):
@@ -45,7 +46,8 @@ class _Config(C.Structure):
 class _KvArgs(C.Structure):
     _fields_ = [("seq", C.c_int32), ("length", C.c_int32), ("k", C.c_void_p), ("v", C.c_void_p),
                 ("k_out", C.c_void_p), ("v_out", C.c_void_p), ("free_list", C.c_void_p),
-                ("host_buf", C.c_void_p), ("host_bytes", C.c_size_t)]
+                ("host_buf", C.c_void_p), ("host_bytes", C.c_size_t), ("dev_buf", C.c_void_p),
+                ("dev_bytes", C.c_size_t)]
 
 
 class _KvResult(C.Structure):
@@ -108,6 +110,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdlm_accept_commit.argtypes = [vp, i32, i32, vp, f32, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_device_status.restype = C.c_int
     lib.sdlm_device_status.argtypes = [vp, vp, i32, vp]
+    lib.sdlm_decode_step.restype = C.c_int
+    lib.sdlm_decode_step.argtypes = [vp, i32, i32, vp, f32, C.c_int] + [vp] * 12
     lib.sdlm_decode_step_host.restype = C.c_int
     lib.sdlm_decode_step_host.argtypes = [vp, i32, i32, vp, f32, C.c_int] + [vp] * 12
     lib.sdlm_set_option.restype = C.c_int
@@ -192,7 +196,7 @@ class Sdlm:
     def kv_pages(self, op: int, seq: int = 0, length: int = 0, k: Optional[torch.Tensor] = None,
                  v: Optional[torch.Tensor] = None, k_out: Optional[torch.Tensor] = None,
                  v_out: Optional[torch.Tensor] = None, free_list: Optional[np.ndarray] = None,
-                 host_buf: Optional[np.ndarray] = None, stream=None) -> _KvResult:
+                 host_buf: Optional[np.ndarray] = None, dev_buf: Optional[torch.Tensor] = None, stream=None) -> _KvResult:
         a = _KvArgs()
         a.seq, a.length = seq, length
         keep = []
@@ -208,6 +212,9 @@ class Sdlm:
             a.free_list = fl.ctypes.data
         if host_buf is not None:
             a.host_buf, a.host_bytes = host_buf.ctypes.data, host_buf.nbytes
+        if dev_buf is not None:
+            _dev(dev_buf, torch.uint8, "dev_buf")
+            a.dev_buf, a.dev_bytes = dev_buf.data_ptr(), dev_buf.numel()
         r = _KvResult()
         self._check("sdlm_kv_pages", self.lib.sdlm_kv_pages(self.ctx, op, C.byref(a), C.byref(r), _stream_ptr(stream)))
         return r
@@ -252,6 +259,16 @@ class Sdlm:
         buf = np.empty(r.table_bytes, dtype=np.uint8)
         self.kv_pages(KV_EXPORT, host_buf=buf)
         return buf
+
+    def kv_save(self, dev_buf: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """Device-side snapshot of the tables (no host synchronisation); returns the buffer."""
+        if dev_buf is None:
+            dev_buf = torch.empty(self.kv_pages(KV_QUERY).table_bytes, dtype=torch.uint8, device=self.device)
+        self.kv_pages(KV_SAVE, dev_buf=dev_buf, stream=stream)
+        return dev_buf
+
+    def kv_restore(self, dev_buf: torch.Tensor, stream=None) -> None:
+        self.kv_pages(KV_RESTORE, dev_buf=dev_buf, stream=stream)
 
     def kv_import(self, buf: np.ndarray) -> None:
         self.kv_pages(KV_IMPORT, host_buf=np.ascontiguousarray(buf))
@@ -323,6 +340,21 @@ class Sdlm:
         self._check("sdlm_device_status", self.lib.sdlm_device_status(self.ctx, out.ctypes.data, int(clear),
                                                                       _stream_ptr(stream)))
         return out
+
+    def decode_step(self, tau: float, q: torch.Tensor, k_blk: torch.Tensor, v_blk: torch.Tensor, hidden: torch.Tensor,
+                    w_lm: torch.Tensor, attn_out: torch.Tensor, token: torch.Tensor, p_top1: torch.Tensor,
+                    entropy: torch.Tensor, accepted_len: torch.Tensor, out_tokens: torch.Tensor,
+                    seq_ids: Optional[torch.Tensor] = None, mode: int = CONF_LOGIT, stream=None) -> None:
+        """Whole step on device tensors: attention, LM-head statistics, accept + commit."""
+        batch, D = int(q.shape[0]), int(q.shape[1])
+        for t, n in ((q, "q"), (k_blk, "k_blk"), (v_blk, "v_blk"), (hidden, "hidden"), (w_lm, "w_lm"), (attn_out, "attn_out")):
+            _dev(t, torch.bfloat16, n)
+        _dev(token, torch.int32, "token"); _dev(p_top1, torch.float32, "p_top1"); _dev(entropy, torch.float32, "entropy")
+        _dev(accepted_len, torch.int32, "accepted_len"); _dev(out_tokens, torch.int32, "out_tokens")
+        self._check("sdlm_decode_step", self.lib.sdlm_decode_step(
+            self.ctx, batch, D, _ptr(seq_ids), float(tau), int(mode), _ptr(q), _ptr(k_blk), _ptr(v_blk), _ptr(hidden),
+            _ptr(w_lm), _ptr(attn_out), _ptr(token), _ptr(p_top1), _ptr(entropy), _ptr(accepted_len),
+            _ptr(out_tokens), _stream_ptr(stream)))
 
     def decode_step_host(self, tau: float, q: torch.Tensor, k_blk: torch.Tensor, v_blk: torch.Tensor,
                          hidden: torch.Tensor, w_lm: torch.Tensor, attn_out: Optional[torch.Tensor] = None,

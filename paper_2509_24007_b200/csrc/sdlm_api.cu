@@ -1,6 +1,7 @@
 // Host side of the C ABI plus the small table kernels: context, page bookkeeping (Fig. 2b's
 // cached KV states as a paged pool), longest-prefix acceptance and commit (Eq. 7, Eq. 4).
 #include "sdlm_internal.h"
+#include "sdlm_ptx.cuh"
 
 #include <math.h>
 #include <new>
@@ -221,6 +222,8 @@ __global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitPar
   __shared__ uint32_t s_head, s_avail;
   __shared__ int s_last;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();  // the statistics this kernel reads come from the kernels before it
   if (tid == 0) {
     s_head = *(volatile uint32_t*)&p.hdr->free_head;
     s_avail = *(volatile uint32_t*)&p.hdr->free_tail - s_head;
@@ -410,6 +413,7 @@ extern "C" sdlm_status sdlm_create(const sdlm_config* cfg, void* kv_pool, size_t
   ctx->free_list = reinterpret_cast<int32_t*>(ctx->ws + ctx->lay.free_list);
   ctx->launches = 0;
   ctx->lmhead_path = 0;
+  ctx->overlap_lmhead = 0;
   ctx->tmap_w_ptr = nullptr;
   ctx->tmap_w_rows = 0;
   if (setup_attn(ctx) != cudaSuccess || setup_lmhead(ctx) != cudaSuccess) { delete ctx; return SDLM_ERR_CUDA; }
@@ -428,6 +432,10 @@ extern "C" sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t v
     case SDLM_OPT_LMHEAD_KERNEL:
       if (value < 0 || value > 2) return SDLM_ERR_INVALID_ARG;
       ctx->lmhead_path = value;
+      return SDLM_OK;
+    case SDLM_OPT_STEP_OVERLAP:
+      if (value < 0 || value > 1) return SDLM_ERR_INVALID_ARG;
+      ctx->overlap_lmhead = value;
       return SDLM_OK;
   }
   return SDLM_ERR_INVALID_ARG;
@@ -499,6 +507,16 @@ extern "C" sdlm_status sdlm_kv_pages(sdlm_ctx* ctx, sdlm_kv_op op, const sdlm_kv
       if (r) r->table_bytes = table_bytes;
       return SDLM_OK;
     }
+    case SDLM_KV_SAVE:
+    case SDLM_KV_RESTORE: {
+      if (!a || !a->dev_buf || a->dev_bytes < table_bytes || !aligned16(a->dev_buf)) return SDLM_ERR_INVALID_ARG;
+      void* tables = ctx->ws + ctx->lay.hdr;
+      const cudaError_t e = op == SDLM_KV_SAVE
+                                ? cudaMemcpyAsync(a->dev_buf, tables, table_bytes, cudaMemcpyDeviceToDevice, st)
+                                : cudaMemcpyAsync(tables, a->dev_buf, table_bytes, cudaMemcpyDeviceToDevice, st);
+      if (r) r->table_bytes = table_bytes;
+      return e == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+    }
     case SDLM_KV_IMPORT: {
       if (!a || !a->host_buf || a->host_bytes < table_bytes) return SDLM_ERR_INVALID_ARG;
       if (cudaStreamSynchronize(st) != cudaSuccess) return SDLM_ERR_CUDA;
@@ -562,9 +580,10 @@ extern "C" sdlm_status sdlm_accept_commit(sdlm_ctx* ctx, int32_t batch, int32_t 
   p.inv_ln_vocab = c.vocab > 1 ? (float)(1.0 / log((double)c.vocab)) : 0.0f;
   p.mode = (int)mode; p.batch = batch; p.D = D; p.Hkv = c.n_kv_heads; p.d = c.head_dim;
   p.mpps = c.max_pages_per_seq; p.num_pages = c.num_pages;
-  accept_commit_kernel<<<batch, kCommitThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+  const cudaError_t e = launch_overlapped(accept_commit_kernel, dim3(batch), dim3(kCommitThreads), 0,
+                                          static_cast<cudaStream_t>(stream), p);
   ctx->launches++;
-  return cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+  return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
 }
 
 extern "C" sdlm_status sdlm_device_status(sdlm_ctx* ctx, int32_t* host_out, int32_t clear, void* stream) {
@@ -574,6 +593,34 @@ extern "C" sdlm_status sdlm_device_status(sdlm_ctx* ctx, int32_t* host_out, int3
   if (clear && cudaMemsetAsync(ctx->hdr->status, 0, 16, st) != cudaSuccess) return SDLM_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return SDLM_ERR_CUDA;
   return SDLM_OK;
+}
+
+// (a) + (b) + (c) on device buffers.  The LM head reads nothing that attention writes, so its stripe
+// kernel is allowed to start while attention's last CTAs are still running.
+static sdlm_status decode_step_device(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, float tau,
+                                      sdlm_conf_mode mode, const void* q, const void* k_blk, const void* v_blk,
+                                      const void* hidden, const void* w_lm, void* attn_out, int32_t* token,
+                                      float* p_top1, float* entropy, int32_t* accepted_len, int32_t* out_tokens,
+                                      void* stream) {
+  sdlm_status s = sdlm_block_attn(ctx, batch, D, seq_ids, q, k_blk, v_blk, attn_out, stream);
+  if (s != SDLM_OK) return s;
+  if (!hidden || !w_lm || !token || !p_top1 || !entropy) return SDLM_ERR_INVALID_ARG;
+  if (!aligned16(hidden) || !aligned16(w_lm)) return SDLM_ERR_INVALID_ARG;
+  s = launch_lmhead(ctx, batch * D, hidden, w_lm, token, p_top1, entropy, nullptr, nullptr,
+                    static_cast<cudaStream_t>(stream), /*independent_of_predecessor=*/ctx->overlap_lmhead != 0);
+  if (s != SDLM_OK) return s;
+  return sdlm_accept_commit(ctx, batch, D, seq_ids, tau, mode, token, p_top1, entropy, k_blk, v_blk, accepted_len,
+                            out_tokens, stream);
+}
+
+extern "C" sdlm_status sdlm_decode_step(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, float tau,
+                                        sdlm_conf_mode mode, const void* q, const void* k_blk, const void* v_blk,
+                                        const void* hidden, const void* w_lm, void* attn_out, int32_t* token,
+                                        float* p_top1, float* entropy, int32_t* accepted_len, int32_t* out_tokens,
+                                        void* stream) {
+  if (!ctx) return SDLM_ERR_INVALID_ARG;
+  return decode_step_device(ctx, batch, D, seq_ids, tau, mode, q, k_blk, v_blk, hidden, w_lm, attn_out, token, p_top1,
+                            entropy, accepted_len, out_tokens, stream);
 }
 
 extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids_host,
@@ -607,12 +654,8 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
   float* d_ent = reinterpret_cast<float*>(ws + L.st_ent);
   int32_t* d_acc = reinterpret_cast<int32_t*>(ws + L.st_acc);
   int32_t* d_out_tokens = reinterpret_cast<int32_t*>(ws + L.st_out_tokens);
-  s = sdlm_block_attn(ctx, batch, D, seq_ids, ws + L.st_q, ws + L.st_k, ws + L.st_v, ws + L.st_out, stream);
-  if (s != SDLM_OK) return s;
-  s = sdlm_lmhead_confidence(ctx, (int32_t)rows, ws + L.st_hidden, w_lm, d_token, d_p, d_ent, nullptr, nullptr, stream);
-  if (s != SDLM_OK) return s;
-  s = sdlm_accept_commit(ctx, batch, D, seq_ids, tau, mode, d_token, d_p, d_ent, ws + L.st_k, ws + L.st_v, d_acc,
-                         d_out_tokens, stream);
+  s = decode_step_device(ctx, batch, D, seq_ids, tau, mode, ws + L.st_q, ws + L.st_k, ws + L.st_v, ws + L.st_hidden, w_lm,
+                         ws + L.st_out, d_token, d_p, d_ent, d_acc, d_out_tokens, stream);
   if (s != SDLM_OK) return s;
   if (attn_out_host) ok &= cudaMemcpyAsync(attn_out_host, ws + L.st_out, q_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   if (token_host) ok &= cudaMemcpyAsync(token_host, d_token, rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;

@@ -202,6 +202,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int GD = p.G * p.D;
+  ptx::grid_dep_wait();    // lengths, page table and pool are written by the kernels before this one
+  ptx::grid_dep_launch();  // only now: a successor that does not wait itself may then rely on them too
 
   // exclusive prefix sum of (pages + 1) per batch row
   if (warp == 0) {
@@ -776,9 +778,9 @@ static cudaError_t attn_launch_one(sdlm_ctx* ctx, AttnParams& p, cudaStream_t st
   p.n_stages = n;
   const size_t smem = (size_t)attn_fixed_smem<HD, NQ>(p.batch) + (size_t)n * (pair_b + 16);
   const int n_cta = ctx->sm_count < kAttnMaxCtas ? ctx->sm_count : kAttnMaxCtas;
-  block_attn_umma_kernel<HD, NQ><<<n_cta, kAttnThreads, smem, st>>>(p);
+  const cudaError_t e = launch_overlapped(block_attn_umma_kernel<HD, NQ>, dim3(n_cta), dim3(kAttnThreads), smem, st, p);
   ctx->launches++;
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t setup_attn(sdlm_ctx* ctx) {

@@ -60,6 +60,7 @@ struct sdlm_ctx {
   int32_t* free_list;
   uint64_t launches;
   int lmhead_path;  // 0 = pick by shape, 1 = force the mma.sync kernel, 2 = force the tcgen05 kernel
+  int overlap_lmhead;  // sdlm_decode_step: let the LM-head stripe kernel start before attention has finished
   // cached TMA descriptor of the LM-head weight (keyed by pointer and tile rows)
   const void* tmap_w_ptr;
   int tmap_w_rows;
@@ -88,11 +89,33 @@ __host__ __device__ inline int vt_tile_elem(int key, int col) {
   return col * kPageSize + (((key >> 3) ^ (col & 7)) << 3) + (key & 7);
 }
 
+// Launch with the programmatic-serialization attribute: the kernel may be scheduled while its
+// predecessor on the stream drains.  Every kernel launched this way calls ptx::grid_dep_wait()
+// before it touches memory the predecessor may write (or, where it needs none of it, before it ends).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                     Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- launchers implemented in the kernel translation units ---------------------------------
 cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, const void* q,
                               const void* k_blk, const void* v_blk, void* out, cudaStream_t st);
+// `independent_of_predecessor`: the caller guarantees that none of the inputs is written by the
+// kernel enqueued just before on `st` (the stripe kernel then overlaps with it).
 sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
-                          float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st);
+                          float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st,
+                          bool independent_of_predecessor = false);
 cudaError_t setup_attn(sdlm_ctx* ctx);
 cudaError_t setup_lmhead(sdlm_ctx* ctx);
 

@@ -53,6 +53,7 @@ struct LmParams {
   DevHeader* hdr;
   int rows, H, V, n_stripes, rows_pad;
   int bn;  // umma path: vocab rows per tile (multiple of 16, <= 256)
+  int wait_at_end;  // 1: no input comes from the kernel before this one; only completion order is kept
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -142,6 +143,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
   volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  ptx::grid_dep_launch();
 
   // this CTA's vocabulary stripe, in groups of 16 rows
   const int groups = (p.V + 15) / 16;
@@ -174,6 +176,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (!p.wait_at_end) ptx::grid_dep_wait();  // the hidden states may come from the kernel before this one
 
   if (warp == 0) {
     if (lane == 0) {  // ---- TMA producer
@@ -293,6 +296,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, 512);
   }
+  // Started without waiting for the kernel before it: do not finish before that kernel has, so that
+  // whatever follows on the stream still sees both completed.
+  if (p.wait_at_end) ptx::grid_dep_wait();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -305,6 +311,8 @@ __global__ void __launch_bounds__(kMmaThreads) lmhead_mma_kernel(const LmParams 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
   const int row_base = blockIdx.y * kMmaBM;
   const int tiles_total = (p.V + kMmaBN - 1) / kMmaBN;
   const int t0 = (int)((long long)blockIdx.x * tiles_total / gridDim.x);
@@ -429,6 +437,8 @@ __global__ void __launch_bounds__(128) lmhead_combine_kernel(const float4* parti
                                                              int32_t* token, float* p_top1, float* entropy,
                                                              float* max_logit, float* lse) {
   const int row = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();  // the partials come from the stripe kernel
   if (row >= rows) return;
   Stat st = stat_empty();
   for (int s = lane; s < n_stripes; s += 32) {
@@ -502,7 +512,7 @@ cudaError_t setup_lmhead(sdlm_ctx* ctx) {
 // `partials` holds one float4 per (stripe, row): [max_stripes][rows_pad].
 static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
                                     float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st,
-                                    float4* partials, int rows_pad, int max_stripes) {
+                                    float4* partials, int rows_pad, int max_stripes, bool independent) {
   const sdlm_config& c = ctx->cfg;
   LmParams p;
   p.hidden = static_cast<const __nv_bfloat16*>(hidden);
@@ -512,6 +522,8 @@ static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden,
   p.rows = rows; p.H = c.hidden; p.V = c.vocab;
   p.rows_pad = rows_pad;
   p.bn = 0;
+  p.wait_at_end = independent ? 1 : 0;
+  cudaError_t le = cudaSuccess;
 
   const bool use_umma = ctx->lmhead_path != 1 && rows <= 256 && c.vocab >= 16;
   if (ctx->lmhead_path == 2 && !use_umma) return SDLM_ERR_UNSUPPORTED;
@@ -538,9 +550,9 @@ static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden,
     const CUtensorMap& tm_w = *reinterpret_cast<const CUtensorMap*>(ctx->tmap_w);
     const size_t smem = (size_t)n_stages * stage_bytes + 1024 + 512;
     if (R == 1)
-      lmhead_umma_kernel<1><<<n_cta, kUmmaThreads, smem, st>>>(tm_h, tm_w, p, n_stages);
+      le = launch_overlapped(lmhead_umma_kernel<1>, dim3(n_cta), dim3(kUmmaThreads), smem, st, tm_h, tm_w, p, n_stages);
     else
-      lmhead_umma_kernel<2><<<n_cta, kUmmaThreads, smem, st>>>(tm_h, tm_w, p, n_stages);
+      le = launch_overlapped(lmhead_umma_kernel<2>, dim3(n_cta), dim3(kUmmaThreads), smem, st, tm_h, tm_w, p, n_stages);
   } else {
     const int tiles_total = (c.vocab + kMmaBN - 1) / kMmaBN;
     int n_cta = ctx->sm_count * 2;
@@ -548,21 +560,22 @@ static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden,
     if (n_cta > max_stripes) n_cta = max_stripes;
     p.n_stripes = n_cta;
     dim3 grid(n_cta, (rows + kMmaBM - 1) / kMmaBM);
-    lmhead_mma_kernel<<<grid, kMmaThreads, kMmaStages * kMmaStageBytes + 128, st>>>(p);
+    le = launch_overlapped(lmhead_mma_kernel, grid, dim3(kMmaThreads), (size_t)(kMmaStages * kMmaStageBytes + 128), st, p);
   }
   ctx->launches++;
-  if (cudaGetLastError() != cudaSuccess) return SDLM_ERR_CUDA;
-  lmhead_combine_kernel<<<(rows + 3) / 4, 128, 0, st>>>(p.partials, p.n_stripes, p.rows_pad, rows, token, p_top1,
-                                                       entropy, max_logit, lse);
+  if (le != cudaSuccess || cudaGetLastError() != cudaSuccess) return SDLM_ERR_CUDA;
+  le = launch_overlapped(lmhead_combine_kernel, dim3((rows + 3) / 4), dim3(128), 0, st, (const float4*)p.partials,
+                         p.n_stripes, p.rows_pad, rows, token, p_top1, entropy, max_logit, lse);
   ctx->launches++;
-  return cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+  return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
 }
 
 sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
-                          float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st) {
+                          float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st,
+                          bool independent_of_predecessor) {
   return launch_lmhead_on(ctx, rows, hidden, w_lm, token, p_top1, entropy, max_logit, lse, st,
                           reinterpret_cast<float4*>(ctx->ws + ctx->lay.lm_partials),
-                          ctx->cfg.max_batch * ctx->cfg.max_block, kLmMaxStripes);
+                          ctx->cfg.max_batch * ctx->cfg.max_block, kLmMaxStripes, independent_of_predecessor);
 }
 
 }  // namespace sdlm
@@ -613,5 +626,5 @@ extern "C" sdlm_status sdlm_lmhead_confidence_static(sdlm_ctx* ctx, int32_t rows
   sdlm_status s = static_partials_for_current_device(device, &partials);
   if (s != SDLM_OK) return s;
   return sdlm::launch_lmhead_on(ctx, rows, hidden, w_lm, token, p_top1, entropy, max_logit, lse,
-                                static_cast<cudaStream_t>(stream), partials, kStaticMaxRows, kStaticMaxStripes);
+                                static_cast<cudaStream_t>(stream), partials, kStaticMaxRows, kStaticMaxStripes, false);
 }

@@ -82,10 +82,14 @@ class DeviceProblem:
                            torch.empty((B, D), dtype=torch.int32, device=dev))
 
     def step(self, x: DeviceBlock, tau: float, out: Optional[StepOutputs] = None, mode: int = CONF_LOGIT,
-             stream=None) -> StepOutputs:
+             stream=None, fused: bool = False) -> StepOutputs:
         """(a) + (b) + (c) on device-resident inputs: three library calls, no host synchronisation."""
         out = out or self.alloc_outputs()
         sd = self.sd
+        if fused:
+            sd.decode_step(tau, x.q, x.k_blk, x.v_blk, x.hidden, self.w_lm, out.attn, out.token, out.p_top1, out.entropy,
+                           out.accepted_len, out.out_tokens, mode=mode, stream=stream)
+            return out
         sd.block_attn(x.q, x.k_blk, x.v_blk, out.attn, stream=stream)
         sd.lmhead_confidence(x.hidden, self.w_lm, out.token, out.p_top1, out.entropy, stream=stream)
         sd.accept_commit(tau, out.token, out.p_top1, out.entropy, x.k_blk, x.v_blk, mode, out.accepted_len,

@@ -41,6 +41,12 @@ def test_add_gather_release_match_oracle(shape):
     dp.sd.kv_add_seq(2, pk.bf16_tensor_from_bits(k), pk.bf16_tensor_from_bits(v))
     cache.add_sequence_fast(2, k, v)
     _tables_equal(dp, cache)
+    # device-side save / restore of the tables, no host round trip
+    saved = dp.sd.kv_save()
+    dp.sd.kv_release_seq(1)
+    assert dp.sd.kv_tables()["seq_len"][1] == 0
+    dp.sd.kv_restore(saved)
+    _tables_equal(dp, cache)
     # export / reset / import restores the tables
     snap = dp.sd.kv_export()
     dp.sd.kv_reset()

@@ -11,6 +11,7 @@ import torch
 
 import paper_2509_24007_b200 as pk
 from paper_2509_24007_b200.harness import DeviceProblem
+from paper_2509_24007_b200.binding import OPT_STEP_OVERLAP
 from oracle import sdlm_oracle as orc
 import sdlm_synth as syn
 from oracle_side import (check_attention, check_confidences, check_gamma, check_tokens, oracle_cache)
@@ -173,3 +174,30 @@ def test_decode_step_host_entry_matches_device_calls():
     assert torch.equal(out_tok, ref.out_tokens.cpu())
     t = dp.sd.kv_tables()
     assert np.array_equal(t["page_table"], t_ref["page_table"]) and np.array_equal(t["seq_len"], t_ref["seq_len"])
+
+
+@pytest.mark.parametrize("name,batch", [("cfg0", 3), ("cfg2_d4", 6)])
+def test_decode_step_device_entry_matches_three_calls(name, batch):
+    """sdlm_decode_step lets attention and the LM head overlap on the GPU; results must not change."""
+    wl = syn.CONFIGS[name].with_(batch=batch, prefix_lo=10, prefix_hi=700)
+    dp = DeviceProblem(wl)
+    for step in range(4):
+        dp.sd.set_option(OPT_STEP_OVERLAP, step % 2)
+        x = dp.block(step)
+        snap = dp.sd.kv_export()
+        ref = dp.step(x, wl.tau)
+        torch.cuda.synchronize()
+        t_ref = dp.sd.kv_tables()
+        k_ref = [dp.sd.kv_gather(b, int(t_ref["seq_len"][b])) for b in range(batch)]
+        dp.sd.kv_import(snap)                       # same starting tables for the fused call
+        out = dp.step(x, wl.tau, fused=True)
+        torch.cuda.synchronize()
+        assert dp.sd.device_status()[0] == 0
+        for a, b_ in zip((out.attn, out.token, out.p_top1, out.entropy, out.accepted_len, out.out_tokens),
+                         (ref.attn, ref.token, ref.p_top1, ref.entropy, ref.accepted_len, ref.out_tokens)):
+            assert torch.equal(a, b_)
+        t = dp.sd.kv_tables()
+        assert np.array_equal(t["page_table"], t_ref["page_table"]) and np.array_equal(t["seq_len"], t_ref["seq_len"])
+        for b in range(batch):
+            k, v = dp.sd.kv_gather(b, int(t["seq_len"][b]))
+            assert torch.equal(k, k_ref[b][0]) and torch.equal(v, k_ref[b][1])
