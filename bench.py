@@ -335,11 +335,11 @@ def main():
             line["extra"] = {wl8.name: {"value": r8["tokens"] / (r8["ms_total"] * 1e-3), "unit": UNIT,
                                         "ms_per_step": r8["ms_per_step"], "lm_ms": r8["lm_ms"], "attn_ms": r8["attn_ms"]}}
             del dp8
-        n_seqs = min(wl.batch, 4)
-        tok, dt = oracle_sample(wl, n_seqs)
+        n_seqs = min(wl.batch, 32)
+        tok, dt = oracle_sample(wl, n_seqs, repeats=2)
         line["cpu_baseline"] = {"value": tok / dt, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
                                 "sample": f"oracle decode_step on the first {n_seqs} of {wl.batch} sequences "
-                                          f"({n_seqs * wl.block} rows; {dt:.1f} s), fp64 numpy"}
+                                          f"({n_seqs * wl.block} rows; best of 2 runs, {dt:.1f} s each), fp64 numpy"}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
