@@ -414,6 +414,7 @@ extern "C" sdlm_status sdlm_create(const sdlm_config* cfg, void* kv_pool, size_t
   ctx->launches = 0;
   ctx->lmhead_path = 0;
   ctx->overlap_lmhead = 0;
+  ctx->attn_item_cost = 12;
   ctx->tmap_w_ptr = nullptr;
   ctx->tmap_w_rows = 0;
   if (setup_attn(ctx) != cudaSuccess || setup_lmhead(ctx) != cudaSuccess) { delete ctx; return SDLM_ERR_CUDA; }
@@ -432,6 +433,10 @@ extern "C" sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t v
     case SDLM_OPT_LMHEAD_KERNEL:
       if (value < 0 || value > 2) return SDLM_ERR_INVALID_ARG;
       ctx->lmhead_path = value;
+      return SDLM_OK;
+    case SDLM_OPT_ATTN_ITEM_COST:
+      if (value < 0 || value > 64) return SDLM_ERR_INVALID_ARG;
+      ctx->attn_item_cost = value;
       return SDLM_OK;
     case SDLM_OPT_STEP_OVERLAP:
       if (value < 0 || value > 1) return SDLM_ERR_INVALID_ARG;

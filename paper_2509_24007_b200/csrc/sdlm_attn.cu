@@ -46,6 +46,7 @@ struct AttnParams {
   DevHeader* hdr;
   float scale_log2;  // softmax scale * log2(e)
   int batch, D, Hq, Hkv, G, mpps, num_pages, n_stages;
+  int item_cost;  // what starting a (sequence, KV head) pair costs a CTA, in tiles (see ItemWalk)
 };
 
 constexpr int kAttnThreads = 256;
@@ -71,16 +72,19 @@ struct Item {
   int pair, c_first, n_splits;
 };
 
+// The sequence that is cut into equal ranges is not the bare tile sequence: every pair is preceded
+// by `item_cost` positions that stand for the fixed work of an item (reference set-up, epilogue,
+// partial results).  A range that contains the start of a pair therefore gets fewer real tiles.
 struct ItemWalk {
-  const int* s_first;  // [batch + 1] exclusive prefix sum of (pages + 1) per batch row
+  const int* s_first;  // [batch + 1] exclusive prefix sum of (item_cost + pages + 1) per batch row
   const int* s_len;    // [batch] cached tokens per batch row
   const int* s_slot;   // [batch] sequence slot per batch row
-  uint32_t total;      // tiles in the whole launch (the host keeps total * gridDim below 2^31)
+  uint32_t total;      // positions in the whole launch (the host keeps total * gridDim below 2^31)
   uint32_t cur, hi;
   uint32_t nc;
 };
 
-__device__ __forceinline__ int tile_owner(uint32_t x, uint32_t total, uint32_t nc) {
+__device__ __forceinline__ int pos_owner(uint32_t x, uint32_t total, uint32_t nc) {
   return (int)(((x + 1) * nc - 1) / total);  // the CTA c with floor(c*total/nc) <= x < floor((c+1)*total/nc)
 }
 
@@ -89,8 +93,7 @@ __device__ __forceinline__ void walk_begin(ItemWalk& w, const int* s_first, int 
   w.s_len = s_first + batch + 1;
   w.s_slot = w.s_len + batch;
   w.total = (uint32_t)s_first[batch] * (uint32_t)Hkv;
-  // never more ranges than tiles: every range is then non-empty and the CTAs that share a pair
-  // are consecutive
+  // never more ranges than positions: every range is then non-empty
   w.nc = min(gridDim.x, w.total);
   if (blockIdx.x >= w.nc) {
     w.cur = w.hi = 0;
@@ -101,28 +104,34 @@ __device__ __forceinline__ void walk_begin(ItemWalk& w, const int* s_first, int 
 }
 
 __device__ __forceinline__ bool walk_next(ItemWalk& w, const AttnParams& p, Item& it) {
-  if (w.cur >= w.hi) return false;
-  int lo = 0, hi = p.batch - 1;
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) >> 1;
-    if ((uint32_t)w.s_first[mid] * (uint32_t)p.Hkv <= w.cur) lo = mid; else hi = mid - 1;
+  const uint32_t cost = (uint32_t)p.item_cost;
+  while (w.cur < w.hi) {
+    int lo = 0, hi = p.batch - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if ((uint32_t)w.s_first[mid] * (uint32_t)p.Hkv <= w.cur) lo = mid; else hi = mid - 1;
+    }
+    const uint32_t span = (uint32_t)(w.s_first[lo + 1] - w.s_first[lo]);  // cost + tiles of one pair
+    const uint32_t row_start = (uint32_t)w.s_first[lo] * (uint32_t)p.Hkv;
+    const uint32_t h = (w.cur - row_start) / span;
+    const uint32_t pair_start = row_start + h * span;
+    const uint32_t a0 = w.cur - pair_start, a1 = min(w.hi, pair_start + span) - pair_start;
+    w.cur = pair_start + a1;
+    if (a1 <= cost) continue;  // only the fixed-cost positions of this pair fall into the range
+    it.b = lo;
+    it.h = (int)h;
+    it.t0 = (int)(max(a0, cost) - cost);
+    it.t1 = (int)(a1 - cost);
+    it.pages = (int)(span - cost) - 1;
+    it.slot = w.s_slot[lo];
+    it.len = w.s_len[lo];
+    it.pair = lo * p.Hkv + it.h;
+    // the CTAs that hold real tiles of this pair are consecutive
+    it.c_first = pos_owner(pair_start + cost, w.total, w.nc);
+    it.n_splits = pos_owner(pair_start + span - 1, w.total, w.nc) - it.c_first + 1;
+    return true;
   }
-  it.b = lo;
-  const uint32_t tiles_b = (uint32_t)(w.s_first[lo + 1] - w.s_first[lo]);
-  const uint32_t row_start = (uint32_t)w.s_first[lo] * (uint32_t)p.Hkv;
-  it.h = (int)((w.cur - row_start) / tiles_b);
-  const uint32_t pair_start = row_start + (uint32_t)it.h * tiles_b;
-  it.t0 = (int)(w.cur - pair_start);
-  const uint32_t end = min(w.hi, pair_start + tiles_b);
-  it.t1 = (int)(end - pair_start);
-  it.pages = (int)tiles_b - 1;
-  it.slot = w.s_slot[lo];
-  it.len = w.s_len[lo];
-  it.pair = lo * p.Hkv + it.h;
-  it.c_first = tile_owner(pair_start, w.total, w.nc);
-  it.n_splits = tile_owner(pair_start + tiles_b - 1, w.total, w.nc) - it.c_first + 1;
-  w.cur = end;
-  return true;
+  return false;
 }
 
 // Ring position of the n-th tile this CTA pushes through its stages.
@@ -215,7 +224,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
         const int len = attn_len(p, i);
         s_first[p.batch + 1 + i] = len;
         s_first[2 * p.batch + 1 + i] = attn_slot(p, i);
-        n = (len + kPageSize - 1) / kPageSize + 1;
+        n = (len + kPageSize - 1) / kPageSize + 1 + p.item_cost;
       }
       int incl = n;
       for (int o = 1; o < 32; o <<= 1) {
@@ -255,8 +264,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
   __syncthreads();
   {
     ItemWalk w0;
+    Item i0;
     walk_begin(w0, s_first, p.batch, p.Hkv);
-    if (w0.cur >= w0.hi) return;  // nothing falls into this CTA's range (uniform for the CTA)
+    if (!walk_next(w0, p, i0)) return;  // no tile falls into this CTA's range (uniform for the CTA)
   }
   if (warp == 1) {
     ptx::tmem_alloc(tmem_slot, TMEM_COLS);
@@ -816,8 +826,10 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
   p.scale_log2 = ctx->scale * 1.4426950408889634f;
   p.batch = batch; p.D = D; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.G = ctx->group;
   p.mpps = c.max_pages_per_seq; p.num_pages = c.num_pages; p.n_stages = 0;
+  p.item_cost = ctx->attn_item_cost;
   // the kernel's tile arithmetic is 32-bit: (tiles of the launch) x (CTAs) must stay below 2^31
-  if ((long long)batch * (c.max_pages_per_seq + 1) * c.n_kv_heads > 13000000ll) return cudaErrorInvalidConfiguration;
+  if ((long long)batch * (c.max_pages_per_seq + 1 + ctx->attn_item_cost) * c.n_kv_heads > 13000000ll)
+    return cudaErrorInvalidConfiguration;
   const bool wide = ctx->group * D > 32;  // stacked query rows padded to 64, else to 32
   if (c.head_dim == 128) return wide ? attn_launch_one<128, 64>(ctx, p, st) : attn_launch_one<128, 32>(ctx, p, st);
   return wide ? attn_launch_one<64, 64>(ctx, p, st) : attn_launch_one<64, 32>(ctx, p, st);

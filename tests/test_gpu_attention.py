@@ -100,6 +100,22 @@ def test_attention_with_scores_that_keep_outgrowing_the_row_reference(D):
     check_attention(pk.bits_from_bf16_tensor(out), ref)
 
 
+@pytest.mark.parametrize("cost", [0, 3, 17, 64])
+def test_attention_schedule_item_cost_does_not_change_results(cost):
+    from paper_2509_24007_b200.binding import OPT_ATTN_ITEM_COST
+    shape = syn.Shape(16, 2, 128, 64, 64)
+    lens = np.array([0, 1, 64, 700, 129, 2500, 63, 300, 5], dtype=np.int32)
+    wl = syn.Workload("attn_cost", shape, len(lens), 4, 0, 0, (0.9,), seed=37)
+    dp = DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16), lengths=lens)
+    dp.sd.set_option(OPT_ATTN_ITEM_COST, cost)
+    x = dp.block(0)
+    out = dp.sd.block_attn(x.q, x.k_blk, x.v_blk)
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+    pk_, pv_ = zip(*dp.prefix)
+    check_attention(pk.bits_from_bf16_tensor(out), orc.block_attention(x.host.q, x.host.k_blk, x.host.v_blk, pk_, pv_))
+
+
 def test_attention_rejects_bad_arguments():
     shape = syn.SHAPE_TINY
     wl = syn.Workload("attn_bad", shape, 2, 4, 8, 8, (0.9,), seed=35)
