@@ -264,25 +264,12 @@ __global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitPar
   }
   const int total_need = s_carry;
 
-  // all reads of the shared tables are done: take a ticket
+  // All reads of the shared tables are done: take a ticket.  Its value is only needed at the very
+  // end, so the round trip of the atomic overlaps this row's copies.
+  uint32_t ticket = 0;
   if (tid == 0) {
     __threadfence();
-    const uint32_t t = atomicAdd(&p.hdr->commit_ticket, 1u);
-    s_last = (t == gridDim.x - 1);
-  }
-  __syncthreads();
-  if (s_last) {
-    __threadfence();
-    for (int i = tid; i < p.batch; i += kCommitThreads) {
-      if (s_state[i] == 0) {
-        const int slot = p.seq_ids ? p.seq_ids[i] : i;
-        p.seq_len[slot] += s_gamma[i];
-      }
-    }
-    if (tid == 0) {
-      p.hdr->free_head = s_head + min((uint32_t)total_need, avail);
-      p.hdr->commit_ticket = 0;
-    }
+    ticket = atomicAdd(&p.hdr->commit_ticket, 1u);
   }
 
   // my row
@@ -294,41 +281,58 @@ __global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitPar
       report_status(p.hdr, state == 1 ? SDLM_ERR_DEVICE_CHECK : SDLM_ERR_OUT_OF_PAGES, slot, len);
     }
     for (int k = tid; k < p.D; k += kCommitThreads) p.out_tokens[b * p.D + k] = -1;
-    return;
-  }
-  const int new_idx = (len + kPageSize - 1) / kPageSize;
-  int new_page = -1;
-  if (need) {
-    new_page = p.free_list[(s_head + (uint32_t)alloc) % (uint32_t)p.num_pages];
-    if (tid == 0) p.page_table[(size_t)slot * p.mpps + new_idx] = new_page;
-  }
-  if (tid == 0) p.accepted_len[b] = g;
-  for (int k = tid; k < p.D; k += kCommitThreads) p.out_tokens[b * p.D + k] = (k < g) ? p.token[b * p.D + k] : -1;
-  if (need) {  // a page fresh from the ring may hold anything: clear its V^T tiles first
-    const int per_head = kPageSize * p.d / 8;
-    for (int idx = tid; idx < p.Hkv * per_head; idx += kCommitThreads)
-      reinterpret_cast<uint4*>(p.pool + kv_tile_offset(new_page, idx / per_head, 1, p.Hkv, p.d))[idx % per_head] =
-          make_uint4(0, 0, 0, 0);
-    __syncthreads();
-  }
-  const int cpr = p.d / 8;
-  const int total = g * p.Hkv * cpr;
-  for (int idx = tid; idx < total; idx += kCommitThreads) {
-    const int c = idx % cpr;
-    int r = idx / cpr;
-    const int h = r % p.Hkv;
-    const int t = r / p.Hkv;
-    const int pos = len + t;
-    const int pidx = pos / kPageSize, key = pos % kPageSize;
-    const int page = (need && pidx == new_idx) ? new_page : p.page_table[(size_t)slot * p.mpps + pidx];
-    const size_t src = (((size_t)b * p.D + t) * p.Hkv + h) * p.d;
-    *reinterpret_cast<uint4*>(p.pool + kv_tile_offset(page, h, 0, p.Hkv, p.d) + k_tile_elem(key, c * 8)) =
-        *(reinterpret_cast<const uint4*>(p.k_blk + src) + c);
-    const uint4 vv = *(reinterpret_cast<const uint4*>(p.v_blk + src) + c);
-    const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(&vv);
-    __nv_bfloat16* v_tile = p.pool + kv_tile_offset(page, h, 1, p.Hkv, p.d);
+  } else {
+    const int new_idx = (len + kPageSize - 1) / kPageSize;
+    int new_page = -1;
+    if (need) {
+      new_page = p.free_list[(s_head + (uint32_t)alloc) % (uint32_t)p.num_pages];
+      if (tid == 0) p.page_table[(size_t)slot * p.mpps + new_idx] = new_page;
+    }
+    if (tid == 0) p.accepted_len[b] = g;
+    for (int k = tid; k < p.D; k += kCommitThreads) p.out_tokens[b * p.D + k] = (k < g) ? p.token[b * p.D + k] : -1;
+    if (need) {  // a page fresh from the ring may hold anything: clear its V^T tiles first
+      const int per_head = kPageSize * p.d / 8;
+      for (int idx = tid; idx < p.Hkv * per_head; idx += kCommitThreads)
+        reinterpret_cast<uint4*>(p.pool + kv_tile_offset(new_page, idx / per_head, 1, p.Hkv, p.d))[idx % per_head] =
+            make_uint4(0, 0, 0, 0);
+      __syncthreads();
+    }
+    const int cpr = p.d / 8;
+    const int total = g * p.Hkv * cpr;
+    for (int idx = tid; idx < total; idx += kCommitThreads) {
+      const int c = idx % cpr;
+      int r = idx / cpr;
+      const int h = r % p.Hkv;
+      const int t = r / p.Hkv;
+      const int pos = len + t;
+      const int pidx = pos / kPageSize, key = pos % kPageSize;
+      const int page = (need && pidx == new_idx) ? new_page : p.page_table[(size_t)slot * p.mpps + pidx];
+      const size_t src = (((size_t)b * p.D + t) * p.Hkv + h) * p.d;
+      *reinterpret_cast<uint4*>(p.pool + kv_tile_offset(page, h, 0, p.Hkv, p.d) + k_tile_elem(key, c * 8)) =
+          *(reinterpret_cast<const uint4*>(p.k_blk + src) + c);
+      const uint4 vv = *(reinterpret_cast<const uint4*>(p.v_blk + src) + c);
+      const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(&vv);
+      __nv_bfloat16* v_tile = p.pool + kv_tile_offset(page, h, 1, p.Hkv, p.d);
 #pragma unroll
-    for (int e = 0; e < 8; ++e) v_tile[vt_tile_elem(key, c * 8 + e)] = ve[e];
+      for (int e = 0; e < 8; ++e) v_tile[vt_tile_elem(key, c * 8 + e)] = ve[e];
+    }
+  }
+
+  // whichever CTA took the last ticket publishes the new lengths and the ring cursor
+  if (tid == 0) s_last = (ticket == gridDim.x - 1);
+  __syncthreads();
+  if (s_last) {
+    __threadfence();
+    for (int i = tid; i < p.batch; i += kCommitThreads) {
+      if (s_state[i] == 0) {
+        const int sl = p.seq_ids ? p.seq_ids[i] : i;
+        p.seq_len[sl] += s_gamma[i];
+      }
+    }
+    if (tid == 0) {
+      p.hdr->free_head = s_head + min((uint32_t)total_need, avail);
+      p.hdr->commit_ticket = 0;
+    }
   }
 }
 

@@ -211,6 +211,34 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int GD = p.G * p.D;
+  // set-up that touches no global memory runs while the kernel before this one drains
+  if (tid == 32) {
+    for (int s = 0; s < NS; ++s) {
+      ptx::mbar_init(&full[s], 2);  // the copies' issuer, plus whoever completes the group (see warp 0)
+      ptx::mbar_init(&stage_free[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      ptx::mbar_init(&s_full[s], 1);
+      ptx::mbar_init(&s_free[s], 4);
+      ptx::mbar_init(&p_full[s], 4);
+      ptx::mbar_init(&p_free[s], 1);
+    }
+    ptx::mbar_init(q_full, 1);
+    ptx::mbar_init(q_free, 1);
+    ptx::mbar_init(o_done, 1);
+    ptx::mbar_init(o_free, 4);
+    ptx::mbar_init(ep_bar, 4);
+    ptx::mbar_init(&drain[0], 1);
+    ptx::mbar_init(&drain[1], 1);
+    *abort = 0;
+    *blk_go = 0;
+    flag[0] = flag[1] = flag[2] = 0;
+    ptx::fence_barrier_init();
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
   ptx::grid_dep_wait();    // lengths, page table and pool are written by the kernels before this one
   ptx::grid_dep_launch();  // only now: a successor that does not wait itself may then rely on them too
 
@@ -238,43 +266,18 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
   }
   // stacked row r = j*G + g is q[b, j, h*G + g, :] (and the same row of out)
   if (tid >= 64 && tid < 128) row_off[tid - 64] = tid - 64 < GD ? (((tid - 64) / p.G) * p.Hq + (tid - 64) % p.G) * HD : -1;
-  if (tid == 32) {
-    for (int s = 0; s < NS; ++s) {
-      ptx::mbar_init(&full[s], 2);  // the copies' issuer, plus whoever completes the group (see warp 0)
-      ptx::mbar_init(&stage_free[s], 1);
-    }
-    for (int s = 0; s < 2; ++s) {
-      ptx::mbar_init(&s_full[s], 1);
-      ptx::mbar_init(&s_free[s], 4);
-      ptx::mbar_init(&p_full[s], 4);
-      ptx::mbar_init(&p_free[s], 1);
-    }
-    ptx::mbar_init(q_full, 1);
-    ptx::mbar_init(q_free, 1);
-    ptx::mbar_init(o_done, 1);
-    ptx::mbar_init(o_free, 4);
-    ptx::mbar_init(ep_bar, 4);
-    ptx::mbar_init(&drain[0], 1);
-    ptx::mbar_init(&drain[1], 1);
-    *abort = 0;
-    *blk_go = 0;
-    flag[0] = flag[1] = flag[2] = 0;
-    ptx::fence_barrier_init();
-  }
+  ptx::tc_fence_before();
   __syncthreads();
+  ptx::tc_fence_after();
   {
     ItemWalk w0;
     Item i0;
     walk_begin(w0, s_first, p.batch, p.Hkv);
-    if (!walk_next(w0, p, i0)) return;  // no tile falls into this CTA's range (uniform for the CTA)
+    if (!walk_next(w0, p, i0)) {  // no tile falls into this CTA's range (uniform for the CTA)
+      if (warp == 1) ptx::tmem_dealloc(*tmem_slot, TMEM_COLS);
+      return;
+    }
   }
-  if (warp == 1) {
-    ptx::tmem_alloc(tmem_slot, TMEM_COLS);
-    ptx::tmem_relinquish();
-  }
-  ptx::tc_fence_before();
-  __syncthreads();
-  ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {

@@ -441,9 +441,14 @@ __global__ void __launch_bounds__(128) lmhead_combine_kernel(const float4* parti
   ptx::grid_dep_wait();  // the partials come from the stripe kernel
   if (row >= rows) return;
   Stat st = stat_empty();
-  for (int s = lane; s < n_stripes; s += 32) {
-    const float4 v = partials[(size_t)s * rows_pad + row];
-    st = stat_merge(st, Stat{v.x, v.y, v.z, __float_as_int(v.w)});
+  for (int s0 = lane; s0 < n_stripes; s0 += 32 * 8) {  // eight loads in flight, merged in index order
+    float4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      if (s0 + 32 * u < n_stripes) v[u] = __ldcg(partials + (size_t)(s0 + 32 * u) * rows_pad + row);
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      if (s0 + 32 * u < n_stripes) st = stat_merge(st, Stat{v[u].x, v[u].y, v[u].z, __float_as_int(v[u].w)});
   }
 #pragma unroll
   for (int o = 16; o; o >>= 1) {
