@@ -91,7 +91,7 @@ def _blas_threads() -> int:
         return os.cpu_count() or 1
 
 
-def oracle_sample(wl: syn.Workload, n_seqs: int, w_bits=None, repeats: int = 1):
+def oracle_sample(wl: syn.Workload, n_seqs: int, w_bits=None, repeats: int = 1, w64=None):
     """Times the CPU oracle (as it stands) on the first n_seqs sequences of the workload's step."""
     from oracle import sdlm_oracle as orc
     sub = wl.with_(batch=n_seqs)
@@ -108,28 +108,36 @@ def oracle_sample(wl: syn.Workload, n_seqs: int, w_bits=None, repeats: int = 1):
         for b in range(n_seqs):
             cache.add_sequence_fast(b, *prefix[b])
         t0 = time.perf_counter()
-        res = orc.decode_step(cache, range(n_seqs), x.q, x.k_blk, x.v_blk, x.hidden, w_bits, wl.tau)
+        res = orc.decode_step(cache, range(n_seqs), x.q, x.k_blk, x.v_blk, x.hidden, w_bits, wl.tau, w64=w64)
         dt = time.perf_counter() - t0
         tokens = int(res.commit.accepted_len.sum())
         best = dt if best is None else min(best, dt)
     return tokens, best
 
 
+REFERENCE_BUDGET_S = 150.0   # the reference arm sizes its per-step sample so that the run ends within this
+
+
 def run_reference(args, wl: syn.Workload):
-    """The reference arm: the CPU oracle timed on host cores, a bounded sample per step."""
+    """The reference arm: the CPU oracle timed on host cores, a bounded sample of the workload per step."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    n_seqs = min(wl.batch, 4)
+    from oracle import sdlm_oracle as orc
     w_bits = syn.lm_head_weight(wl)
+    w64 = orc.widen(w_bits)                      # the weight in the oracle's own precision, prepared once (untimed)
+    _, t1 = oracle_sample(wl, 1, w_bits, w64=w64)   # calibration: one sequence per step
+    per_step = REFERENCE_BUDGET_S / max(1, args.steps + args.warmup)
+    n_seqs = int(max(1, min(wl.batch, 4, per_step // max(t1, 1e-3))))
     times, tokens = [], 0
     for i in range(args.warmup + args.steps):
-        tok, dt = oracle_sample(wl, n_seqs, w_bits)
+        tok, dt = oracle_sample(wl, n_seqs, w_bits, w64=w64)
         if i >= args.warmup:
             times.append(dt); tokens += tok
     total = sum(times)
     value = tokens / total
-    sample = f"oracle decode_step on the first {n_seqs} of {wl.batch} sequences ({n_seqs * wl.block} rows), fp64 numpy"
+    sample = (f"oracle decode_step on the first {n_seqs} of {wl.batch} sequences ({n_seqs * wl.block} rows) per step, "
+              f"fp64 numpy, LM-head weight widened to fp64 once beforehand")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / max(1, args.steps),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
