@@ -53,6 +53,7 @@ struct LmParams {
   DevHeader* hdr;
   int rows, H, V, n_stripes, rows_pad;
   int bn;  // umma path: vocab rows per tile (multiple of 16, <= 256)
+  int a_box_rows;   // umma path: hidden-state rows one TMA box brings in (<= 128; rows beyond it are never read back)
   int wait_at_end;  // 1: no input comes from the kernel before this one; only completion order is kept
 };
 
@@ -191,7 +192,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
             break;
           }
           uint8_t* st = smem + (size_t)s * stage_bytes;
-          ptx::mbar_arrive_expect_tx(&full[s], (uint32_t)stage_bytes);
+          ptx::mbar_arrive_expect_tx(&full[s], (uint32_t)(R * p.a_box_rows * kBK * 2 + w_tile_bytes));
 #pragma unroll
           for (int r = 0; r < R; ++r) ptx::tma_load_2d(st + r * kATileBytes, &tmap_h, kc * kBK, r * 128, &full[s]);
           ptx::tma_load_2d(st + R * kATileBytes, &tmap_w, kc * kBK, n0, &full[s]);
@@ -527,6 +528,7 @@ static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden,
   p.rows = rows; p.H = c.hidden; p.V = c.vocab;
   p.rows_pad = rows_pad;
   p.bn = 0;
+  p.a_box_rows = 128;
   p.wait_at_end = independent ? 1 : 0;
   cudaError_t le = cudaSuccess;
 
@@ -546,7 +548,10 @@ static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden,
     if (n_stages > 8) n_stages = 8;
     if (n_stages < 2) return SDLM_ERR_UNSUPPORTED;
     CUtensorMap tm_h;
-    if (!make_tmap(&tm_h, hidden, rows, c.hidden, 128)) return SDLM_ERR_CUDA;
+    // With few rows the box only covers them (rounded up to the 8-row swizzle group): the other
+    // accumulator lanes then compute on whatever the stage held before, and are never read back.
+    p.a_box_rows = R == 1 ? ((rows + 7) / 8 * 8 < 128 ? (rows + 7) / 8 * 8 : 128) : 128;
+    if (!make_tmap(&tm_h, hidden, rows, c.hidden, p.a_box_rows)) return SDLM_ERR_CUDA;
     if (ctx->tmap_w_ptr != w_lm || ctx->tmap_w_rows != p.bn) {
       if (!make_tmap(reinterpret_cast<CUtensorMap*>(ctx->tmap_w), w_lm, c.vocab, c.hidden, p.bn)) return SDLM_ERR_CUDA;
       ctx->tmap_w_ptr = w_lm;
