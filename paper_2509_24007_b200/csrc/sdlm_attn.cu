@@ -176,13 +176,15 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
   constexpr int Q_PANEL_B = NQ * 128;
   constexpr int P_PANEL_B = NQ * 128;             // P^T of one tile: NQ rows x 64 keys
   constexpr int P_BUF_B = 2 * P_PANEL_B;
+  // two P^T buffers, except where a third two-tile ring stage is worth more than the second buffer
+  constexpr int PB = (HD == 128 && NQ == 64) ? 1 : 2;
   constexpr uint32_t O_COL = 128, TMEM_COLS = 256;  // S^T buffers at columns 0 and NQ
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* q_s = smem;
   uint8_t* p_s = q_s + KH * Q_PANEL_B;
-  uint8_t* stages = p_s + 2 * P_BUF_B;
+  uint8_t* stages = p_s + PB * P_BUF_B;
   const int NS = p.n_stages;
   uint64_t* full = reinterpret_cast<uint64_t*>(stages + (size_t)NS * PAIR_B);
   uint64_t* stage_free = full + NS;
@@ -202,11 +204,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
   volatile int* blk_go = abort + 2;     // warp 0 -> warp 6: block-tile ring slots that are free so far
   volatile int* flag = abort + 3;       // [3] "some score outgrew its reference", by group mod 3
   float* mref = reinterpret_cast<float*>(const_cast<int*>(abort) + 7);  // [64] row references (log2 units); 16-byte aligned
-  float* mnew = mref + 64;              // [64]
-  float* fbuf = mnew + 64;              // [64] rescale factors of a reference move
-  int* mx = reinterpret_cast<int*>(fbuf + 64);                          // [4][64] per-warp row maxima
-  float* lsum = reinterpret_cast<float*>(mx + 256);                     // [2][4][64] per-warp row sums, by item parity
-  int* row_off = reinterpret_cast<int*>(lsum + 512);  // [64] element offset of stacked row r inside a (b, KV head) slab
+  float* fbuf = mref + 64;              // [64] rescale factors of a reference move; 1 / row sum in a merge
+  int* row_off = reinterpret_cast<int*>(fbuf + 64);  // [64] element offset of stacked row r inside a (b, KV head) slab
+  // Scratch that is only needed while no O^T instruction can be reading P^T (a reference move waits
+  // for the previous one, the end of an item for the last one) lives in the P^T buffers:
+  float* mnew = reinterpret_cast<float*>(p_s);   // [64] references after a move
+  int* mx = reinterpret_cast<int*>(p_s) + 64;    // [4][64] per-warp row maxima
+  float* lsum = reinterpret_cast<float*>(p_s) + 320;  // [4][64] per-warp row sums
   int* s_first = row_off + 64;                         // [batch + 1], then lengths [batch], then slots [batch]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -396,8 +400,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
       while (ok && walk_next(w, p, it)) {
         const int n = it.t1 - it.t0, ng = (n + 1) / 2;
         for (int g = 0; g < ng; ++g) {
-          const uint32_t pb = gc & 1u;
-          if (!ptx::mbar_wait(&p_full[pb], (gc >> 1) & 1u, abort)) { ok = false; break; }
+          const uint32_t pb = gc % PB;
+          if (!ptx::mbar_wait(&p_full[pb], (gc / PB) & 1u, abort)) { ok = false; break; }
           // the first instruction of an item overwrites O^T: the previous item's must have been read out
           if (g == 0 && item_idx > 0 && !ptx::mbar_wait(o_free, (item_idx - 1) & 1u, abort)) { ok = false; break; }
           ptx::tc_fence_after();
@@ -485,7 +489,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
           moved = flag[fi] != 0;
         }
         if (moved) {
-          // ---- move the row references to max(old reference, this group's row maxima)
+          // ---- move the row references to max(old reference, this group's row maxima).  The scratch
+          // for this sits in the P^T buffers and O^T is about to be rescaled: the previous O^T
+          // instruction must be done (for the first group of an item the previous item's end saw to it).
+          if (!first) {
+            const uint32_t prev = gc - 1;
+            if (!__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[prev % PB], (prev / PB) & 1u, abort))) { ok = false; break; }
+          }
 #pragma unroll
           for (int q = 0; q < NQ; ++q) {
             const int v = __reduce_max_sync(0xffffffffu, mine ? ordered_int(x[q] * p.scale_log2) : kIntMin);
@@ -504,10 +514,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
           }
           if (!meet()) { ok = false; break; }  // everybody has read the old references
           if (kg < NQ) mref[kg] = mnew[kg];
-          if (!first) {
-            // O^T holds sums relative to the old references; the previous O^T instruction must be done
-            const uint32_t prev = gc - 1;
-            if (!__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[prev & 1u], (prev >> 1) & 1u, abort))) { ok = false; break; }
+          if (!first) {  // O^T holds sums relative to the old references
             ptx::tc_fence_after();
 #pragma unroll
             for (int c = 0; c < NQ / 16; ++c) {
@@ -531,8 +538,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
           }
         }
         // P^T column of my key: 2^(s*scale - reference), rounded to bf16; absent keys give 0
-        if (gc >= 2 && !__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[sb], ((gc >> 1) & 1u) ^ 1u, abort))) { ok = false; break; }
-        uint8_t* pcol = p_s + sb * P_BUF_B + tj * P_PANEL_B + (kt & 7) * 2;
+        const uint32_t pbuf = gc % PB;
+        if (gc >= (uint32_t)PB && !__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[pbuf], ((gc / PB) & 1u) ^ 1u, abort))) { ok = false; break; }
+        uint8_t* pcol = p_s + pbuf * P_BUF_B + tj * P_PANEL_B + (kt & 7) * 2;
 #pragma unroll
         for (int q = 0; q < NQ; ++q) {
           e[q] = mine ? ptx::ex2(e[q]) : 0.f;
@@ -544,12 +552,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
         ptx::fence_proxy_async();
         ptx::tc_fence_before();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&p_full[sb]);
+        if (lane == 0) ptx::mbar_arrive(&p_full[pbuf]);
       }
       if (!ok) break;
 
       // ---- end of item: row sums over all keys (lane q of each warp ends up with the warp's sum of row q)
-      float* ls = lsum + (item_idx & 1u) * 256;
+      float* ls = lsum;
+      float lwarp[NQ / 32];
 #pragma unroll
       for (int half = 0; half < NQ / 32; ++half) {
         float* v = &l[half * 32];
@@ -562,11 +571,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
             v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
           }
         }
-        ls[qd * 64 + half * 32 + lane] = v[0];
+        lwarp[half] = v[0];
       }
-      if (!meet()) { ok = false; break; }
+      // the last O^T instruction of the item is done: O^T is complete and the P^T buffers are idle
       if (!__all_sync(0xffffffffu, ptx::mbar_wait(o_done, item_idx & 1u, abort))) { ok = false; break; }
       ptx::tc_fence_after();
+#pragma unroll
+      for (int half = 0; half < NQ / 32; ++half) ls[qd * 64 + half * 32 + lane] = lwarp[half];
+      if (!meet()) { ok = false; break; }
       float o[NQ];  // O^T row d = kg: one value per query row
 #pragma unroll
       for (int c = 0; c < NQ / 16; ++c)
@@ -613,7 +625,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
           // split s is 2^(m_s - m) with m = max_s m_s; the weights go through the (now idle) P^T
           // buffers, every thread sums four output columns, and the row sum L divides at the end.
           __threadfence();
-          constexpr int kCap = 128;  // splits whose weights fit into the P^T buffers at once
+          constexpr int kCap = PB * P_BUF_B / 4 / NQ;  // splits whose weights fit into the P^T buffers at once
           float* wbuf = reinterpret_cast<float*>(p_s);
           const size_t first_row = (size_t)(it.c_first + it.pair) * NQ;
           float m = -INFINITY, L = 0.f;
@@ -776,9 +788,10 @@ constexpr int kAttnSmemLimit = 232448;  // largest dynamic shared memory of one 
 
 template <int HD, int NQ>
 static int attn_fixed_smem(int batch) {
-  // alignment slack, Q, two P^T buffers, 15 barriers, flags, row scratch, prefix sums; for d = 64 the
+  // alignment slack, Q, the P^T buffers, 16 barrier slots, flags, row scratch, prefix sums; for d = 64 the
   // M = 128 O^T instruction reads 64 rows past the last V^T tile, which must still be shared memory
-  return 1024 + (HD / 64) * NQ * 128 + 4 * NQ * 128 + 16 * 8 + 32 + 960 * 4 + 64 * 4 + (batch + 1) * 12 + 64 +
+  const int p_buffers = (HD == 128 && NQ == 64) ? 1 : 2;
+  return 1024 + (HD / 64) * NQ * 128 + p_buffers * 2 * NQ * 128 + 16 * 8 + 32 + 3 * 64 * 4 + (batch + 1) * 12 + 64 +
          (HD == 64 ? 8192 : 0);
 }
 
