@@ -247,6 +247,20 @@ def time_e2e(torch, dp, wl, steps, warmup, n_blocks=4):
             "ms_per_step": 1e3 * dt / steps}
 
 
+def aggregate_over_ranks(dist, torch, ms_total, tokens, e2e_value, device):
+    """Whole-job figures from per-rank ones: every rank ran its own replica of the workload, so the
+    job's time is the slowest rank's and its tokens (and end-to-end rate) are the sum over ranks."""
+    if dist is None:
+        return ms_total, tokens, e2e_value
+    t = torch.tensor([ms_total], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    n = torch.tensor([tokens], dtype=torch.int64, device=device)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    e = torch.tensor([e2e_value], dtype=torch.float64, device=device)
+    dist.all_reduce(e, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(n.item()), float(e.item())
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -291,19 +305,8 @@ def main():
     res = time_workload(torch, dp, wl_run, args.steps, args.warmup)
     barrier()
     clocks = sampler.stop() if rank == 0 else None
-    ms_total, tokens = res["ms_total"], res["tokens"]
-    if dist is not None:
-        t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-        n = torch.tensor([tokens], dtype=torch.int64, device="cuda")
-        dist.all_reduce(n, op=dist.ReduceOp.SUM)
-        tokens = int(n.item())
     e2e = time_e2e(torch, dp, wl_run, max(3, min(args.steps, 100)), 3)
-    if dist is not None:
-        t = torch.tensor([e2e["value"]], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.SUM)
-        e2e["value"] = float(t.item())
+    ms_total, tokens, e2e["value"] = aggregate_over_ranks(dist, torch, res["ms_total"], res["tokens"], e2e["value"], "cuda")
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()

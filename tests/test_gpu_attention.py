@@ -116,6 +116,16 @@ def test_attention_schedule_item_cost_does_not_change_results(cost):
     check_attention(pk.bits_from_bf16_tensor(out), orc.block_attention(x.host.q, x.host.k_blk, x.host.v_blk, pk_, pv_))
 
 
+def test_attention_many_short_sequences_many_items_per_thread_block():
+    """600 sequences, most of them shorter than a page: more (sequence, head) pairs than thread blocks,
+    several items per thread block, a long prefix-sum table in shared memory."""
+    shape = syn.Shape(4, 2, 64, 64, 64)
+    rng = np.random.default_rng(7)
+    lens = rng.integers(0, 200, size=600).astype(np.int32)
+    lens[::37] = 0
+    _attn_case(shape, lens, 2, seed=38)
+
+
 def test_attention_rejects_bad_arguments():
     shape = syn.SHAPE_TINY
     wl = syn.Workload("attn_bad", shape, 2, 4, 8, 8, (0.9,), seed=35)

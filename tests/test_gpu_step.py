@@ -201,3 +201,14 @@ def test_decode_step_device_entry_matches_three_calls(name, batch):
         for b in range(batch):
             k, v = dp.sd.kv_gather(b, int(t["seq_len"][b]))
             assert torch.equal(k, k_ref[b][0]) and torch.equal(v, k_ref[b][1])
+
+
+def test_block_size_one_is_next_token_decode_on_the_gpu():
+    """D = 1: every sequence commits exactly one token whatever tau is, and the step equals the oracle's."""
+    wl = syn.CONFIGS["cfg0"].with_(batch=5, block=1, prefix_lo=0, prefix_hi=300)
+    dp = DeviceProblem(wl)
+    cache = oracle_cache(wl, dp.lengths, dp.num_pages, dp.mpps, dp.prefix)
+    for step, tau in enumerate((0.9, 0.0, 1.5)):
+        out, stats, res, n_bad = _one_step(dp, cache, tau, step)
+        assert n_bad == 0 and out.accepted_len.cpu().tolist() == [1] * wl.batch
+        _compare_tables(dp, cache)
