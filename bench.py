@@ -160,6 +160,7 @@ def _config(wl: syn.Workload, lengths=None):
     return c
 
 
+LMHEAD_NCU_TRAFFIC = 635448832   # bytes per launch of lmhead_umma_kernel<1> at cfg2_d4 (ncu, see profiles/)
 RESTORE_EVERY = 8   # steps between restores of the cache tables, so that prefix lengths stay the workload's
 
 
@@ -329,7 +330,9 @@ def main():
         "roofline": {"bound": "hbm", "kernel": "lmhead_umma_kernel (sdlm_lmhead_confidence: stripe kernel + merge of the stripes)",
                      "timing": "CUDA events around the call on its stream, mean over a second pass of the timed steps",
                      "achieved": lm_gbs, "peak": peak, "unit": "GB/s", "frac": lm_gbs / peak,
-                     "peak_source": peak_src, "traffic": None, "algorithmic_bytes": lm_bytes,
+                     "peak_source": peak_src, "traffic": LMHEAD_NCU_TRAFFIC if wl.name == "cfg2_3b_b32_d4" else None,
+                     "traffic_source": "dram__bytes_read.sum + dram__bytes_write.sum of one launch, profiles/lmhead_umma_and_block_attn_umma__cfg2_d4.md",
+                     "algorithmic_bytes": lm_bytes,
                      "launch_ms": res["lm_ms"]},
         "step": {"algorithmic_bytes": step_bytes, "achieved_gbs": step_bytes / (ms_total / args.steps * 1e-3) / 1e9,
                  "frac_of_peak": step_bytes / (ms_total / args.steps * 1e-3) / 1e9 / peak,
