@@ -49,7 +49,8 @@ struct AttnParams {
   int item_cost;  // what starting a (sequence, KV head) pair costs a CTA, in tiles (see ItemWalk)
 };
 
-constexpr int kAttnThreads = 256;
+// 8 warps; 12 when 64 stacked query rows need a second set of softmax warps
+constexpr int attn_threads(int nq) { return nq == 64 ? 384 : 256; }
 constexpr float kRebaseThreshold = 32.0f;  // log2 units a score may exceed its row reference by
 
 __device__ __forceinline__ int attn_slot(const AttnParams& p, int i) { return p.seq_ids ? p.seq_ids[i] : i; }
@@ -166,7 +167,7 @@ __device__ __forceinline__ int tile_valid(const Item& it, int ti, int D) {
 }
 
 template <int HD, int NQ>
-__global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(const AttnParams p) {
   constexpr int KH = HD / 64;                 // 64-wide panels of K and of Q
   constexpr int K_PANEL_B = kPageSize * 128;  // one tile's panel: 64 keys x 128 bytes
   constexpr int VT_B = HD * 128;              // one tile's V^T: d rows x 128 bytes
@@ -223,15 +224,15 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
     }
     for (int s = 0; s < 2; ++s) {
       ptx::mbar_init(&s_full[s], 1);
-      ptx::mbar_init(&s_free[s], 4);
-      ptx::mbar_init(&p_full[s], 4);
+      ptx::mbar_init(&s_free[s], NQ / 8);  // one arrival per softmax warp
+      ptx::mbar_init(&p_full[s], NQ / 8);
       ptx::mbar_init(&p_free[s], 1);
     }
     ptx::mbar_init(q_full, 1);
     ptx::mbar_init(q_free, 1);
     ptx::mbar_init(o_done, 1);
-    ptx::mbar_init(o_free, 4);
-    ptx::mbar_init(ep_bar, 4);
+    ptx::mbar_init(o_free, NQ / 8);
+    ptx::mbar_init(ep_bar, NQ / 8);
     ptx::mbar_init(&drain[0], 1);
     ptx::mbar_init(&drain[1], 1);
     *abort = 0;
@@ -429,9 +430,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
       }
     }
     __syncwarp();
-  } else if (warp < 6) {
+  } else if (warp < 6 || warp >= 8) {
     // ---------------------------------------------------------------- softmax: thread = key of the group
-    const int qd = warp & 3;             // TMEM lane quarter of this warp
+    // Four warps cover the 128 keys of a group; with 64 stacked query rows a second set of four
+    // (warps 8..11) takes the upper 32 rows, so that no thread handles more than 32 values per group.
+    constexpr int QV = 32;                          // query rows (columns of S^T) per thread
+    const int qd = warp & 3;                        // TMEM lane quarter of this warp
+    const int qb = warp >= 8 ? 32 : 0;              // first query row of this warp's set
+    const int sw = (warp >= 8 ? 4 : 0) + qd;        // index among the softmax warps
     const int kg = qd * 32 + lane;       // key within the group = accumulator lane; also the d index at the end
     const int tj = kg >> 6, kt = kg & 63;  // tile of the group, key within that tile
     const uint32_t lane_addr = tmem_base + ((uint32_t)(qd * 32) << 16);
@@ -440,7 +446,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
     Item it;
     uint32_t gc = 0, item_idx = 0, ep_uses = 0;
     bool ok = true;
-    // all four softmax warps meet; false when a wait ran out
+    // all softmax warps meet; false when a wait ran out
     auto meet = [&]() -> bool {
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(ep_bar);
@@ -449,19 +455,19 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
       return r;
     };
     while (ok && walk_next(w, p, it)) {
-      float l[NQ];  // this key subset's share of every row sum
+      float l[QV];  // this key subset's share of every row sum
 #pragma unroll
-      for (int q = 0; q < NQ; ++q) l[q] = 0.f;
+      for (int q = 0; q < QV; ++q) l[q] = 0.f;
       const int n = it.t1 - it.t0, ng = (n + 1) / 2;
       for (int g = 0; g < ng; ++g, ++gc) {
         const uint32_t sb = gc & 1u;
         const bool mine = kt < tile_valid(it, it.t0 + 2 * g + tj, p.D);  // does my key exist?
         if (!__all_sync(0xffffffffu, ptx::mbar_wait(&s_full[sb], (gc >> 1) & 1u, abort))) { ok = false; break; }
         ptx::tc_fence_after();
-        float x[NQ];  // my key's score for every row, then its exponent relative to the row reference
+        float x[QV];  // my key's score for every row, then its exponent relative to the row reference
 #pragma unroll
-        for (int c = 0; c < NQ / 16; ++c)
-          ptx::tmem_ld16(lane_addr + sb * NQ + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&x[c * 16]));
+        for (int c = 0; c < QV / 16; ++c)
+          ptx::tmem_ld16(lane_addr + sb * NQ + qb + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&x[c * 16]));
         ptx::tmem_ld_wait();
         ptx::tc_fence_before();
         __syncwarp();
@@ -471,12 +477,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
         bool moved = first;  // the first group of an item always sets the references
         const uint32_t fi = gc % 3u;
         if (warp == 2 && lane == 0) flag[(fi + 1u) % 3u] = 0;  // last read two groups ago
-        float e[NQ];  // exponents of my key relative to the row references
+        float e[QV];  // exponents of my key relative to the row references
         if (!first) {
           float xm = -INFINITY;
 #pragma unroll
-          for (int q4 = 0; q4 < NQ; q4 += 4) {
-            const float4 mr = *reinterpret_cast<const float4*>(mref + q4);
+          for (int q4 = 0; q4 < QV; q4 += 4) {
+            const float4 mr = *reinterpret_cast<const float4*>(mref + qb + q4);
             e[q4] = fmaf(x[q4], p.scale_log2, -mr.x);
             e[q4 + 1] = fmaf(x[q4 + 1], p.scale_log2, -mr.y);
             e[q4 + 2] = fmaf(x[q4 + 2], p.scale_log2, -mr.z);
@@ -497,40 +503,40 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
             if (!__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[prev % PB], (prev / PB) & 1u, abort))) { ok = false; break; }
           }
 #pragma unroll
-          for (int q = 0; q < NQ; ++q) {
+          for (int q = 0; q < QV; ++q) {
             const int v = __reduce_max_sync(0xffffffffu, mine ? ordered_int(x[q] * p.scale_log2) : kIntMin);
-            if (lane == (q & 31)) mx[qd * 64 + q] = v;
+            if (lane == q) mx[qd * 64 + qb + q] = v;
           }
           if (!meet()) { ok = false; break; }
 #pragma unroll
-          for (int q = 0; q < NQ; ++q) {
-            const int gi = max(max(mx[q], mx[64 + q]), max(mx[128 + q], mx[192 + q]));
-            const float m_old = first ? -INFINITY : mref[q];
+          for (int q = 0; q < QV; ++q) {
+            const int gi = max(max(mx[qb + q], mx[64 + qb + q]), max(mx[128 + qb + q], mx[192 + qb + q]));
+            const float m_old = first ? -INFINITY : mref[qb + q];
             float m_new = gi == kIntMin ? m_old : fmaxf(m_old, ordered_float(gi));
             if (m_new == -INFINITY) m_new = 0.f;  // no key at all (cannot happen: every group has one)
             const float f = first ? 0.f : ptx::ex2(m_old - m_new);
             l[q] *= f;
-            if (kg == q) { mnew[q] = m_new; fbuf[q] = f; }
+            if (kg == q) { mnew[qb + q] = m_new; fbuf[qb + q] = f; }
           }
           if (!meet()) { ok = false; break; }  // everybody has read the old references
-          if (kg < NQ) mref[kg] = mnew[kg];
+          if (kg < QV) mref[qb + kg] = mnew[qb + kg];
           if (!first) {  // O^T holds sums relative to the old references
             ptx::tc_fence_after();
 #pragma unroll
-            for (int c = 0; c < NQ / 16; ++c) {
+            for (int c = 0; c < QV / 16; ++c) {
               uint32_t o[16];
-              ptx::tmem_ld16(lane_addr + O_COL + c * 16, o);
+              ptx::tmem_ld16(lane_addr + O_COL + qb + c * 16, o);
               ptx::tmem_ld_wait();
 #pragma unroll
-              for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * fbuf[c * 16 + i]);
-              ptx::tmem_st16(lane_addr + O_COL + c * 16, o);
+              for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * fbuf[qb + c * 16 + i]);
+              ptx::tmem_st16(lane_addr + O_COL + qb + c * 16, o);
             }
             ptx::tmem_st_wait();
           }
           if (!meet()) { ok = false; break; }  // the new references are visible
 #pragma unroll
-          for (int q4 = 0; q4 < NQ; q4 += 4) {
-            const float4 mr = *reinterpret_cast<const float4*>(mref + q4);
+          for (int q4 = 0; q4 < QV; q4 += 4) {
+            const float4 mr = *reinterpret_cast<const float4*>(mref + qb + q4);
             e[q4] = fmaf(x[q4], p.scale_log2, -mr.x);
             e[q4 + 1] = fmaf(x[q4 + 1], p.scale_log2, -mr.y);
             e[q4 + 2] = fmaf(x[q4 + 2], p.scale_log2, -mr.z);
@@ -542,13 +548,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
         if (gc >= (uint32_t)PB && !__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[pbuf], ((gc / PB) & 1u) ^ 1u, abort))) { ok = false; break; }
         uint8_t* pcol = p_s + pbuf * P_BUF_B + tj * P_PANEL_B + (kt & 7) * 2;
 #pragma unroll
-        for (int q = 0; q < NQ; ++q) {
+        for (int q = 0; q < QV; ++q) {
           e[q] = mine ? ptx::ex2(e[q]) : 0.f;
           l[q] += e[q];
         }
 #pragma unroll
-        for (int q = 0; q < NQ; ++q)
-          *reinterpret_cast<__nv_bfloat16*>(pcol + q * 128 + (((kt >> 3) ^ (q & 7)) << 4)) = __float2bfloat16_rn(e[q]);
+        for (int q = 0; q < QV; ++q)
+          *reinterpret_cast<__nv_bfloat16*>(pcol + (qb + q) * 128 + (((kt >> 3) ^ (q & 7)) << 4)) = __float2bfloat16_rn(e[q]);
         ptx::fence_proxy_async();
         ptx::tc_fence_before();
         __syncwarp();
@@ -558,9 +564,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
 
       // ---- end of item: row sums over all keys (lane q of each warp ends up with the warp's sum of row q)
       float* ls = lsum;
-      float lwarp[NQ / 32];
+      float lwarp[QV / 32];
 #pragma unroll
-      for (int half = 0; half < NQ / 32; ++half) {
+      for (int half = 0; half < QV / 32; ++half) {
         float* v = &l[half * 32];
 #pragma unroll
         for (int off = 16; off >= 1; off >>= 1) {
@@ -577,12 +583,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
       if (!__all_sync(0xffffffffu, ptx::mbar_wait(o_done, item_idx & 1u, abort))) { ok = false; break; }
       ptx::tc_fence_after();
 #pragma unroll
-      for (int half = 0; half < NQ / 32; ++half) ls[qd * 64 + half * 32 + lane] = lwarp[half];
+      for (int half = 0; half < QV / 32; ++half) ls[qd * 64 + qb + half * 32 + lane] = lwarp[half];
       if (!meet()) { ok = false; break; }
-      float o[NQ];  // O^T row d = kg: one value per query row
+      float o[QV];  // O^T row d = kg: one value per query row of this warp's set
 #pragma unroll
-      for (int c = 0; c < NQ / 16; ++c)
-        ptx::tmem_ld16(lane_addr + O_COL + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&o[c * 16]));
+      for (int c = 0; c < QV / 16; ++c)
+        ptx::tmem_ld16(lane_addr + O_COL + qb + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&o[c * 16]));
       ptx::tmem_ld_wait();
       ptx::tc_fence_before();
       __syncwarp();
@@ -595,10 +601,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
       if (it.n_splits == 1) {
         if (d < HD) {
 #pragma unroll
-          for (int q = 0; q < NQ; ++q) {
-            if (q < GD) {
-              const float lt = ls[q] + ls[64 + q] + ls[128 + q] + ls[192 + q];
-              out_base[row_off[q]] = __float2bfloat16_rn(o[q] / lt);
+          for (int q = 0; q < QV; ++q) {
+            if (qb + q < GD) {
+              const float lt = ls[qb + q] + ls[64 + qb + q] + ls[128 + qb + q] + ls[192 + qb + q];
+              out_base[row_off[qb + q]] = __float2bfloat16_rn(o[q] / lt);
             }
           }
         }
@@ -606,11 +612,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
         const size_t slot_row = (size_t)(blockIdx.x + it.pair) * NQ;
         if (d < HD) {
 #pragma unroll
-          for (int q = 0; q < NQ; ++q) p.part_o[(slot_row + q) * HD + d] = o[q];
+          for (int q = 0; q < QV; ++q) p.part_o[(slot_row + qb + q) * HD + d] = o[q];
         }
-        if (kg < NQ)
-          *reinterpret_cast<float2*>(p.part_ml + (slot_row + kg) * 2) =
-              make_float2(mref[kg], ls[kg] + ls[64 + kg] + ls[128 + kg] + ls[192 + kg]);
+        const int mrow = qb + kg;  // the query row this thread looks after where one thread per row is needed
+        if (kg < QV)
+          *reinterpret_cast<float2*>(p.part_ml + (slot_row + mrow) * 2) =
+              make_float2(mref[mrow], ls[mrow] + ls[64 + mrow] + ls[128 + mrow] + ls[192 + mrow]);
         __threadfence();
         if (!meet()) { ok = false; break; }
         if (warp == 2 && lane == 0) {  // every split of the pair counts once; the last one merges
@@ -629,24 +636,26 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
           float* wbuf = reinterpret_cast<float*>(p_s);
           const size_t first_row = (size_t)(it.c_first + it.pair) * NQ;
           float m = -INFINITY, L = 0.f;
-          if (kg < GD) {
+          const bool row_thread = kg < QV && mrow < GD;
+          if (row_thread) {
 #pragma unroll 8
-            for (int s = 0; s < it.n_splits; ++s) m = fmaxf(m, __ldcg(p.part_ml + (first_row + (size_t)s * NQ + kg) * 2));
+            for (int s = 0; s < it.n_splits; ++s) m = fmaxf(m, __ldcg(p.part_ml + (first_row + (size_t)s * NQ + mrow) * 2));
           }
-          const int dq = tid & 31, qg = (tid >> 5) & 3;  // four columns 4*dq.. of the rows q = qg mod 4
-          float acc[NQ / 4][4];
+          constexpr int NSW = NQ / 8;           // softmax warps
+          const int dq = lane, qg = sw;         // four columns 4*dq.. of the rows q = qg mod NSW
+          float acc[NQ / NSW][4];
 #pragma unroll
-          for (int i = 0; i < NQ / 4; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
+          for (int i = 0; i < NQ / NSW; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
           for (int c0 = 0; c0 < it.n_splits; c0 += kCap) {
             const int cn = min(kCap, it.n_splits - c0);
             if (c0 > 0 && !meet()) { ok = false; break; }  // the previous chunk's weights are no longer read
-            if (kg < GD) {
+            if (row_thread) {
 #pragma unroll 8
               for (int s = 0; s < cn; ++s) {
-                const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (first_row + (size_t)(c0 + s) * NQ + kg) * 2));
+                const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (first_row + (size_t)(c0 + s) * NQ + mrow) * 2));
                 const float a = ptx::ex2(ml.x - m);
                 L = fmaf(a, ml.y, L);
-                wbuf[s * NQ + kg] = a;
+                wbuf[s * NQ + mrow] = a;
               }
             }
             if (!meet()) { ok = false; break; }
@@ -655,8 +664,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
               for (int s = 0; s < cn; ++s) {
                 const float* src = p.part_o + (first_row + (size_t)(c0 + s) * NQ) * HD + 4 * dq;
 #pragma unroll
-                for (int i = 0; i < NQ / 4; ++i) {
-                  const int q = qg + 4 * i;
+                for (int i = 0; i < NQ / NSW; ++i) {
+                  const int q = qg + NSW * i;
                   if (q < GD) {
                     const float wq = wbuf[s * NQ + q];
                     const float4 v = __ldcg(reinterpret_cast<const float4*>(src + (size_t)q * HD));
@@ -670,13 +679,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) block_attn_umma_kernel(const 
             }
           }
           if (!ok) break;
-          if (kg < GD) fbuf[kg] = 1.0f / L;
+          if (row_thread) fbuf[mrow] = 1.0f / L;
           if (!meet()) { ok = false; break; }
           if (4 * dq < HD) {
             __nv_bfloat16* ob = p.out + ((size_t)it.b * p.D * p.Hq + it.h * p.G) * HD + 4 * dq;
 #pragma unroll
-            for (int i = 0; i < NQ / 4; ++i) {
-              const int q = qg + 4 * i;
+            for (int i = 0; i < NQ / NSW; ++i) {
+              const int q = qg + NSW * i;
               if (q < GD) {
                 const float inv = fbuf[q];
                 uint2 v;
@@ -804,7 +813,7 @@ static cudaError_t attn_launch_one(sdlm_ctx* ctx, AttnParams& p, cudaStream_t st
   p.n_stages = n;
   const size_t smem = (size_t)attn_fixed_smem<HD, NQ>(p.batch) + (size_t)n * (pair_b + 16);
   const int n_cta = ctx->sm_count < kAttnMaxCtas ? ctx->sm_count : kAttnMaxCtas;
-  const cudaError_t e = launch_overlapped(block_attn_umma_kernel<HD, NQ>, dim3(n_cta), dim3(kAttnThreads), smem, st, p);
+  const cudaError_t e = launch_overlapped(block_attn_umma_kernel<HD, NQ>, dim3(n_cta), dim3(attn_threads(NQ)), smem, st, p);
   ctx->launches++;
   return e != cudaSuccess ? e : cudaGetLastError();
 }
