@@ -18,9 +18,10 @@
 //               tensor-core shared-memory layout) into a ring of two-tile buffers;
 //   warp 1      one thread issues the S^T instructions (S^T double-buffered in tensor memory);
 //   warp 7      one thread issues the O^T instructions;
-//   warps 2..5  softmax: thread = accumulator lane = one key; it holds that key's score for every
-//               query row, exponentiates against a per-row reference kept in shared memory, adds to
-//               its private row sums and writes its column of P^T (bf16) into the B-operand buffer;
+//   warps 2..5  softmax: thread = accumulator lane = one key; it holds that key's score for 32
+//               query rows, exponentiates against per-row references kept in shared memory, adds to
+//               its private row sums and writes its column of P^T (bf16) into the B-operand buffer
+//               (with 64 stacked rows warps 8..11 do the same for rows 32..63);
 //   warp 6      stages the stacked query rows (fetched one item ahead) and the block's own K/V rows.
 // The reference of a row is not the running maximum: it is only moved (and O^T, sums rescaled)
 // when some score exceeds it by more than 2^32, which the softmax warps agree on once per group;
@@ -709,25 +710,35 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     Ring ring{0, 0};
     uint32_t blk_idx = 0, item_idx = 0;
     bool ok = true;
-    uint4 qreg[NQC];
+    // At most 16 chunks per lane are kept in registers at a time (more would spill and serialise the
+    // loads): those are fetched one item ahead, the rest (only with 64 stacked rows) when the item starts.
+    constexpr int NQR = NQC < 16 ? NQC : 16;
+    uint4 qreg[NQR];
     // stacked query rows: row r = j*G + g  <->  q[b, j, h*G + g, :]; rows beyond G*D are zero
-    auto fetch_q = [&](const Item& x) {
+    auto fetch_q = [&](const Item& x, int first) {
 #pragma unroll
-      for (int i = 0; i < NQC; ++i) {
-        const int idx = i * 32 + lane, r = idx / (HD / 8), c = idx % (HD / 8);
+      for (int i = 0; i < NQR; ++i) {
+        const int idx = (first + i) * 32 + lane, r = idx / (HD / 8), c = idx % (HD / 8);
         qreg[i] = make_uint4(0, 0, 0, 0);
         if (r < GD)
           qreg[i] = __ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)x.b * p.D * p.Hq + x.h * p.G) * HD + row_off[r]) + c);
       }
     };
+    auto store_q = [&](int first) {
+#pragma unroll
+      for (int i = 0; i < NQR; ++i) {
+        const int idx = (first + i) * 32 + lane, r = idx / (HD / 8), c = idx % (HD / 8);
+        *reinterpret_cast<uint4*>(q_s + (c >> 3) * Q_PANEL_B + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = qreg[i];
+      }
+    };
     bool have = walk_next(w, p, it);
-    if (have) fetch_q(it);
+    if (have) fetch_q(it, 0);
     while (ok && have) {
       if (item_idx > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait(q_free, (item_idx - 1) & 1u, abort))) { ok = false; break; }
-#pragma unroll
-      for (int i = 0; i < NQC; ++i) {
-        const int idx = i * 32 + lane, r = idx / (HD / 8), c = idx % (HD / 8);
-        *reinterpret_cast<uint4*>(q_s + (c >> 3) * Q_PANEL_B + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = qreg[i];
+      store_q(0);
+      for (int first = NQR; first < NQC; first += NQR) {
+        fetch_q(it, first);
+        store_q(first);
       }
       ptx::fence_proxy_async();
       __syncwarp();
@@ -736,7 +747,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
 
       // the next item's query rows travel while this item is being processed
       have = walk_next(w, p, nxt);
-      if (have) fetch_q(nxt);
+      if (have) fetch_q(nxt, 0);
 
       const int n = it.t1 - it.t0, ng = (n + 1) / 2;
       for (int g = 0; g + 1 < ng; ++g) ring.advance(NS);
