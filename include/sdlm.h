@@ -243,9 +243,10 @@ sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const
  * LM-head kernel while attention's last thread blocks are still running (default 0: in order).
  * SDLM_OPT_ATTN_ITEM_COST: 0..64, how many cache pages' worth of work the attention schedule
  * charges a thread block for every (sequence, KV head) pair it starts (default 12); results do not
- * depend on it.
+ * depend on it.  SDLM_OPT_ATTN_MIN_RANGE: 1..4096, the fewest schedule positions (pages plus item
+ * costs) one thread block is given, which bounds how finely a short workload is split.
  * Errors: INVALID_ARG. */
-typedef enum sdlm_option { SDLM_OPT_LMHEAD_KERNEL = 0, SDLM_OPT_STEP_OVERLAP = 1, SDLM_OPT_ATTN_ITEM_COST = 2 } sdlm_option;
+typedef enum sdlm_option { SDLM_OPT_LMHEAD_KERNEL = 0, SDLM_OPT_STEP_OVERLAP = 1, SDLM_OPT_ATTN_ITEM_COST = 2, SDLM_OPT_ATTN_MIN_RANGE = 3 } sdlm_option;
 sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t value);
 
 /* Number of kernels the library has launched through this context since it was created. */

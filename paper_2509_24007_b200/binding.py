@@ -23,6 +23,7 @@ KV_RESET, KV_ADD_SEQ, KV_RELEASE_SEQ, KV_QUERY, KV_GATHER, KV_EXPORT, KV_IMPORT,
 OPT_LMHEAD_KERNEL = 0
 OPT_STEP_OVERLAP = 1
 OPT_ATTN_ITEM_COST = 2
+OPT_ATTN_MIN_RANGE = 3
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "UNSUPPORTED", 4: "OUT_OF_PAGES", 5: "CUDA",
                 6: "TIMEOUT", 7: "DEVICE_CHECK", 8: "WORKSPACE"}

@@ -419,6 +419,7 @@ extern "C" sdlm_status sdlm_create(const sdlm_config* cfg, void* kv_pool, size_t
   ctx->lmhead_path = 0;
   ctx->overlap_lmhead = 0;
   ctx->attn_item_cost = 12;
+  ctx->attn_min_range = 8;
   ctx->tmap_w_ptr = nullptr;
   ctx->tmap_w_rows = 0;
   if (setup_attn(ctx) != cudaSuccess || setup_lmhead(ctx) != cudaSuccess) { delete ctx; return SDLM_ERR_CUDA; }
@@ -441,6 +442,10 @@ extern "C" sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t v
     case SDLM_OPT_ATTN_ITEM_COST:
       if (value < 0 || value > 64) return SDLM_ERR_INVALID_ARG;
       ctx->attn_item_cost = value;
+      return SDLM_OK;
+    case SDLM_OPT_ATTN_MIN_RANGE:
+      if (value < 1 || value > 4096) return SDLM_ERR_INVALID_ARG;
+      ctx->attn_min_range = value;
       return SDLM_OK;
     case SDLM_OPT_STEP_OVERLAP:
       if (value < 0 || value > 1) return SDLM_ERR_INVALID_ARG;

@@ -47,6 +47,7 @@ struct AttnParams {
   DevHeader* hdr;
   float scale_log2;  // softmax scale * log2(e)
   int batch, D, Hq, Hkv, G, mpps, num_pages, n_stages;
+  int min_range;  // shortest range of positions worth a CTA of its own
   int item_cost;  // what starting a (sequence, KV head) pair costs a CTA, in tiles (see ItemWalk)
 };
 
@@ -90,13 +91,15 @@ __device__ __forceinline__ int pos_owner(uint32_t x, uint32_t total, uint32_t nc
   return (int)(((x + 1) * nc - 1) / total);  // the CTA c with floor(c*total/nc) <= x < floor((c+1)*total/nc)
 }
 
-__device__ __forceinline__ void walk_begin(ItemWalk& w, const int* s_first, int batch, int Hkv) {
+__device__ __forceinline__ void walk_begin(ItemWalk& w, const int* s_first, int batch, int Hkv, int p_min_range) {
   w.s_first = s_first;
   w.s_len = s_first + batch + 1;
   w.s_slot = w.s_len + batch;
   w.total = (uint32_t)s_first[batch] * (uint32_t)Hkv;
-  // never more ranges than positions: every range is then non-empty
-  w.nc = min(gridDim.x, w.total);
+  // Never more ranges than positions (every range is then non-empty), and no range shorter than a
+  // few tiles: below that the fixed cost of a CTA and of merging its partial result outweighs
+  // the parallelism.
+  w.nc = min(gridDim.x, max(1u, w.total / (uint32_t)max(1, p_min_range)));
   if (blockIdx.x >= w.nc) {
     w.cur = w.hi = 0;
     return;
@@ -278,7 +281,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
   {
     ItemWalk w0;
     Item i0;
-    walk_begin(w0, s_first, p.batch, p.Hkv);
+    walk_begin(w0, s_first, p.batch, p.Hkv, p.min_range);
     if (!walk_next(w0, p, i0)) {  // no tile falls into this CTA's range (uniform for the CTA)
       if (warp == 1) ptx::tmem_dealloc(*tmem_slot, TMEM_COLS);
       return;
@@ -289,7 +292,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
   if (warp == 0) {
     // ---------------------------------------------------------------- cached tiles: bulk copies
     ItemWalk w;
-    walk_begin(w, s_first, p.batch, p.Hkv);
+    walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
     Item it;
     Ring ring{0, 0};
     uint32_t issued = 0;  // groups so far
@@ -354,7 +357,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NQ >> 3) << 17) | ((128u >> 4) << 24);
       const uint32_t q_addr = ptx::smem_u32(q_s), st_addr = ptx::smem_u32(stages);
       ItemWalk w;
-      walk_begin(w, s_first, p.batch, p.Hkv);
+      walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
       Item it;
       Ring ring{0, 0};
       uint32_t gc = 0, item_idx = 0;
@@ -394,7 +397,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NQ >> 3) << 17) | ((128u >> 4) << 24);
       const uint32_t p_addr = ptx::smem_u32(p_s), st_addr = ptx::smem_u32(stages);
       ItemWalk w;
-      walk_begin(w, s_first, p.batch, p.Hkv);
+      walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
       Item it;
       Ring ring{0, 0};
       uint32_t gc = 0, item_idx = 0;
@@ -443,7 +446,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     const int tj = kg >> 6, kt = kg & 63;  // tile of the group, key within that tile
     const uint32_t lane_addr = tmem_base + ((uint32_t)(qd * 32) << 16);
     ItemWalk w;
-    walk_begin(w, s_first, p.batch, p.Hkv);
+    walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
     Item it;
     uint32_t gc = 0, item_idx = 0, ep_uses = 0;
     bool ok = true;
@@ -705,7 +708,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     // ---------------------------------------------------------------- warp 6: Q rows and the block's own tile
     constexpr int NQC = NQ * (HD / 8) / 32;  // 16-byte chunks of the stacked query rows per lane
     ItemWalk w;
-    walk_begin(w, s_first, p.batch, p.Hkv);
+    walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
     Item it, nxt;
     Ring ring{0, 0};
     uint32_t blk_idx = 0, item_idx = 0;
@@ -863,6 +866,7 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
   p.batch = batch; p.D = D; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.G = ctx->group;
   p.mpps = c.max_pages_per_seq; p.num_pages = c.num_pages; p.n_stages = 0;
   p.item_cost = ctx->attn_item_cost;
+  p.min_range = ctx->attn_min_range;
   // the kernel's tile arithmetic is 32-bit: (tiles of the launch) x (CTAs) must stay below 2^31
   if ((long long)batch * (c.max_pages_per_seq + 1 + ctx->attn_item_cost) * c.n_kv_heads > 13000000ll)
     return cudaErrorInvalidConfiguration;

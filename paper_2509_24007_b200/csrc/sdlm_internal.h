@@ -60,6 +60,7 @@ struct sdlm_ctx {
   int32_t* free_list;
   uint64_t launches;
   int lmhead_path;  // 0 = pick by shape, 1 = force the mma.sync kernel, 2 = force the tcgen05 kernel
+  int attn_min_range;  // shortest range of schedule positions given to one attention thread block
   int attn_item_cost;  // positions the attention schedule charges for starting a (sequence, KV head) pair
   int overlap_lmhead;  // sdlm_decode_step: let the LM-head stripe kernel start before attention has finished
   // cached TMA descriptor of the LM-head weight (keyed by pointer and tile rows)
