@@ -164,7 +164,7 @@ LMHEAD_NCU_TRAFFIC = 635448832   # bytes per launch of lmhead_umma_kernel<1> at 
 RESTORE_EVERY = 8   # steps between restores of the cache tables, so that prefix lengths stay the workload's
 
 
-def time_workload(torch, dp, wl, steps, warmup, n_blocks=4):
+def time_workload(torch, dp, wl, steps, warmup, n_blocks=4, use_graph=True):
     """Device-timed region of `steps` whole steps (three library calls each, nothing else on the stream
     but a table restore every RESTORE_EVERY steps).  A second pass of the same steps brackets the
     LM-head call with events: that is the dominant kernel's launch duration for the roofline."""
@@ -192,13 +192,44 @@ def time_workload(torch, dp, wl, steps, warmup, n_blocks=4):
     run(warmup, 0)
     torch.cuda.synchronize()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    graph, per_graph = None, 0
+    if use_graph and steps >= RESTORE_EVERY:
+        # RESTORE_EVERY steps (with their table restore) captured once and replayed: the library never
+        # synchronises with the host, so the whole loop can live in a CUDA graph
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        graph = torch.cuda.CUDAGraph()
+        acc_g = torch.zeros((RESTORE_EVERY, wl.batch), dtype=torch.int32, device=sd.device)
+        with torch.cuda.stream(side):
+            n0 = sd.launch_count()
+            with torch.cuda.graph(graph, stream=side):
+                for i in range(RESTORE_EVERY):
+                    x = blocks[(warmup + i) % n_blocks]
+                    if i == 0:
+                        sd.kv_restore(saved, stream=side)
+                    sd.block_attn(x.q, x.k_blk, x.v_blk, out.attn, stream=side)
+                    sd.lmhead_confidence(x.hidden, dp.w_lm, out.token, out.p_top1, out.entropy, stream=side)
+                    sd.accept_commit(wl.tau, out.token, out.p_top1, out.entropy, x.k_blk, x.v_blk, 0, acc_g[i],
+                                     out.out_tokens, stream=side)
+            per_graph = sd.launch_count() - n0
+        stream.wait_stream(side)
+        for _ in range(2):
+            graph.replay()
+        torch.cuda.synchronize()
     launches0 = sd.launch_count()
+    replays = steps // RESTORE_EVERY if graph is not None else 0
+    rest = steps - replays * RESTORE_EVERY
     ev0.record(stream)
-    run(steps, warmup, acc_buf)
+    for _ in range(replays):
+        graph.replay()
+    run(rest, warmup, acc_buf)
     ev1.record(stream)
     torch.cuda.synchronize()
-    launches = sd.launch_count() - launches0
+    launches = sd.launch_count() - launches0 + replays * per_graph
     ms = ev0.elapsed_time(ev1)
+    tokens = int(acc_buf[:rest].clamp(min=0).sum().item())
+    if graph is not None:
+        tokens += replays * int(acc_g.clamp(min=0).sum().item())
     # second pass: per-call device times
     n2 = min(steps, 200)
     mk = lambda: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n2)]
@@ -210,8 +241,8 @@ def time_workload(torch, dp, wl, steps, warmup, n_blocks=4):
     sd.kv_restore(saved)
     torch.cuda.synchronize()
     assert int(sd.device_status()[0]) == 0, "device status set during the timed region"
-    return {"ms_total": ms, "ms_per_step": ms / steps, "tokens": int(acc_buf.clamp(min=0).sum().item()), "lm_ms": lm_ms,
-            "attn_ms": at_ms, "launches": launches}
+    return {"ms_total": ms, "ms_per_step": ms / steps, "tokens": tokens, "lm_ms": lm_ms,
+            "attn_ms": at_ms, "launches": launches, "graph": graph is not None}
 
 
 def time_e2e(torch, dp, wl, steps, warmup, n_blocks=4):
@@ -269,6 +300,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg2_d4", choices=syn.workloads())
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--no-graph", action="store_true", help="enqueue every step from the host instead of replaying a CUDA graph")
     ap.add_argument("--no-extra", action="store_true", help="skip the D=8 companion measurement and the CPU baseline")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
@@ -303,7 +335,7 @@ def main():
     barrier()
     if rank == 0:
         sampler.start()
-    res = time_workload(torch, dp, wl_run, args.steps, args.warmup)
+    res = time_workload(torch, dp, wl_run, args.steps, args.warmup, use_graph=not args.no_graph)
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     e2e = time_e2e(torch, dp, wl_run, max(3, min(args.steps, 100)), 3)
@@ -325,6 +357,7 @@ def main():
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": _config(wl, lengths),
         "tokens_per_step": tokens / args.steps / world,
         "gpu_launches": res["launches"],
+        "launch_mode": (f"CUDA graph of {RESTORE_EVERY} steps replayed" if res["graph"] else "one host call per library call"),
         "clocks": clocks,
         "e2e": e2e,
         "roofline": {"bound": "hbm", "kernel": "lmhead_umma_kernel (sdlm_lmhead_confidence: stripe kernel + merge of the stripes)",

@@ -212,3 +212,38 @@ def test_block_size_one_is_next_token_decode_on_the_gpu():
         out, stats, res, n_bad = _one_step(dp, cache, tau, step)
         assert n_bad == 0 and out.accepted_len.cpu().tolist() == [1] * wl.batch
         _compare_tables(dp, cache)
+
+
+def test_steps_replayed_from_a_cuda_graph_match_eager_steps():
+    """The three calls never synchronise with the host, so a run of steps can be captured once and
+    replayed; accepted lengths, tokens and tables must equal the eager run."""
+    wl = syn.CONFIGS["cfg0"].with_(batch=4, prefix_lo=50, prefix_hi=260)
+    dp = DeviceProblem(wl)
+    blocks = [dp.block(i) for i in range(3)]
+    outs = [dp.alloc_outputs() for _ in range(3)]
+    saved = dp.sd.kv_save()
+    for x, o in zip(blocks, outs):                       # eager reference
+        dp.step(x, wl.tau, o)
+    torch.cuda.synchronize()
+    ref = [(o.accepted_len.clone(), o.out_tokens.clone(), o.attn.clone()) for o in outs]
+    t_ref = dp.sd.kv_tables()
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        dp.sd.kv_restore(saved, stream=stream)
+        dp.step(blocks[0], wl.tau, outs[0], stream=stream)     # warm-up on the capture stream
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=stream):
+            dp.sd.kv_restore(saved, stream=stream)
+            for x, o in zip(blocks, outs):
+                dp.step(x, wl.tau, o, stream=stream)
+    for _ in range(2):
+        for o in outs:
+            o.accepted_len.zero_(); o.out_tokens.zero_(); o.attn.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for o, (acc, tok, attn) in zip(outs, ref):
+            assert torch.equal(o.accepted_len, acc) and torch.equal(o.out_tokens, tok) and torch.equal(o.attn, attn)
+        t = dp.sd.kv_tables()
+        assert np.array_equal(t["seq_len"], t_ref["seq_len"]) and np.array_equal(t["page_table"], t_ref["page_table"])
+        assert t["status"][0] == 0
