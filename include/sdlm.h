@@ -239,8 +239,10 @@ sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const
 /* Tuning / test knobs (the paper has no counterpart).  SDLM_OPT_LMHEAD_KERNEL: which stripe kernel
  * sdlm_lmhead_confidence uses: 0 = chosen from the shape (default), 1 = warp-level mma.sync
  * kernel, 2 = tcgen05 / TMA kernel (the call then fails with UNSUPPORTED for rows > 256 or
- * |V| < 16).  SDLM_OPT_STEP_OVERLAP: 1 lets sdlm_decode_step / sdlm_decode_step_host start the
- * LM-head kernel while attention's last thread blocks are still running (default 0: in order).
+ * |V| < 16).  SDLM_OPT_STEP_OVERLAP: A in 0..SMs-1.  With A > 0 sdlm_decode_step /
+ * sdlm_decode_step_host run attention on A SMs and the LM-head kernel at the same time on the
+ * other SMs (the work is split over fewer thread blocks each, so results agree to rounding, not
+ * bit for bit; default 0: one after the other on all SMs).
  * SDLM_OPT_ATTN_ITEM_COST: 0..64, how many cache pages' worth of work the attention schedule
  * charges a thread block for every (sequence, KV head) pair it starts (default 12); results do not
  * depend on it.  SDLM_OPT_ATTN_MIN_RANGE: 1..4096, the fewest schedule positions (pages plus item

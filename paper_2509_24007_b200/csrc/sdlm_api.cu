@@ -448,7 +448,7 @@ extern "C" sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t v
       ctx->attn_min_range = value;
       return SDLM_OK;
     case SDLM_OPT_STEP_OVERLAP:
-      if (value < 0 || value > 1) return SDLM_ERR_INVALID_ARG;
+      if (value < 0 || value >= ctx->sm_count) return SDLM_ERR_INVALID_ARG;
       ctx->overlap_lmhead = value;
       return SDLM_OK;
   }
@@ -609,19 +609,30 @@ extern "C" sdlm_status sdlm_device_status(sdlm_ctx* ctx, int32_t* host_out, int3
   return SDLM_OK;
 }
 
-// (a) + (b) + (c) on device buffers.  The LM head reads nothing that attention writes, so its stripe
-// kernel is allowed to start while attention's last CTAs are still running.
+// (a) + (b) + (c) on device buffers.  The LM head reads nothing that attention writes.  With the
+// overlap option set to A, attention is launched on A thread blocks and the LM-head stripe kernel on
+// (SMs - A), and the stripe kernel does not wait for attention before it starts: the two then run side
+// by side on disjoint SMs, attention's latency-bound gathers hidden under the LM head's weight stream.
+// Both are one thread block per SM, so neither can crowd the other out; the stripe kernel still waits
+// for attention to have finished before it exits, which orders the commit kernel after both.
 static sdlm_status decode_step_device(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, float tau,
                                       sdlm_conf_mode mode, const void* q, const void* k_blk, const void* v_blk,
                                       const void* hidden, const void* w_lm, void* attn_out, int32_t* token,
                                       float* p_top1, float* entropy, int32_t* accepted_len, int32_t* out_tokens,
                                       void* stream) {
-  sdlm_status s = sdlm_block_attn(ctx, batch, D, seq_ids, q, k_blk, v_blk, attn_out, stream);
+  if (!ctx || !q || !k_blk || !v_blk || !attn_out) return SDLM_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(attn_out)) return SDLM_ERR_INVALID_ARG;
+  sdlm_status s = check_batch(ctx, batch, D);
   if (s != SDLM_OK) return s;
+  const int a_sms = ctx->overlap_lmhead;
+  if (launch_block_attn(ctx, batch, D, seq_ids, q, k_blk, v_blk, attn_out, static_cast<cudaStream_t>(stream), a_sms) !=
+      cudaSuccess)
+    return SDLM_ERR_CUDA;
   if (!hidden || !w_lm || !token || !p_top1 || !entropy) return SDLM_ERR_INVALID_ARG;
   if (!aligned16(hidden) || !aligned16(w_lm)) return SDLM_ERR_INVALID_ARG;
   s = launch_lmhead(ctx, batch * D, hidden, w_lm, token, p_top1, entropy, nullptr, nullptr,
-                    static_cast<cudaStream_t>(stream), /*independent_of_predecessor=*/ctx->overlap_lmhead != 0);
+                    static_cast<cudaStream_t>(stream), /*independent_of_predecessor=*/a_sms > 0,
+                    a_sms > 0 ? ctx->sm_count - a_sms : 0);
   if (s != SDLM_OK) return s;
   return sdlm_accept_commit(ctx, batch, D, seq_ids, tau, mode, token, p_top1, entropy, k_blk, v_blk, accepted_len,
                             out_tokens, stream);

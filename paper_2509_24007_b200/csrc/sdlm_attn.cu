@@ -819,14 +819,15 @@ static int attn_fixed_smem(int batch) {
 }
 
 template <int HD, int NQ>
-static cudaError_t attn_launch_one(sdlm_ctx* ctx, AttnParams& p, cudaStream_t st) {
+static cudaError_t attn_launch_one(sdlm_ctx* ctx, AttnParams& p, cudaStream_t st, int cta_cap) {
   const int pair_b = 2 * (2 * kPageSize * HD * 2);
   int n = (kAttnSmemLimit - attn_fixed_smem<HD, NQ>(p.batch)) / (pair_b + 16);
   if (n > 6) n = 6;
   if (n < 2) return cudaErrorLaunchOutOfResources;
   p.n_stages = n;
   const size_t smem = (size_t)attn_fixed_smem<HD, NQ>(p.batch) + (size_t)n * (pair_b + 16);
-  const int n_cta = ctx->sm_count < kAttnMaxCtas ? ctx->sm_count : kAttnMaxCtas;
+  int n_cta = ctx->sm_count < kAttnMaxCtas ? ctx->sm_count : kAttnMaxCtas;
+  if (cta_cap > 0 && cta_cap < n_cta) n_cta = cta_cap;
   const cudaError_t e = launch_overlapped(block_attn_umma_kernel<HD, NQ>, dim3(n_cta), dim3(attn_threads(NQ)), smem, st, p);
   ctx->launches++;
   return e != cudaSuccess ? e : cudaGetLastError();
@@ -847,7 +848,7 @@ cudaError_t setup_attn(sdlm_ctx* ctx) {
 }
 
 cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, const void* q,
-                              const void* k_blk, const void* v_blk, void* out, cudaStream_t st) {
+                              const void* k_blk, const void* v_blk, void* out, cudaStream_t st, int cta_cap) {
   const sdlm_config& c = ctx->cfg;
   AttnParams p;
   p.pool = reinterpret_cast<const __nv_bfloat16*>(ctx->pool);
@@ -871,8 +872,9 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
   if ((long long)batch * (c.max_pages_per_seq + 1 + ctx->attn_item_cost) * c.n_kv_heads > 13000000ll)
     return cudaErrorInvalidConfiguration;
   const bool wide = ctx->group * D > 32;  // stacked query rows padded to 64, else to 32
-  if (c.head_dim == 128) return wide ? attn_launch_one<128, 64>(ctx, p, st) : attn_launch_one<128, 32>(ctx, p, st);
-  return wide ? attn_launch_one<64, 64>(ctx, p, st) : attn_launch_one<64, 32>(ctx, p, st);
+  if (c.head_dim == 128)
+    return wide ? attn_launch_one<128, 64>(ctx, p, st, cta_cap) : attn_launch_one<128, 32>(ctx, p, st, cta_cap);
+  return wide ? attn_launch_one<64, 64>(ctx, p, st, cta_cap) : attn_launch_one<64, 32>(ctx, p, st, cta_cap);
 }
 
 }  // namespace sdlm

@@ -62,7 +62,7 @@ struct sdlm_ctx {
   int lmhead_path;  // 0 = pick by shape, 1 = force the mma.sync kernel, 2 = force the tcgen05 kernel
   int attn_min_range;  // shortest range of schedule positions given to one attention thread block
   int attn_item_cost;  // positions the attention schedule charges for starting a (sequence, KV head) pair
-  int overlap_lmhead;  // sdlm_decode_step: let the LM-head stripe kernel start before attention has finished
+  int overlap_lmhead;  // sdlm_decode_step: SMs given to attention while the LM head runs on the rest (0: one after the other)
   // cached TMA descriptor of the LM-head weight (keyed by pointer and tile rows)
   const void* tmap_w_ptr;
   int tmap_w_rows;
@@ -112,12 +112,13 @@ inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 b
 
 // ---- launchers implemented in the kernel translation units ---------------------------------
 cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, const void* q,
-                              const void* k_blk, const void* v_blk, void* out, cudaStream_t st);
+                              const void* k_blk, const void* v_blk, void* out, cudaStream_t st,
+                              int cta_cap = 0);
 // `independent_of_predecessor`: the caller guarantees that none of the inputs is written by the
 // kernel enqueued just before on `st` (the stripe kernel then overlaps with it).
 sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
                           float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st,
-                          bool independent_of_predecessor = false);
+                          bool independent_of_predecessor = false, int cta_cap = 0);
 cudaError_t setup_attn(sdlm_ctx* ctx);
 cudaError_t setup_lmhead(sdlm_ctx* ctx);
 

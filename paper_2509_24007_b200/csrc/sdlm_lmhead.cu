@@ -518,7 +518,8 @@ cudaError_t setup_lmhead(sdlm_ctx* ctx) {
 // `partials` holds one float4 per (stripe, row): [max_stripes][rows_pad].
 static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
                                     float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st,
-                                    float4* partials, int rows_pad, int max_stripes, bool independent) {
+                                    float4* partials, int rows_pad, int max_stripes, bool independent,
+                                    int cta_cap = 0) {
   const sdlm_config& c = ctx->cfg;
   LmParams p;
   p.hidden = static_cast<const __nv_bfloat16*>(hidden);
@@ -538,6 +539,7 @@ static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden,
     const int groups = (c.vocab + 15) / 16;
     int n_cta = groups < ctx->sm_count ? groups : ctx->sm_count;
     if (n_cta > max_stripes) n_cta = max_stripes;
+    if (cta_cap > 0 && cta_cap < n_cta) n_cta = cta_cap;
     const int gmax = (groups + n_cta - 1) / n_cta;
     const int tiles = (gmax * 16 + 255) / 256;
     p.bn = 16 * ((gmax + tiles - 1) / tiles);
@@ -582,10 +584,10 @@ static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden,
 
 sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
                           float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st,
-                          bool independent_of_predecessor) {
+                          bool independent_of_predecessor, int cta_cap) {
   return launch_lmhead_on(ctx, rows, hidden, w_lm, token, p_top1, entropy, max_logit, lse, st,
                           reinterpret_cast<float4*>(ctx->ws + ctx->lay.lm_partials),
-                          ctx->cfg.max_batch * ctx->cfg.max_block, kLmMaxStripes, independent_of_predecessor);
+                          ctx->cfg.max_batch * ctx->cfg.max_block, kLmMaxStripes, independent_of_predecessor, cta_cap);
 }
 
 }  // namespace sdlm

@@ -178,11 +178,11 @@ def test_decode_step_host_entry_matches_device_calls():
 
 @pytest.mark.parametrize("name,batch", [("cfg0", 3), ("cfg2_d4", 6)])
 def test_decode_step_device_entry_matches_three_calls(name, batch):
-    """sdlm_decode_step lets attention and the LM head overlap on the GPU; results must not change."""
+    """sdlm_decode_step may run attention and the LM head side by side on disjoint SMs; results must not change."""
     wl = syn.CONFIGS[name].with_(batch=batch, prefix_lo=10, prefix_hi=700)
     dp = DeviceProblem(wl)
     for step in range(4):
-        dp.sd.set_option(OPT_STEP_OVERLAP, step % 2)
+        dp.sd.set_option(OPT_STEP_OVERLAP, (0, 40, 1, 147)[step])   # SMs given to attention; 0: in order
         x = dp.block(step)
         snap = dp.sd.kv_export()
         ref = dp.step(x, wl.tau)
@@ -193,8 +193,14 @@ def test_decode_step_device_entry_matches_three_calls(name, batch):
         out = dp.step(x, wl.tau, fused=True)
         torch.cuda.synchronize()
         assert dp.sd.device_status()[0] == 0
-        for a, b_ in zip((out.attn, out.token, out.p_top1, out.entropy, out.accepted_len, out.out_tokens),
-                         (ref.attn, ref.token, ref.p_top1, ref.entropy, ref.accepted_len, ref.out_tokens)):
+        if step == 0:      # in order on all SMs: the same launches as the three calls, bit for bit
+            assert torch.equal(out.attn, ref.attn) and torch.equal(out.p_top1, ref.p_top1)
+            assert torch.equal(out.entropy, ref.entropy)
+        else:              # fewer thread blocks each: the work is split, and so rounded, differently
+            assert (out.attn.float() - ref.attn.float()).abs().max().item() <= 2e-2
+            assert (out.p_top1 - ref.p_top1).abs().max().item() <= 1e-3
+            assert (out.entropy - ref.entropy).abs().max().item() <= 1e-3
+        for a, b_ in zip((out.token, out.accepted_len, out.out_tokens), (ref.token, ref.accepted_len, ref.out_tokens)):
             assert torch.equal(a, b_)
         t = dp.sd.kv_tables()
         assert np.array_equal(t["page_table"], t_ref["page_table"]) and np.array_equal(t["seq_len"], t_ref["seq_len"])
