@@ -164,10 +164,13 @@ LMHEAD_NCU_TRAFFIC = 635448832   # bytes per launch of lmhead_umma_kernel<1> at 
 RESTORE_EVERY = 8   # steps between restores of the cache tables, so that prefix lengths stay the workload's
 
 
-def time_workload(torch, dp, wl, steps, warmup, n_blocks=4, use_graph=True):
-    """Device-timed region of `steps` whole steps (three library calls each, nothing else on the stream
-    but a table restore every RESTORE_EVERY steps).  A second pass of the same steps brackets the
-    LM-head call with events: that is the dominant kernel's launch duration for the roofline."""
+def time_workload(torch, dp, wl, steps, warmup, n_blocks=4, use_graph=True, overlap=True):
+    """Device-timed region of `steps` whole steps (one sdlm_decode_step call each, nothing else on the
+    stream but a table restore every RESTORE_EVERY steps).  Before it, un-timed: warm-up steps, the
+    three calls timed one by one (attention and the LM-head call bracketed by events: the latter is the
+    dominant kernel's launch duration for the roofline), and the choice of how many SMs attention gets
+    when the step runs attention and the LM head side by side."""
+    from paper_2509_24007_b200.binding import OPT_STEP_OVERLAP
     blocks = [dp.block(i) for i in range(n_blocks)]
     out = dp.alloc_outputs()
     stream = torch.cuda.current_stream()
@@ -175,21 +178,62 @@ def time_workload(torch, dp, wl, steps, warmup, n_blocks=4, use_graph=True):
     acc_buf = torch.zeros((steps, wl.batch), dtype=torch.int32, device=sd.device)   # gamma of every timed step
     saved = sd.kv_save()
 
-    def run(n, first, acc=None, lm_ev=None, at_ev=None):
+    def one_step(x, acc, st=None):
+        sd.decode_step(wl.tau, x.q, x.k_blk, x.v_blk, x.hidden, dp.w_lm, out.attn, out.token, out.p_top1, out.entropy,
+                       acc, out.out_tokens, stream=st)
+
+    def run(n, first, acc=None):
+        for i in range(n):
+            if i % RESTORE_EVERY == 0:
+                sd.kv_restore(saved)
+            one_step(blocks[(first + i) % n_blocks], acc[i] if acc is not None else out.accepted_len)
+
+    def run_three_calls(n, first, lm_ev, at_ev):
         for i in range(n):
             x = blocks[(first + i) % n_blocks]
             if i % RESTORE_EVERY == 0:
                 sd.kv_restore(saved)
-            if at_ev: at_ev[i][0].record(stream)
+            at_ev[i][0].record(stream)
             sd.block_attn(x.q, x.k_blk, x.v_blk, out.attn)
-            if at_ev: at_ev[i][1].record(stream)
-            if lm_ev: lm_ev[i][0].record(stream)
+            at_ev[i][1].record(stream)
+            lm_ev[i][0].record(stream)
             sd.lmhead_confidence(x.hidden, dp.w_lm, out.token, out.p_top1, out.entropy)
-            if lm_ev: lm_ev[i][1].record(stream)
-            sd.accept_commit(wl.tau, out.token, out.p_top1, out.entropy, x.k_blk, x.v_blk, 0,
-                             acc[i] if acc is not None else out.accepted_len, out.out_tokens)
+            lm_ev[i][1].record(stream)
+            sd.accept_commit(wl.tau, out.token, out.p_top1, out.entropy, x.k_blk, x.v_blk, 0, out.accepted_len,
+                             out.out_tokens)
 
+    def timed(n, first):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        run(n, first)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    sd.set_option(OPT_STEP_OVERLAP, 0)
     run(warmup, 0)
+    # per-call device times, each call on all SMs
+    n2 = min(max(steps, 8), 200)
+    mk = lambda: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n2)]
+    lm_ev, at_ev = mk(), mk()
+    run_three_calls(n2, warmup, lm_ev, at_ev)
+    torch.cuda.synchronize()
+    lm_ms = float(np.mean([a.elapsed_time(b) for a, b in lm_ev]))
+    at_ms = float(np.mean([a.elapsed_time(b) for a, b in at_ev]))
+    # side by side: attention's share of the SMs starts from its share of the two calls' SM-time and
+    # is settled by timing a few neighbours (and the in-order step) on RESTORE_EVERY * 3 steps each
+    a_sms, sweep = 0, {}
+    if overlap:
+        sms = torch.cuda.get_device_properties(sd.device).multi_processor_count
+        a0 = int(round(sms * at_ms / (at_ms + lm_ms)))
+        for a in [0] + sorted({min(max(a0 + d, 1), sms - 1) for d in (-8, -6, -4, -2, 0, 2, 4, 6, 8)}):
+            sd.set_option(OPT_STEP_OVERLAP, a)
+            run(RESTORE_EVERY, warmup)
+            sweep[a] = min(timed(RESTORE_EVERY * 3, warmup) for _ in range(2))
+        a_sms = min(sweep, key=sweep.get)
+    sd.set_option(OPT_STEP_OVERLAP, a_sms)
+    run(max(warmup, RESTORE_EVERY), 0)
     torch.cuda.synchronize()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     graph, per_graph = None, 0
@@ -203,14 +247,9 @@ def time_workload(torch, dp, wl, steps, warmup, n_blocks=4, use_graph=True):
         with torch.cuda.stream(side):
             n0 = sd.launch_count()
             with torch.cuda.graph(graph, stream=side):
+                sd.kv_restore(saved, stream=side)
                 for i in range(RESTORE_EVERY):
-                    x = blocks[(warmup + i) % n_blocks]
-                    if i == 0:
-                        sd.kv_restore(saved, stream=side)
-                    sd.block_attn(x.q, x.k_blk, x.v_blk, out.attn, stream=side)
-                    sd.lmhead_confidence(x.hidden, dp.w_lm, out.token, out.p_top1, out.entropy, stream=side)
-                    sd.accept_commit(wl.tau, out.token, out.p_top1, out.entropy, x.k_blk, x.v_blk, 0, acc_g[i],
-                                     out.out_tokens, stream=side)
+                    one_step(blocks[(warmup + i) % n_blocks], acc_g[i], side)
             per_graph = sd.launch_count() - n0
         stream.wait_stream(side)
         for _ in range(2):
@@ -230,19 +269,12 @@ def time_workload(torch, dp, wl, steps, warmup, n_blocks=4, use_graph=True):
     tokens = int(acc_buf[:rest].clamp(min=0).sum().item())
     if graph is not None:
         tokens += replays * int(acc_g.clamp(min=0).sum().item())
-    # second pass: per-call device times
-    n2 = min(steps, 200)
-    mk = lambda: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n2)]
-    lm_ev, at_ev = mk(), mk()
-    run(n2, warmup, None, lm_ev, at_ev)
-    torch.cuda.synchronize()
-    lm_ms = float(np.mean([a.elapsed_time(b) for a, b in lm_ev]))
-    at_ms = float(np.mean([a.elapsed_time(b) for a, b in at_ev]))
     sd.kv_restore(saved)
     torch.cuda.synchronize()
     assert int(sd.device_status()[0]) == 0, "device status set during the timed region"
     return {"ms_total": ms, "ms_per_step": ms / steps, "tokens": tokens, "lm_ms": lm_ms,
-            "attn_ms": at_ms, "launches": launches, "graph": graph is not None}
+            "attn_ms": at_ms, "launches": launches, "graph": graph is not None, "attn_sms": a_sms,
+            "sweep_us": {str(k): round(v * 1e3, 1) for k, v in sweep.items()}}
 
 
 def time_e2e(torch, dp, wl, steps, warmup, n_blocks=4):
@@ -301,6 +333,7 @@ def main():
     ap.add_argument("--workload", default="cfg2_d4", choices=syn.workloads())
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="enqueue every step from the host instead of replaying a CUDA graph")
+    ap.add_argument("--no-overlap", action="store_true", help="attention, then the LM head, each on all SMs (no side-by-side step)")
     ap.add_argument("--no-extra", action="store_true", help="skip the D=8 companion measurement and the CPU baseline")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
@@ -335,7 +368,7 @@ def main():
     barrier()
     if rank == 0:
         sampler.start()
-    res = time_workload(torch, dp, wl_run, args.steps, args.warmup, use_graph=not args.no_graph)
+    res = time_workload(torch, dp, wl_run, args.steps, args.warmup, use_graph=not args.no_graph, overlap=not args.no_overlap)
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     e2e = time_e2e(torch, dp, wl_run, max(3, min(args.steps, 100)), 3)
@@ -358,10 +391,14 @@ def main():
         "tokens_per_step": tokens / args.steps / world,
         "gpu_launches": res["launches"],
         "launch_mode": (f"CUDA graph of {RESTORE_EVERY} steps replayed" if res["graph"] else "one host call per library call"),
+        "step_mode": ({"side_by_side": True, "attention_sms": res["attn_sms"], "lm_head_sms": "the rest",
+                       "chosen": "un-timed sweep before the timed region (us/step by attention SMs; 0 = in order)",
+                       "sweep_us": res["sweep_us"]} if res["attn_sms"] else
+                      {"side_by_side": False, "sweep_us": res["sweep_us"]}),
         "clocks": clocks,
         "e2e": e2e,
         "roofline": {"bound": "hbm", "kernel": "lmhead_umma_kernel (sdlm_lmhead_confidence: stripe kernel + merge of the stripes)",
-                     "timing": "CUDA events around the call on its stream, mean over a second pass of the timed steps",
+                     "timing": "CUDA events around the call on its stream (the call alone on all SMs), mean over the same steps run as three calls just before the timed region",
                      "achieved": lm_gbs, "peak": peak, "unit": "GB/s", "frac": lm_gbs / peak,
                      "peak_source": peak_src, "traffic": LMHEAD_NCU_TRAFFIC if wl.name == "cfg2_3b_b32_d4" else None,
                      "traffic_source": "dram__bytes_read.sum + dram__bytes_write.sum of one launch, profiles/lmhead_umma_and_block_attn_umma__cfg2_d4.md",
@@ -378,9 +415,11 @@ def main():
             del dp
             torch.cuda.empty_cache()
             dp8 = DeviceProblem(wl8, keep_prefix=False)
-            r8 = time_workload(torch, dp8, wl8, max(5, min(args.steps, 200)), 3)
+            r8 = time_workload(torch, dp8, wl8, max(8, min(args.steps, 200)), 3, use_graph=not args.no_graph,
+                               overlap=not args.no_overlap)
             line["extra"] = {wl8.name: {"value": r8["tokens"] / (r8["ms_total"] * 1e-3), "unit": UNIT,
-                                        "ms_per_step": r8["ms_per_step"], "lm_ms": r8["lm_ms"], "attn_ms": r8["attn_ms"]}}
+                                        "ms_per_step": r8["ms_per_step"], "lm_ms": r8["lm_ms"], "attn_ms": r8["attn_ms"],
+                                        "attention_sms": r8["attn_sms"]}}
             del dp8
         n_seqs = min(wl.batch, 32)
         tok, dt = oracle_sample(wl, n_seqs, repeats=2)
