@@ -214,7 +214,10 @@ sdlm_status sdlm_device_status(sdlm_ctx* ctx, int32_t* host_out, int32_t clear, 
 /* ---- whole step on device memory: (a) + (b) + (c) in one call, same arguments and results as the
  * three calls made one after the other (Sec. 3.2: one forward pass, then Decode).  The library
  * knows here that the LM head reads nothing attention writes, so with SDLM_OPT_STEP_OVERLAP it
- * may overlap the two on the GPU; `hidden` and `w_lm` must not alias `attn_out`.  All pointers are DEVICE
+ * may overlap the two on the GPU; `hidden` and `w_lm` must not alias `attn_out`.  With that option the
+ * LM-head kernel may also begin to read `hidden` and `w_lm` while work enqueued on the stream before
+ * this call (the previous step's commit, say) is still running: their contents must be final when the
+ * call is made, not the pending output of earlier work on the stream.  All pointers are DEVICE
  * memory and required (seq_ids may be NULL).
  * Errors: as the three calls. */
 sdlm_status sdlm_decode_step(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, float tau,

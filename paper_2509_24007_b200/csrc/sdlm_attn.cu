@@ -49,6 +49,7 @@ struct AttnParams {
   int batch, D, Hq, Hkv, G, mpps, num_pages, n_stages;
   int min_range;  // shortest range of positions worth a CTA of its own
   int item_cost;  // what starting a (sequence, KV head) pair costs a CTA, in tiles (see ItemWalk)
+  int release_first;  // let the next kernel on the stream start before this one has waited for the one before it
 };
 
 // 8 warps; 12 when 64 stacked query rows need a second set of softmax warps
@@ -248,8 +249,13 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     ptx::tmem_alloc(tmem_slot, TMEM_COLS);
     ptx::tmem_relinquish();
   }
-  ptx::grid_dep_wait();    // lengths, page table and pool are written by the kernels before this one
-  ptx::grid_dep_launch();  // only now: a successor that does not wait itself may then rely on them too
+  // Lengths, page table and pool are written by the kernels before this one.  The next kernel is let go
+  // only after the wait, so that a successor that does not wait itself may rely on them too; the
+  // side-by-side step lets its LM-head kernel go first: that kernel reads nothing a predecessor wrote
+  // and takes its own wait before it writes.
+  if (p.release_first) ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
+  if (!p.release_first) ptx::grid_dep_launch();
 
   // exclusive prefix sum of (pages + 1) per batch row
   if (warp == 0) {
@@ -868,6 +874,7 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
   p.mpps = c.max_pages_per_seq; p.num_pages = c.num_pages; p.n_stages = 0;
   p.item_cost = ctx->attn_item_cost;
   p.min_range = ctx->attn_min_range;
+  p.release_first = cta_cap > 0 ? 1 : 0;
   // the kernel's tile arithmetic is 32-bit: (tiles of the launch) x (CTAs) must stay below 2^31
   if ((long long)batch * (c.max_pages_per_seq + 1 + ctx->attn_item_cost) * c.n_kv_heads > 13000000ll)
     return cudaErrorInvalidConfiguration;

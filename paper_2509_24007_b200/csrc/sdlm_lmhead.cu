@@ -283,6 +283,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&acc_empty[as]);
     }
+    // started without waiting: the merge kernel of an earlier call may still be reading the partials
+    if (p.wait_at_end) ptx::grid_dep_wait();
 #pragma unroll
     for (int r = 0; r < R; ++r) {
       const int row = r * 128 + q * 32 + lane;
