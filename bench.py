@@ -227,10 +227,22 @@ def time_workload(torch, dp, wl, steps, warmup, n_blocks=4, use_graph=True, over
     if overlap:
         sms = torch.cuda.get_device_properties(sd.device).multi_processor_count
         a0 = int(round(sms * at_ms / (at_ms + lm_ms)))
-        for a in [0] + sorted({min(max(a0 + d, 1), sms - 1) for d in (-8, -6, -4, -2, 0, 2, 4, 6, 8)}):
-            sd.set_option(OPT_STEP_OVERLAP, a)
-            run(RESTORE_EVERY, warmup)
-            sweep[a] = min(timed(RESTORE_EVERY * 3, warmup) for _ in range(2))
+        def try_sms(a):
+            if a not in sweep and (a == 0 or 1 <= a < sms):
+                sd.set_option(OPT_STEP_OVERLAP, a)
+                run(RESTORE_EVERY, warmup)
+                sweep[a] = min(timed(RESTORE_EVERY * 3, warmup) for _ in range(2))
+        for a in [0] + [a0 + d for d in (-8, -6, -4, -2, 0, 2, 4, 6, 8)]:
+            try_sms(a)
+        for _ in range(4):   # the best at an end of the range tried: look further that way
+            split = {a: t for a, t in sweep.items() if a > 0}
+            best = min(split, key=split.get)
+            if best == min(split):
+                for d in (2, 4, 6): try_sms(best - d)
+            elif best == max(split):
+                for d in (2, 4, 6): try_sms(best + d)
+            else:
+                break
         a_sms = min(sweep, key=sweep.get)
     sd.set_option(OPT_STEP_OVERLAP, a_sms)
     run(max(warmup, RESTORE_EVERY), 0)
@@ -274,7 +286,7 @@ def time_workload(torch, dp, wl, steps, warmup, n_blocks=4, use_graph=True, over
     assert int(sd.device_status()[0]) == 0, "device status set during the timed region"
     return {"ms_total": ms, "ms_per_step": ms / steps, "tokens": tokens, "lm_ms": lm_ms,
             "attn_ms": at_ms, "launches": launches, "graph": graph is not None, "attn_sms": a_sms,
-            "sweep_us": {str(k): round(v * 1e3, 1) for k, v in sweep.items()}}
+            "sweep_us": {str(k): round(v * 1e3, 1) for k, v in sorted(sweep.items())}}
 
 
 def time_e2e(torch, dp, wl, steps, warmup, n_blocks=4):
