@@ -242,7 +242,8 @@ sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const
 /* Tuning / test knobs (the paper has no counterpart).  SDLM_OPT_LMHEAD_KERNEL: which stripe kernel
  * sdlm_lmhead_confidence uses: 0 = chosen from the shape (default), 1 = warp-level mma.sync
  * kernel, 2 = tcgen05 / TMA kernel (the call then fails with UNSUPPORTED for rows > 256 or
- * |V| < 16).  SDLM_OPT_STEP_OVERLAP: A in 0..SMs-1.  With A > 0 sdlm_decode_step /
+ * |V| < 16), 3 = as 2 but with one thread block per tile also for 129..256 rows, where 0 and 2 let
+ * two thread blocks share a tile.  SDLM_OPT_STEP_OVERLAP: A in 0..SMs-1.  With A > 0 sdlm_decode_step /
  * sdlm_decode_step_host run attention on A SMs and the LM-head kernel at the same time on the
  * other SMs (the work is split over fewer thread blocks each, so results agree to rounding, not
  * bit for bit; default 0: one after the other on all SMs).

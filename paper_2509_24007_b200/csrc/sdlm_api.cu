@@ -436,7 +436,7 @@ extern "C" sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t v
   if (!ctx) return SDLM_ERR_INVALID_ARG;
   switch (opt) {
     case SDLM_OPT_LMHEAD_KERNEL:
-      if (value < 0 || value > 2) return SDLM_ERR_INVALID_ARG;
+      if (value < 0 || value > 3) return SDLM_ERR_INVALID_ARG;
       ctx->lmhead_path = value;
       return SDLM_OK;
     case SDLM_OPT_ATTN_ITEM_COST:

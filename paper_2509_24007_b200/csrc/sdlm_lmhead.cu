@@ -77,23 +77,35 @@ __device__ __forceinline__ void lm_timeout(DevHeader* hdr, int where) {
   }
 }
 
-// Folds 16 consecutive logits (vocab indices n0 .. n0+15, those >= n_end ignored) into a row's statistics.
-__device__ __forceinline__ void fold16(const uint32_t (&v)[16], int n0, int n_end, Stat& st) {
-  float z[16];
+// Folds NC consecutive logits (vocab indices n0 .. n0+NC-1, those >= n_end ignored) into a row's statistics.
+// An epilogue warp has at most one other warp on its scheduler to hide latencies behind, so the work
+// is arranged as few, wide dependency chains: one maximum and one rescale per call, then the
+// exponentials with `kChains` independent accumulators.  Per element that leaves the exponent
+// argument, the exponential and two accumulations, the three FP32 ones as packed two-wide operations:
+// sum e and sum e*z are accumulated, and sum e*(z-m) = sum e*z - m * sum e is formed once per call.
+template <int NC>
+__device__ __forceinline__ void fold(const uint32_t (&v)[NC], int n0, int n_end, Stat& st) {
+  static_assert(NC % 16 == 0, "whole 16-column groups");
+  float z[NC];
 #pragma unroll
-  for (int i = 0; i < 16; ++i) z[i] = __uint_as_float(v[i]);
-  if (n0 + 16 > n_end) {
+  for (int i = 0; i < NC; ++i) z[i] = __uint_as_float(v[i]);
+  if (n0 + NC > n_end) {
 #pragma unroll
-    for (int i = 0; i < 16; ++i)
+    for (int i = 0; i < NC; ++i)
       if (n0 + i >= n_end) z[i] = kNegInit;
   }
-  float cm = z[0];
+  float cm = kNegInit;
 #pragma unroll
-  for (int i = 1; i < 16; ++i) cm = fmaxf(cm, z[i]);
+  for (int g = 0; g < NC; g += 16) {
+    float gm = ptx::max3(ptx::max3(z[g], z[g + 1], z[g + 2]), ptx::max3(z[g + 3], z[g + 4], z[g + 5]),
+                         ptx::max3(z[g + 6], z[g + 7], z[g + 8]));
+    gm = ptx::max3(gm, ptx::max3(z[g + 9], z[g + 10], z[g + 11]), ptx::max3(z[g + 12], z[g + 13], z[g + 14]));
+    cm = ptx::max3(cm, gm, z[g + 15]);
+  }
   if (cm > st.m) {  // new running maximum: remember its first position, rescale the sums
-    int first = 15;
+    int first = NC - 1;
 #pragma unroll
-    for (int i = 14; i >= 0; --i)
+    for (int i = NC - 2; i >= 0; --i)
       if (z[i] == cm) first = i;
     st.idx = n0 + first;
     const float dm = st.m - cm;
@@ -102,17 +114,34 @@ __device__ __forceinline__ void fold16(const uint32_t (&v)[16], int n0, int n_en
     st.S = a * st.S;
     st.m = cm;
   }
-  const float m_l2 = st.m * kLog2e;
-  float S = 0.f, T = 0.f;
+  constexpr int kChains = NC >= 32 ? 4 : 2;
+  const float nm = -st.m * kLog2e;
+  const uint64_t nm2 = ptx::pack2(nm, nm), l2 = ptx::pack2(kLog2e, kLog2e);
+  uint64_t S2[kChains], U2[kChains];
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const float e = ptx::ex2(fmaf(z[i], kLog2e, -m_l2));
-    S += e;
-    T = fmaf(e, z[i] - st.m, T);
+  for (int c = 0; c < kChains; ++c) S2[c] = U2[c] = ptx::pack2(0.f, 0.f);
+#pragma unroll
+  for (int i = 0; i < NC; i += 2) {
+    const uint64_t zz = ptx::pack2(z[i], z[i + 1]);
+    float a0, a1;
+    ptx::unpack2(ptx::fma2(zz, l2, nm2), a0, a1);
+    const uint64_t ee = ptx::pack2(ptx::ex2(a0), ptx::ex2(a1));
+    S2[(i / 2) % kChains] = ptx::add2(S2[(i / 2) % kChains], ee);
+    U2[(i / 2) % kChains] = ptx::fma2(ee, zz, U2[(i / 2) % kChains]);
   }
+#pragma unroll
+  for (int c = 1; c < kChains; ++c) {
+    S2[0] = ptx::add2(S2[0], S2[c]);
+    U2[0] = ptx::add2(U2[0], U2[c]);
+  }
+  float s0, s1, u0, u1;
+  ptx::unpack2(S2[0], s0, s1);
+  ptx::unpack2(U2[0], u0, u1);
+  const float S = s0 + s1;
   st.S += S;
-  st.T += T;
+  st.T += fmaf(-st.m, S, u0 + u1);
 }
+__device__ __forceinline__ void fold16(const uint32_t (&v)[16], int n0, int n_end, Stat& st) { fold<16>(v, n0, n_end, st); }
 
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
   asm volatile(
@@ -301,6 +330,201 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
   }
   // Started without waiting for the kernel before it: do not finish before that kernel has, so that
   // whatever follows on the stream still sees both completed.
+  if (p.wait_at_end) ptx::grid_dep_wait();
+}
+
+// ---------------------------------------------------------------------------------------------
+// tcgen05 stripe kernel for 129..256 hidden-state rows: two CTAs share one 256-row x 2N-column tile
+// ---------------------------------------------------------------------------------------------
+// With more than 128 rows the single-CTA kernel needs the whole 256-row hidden slab again for every
+// N <= 256 vocabulary rows (about 2.2 bytes into the SM per byte of W) and its one accumulator set
+// leaves the epilogue of both row blocks exposed.  Here a cluster of two CTAs works on one tile of
+// 256 rows x 2N vocabulary entries (tcgen05 cta_group::2, M = 256): each CTA stages only its own 128
+// hidden rows and half of each of the two N-row slabs of W per K step (1.5 bytes per byte of W), holds
+// its rows' two accumulators (2 x 256 columns of its tensor memory) and folds them in its own warps.
+// The first CTA of the pair issues the MMAs; the copies of both CTAs are counted on its `full`
+// barriers, and tcgen05.commit reports to the `empty` / `acc_full` barriers of both.  The accumulators
+// fill the tensor memory, so the next tile's MMAs wait for the epilogue: eight epilogue warps (four per
+// accumulator, two per scheduler so that one hides the other's latencies) keep that wait short, and
+// each accumulator's columns leave their own partial record (2 per pair and row).
+constexpr int kPairThreads = 320;  // warp 0 producer, warp 1 MMA + TMEM, warps 2..5 / 6..9 epilogue of accumulator 0 / 1
+__global__ void __launch_bounds__(kPairThreads, 1)
+    lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_w,
+                       const LmParams p, int n_stages) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int N = p.bn;                          // vocabulary rows per MMA; a tile is two of them
+  const int w_half_bytes = (N / 2) * kBK * 2;  // this CTA's part of one N-row slab
+  const int stage_bytes = kATileBytes + 2 * w_half_bytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)n_stages * stage_bytes);
+  uint64_t* empty = full + n_stages;
+  uint64_t* acc_full = empty + n_stages;
+  uint64_t* acc_empty = acc_full + 1;
+  uint64_t* drain = acc_empty + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+  volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t cta = ptx::cluster_ctarank();  // 0 issues the MMAs
+  ptx::grid_dep_launch();
+
+  // the pair's vocabulary stripe, in groups of 32 rows
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int groups = (p.V + 31) / 32;
+  const int g0 = (int)((long long)pair * groups / n_pairs);
+  const int g1 = (int)((long long)(pair + 1) * groups / n_pairs);
+  const int n_begin = g0 * 32, n_end = min(p.V, g1 * 32);
+  const int n_tiles = (n_end - n_begin + 2 * N - 1) / (2 * N);
+  const int KC = (p.H + kBK - 1) / kBK;
+
+  if (tid == 0) {
+    for (int s = 0; s < n_stages; ++s) {
+      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&empty[s], 1);
+    }
+    ptx::mbar_init(acc_full, 1);
+    ptx::mbar_init(acc_empty, 16);  // the eight epilogue warps of each CTA
+    ptx::mbar_init(drain, 1);
+    *abort = 0;
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmap_h);
+    ptx::prefetch_tmap(&tmap_w);
+  }
+  __syncthreads();
+  if (warp == 1) {  // the same warp in both CTAs: the allocation is one operation of the pair
+    ptx::tmem_alloc_pair(tmem_slot, 512);
+    ptx::tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before();
+  ptx::cluster_sync_all();  // barriers of both CTAs exist before anything is counted on them
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  if (!p.wait_at_end) ptx::grid_dep_wait();
+
+  if (warp == 0) {
+    if (lane == 0) {  // ---- TMA producer (both CTAs; completion counted in the first CTA)
+      uint32_t it = 0;
+      bool ok = true;
+      const uint32_t full0 = ptx::mapa_u32(ptx::smem_u32(full), 0);
+      const uint32_t tx_bytes = 2u * (uint32_t)stage_bytes;
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const int n0 = n_begin + t * 2 * N + (int)cta * (N / 2);
+        for (int kc = 0; kc < KC; ++kc, ++it) {
+          const int s = it % n_stages;
+          if (it >= (uint32_t)n_stages && !ptx::mbar_wait_cluster(&empty[s], ((it / n_stages) & 1) ^ 1, abort)) {
+            ok = false;
+            break;
+          }
+          uint8_t* st = smem + (size_t)s * stage_bytes;
+          if (cta == 0) ptx::mbar_arrive_expect_tx(&full[s], tx_bytes);
+          const uint32_t bar = full0 + (uint32_t)s * 8u;
+          ptx::tma_load_2d_pair(st, &tmap_h, kc * kBK, (int)cta * 128, bar);
+          ptx::tma_load_2d_pair(st + kATileBytes, &tmap_w, kc * kBK, n0, bar);
+          ptx::tma_load_2d_pair(st + kATileBytes + w_half_bytes, &tmap_w, kc * kBK, n0 + N, bar);
+        }
+      }
+      if (!ok || *abort) {  // winding down: let the copies already issued land before the CTA goes away
+        lm_timeout(p.hdr, 6);
+        if (cta == 0) {
+          const uint32_t first = it > (uint32_t)n_stages ? it - n_stages : 0;
+          for (uint32_t j = first; j < it; ++j) ptx::mbar_wait_brief(&full[j % n_stages], (j / n_stages) & 1);
+        } else {
+          for (int i = 0; i < 256; ++i) __nanosleep(1000);  // its copies are counted in the other CTA
+        }
+      }
+    }
+    __syncwarp();  // the warp arrives at the closing barrier as a whole
+  } else if (warp == 1) {
+    if (lane == 0 && cta == 0) {  // ---- MMA issuer of the pair
+      // instruction descriptor: D fp32, A and B bf16, both K-major, N, M = 256 over the two CTAs
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((256u >> 4) << 24);
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        // one accumulator set: both CTAs' epilogues must have read tile t-1
+        if (t > 0 && !ptx::mbar_wait_cluster(acc_empty, (uint32_t)(t - 1) & 1u, abort)) {
+          ok = false;
+          break;
+        }
+        ptx::tc_fence_after();
+        for (int kc = 0; kc < KC; ++kc, ++it) {
+          const int s = it % n_stages;
+          if (!ptx::mbar_wait_cluster(&full[s], (it / n_stages) & 1, abort)) {
+            ok = false;
+            break;
+          }
+          ptx::tc_fence_after();
+          const uint32_t a_addr = ptx::smem_u32(smem + (size_t)s * stage_bytes);
+          const uint32_t b_addr = a_addr + kATileBytes;
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+#pragma unroll
+            for (int k = 0; k < kBK / 16; ++k)
+              ptx::umma_bf16_ss_pair(tmem_base + (uint32_t)(j * 256), umma_smem_desc(a_addr + k * 32),
+                                     umma_smem_desc(b_addr + j * w_half_bytes + k * 32), idesc, (kc | k) ? 1u : 0u);
+          }
+          ptx::umma_commit_pair(&empty[s], 3);  // the stage is reusable in both CTAs once these MMAs have read it
+        }
+        if (ok) ptx::umma_commit_pair(acc_full, 3);  // both CTAs' accumulators complete
+      }
+      if (!ok) {  // winding down: the MMAs already issued must finish before TMEM and smem are released
+        lm_timeout(p.hdr, 7);
+        ptx::umma_commit_pair_local(drain);
+        ptx::mbar_wait_brief(drain, 0);
+      }
+    }
+    __syncwarp();
+  } else {  // ---- epilogue: TMEM lane = hidden-state row cta*128 + lane; warps 2..5 take accumulator 0, 6..9 accumulator 1
+    const int q = warp & 3;  // TMEM lane quarter this warp may touch
+    const int j = warp >= 6 ? 1 : 0;
+    Stat st = stat_empty();
+    const uint32_t acc_empty0 = ptx::mapa_u32(ptx::smem_u32(acc_empty), 0);
+    const int n_chunks = N / 16;
+    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(j * 256);
+    for (int t = 0; t < n_tiles; ++t) {
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait_cluster(acc_full, (uint32_t)t & 1u, abort))) {
+        if (lane == 0) lm_timeout(p.hdr, 8);
+        break;
+      }
+      ptx::tc_fence_after();
+      const int n0 = n_begin + t * 2 * N + j * N;
+      // 32 columns per load and fold, the next load in flight meanwhile; an odd last 16 on their own
+      const int n_u = N / 32;
+      uint32_t a[32], b[32];
+      if (n_u > 0) ptx::tmem_ld_32x32b_x32(taddr, a);
+      for (int u = 0; u < n_u; u += 2) {
+        ptx::tmem_ld_wait();
+        if (u + 1 < n_u) ptx::tmem_ld_32x32b_x32(taddr + (u + 1) * 32, b);
+        if (n0 + u * 32 < n_end) fold<32>(a, n0 + u * 32, n_end, st);
+        if (u + 1 < n_u) {
+          ptx::tmem_ld_wait();
+          if (u + 2 < n_u) ptx::tmem_ld_32x32b_x32(taddr + (u + 2) * 32, a);
+          if (n0 + (u + 1) * 32 < n_end) fold<32>(b, n0 + (u + 1) * 32, n_end, st);
+        }
+      }
+      for (int c = n_u * 2; c < n_chunks; ++c) {
+        uint32_t v[16];
+        tmem_ld16(taddr + c * 16, v);
+        ptx::tmem_ld_wait();
+        if (n0 + c * 16 < n_end) fold<16>(v, n0 + c * 16, n_end, st);
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive_cluster(acc_empty0);
+    }
+    // started without waiting: the merge kernel of an earlier call may still be reading the partials
+    if (p.wait_at_end) ptx::grid_dep_wait();
+    const int row = (int)cta * 128 + q * 32 + lane;
+    if (row < p.rows)
+      p.partials[(size_t)(2 * pair + j) * p.rows_pad + row] = make_float4(st.m, st.S, st.T, __int_as_float(st.idx));
+  }
+  // Neither CTA may go while the other can still reach its shared memory or barriers.
+  ptx::tc_fence_before();
+  ptx::cluster_sync_all();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc_pair(tmem_base, 512);
+  }
   if (p.wait_at_end) ptx::grid_dep_wait();
 }
 
@@ -513,6 +737,8 @@ cudaError_t setup_lmhead(sdlm_ctx* ctx) {
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(lmhead_umma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmemBudget + 2048);
   if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(lmhead_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmemBudget + 2048);
+  if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(lmhead_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               kMmaStages * kMmaStageBytes + 128);
 }
@@ -536,12 +762,39 @@ static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden,
   cudaError_t le = cudaSuccess;
 
   const bool use_umma = ctx->lmhead_path != 1 && rows <= 256 && c.vocab >= 16;
-  if (ctx->lmhead_path == 2 && !use_umma) return SDLM_ERR_UNSUPPORTED;
-  if (use_umma) {
+  if (ctx->lmhead_path >= 2 && !use_umma) return SDLM_ERR_UNSUPPORTED;
+  int sm_avail = ctx->sm_count;
+  if (cta_cap > 0 && cta_cap < sm_avail) sm_avail = cta_cap;
+  // more than 128 rows: two CTAs per tile (lmhead_path 3 keeps the single-CTA kernel, for comparison)
+  const bool use_pair = use_umma && rows > 128 && ctx->lmhead_path != 3 && sm_avail >= 2 && c.vocab >= 32;
+  if (use_pair) {
+    const int groups = (c.vocab + 31) / 32;
+    int pairs = sm_avail / 2;
+    if (pairs > groups) pairs = groups;
+    if (2 * pairs > max_stripes) pairs = max_stripes / 2;  // two partial records per pair
+    const int gmax = (groups + pairs - 1) / pairs;
+    const int tiles = (gmax * 32 + 511) / 512;
+    p.bn = 16 * ((gmax + tiles - 1) / tiles);  // N of one MMA; a tile is 2N vocabulary rows
+    p.n_stripes = 2 * pairs;
+    const int stage_bytes = kATileBytes + p.bn * kBK * 2;
+    int n_stages = kUmmaSmemBudget / stage_bytes;
+    if (n_stages > 8) n_stages = 8;
+    CUtensorMap tm_h;
+    if (!make_tmap(&tm_h, hidden, rows, c.hidden, 128)) return SDLM_ERR_CUDA;
+    if (ctx->tmap_w_ptr != w_lm || ctx->tmap_w_rows != p.bn / 2) {
+      if (!make_tmap(reinterpret_cast<CUtensorMap*>(ctx->tmap_w), w_lm, c.vocab, c.hidden, p.bn / 2)) return SDLM_ERR_CUDA;
+      ctx->tmap_w_ptr = w_lm;
+      ctx->tmap_w_rows = p.bn / 2;
+    }
+    const CUtensorMap& tm_w = *reinterpret_cast<const CUtensorMap*>(ctx->tmap_w);
+    const size_t smem = (size_t)n_stages * stage_bytes + 1024 + 512;
+    le = launch_overlapped_cluster(lmhead_pair_kernel, dim3(2 * pairs), dim3(kPairThreads), smem, st, 2, tm_h, tm_w, p,
+                                   n_stages);
+  } else if (use_umma) {
     const int groups = (c.vocab + 15) / 16;
     int n_cta = groups < ctx->sm_count ? groups : ctx->sm_count;
     if (n_cta > max_stripes) n_cta = max_stripes;
-    if (cta_cap > 0 && cta_cap < n_cta) n_cta = cta_cap;
+    if (sm_avail < n_cta) n_cta = sm_avail;
     const int gmax = (groups + n_cta - 1) / n_cta;
     const int tiles = (gmax * 16 + 255) / 256;
     p.bn = 16 * ((gmax + tiles - 1) / tiles);
