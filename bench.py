@@ -226,7 +226,7 @@ def time_workload(torch, dp, wl, steps, warmup, n_blocks=4, use_graph=True, over
     a_sms, sweep = 0, {}
     if overlap:
         sms = torch.cuda.get_device_properties(sd.device).multi_processor_count
-        a0 = int(round(sms * at_ms / (at_ms + lm_ms)))
+        a0 = 2 * int(round(sms * at_ms / (at_ms + lm_ms) / 2))   # even: with more than 128 rows both kernels take whole SM pairs
         def try_sms(a):
             if a not in sweep and (a == 0 or 1 <= a < sms):
                 sd.set_option(OPT_STEP_OVERLAP, a)

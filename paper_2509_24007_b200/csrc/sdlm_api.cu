@@ -625,8 +625,9 @@ static sdlm_status decode_step_device(sdlm_ctx* ctx, int32_t batch, int32_t D, c
   sdlm_status s = check_batch(ctx, batch, D);
   if (s != SDLM_OK) return s;
   const int a_sms = ctx->overlap_lmhead;
-  if (launch_block_attn(ctx, batch, D, seq_ids, q, k_blk, v_blk, attn_out, static_cast<cudaStream_t>(stream), a_sms) !=
-      cudaSuccess)
+  // with more than 128 rows the LM head runs as CTA pairs: attention then takes whole pairs of SMs
+  if (launch_block_attn(ctx, batch, D, seq_ids, q, k_blk, v_blk, attn_out, static_cast<cudaStream_t>(stream), a_sms,
+                        a_sms > 0 && batch * D > 128) != cudaSuccess)
     return SDLM_ERR_CUDA;
   if (!hidden || !w_lm || !token || !p_top1 || !entropy) return SDLM_ERR_INVALID_ARG;
   if (!aligned16(hidden) || !aligned16(w_lm)) return SDLM_ERR_INVALID_ARG;

@@ -825,7 +825,7 @@ static int attn_fixed_smem(int batch) {
 }
 
 template <int HD, int NQ>
-static cudaError_t attn_launch_one(sdlm_ctx* ctx, AttnParams& p, cudaStream_t st, int cta_cap) {
+static cudaError_t attn_launch_one(sdlm_ctx* ctx, AttnParams& p, cudaStream_t st, int cta_cap, bool whole_tpcs) {
   const int pair_b = 2 * (2 * kPageSize * HD * 2);
   int n = (kAttnSmemLimit - attn_fixed_smem<HD, NQ>(p.batch)) / (pair_b + 16);
   if (n > 6) n = 6;
@@ -834,7 +834,13 @@ static cudaError_t attn_launch_one(sdlm_ctx* ctx, AttnParams& p, cudaStream_t st
   const size_t smem = (size_t)attn_fixed_smem<HD, NQ>(p.batch) + (size_t)n * (pair_b + 16);
   int n_cta = ctx->sm_count < kAttnMaxCtas ? ctx->sm_count : kAttnMaxCtas;
   if (cta_cap > 0 && cta_cap < n_cta) n_cta = cta_cap;
-  const cudaError_t e = launch_overlapped(block_attn_umma_kernel<HD, NQ>, dim3(n_cta), dim3(attn_threads(NQ)), smem, st, p);
+  // Beside a kernel that runs as CTA pairs, attention is launched as clusters of two as well (it uses
+  // nothing of the cluster): its thread blocks then fill whole pairs of SMs instead of one SM of many pairs.
+  if (whole_tpcs && n_cta >= 2) n_cta &= ~1;
+  const cudaError_t e =
+      whole_tpcs && n_cta >= 2
+          ? launch_overlapped_cluster(block_attn_umma_kernel<HD, NQ>, dim3(n_cta), dim3(attn_threads(NQ)), smem, st, 2, p)
+          : launch_overlapped(block_attn_umma_kernel<HD, NQ>, dim3(n_cta), dim3(attn_threads(NQ)), smem, st, p);
   ctx->launches++;
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -854,7 +860,8 @@ cudaError_t setup_attn(sdlm_ctx* ctx) {
 }
 
 cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, const void* q,
-                              const void* k_blk, const void* v_blk, void* out, cudaStream_t st, int cta_cap) {
+                              const void* k_blk, const void* v_blk, void* out, cudaStream_t st, int cta_cap,
+                              bool whole_tpcs) {
   const sdlm_config& c = ctx->cfg;
   AttnParams p;
   p.pool = reinterpret_cast<const __nv_bfloat16*>(ctx->pool);
@@ -880,8 +887,10 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
     return cudaErrorInvalidConfiguration;
   const bool wide = ctx->group * D > 32;  // stacked query rows padded to 64, else to 32
   if (c.head_dim == 128)
-    return wide ? attn_launch_one<128, 64>(ctx, p, st, cta_cap) : attn_launch_one<128, 32>(ctx, p, st, cta_cap);
-  return wide ? attn_launch_one<64, 64>(ctx, p, st, cta_cap) : attn_launch_one<64, 32>(ctx, p, st, cta_cap);
+    return wide ? attn_launch_one<128, 64>(ctx, p, st, cta_cap, whole_tpcs)
+                : attn_launch_one<128, 32>(ctx, p, st, cta_cap, whole_tpcs);
+  return wide ? attn_launch_one<64, 64>(ctx, p, st, cta_cap, whole_tpcs)
+              : attn_launch_one<64, 32>(ctx, p, st, cta_cap, whole_tpcs);
 }
 
 }  // namespace sdlm
