@@ -230,7 +230,10 @@ sdlm_status sdlm_decode_step(sdlm_ctx* ctx, int32_t batch, int32_t D, const int3
  * best speed), and seq_ids (HOST int32 [batch] or NULL), to workspace staging; runs the three
  * calls on `stream`; copies attn_out [batch,D,Hq,d] bf16, token / p_top1 / entropy [batch*D],
  * accepted_len [batch] and out_tokens [batch,D] back to HOST (any may be NULL to skip) and
- * synchronises `stream` before returning.  w_lm stays a DEVICE pointer (model state).
+ * synchronises `stream` before returning.  A result buffer that is page-locked host memory the GPU
+ * can address (cudaHostAlloc / cudaHostRegister) is written by the kernels directly, without a
+ * copy after the step; its contents are defined once the call has returned.  w_lm stays a DEVICE
+ * pointer (model state).
  * Errors: as the three calls, plus CUDA. */
 sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids_host,
                                   float tau, sdlm_conf_mode mode, const void* q_host, const void* k_blk_host,

@@ -190,6 +190,11 @@ struct CommitParams {
   const __nv_bfloat16* v_blk;
   int32_t* accepted_len;
   int32_t* out_tokens;
+  // optional second copies of the per-row statistics this kernel reads (mapped host memory of the
+  // host-buffer step: written here, they need no copy after the step); any may be null
+  int32_t* token_copy;
+  float* p_top1_copy;
+  float* entropy_copy;
   float tau, inv_ln_vocab;
   int mode, batch, D, Hkv, d, mpps, num_pages;
 };
@@ -275,6 +280,11 @@ __global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitPar
   // my row
   const int g = s_mine[0], need = s_mine[1], alloc = s_mine[2], len = s_mine[3], state = s_mine[4];
   const int slot = p.seq_ids ? p.seq_ids[b] : b;
+  for (int k = tid; k < p.D; k += kCommitThreads) {
+    if (p.token_copy) p.token_copy[b * p.D + k] = p.token[b * p.D + k];
+    if (p.p_top1_copy) p.p_top1_copy[b * p.D + k] = p.p_top1[b * p.D + k];
+    if (p.entropy_copy) p.entropy_copy[b * p.D + k] = p.entropy[b * p.D + k];
+  }
   if (state != 0) {
     if (tid == 0) {
       p.accepted_len[b] = -1;
@@ -572,10 +582,17 @@ extern "C" sdlm_status sdlm_lmhead_confidence(sdlm_ctx* ctx, int32_t rows, const
                        static_cast<cudaStream_t>(stream));
 }
 
-extern "C" sdlm_status sdlm_accept_commit(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, float tau,
-                                          sdlm_conf_mode mode, const int32_t* token, const float* p_top1,
-                                          const float* entropy, const void* k_blk, const void* v_blk,
-                                          int32_t* accepted_len, int32_t* out_tokens, void* stream) {
+struct StatCopies {
+  int32_t* token = nullptr;
+  float* p_top1 = nullptr;
+  float* entropy = nullptr;
+};
+
+static sdlm_status accept_commit_launch(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, float tau,
+                                        sdlm_conf_mode mode, const int32_t* token, const float* p_top1,
+                                        const float* entropy, const void* k_blk, const void* v_blk,
+                                        int32_t* accepted_len, int32_t* out_tokens, const StatCopies& copies,
+                                        void* stream) {
   if (!ctx || !token || !p_top1 || !entropy || !k_blk || !v_blk || !accepted_len || !out_tokens)
     return SDLM_ERR_INVALID_ARG;
   if (!aligned16(k_blk) || !aligned16(v_blk)) return SDLM_ERR_INVALID_ARG;
@@ -590,6 +607,7 @@ extern "C" sdlm_status sdlm_accept_commit(sdlm_ctx* ctx, int32_t batch, int32_t 
   p.seq_ids = seq_ids; p.token = token; p.p_top1 = p_top1; p.entropy = entropy;
   p.k_blk = static_cast<const __nv_bfloat16*>(k_blk); p.v_blk = static_cast<const __nv_bfloat16*>(v_blk);
   p.accepted_len = accepted_len; p.out_tokens = out_tokens;
+  p.token_copy = copies.token; p.p_top1_copy = copies.p_top1; p.entropy_copy = copies.entropy;
   p.tau = tau;
   p.inv_ln_vocab = c.vocab > 1 ? (float)(1.0 / log((double)c.vocab)) : 0.0f;
   p.mode = (int)mode; p.batch = batch; p.D = D; p.Hkv = c.n_kv_heads; p.d = c.head_dim;
@@ -598,6 +616,14 @@ extern "C" sdlm_status sdlm_accept_commit(sdlm_ctx* ctx, int32_t batch, int32_t 
                                           static_cast<cudaStream_t>(stream), p);
   ctx->launches++;
   return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+}
+
+extern "C" sdlm_status sdlm_accept_commit(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, float tau,
+                                          sdlm_conf_mode mode, const int32_t* token, const float* p_top1,
+                                          const float* entropy, const void* k_blk, const void* v_blk,
+                                          int32_t* accepted_len, int32_t* out_tokens, void* stream) {
+  return accept_commit_launch(ctx, batch, D, seq_ids, tau, mode, token, p_top1, entropy, k_blk, v_blk, accepted_len,
+                              out_tokens, StatCopies{}, stream);
 }
 
 extern "C" sdlm_status sdlm_device_status(sdlm_ctx* ctx, int32_t* host_out, int32_t clear, void* stream) {
@@ -619,7 +645,7 @@ static sdlm_status decode_step_device(sdlm_ctx* ctx, int32_t batch, int32_t D, c
                                       sdlm_conf_mode mode, const void* q, const void* k_blk, const void* v_blk,
                                       const void* hidden, const void* w_lm, void* attn_out, int32_t* token,
                                       float* p_top1, float* entropy, int32_t* accepted_len, int32_t* out_tokens,
-                                      void* stream) {
+                                      const StatCopies& copies, void* stream) {
   if (!ctx || !q || !k_blk || !v_blk || !attn_out) return SDLM_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(attn_out)) return SDLM_ERR_INVALID_ARG;
   sdlm_status s = check_batch(ctx, batch, D);
@@ -635,8 +661,8 @@ static sdlm_status decode_step_device(sdlm_ctx* ctx, int32_t batch, int32_t D, c
                     static_cast<cudaStream_t>(stream), /*independent_of_predecessor=*/a_sms > 0,
                     a_sms > 0 ? ctx->sm_count - a_sms : 0);
   if (s != SDLM_OK) return s;
-  return sdlm_accept_commit(ctx, batch, D, seq_ids, tau, mode, token, p_top1, entropy, k_blk, v_blk, accepted_len,
-                            out_tokens, stream);
+  return accept_commit_launch(ctx, batch, D, seq_ids, tau, mode, token, p_top1, entropy, k_blk, v_blk, accepted_len,
+                              out_tokens, copies, stream);
 }
 
 extern "C" sdlm_status sdlm_decode_step(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, float tau,
@@ -646,7 +672,7 @@ extern "C" sdlm_status sdlm_decode_step(sdlm_ctx* ctx, int32_t batch, int32_t D,
                                         void* stream) {
   if (!ctx) return SDLM_ERR_INVALID_ARG;
   return decode_step_device(ctx, batch, D, seq_ids, tau, mode, q, k_blk, v_blk, hidden, w_lm, attn_out, token, p_top1,
-                            entropy, accepted_len, out_tokens, stream);
+                            entropy, accepted_len, out_tokens, StatCopies{}, stream);
 }
 
 extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids_host,
@@ -680,15 +706,39 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
   float* d_ent = reinterpret_cast<float*>(ws + L.st_ent);
   int32_t* d_acc = reinterpret_cast<int32_t*>(ws + L.st_acc);
   int32_t* d_out_tokens = reinterpret_cast<int32_t*>(ws + L.st_out_tokens);
+  // A result buffer in page-locked host memory that the GPU can address is written by the kernels
+  // themselves (attention's output rows during the step, the small per-row results by the commit
+  // kernel), which saves a copy after the step; any other host buffer is filled by a copy.
+  auto mapped = [](void* host_ptr) -> void* {
+    if (!host_ptr) return nullptr;
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, host_ptr) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    return a.type == cudaMemoryTypeHost ? a.devicePointer : nullptr;
+  };
+  void* m_attn = mapped(attn_out_host);
+  if (m_attn && !aligned16(m_attn)) m_attn = nullptr;
+  int32_t* m_acc = static_cast<int32_t*>(mapped(accepted_len_host));
+  int32_t* m_out_tokens = static_cast<int32_t*>(mapped(out_tokens_host));
+  StatCopies copies;
+  copies.token = static_cast<int32_t*>(mapped(token_host));
+  copies.p_top1 = static_cast<float*>(mapped(p_top1_host));
+  copies.entropy = static_cast<float*>(mapped(entropy_host));
   s = decode_step_device(ctx, batch, D, seq_ids, tau, mode, ws + L.st_q, ws + L.st_k, ws + L.st_v, ws + L.st_hidden, w_lm,
-                         ws + L.st_out, d_token, d_p, d_ent, d_acc, d_out_tokens, stream);
+                         m_attn ? m_attn : ws + L.st_out, d_token, d_p, d_ent, m_acc ? m_acc : d_acc,
+                         m_out_tokens ? m_out_tokens : d_out_tokens, copies, stream);
   if (s != SDLM_OK) return s;
-  if (attn_out_host) ok &= cudaMemcpyAsync(attn_out_host, ws + L.st_out, q_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  if (token_host) ok &= cudaMemcpyAsync(token_host, d_token, rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  if (p_top1_host) ok &= cudaMemcpyAsync(p_top1_host, d_p, rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  if (entropy_host) ok &= cudaMemcpyAsync(entropy_host, d_ent, rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  if (accepted_len_host) ok &= cudaMemcpyAsync(accepted_len_host, d_acc, (size_t)batch * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  if (out_tokens_host) ok &= cudaMemcpyAsync(out_tokens_host, d_out_tokens, rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (attn_out_host && !m_attn)
+    ok &= cudaMemcpyAsync(attn_out_host, ws + L.st_out, q_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (token_host && !copies.token) ok &= cudaMemcpyAsync(token_host, d_token, rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (p_top1_host && !copies.p_top1) ok &= cudaMemcpyAsync(p_top1_host, d_p, rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (entropy_host && !copies.entropy) ok &= cudaMemcpyAsync(entropy_host, d_ent, rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (accepted_len_host && !m_acc)
+    ok &= cudaMemcpyAsync(accepted_len_host, d_acc, (size_t)batch * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (out_tokens_host && !m_out_tokens)
+    ok &= cudaMemcpyAsync(out_tokens_host, d_out_tokens, rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   if (!ok || cudaStreamSynchronize(st) != cudaSuccess) return SDLM_ERR_CUDA;
   return SDLM_OK;
 }

@@ -151,7 +151,10 @@ def test_cfg4_long_prefix_multi_step_loop():
     print("cfg4 committed", total_ref, "tokens in", wl.steps, "steps; flagged", flagged)
 
 
-def test_decode_step_host_entry_matches_device_calls():
+@pytest.mark.parametrize("results", ["page-locked", "pageable", "mixed"])
+def test_decode_step_host_entry_matches_device_calls(results):
+    """Page-locked result buffers are written by the kernels themselves, pageable ones by copies after
+    the step: the host sees the same values either way, and entropy too."""
     wl = syn.CONFIGS["cfg0"].with_(batch=3, prefix_lo=10, prefix_hi=200)
     dp = DeviceProblem(wl)
     x = dp.block(0)
@@ -161,17 +164,21 @@ def test_decode_step_host_entry_matches_device_calls():
     dp.reset_cache()
     pin = lambda t: t.cpu().pin_memory()
     B, D, s = wl.batch, wl.block, wl.shape
-    attn = torch.empty((B, D, s.n_q_heads, s.head_dim), dtype=torch.bfloat16).pin_memory()
-    tok = torch.empty((B, D), dtype=torch.int32).pin_memory()
-    p = torch.empty((B, D), dtype=torch.float32).pin_memory()
-    ent = torch.empty((B, D), dtype=torch.float32).pin_memory()
-    acc = torch.empty(B, dtype=torch.int32).pin_memory()
-    out_tok = torch.empty((B, D), dtype=torch.int32).pin_memory()
+    def buf(shape, dtype, i):
+        t = torch.full(shape, -7, dtype=dtype)
+        locked = results == "page-locked" or (results == "mixed" and i % 2 == 0)
+        return t.pin_memory() if locked else t
+    attn = buf((B, D, s.n_q_heads, s.head_dim), torch.bfloat16, 0)
+    tok = buf((B, D), torch.int32, 1)
+    p = buf((B, D), torch.float32, 2)
+    ent = buf((B, D), torch.float32, 3)
+    acc = buf((B,), torch.int32, 4)
+    out_tok = buf((B, D), torch.int32, 5)
     dp.sd.decode_step_host(wl.tau, pin(x.q), pin(x.k_blk), pin(x.v_blk), pin(x.hidden), dp.w_lm, attn, tok, p, ent,
                            acc, out_tok)
     assert torch.equal(attn, ref.attn.cpu()) and torch.equal(tok, ref.token.cpu())
     assert torch.equal(p, ref.p_top1.cpu()) and torch.equal(acc, ref.accepted_len.cpu())
-    assert torch.equal(out_tok, ref.out_tokens.cpu())
+    assert torch.equal(out_tok, ref.out_tokens.cpu()) and torch.equal(ent, ref.entropy.cpu())
     t = dp.sd.kv_tables()
     assert np.array_equal(t["page_table"], t_ref["page_table"]) and np.array_equal(t["seq_len"], t_ref["seq_len"])
 
