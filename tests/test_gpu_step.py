@@ -32,12 +32,18 @@ def _compare_tables(dp, cache, sample_seqs=None):
         assert np.array_equal(pk.bits_from_bf16_tensor(k), ok) and np.array_equal(pk.bits_from_bf16_tensor(v), ov)
 
 
-def _one_step(dp, cache, tau, step=0, mode=orc.CONF_LOGIT, w64=None, attn_rows=None, report=None):
-    """Runs step `step` on both sides; returns (gpu outputs, oracle StepResult)."""
+def _one_step(dp, cache, tau, step=0, mode=orc.CONF_LOGIT, w64=None, attn_rows=None, report=None, attn_sms=None):
+    """Runs step `step` on both sides; returns (gpu outputs, oracle StepResult).  `attn_sms`: None = three
+    library calls; a number = one sdlm_decode_step call with that many SMs for attention beside the LM
+    head (0: in order), the launch configuration the benchmark times."""
     report = report if report is not None else []
     wl = dp.wl
     x = dp.block(step)
-    out = dp.step(x, tau, mode=mode)
+    if attn_sms is None:
+        out = dp.step(x, tau, mode=mode)
+    else:
+        dp.sd.set_option(OPT_STEP_OVERLAP, attn_sms)
+        out = dp.step(x, tau, mode=mode, fused=True)
     torch.cuda.synchronize()
     # oracle: attention over the cache as it was before the commit
     seqs = list(range(wl.batch)) if attn_rows is None else attn_rows
@@ -84,13 +90,16 @@ def test_cfg1_3b_single_sequence_tau_sweep():
     assert gammas == sorted(gammas, reverse=True)          # a higher threshold never accepts more
 
 
-@pytest.mark.parametrize("name", ["cfg2", "cfg2_d4"])
-def test_cfg2_3b_ragged_batch(name):
+@pytest.mark.parametrize("name,attn_sms", [("cfg2", None), ("cfg2_d4", None), ("cfg2", 36), ("cfg2_d4", 42), ("cfg2_d4", 0)])
+def test_cfg2_3b_ragged_batch(name, attn_sms):
+    """Full-size batch-32 step against the oracle: as three calls, and as the one call the benchmark
+    times (attention on 36 / 42 SMs beside the LM head; with D = 8 the LM head then runs as CTA pairs
+    and attention as clusters of two)."""
     wl = syn.CONFIGS[name]
     dp = DeviceProblem(wl)
     cache = oracle_cache(wl, dp.lengths, dp.num_pages, dp.mpps, dp.prefix)
     report = []
-    out, stats, res, n_bad = _one_step(dp, cache, wl.tau, 0, report=report)
+    out, stats, res, n_bad = _one_step(dp, cache, wl.tau, 0, report=report, attn_sms=attn_sms)
     print(name, "flagged:", report, "gamma hist:", np.bincount(res.accepted_len, minlength=wl.block + 1).tolist())
     _compare_if_in_sync(dp, cache, n_bad)
     assert 1.0 <= res.accepted_len.mean() <= wl.block
@@ -125,12 +134,16 @@ def test_cfg4_long_prefix_multi_step_loop():
     flagged = []
     for step in range(wl.steps):
         x = dp.block(step)
-        check_attn = step in (0, wl.steps // 2, wl.steps - 1)
+        check_attn = step in (0, wl.steps // 2, wl.steps // 2 + 1, wl.steps - 1)
         if check_attn:
             seqs = [0, wl.batch - 1]
             pk_, pv_ = zip(*[cache.gather_fast(b) for b in seqs])
             ref_attn = orc.block_attention(x.host.q[seqs], x.host.k_blk[seqs], x.host.v_blk[seqs], pk_, pv_)
-        dp.step(x, wl.tau, outs)
+        if step % 2:      # every other step as the one call the benchmark times, attention on 68 SMs beside the LM head
+            dp.sd.set_option(OPT_STEP_OVERLAP, 68)
+            dp.step(x, wl.tau, outs, fused=True)
+        else:
+            dp.step(x, wl.tau, outs)
         torch.cuda.synchronize()
         if check_attn:
             check_attention(pk.bits_from_bf16_tensor(outs.attn)[seqs], ref_attn)
