@@ -256,6 +256,30 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
   if (p.release_first) ptx::grid_dep_launch();
   ptx::grid_dep_wait();
   if (!p.release_first) ptx::grid_dep_launch();
+  // The start-up chain is lengths -> page table -> first tiles (and query rows), each a trip to DRAM
+  // that costs several microseconds under a concurrent weight stream.  Pulling the page table and the
+  // block's query / key / value rows towards L2 now, alongside the load of the lengths, takes the
+  // second trip out of the chain.  (Earlier, before the wait, is too early: the thread blocks may sit
+  // there for tens of microseconds while the weight stream turns L2 over.)
+  {
+    const size_t line = 128;
+    // with seq_ids the rows of the first `batch` slots may not be the ones used: harmless, they exist
+    const size_t lim_len = ((size_t)p.batch * 4 + line - 1) / line;
+    const size_t n_tab = ((size_t)p.batch * p.mpps * 4 + line - 1) / line;
+    const size_t n_q = ((size_t)p.batch * p.D * p.Hq * HD * 2 + line - 1) / line;
+    const size_t n_kv = ((size_t)p.batch * p.D * p.Hkv * HD * 2 + line - 1) / line;
+    const size_t total = lim_len + n_tab + n_q + 2 * n_kv;  // (the lengths too: one line, for the other thread blocks)
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + tid; i < total; i += (size_t)gridDim.x * blockDim.x) {
+      const char* a;
+      size_t k = i;
+      if (k < lim_len) a = reinterpret_cast<const char*>(p.seq_len) + k * line;
+      else if ((k -= lim_len) < n_tab) a = reinterpret_cast<const char*>(p.page_table) + k * line;
+      else if ((k -= n_tab) < n_q) a = reinterpret_cast<const char*>(p.q) + k * line;
+      else if ((k -= n_q) < n_kv) a = reinterpret_cast<const char*>(p.k_blk) + k * line;
+      else a = reinterpret_cast<const char*>(p.v_blk) + (k - n_kv) * line;
+      ptx::prefetch_l2(a);
+    }
+  }
 
   // exclusive prefix sum of (pages + 1) per batch row
   if (warp == 0) {
@@ -302,6 +326,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     Item it;
     Ring ring{0, 0};
     uint32_t issued = 0;  // groups so far
+    const uint64_t kv_policy = ptx::l2_evict_first_policy();  // cached tiles are read once per call
     bool ok = true;
     while (ok && walk_next(w, p, it)) {
       const int32_t* ptab = p.page_table + (size_t)it.slot * p.mpps;
@@ -328,8 +353,9 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
               const uint8_t* src = reinterpret_cast<const uint8_t*>(p.pool + kv_tile_offset(page, it.h, 0, p.Hkv, HD));
 #pragma unroll
               for (int kh = 0; kh < KH; ++kh)
-                ptx::bulk_g2s(st + kh * 2 * K_PANEL_B + j * K_PANEL_B, src + kh * K_PANEL_B, K_PANEL_B, &full[ring.stage]);
-              ptx::bulk_g2s(st + K_REGION_B + j * VT_B, src + KH * K_PANEL_B, VT_B, &full[ring.stage]);
+                ptx::bulk_g2s_hint(st + kh * 2 * K_PANEL_B + j * K_PANEL_B, src + kh * K_PANEL_B, K_PANEL_B,
+                                   &full[ring.stage], kv_policy);
+              ptx::bulk_g2s_hint(st + K_REGION_B + j * VT_B, src + KH * K_PANEL_B, VT_B, &full[ring.stage], kv_policy);
             }
             if (has_blk) {
               // The block's own tile is written by warp 6, which then gives the group's second

@@ -212,6 +212,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
     if (lane == 0) {  // ---- TMA producer
       uint32_t it = 0;
       bool ok = true;
+      const uint64_t w_policy = ptx::l2_evict_first_policy();  // W is read once per call
       for (int t = 0; t < n_tiles && ok; ++t) {
         const int n0 = n_begin + t * p.bn;
         for (int kc = 0; kc < KC; ++kc, ++it) {
@@ -224,7 +225,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
           ptx::mbar_arrive_expect_tx(&full[s], (uint32_t)(R * p.a_box_rows * kBK * 2 + w_tile_bytes));
 #pragma unroll
           for (int r = 0; r < R; ++r) ptx::tma_load_2d(st + r * kATileBytes, &tmap_h, kc * kBK, r * 128, &full[s]);
-          ptx::tma_load_2d(st + R * kATileBytes, &tmap_w, kc * kBK, n0, &full[s]);
+          ptx::tma_load_2d_hint(st + R * kATileBytes, &tmap_w, kc * kBK, n0, &full[s], w_policy);
         }
       }
       if (!ok || *abort) {  // winding down: let the copies already issued land before the CTA goes away
@@ -407,6 +408,7 @@ __global__ void __launch_bounds__(kPairThreads, 1)
       bool ok = true;
       const uint32_t full0 = ptx::mapa_u32(ptx::smem_u32(full), 0);
       const uint32_t tx_bytes = 2u * (uint32_t)stage_bytes;
+      const uint64_t w_policy = ptx::l2_evict_first_policy();  // W is read once per call
       for (int t = 0; t < n_tiles && ok; ++t) {
         const int n0 = n_begin + t * 2 * N + (int)cta * (N / 2);
         for (int kc = 0; kc < KC; ++kc, ++it) {
@@ -419,8 +421,8 @@ __global__ void __launch_bounds__(kPairThreads, 1)
           if (cta == 0) ptx::mbar_arrive_expect_tx(&full[s], tx_bytes);
           const uint32_t bar = full0 + (uint32_t)s * 8u;
           ptx::tma_load_2d_pair(st, &tmap_h, kc * kBK, (int)cta * 128, bar);
-          ptx::tma_load_2d_pair(st + kATileBytes, &tmap_w, kc * kBK, n0, bar);
-          ptx::tma_load_2d_pair(st + kATileBytes + w_half_bytes, &tmap_w, kc * kBK, n0 + N, bar);
+          ptx::tma_load_2d_pair_hint(st + kATileBytes, &tmap_w, kc * kBK, n0, bar, w_policy);
+          ptx::tma_load_2d_pair_hint(st + kATileBytes + w_half_bytes, &tmap_w, kc * kBK, n0 + N, bar, w_policy);
         }
       }
       if (!ok || *abort) {  // winding down: let the copies already issued land before the CTA goes away
