@@ -153,14 +153,14 @@ def _config(wl: syn.Workload, lengths=None):
          "shape": {"q_heads": s.n_q_heads, "kv_heads": s.n_kv_heads, "head_dim": s.head_dim, "hidden": s.hidden,
                    "vocab": s.vocab, "page": s.page_size},
          "prefix": [wl.prefix_lo, wl.prefix_hi], "s_max": round(wl.resolved_s_max(), 3), "seed": wl.seed,
-         "l2": "inputs larger than L2: the LM-head weight streamed each step exceeds the 126 MB L2",
+         "l2": "inputs larger than L2: the LM-head weight streamed each step exceeds the 126 MB L2; streamed loads are evict-first, and on cfg2_d4 ncu --cache-control none shows about a quarter of the cached K/V still in L2 from the step before (profiles/)",
          "tables": f"cache tables restored on the device every {RESTORE_EVERY} steps so prefix lengths stay as drawn"}
     if lengths is not None:
         c["prefix_tokens_total"] = int(np.sum(lengths))
     return c
 
 
-LMHEAD_NCU_TRAFFIC = 636448512   # bytes per launch of lmhead_umma_kernel<1> at cfg2_d4 (ncu, see profiles/)
+LMHEAD_NCU_TRAFFIC = 634270464   # bytes per launch of lmhead_umma_kernel<1> at cfg2_d4 (ncu, see profiles/)
 RESTORE_EVERY = 8   # steps between restores of the cache tables, so that prefix lengths stay the workload's
 
 
