@@ -39,6 +39,13 @@ formula on a hand-worked example and exhaustive brute force; gamma-append
 equals single appends.  The synthetic acceptance *statistics* versus the
 paper's tokens-per-pass tables are "parity unpinned" (they depend on trained
 weights) and are context only.
+
+Beyond the confidence-thresholded step: block_attention_masked (explicit visibility of the block's own
+keys) and verified_length / verify_and_commit (self-speculative decoding, Sec. 3.4).  Pins
+(tests/test_oracle_masked.py): all-visible equals block_attention; a position that sees one key
+returns that key's value row; invisible keys can hold anything; the causal mask equals token-by-token
+decoding with block_attention; permuting block keys together with the mask bits changes nothing;
+verified_length on hand-worked cases, against brute force, and where it parts from the printed formula.
 """
 from __future__ import annotations
 
@@ -89,6 +96,56 @@ def block_attention(q_bits: np.ndarray, k_blk_bits: np.ndarray, v_blk_bits: np.n
                     wgt = np.exp(s - m)
                     out[b, j, h] = (wgt @ vals) / np.sum(wgt)
     return out
+
+
+def block_attention_masked(q_bits: np.ndarray, k_blk_bits: np.ndarray, v_blk_bits: np.ndarray,
+                           prefix_k_bits: Sequence[np.ndarray], prefix_v_bits: Sequence[np.ndarray],
+                           vis: np.ndarray, scale: Optional[float] = None) -> np.ndarray:
+    """Block attention in which each query position sees all of the history but only chosen block keys.
+
+    q: [B, R, Hq, d]; k_blk, v_blk: [B, T, Hkv, d]; vis: [B, R] integers, bit t of vis[b, j] set when
+    query position j may attend to block key t.  out[b, j, h, :] = softmax over {all P_b cached
+    tokens} U {block keys t with bit t set} of q . K * scale, times V.  Returns float64 [B, R, Hq, d].
+
+    Two uses, both statements of the paper's masks with the block's own keys listed explicitly:
+      * verification inputs of self-speculative decoding (Sec. 3.4): position j sees the already
+        sampled tokens before it and the one [m] appended at the first unverified position;
+      * blocks whose first rows are real tokens attending causally, A_uv = 1[v <= u] for u < i
+        (Sec. 3.3), followed by the bidirectional noise block.
+    With every bit set (and R = T = D) this is block_attention.  A position that sees no key at all
+    (empty history and vis = 0) has no softmax; it is rejected.
+    """
+    B, R, Hq, d = q_bits.shape
+    T, Hkv = k_blk_bits.shape[1], k_blk_bits.shape[2]
+    G = Hq // Hkv
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    q = widen(q_bits)
+    out = np.zeros((B, R, Hq, d), dtype=np.float64)
+    for b in range(B):
+        P = prefix_k_bits[b].shape[0]
+        for j in range(R):
+            seen = [t for t in range(T) if (int(vis[b, j]) >> t) & 1]
+            if P + len(seen) == 0:
+                raise ValueError(f"query position {j} of sequence {b} sees no key")
+            for hk in range(Hkv):
+                keys = np.concatenate([widen(prefix_k_bits[b][:, hk, :]), widen(k_blk_bits[b, seen, hk, :])], axis=0)
+                vals = np.concatenate([widen(prefix_v_bits[b][:, hk, :]), widen(v_blk_bits[b, seen, hk, :])], axis=0)
+                for h in range(hk * G, (hk + 1) * G):
+                    s = (keys @ q[b, j, h]) * scale
+                    m = np.max(s)
+                    wgt = np.exp(s - m)
+                    out[b, j, h] = (wgt @ vals) / np.sum(wgt)
+    return out
+
+
+def verification_visibility(D: int) -> np.ndarray:
+    """vis[j] for the D verification inputs of one block (Sec. 3.4, self-speculative decoding), with
+    the block's keys listed as T = 2D rows: keys 0..D-1 are the real tokens [x^{i-1}, y^1, ..,
+    y^{D-1}] and keys D..2D-1 the [m] of each position.  Verification input j consists of the tokens
+    before position j and one [m] at position j, so position j sees real keys t < j and key D + j.
+    (Position 0 holds x^{i-1} itself: its 'mask' key D + 0 is that token's own key.)"""
+    return np.array([((1 << j) - 1) | (1 << (D + j)) for j in range(D)], dtype=np.int64)
 
 
 # ----------------------------------------------------------------------------
@@ -172,6 +229,44 @@ def accepted_length(conf: Sequence[float], tau: float) -> Tuple[int, float]:
         if prod >= tau:
             admissible.add(j)
     return max(admissible), margin
+
+
+def verified_length(draft: Sequence[int], verify: Sequence[int]) -> int:
+    """gamma_verify of Sec. 3.4: how many of the D speculative tokens y^ are kept after the second
+    pass produced y~.  Read as the longest prefix on which the two agree, floored at 1 (the section
+    is "Longest Prefix Decoding", and a token after a disagreement was sampled on a rejected
+    context); the printed formula, max{ j : y^_j = y~_j } U {1}, would also keep tokens after a
+    disagreement whenever a later position happens to agree."""
+    g = 0
+    for a, b in zip(draft, verify):
+        if int(a) != int(b):
+            break
+        g += 1
+    return max(g, 1)
+
+
+def verified_length_as_printed(draft: Sequence[int], verify: Sequence[int]) -> int:
+    """The formula exactly as printed (largest agreeing index, floored at 1); kept to show where the
+    two readings part."""
+    agree = {j for j in range(1, len(draft) + 1) if int(draft[j - 1]) == int(verify[j - 1])}
+    return max(agree | {1})
+
+
+def verify_and_commit(cache: "PagedKVCache", seq_ids: Sequence[int], draft: np.ndarray, verify: np.ndarray,
+                      k_real_bits: np.ndarray, v_real_bits: np.ndarray) -> "CommitResult":
+    """Self-speculative acceptance: gamma_verify per sequence, emit the first gamma speculative tokens
+    and append the K/V rows of those positions (the real tokens' rows of the verification pass) as
+    gamma single-token appends, sequences in batch order."""
+    B, D = draft.shape
+    acc = np.zeros(B, np.int32)
+    out = np.full((B, D), -1, np.int32)
+    for b in range(B):
+        g = verified_length(draft[b], verify[b])
+        for t in range(g):
+            cache.append_token(int(seq_ids[b]), k_real_bits[b, t], v_real_bits[b, t])
+        acc[b] = g
+        out[b, :g] = draft[b, :g]
+    return CommitResult(acc, out, np.full(B, np.inf))
 
 
 # ----------------------------------------------------------------------------

@@ -1,0 +1,161 @@
+"""Pins for the oracle's block attention with explicit visibility of the block's own keys and for the
+self-speculative acceptance rule (Sec. 3.3 mask, Sec. 3.4 "Self-Speculative Decoding")."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import sdlm_oracle as orc
+import sdlm_synth as syn
+
+
+def _rand_bits(rng, shape):
+    return syn.f32_to_bf16_bits(rng.normal(size=shape).astype(np.float32))
+
+
+def _case(seed, B, R, T, Hq, Hkv, d, prefix):
+    rng = np.random.default_rng(seed)
+    q = _rand_bits(rng, (B, R, Hq, d))
+    k = _rand_bits(rng, (B, T, Hkv, d))
+    v = _rand_bits(rng, (B, T, Hkv, d))
+    pk = [_rand_bits(rng, (p, Hkv, d)) for p in prefix]
+    pv = [_rand_bits(rng, (p, Hkv, d)) for p in prefix]
+    return q, k, v, pk, pv
+
+
+def test_every_key_visible_is_the_unmasked_block_attention():
+    q, k, v, pk, pv = _case(1, 3, 4, 4, 4, 2, 16, (0, 5, 70))
+    vis = np.full((3, 4), 0b1111, dtype=np.int64)
+    a = orc.block_attention_masked(q, k, v, pk, pv, vis)
+    b = orc.block_attention(q, k, v, pk, pv)
+    assert np.array_equal(a, b)
+
+
+def test_a_position_that_sees_a_single_key_returns_that_value_row():
+    """softmax over one key is 1: the output is the value row itself, whatever the scores are."""
+    q, k, v, pk, pv = _case(2, 2, 3, 5, 4, 2, 8, (0, 0))
+    vis = np.array([[1 << 4, 1 << 0, 1 << 2], [1 << 1, 1 << 3, 1 << 3]], dtype=np.int64)
+    out = orc.block_attention_masked(q, k, v, pk, pv, vis)
+    vf = syn.bf16_bits_to_f32(v).astype(np.float64)
+    for b in range(2):
+        for j in range(3):
+            t = int(vis[b, j]).bit_length() - 1
+            for h in range(4):
+                assert np.array_equal(out[b, j, h], vf[b, t, h // 2])
+
+
+def test_keys_a_position_does_not_see_can_hold_anything():
+    q, k, v, pk, pv = _case(3, 2, 4, 6, 2, 1, 8, (3, 11))
+    vis = np.array([[0b000101, 0b110000, 0b000001, 0b111111]] * 2, dtype=np.int64)
+    ref = orc.block_attention_masked(q, k, v, pk, pv, vis)
+    k2, v2 = k.copy(), v.copy()
+    k2[:, 1] = syn.f32_to_bf16_bits(np.full(k[:, 1].shape, 1e30, np.float32))     # key 1: unseen by rows 0..2
+    v2[:, 3] = syn.f32_to_bf16_bits(np.full(v[:, 3].shape, -7.5, np.float32))    # key 3: unseen by rows 0..2
+    out = orc.block_attention_masked(q, k2, v2, pk, pv, vis)
+    assert np.array_equal(out[:, :3], ref[:, :3])
+    assert not np.array_equal(out[:, 3], ref[:, 3])          # the row that sees them does change
+
+
+def test_causal_visibility_is_token_by_token_decoding():
+    """A_uv = 1[v <= u] inside the block: row j equals a D = 1 step whose history is [history ; rows < j]
+    (block_attention with D = 1 is pinned separately against next-token decode)."""
+    B, R, Hq, Hkv, d = 2, 5, 4, 2, 16
+    q, k, v, pk, pv = _case(4, B, R, R, Hq, Hkv, d, (6, 0))
+    vis = np.array([[(1 << (j + 1)) - 1 for j in range(R)]] * B, dtype=np.int64)
+    out = orc.block_attention_masked(q, k, v, pk, pv, vis)
+    for j in range(R):
+        hist_k = [np.concatenate([pk[b], k[b, :j]], axis=0) for b in range(B)]
+        hist_v = [np.concatenate([pv[b], v[b, :j]], axis=0) for b in range(B)]
+        one = orc.block_attention(q[:, j:j + 1], k[:, j:j + 1], v[:, j:j + 1], hist_k, hist_v)
+        assert np.allclose(out[:, j], one[:, 0], rtol=0, atol=1e-14)
+
+
+def test_permuting_block_keys_together_with_the_mask_bits_changes_nothing():
+    q, k, v, pk, pv = _case(5, 2, 3, 6, 2, 2, 8, (4, 9))
+    rng = np.random.default_rng(0)
+    vis = rng.integers(1, 1 << 6, size=(2, 3)).astype(np.int64)
+    ref = orc.block_attention_masked(q, k, v, pk, pv, vis)
+    perm = np.array([3, 0, 5, 1, 4, 2])                      # new key t' holds old key perm[t']
+    vis2 = np.zeros_like(vis)
+    for t_new, t_old in enumerate(perm):
+        vis2 |= ((vis >> t_old) & 1) << t_new
+    out = orc.block_attention_masked(q, k[:, perm], v[:, perm], pk, pv, vis2)
+    assert np.allclose(out, ref, rtol=0, atol=1e-14)
+
+
+def test_against_dense_attention_with_an_explicit_mask_matrix():
+    """torch softmax over [history ; block keys] with -inf where the bit is clear."""
+    B, R, T, Hq, Hkv, d = 1, 4, 7, 4, 2, 8
+    q, k, v, pk, pv = _case(6, B, R, T, Hq, Hkv, d, (10,))
+    vis = np.array([[0b1000001, 0b0101010, 0b1111111, 0b0010000]], dtype=np.int64)
+    out = orc.block_attention_masked(q, k, v, pk, pv, vis)
+    f = lambda bits: torch.from_numpy(syn.bf16_bits_to_f32(bits).astype(np.float64))
+    keys = torch.cat([f(pk[0]), f(k[0])], 0)                 # [P+T, Hkv, d]
+    vals = torch.cat([f(pv[0]), f(v[0])], 0)
+    for j in range(R):
+        allowed = torch.tensor([True] * 10 + [bool((int(vis[0, j]) >> t) & 1) for t in range(T)])
+        for h in range(Hq):
+            s = (keys[:, h // 2] @ f(q[0, j, h])) / np.sqrt(d)
+            s = torch.where(allowed, s, torch.tensor(float("-inf"), dtype=torch.float64))
+            ref = torch.softmax(s, 0) @ vals[:, h // 2]
+            assert torch.allclose(torch.from_numpy(out[0, j, h]), ref, rtol=0, atol=1e-13)
+
+
+def test_a_position_without_any_key_is_rejected():
+    q, k, v, pk, pv = _case(7, 1, 2, 2, 2, 1, 8, (0,))
+    with pytest.raises(ValueError):
+        orc.block_attention_masked(q, k, v, pk, pv, np.array([[0b01, 0]], dtype=np.int64))
+
+
+def test_verification_visibility_lists_the_tokens_before_and_one_mask():
+    vis = orc.verification_visibility(4)
+    # position j: real keys 0..j-1 and mask key 4 + j
+    assert [bin(int(x)) for x in vis] == ["0b10000", "0b100001", "0b1000011", "0b10000111"]
+
+
+# ---- gamma_verify ------------------------------------------------------------------------------
+@pytest.mark.parametrize("draft,verify,gamma", [
+    ([5, 6, 7, 8], [5, 6, 7, 8], 4),      # all consistent: the whole block is kept
+    ([5, 6, 7, 8], [5, 6, 9, 8], 2),      # first disagreement at position 3
+    ([5, 6, 7, 8], [4, 6, 7, 8], 1),      # disagreement at position 1: the floor of 1 applies
+    ([5, 6, 7, 8], [5, 0, 0, 0], 1),
+    ([3], [9], 1),
+    ([3], [3], 1),
+])
+def test_verified_length_hand_worked(draft, verify, gamma):
+    assert orc.verified_length(draft, verify) == gamma
+
+
+def test_verified_length_against_brute_force_over_all_agreement_patterns():
+    D = 6
+    for pattern in itertools.product([0, 1], repeat=D):
+        draft = list(range(10, 10 + D))
+        verify = [d if a else -1 for d, a in zip(draft, pattern)]
+        want = 1
+        for j in range(1, D + 1):
+            if all(pattern[:j]):
+                want = max(want, j)
+        assert orc.verified_length(draft, verify) == want
+        # the printed formula keeps a later agreeing position: it is never shorter, and differs
+        # exactly when some position after the first disagreement agrees
+        printed = orc.verified_length_as_printed(draft, verify)
+        assert printed >= want
+        first_bad = pattern.index(0) if 0 in pattern else D
+        assert (printed > want) == any(pattern[first_bad + 1:])
+
+
+def test_verify_and_commit_appends_the_kept_rows_like_single_appends():
+    rng = np.random.default_rng(3)
+    shape = syn.Shape(4, 2, 64, 64, 128)
+    cache = orc.PagedKVCache(num_pages=8, page_size=64, n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim, max_batch=2,
+                             max_pages_per_seq=4)
+    for b, n in enumerate((63, 5)):
+        cache.add_sequence(b, _rand_bits(rng, (n, 2, 64)), _rand_bits(rng, (n, 2, 64)))
+    k = _rand_bits(rng, (2, 4, 2, 64)); v = _rand_bits(rng, (2, 4, 2, 64))
+    draft = np.array([[1, 2, 3, 4], [1, 2, 3, 4]]); verify = np.array([[1, 2, 3, 9], [7, 2, 3, 4]])
+    res = orc.verify_and_commit(cache, [0, 1], draft, verify, k, v)
+    assert res.accepted_len.tolist() == [3, 1] and res.out_tokens.tolist() == [[1, 2, 3, -1], [1, -1, -1, -1]]
+    assert cache.seq_len[:2].tolist() == [66, 6]
+    k0, v0 = cache.gather_fast(0)
+    assert np.array_equal(k0[63:], k[0, :3]) and np.array_equal(v0[63:], v[0, :3])
