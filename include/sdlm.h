@@ -154,6 +154,22 @@ sdlm_status sdlm_kv_pages(sdlm_ctx* ctx, sdlm_kv_op op, const sdlm_kv_args* args
 sdlm_status sdlm_block_attn(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, const void* q,
                             const void* k_blk, const void* v_blk, void* out, void* stream);
 
+/* ---- (a') block attention with an explicit visibility mask over the block's own keys.
+ * Sec. 3.4, self-speculative decoding: the D verification inputs of a block are the sampled tokens
+ * before position j plus one [m] at position j; Sec. 3.3: rows of real tokens attend causally,
+ * A_uv = 1[v <= u].  Both are this call with the block's keys listed explicitly:
+ *   out[b,j,h,:] = softmax_t( q[b,j,h,:] . K_t * scale ) V_t,  t over the slot's cached tokens (all
+ *   visible) followed by those of the n_k rows k_blk[b,t,h/G,:] whose bit t is set in vis[b,j].
+ * q, out [batch, n_q, Hq, d]; k_blk / v_blk [batch, n_k, Hkv, d]: device bf16; vis: device uint32
+ * [batch, n_q]; seq_ids: device int32 [batch] or NULL.  1 <= n_q <= max_block with (Hq/Hkv) * n_q <= 64;
+ * 1 <= n_k <= 16.  Every query position must see at least one key (a cached token or a block key);
+ * the output of one that sees none is undefined.  Arithmetic, scratch and overlap rules as
+ * sdlm_block_attn; with every bit set and n_q = n_k it computes the same values.
+ * Errors: INVALID_ARG, SHAPE, UNSUPPORTED (softmax_scale = 0: masking needs a positive scale). */
+sdlm_status sdlm_block_attn_masked(sdlm_ctx* ctx, int32_t batch, int32_t n_q, int32_t n_k, const int32_t* seq_ids,
+                                   const void* q, const void* k_blk, const void* v_blk, const uint32_t* vis,
+                                   void* out, void* stream);
+
 /* ---- (b) LM head -> softmax statistics -- Sec. 3.2 (Z in R^{D x |V|}), Eq. 8, Eq. 9.
  * For each of `rows` hidden states: z = W h (|V| logits, fp32 accumulate, never stored);
  *   token   = argmax_n z_n (lowest n on exact ties)
@@ -205,6 +221,18 @@ sdlm_status sdlm_accept_commit(sdlm_ctx* ctx, int32_t batch, int32_t D, const in
                                sdlm_conf_mode mode, const int32_t* token, const float* p_top1,
                                const float* entropy, const void* k_blk, const void* v_blk,
                                int32_t* accepted_len, int32_t* out_tokens, void* stream);
+
+/* ---- (c') self-speculative acceptance + commit -- Sec. 3.4, gamma_verify.
+ * draft_token [batch, D] are the tokens of the first pass, verify_token [batch, D] those of the
+ * verification pass (device int32).  accepted_len[b] = length of the longest prefix on which the two
+ * agree, at least 1 (the printed formula takes the largest agreeing index; read here as the longest
+ * agreeing prefix, the section's "Longest Prefix Decoding"); out_tokens[b,k] = draft_token[b,k] for
+ * k < accepted_len[b], else -1; rows 0..accepted_len[b]-1 of k_blk / v_blk [batch, D, Hkv, d] (the
+ * real tokens' rows of the verification pass) are appended to the cache exactly as
+ * sdlm_accept_commit appends them.  Errors and device-side checks: as sdlm_accept_commit. */
+sdlm_status sdlm_verify_commit(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids,
+                               const int32_t* draft_token, const int32_t* verify_token, const void* k_blk,
+                               const void* v_blk, int32_t* accepted_len, int32_t* out_tokens, void* stream);
 
 /* Synchronises `stream` and copies the sticky device status words to host_out[4]:
  * {sdlm_status (0 = none), sequence slot of the first failure, detail, number of failures}.

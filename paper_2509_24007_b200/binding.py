@@ -30,7 +30,8 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "UNSUPPORTED", 4: "OUT
 
 EXPORTED = ["sdlm_pool_bytes", "sdlm_workspace_bytes", "sdlm_create", "sdlm_destroy", "sdlm_status_str",
             "sdlm_kv_pages", "sdlm_block_attn", "sdlm_lmhead_confidence", "sdlm_lmhead_confidence_static", "sdlm_accept_commit",
-            "sdlm_device_status", "sdlm_decode_step", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count"]
+            "sdlm_device_status", "sdlm_decode_step", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count",
+            "sdlm_block_attn_masked", "sdlm_verify_commit"]
 
 
 class SdlmError(RuntimeError):
@@ -108,6 +109,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdlm_lmhead_confidence.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_lmhead_confidence_static.restype = C.c_int
     lib.sdlm_lmhead_confidence_static.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_block_attn_masked.restype = C.c_int
+    lib.sdlm_block_attn_masked.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_verify_commit.restype = C.c_int
+    lib.sdlm_verify_commit.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_accept_commit.restype = C.c_int
     lib.sdlm_accept_commit.argtypes = [vp, i32, i32, vp, f32, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_device_status.restype = C.c_int
@@ -288,6 +293,42 @@ class Sdlm:
                                                                 _ptr(v_blk), _ptr(_dev(out, torch.bfloat16, "out")),
                                                                 _stream_ptr(stream)))
         return out
+
+    def block_attn_masked(self, q: torch.Tensor, k_blk: torch.Tensor, v_blk: torch.Tensor, vis: torch.Tensor,
+                          out: Optional[torch.Tensor] = None, seq_ids: Optional[torch.Tensor] = None,
+                          stream=None) -> torch.Tensor:
+        """sdlm_block_attn_masked: vis [batch, n_q] int32 holds the uint32 visibility words."""
+        batch, n_q, n_k = int(q.shape[0]), int(q.shape[1]), int(k_blk.shape[1])
+        _dev(q, torch.bfloat16, "q"); _dev(k_blk, torch.bfloat16, "k_blk"); _dev(v_blk, torch.bfloat16, "v_blk")
+        _dev(vis, torch.int32, "vis")
+        if tuple(vis.shape) != (batch, n_q):
+            raise ValueError("vis must be [batch, n_q]")
+        if out is None:
+            out = torch.empty_like(q)
+        if seq_ids is not None:
+            _dev(seq_ids, torch.int32, "seq_ids")
+        self._check("sdlm_block_attn_masked", self.lib.sdlm_block_attn_masked(
+            self.ctx, batch, n_q, n_k, _ptr(seq_ids), _ptr(q), _ptr(k_blk), _ptr(v_blk), _ptr(vis),
+            _ptr(_dev(out, torch.bfloat16, "out")), _stream_ptr(stream)))
+        return out
+
+    def verify_commit(self, draft_token: torch.Tensor, verify_token: torch.Tensor, k_blk: torch.Tensor,
+                      v_blk: torch.Tensor, accepted_len: Optional[torch.Tensor] = None,
+                      out_tokens: Optional[torch.Tensor] = None, seq_ids: Optional[torch.Tensor] = None, stream=None):
+        batch, D = int(k_blk.shape[0]), int(k_blk.shape[1])
+        _dev(draft_token, torch.int32, "draft_token"); _dev(verify_token, torch.int32, "verify_token")
+        _dev(k_blk, torch.bfloat16, "k_blk"); _dev(v_blk, torch.bfloat16, "v_blk")
+        if accepted_len is None:
+            accepted_len = torch.empty(batch, dtype=torch.int32, device=self.device)
+        if out_tokens is None:
+            out_tokens = torch.empty((batch, D), dtype=torch.int32, device=self.device)
+        if seq_ids is not None:
+            _dev(seq_ids, torch.int32, "seq_ids")
+        self._check("sdlm_verify_commit", self.lib.sdlm_verify_commit(
+            self.ctx, batch, D, _ptr(seq_ids), _ptr(draft_token), _ptr(verify_token), _ptr(k_blk), _ptr(v_blk),
+            _ptr(_dev(accepted_len, torch.int32, "accepted_len")), _ptr(_dev(out_tokens, torch.int32, "out_tokens")),
+            _stream_ptr(stream)))
+        return accepted_len, out_tokens
 
     def lmhead_confidence_static(self, hidden: torch.Tensor, w_lm: torch.Tensor, token: torch.Tensor,
                                  p_top1: torch.Tensor, entropy: torch.Tensor, max_logit: Optional[torch.Tensor] = None,

@@ -195,6 +195,7 @@ struct CommitParams {
   int32_t* token_copy;
   float* p_top1_copy;
   float* entropy_copy;
+  const int32_t* verify_token;  // null: gamma_tau of Eq. 7; else gamma_verify against these tokens
   float tau, inv_ln_vocab;
   int mode, batch, D, Hkv, d, mpps, num_pages;
 };
@@ -204,6 +205,11 @@ struct CommitParams {
 __device__ inline int gamma_tau(const CommitParams& p, int row) {
   float prod = 1.0f;
   int g = 1;
+  if (p.verify_token) {  // self-speculative acceptance (Sec. 3.4): the longest prefix on which both passes agree
+    int k = 0;
+    while (k < p.D && p.token[row * p.D + k] == p.verify_token[row * p.D + k]) ++k;
+    return k > 1 ? k : 1;
+  }
   for (int k = 0; k < p.D; ++k) {
     float c = (p.mode == SDLM_CONF_LOGIT) ? p.p_top1[row * p.D + k]
                                           : __fsub_rn(1.0f, __fmul_rn(p.entropy[row * p.D + k], p.inv_ln_vocab));
@@ -592,9 +598,9 @@ static sdlm_status accept_commit_launch(sdlm_ctx* ctx, int32_t batch, int32_t D,
                                         sdlm_conf_mode mode, const int32_t* token, const float* p_top1,
                                         const float* entropy, const void* k_blk, const void* v_blk,
                                         int32_t* accepted_len, int32_t* out_tokens, const StatCopies& copies,
-                                        void* stream) {
-  if (!ctx || !token || !p_top1 || !entropy || !k_blk || !v_blk || !accepted_len || !out_tokens)
-    return SDLM_ERR_INVALID_ARG;
+                                        void* stream, const int32_t* verify_token = nullptr) {
+  if (!ctx || !token || !k_blk || !v_blk || !accepted_len || !out_tokens) return SDLM_ERR_INVALID_ARG;
+  if (!verify_token && (!p_top1 || !entropy)) return SDLM_ERR_INVALID_ARG;
   if (!aligned16(k_blk) || !aligned16(v_blk)) return SDLM_ERR_INVALID_ARG;
   if (mode != SDLM_CONF_LOGIT && mode != SDLM_CONF_ENTROPY) return SDLM_ERR_INVALID_ARG;
   if (!isfinite(tau)) return SDLM_ERR_INVALID_ARG;
@@ -608,6 +614,7 @@ static sdlm_status accept_commit_launch(sdlm_ctx* ctx, int32_t batch, int32_t D,
   p.k_blk = static_cast<const __nv_bfloat16*>(k_blk); p.v_blk = static_cast<const __nv_bfloat16*>(v_blk);
   p.accepted_len = accepted_len; p.out_tokens = out_tokens;
   p.token_copy = copies.token; p.p_top1_copy = copies.p_top1; p.entropy_copy = copies.entropy;
+  p.verify_token = verify_token;
   p.tau = tau;
   p.inv_ln_vocab = c.vocab > 1 ? (float)(1.0 / log((double)c.vocab)) : 0.0f;
   p.mode = (int)mode; p.batch = batch; p.D = D; p.Hkv = c.n_kv_heads; p.d = c.head_dim;
@@ -624,6 +631,32 @@ extern "C" sdlm_status sdlm_accept_commit(sdlm_ctx* ctx, int32_t batch, int32_t 
                                           int32_t* accepted_len, int32_t* out_tokens, void* stream) {
   return accept_commit_launch(ctx, batch, D, seq_ids, tau, mode, token, p_top1, entropy, k_blk, v_blk, accepted_len,
                               out_tokens, StatCopies{}, stream);
+}
+
+extern "C" sdlm_status sdlm_verify_commit(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids,
+                                          const int32_t* draft_token, const int32_t* verify_token, const void* k_blk,
+                                          const void* v_blk, int32_t* accepted_len, int32_t* out_tokens,
+                                          void* stream) {
+  if (!verify_token) return SDLM_ERR_INVALID_ARG;
+  return accept_commit_launch(ctx, batch, D, seq_ids, 0.5f, SDLM_CONF_LOGIT, draft_token, nullptr, nullptr, k_blk, v_blk,
+                              accepted_len, out_tokens, StatCopies{}, stream, verify_token);
+}
+
+extern "C" sdlm_status sdlm_block_attn_masked(sdlm_ctx* ctx, int32_t batch, int32_t n_q, int32_t n_k,
+                                              const int32_t* seq_ids, const void* q, const void* k_blk,
+                                              const void* v_blk, const uint32_t* vis, void* out, void* stream) {
+  if (!ctx || !q || !k_blk || !v_blk || !vis || !out) return SDLM_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out)) return SDLM_ERR_INVALID_ARG;
+  sdlm_status s = check_batch(ctx, batch, n_q);
+  if (s != SDLM_OK) return s;
+  if (n_k < 1) return SDLM_ERR_INVALID_ARG;
+  if (n_k > kMaxBlockKeys) return SDLM_ERR_SHAPE;
+  if (ctx->group * n_q > kMaxQRows) return SDLM_ERR_SHAPE;
+  if (!(ctx->scale > 0.0f)) return SDLM_ERR_UNSUPPORTED;  // masking is by -inf scores: needs a positive scale
+  return launch_block_attn(ctx, batch, n_q, seq_ids, q, k_blk, v_blk, out, static_cast<cudaStream_t>(stream), 0, false,
+                           n_k, vis) == cudaSuccess
+             ? SDLM_OK
+             : SDLM_ERR_CUDA;
 }
 
 extern "C" sdlm_status sdlm_device_status(sdlm_ctx* ctx, int32_t* host_out, int32_t clear, void* stream) {

@@ -50,6 +50,11 @@ struct AttnParams {
   int min_range;  // shortest range of positions worth a CTA of its own
   int item_cost;  // what starting a (sequence, KV head) pair costs a CTA, in tiles (see ItemWalk)
   int release_first;  // let the next kernel on the stream start before this one has waited for the one before it
+  // Block-tile keys and who sees them.  Dk = rows of k_blk / v_blk per sequence (D unless masked);
+  // vis = null (every query position sees every block key) or [batch][D] words, bit t of word j set
+  // when query position j sees block key t.  The cached history is visible to every position.
+  int Dk;
+  const uint32_t* vis;
 };
 
 // 8 warps; 12 when 64 stacked query rows need a second set of softmax warps
@@ -267,7 +272,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     const size_t lim_len = ((size_t)p.batch * 4 + line - 1) / line;
     const size_t n_tab = ((size_t)p.batch * p.mpps * 4 + line - 1) / line;
     const size_t n_q = ((size_t)p.batch * p.D * p.Hq * HD * 2 + line - 1) / line;
-    const size_t n_kv = ((size_t)p.batch * p.D * p.Hkv * HD * 2 + line - 1) / line;
+    const size_t n_kv = ((size_t)p.batch * p.Dk * p.Hkv * HD * 2 + line - 1) / line;
     const size_t total = lim_len + n_tab + n_q + 2 * n_kv;  // (the lengths too: one line, for the other thread blocks)
     for (size_t i = (size_t)blockIdx.x * blockDim.x + tid; i < total; i += (size_t)gridDim.x * blockDim.x) {
       const char* a;
@@ -495,9 +500,26 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
 #pragma unroll
       for (int q = 0; q < QV; ++q) l[q] = 0.f;
       const int n = it.t1 - it.t0, ng = (n + 1) / 2;
+      // which of my 32 query rows see my key if it turns out to be a block key (bit q: row qb + q)
+      uint32_t visq = 0xffffffffu;
+      if (p.vis != nullptr && it.t1 > it.pages) {
+        visq = 0;
+        int j = qb / p.G, rem = qb % p.G;
+        uint32_t vj = j < p.D ? p.vis[(size_t)it.b * p.D + j] : 0u;
+#pragma unroll
+        for (int q = 0; q < QV; ++q) {
+          const uint32_t bit = qb + q < GD ? (kt < 32 ? (vj >> kt) & 1u : 0u) : 1u;  // padding rows: no mask
+          visq |= bit << q;
+          if (++rem == p.G) {
+            rem = 0;
+            ++j;
+            vj = j < p.D ? p.vis[(size_t)it.b * p.D + j] : 0u;
+          }
+        }
+      }
       for (int g = 0; g < ng; ++g, ++gc) {
         const uint32_t sb = gc & 1u;
-        const bool mine = kt < tile_valid(it, it.t0 + 2 * g + tj, p.D);  // does my key exist?
+        const bool mine = kt < tile_valid(it, it.t0 + 2 * g + tj, p.Dk);  // does my key exist?
         if (!__all_sync(0xffffffffu, ptx::mbar_wait(&s_full[sb], (gc >> 1) & 1u, abort))) { ok = false; break; }
         ptx::tc_fence_after();
         float x[QV];  // my key's score for every row, then its exponent relative to the row reference
@@ -508,6 +530,11 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&s_free[sb]);
+        if (visq != 0xffffffffu && it.t0 + 2 * g + tj == it.pages) {  // my key is a block key some rows do not see
+#pragma unroll
+          for (int q = 0; q < QV; ++q)
+            if (!((visq >> q) & 1u)) x[q] = -INFINITY;
+        }
 
         const bool first = g == 0;
         bool moved = first;  // the first group of an item always sets the references
@@ -651,9 +678,12 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
           for (int q = 0; q < QV; ++q) p.part_o[(slot_row + qb + q) * HD + d] = o[q];
         }
         const int mrow = qb + kg;  // the query row this thread looks after where one thread per row is needed
-        if (kg < QV)
+        if (kg < QV) {
+          // a row that saw no key in this split (all of them masked) takes no part in the merge
+          const float lrow = ls[mrow] + ls[64 + mrow] + ls[128 + mrow] + ls[192 + mrow];
           *reinterpret_cast<float2*>(p.part_ml + (slot_row + mrow) * 2) =
-              make_float2(mref[mrow], ls[mrow] + ls[64 + mrow] + ls[128 + mrow] + ls[192 + mrow]);
+              make_float2(lrow > 0.f ? mref[mrow] : -INFINITY, lrow);
+        }
         __threadfence();
         if (!meet()) { ok = false; break; }
         if (warp == 2 && lane == 0) {  // every split of the pair counts once; the last one merges
@@ -786,19 +816,22 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
 
       const int n = it.t1 - it.t0, ng = (n + 1) / 2;
       for (int g = 0; g + 1 < ng; ++g) ring.advance(NS);
-      if (it.t1 > it.pages) {  // the item's last group holds the block's own D keys
-        constexpr int NB = kMaxBlock * (HD / 8) / 32;  // chunks of the block's K (and V) rows per lane
+      if (it.t1 > it.pages) {  // the item's last group holds the block's own keys (D of them, Dk when masked)
+        constexpr int NB = kMaxBlock * (HD / 8) / 32;  // chunks of eight of the block's K (and V) rows per lane
         uint4 kreg[NB], vreg[NB];
+        auto load_rows = [&](int k0) {
 #pragma unroll
-        for (int i = 0; i < NB; ++i) {
-          const int idx = i * 32 + lane, key = idx / (HD / 8), c = idx % (HD / 8);
-          kreg[i] = vreg[i] = make_uint4(0, 0, 0, 0);
-          if (key < p.D) {
-            const size_t src = (((size_t)it.b * p.D + key) * p.Hkv + it.h) * HD;
-            kreg[i] = __ldg(reinterpret_cast<const uint4*>(p.k_blk + src) + c);
-            vreg[i] = __ldg(reinterpret_cast<const uint4*>(p.v_blk + src) + c);
+          for (int i = 0; i < NB; ++i) {
+            const int idx = i * 32 + lane, key = k0 + idx / (HD / 8), c = idx % (HD / 8);
+            kreg[i] = vreg[i] = make_uint4(0, 0, 0, 0);
+            if (key < p.Dk) {
+              const size_t src = (((size_t)it.b * p.Dk + key) * p.Hkv + it.h) * HD;
+              kreg[i] = __ldg(reinterpret_cast<const uint4*>(p.k_blk + src) + c);
+              vreg[i] = __ldg(reinterpret_cast<const uint4*>(p.v_blk + src) + c);
+            }
           }
-        }
+        };
+        load_rows(0);
         if (!__all_sync(0xffffffffu, ptx::counter_wait(blk_go, (int)blk_idx, abort))) {
           ok = false;
           break;
@@ -807,18 +840,21 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
         const int tj = (n - 1) & 1;  // the block's tile is the group's first or second
         uint8_t* st = stages + (size_t)ring.stage * PAIR_B;
         uint8_t* v_t = st + K_REGION_B + tj * VT_B;
-        // V^T columns of keys beyond D must be zeros (0 * stale bits could be NaN); K rows beyond D
-        // only produce scores that are masked
+        // V^T columns of keys beyond the block's must be zeros (0 * stale bits could be NaN); K rows
+        // beyond them only produce scores that are masked
         for (int idx = lane; idx < VT_B / 16; idx += 32) reinterpret_cast<uint4*>(v_t)[idx] = make_uint4(0, 0, 0, 0);
         __syncwarp();
+        for (int k0 = 0; k0 < p.Dk; k0 += kMaxBlock) {
+          if (k0 > 0) load_rows(k0);
 #pragma unroll
-        for (int i = 0; i < NB; ++i) {
-          const int idx = i * 32 + lane, key = idx / (HD / 8), c = idx % (HD / 8);
-          if (key < p.D) {
-            *reinterpret_cast<uint4*>(st + (c >> 3) * 2 * K_PANEL_B + tj * K_PANEL_B + key * 128 + (((c & 7) ^ (key & 7)) << 4)) = kreg[i];
-            const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(&vreg[i]);
+          for (int i = 0; i < NB; ++i) {
+            const int idx = i * 32 + lane, key = k0 + idx / (HD / 8), c = idx % (HD / 8);
+            if (key < p.Dk) {
+              *reinterpret_cast<uint4*>(st + (c >> 3) * 2 * K_PANEL_B + tj * K_PANEL_B + key * 128 + (((c & 7) ^ (key & 7)) << 4)) = kreg[i];
+              const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(&vreg[i]);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) reinterpret_cast<__nv_bfloat16*>(v_t)[vt_tile_elem(key, c * 8 + e)] = ve[e];
+              for (int e = 0; e < 8; ++e) reinterpret_cast<__nv_bfloat16*>(v_t)[vt_tile_elem(key, c * 8 + e)] = ve[e];
+            }
           }
         }
         ptx::fence_proxy_async();
@@ -887,7 +923,7 @@ cudaError_t setup_attn(sdlm_ctx* ctx) {
 
 cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, const void* q,
                               const void* k_blk, const void* v_blk, void* out, cudaStream_t st, int cta_cap,
-                              bool whole_tpcs) {
+                              bool whole_tpcs, int n_blk_keys, const uint32_t* vis) {
   const sdlm_config& c = ctx->cfg;
   AttnParams p;
   p.pool = reinterpret_cast<const __nv_bfloat16*>(ctx->pool);
@@ -908,6 +944,8 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
   p.item_cost = ctx->attn_item_cost;
   p.min_range = ctx->attn_min_range;
   p.release_first = cta_cap > 0 ? 1 : 0;
+  p.Dk = n_blk_keys > 0 ? n_blk_keys : D;
+  p.vis = vis;
   // the kernel's tile arithmetic is 32-bit: (tiles of the launch) x (CTAs) must stay below 2^31
   if ((long long)batch * (c.max_pages_per_seq + 1 + ctx->attn_item_cost) * c.n_kv_heads > 13000000ll)
     return cudaErrorInvalidConfiguration;

@@ -12,6 +12,7 @@ namespace sdlm {
 
 constexpr int kPageSize = 64;        // tokens per KV page
 constexpr int kMaxBlock = 8;         // largest D
+constexpr int kMaxBlockKeys = 16;    // rows of k_blk / v_blk per sequence in the masked variant
 constexpr int kMaxQRows = 64;        // (Hq/Hkv) * D stacked query rows per KV head
 constexpr int kMaxBatch = 4096;
 constexpr int kLmMaxStripes = 1024;  // upper bound on vocab stripes (one partial per stripe per row)
@@ -134,7 +135,8 @@ inline cudaError_t launch_overlapped_cluster(void (*kernel)(KArgs...), dim3 grid
 // ---- launchers implemented in the kernel translation units ---------------------------------
 cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, const void* q,
                               const void* k_blk, const void* v_blk, void* out, cudaStream_t st,
-                              int cta_cap = 0, bool whole_tpcs = false);
+                              int cta_cap = 0, bool whole_tpcs = false, int n_blk_keys = 0,
+                              const uint32_t* vis = nullptr);
 // `independent_of_predecessor`: the caller guarantees that none of the inputs is written by the
 // kernel enqueued just before on `st` (the stripe kernel then overlaps with it).
 sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,

@@ -16,6 +16,13 @@ import sdlm_synth as syn
 from .binding import CONF_LOGIT, Sdlm, SdlmConfig, bf16_tensor_from_bits
 
 
+def verification_mask(D: int) -> np.ndarray:
+    """Visibility words for sdlm_block_attn_masked in the verification pass of a self-speculative step
+    (Sec. 3.4), with the block's 2D keys laid out as [real tokens 0..D-1, [m] of positions 0..D-1]:
+    position j sees the real tokens before it and the [m] at its own position."""
+    return np.array([((1 << j) - 1) + (1 << (D + j)) for j in range(D)], dtype=np.uint32)
+
+
 @dataclass
 class DeviceBlock:
     q: torch.Tensor

@@ -34,6 +34,7 @@ _CHUNK = 1 << 22  # elements per independently seeded chunk
 # tensor ids: the high half of the Philox key
 _T_WLM, _T_PREFIX_LEN, _T_FREE, _T_KPREF, _T_VPREF = 1, 2, 3, 4, 5
 _T_Q, _T_KBLK, _T_VBLK, _T_HNOISE, _T_TARGET, _T_SCALE = 6, 7, 8, 9, 10, 11
+_T_QVER, _T_KMASK, _T_VMASK, _T_VIS, _T_AGREE = 12, 13, 14, 15, 16
 
 
 # ----------------------------------------------------------------------------
@@ -227,6 +228,40 @@ def block_inputs(w: Workload, w_lm_bits: np.ndarray, step: int = 0) -> BlockInpu
     planted = bf16_bits_to_f32(w_lm_bits[target.reshape(-1)]).reshape(B, D, s.hidden)
     hidden = f32_to_bf16_bits(noise + scale[..., None] * planted).reshape(B, D, s.hidden)
     return BlockInputs(q, k_blk, v_blk, hidden, target, scale)
+
+
+@dataclass
+class VerifyInputs:
+    q: np.ndarray        # [B, D, Hq, d]  queries of the verification pass
+    k_blk: np.ndarray    # [B, 2D, Hkv, d] rows 0..D-1: the real tokens' keys (= the block's k_blk), D..2D-1: the [m] keys
+    v_blk: np.ndarray    # [B, 2D, Hkv, d]
+
+
+def verify_inputs(w: Workload, w_lm_bits: np.ndarray, step: int = 0) -> VerifyInputs:
+    """Inputs of the second (verification) pass of a self-speculative step: new query rows and the
+    keys / values of the [m] placed at each position, on top of the block's own rows as the real
+    tokens' keys / values.  A pure function of (seed, step); values ~ N(0,1)."""
+    s = w.shape
+    B, D = w.batch, w.block
+    x = block_inputs(w, w_lm_bits, step)
+    q = normal_bf16(w.seed, _T_QVER, (B, D, s.n_q_heads, s.head_dim), sub=step)
+    k_m = normal_bf16(w.seed, _T_KMASK, (B, D, s.n_kv_heads, s.head_dim), sub=step)
+    v_m = normal_bf16(w.seed, _T_VMASK, (B, D, s.n_kv_heads, s.head_dim), sub=step)
+    return VerifyInputs(q, np.concatenate([x.k_blk, k_m], axis=1), np.concatenate([x.v_blk, v_m], axis=1))
+
+
+def random_visibility(seed: int, batch: int, n_q: int, n_k: int, step: int = 0) -> np.ndarray:
+    """Random visibility words [batch, n_q] (uint32): each block key is visible with probability 1/2,
+    and position j always sees key j mod n_k, so no position is left without a key."""
+    bits = _rng(seed, _T_VIS, step).integers(0, 2, size=(batch, n_q, n_k), dtype=np.int64)
+    for j in range(n_q):
+        bits[:, j, j % n_k] = 1
+    return (bits << np.arange(n_k, dtype=np.int64)).sum(axis=2).astype(np.uint32)
+
+
+def agreement_pattern(seed: int, batch: int, D: int, p_agree: float = 0.8, step: int = 0) -> np.ndarray:
+    """[batch, D] booleans: where a synthetic verification pass repeats the first pass's token."""
+    return _rng(seed, _T_AGREE, step).random((batch, D)) < p_agree
 
 
 def kv_read_bytes(w: Workload, lengths: np.ndarray) -> int:

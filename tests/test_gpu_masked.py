@@ -1,0 +1,147 @@
+"""GPU parity of the masked block attention and the self-speculative acceptance (Sec. 3.3, Sec. 3.4)
+with the oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2509_24007_b200 as pk
+from paper_2509_24007_b200.binding import SdlmError
+from paper_2509_24007_b200.harness import DeviceProblem, verification_mask
+from oracle import sdlm_oracle as orc
+import sdlm_synth as syn
+from oracle_side import check_attention, oracle_cache
+
+pytestmark = pytest.mark.gpu
+
+
+def _dev_bits(bits):
+    return pk.bf16_tensor_from_bits(bits)
+
+
+def _vis_tensor(vis):
+    return torch.from_numpy(np.ascontiguousarray(vis.astype(np.uint32)).view(np.int32)).cuda()
+
+
+def _problem(shape, lens, D, seed):
+    lens = np.asarray(lens, dtype=np.int32)
+    wl = syn.Workload("masked", shape, len(lens), D, 0, 0, (0.9,), seed=seed)
+    return wl, DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16), lengths=lens)
+
+
+def _rows(wl, n_rows, step, shape_heads):
+    """n_rows block rows per sequence ([B, n_rows, heads, d] bf16 bits), drawn D at a time."""
+    parts, got, i = [], 0, 0
+    while got < n_rows:
+        x = syn.block_inputs(wl, np.zeros((wl.shape.vocab, wl.shape.hidden), np.uint16), step * 16 + i)
+        parts.append(x.q if shape_heads == "q" else (x.k_blk if shape_heads == "k" else x.v_blk))
+        got += wl.block; i += 1
+    return np.ascontiguousarray(np.concatenate(parts, axis=1)[:, :n_rows])
+
+
+@pytest.mark.parametrize("Hq,Hkv,d", [(4, 2, 64), (16, 2, 128), (8, 1, 64), (2, 2, 128)])
+@pytest.mark.parametrize("n_q,n_k", [(4, 4), (4, 8), (3, 16), (8, 5), (1, 9), (7, 7)])
+def test_masked_attention_random_visibility(Hq, Hkv, d, n_q, n_k):
+    if (Hq // Hkv) * n_q > 64:
+        pytest.skip("more than 64 stacked query rows")
+    shape = syn.Shape(Hq, Hkv, d, 64, 64)
+    lens = [0, 1, 63, 64, 65, 200, 1000]
+    wl, dp = _problem(shape, lens, n_q, seed=700 + Hq + n_q + n_k)
+    q = _rows(wl, n_q, 0, "q"); k = _rows(wl, n_k, 1, "k"); v = _rows(wl, n_k, 2, "v")
+    vis = syn.random_visibility(wl.seed, len(lens), n_q, n_k)
+    out = dp.sd.block_attn_masked(_dev_bits(q), _dev_bits(k), _dev_bits(v), _vis_tensor(vis))
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+    pk_, pv_ = zip(*dp.prefix)
+    ref = orc.block_attention_masked(q, k, v, pk_, pv_, vis.astype(np.int64))
+    check_attention(pk.bits_from_bf16_tensor(out), ref)
+
+
+def test_masked_attention_with_every_bit_set_is_the_unmasked_call_bit_for_bit():
+    shape = syn.Shape(16, 2, 128, 64, 64)
+    wl, dp = _problem(shape, [5, 130, 4000], 4, seed=41)
+    x = dp.block(0)
+    vis = _vis_tensor(np.full((3, 4), 0xF, dtype=np.uint32))
+    a = dp.sd.block_attn_masked(x.q, x.k_blk, x.v_blk, vis)
+    b = dp.sd.block_attn(x.q, x.k_blk, x.v_blk)
+    assert torch.equal(a, b)
+
+
+def test_masked_attention_long_prefix_split_over_many_thread_blocks():
+    """A range that holds only the block's tile meets rows that see none of its keys there."""
+    shape = syn.Shape(16, 2, 128, 64, 64)
+    wl, dp = _problem(shape, [20000, 64 * 9, 3], 4, seed=43)
+    q = _rows(wl, 4, 0, "q"); k = _rows(wl, 8, 1, "k"); v = _rows(wl, 8, 2, "v")
+    vis = np.tile(orc.verification_visibility(4).astype(np.uint32), (3, 1))
+    vis[1] = [1 << 7, 1 << 0, 0, 0b10101010]          # sequence 1: a position that sees no block key at all
+    out = dp.sd.block_attn_masked(_dev_bits(q), _dev_bits(k), _dev_bits(v), _vis_tensor(vis))
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+    pk_, pv_ = zip(*dp.prefix)
+    check_attention(pk.bits_from_bf16_tensor(out), orc.block_attention_masked(q, k, v, pk_, pv_, vis.astype(np.int64)))
+
+
+def test_the_library_side_verification_mask_is_the_oracles():
+    for D in range(1, 9):
+        assert np.array_equal(verification_mask(D).astype(np.int64), orc.verification_visibility(D))
+
+
+@pytest.mark.parametrize("name", ["cfg2_d4", "cfg2"])
+def test_verification_pass_attention_at_full_size(name):
+    """Batch 32, ragged 512..4096 prefixes: the verification pass's attention (2D block keys) on a sample."""
+    wl = syn.CONFIGS[name]
+    dp = DeviceProblem(wl, keep_prefix=True)
+    ver = syn.verify_inputs(wl, dp.w_bits, 0)
+    vis = np.tile(verification_mask(wl.block), (wl.batch, 1))
+    out = dp.sd.block_attn_masked(_dev_bits(ver.q), _dev_bits(ver.k_blk), _dev_bits(ver.v_blk), _vis_tensor(vis))
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+    order = np.argsort(dp.lengths)
+    sample = sorted({int(order[0]), int(order[-1]), 0, wl.batch - 1, 13})
+    pk_, pv_ = zip(*[dp.prefix[b] for b in sample])
+    ref = orc.block_attention_masked(ver.q[sample], ver.k_blk[sample], ver.v_blk[sample], pk_, pv_,
+                                     vis[sample].astype(np.int64))
+    check_attention(pk.bits_from_bf16_tensor(out)[sample], ref)
+
+
+@pytest.mark.parametrize("D,p_agree", [(4, 0.8), (8, 0.9), (1, 0.5), (8, 0.0), (5, 1.0)])
+def test_verify_commit_matches_the_oracle(D, p_agree):
+    shape = syn.SHAPE_TINY
+    lens = np.array([0, 60, 64, 127, 300, 63], dtype=np.int32)
+    wl = syn.Workload("verify", shape, len(lens), D, 0, 0, (0.9,), seed=900 + D)
+    dp = DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16), lengths=lens)
+    cache = oracle_cache(wl, dp.lengths, dp.num_pages, dp.mpps, dp.prefix)
+    rng = np.random.default_rng(D)
+    for step in range(3):
+        x = syn.block_inputs(wl, dp.w_bits, step)
+        draft = rng.integers(0, shape.vocab, size=(len(lens), D)).astype(np.int32)
+        agree = syn.agreement_pattern(wl.seed, len(lens), D, p_agree, step)
+        verify = np.where(agree, draft, (draft + 1) % shape.vocab).astype(np.int32)
+        acc, out_tok = dp.sd.verify_commit(torch.from_numpy(draft).cuda(), torch.from_numpy(verify).cuda(),
+                                           _dev_bits(x.k_blk), _dev_bits(x.v_blk))
+        torch.cuda.synchronize()
+        res = orc.verify_and_commit(cache, range(len(lens)), draft, verify, x.k_blk, x.v_blk)
+        assert np.array_equal(acc.cpu().numpy(), res.accepted_len)
+        assert np.array_equal(out_tok.cpu().numpy(), res.out_tokens)
+        t = dp.sd.kv_tables()
+        assert t["status"][0] == 0
+        assert np.array_equal(t["page_table"], cache.page_table) and np.array_equal(t["seq_len"], cache.seq_len)
+        for b in range(len(lens)):
+            k, v = dp.sd.kv_gather(b, int(cache.seq_len[b]))
+            ok, ov = cache.gather_fast(b)
+            assert np.array_equal(pk.bits_from_bf16_tensor(k), ok) and np.array_equal(pk.bits_from_bf16_tensor(v), ov)
+
+
+def test_masked_attention_rejects_bad_arguments():
+    shape = syn.Shape(16, 2, 128, 64, 64)
+    wl, dp = _problem(shape, [10, 20], 4, seed=5)
+    x = dp.block(0)
+    vis = _vis_tensor(np.full((2, 4), 1, dtype=np.uint32))
+    big = torch.zeros((2, 17, 2, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(SdlmError) as e:
+        dp.sd.block_attn_masked(x.q, big, big, vis)
+    assert e.value.code == 2          # SDLM_ERR_SHAPE
+    q9 = torch.zeros((2, 9, 16, 128), dtype=torch.bfloat16, device="cuda")     # 8 * 9 stacked rows > 64 (and > max_block)
+    with pytest.raises(SdlmError):
+        dp.sd.block_attn_masked(q9, x.k_blk, x.v_blk, _vis_tensor(np.full((2, 9), 1, dtype=np.uint32)))
+    with pytest.raises(ValueError):
+        dp.sd.block_attn_masked(x.q, x.k_blk, x.v_blk, _vis_tensor(np.full((2, 3), 1, dtype=np.uint32)))
