@@ -289,6 +289,43 @@ def time_workload(torch, dp, wl, steps, warmup, n_blocks=4, use_graph=True, over
             "sweep_us": {str(k): round(v * 1e3, 1) for k, v in sorted(sweep.items())}}
 
 
+def time_speculative(torch, dp, wl, steps, warmup, n_blocks=4, p_agree=0.8):
+    """Self-speculative steps (Sec. 3.4): first pass, verification pass (masked attention over 2D block
+    keys), gamma_verify + commit; five library calls per step, device-timed like the main loop."""
+    sd = dp.sd
+    blocks = [(dp.block(i), dp.verify_block(i, p_agree)) for i in range(n_blocks)]
+    out, out_v = dp.alloc_outputs(), dp.alloc_outputs()
+    acc = torch.zeros((steps, wl.batch), dtype=torch.int32, device=sd.device)
+    saved = sd.kv_save()
+    stream = torch.cuda.current_stream()
+
+    def run(n, first, keep):
+        for i in range(n):
+            if i % RESTORE_EVERY == 0:
+                sd.kv_restore(saved)
+            x, xv = blocks[(first + i) % n_blocks]
+            dp.speculative_step(x, xv, out, out_v)
+            if keep:
+                acc[i].copy_(out.accepted_len, non_blocking=True)
+
+    run(warmup, 0, False)
+    torch.cuda.synchronize()
+    n0 = sd.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    run(steps, warmup, True)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    sd.kv_restore(saved)
+    torch.cuda.synchronize()
+    assert int(sd.device_status()[0]) == 0, "device status set during the self-speculative steps"
+    tokens = int(acc.clamp(min=0).sum().item())
+    return {"value": tokens / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / steps, "tokens_per_step": tokens / steps,
+            "launches_per_step": (sd.launch_count() - n0) / steps,
+            "what": f"first pass + verification pass + verified commit, synthetic agreement {p_agree} per position"}
+
+
 def time_e2e(torch, dp, wl, steps, warmup, n_blocks=4):
     """Same metric through sdlm_decode_step_host: pinned host inputs copied in, results copied out, every step."""
     s = wl.shape
@@ -433,6 +470,11 @@ def main():
                                         "ms_per_step": r8["ms_per_step"], "lm_ms": r8["lm_ms"], "attn_ms": r8["attn_ms"],
                                         "attention_sms": r8["attn_sms"]}}
             del dp8
+        if args.workload == "cfg2_d4":
+            dps = DeviceProblem(wl_run, keep_prefix=False)
+            line["extra"]["self_speculative_" + wl.name] = time_speculative(torch, dps, wl_run, max(8, min(args.steps, 200)), 3)
+            del dps
+            torch.cuda.empty_cache()
         n_seqs = min(wl.batch, 32)
         tok, dt = oracle_sample(wl, n_seqs, repeats=2)
         line["cpu_baseline"] = {"value": tok / dt, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",

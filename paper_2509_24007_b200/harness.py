@@ -33,6 +33,18 @@ class DeviceBlock:
 
 
 @dataclass
+class DeviceVerify:
+    q: torch.Tensor        # [B, D, Hq, d]
+    k_blk: torch.Tensor    # [B, 2D, Hkv, d]: real tokens' keys, then the [m] keys
+    v_blk: torch.Tensor
+    hidden: torch.Tensor   # [B, D, H]
+    vis: torch.Tensor      # [B, D] int32 (uint32 visibility words)
+    host: "syn.VerifyInputs"
+    host_hidden: np.ndarray
+    host_vis: np.ndarray
+
+
+@dataclass
 class StepOutputs:
     attn: torch.Tensor
     token: torch.Tensor
@@ -77,6 +89,28 @@ class DeviceProblem:
         x = syn.block_inputs(self.wl, self.w_bits, step)
         return DeviceBlock(bf16_tensor_from_bits(x.q), bf16_tensor_from_bits(x.k_blk), bf16_tensor_from_bits(x.v_blk),
                            bf16_tensor_from_bits(x.hidden), x)
+
+    def verify_block(self, step: int = 0, p_agree: float = 0.8) -> "DeviceVerify":
+        """Device copies of the verification pass's inputs of step `step` (self-speculative decoding)."""
+        wl = self.wl
+        v = syn.verify_inputs(wl, self.w_bits, step)
+        h = syn.verify_hidden(wl, self.w_bits, step, p_agree)
+        vis = np.tile(verification_mask(wl.block), (wl.batch, 1))
+        return DeviceVerify(bf16_tensor_from_bits(v.q), bf16_tensor_from_bits(v.k_blk), bf16_tensor_from_bits(v.v_blk),
+                            bf16_tensor_from_bits(h), torch.from_numpy(vis.view(np.int32)).to(self.sd.device), v, h, vis)
+
+    def speculative_step(self, x: DeviceBlock, xv: "DeviceVerify", out: StepOutputs, out_v: StepOutputs,
+                         stream=None) -> None:
+        """One self-speculative step (Sec. 3.4) on device-resident inputs, five library calls: first pass
+        (attention, LM head -> speculative tokens), verification pass (masked attention over the real
+        tokens' and the [m] keys, LM head -> verification tokens), then gamma_verify and the commit of
+        the kept real-token rows.  No host synchronisation."""
+        sd = self.sd
+        sd.block_attn(x.q, x.k_blk, x.v_blk, out.attn, stream=stream)
+        sd.lmhead_confidence(x.hidden, self.w_lm, out.token, out.p_top1, out.entropy, stream=stream)
+        sd.block_attn_masked(xv.q, xv.k_blk, xv.v_blk, xv.vis, out_v.attn, stream=stream)
+        sd.lmhead_confidence(xv.hidden, self.w_lm, out_v.token, out_v.p_top1, out_v.entropy, stream=stream)
+        sd.verify_commit(out.token, out_v.token, x.k_blk, x.v_blk, out.accepted_len, out.out_tokens, stream=stream)
 
     def alloc_outputs(self) -> StepOutputs:
         wl, s, dev = self.wl, self.wl.shape, self.sd.device

@@ -250,6 +250,17 @@ def verify_inputs(w: Workload, w_lm_bits: np.ndarray, step: int = 0) -> VerifyIn
     return VerifyInputs(q, np.concatenate([x.k_blk, k_m], axis=1), np.concatenate([x.v_blk, v_m], axis=1))
 
 
+def verify_hidden(w: Workload, w_lm_bits: np.ndarray, step: int = 0, p_agree: float = 0.8) -> np.ndarray:
+    """Hidden states [B, D, H] of the verification pass: the first pass's row where the synthetic
+    agreement pattern says the two passes agree (so both heads give the same token), a row drawn for
+    another step elsewhere.  Position 0 always agrees (same input in both passes)."""
+    x = block_inputs(w, w_lm_bits, step)
+    other = block_inputs(w, w_lm_bits, step + 7919)
+    agree = agreement_pattern(w.seed, w.batch, w.block, p_agree, step)
+    agree[:, 0] = True
+    return np.where(agree[..., None], x.hidden, other.hidden)
+
+
 def random_visibility(seed: int, batch: int, n_q: int, n_k: int, step: int = 0) -> np.ndarray:
     """Random visibility words [batch, n_q] (uint32): each block key is visible with probability 1/2,
     and position j always sees key j mod n_k, so no position is left without a key."""

@@ -131,6 +131,47 @@ def test_verify_commit_matches_the_oracle(D, p_agree):
             assert np.array_equal(pk.bits_from_bf16_tensor(k), ok) and np.array_equal(pk.bits_from_bf16_tensor(v), ov)
 
 
+@pytest.mark.parametrize("name,batch", [("cfg0", 4), ("cfg2_d4", 8), ("cfg2", 5)])
+def test_self_speculative_step_matches_the_oracle(name, batch):
+    """Two passes and the verified commit, several steps in a row, against the oracle's composition."""
+    from oracle_side import check_tokens, check_confidences
+    wl = syn.CONFIGS[name].with_(batch=batch, prefix_lo=30, prefix_hi=500, steps=8)
+    dp = DeviceProblem(wl)
+    cache = oracle_cache(wl, dp.lengths, dp.num_pages, dp.mpps, dp.prefix)
+    out, out_v = dp.alloc_outputs(), dp.alloc_outputs()
+    w64 = orc.widen(dp.w_bits) if name == "cfg0" else None
+    kept = []
+    for step in range(3):
+        x, xv = dp.block(step), dp.verify_block(step, p_agree=0.7)
+        pk_, pv_ = zip(*[cache.gather_fast(b) for b in range(batch)])
+        dp.speculative_step(x, xv, out, out_v)
+        torch.cuda.synchronize()
+        assert dp.sd.device_status()[0] == 0
+        check_attention(pk.bits_from_bf16_tensor(out.attn), orc.block_attention(x.host.q, x.host.k_blk, x.host.v_blk, pk_, pv_))
+        check_attention(pk.bits_from_bf16_tensor(out_v.attn),
+                        orc.block_attention_masked(xv.host.q, xv.host.k_blk, xv.host.v_blk, pk_, pv_,
+                                                   xv.host_vis.astype(np.int64)))
+        flagged = []
+        st1 = orc.lm_head_statistics(x.host.hidden, dp.w_bits, w64)
+        st2 = orc.lm_head_statistics(xv.host_hidden, dp.w_bits, w64)
+        check_tokens(out.token.cpu().numpy(), st1, flagged)
+        check_tokens(out_v.token.cpu().numpy(), st2, flagged)
+        check_confidences(out_v.p_top1.cpu().numpy(), out_v.entropy.cpu().numpy(), st2)
+        assert not flagged, flagged      # no near-tie among these seeds: both sides decode the same tokens
+        res = orc.verify_and_commit(cache, range(batch), st1.token.reshape(batch, wl.block),
+                                    st2.token.reshape(batch, wl.block), x.host.k_blk, x.host.v_blk)
+        assert np.array_equal(out.accepted_len.cpu().numpy(), res.accepted_len)
+        assert np.array_equal(out.out_tokens.cpu().numpy(), res.out_tokens)
+        t = dp.sd.kv_tables()
+        assert np.array_equal(t["page_table"], cache.page_table) and np.array_equal(t["seq_len"], cache.seq_len)
+        kept += res.accepted_len.tolist()
+    assert min(kept) >= 1 and max(kept) > 1        # the synthetic agreement pattern keeps more than one token somewhere
+    for b in range(batch):
+        k, v = dp.sd.kv_gather(b, int(cache.seq_len[b]))
+        ok, ov = cache.gather_fast(b)
+        assert np.array_equal(pk.bits_from_bf16_tensor(k), ok) and np.array_equal(pk.bits_from_bf16_tensor(v), ov)
+
+
 def test_masked_attention_rejects_bad_arguments():
     shape = syn.Shape(16, 2, 128, 64, 64)
     wl, dp = _problem(shape, [10, 20], 4, seed=5)
