@@ -46,6 +46,9 @@ keys) and verified_length / verify_and_commit (self-speculative decoding, Sec. 3
 returns that key's value row; invisible keys can hold anything; the causal mask equals token-by-token
 decoding with block_attention; permuting block keys together with the mask bits changes nothing;
 verified_length on hand-worked cases, against brute force, and where it parts from the printed formula.
+carry_visibility / accept_and_commit_carry (a block preceded by rows of real tokens): the words equal
+the literal mask A_uv over [history ; carry ; block]; attention under them equals dense attention under
+that mask; a loop of such steps leaves in the cache exactly the real tokens' rows whatever gamma was.
 """
 from __future__ import annotations
 
@@ -137,6 +140,23 @@ def block_attention_masked(q_bits: np.ndarray, k_blk_bits: np.ndarray, v_blk_bit
                     wgt = np.exp(s - m)
                     out[b, j, h] = (wgt @ vals) / np.sum(wgt)
     return out
+
+
+def carry_visibility(carry_len: Sequence[int], c_max: int, D: int) -> np.ndarray:
+    """vis[b, r] for a block that is preceded by carry_len[b] <= c_max rows of real tokens (the tokens
+    accepted in the previous step whose K/V were never computed from real inputs), laid out as
+    c_max + D rows / keys: rows 0..c_max-1 the carry rows (those >= carry_len[b] are padding), rows
+    c_max.. the D block positions.  With i the block's first position, Sec. 3.3's mask
+    A_uv = 1[v <= u] OR 1[u >= i and v >= i] gives: carry row r sees carry keys <= r (strictly causal,
+    u < i); a block position sees every carry key of the sequence and every block key.  A padding
+    row sees only its own key (its output is unused; this keeps its softmax defined)."""
+    vis = np.zeros((len(carry_len), c_max + D), dtype=np.int64)
+    block_bits = ((1 << D) - 1) << c_max
+    for b, c in enumerate(carry_len):
+        for r in range(c_max):
+            vis[b, r] = (1 << (r + 1)) - 1 if r < c else 1 << r
+        vis[b, c_max:] = ((1 << int(c)) - 1) | block_bits
+    return vis
 
 
 def verification_visibility(D: int) -> np.ndarray:
@@ -391,6 +411,27 @@ def accept_and_commit(cache: PagedKVCache, seq_ids: Sequence[int], token: np.nda
         g, margin[b] = accepted_length([float(c) for c in conf[b]], tau)
         for t in range(g):
             cache.append_token(int(seq_ids[b]), k_blk_bits[b, t], v_blk_bits[b, t])
+        acc[b] = g
+        out[b, :g] = token[b, :g]
+    return CommitResult(acc, out, margin)
+
+
+def accept_and_commit_carry(cache: PagedKVCache, seq_ids: Sequence[int], token: np.ndarray, conf: np.ndarray,
+                            tau: float, carry_len: Sequence[int], c_max: int, k_rows_bits: np.ndarray,
+                            v_rows_bits: np.ndarray) -> CommitResult:
+    """Acceptance as accept_and_commit (gamma of Eq. 7 over the D block positions, first gamma tokens
+    emitted), but only K/V computed from real tokens enter the cache: the carry_len[b] carry rows
+    (rows 0.. of k_rows / v_rows [B, c_max + D, Hkv, d]) and block position 0 (row c_max, the token
+    x^{i-1}), as carry_len[b] + 1 single-token appends, sequences in batch order.  The gamma - 1
+    tokens accepted beyond position 0 are the next step's carry rows."""
+    B, D = token.shape
+    acc = np.zeros(B, np.int32)
+    out = np.full((B, D), -1, np.int32)
+    margin = np.zeros(B)
+    for b in range(B):
+        g, margin[b] = accepted_length([float(c) for c in conf[b]], tau)
+        for r in list(range(int(carry_len[b]))) + [c_max]:
+            cache.append_token(int(seq_ids[b]), k_rows_bits[b, r], v_rows_bits[b, r])
         acc[b] = g
         out[b, :g] = token[b, :g]
     return CommitResult(acc, out, margin)

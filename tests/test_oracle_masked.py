@@ -159,3 +159,83 @@ def test_verify_and_commit_appends_the_kept_rows_like_single_appends():
     assert cache.seq_len[:2].tolist() == [66, 6]
     k0, v0 = cache.gather_fast(0)
     assert np.array_equal(k0[63:], k[0, :3]) and np.array_equal(v0[63:], v[0, :3])
+
+
+# ---- a block preceded by rows of real tokens (carry rows) ----------------------------------------
+def _literal_mask(P, D):
+    """A_uv = 1[v <= u] OR 1[u >= i and v >= i] with i = P, as a (P+D)x(P+D) 0/1 matrix (Sec. 3.3)."""
+    n = P + D
+    A = np.zeros((n, n), dtype=bool)
+    for u in range(n):
+        for v in range(n):
+            A[u, v] = (v <= u) or (u >= P and v >= P)
+    return A
+
+
+@pytest.mark.parametrize("P,c,D", [(0, 0, 4), (3, 2, 4), (5, 3, 4), (2, 7, 8), (0, 1, 1)])
+def test_carry_visibility_is_the_literal_mask_over_history_carry_block(P, c, D):
+    """Rows of [history ; carry ; block] from the first carry row on, columns of carry and block keys."""
+    A = _literal_mask(P + c, D)                       # the block starts after history and carry rows
+    vis = orc.carry_visibility([c], c, D)[0]          # no padding rows: c_max = c
+    for r in range(c + D):
+        for t in range(c + D):
+            assert bool((int(vis[r]) >> t) & 1) == bool(A[P + r, P + t])
+        assert all(A[P + r, :P])                      # and the whole history, which the call always shows
+
+
+def test_carry_attention_equals_dense_attention_under_the_literal_mask():
+    P, c, D, Hq, Hkv, d = 6, 3, 4, 4, 2, 8
+    rng = np.random.default_rng(11)
+    n = P + c + D
+    q_all, k_all, v_all = (_rand_bits(rng, (n, h, d)) for h in (Hq, Hkv, Hkv))
+    f = lambda bits: torch.from_numpy(syn.bf16_bits_to_f32(bits).astype(np.float64))
+    A = torch.from_numpy(_literal_mask(P + c, D))
+    vis = orc.carry_visibility([c], c, D)
+    out = orc.block_attention_masked(q_all[None, P:], k_all[None, P:], v_all[None, P:], [k_all[:P]], [v_all[:P]], vis)
+    for u in range(P, n):
+        for h in range(Hq):
+            s = (f(k_all)[:, h // 2] @ f(q_all)[u, h]) / np.sqrt(d)
+            s = torch.where(A[u], s, torch.tensor(float("-inf"), dtype=torch.float64))
+            ref = torch.softmax(s, 0) @ f(v_all)[:, h // 2]
+            assert torch.allclose(torch.from_numpy(out[0, u - P, h]), ref, rtol=0, atol=1e-13)
+
+
+def test_padding_carry_rows_change_nothing_for_the_real_rows():
+    """c_max = 3 with carry_len = 1: the two padding rows / keys may hold anything."""
+    P, D, Hq, Hkv, d = 4, 4, 2, 1, 8
+    q, k, v, pk, pv = _case(12, 1, 1 + D, 1 + D, Hq, Hkv, d, (P,))
+    tight = orc.block_attention_masked(q, k, v, pk, pv, orc.carry_visibility([1], 1, D))
+    rng = np.random.default_rng(13)
+    pad = lambda x, h: np.concatenate([x[:, :1], _rand_bits(rng, (1, 2, h, d)), x[:, 1:]], axis=1)
+    padded = orc.block_attention_masked(pad(q, Hq), pad(k, Hkv), pad(v, Hkv), pk, pv, orc.carry_visibility([1], 3, D))
+    assert np.array_equal(padded[:, [0, 3, 4, 5, 6]], tight)
+
+
+def test_a_loop_of_carry_steps_leaves_only_real_token_rows_in_the_cache():
+    """Every token position has one true K/V row; [m] rows are junk.  Whatever tau accepts, after N
+    steps the cache is exactly the true rows of the positions it covers (what commit rows 0..gamma-1
+    of the block, masks included, cannot give)."""
+    D, c_max, Hkv, d, B = 4, 3, 2, 64, 3
+    rng = np.random.default_rng(21)
+    true_k, true_v = _rand_bits(rng, (B, 400, Hkv, d)), _rand_bits(rng, (B, 400, Hkv, d))
+    cache = orc.PagedKVCache(num_pages=24, page_size=64, n_kv_heads=Hkv, head_dim=d, max_batch=B, max_pages_per_seq=8)
+    start = [60, 0, 130]
+    for b in range(B):
+        cache.add_sequence(b, true_k[b, :start[b]], true_v[b, :start[b]])
+    carry = [0] * B
+    for step in range(12):
+        k_rows, v_rows = _rand_bits(rng, (B, c_max + D, Hkv, d)), _rand_bits(rng, (B, c_max + D, Hkv, d))   # junk
+        for b in range(B):
+            L = int(cache.seq_len[b])
+            for r in range(carry[b]):                         # carry rows: the real tokens right after the cache
+                k_rows[b, r], v_rows[b, r] = true_k[b, L + r], true_v[b, L + r]
+            k_rows[b, c_max], v_rows[b, c_max] = true_k[b, L + carry[b]], true_v[b, L + carry[b]]   # slot 0 = x^{i-1}
+        conf = rng.random((B, D)) * 0.5 + 0.5
+        token = rng.integers(0, 1000, size=(B, D)).astype(np.int32)
+        res = orc.accept_and_commit_carry(cache, range(B), token, conf, 0.6, carry, c_max, k_rows, v_rows)
+        carry = [int(g) - 1 for g in res.accepted_len]
+        assert all(0 <= c <= c_max for c in carry)
+    for b in range(B):
+        L = int(cache.seq_len[b])
+        k, v = cache.gather_fast(b)
+        assert L > start[b] and np.array_equal(k, true_k[b, :L]) and np.array_equal(v, true_v[b, :L])
