@@ -234,6 +234,22 @@ sdlm_status sdlm_verify_commit(sdlm_ctx* ctx, int32_t batch, int32_t D, const in
                                const int32_t* draft_token, const int32_t* verify_token, const void* k_blk,
                                const void* v_blk, int32_t* accepted_len, int32_t* out_tokens, void* stream);
 
+/* ---- (c'') acceptance + commit for a block preceded by carry rows -- Sec. 3.3 / 3.2: the tokens a
+ * step accepts beyond position 0 were predicted at [m] inputs, so their K/V do not exist yet; the
+ * next step feeds them as rows of real tokens in front of its block (attending causally:
+ * sdlm_block_attn_masked with causal words for those rows), and only K/V of real tokens enter the cache.
+ * k_rows / v_rows [batch, c_max + D, Hkv, d]: rows 0..carry_len[b]-1 the carry rows of sequence b
+ * (device int32 carry_len [batch], each in 0..c_max; the rows up to c_max are padding), row c_max the
+ * block's position 0 (x^{i-1}).  accepted_len / out_tokens: exactly as sdlm_accept_commit (Eq. 7 over
+ * the D block positions); the cache grows by the carry_len[b] + 1 real rows, appended as single
+ * tokens in order.  accepted_len[b] - 1 is the next step's carry_len[b].  c_max + D <= 16.
+ * Errors and device-side checks: as sdlm_accept_commit; a carry_len outside 0..c_max is reported as
+ * SDLM_ERR_DEVICE_CHECK and that sequence is left unchanged. */
+sdlm_status sdlm_accept_commit_carry(sdlm_ctx* ctx, int32_t batch, int32_t D, int32_t c_max, const int32_t* seq_ids,
+                                     const int32_t* carry_len, float tau, sdlm_conf_mode mode, const int32_t* token,
+                                     const float* p_top1, const float* entropy, const void* k_rows,
+                                     const void* v_rows, int32_t* accepted_len, int32_t* out_tokens, void* stream);
+
 /* Synchronises `stream` and copies the sticky device status words to host_out[4]:
  * {sdlm_status (0 = none), sequence slot of the first failure, detail, number of failures}.
  * `clear` != 0 resets them afterwards. */

@@ -31,7 +31,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "UNSUPPORTED", 4: "OUT
 EXPORTED = ["sdlm_pool_bytes", "sdlm_workspace_bytes", "sdlm_create", "sdlm_destroy", "sdlm_status_str",
             "sdlm_kv_pages", "sdlm_block_attn", "sdlm_lmhead_confidence", "sdlm_lmhead_confidence_static", "sdlm_accept_commit",
             "sdlm_device_status", "sdlm_decode_step", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count",
-            "sdlm_block_attn_masked", "sdlm_verify_commit"]
+            "sdlm_block_attn_masked", "sdlm_verify_commit", "sdlm_accept_commit_carry"]
 
 
 class SdlmError(RuntimeError):
@@ -111,6 +111,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdlm_lmhead_confidence_static.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_block_attn_masked.restype = C.c_int
     lib.sdlm_block_attn_masked.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_accept_commit_carry.restype = C.c_int
+    lib.sdlm_accept_commit_carry.argtypes = [vp, i32, i32, i32, vp, vp, f32, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_verify_commit.restype = C.c_int
     lib.sdlm_verify_commit.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_accept_commit.restype = C.c_int
@@ -326,6 +328,31 @@ class Sdlm:
             _dev(seq_ids, torch.int32, "seq_ids")
         self._check("sdlm_verify_commit", self.lib.sdlm_verify_commit(
             self.ctx, batch, D, _ptr(seq_ids), _ptr(draft_token), _ptr(verify_token), _ptr(k_blk), _ptr(v_blk),
+            _ptr(_dev(accepted_len, torch.int32, "accepted_len")), _ptr(_dev(out_tokens, torch.int32, "out_tokens")),
+            _stream_ptr(stream)))
+        return accepted_len, out_tokens
+
+    def accept_commit_carry(self, tau: float, carry_len: torch.Tensor, c_max: int, token: torch.Tensor,
+                            p_top1: torch.Tensor, entropy: torch.Tensor, k_rows: torch.Tensor, v_rows: torch.Tensor,
+                            mode: int = CONF_LOGIT, accepted_len: Optional[torch.Tensor] = None,
+                            out_tokens: Optional[torch.Tensor] = None, seq_ids: Optional[torch.Tensor] = None,
+                            stream=None):
+        """sdlm_accept_commit_carry: k_rows / v_rows are [batch, c_max + D, Hkv, d]."""
+        batch, D = int(token.shape[0]), int(token.shape[1])
+        _dev(carry_len, torch.int32, "carry_len"); _dev(token, torch.int32, "token")
+        _dev(p_top1, torch.float32, "p_top1"); _dev(entropy, torch.float32, "entropy")
+        _dev(k_rows, torch.bfloat16, "k_rows"); _dev(v_rows, torch.bfloat16, "v_rows")
+        if int(k_rows.shape[1]) != c_max + D:
+            raise ValueError("k_rows must hold c_max + D rows per sequence")
+        if accepted_len is None:
+            accepted_len = torch.empty(batch, dtype=torch.int32, device=self.device)
+        if out_tokens is None:
+            out_tokens = torch.empty((batch, D), dtype=torch.int32, device=self.device)
+        if seq_ids is not None:
+            _dev(seq_ids, torch.int32, "seq_ids")
+        self._check("sdlm_accept_commit_carry", self.lib.sdlm_accept_commit_carry(
+            self.ctx, batch, D, int(c_max), _ptr(seq_ids), _ptr(carry_len), float(tau), int(mode), _ptr(token),
+            _ptr(p_top1), _ptr(entropy), _ptr(k_rows), _ptr(v_rows),
             _ptr(_dev(accepted_len, torch.int32, "accepted_len")), _ptr(_dev(out_tokens, torch.int32, "out_tokens")),
             _stream_ptr(stream)))
         return accepted_len, out_tokens

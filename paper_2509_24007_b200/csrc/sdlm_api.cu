@@ -196,6 +196,11 @@ struct CommitParams {
   float* p_top1_copy;
   float* entropy_copy;
   const int32_t* verify_token;  // null: gamma_tau of Eq. 7; else gamma_verify against these tokens
+  // Carry mode (carry_len != null): k_blk / v_blk hold c_max + D rows per sequence, the first
+  // carry_len[b] of them real tokens accepted in the step before, row c_max the block's position 0.
+  // Those carry_len[b] + 1 rows are appended instead of block rows 0..gamma-1; gamma is still output.
+  const int32_t* carry_len;
+  int c_max;
   float tau, inv_ln_vocab;
   int mode, batch, D, Hkv, d, mpps, num_pages;
 };
@@ -229,7 +234,7 @@ __global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitPar
   __shared__ int8_t s_gamma[kMaxBatch];
   __shared__ int8_t s_state[kMaxBatch];  // 0 ok, 1 capacity failure, 2 out of pages
   __shared__ int s_warp[kCommitThreads / 32];
-  __shared__ int s_carry, s_mine[5];     // my row: gamma, need, alloc index, len, state
+  __shared__ int s_carry, s_mine[6];     // my row: gamma, need, alloc index, len, state, rows to append
   __shared__ uint32_t s_head, s_avail;
   __shared__ int s_last;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -244,13 +249,19 @@ __global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitPar
   const uint32_t avail = s_avail;
   for (int base = 0; base < p.batch; base += kCommitThreads) {
     const int i = base + tid;
-    int g = 0, need = 0, state = 0, len = 0;
+    int g = 0, na = 0, need = 0, state = 0, len = 0;
     if (i < p.batch) {
       const int slot = p.seq_ids ? p.seq_ids[i] : i;
       len = *(volatile int32_t*)&p.seq_len[slot];
       g = gamma_tau(p, i);
-      if (len + g > p.mpps * kPageSize) state = 1;
-      else need = (len % kPageSize == 0) || (len % kPageSize + g > kPageSize);
+      na = g;
+      if (p.carry_len) {
+        const int c = p.carry_len[i];
+        if (c < 0 || c > p.c_max) state = 1;  // not a carry length: reported like a capacity failure
+        na = min(max(c, 0), p.c_max) + 1;
+      }
+      if (len + na > p.mpps * kPageSize) state = 1;
+      if (state == 0) need = (len % kPageSize == 0) || (len % kPageSize + na > kPageSize);
     }
     // exclusive scan of `need` in batch order
     int incl = need;
@@ -265,9 +276,9 @@ __global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitPar
     const int alloc = before + incl - need;
     if (need && (uint32_t)alloc >= avail) { state = 2; }
     if (i < p.batch) {
-      s_gamma[i] = (int8_t)g;
+      s_gamma[i] = (int8_t)na;   // what the sequence grows by
       s_state[i] = (int8_t)state;
-      if (i == b) { s_mine[0] = g; s_mine[1] = need; s_mine[2] = alloc; s_mine[3] = len; s_mine[4] = state; }
+      if (i == b) { s_mine[0] = g; s_mine[1] = need; s_mine[2] = alloc; s_mine[3] = len; s_mine[4] = state; s_mine[5] = na; }
     }
     __syncthreads();
     if (tid == kCommitThreads - 1) s_carry = before + incl;
@@ -284,7 +295,7 @@ __global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitPar
   }
 
   // my row
-  const int g = s_mine[0], need = s_mine[1], alloc = s_mine[2], len = s_mine[3], state = s_mine[4];
+  const int g = s_mine[0], need = s_mine[1], alloc = s_mine[2], len = s_mine[3], state = s_mine[4], na = s_mine[5];
   const int slot = p.seq_ids ? p.seq_ids[b] : b;
   for (int k = tid; k < p.D; k += kCommitThreads) {
     if (p.token_copy) p.token_copy[b * p.D + k] = p.token[b * p.D + k];
@@ -314,7 +325,8 @@ __global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitPar
       __syncthreads();
     }
     const int cpr = p.d / 8;
-    const int total = g * p.Hkv * cpr;
+    const int total = na * p.Hkv * cpr;
+    const int rows_per_seq = p.carry_len ? p.c_max + p.D : p.D;
     for (int idx = tid; idx < total; idx += kCommitThreads) {
       const int c = idx % cpr;
       int r = idx / cpr;
@@ -323,7 +335,8 @@ __global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitPar
       const int pos = len + t;
       const int pidx = pos / kPageSize, key = pos % kPageSize;
       const int page = (need && pidx == new_idx) ? new_page : p.page_table[(size_t)slot * p.mpps + pidx];
-      const size_t src = (((size_t)b * p.D + t) * p.Hkv + h) * p.d;
+      const int srow = p.carry_len ? (t < na - 1 ? t : p.c_max) : t;  // carry rows, then the block's position 0
+      const size_t src = (((size_t)b * rows_per_seq + srow) * p.Hkv + h) * p.d;
       *reinterpret_cast<uint4*>(p.pool + kv_tile_offset(page, h, 0, p.Hkv, p.d) + k_tile_elem(key, c * 8)) =
           *(reinterpret_cast<const uint4*>(p.k_blk + src) + c);
       const uint4 vv = *(reinterpret_cast<const uint4*>(p.v_blk + src) + c);
@@ -598,7 +611,8 @@ static sdlm_status accept_commit_launch(sdlm_ctx* ctx, int32_t batch, int32_t D,
                                         sdlm_conf_mode mode, const int32_t* token, const float* p_top1,
                                         const float* entropy, const void* k_blk, const void* v_blk,
                                         int32_t* accepted_len, int32_t* out_tokens, const StatCopies& copies,
-                                        void* stream, const int32_t* verify_token = nullptr) {
+                                        void* stream, const int32_t* verify_token = nullptr,
+                                        const int32_t* carry_len = nullptr, int c_max = 0) {
   if (!ctx || !token || !k_blk || !v_blk || !accepted_len || !out_tokens) return SDLM_ERR_INVALID_ARG;
   if (!verify_token && (!p_top1 || !entropy)) return SDLM_ERR_INVALID_ARG;
   if (!aligned16(k_blk) || !aligned16(v_blk)) return SDLM_ERR_INVALID_ARG;
@@ -615,6 +629,8 @@ static sdlm_status accept_commit_launch(sdlm_ctx* ctx, int32_t batch, int32_t D,
   p.accepted_len = accepted_len; p.out_tokens = out_tokens;
   p.token_copy = copies.token; p.p_top1_copy = copies.p_top1; p.entropy_copy = copies.entropy;
   p.verify_token = verify_token;
+  p.carry_len = carry_len;
+  p.c_max = c_max;
   p.tau = tau;
   p.inv_ln_vocab = c.vocab > 1 ? (float)(1.0 / log((double)c.vocab)) : 0.0f;
   p.mode = (int)mode; p.batch = batch; p.D = D; p.Hkv = c.n_kv_heads; p.d = c.head_dim;
@@ -640,6 +656,17 @@ extern "C" sdlm_status sdlm_verify_commit(sdlm_ctx* ctx, int32_t batch, int32_t 
   if (!verify_token) return SDLM_ERR_INVALID_ARG;
   return accept_commit_launch(ctx, batch, D, seq_ids, 0.5f, SDLM_CONF_LOGIT, draft_token, nullptr, nullptr, k_blk, v_blk,
                               accepted_len, out_tokens, StatCopies{}, stream, verify_token);
+}
+
+extern "C" sdlm_status sdlm_accept_commit_carry(sdlm_ctx* ctx, int32_t batch, int32_t D, int32_t c_max,
+                                                const int32_t* seq_ids, const int32_t* carry_len, float tau,
+                                                sdlm_conf_mode mode, const int32_t* token, const float* p_top1,
+                                                const float* entropy, const void* k_rows, const void* v_rows,
+                                                int32_t* accepted_len, int32_t* out_tokens, void* stream) {
+  if (!carry_len || c_max < 0) return SDLM_ERR_INVALID_ARG;
+  if (c_max + D > kMaxBlockKeys) return SDLM_ERR_SHAPE;
+  return accept_commit_launch(ctx, batch, D, seq_ids, tau, mode, token, p_top1, entropy, k_rows, v_rows, accepted_len,
+                              out_tokens, StatCopies{}, stream, nullptr, carry_len, c_max);
 }
 
 extern "C" sdlm_status sdlm_block_attn_masked(sdlm_ctx* ctx, int32_t batch, int32_t n_q, int32_t n_k,

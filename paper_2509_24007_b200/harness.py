@@ -32,6 +32,20 @@ class DeviceBlock:
     host: syn.BlockInputs
 
 
+def carry_mask(carry_len, c_max: int, D: int) -> np.ndarray:
+    """Visibility words [batch, c_max + D] for sdlm_block_attn_masked when each block is preceded by
+    carry_len[b] <= c_max rows of real tokens (rows / keys 0..c_max-1, padded; then the D block positions):
+    a carry row sees the carry keys up to itself, a padding row only itself, a block position every
+    carry key of its sequence and every block key (Sec. 3.3)."""
+    carry_len = np.asarray(carry_len, dtype=np.int64)
+    out = np.empty((len(carry_len), c_max + D), dtype=np.uint32)
+    r = np.arange(c_max, dtype=np.int64)
+    for b, c in enumerate(carry_len):
+        out[b, :c_max] = np.where(r < c, (np.int64(2) << r) - 1, np.int64(1) << r)
+        out[b, c_max:] = ((1 << int(c)) - 1) + (((1 << D) - 1) << c_max)
+    return out
+
+
 @dataclass
 class DeviceVerify:
     q: torch.Tensor        # [B, D, Hq, d]

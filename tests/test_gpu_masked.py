@@ -186,3 +186,92 @@ def test_masked_attention_rejects_bad_arguments():
         dp.sd.block_attn_masked(q9, x.k_blk, x.v_blk, _vis_tensor(np.full((2, 9), 1, dtype=np.uint32)))
     with pytest.raises(ValueError):
         dp.sd.block_attn_masked(x.q, x.k_blk, x.v_blk, _vis_tensor(np.full((2, 3), 1, dtype=np.uint32)))
+
+
+# ---- a block preceded by carry rows of real tokens ----------------------------------------------
+def test_the_library_side_carry_mask_is_the_oracles():
+    from paper_2509_24007_b200.harness import carry_mask
+    for c_max, D in ((0, 4), (3, 4), (7, 8), (2, 1)):
+        lens = list(range(c_max + 1)) * 2
+        assert np.array_equal(carry_mask(lens, c_max, D).astype(np.int64), orc.carry_visibility(lens, c_max, D))
+
+
+@pytest.mark.parametrize("shape_name,D,c_max", [("tiny", 4, 3), ("3b", 4, 3), ("tiny", 3, 2), ("tiny", 1, 0)])
+def test_carry_step_loop_matches_the_oracle_and_caches_only_real_rows(shape_name, D, c_max):
+    """Several steps of: masked attention over [carry rows ; block], LM head on the block positions,
+    Eq. 7, commit of the real-token rows.  Against the oracle step by step; and at the end the cache
+    holds exactly the true rows of the positions it covers (the junk [m] rows never enter it)."""
+    from paper_2509_24007_b200.harness import carry_mask
+    from oracle_side import check_tokens, check_confidences, check_gamma
+    shape = syn.SHAPE_TINY if shape_name == "tiny" else syn.Shape(16, 2, 128, 256, 1024)
+    B = 4
+    lens = np.array([0, 62, 64, 300], dtype=np.int32)
+    wl = syn.Workload("carry", shape, B, D, 0, 0, (0.9,), steps=8, seed=1200 + D)
+    dp = DeviceProblem(wl, lengths=lens, max_block=c_max + D)
+    cache = oracle_cache(wl, dp.lengths, dp.num_pages, dp.mpps, dp.prefix)
+    rng = np.random.default_rng(D)
+    Hkv, d = shape.n_kv_heads, shape.head_dim
+    true_k = syn.f32_to_bf16_bits(rng.normal(size=(B, 600, Hkv, d)).astype(np.float32))
+    true_v = syn.f32_to_bf16_bits(rng.normal(size=(B, 600, Hkv, d)).astype(np.float32))
+    for b in range(B):                                   # the prefixes the problem was built with are "true" rows too
+        true_k[b, :lens[b]], true_v[b, :lens[b]] = dp.prefix[b]
+    w64 = orc.widen(dp.w_bits)
+    carry = np.zeros(B, dtype=np.int32)
+    R = c_max + D
+    for step in range(5):
+        x = syn.block_inputs(wl, dp.w_bits, step)
+        q = syn.f32_to_bf16_bits(rng.normal(size=(B, R, shape.n_q_heads, d)).astype(np.float32))
+        k_rows = syn.f32_to_bf16_bits(rng.normal(size=(B, R, Hkv, d)).astype(np.float32))     # junk unless overwritten
+        v_rows = syn.f32_to_bf16_bits(rng.normal(size=(B, R, Hkv, d)).astype(np.float32))
+        for b in range(B):
+            L = int(cache.seq_len[b])
+            for r in range(int(carry[b])):
+                k_rows[b, r], v_rows[b, r] = true_k[b, L + r], true_v[b, L + r]
+            k_rows[b, c_max], v_rows[b, c_max] = true_k[b, L + carry[b]], true_v[b, L + carry[b]]
+        vis = carry_mask(carry, c_max, D)
+        pk_, pv_ = zip(*[cache.gather_fast(b) for b in range(B)])
+        dk, dv = _dev_bits(k_rows), _dev_bits(v_rows)
+        attn = dp.sd.block_attn_masked(_dev_bits(q), dk, dv, _vis_tensor(vis))
+        tok, p, ent = dp.sd.lmhead_confidence(_dev_bits(x.hidden), dp.w_lm)[:3]
+        acc, out_tok = dp.sd.accept_commit_carry(wl.tau, torch.from_numpy(carry).cuda(), c_max, tok.view(B, D),
+                                                 p.view(B, D), ent.view(B, D), dk, dv)
+        torch.cuda.synchronize()
+        assert dp.sd.device_status()[0] == 0
+        ref = orc.block_attention_masked(q, k_rows, v_rows, pk_, pv_, vis.astype(np.int64))
+        real = [(b, r) for b in range(B) for r in list(range(int(carry[b]))) + list(range(c_max, R))]
+        got = pk.bits_from_bf16_tensor(attn)
+        idx = tuple(np.array(real).T)
+        check_attention(got[idx], ref[idx])                # padding rows are not outputs
+        stats = orc.lm_head_statistics(x.hidden, dp.w_bits, w64)
+        flagged = []
+        check_tokens(tok.cpu().numpy(), stats, flagged)
+        check_confidences(p.cpu().numpy(), ent.cpu().numpy(), stats)
+        res = orc.accept_and_commit_carry(cache, range(B), stats.token.reshape(B, D), stats.p_top1.reshape(B, D), wl.tau,
+                                          carry, c_max, k_rows, v_rows)
+        assert check_gamma(acc.cpu().numpy(), res, flagged) == 0 and not flagged, flagged
+        assert np.array_equal(out_tok.cpu().numpy(), res.out_tokens)
+        t = dp.sd.kv_tables()
+        assert np.array_equal(t["page_table"], cache.page_table) and np.array_equal(t["seq_len"], cache.seq_len)
+        carry = (res.accepted_len - 1).astype(np.int32)
+    for b in range(B):
+        L = int(cache.seq_len[b])
+        k, v = dp.sd.kv_gather(b, L)
+        assert L > lens[b]
+        assert np.array_equal(pk.bits_from_bf16_tensor(k), true_k[b, :L]) and np.array_equal(pk.bits_from_bf16_tensor(v), true_v[b, :L])
+
+
+def test_carry_commit_reports_a_carry_length_out_of_range():
+    shape = syn.SHAPE_TINY
+    wl = syn.Workload("carry_bad", shape, 2, 4, 0, 0, (0.9,), steps=4, seed=7)
+    dp = DeviceProblem(wl, lengths=np.array([10, 20], dtype=np.int32), max_block=7)
+    x = syn.block_inputs(wl, dp.w_bits, 0)
+    rows = torch.zeros((2, 7, shape.n_kv_heads, shape.head_dim), dtype=torch.bfloat16, device="cuda")
+    tok, p, ent = dp.sd.lmhead_confidence(_dev_bits(x.hidden), dp.w_lm)[:3]
+    acc, _ = dp.sd.accept_commit_carry(0.9, torch.tensor([5, 1], dtype=torch.int32).cuda(), 3, tok.view(2, 4), p.view(2, 4),
+                                       ent.view(2, 4), rows, rows)
+    torch.cuda.synchronize()
+    st = dp.sd.device_status(clear=True)
+    assert st[0] == 7                          # SDLM_ERR_DEVICE_CHECK
+    assert int(acc[0]) == -1 and int(acc[1]) >= 1
+    t = dp.sd.kv_tables()
+    assert t["seq_len"][0] == 10 and t["seq_len"][1] == 22
