@@ -326,6 +326,57 @@ def time_speculative(torch, dp, wl, steps, warmup, n_blocks=4, p_agree=0.8):
             "what": f"first pass + verification pass + verified commit, synthetic agreement {p_agree} per position"}
 
 
+def time_carry(torch, pk, DeviceProblem, wl, steps, warmup, n_blocks=4):
+    """Steps whose block is preceded by up to D-1 carry rows of real tokens (Sec. 3.3 causal rows):
+    masked attention over c_max + D rows / block keys, LM head on the D block positions, Eq. 7, commit
+    of the real-token rows only.  Three library calls per step.  The carry lengths are those a first
+    step's acceptance gives and are held fixed, so that every timed step does the same work."""
+    from paper_2509_24007_b200.harness import carry_mask
+    D, c_max = wl.block, wl.block - 1
+    R = c_max + D
+    dp = DeviceProblem(wl, keep_prefix=False, max_block=R)
+    sd = dp.sd
+    wide = wl.with_(block=R)
+    rows = [syn.block_inputs(wide, dp.w_bits, 300 + i) for i in range(n_blocks)]
+    blocks = [(pk.bf16_tensor_from_bits(r.q), pk.bf16_tensor_from_bits(r.k_blk), pk.bf16_tensor_from_bits(r.v_blk),
+               dp.block(i).hidden) for i, r in enumerate(rows)]
+    out = dp.alloc_outputs()
+    attn = torch.empty((wl.batch, R, wl.shape.n_q_heads, wl.shape.head_dim), dtype=torch.bfloat16, device=sd.device)
+    saved = sd.kv_save()
+    first = dp.step(dp.block(0), wl.tau)                      # a plain step: its gamma - 1 are the carry lengths
+    torch.cuda.synchronize()
+    carry_host = (first.accepted_len.cpu().numpy() - 1).clip(0, c_max).astype(np.int32)
+    carry = torch.from_numpy(carry_host).to(sd.device)
+    vis = torch.from_numpy(carry_mask(carry_host, c_max, D).view(np.int32)).to(sd.device)
+    sd.kv_restore(saved)
+    acc = torch.zeros((steps, wl.batch), dtype=torch.int32, device=sd.device)
+    stream = torch.cuda.current_stream()
+
+    def run(n, first_i, keep):
+        for i in range(n):
+            if i % RESTORE_EVERY == 0:
+                sd.kv_restore(saved)
+            q, k, v, hidden = blocks[(first_i + i) % n_blocks]
+            sd.block_attn_masked(q, k, v, vis, attn)
+            sd.lmhead_confidence(hidden, dp.w_lm, out.token, out.p_top1, out.entropy)
+            sd.accept_commit_carry(wl.tau, carry, c_max, out.token, out.p_top1, out.entropy, k, v, 0,
+                                   acc[i] if keep else out.accepted_len, out.out_tokens)
+
+    run(warmup, 0, False)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    run(steps, warmup, True)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    assert int(sd.device_status()[0]) == 0, "device status set during the carry steps"
+    tokens = int(acc.clamp(min=0).sum().item())
+    return {"value": tokens / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / steps, "tokens_per_step": tokens / steps,
+            "rows_appended_per_step": int(carry_host.sum()) + wl.batch, "query_positions": R,
+            "what": "block preceded by gamma_prev - 1 carry rows of real tokens; only real-token K/V are cached"}
+
+
 def time_e2e(torch, dp, wl, steps, warmup, n_blocks=4):
     """Same metric through sdlm_decode_step_host: pinned host inputs copied in, results copied out, every step."""
     s = wl.shape
@@ -474,6 +525,9 @@ def main():
             dps = DeviceProblem(wl_run, keep_prefix=False)
             line["extra"]["self_speculative_" + wl.name] = time_speculative(torch, dps, wl_run, max(8, min(args.steps, 200)), 3)
             del dps
+            torch.cuda.empty_cache()
+        if args.workload == "cfg2_d4":
+            line["extra"]["carry_over_" + wl.name] = time_carry(torch, pk, DeviceProblem, wl_run, max(8, min(args.steps, 200)), 3)
             torch.cuda.empty_cache()
         n_seqs = min(wl.batch, 32)
         tok, dt = oracle_sample(wl, n_seqs, repeats=2)
