@@ -286,6 +286,31 @@ sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const
                                   float* entropy_host, int32_t* accepted_len_host, int32_t* out_tokens_host,
                                   void* stream);
 
+/* ---- the rest of a decoder layer around (a) (widening; Sec. 4.1: the models are built on the
+ * Qwen-2.5 backbone: RMSNorm, rotary positions in the rotate-half convention, grouped-query attention
+ * with biased q/k/v projections, SwiGLU MLP).  All tensors DEVICE bf16, row-major, 16-byte aligned;
+ * arithmetic fp32, one rounding to bf16 at the end.  None of these touches the cache.
+ *
+ * sdlm_linear:   out[r, n] = sum_k x[r, k] * w[n, k] (+ bias[n]) (+ residual[r, n]); x [rows, K],
+ *                w [N, K], out / residual [rows, N] (out may be residual: in-place accumulation into the
+ *                residual stream).  K % 8 == 0, N % 16 == 0 (else UNSUPPORTED).  Runs on the LM head's
+ *                tcgen05 / TMA stripe kernel, W streamed once per 128 rows.
+ * sdlm_rmsnorm:  out[r, :] = x[r, :] / sqrt(mean_k x[r, k]^2 + eps) * weight[:]; H % 8 == 0.
+ * sdlm_rope_block: rotary embedding, in place, of x [batch, D, n_heads, head_dim]: the position of row
+ *                (b, j) is (length of slot seq_ids[b], or b, as the tables stand on the stream) + j;
+ *                x'[i] = x[i] cos a - x[i + d/2] sin a, x'[i + d/2] = x[i + d/2] cos a + x[i] sin a,
+ *                a = position * theta^(-2i/d), i < d/2.
+ * sdlm_swiglu:   out[r, i] = silu(gate_up[r, i]) * gate_up[r, I + i], silu(g) = g / (1 + e^-g);
+ *                gate_up [rows, 2I], out [rows, I]; I % 8 == 0.
+ * Errors: INVALID_ARG, SHAPE, UNSUPPORTED, CUDA. */
+sdlm_status sdlm_linear(sdlm_ctx* ctx, int32_t rows, int32_t K, int32_t N, const void* x, const void* w,
+                        const void* bias, const void* residual, void* out, void* stream);
+sdlm_status sdlm_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t H, const void* x, const void* weight, float eps,
+                         void* out, void* stream);
+sdlm_status sdlm_rope_block(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, int32_t n_heads, void* x,
+                            float theta, void* stream);
+sdlm_status sdlm_swiglu(sdlm_ctx* ctx, int32_t rows, int32_t I, const void* gate_up, void* out, void* stream);
+
 /* Tuning / test knobs (the paper has no counterpart).  SDLM_OPT_LMHEAD_KERNEL: which stripe kernel
  * sdlm_lmhead_confidence uses: 0 = chosen from the shape (default), 1 = warp-level mma.sync
  * kernel, 2 = tcgen05 / TMA kernel (the call then fails with UNSUPPORTED for rows > 256 or

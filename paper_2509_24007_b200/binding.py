@@ -31,7 +31,8 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "UNSUPPORTED", 4: "OUT
 EXPORTED = ["sdlm_pool_bytes", "sdlm_workspace_bytes", "sdlm_create", "sdlm_destroy", "sdlm_status_str",
             "sdlm_kv_pages", "sdlm_block_attn", "sdlm_lmhead_confidence", "sdlm_lmhead_confidence_static", "sdlm_accept_commit",
             "sdlm_device_status", "sdlm_decode_step", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count",
-            "sdlm_block_attn_masked", "sdlm_verify_commit", "sdlm_accept_commit_carry"]
+            "sdlm_block_attn_masked", "sdlm_verify_commit", "sdlm_accept_commit_carry",
+            "sdlm_linear", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu"]
 
 
 class SdlmError(RuntimeError):
@@ -113,6 +114,14 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdlm_block_attn_masked.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_accept_commit_carry.restype = C.c_int
     lib.sdlm_accept_commit_carry.argtypes = [vp, i32, i32, i32, vp, vp, f32, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_linear.restype = C.c_int
+    lib.sdlm_linear.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_rmsnorm.restype = C.c_int
+    lib.sdlm_rmsnorm.argtypes = [vp, i32, i32, vp, vp, f32, vp, vp]
+    lib.sdlm_rope_block.restype = C.c_int
+    lib.sdlm_rope_block.argtypes = [vp, i32, i32, vp, i32, vp, f32, vp]
+    lib.sdlm_swiglu.restype = C.c_int
+    lib.sdlm_swiglu.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.sdlm_verify_commit.restype = C.c_int
     lib.sdlm_verify_commit.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_accept_commit.restype = C.c_int
@@ -356,6 +365,46 @@ class Sdlm:
             _ptr(_dev(accepted_len, torch.int32, "accepted_len")), _ptr(_dev(out_tokens, torch.int32, "out_tokens")),
             _stream_ptr(stream)))
         return accepted_len, out_tokens
+
+    def linear(self, x: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor] = None,
+               residual: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """sdlm_linear: out = x w^T (+ bias) (+ residual); x [rows, K], w [N, K]."""
+        _dev(x, torch.bfloat16, "x"); _dev(w, torch.bfloat16, "w")
+        K, N = int(w.shape[1]), int(w.shape[0])
+        rows = x.numel() // K
+        if out is None:
+            out = torch.empty((rows, N), dtype=torch.bfloat16, device=self.device)
+        self._check("sdlm_linear", self.lib.sdlm_linear(self.ctx, rows, K, N, _ptr(x), _ptr(w), _ptr(bias), _ptr(residual),
+                                                        _ptr(_dev(out, torch.bfloat16, "out")), _stream_ptr(stream)))
+        return out
+
+    def rmsnorm(self, x: torch.Tensor, weight: torch.Tensor, eps: float, out: Optional[torch.Tensor] = None,
+                stream=None) -> torch.Tensor:
+        _dev(x, torch.bfloat16, "x"); _dev(weight, torch.bfloat16, "weight")
+        H = int(weight.numel())
+        if out is None:
+            out = torch.empty_like(x)
+        self._check("sdlm_rmsnorm", self.lib.sdlm_rmsnorm(self.ctx, x.numel() // H, H, _ptr(x), _ptr(weight), float(eps),
+                                                          _ptr(_dev(out, torch.bfloat16, "out")), _stream_ptr(stream)))
+        return out
+
+    def rope_block(self, x: torch.Tensor, theta: float, seq_ids: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """sdlm_rope_block, in place: x [batch, D, n_heads, head_dim]."""
+        _dev(x, torch.bfloat16, "x")
+        batch, D, n_heads = int(x.shape[0]), int(x.shape[1]), int(x.shape[2])
+        self._check("sdlm_rope_block", self.lib.sdlm_rope_block(self.ctx, batch, D, _ptr(seq_ids), n_heads, _ptr(x),
+                                                                float(theta), _stream_ptr(stream)))
+        return x
+
+    def swiglu(self, gate_up: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        _dev(gate_up, torch.bfloat16, "gate_up")
+        I = int(gate_up.shape[-1]) // 2
+        rows = gate_up.numel() // (2 * I)
+        if out is None:
+            out = torch.empty((rows, I), dtype=torch.bfloat16, device=self.device)
+        self._check("sdlm_swiglu", self.lib.sdlm_swiglu(self.ctx, rows, I, _ptr(gate_up),
+                                                        _ptr(_dev(out, torch.bfloat16, "out")), _stream_ptr(stream)))
+        return out
 
     def lmhead_confidence_static(self, hidden: torch.Tensor, w_lm: torch.Tensor, token: torch.Tensor,
                                  p_top1: torch.Tensor, entropy: torch.Tensor, max_logit: Optional[torch.Tensor] = None,

@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsdlm.so")
-SOURCES = ["sdlm_api.cu", "sdlm_attn.cu", "sdlm_lmhead.cu"]
+SOURCES = ["sdlm_api.cu", "sdlm_attn.cu", "sdlm_lmhead.cu", "sdlm_layer.cu"]
 HEADERS = ["sdlm_internal.h", "sdlm_ptx.cuh", os.path.join("..", "..", "include", "sdlm.h")]
 
 

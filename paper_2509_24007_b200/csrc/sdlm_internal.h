@@ -142,6 +142,8 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
 sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
                           float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st,
                           bool independent_of_predecessor = false, int cta_cap = 0);
+sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, const void* w, const void* bias,
+                          const void* residual, void* out, cudaStream_t st);
 cudaError_t setup_attn(sdlm_ctx* ctx);
 cudaError_t setup_lmhead(sdlm_ctx* ctx);
 

@@ -1,0 +1,151 @@
+// The pieces of a decoder layer around the block attention (Sec. 4.1: the models are built on the
+// Qwen-2.5 backbone: RMSNorm, rotary position embedding in the rotate-half convention, grouped-query
+// attention, SwiGLU MLP).  The matrix products run on the LM-head stripe kernel's second epilogue
+// (sdlm_lmhead.cu); here are the memory-bound row-wise operations and the entry points.
+#include "sdlm_internal.h"
+#include "sdlm_ptx.cuh"
+
+#include <math.h>
+
+namespace sdlm {
+
+// out[r, :] = x[r, :] / sqrt(mean(x[r, :]^2) + eps) * weight[:]; one warp per row, fp32 arithmetic.
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const __nv_bfloat16* x, const __nv_bfloat16* weight,
+                                                      __nv_bfloat16* out, int rows, int H, float eps) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * H);
+  float ss = 0.f;
+  for (int c = lane; c < H / 8; c += 32) {
+    const uint4 v = xr[c];
+    const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float f = __bfloat162float(e[i]);
+      ss = fmaf(f, f, ss);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const float inv = rsqrtf(ss / (float)H + eps);
+  const uint4* wr = reinterpret_cast<const uint4*>(weight);
+  uint4* orow = reinterpret_cast<uint4*>(out + (size_t)row * H);
+  for (int c = lane; c < H / 8; c += 32) {
+    const uint4 v = xr[c], w = wr[c];
+    const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
+    const __nv_bfloat16* g = reinterpret_cast<const __nv_bfloat16*>(&w);
+    uint4 o;
+    uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      ow[i] = ptx::pack_bf16(__bfloat162float(e[2 * i]) * inv * __bfloat162float(g[2 * i]),
+                             __bfloat162float(e[2 * i + 1]) * inv * __bfloat162float(g[2 * i + 1]));
+    orow[c] = o;
+  }
+}
+
+// Rotary embedding of the block's rows, in place: position of row (b, j) is seq_len[slot_b] + j, the
+// first position after the cached history.  Rotate-half convention: element i < d/2 pairs with i + d/2,
+//   x'[i] = x[i] cos(a_i) - x[i+d/2] sin(a_i),  x'[i+d/2] = x[i+d/2] cos(a_i) + x[i] sin(a_i),
+//   a_i = pos * theta^(-2i/d).   One thread per (row, head, i).
+__global__ void __launch_bounds__(256) rope_block_kernel(__nv_bfloat16* x, const int32_t* seq_len, const int32_t* seq_ids,
+                                                         int batch, int D, int n_heads, int d, float log2_theta) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
+  const int half = d / 2;
+  const size_t total = (size_t)batch * D * n_heads * half;
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
+    const int i = (int)(idx % half);
+    size_t r = idx / half;
+    const int h = (int)(r % n_heads); r /= n_heads;
+    const int j = (int)(r % D), b = (int)(r / D);
+    const int slot = seq_ids ? seq_ids[b] : b;
+    const float pos = (float)(seq_len[slot] + j);
+    const float inv_freq = exp2f(-log2_theta * (float)(2 * i) / (float)d);
+    float sn, cs;
+    sincosf(pos * inv_freq, &sn, &cs);
+    __nv_bfloat16* p = x + (((size_t)b * D + j) * n_heads + h) * d;
+    const float a = __bfloat162float(p[i]), c = __bfloat162float(p[i + half]);
+    p[i] = __float2bfloat16_rn(a * cs - c * sn);
+    p[i + half] = __float2bfloat16_rn(c * cs + a * sn);
+  }
+}
+
+// out[r, i] = silu(gate_up[r, i]) * gate_up[r, I + i], silu(g) = g / (1 + exp(-g)); eight elements per thread.
+__global__ void __launch_bounds__(256) swiglu_kernel(const __nv_bfloat16* gate_up, __nv_bfloat16* out, int rows, int I) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
+  const size_t total = (size_t)rows * (I / 8);
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
+    const int c = (int)(idx % (I / 8));
+    const size_t r = idx / (I / 8);
+    const uint4 g = *(reinterpret_cast<const uint4*>(gate_up + r * 2 * I) + c);
+    const uint4 u = *(reinterpret_cast<const uint4*>(gate_up + r * 2 * I + I) + c);
+    const __nv_bfloat16* ge = reinterpret_cast<const __nv_bfloat16*>(&g);
+    const __nv_bfloat16* ue = reinterpret_cast<const __nv_bfloat16*>(&u);
+    uint4 o;
+    uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float g0 = __bfloat162float(ge[2 * i]), g1 = __bfloat162float(ge[2 * i + 1]);
+      ow[i] = ptx::pack_bf16(g0 / (1.f + __expf(-g0)) * __bfloat162float(ue[2 * i]),
+                             g1 / (1.f + __expf(-g1)) * __bfloat162float(ue[2 * i + 1]));
+    }
+    *(reinterpret_cast<uint4*>(out + r * I) + c) = o;
+  }
+}
+
+static inline bool a16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace sdlm
+
+using namespace sdlm;
+
+extern "C" sdlm_status sdlm_linear(sdlm_ctx* ctx, int32_t rows, int32_t K, int32_t N, const void* x, const void* w,
+                                   const void* bias, const void* residual, void* out, void* stream) {
+  if (!ctx || !x || !w || !out || rows < 1 || K < 8 || N < 16) return SDLM_ERR_INVALID_ARG;
+  if (!a16(x) || !a16(w) || !a16(out) || (bias && !a16(bias)) || (residual && !a16(residual))) return SDLM_ERR_INVALID_ARG;
+  if (K % 8 || N % 16) return SDLM_ERR_UNSUPPORTED;
+  return launch_linear(ctx, rows, K, N, x, w, bias, residual, out, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" sdlm_status sdlm_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t H, const void* x, const void* weight, float eps,
+                                    void* out, void* stream) {
+  if (!ctx || !x || !weight || !out || rows < 1 || H < 8 || !(eps >= 0.f)) return SDLM_ERR_INVALID_ARG;
+  if (!a16(x) || !a16(weight) || !a16(out)) return SDLM_ERR_INVALID_ARG;
+  if (H % 8) return SDLM_ERR_UNSUPPORTED;
+  const cudaError_t e = launch_overlapped(rmsnorm_kernel, dim3((rows + 7) / 8), dim3(256), 0, static_cast<cudaStream_t>(stream),
+                                          static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(weight),
+                                          static_cast<__nv_bfloat16*>(out), (int)rows, (int)H, eps);
+  ctx->launches++;
+  return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+}
+
+extern "C" sdlm_status sdlm_rope_block(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, int32_t n_heads,
+                                       void* x, float theta, void* stream) {
+  if (!ctx || !x || batch < 1 || D < 1 || n_heads < 1 || !(theta > 1.f)) return SDLM_ERR_INVALID_ARG;
+  if (batch > ctx->cfg.max_batch) return SDLM_ERR_SHAPE;
+  const int d = ctx->cfg.head_dim;
+  const size_t total = (size_t)batch * D * n_heads * (d / 2);
+  const int blocks = (int)((total + 255) / 256 < 1184 ? (total + 255) / 256 : 1184);
+  const cudaError_t e = launch_overlapped(rope_block_kernel, dim3(blocks), dim3(256), 0, static_cast<cudaStream_t>(stream),
+                                          static_cast<__nv_bfloat16*>(x), (const int32_t*)ctx->seq_len, seq_ids, (int)batch,
+                                          (int)D, (int)n_heads, d, log2f(theta));
+  ctx->launches++;
+  return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+}
+
+extern "C" sdlm_status sdlm_swiglu(sdlm_ctx* ctx, int32_t rows, int32_t I, const void* gate_up, void* out, void* stream) {
+  if (!ctx || !gate_up || !out || rows < 1 || I < 8) return SDLM_ERR_INVALID_ARG;
+  if (!a16(gate_up) || !a16(out)) return SDLM_ERR_INVALID_ARG;
+  if (I % 8) return SDLM_ERR_UNSUPPORTED;
+  const size_t total = (size_t)rows * (I / 8);
+  const int blocks = (int)((total + 255) / 256 < 1184 ? (total + 255) / 256 : 1184);
+  const cudaError_t e = launch_overlapped(swiglu_kernel, dim3(blocks), dim3(256), 0, static_cast<cudaStream_t>(stream),
+                                          static_cast<const __nv_bfloat16*>(gate_up), static_cast<__nv_bfloat16*>(out),
+                                          (int)rows, (int)I);
+  ctx->launches++;
+  return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+}

@@ -55,6 +55,10 @@ struct LmParams {
   int bn;  // umma path: vocab rows per tile (multiple of 16, <= 256)
   int a_box_rows;   // umma path: hidden-state rows one TMA box brings in (<= 128; rows beyond it are never read back)
   int wait_at_end;  // 1: no input comes from the kernel before this one; only completion order is kept
+  // linear mode (the kernel's second epilogue): out[row, n] = bf16(z[row, n] (+ residual[row, n])), row pitch V
+  __nv_bfloat16* out;
+  const __nv_bfloat16* residual;
+  const __nv_bfloat16* bias;  // [V] or null
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -155,7 +159,36 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
 
 // R = number of 128-row blocks of hidden states (1 or 2).  R == 1 double-buffers the accumulator
 // (2 x 256 TMEM columns); R == 2 uses one accumulator per row block.
-template <int R>
+__device__ __forceinline__ void add16(float (&z)[16], const __nv_bfloat16* src) {
+  const uint4 r0 = *reinterpret_cast<const uint4*>(src), r1 = *(reinterpret_cast<const uint4*>(src) + 1);
+  const __nv_bfloat16* rb0 = reinterpret_cast<const __nv_bfloat16*>(&r0);
+  const __nv_bfloat16* rb1 = reinterpret_cast<const __nv_bfloat16*>(&r1);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    z[i] += __bfloat162float(rb0[i]);
+    z[8 + i] += __bfloat162float(rb1[i]);
+  }
+}
+// Sixteen outputs of one row: fp32 accumulator, plus bias, plus residual (in that order), rounded to bf16 once.
+__device__ __forceinline__ void store16(const uint32_t (&v)[16], __nv_bfloat16* out, const __nv_bfloat16* residual,
+                                        const __nv_bfloat16* bias) {
+  float z[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) z[i] = __uint_as_float(v[i]);
+  if (bias) add16(z, bias);
+  if (residual) add16(z, residual);
+  uint4 o0, o1;
+  o0.x = ptx::pack_bf16(z[0], z[1]); o0.y = ptx::pack_bf16(z[2], z[3]);
+  o0.z = ptx::pack_bf16(z[4], z[5]); o0.w = ptx::pack_bf16(z[6], z[7]);
+  o1.x = ptx::pack_bf16(z[8], z[9]); o1.y = ptx::pack_bf16(z[10], z[11]);
+  o1.z = ptx::pack_bf16(z[12], z[13]); o1.w = ptx::pack_bf16(z[14], z[15]);
+  *reinterpret_cast<uint4*>(out) = o0;
+  *(reinterpret_cast<uint4*>(out) + 1) = o1;
+}
+
+// LINEAR = false: the statistics epilogue of the LM head.  LINEAR = true: the same pipeline as a plain
+// skinny matrix product out = x W^T (rows <= 128 per row block), its epilogue storing bf16 outputs.
+template <int R, bool LINEAR = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
     lmhead_umma_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_w,
                        const LmParams p, int n_stages) {
@@ -301,11 +334,26 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
         for (int c = 0; c < n_chunks; c += 2) {
           ptx::tmem_ld_wait();
           if (c + 1 < n_chunks) tmem_ld16(taddr + (c + 1) * 16, v1);
-          if (n0 + c * 16 < n_end) fold16(v0, n0 + c * 16, n_end, st[r]);
+          const int row = r * 128 + q * 32 + lane;
+          if constexpr (LINEAR) {
+            if (n0 + c * 16 < n_end && row < p.rows)
+              store16(v0, p.out + (size_t)row * p.V + n0 + c * 16,
+                      p.residual ? p.residual + (size_t)row * p.V + n0 + c * 16 : nullptr,
+                      p.bias ? p.bias + n0 + c * 16 : nullptr);
+          } else {
+            if (n0 + c * 16 < n_end) fold16(v0, n0 + c * 16, n_end, st[r]);
+          }
           if (c + 1 < n_chunks) {
             ptx::tmem_ld_wait();
             if (c + 2 < n_chunks) tmem_ld16(taddr + (c + 2) * 16, v0);
-            if (n0 + (c + 1) * 16 < n_end) fold16(v1, n0 + (c + 1) * 16, n_end, st[r]);
+            if constexpr (LINEAR) {
+              if (n0 + (c + 1) * 16 < n_end && row < p.rows)
+                store16(v1, p.out + (size_t)row * p.V + n0 + (c + 1) * 16,
+                        p.residual ? p.residual + (size_t)row * p.V + n0 + (c + 1) * 16 : nullptr,
+                        p.bias ? p.bias + n0 + (c + 1) * 16 : nullptr);
+            } else {
+              if (n0 + (c + 1) * 16 < n_end) fold16(v1, n0 + (c + 1) * 16, n_end, st[r]);
+            }
           }
         }
       }
@@ -313,14 +361,16 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&acc_empty[as]);
     }
-    // started without waiting: the merge kernel of an earlier call may still be reading the partials
-    if (p.wait_at_end) ptx::grid_dep_wait();
+    if constexpr (!LINEAR) {
+      // started without waiting: the merge kernel of an earlier call may still be reading the partials
+      if (p.wait_at_end) ptx::grid_dep_wait();
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-      const int row = r * 128 + q * 32 + lane;
-      if (row < p.rows)
-        p.partials[(size_t)blockIdx.x * p.rows_pad + row] =
-            make_float4(st[r].m, st[r].S, st[r].T, __int_as_float(st[r].idx));
+      for (int r = 0; r < R; ++r) {
+        const int row = r * 128 + q * 32 + lane;
+        if (row < p.rows)
+          p.partials[(size_t)blockIdx.x * p.rows_pad + row] =
+              make_float4(st[r].m, st[r].S, st[r].T, __int_as_float(st[r].idx));
+      }
     }
   }
   ptx::tc_fence_before();
@@ -741,6 +791,8 @@ cudaError_t setup_lmhead(sdlm_ctx* ctx) {
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(lmhead_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmemBudget + 2048);
   if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(lmhead_umma_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmemBudget + 2048);
+  if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(lmhead_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               kMmaStages * kMmaStageBytes + 128);
 }
@@ -837,6 +889,41 @@ static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden,
                          p.n_stripes, p.rows_pad, rows, token, p_top1, entropy, max_logit, lse);
   ctx->launches++;
   return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+}
+
+// out[rows, N] = x[rows, K] W[N, K]^T (+ residual), bf16 in and out, fp32 accumulation; row blocks of 128.
+sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, const void* w, const void* bias,
+                          const void* residual, void* out, cudaStream_t st) {
+  for (int r0 = 0; r0 < rows; r0 += 128) {
+    const int nr = rows - r0 < 128 ? rows - r0 : 128;
+    LmParams p{};
+    p.hidden = static_cast<const __nv_bfloat16*>(x) + (size_t)r0 * K;
+    p.w = static_cast<const __nv_bfloat16*>(w);
+    p.hdr = ctx->hdr;
+    p.rows = nr; p.H = K; p.V = N; p.rows_pad = 0; p.partials = nullptr;
+    p.out = static_cast<__nv_bfloat16*>(out) + (size_t)r0 * N;
+    p.residual = residual ? static_cast<const __nv_bfloat16*>(residual) + (size_t)r0 * N : nullptr;
+    p.bias = static_cast<const __nv_bfloat16*>(bias);
+    p.wait_at_end = 0;
+    const int groups = N / 16;
+    int n_cta = groups < ctx->sm_count ? groups : ctx->sm_count;
+    const int gmax = (groups + n_cta - 1) / n_cta;
+    const int tiles = (gmax * 16 + 255) / 256;
+    p.bn = 16 * ((gmax + tiles - 1) / tiles);
+    p.n_stripes = n_cta;
+    p.a_box_rows = (nr + 7) / 8 * 8 < 128 ? (nr + 7) / 8 * 8 : 128;
+    const int stage_bytes = kATileBytes + p.bn * kBK * 2;
+    int n_stages = kUmmaSmemBudget / stage_bytes;
+    if (n_stages > 8) n_stages = 8;
+    CUtensorMap tm_x, tm_w;
+    if (!make_tmap(&tm_x, p.hidden, nr, K, p.a_box_rows) || !make_tmap(&tm_w, w, N, K, p.bn)) return SDLM_ERR_CUDA;
+    const size_t smem = (size_t)n_stages * stage_bytes + 1024 + 512;
+    const cudaError_t le = launch_overlapped(lmhead_umma_kernel<1, true>, dim3(n_cta), dim3(kUmmaThreads), smem, st, tm_x,
+                                             tm_w, p, n_stages);
+    ctx->launches++;
+    if (le != cudaSuccess || cudaGetLastError() != cudaSuccess) return SDLM_ERR_CUDA;
+  }
+  return SDLM_OK;
 }
 
 sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
