@@ -70,3 +70,36 @@ def to_bits(x: np.ndarray) -> np.ndarray:
     f = np.asarray(x, dtype=np.float32)
     u = f.view(np.uint32).astype(np.uint64)
     return (((u + 0x7FFF + ((u >> 16) & 1)) >> 16) & 0xFFFF).astype(np.uint16)
+
+
+def decoder_stack_hidden(h0: np.ndarray, layers, caches, seq_ids, n_q_heads: int, n_kv_heads: int, head_dim: int,
+                         eps: float, theta: float):
+    """The residual stream of one whole-model block step, [B, D, H] -> [B*D, H], through pre-norm decoder
+    layers: h += Wo attn(rope(Wq x + bq), rope(Wk x + bk), Wv x + bv | that layer's cache), x = rms_norm(h);
+    h += Wdown swiglu(Wgu rms_norm(h)).  `layers` is a list of dicts of float64 arrays (ln1, wq, bq, wk,
+    bk, wv, bv, wo, ln2, wgu, wdown); `caches` one PagedKVCache per layer.  Every operation's result is
+    rounded to bf16, as each is a tensor of that type between two library calls.  Returns the final
+    stream (float64 of bf16 values) and the per-layer K / V rows of the block as bf16 bits
+    [B, D, Hkv, d] (what a commit appends).  The composition has no published worked example to pin it
+    to: "parity unpinned" as a whole; every part is pinned on its own."""
+    from .sdlm_oracle import block_attention
+    B, D, H = h0.shape
+    rows = B * D
+    h = round_bf16(h0.reshape(rows, H))
+    k_rows, v_rows = [], []
+    for w, cache in zip(layers, caches):
+        x = round_bf16(rms_norm(h, w["ln1"], eps))
+        q = round_bf16(linear(x, w["wq"], w["bq"])).reshape(B, D, n_q_heads, head_dim)
+        k = round_bf16(linear(x, w["wk"], w["bk"])).reshape(B, D, n_kv_heads, head_dim)
+        v = round_bf16(linear(x, w["wv"], w["bv"])).reshape(B, D, n_kv_heads, head_dim)
+        pos = np.array([int(cache.seq_len[int(s)]) for s in seq_ids])[:, None] + np.arange(D)[None, :]
+        q, k = round_bf16(rope(q, pos, theta)), round_bf16(rope(k, pos, theta))
+        pk, pv = zip(*[cache.gather_fast(int(s)) for s in seq_ids])
+        attn = round_bf16(block_attention(to_bits(q), to_bits(k), to_bits(v), pk, pv))
+        h = round_bf16(linear(attn.reshape(rows, n_q_heads * head_dim), w["wo"], None, h))
+        x = round_bf16(rms_norm(h, w["ln2"], eps))
+        act = round_bf16(swiglu(round_bf16(linear(x, w["wgu"]))))
+        h = round_bf16(linear(act, w["wdown"], None, h))
+        k_rows.append(to_bits(k))
+        v_rows.append(to_bits(v))
+    return h, k_rows, v_rows

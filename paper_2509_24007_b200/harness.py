@@ -150,3 +150,95 @@ class DeviceProblem:
         sd.accept_commit(tau, out.token, out.p_top1, out.entropy, x.k_blk, x.v_blk, mode, out.accepted_len,
                          out.out_tokens, stream=stream)
         return out
+
+
+# ---- a stack of decoder layers around the path (Qwen-2.5 shape) -------------------------------------
+@dataclass
+class LayerWeights:
+    ln1: torch.Tensor    # [H]
+    wq: torch.Tensor     # [Hq*d, H]
+    bq: torch.Tensor     # [Hq*d]
+    wk: torch.Tensor     # [Hkv*d, H]
+    bk: torch.Tensor
+    wv: torch.Tensor
+    bv: torch.Tensor
+    wo: torch.Tensor     # [H, Hq*d]
+    ln2: torch.Tensor    # [H]
+    wgu: torch.Tensor    # [2I, H]: gate rows, then up rows
+    wdown: torch.Tensor  # [H, I]
+
+
+class DecoderStack:
+    """n_layers pre-norm decoder layers (RMSNorm, biased q/k/v projections, rotary positions, block
+    attention over that layer's own paged cache, output projection, SwiGLU MLP), a final RMSNorm and the
+    LM head with acceptance: one whole-model NSP decode step, every operation a library call.  Every
+    layer has its own context (KV pool and tables); all tables move in lockstep because every layer
+    commits the same accepted lengths."""
+
+    EPS = 1e-6
+    THETA = 1.0e6
+
+    def __init__(self, wl: syn.Workload, n_layers: int, intermediate: int, lengths: np.ndarray, layers, ln_f, w_lm,
+                 prefix_fn):
+        """layers: list of LayerWeights; prefix_fn(layer, b, length) -> (k, v) device tensors [length, Hkv, d]."""
+        s = wl.shape
+        self.wl, self.L, self.I = wl, n_layers, intermediate
+        self.lengths = np.asarray(lengths, dtype=np.int32)
+        self.num_pages, self.mpps = syn.pages_needed(wl, self.lengths)
+        self.free_list = syn.free_list_permutation(wl, self.num_pages)
+        cfg = SdlmConfig(s.n_q_heads, s.n_kv_heads, s.head_dim, s.hidden, s.vocab, self.num_pages, wl.batch, self.mpps,
+                         max_block=wl.block, page_size=s.page_size)
+        self.ctx = [Sdlm(cfg) for _ in range(n_layers)]
+        self.layers, self.ln_f, self.w_lm = layers, ln_f, w_lm
+        for l, sd in enumerate(self.ctx):
+            sd.kv_reset(self.free_list)
+            for b in range(wl.batch):
+                if self.lengths[b] > 0:
+                    k, v = prefix_fn(l, b, int(self.lengths[b]))
+                    sd.kv_add_seq(b, k, v)
+        dev = self.ctx[0].device
+        B, D, rows = wl.batch, wl.block, wl.batch * wl.block
+        e = lambda *shape: torch.empty(shape, dtype=torch.bfloat16, device=dev)
+        self.h, self.x = e(rows, s.hidden), e(rows, s.hidden)
+        self.q, self.attn = e(B, D, s.n_q_heads, s.head_dim), e(B, D, s.n_q_heads, s.head_dim)
+        self.k = [e(B, D, s.n_kv_heads, s.head_dim) for _ in range(n_layers)]
+        self.v = [e(B, D, s.n_kv_heads, s.head_dim) for _ in range(n_layers)]
+        self.gu, self.act = e(rows, 2 * intermediate), e(rows, intermediate)
+        self.saved = [sd.kv_save() for sd in self.ctx]
+        torch.cuda.synchronize()
+
+    def restore(self, stream=None) -> None:
+        for sd, sv in zip(self.ctx, self.saved):
+            sd.kv_restore(sv, stream=stream)
+
+    def step(self, h0: torch.Tensor, tau: float, out: StepOutputs, stream=None) -> None:
+        """h0 [B, D, H]: the block's input embeddings.  out.attn is not used (attention is per layer)."""
+        wl, s = self.wl, self.wl.shape
+        self.h.copy_(h0.reshape(self.h.shape))
+        for l, (sd, w) in enumerate(zip(self.ctx, self.layers)):
+            sd.rmsnorm(self.h, w.ln1, self.EPS, self.x, stream=stream)
+            sd.linear(self.x, w.wq, w.bq, None, self.q, stream=stream)
+            sd.linear(self.x, w.wk, w.bk, None, self.k[l], stream=stream)
+            sd.linear(self.x, w.wv, w.bv, None, self.v[l], stream=stream)
+            sd.rope_block(self.q, self.THETA, stream=stream)
+            sd.rope_block(self.k[l], self.THETA, stream=stream)
+            sd.block_attn(self.q, self.k[l], self.v[l], self.attn, stream=stream)
+            sd.linear(self.attn, w.wo, None, self.h, self.h, stream=stream)
+            sd.rmsnorm(self.h, w.ln2, self.EPS, self.x, stream=stream)
+            sd.linear(self.x, w.wgu, None, None, self.gu, stream=stream)
+            sd.swiglu(self.gu, self.act, stream=stream)
+            sd.linear(self.act, w.wdown, None, self.h, self.h, stream=stream)
+        sd0 = self.ctx[0]
+        sd0.rmsnorm(self.h, self.ln_f, self.EPS, self.x, stream=stream)
+        sd0.lmhead_confidence(self.x, self.w_lm, out.token, out.p_top1, out.entropy, stream=stream)
+        for l, sd in enumerate(self.ctx):
+            sd.accept_commit(tau, out.token, out.p_top1, out.entropy, self.k[l], self.v[l], 0, out.accepted_len,
+                             out.out_tokens, stream=stream)
+
+    def launches(self) -> int:
+        return sum(sd.launch_count() for sd in self.ctx)
+
+    def weight_bytes(self) -> int:
+        per = sum(t.numel() * 2 for t in (self.layers[0].wq, self.layers[0].wk, self.layers[0].wv, self.layers[0].wo,
+                                          self.layers[0].wgu, self.layers[0].wdown))
+        return per * self.L + self.w_lm.numel() * 2

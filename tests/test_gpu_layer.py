@@ -117,3 +117,79 @@ def test_layer_pieces_reject_bad_arguments():
     with pytest.raises(pk.SdlmError):
         dp.sd.linear(torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda"),
                      torch.zeros((8, 64), dtype=torch.bfloat16, device="cuda"))   # N < 16
+
+
+def test_two_layer_stack_step_matches_the_oracle_composition():
+    """A tiny whole-model step: the residual stream after two layers, then LM head and acceptance on the
+    GPU's own final hidden state (so that the integer results are compared without accumulated drift),
+    and every layer's cache grown by the same accepted rows."""
+    from paper_2509_24007_b200.harness import DecoderStack, LayerWeights
+    from oracle import sdlm_oracle as orc
+    from oracle_side import oracle_cache, check_tokens, check_confidences, check_gamma
+    shape = syn.SHAPE_TINY                                   # Hq 4, Hkv 2, d 64, H 256, V 1024
+    B, D, L, I = 3, 4, 2, 512
+    lens = np.array([0, 70, 200], dtype=np.int32)
+    wl = syn.Workload("stack", shape, B, D, 0, 0, (0.9,), steps=4, seed=4242)
+    rng = np.random.default_rng(1)
+    H, Hq, Hkv, d = shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+    host_layers, dev_layers = [], []
+    for l in range(L):
+        spec = {"ln1": ((H,), 1.0, 1.0), "wq": ((Hq * d, H), 0.0, H ** -0.5), "bq": ((Hq * d,), 0.0, 0.1),
+                "wk": ((Hkv * d, H), 0.0, H ** -0.5), "bk": ((Hkv * d,), 0.0, 0.1), "wv": ((Hkv * d, H), 0.0, H ** -0.5),
+                "bv": ((Hkv * d,), 0.0, 0.1), "wo": ((H, Hq * d), 0.0, (Hq * d) ** -0.5), "ln2": ((H,), 1.0, 0.1),
+                "wgu": ((2 * I, H), 0.0, H ** -0.5), "wdown": ((H, I), 0.0, I ** -0.5)}
+        hw, dw = {}, {}
+        for name, (shp, mean, std) in spec.items():
+            bits = syn.f32_to_bf16_bits((mean + std * rng.normal(size=shp)).astype(np.float32))
+            hw[name] = syn.bf16_bits_to_f32(bits).astype(np.float64)
+            dw[name] = pk.bf16_tensor_from_bits(bits)
+        host_layers.append(hw)
+        dev_layers.append(LayerWeights(**dw))
+    lnf_bits = syn.f32_to_bf16_bits((1.0 + 0.1 * rng.normal(size=H)).astype(np.float32))
+    w_bits = syn.lm_head_weight(wl)
+    prefixes = [[syn.prefix_kv(wl.with_(seed=wl.seed + 17 * l), b, int(lens[b])) for b in range(B)] for l in range(L)]
+    stack = DecoderStack(wl, L, I, lens, dev_layers, pk.bf16_tensor_from_bits(lnf_bits), pk.bf16_tensor_from_bits(w_bits),
+                         lambda l, b, n: tuple(pk.bf16_tensor_from_bits(t) for t in prefixes[l][b]))
+    caches = [oracle_cache(wl, lens, stack.num_pages, stack.mpps, prefixes[l]) for l in range(L)]
+    out = StepOutputs_like(stack)
+    for step in range(2):
+        h0_bits = syn.f32_to_bf16_bits(rng.normal(size=(B, D, H)).astype(np.float32))
+        stack.step(pk.bf16_tensor_from_bits(h0_bits), wl.tau, out)
+        torch.cuda.synchronize()
+        assert all(sd.device_status()[0] == 0 for sd in stack.ctx)
+        h_ref, k_ref, v_ref = lo.decoder_stack_hidden(syn.bf16_bits_to_f32(h0_bits).astype(np.float64), host_layers, caches,
+                                                     range(B), Hq, Hkv, d, stack.EPS, stack.THETA)
+        h_gpu = _f64(stack.h)
+        scale = np.max(np.abs(h_ref))
+        assert np.max(np.abs(h_gpu - h_ref)) <= 0.03 * scale, (np.max(np.abs(h_gpu - h_ref)), scale)
+        for l in range(L):                                   # the rows each layer is about to commit
+            for got, ref in ((stack.k[l], k_ref[l]), (stack.v[l], v_ref[l])):
+                r64 = syn.bf16_bits_to_f32(ref).astype(np.float64)
+                assert np.max(np.abs(_f64(got) - r64)) <= 0.03 * np.max(np.abs(r64))
+        # head and acceptance: from the GPU's own final normalised hidden state
+        x_bits = pk.bits_from_bf16_tensor(stack.x).reshape(B, D, H)
+        stats = orc.lm_head_statistics(x_bits, w_bits)
+        flagged = []
+        check_tokens(out.token.cpu().numpy(), stats, flagged)
+        check_confidences(out.p_top1.cpu().numpy(), out.entropy.cpu().numpy(), stats)
+        conf = stats.p_top1.reshape(B, D)
+        for l in range(L):
+            kb, vb = pk.bits_from_bf16_tensor(stack.k[l]), pk.bits_from_bf16_tensor(stack.v[l])
+            res = orc.accept_and_commit(caches[l], range(B), stats.token.reshape(B, D), conf, wl.tau, kb, vb)
+            t = stack.ctx[l].kv_tables()
+            assert np.array_equal(t["page_table"], caches[l].page_table) and np.array_equal(t["seq_len"], caches[l].seq_len)
+            for b in range(B):
+                k, v = stack.ctx[l].kv_gather(b, int(caches[l].seq_len[b]))
+                ok, ov = caches[l].gather_fast(b)
+                assert np.array_equal(pk.bits_from_bf16_tensor(k), ok) and np.array_equal(pk.bits_from_bf16_tensor(v), ov)
+        assert check_gamma(out.accepted_len.cpu().numpy(), res, flagged) == 0
+
+
+def StepOutputs_like(stack):
+    from paper_2509_24007_b200.harness import StepOutputs
+    wl, s, dev = stack.wl, stack.wl.shape, stack.ctx[0].device
+    B, D = wl.batch, wl.block
+    return StepOutputs(torch.empty((B, D, s.n_q_heads, s.head_dim), dtype=torch.bfloat16, device=dev),
+                       torch.empty((B, D), dtype=torch.int32, device=dev), torch.empty((B, D), dtype=torch.float32, device=dev),
+                       torch.empty((B, D), dtype=torch.float32, device=dev), torch.empty(B, dtype=torch.int32, device=dev),
+                       torch.empty((B, D), dtype=torch.int32, device=dev))
