@@ -377,6 +377,62 @@ def time_carry(torch, pk, DeviceProblem, wl, steps, warmup, n_blocks=4):
             "what": "block preceded by gamma_prev - 1 carry rows of real tokens; only real-token K/V are cached"}
 
 
+def time_model_level(torch, pk, wl, lengths, n_layers, intermediate, steps, warmup=2):
+    """Whole-model NSP decode steps: n_layers decoder layers of the Qwen-2.5 shape (random weights made
+    on the device) around the block attention, final norm, LM head, acceptance and one commit per layer.
+    One CUDA graph holds a table restore of every layer and one step; it is replayed `steps` times."""
+    from paper_2509_24007_b200.harness import DecoderStack, LayerWeights, StepOutputs
+    s = wl.shape
+    dev = torch.device("cuda", torch.cuda.current_device())
+    g = torch.Generator(device=dev)
+    g.manual_seed(wl.seed)
+    H, Hq, Hkv, d, I = s.hidden, s.n_q_heads, s.n_kv_heads, s.head_dim, intermediate
+    rnd = lambda shape, std, mean=0.0: (mean + std * torch.randn(shape, generator=g, device=dev, dtype=torch.float32)).to(torch.bfloat16)
+    layers = [LayerWeights(rnd((H,), 0.05, 1.0), rnd((Hq * d, H), H ** -0.5), rnd((Hq * d,), 0.05), rnd((Hkv * d, H), H ** -0.5),
+                           rnd((Hkv * d,), 0.05), rnd((Hkv * d, H), H ** -0.5), rnd((Hkv * d,), 0.05),
+                           rnd((H, Hq * d), (Hq * d) ** -0.5), rnd((H,), 0.05, 1.0), rnd((2 * I, H), H ** -0.5),
+                           rnd((H, I), I ** -0.5)) for _ in range(n_layers)]
+    w_lm = pk.bf16_tensor_from_bits(syn.lm_head_weight(wl))
+    stack = DecoderStack(wl, n_layers, I, lengths, layers, rnd((H,), 0.05, 1.0), w_lm,
+                         lambda l, b, n: (rnd((n, Hkv, d), 1.0), rnd((n, Hkv, d), 1.0)))
+    B, D = wl.batch, wl.block
+    out = StepOutputs(torch.empty((B, D, Hq, d), dtype=torch.bfloat16, device=dev), torch.empty((B, D), dtype=torch.int32, device=dev),
+                      torch.empty((B, D), dtype=torch.float32, device=dev), torch.empty((B, D), dtype=torch.float32, device=dev),
+                      torch.empty(B, dtype=torch.int32, device=dev), torch.empty((B, D), dtype=torch.int32, device=dev))
+    h0 = rnd((B, D, H), 1.0)
+    for _ in range(warmup):
+        stack.restore()
+        stack.step(h0, wl.tau, out)
+    torch.cuda.synchronize()
+    n0 = stack.launches()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            stack.restore(stream=side)
+            stack.step(h0, wl.tau, out, stream=side)
+    per_step = stack.launches() - n0
+    torch.cuda.current_stream().wait_stream(side)
+    graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    assert all(int(sd.device_status()[0]) == 0 for sd in stack.ctx), "device status set during the model-level steps"
+    tokens = int(out.accepted_len.clamp(min=0).sum().item())
+    kv = syn.kv_read_bytes(wl, lengths) * n_layers
+    return {"value": tokens / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "tokens_per_step": tokens,
+            "layers": n_layers, "intermediate": I, "library_launches_per_step": per_step,
+            "weight_bytes": stack.weight_bytes(), "kv_bytes": kv,
+            "achieved_gbs": (stack.weight_bytes() + kv) / (ms * 1e-3) / 1e9,
+            "what": "whole-model step (random weights of the 3B shape), every operation a library call, one CUDA graph per step"}
+
+
 def time_e2e(torch, dp, wl, steps, warmup, n_blocks=4):
     """Same metric through sdlm_decode_step_host: pinned host inputs copied in, results copied out, every step."""
     s = wl.shape
@@ -528,6 +584,10 @@ def main():
             torch.cuda.empty_cache()
         if args.workload == "cfg2_d4":
             line["extra"]["carry_over_" + wl.name] = time_carry(torch, pk, DeviceProblem, wl_run, max(8, min(args.steps, 200)), 3)
+            torch.cuda.empty_cache()
+        if args.workload == "cfg2_d4":      # Qwen2.5-3B: 36 layers, intermediate size 11008
+            line["extra"]["model_level_3b_" + wl.name] = time_model_level(torch, pk, wl_run, lengths, 36, 11008,
+                                                                          max(4, min(args.steps, 30)))
             torch.cuda.empty_cache()
         n_seqs = min(wl.batch, 32)
         tok, dt = oracle_sample(wl, n_seqs, repeats=2)
