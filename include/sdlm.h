@@ -295,6 +295,9 @@ sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const
  *                w [N, K], out / residual [rows, N] (out may be residual: in-place accumulation into the
  *                residual stream).  K % 8 == 0, N % 16 == 0 (else UNSUPPORTED).  Runs on the LM head's
  *                tcgen05 / TMA stripe kernel, W streamed once per 128 rows.
+ * sdlm_linear3:  one product whose N1 + N2 + N3 output columns go to three dense tensors out1 [rows, N1],
+ *                out2 [rows, N2], out3 [rows, N3] (the q / k / v projections of a layer from the stacked
+ *                weight [N1 + N2 + N3, K] and bias); N1, N2, N3 multiples of 16; no residual.
  * sdlm_rmsnorm:  out[r, :] = x[r, :] / sqrt(mean_k x[r, k]^2 + eps) * weight[:]; H % 8 == 0.
  * sdlm_rope_block: rotary embedding, in place, of x [batch, D, n_heads, head_dim]: the position of row
  *                (b, j) is (length of slot seq_ids[b], or b, as the tables stand on the stream) + j;
@@ -305,6 +308,8 @@ sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const
  * Errors: INVALID_ARG, SHAPE, UNSUPPORTED, CUDA. */
 sdlm_status sdlm_linear(sdlm_ctx* ctx, int32_t rows, int32_t K, int32_t N, const void* x, const void* w,
                         const void* bias, const void* residual, void* out, void* stream);
+sdlm_status sdlm_linear3(sdlm_ctx* ctx, int32_t rows, int32_t K, int32_t N1, int32_t N2, int32_t N3, const void* x,
+                         const void* w, const void* bias, void* out1, void* out2, void* out3, void* stream);
 sdlm_status sdlm_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t H, const void* x, const void* weight, float eps,
                          void* out, void* stream);
 sdlm_status sdlm_rope_block(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, int32_t n_heads, void* x,

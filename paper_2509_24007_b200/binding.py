@@ -32,7 +32,7 @@ EXPORTED = ["sdlm_pool_bytes", "sdlm_workspace_bytes", "sdlm_create", "sdlm_dest
             "sdlm_kv_pages", "sdlm_block_attn", "sdlm_lmhead_confidence", "sdlm_lmhead_confidence_static", "sdlm_accept_commit",
             "sdlm_device_status", "sdlm_decode_step", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count",
             "sdlm_block_attn_masked", "sdlm_verify_commit", "sdlm_accept_commit_carry",
-            "sdlm_linear", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu"]
+            "sdlm_linear", "sdlm_linear3", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu"]
 
 
 class SdlmError(RuntimeError):
@@ -116,6 +116,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdlm_accept_commit_carry.argtypes = [vp, i32, i32, i32, vp, vp, f32, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_linear.restype = C.c_int
     lib.sdlm_linear.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_linear3.restype = C.c_int
+    lib.sdlm_linear3.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_rmsnorm.restype = C.c_int
     lib.sdlm_rmsnorm.argtypes = [vp, i32, i32, vp, vp, f32, vp, vp]
     lib.sdlm_rope_block.restype = C.c_int
@@ -377,6 +379,20 @@ class Sdlm:
         self._check("sdlm_linear", self.lib.sdlm_linear(self.ctx, rows, K, N, _ptr(x), _ptr(w), _ptr(bias), _ptr(residual),
                                                         _ptr(_dev(out, torch.bfloat16, "out")), _stream_ptr(stream)))
         return out
+
+    def linear3(self, x: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor], out1: torch.Tensor,
+                out2: torch.Tensor, out3: torch.Tensor, stream=None) -> None:
+        """sdlm_linear3: x w^T (+ bias) with the output columns dealt to three dense tensors."""
+        _dev(x, torch.bfloat16, "x"); _dev(w, torch.bfloat16, "w")
+        K = int(w.shape[1])
+        rows = x.numel() // K
+        n = [t.numel() // rows for t in (out1, out2, out3)]
+        if sum(n) != int(w.shape[0]):
+            raise ValueError("the three outputs must take all of w's rows")
+        self._check("sdlm_linear3", self.lib.sdlm_linear3(self.ctx, rows, K, n[0], n[1], n[2], _ptr(x), _ptr(w), _ptr(bias),
+                                                          _ptr(_dev(out1, torch.bfloat16, "out1")),
+                                                          _ptr(_dev(out2, torch.bfloat16, "out2")),
+                                                          _ptr(_dev(out3, torch.bfloat16, "out3")), _stream_ptr(stream)))
 
     def rmsnorm(self, x: torch.Tensor, weight: torch.Tensor, eps: float, out: Optional[torch.Tensor] = None,
                 stream=None) -> torch.Tensor:

@@ -36,6 +36,7 @@ WorkspaceLayout workspace_layout(const sdlm_config& c) {
   L.free_list = take((size_t)c.num_pages * 4);
   L.table_end = off;
   L.lm_partials = take((size_t)kLmMaxStripes * rows * 16);
+  L.lin_part = take((size_t)kLinSplitMax * 128 * kLinSplitMaxN * 4);
   const int G = c.n_q_heads / c.n_kv_heads;
   L.q_rows_pad = G * c.max_block <= 32 ? 32 : 64;
   L.attn_max_items = kAttnMaxCtas + c.max_batch * c.n_kv_heads;

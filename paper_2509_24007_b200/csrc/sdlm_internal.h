@@ -15,6 +15,8 @@ constexpr int kMaxBlock = 8;         // largest D
 constexpr int kMaxBlockKeys = 16;    // rows of k_blk / v_blk per sequence in the masked variant
 constexpr int kMaxQRows = 64;        // (Hq/Hkv) * D stacked query rows per KV head
 constexpr int kMaxBatch = 4096;
+constexpr int kLinSplitMax = 12;      // most K ranges of a split-K linear
+constexpr int kLinSplitMaxN = 4096;   // widest output a split-K linear takes
 constexpr int kLmMaxStripes = 1024;  // upper bound on vocab stripes (one partial per stripe per row)
 constexpr int kAttnMaxCtas = 160;    // upper bound on the attention grid (one CTA per SM)
 
@@ -32,6 +34,7 @@ static_assert(sizeof(DevHeader) == 64, "header is 64 bytes");
 
 struct WorkspaceLayout {
   size_t hdr, page_table, seq_len, free_list, table_end;  // [hdr, table_end) is the exportable state
+  size_t lin_part;                                         // float [kLinSplitMax][128][kLinSplitMaxN]
   size_t lm_partials;                                      // float4 [kLmMaxStripes][max_rows]
   size_t attn_ml, attn_o;                                  // split-KV partial (m, l) and O
   size_t attn_cnt;                                         // per (batch row, KV head) arrival counters
@@ -143,7 +146,8 @@ sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const voi
                           float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st,
                           bool independent_of_predecessor = false, int cta_cap = 0);
 sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, const void* w, const void* bias,
-                          const void* residual, void* out, cudaStream_t st);
+                          const void* residual, void* out, cudaStream_t st, int seg1 = 0, int seg2 = 0,
+                          void* out2 = nullptr, void* out3 = nullptr);
 cudaError_t setup_attn(sdlm_ctx* ctx);
 cudaError_t setup_lmhead(sdlm_ctx* ctx);
 

@@ -111,6 +111,17 @@ extern "C" sdlm_status sdlm_linear(sdlm_ctx* ctx, int32_t rows, int32_t K, int32
   return launch_linear(ctx, rows, K, N, x, w, bias, residual, out, static_cast<cudaStream_t>(stream));
 }
 
+extern "C" sdlm_status sdlm_linear3(sdlm_ctx* ctx, int32_t rows, int32_t K, int32_t N1, int32_t N2, int32_t N3,
+                                    const void* x, const void* w, const void* bias, void* out1, void* out2, void* out3,
+                                    void* stream) {
+  if (!ctx || !x || !w || !out1 || !out2 || !out3 || rows < 1 || K < 8 || N1 < 16 || N2 < 16 || N3 < 16)
+    return SDLM_ERR_INVALID_ARG;
+  if (!a16(x) || !a16(w) || !a16(out1) || !a16(out2) || !a16(out3) || (bias && !a16(bias))) return SDLM_ERR_INVALID_ARG;
+  if (K % 8 || N1 % 16 || N2 % 16 || N3 % 16) return SDLM_ERR_UNSUPPORTED;
+  return launch_linear(ctx, rows, K, N1 + N2 + N3, x, w, bias, nullptr, out1, static_cast<cudaStream_t>(stream), N1,
+                       N1 + N2, out2, out3);
+}
+
 extern "C" sdlm_status sdlm_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t H, const void* x, const void* weight, float eps,
                                     void* out, void* stream) {
   if (!ctx || !x || !weight || !out || rows < 1 || H < 8 || !(eps >= 0.f)) return SDLM_ERR_INVALID_ARG;

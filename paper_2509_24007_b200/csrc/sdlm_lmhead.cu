@@ -60,7 +60,24 @@ struct LmParams {
   __nv_bfloat16* out;
   const __nv_bfloat16* residual;
   const __nv_bfloat16* bias;  // [V] or null
+  // split-K (linear mode, ksplit > 1): thread block (stripe ct, split ks) = blockIdx.x = ks * n_stripes + ct
+  // covers K steps [ks * kc_per, (ks + 1) * kc_per) and leaves fp32 partials part[ks][row][n]; a second
+  // kernel adds them up in split order
+  int ksplit, kc_per;
+  float* part;
+  // three outputs from one product (seg1 > 0): columns [0, seg1) go to out (row pitch seg1), [seg1, seg2)
+  // to out2, [seg2, V) to out3, each a dense tensor of its own; no residual, no split-K then
+  int seg1, seg2;
+  __nv_bfloat16* out2;
+  __nv_bfloat16* out3;
 };
+
+__device__ __forceinline__ __nv_bfloat16* linear_dst(const LmParams& p, int row, int n) {
+  if (p.seg1 == 0) return p.out + (size_t)row * p.V + n;
+  if (n < p.seg1) return p.out + (size_t)row * p.seg1 + n;
+  if (n < p.seg2) return p.out2 + (size_t)row * (p.seg2 - p.seg1) + (n - p.seg1);
+  return p.out3 + (size_t)row * (p.V - p.seg2) + (n - p.seg2);
+}
 
 // ---------------------------------------------------------------------------------------------
 // tcgen05 / TMA stripe kernel
@@ -187,6 +204,12 @@ __device__ __forceinline__ void store16(const uint32_t (&v)[16], __nv_bfloat16* 
   *(reinterpret_cast<uint4*>(out) + 1) = o1;
 }
 
+__device__ __forceinline__ void store16_f32(const uint32_t (&v)[16], float* dst) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    reinterpret_cast<uint4*>(dst)[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+}
+
 // LINEAR = false: the statistics epilogue of the LM head.  LINEAR = true: the same pipeline as a plain
 // skinny matrix product out = x W^T (rows <= 128 per row block), its epilogue storing bf16 outputs.
 template <int R, bool LINEAR = false>
@@ -211,11 +234,15 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
 
   // this CTA's vocabulary stripe, in groups of 16 rows
   const int groups = (p.V + 15) / 16;
-  const int g0 = (int)((long long)blockIdx.x * groups / gridDim.x);
-  const int g1 = (int)((long long)(blockIdx.x + 1) * groups / gridDim.x);
+  const int n_ct = LINEAR ? p.n_stripes : (int)gridDim.x;
+  const int ct = LINEAR ? (int)blockIdx.x % n_ct : (int)blockIdx.x, ks = LINEAR ? (int)blockIdx.x / n_ct : 0;
+  const int g0 = (int)((long long)ct * groups / n_ct);
+  const int g1 = (int)((long long)(ct + 1) * groups / n_ct);
   const int n_begin = g0 * 16, n_end = min(p.V, g1 * 16);
   const int n_tiles = (n_end - n_begin + p.bn - 1) / p.bn;
-  const int KC = (p.H + kBK - 1) / kBK;
+  const int KC_all = (p.H + kBK - 1) / kBK;
+  const int kc0 = LINEAR && p.ksplit > 1 ? ks * p.kc_per : 0;                       // this block's K steps
+  const int KC = LINEAR && p.ksplit > 1 ? max(0, min(KC_all, kc0 + p.kc_per) - kc0) : KC_all;
 
   if (tid == 0) {
     for (int s = 0; s < n_stages; ++s) {
@@ -258,8 +285,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
           uint8_t* st = smem + (size_t)s * stage_bytes;
           ptx::mbar_arrive_expect_tx(&full[s], (uint32_t)(R * p.a_box_rows * kBK * 2 + w_tile_bytes));
 #pragma unroll
-          for (int r = 0; r < R; ++r) ptx::tma_load_2d(st + r * kATileBytes, &tmap_h, kc * kBK, r * 128, &full[s]);
-          ptx::tma_load_2d_hint(st + R * kATileBytes, &tmap_w, kc * kBK, n0, &full[s], w_policy);
+          for (int r = 0; r < R; ++r) ptx::tma_load_2d(st + r * kATileBytes, &tmap_h, (kc0 + kc) * kBK, r * 128, &full[s]);
+          ptx::tma_load_2d_hint(st + R * kATileBytes, &tmap_w, (kc0 + kc) * kBK, n0, &full[s], w_policy);
         }
       }
       if (!ok || *abort) {  // winding down: let the copies already issued land before the CTA goes away
@@ -337,8 +364,10 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
           if (c + 1 < n_chunks) tmem_ld16(taddr + (c + 1) * 16, v1);
           const int row = r * 128 + q * 32 + lane;
           if constexpr (LINEAR) {
-            if (n0 + c * 16 < n_end && row < p.rows)
-              store16(v0, p.out + (size_t)row * p.V + n0 + c * 16,
+            if (p.ksplit > 1) {
+              if (n0 + c * 16 < n_end && row < p.rows) store16_f32(v0, p.part + ((size_t)ks * 128 + row) * p.V + n0 + c * 16);
+            } else if (n0 + c * 16 < n_end && row < p.rows)
+              store16(v0, linear_dst(p, row, n0 + c * 16),
                       p.residual ? p.residual + (size_t)row * p.V + n0 + c * 16 : nullptr,
                       p.bias ? p.bias + n0 + c * 16 : nullptr);
           } else {
@@ -348,8 +377,11 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
             ptx::tmem_ld_wait();
             if (c + 2 < n_chunks) tmem_ld16(taddr + (c + 2) * 16, v0);
             if constexpr (LINEAR) {
-              if (n0 + (c + 1) * 16 < n_end && row < p.rows)
-                store16(v1, p.out + (size_t)row * p.V + n0 + (c + 1) * 16,
+              if (p.ksplit > 1) {
+                if (n0 + (c + 1) * 16 < n_end && row < p.rows)
+                  store16_f32(v1, p.part + ((size_t)ks * 128 + row) * p.V + n0 + (c + 1) * 16);
+              } else if (n0 + (c + 1) * 16 < n_end && row < p.rows)
+                store16(v1, linear_dst(p, row, n0 + (c + 1) * 16),
                         p.residual ? p.residual + (size_t)row * p.V + n0 + (c + 1) * 16 : nullptr,
                         p.bias ? p.bias + n0 + (c + 1) * 16 : nullptr);
             } else {
@@ -711,6 +743,44 @@ __global__ void __launch_bounds__(kMmaThreads) lmhead_mma_kernel(const LmParams 
 }
 
 // ---------------------------------------------------------------------------------------------
+// split-K linear: out = bf16(sum_s part[s] + bias + residual), splits added in index order
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) linear_reduce_kernel(const float* part, int ksplit, int rows, int N,
+                                                            const __nv_bfloat16* bias, const __nv_bfloat16* residual,
+                                                            __nv_bfloat16* out) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
+  const size_t total = (size_t)rows * (N / 8);
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
+    const int c = (int)(idx % (N / 8));
+    const size_t row = idx / (N / 8);
+    float z[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int s = 0; s < ksplit; ++s) {
+      const float4* src = reinterpret_cast<const float4*>(part + ((size_t)s * 128 + row) * N) + 2 * c;
+      const float4 a = __ldcg(src), b = __ldcg(src + 1);
+      z[0] += a.x; z[1] += a.y; z[2] += a.z; z[3] += a.w;
+      z[4] += b.x; z[5] += b.y; z[6] += b.z; z[7] += b.w;
+    }
+    if (bias) {
+      const uint4 v = *(reinterpret_cast<const uint4*>(bias) + c);
+      const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) z[i] += __bfloat162float(e[i]);
+    }
+    if (residual) {
+      const uint4 v = *(reinterpret_cast<const uint4*>(residual + row * N) + c);
+      const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) z[i] += __bfloat162float(e[i]);
+    }
+    uint4 o;
+    o.x = ptx::pack_bf16(z[0], z[1]); o.y = ptx::pack_bf16(z[2], z[3]);
+    o.z = ptx::pack_bf16(z[4], z[5]); o.w = ptx::pack_bf16(z[6], z[7]);
+    *(reinterpret_cast<uint4*>(out + row * N) + c) = o;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // merge of the per-stripe partials: one warp per row, fixed order
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(128) lmhead_combine_kernel(const float4* partials, int n_stripes, int rows_pad, int rows,
@@ -894,7 +964,7 @@ static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden,
 
 // out[rows, N] = x[rows, K] W[N, K]^T (+ residual), bf16 in and out, fp32 accumulation; row blocks of 128.
 sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, const void* w, const void* bias,
-                          const void* residual, void* out, cudaStream_t st) {
+                          const void* residual, void* out, cudaStream_t st, int seg1, int seg2, void* out2, void* out3) {
   for (int r0 = 0; r0 < rows; r0 += 128) {
     const int nr = rows - r0 < 128 ? rows - r0 : 128;
     LmParams p{};
@@ -906,6 +976,12 @@ sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, 
     p.residual = residual ? static_cast<const __nv_bfloat16*>(residual) + (size_t)r0 * N : nullptr;
     p.bias = static_cast<const __nv_bfloat16*>(bias);
     p.wait_at_end = 0;
+    p.seg1 = seg1; p.seg2 = seg2;
+    if (seg1 > 0) {
+      p.out = static_cast<__nv_bfloat16*>(out) + (size_t)r0 * seg1;
+      p.out2 = static_cast<__nv_bfloat16*>(out2) + (size_t)r0 * (seg2 - seg1);
+      p.out3 = static_cast<__nv_bfloat16*>(out3) + (size_t)r0 * (N - seg2);
+    }
     const int groups = N / 16;
     // How many thread blocks: every one re-reads the x rows (from L2) for each of its output tiles, so
     // with few output columns per block that traffic, not the weight stream, sets the time.  Pick the
@@ -926,6 +1002,23 @@ sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, 
       }
       n_cta = best_n;
     }
+    // Narrow products (few output columns, long K) cannot keep enough weight bytes in flight with one
+    // thread block per column stripe: cut K as well.  Stripes of 128 columns, as many K ranges as SMs allow.
+    const int KC_all = (K + kBK - 1) / kBK;
+    p.ksplit = 1;
+    p.kc_per = KC_all;
+    p.part = reinterpret_cast<float*>(ctx->ws + ctx->lay.lin_part);
+    if (N <= kLinSplitMaxN && KC_all >= 64 && seg1 == 0) {  // (with 32 K steps the second launch costs more than it saves)
+      const int n_ct = (N + 127) / 128;
+      int ks = ctx->sm_count / n_ct;
+      if (ks > kLinSplitMax) ks = kLinSplitMax;
+      if (ks > KC_all / 4) ks = KC_all / 4;
+      if (ks >= 2) {
+        p.kc_per = (KC_all + ks - 1) / ks;
+        p.ksplit = (KC_all + p.kc_per - 1) / p.kc_per;  // every range non-empty
+        n_cta = n_ct;
+      }
+    }
     const int gmax = (groups + n_cta - 1) / n_cta;
     const int tiles = (gmax * 16 + 255) / 256;
     p.bn = 16 * ((gmax + tiles - 1) / tiles);
@@ -937,10 +1030,18 @@ sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, 
     CUtensorMap tm_x, tm_w;
     if (!make_tmap(&tm_x, p.hidden, nr, K, p.a_box_rows) || !make_tmap(&tm_w, w, N, K, p.bn)) return SDLM_ERR_CUDA;
     const size_t smem = (size_t)n_stages * stage_bytes + 1024 + 512;
-    const cudaError_t le = launch_overlapped(lmhead_umma_kernel<1, true>, dim3(n_cta), dim3(kUmmaThreads), smem, st, tm_x,
-                                             tm_w, p, n_stages);
+    cudaError_t le = launch_overlapped(lmhead_umma_kernel<1, true>, dim3(n_cta * p.ksplit), dim3(kUmmaThreads), smem, st,
+                                       tm_x, tm_w, p, n_stages);
     ctx->launches++;
     if (le != cudaSuccess || cudaGetLastError() != cudaSuccess) return SDLM_ERR_CUDA;
+    if (p.ksplit > 1) {
+      const size_t total = (size_t)nr * (N / 8);
+      const int blocks = (int)((total + 255) / 256);
+      le = launch_overlapped(linear_reduce_kernel, dim3(blocks), dim3(256), 0, st, (const float*)p.part, p.ksplit, nr, N,
+                             p.bias, p.residual, p.out);
+      ctx->launches++;
+      if (le != cudaSuccess || cudaGetLastError() != cudaSuccess) return SDLM_ERR_CUDA;
+    }
   }
   return SDLM_OK;
 }

@@ -190,6 +190,9 @@ class DecoderStack:
                          max_block=wl.block, page_size=s.page_size)
         self.ctx = [Sdlm(cfg) for _ in range(n_layers)]
         self.layers, self.ln_f, self.w_lm = layers, ln_f, w_lm
+        # q, k and v come from one product over the stacked weight
+        self.wqkv = [torch.cat([w.wq, w.wk, w.wv], dim=0).contiguous() for w in layers]
+        self.bqkv = [torch.cat([w.bq, w.bk, w.bv], dim=0).contiguous() for w in layers]
         for l, sd in enumerate(self.ctx):
             sd.kv_reset(self.free_list)
             for b in range(wl.batch):
@@ -217,9 +220,7 @@ class DecoderStack:
         self.h.copy_(h0.reshape(self.h.shape))
         for l, (sd, w) in enumerate(zip(self.ctx, self.layers)):
             sd.rmsnorm(self.h, w.ln1, self.EPS, self.x, stream=stream)
-            sd.linear(self.x, w.wq, w.bq, None, self.q, stream=stream)
-            sd.linear(self.x, w.wk, w.bk, None, self.k[l], stream=stream)
-            sd.linear(self.x, w.wv, w.bv, None, self.v[l], stream=stream)
+            sd.linear3(self.x, self.wqkv[l], self.bqkv[l], self.q, self.k[l], self.v[l], stream=stream)
             sd.rope_block(self.q, self.THETA, stream=stream)
             sd.rope_block(self.k[l], self.THETA, stream=stream)
             sd.block_attn(self.q, self.k[l], self.v[l], self.attn, stream=stream)

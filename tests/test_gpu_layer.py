@@ -52,6 +52,25 @@ def test_linear_matches_the_oracle(rows, K, N, extras):
     _check_bf16(_f64(out), ref, "linear")
 
 
+@pytest.mark.parametrize("rows,K,n", [(128, 2048, (2048, 256, 256)), (37, 256, (64, 16, 32)), (200, 512, (256, 128, 128))])
+def test_linear_with_three_outputs_matches_three_products(rows, K, n):
+    """The q / k / v projections from one product over the stacked weight."""
+    dp = _ctx()
+    rng = np.random.default_rng(rows + K)
+    _, x64, x = _bf16(rng, (rows, K))
+    _, w64, w = _bf16(rng, (sum(n), K), std=K ** -0.5)
+    _, b64, b = _bf16(rng, (sum(n),))
+    outs = [torch.full((rows, m), 7.0, dtype=torch.bfloat16, device="cuda") for m in n]
+    dp.sd.linear3(x, w, b, *outs)
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+    ref = lo.linear(x64, w64, b64)
+    c = 0
+    for o, m in zip(outs, n):
+        _check_bf16(_f64(o), ref[:, c:c + m], "linear3")
+        c += m
+
+
 def test_linear_in_place_on_the_residual_stream():
     dp = _ctx()
     rng = np.random.default_rng(9)
