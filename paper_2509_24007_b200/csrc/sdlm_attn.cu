@@ -176,7 +176,9 @@ __device__ __forceinline__ int tile_valid(const Item& it, int ti, int D) {
   return ti == it.pages - 1 ? it.len - ti * kPageSize : kPageSize;
 }
 
-template <int HD, int NQ>
+// MASKED: the variant behind sdlm_block_attn_masked (visibility words, up to 16 block keys); kept out of
+// the plain kernel, whose instruction footprint matters (see the no-instruction stalls in profiles/).
+template <int HD, int NQ, bool MASKED = false>
 __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(const AttnParams p) {
   constexpr int KH = HD / 64;                 // 64-wide panels of K and of Q
   constexpr int K_PANEL_B = kPageSize * 128;  // one tile's panel: 64 keys x 128 bytes
@@ -501,8 +503,8 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       for (int q = 0; q < QV; ++q) l[q] = 0.f;
       const int n = it.t1 - it.t0, ng = (n + 1) / 2;
       // which of my 32 query rows see my key if it turns out to be a block key (bit q: row qb + q)
-      uint32_t visq = 0xffffffffu;
-      if (p.vis != nullptr && it.t1 > it.pages) {
+      [[maybe_unused]] uint32_t visq = 0xffffffffu;
+      if (MASKED && p.vis != nullptr && it.t1 > it.pages) {
         visq = 0;
         int j = qb / p.G, rem = qb % p.G;
         uint32_t vj = j < p.D ? p.vis[(size_t)it.b * p.D + j] : 0u;
@@ -530,10 +532,12 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&s_free[sb]);
-        if (visq != 0xffffffffu && it.t0 + 2 * g + tj == it.pages) {  // my key is a block key some rows do not see
+        if constexpr (MASKED) {
+          if (visq != 0xffffffffu && it.t0 + 2 * g + tj == it.pages) {  // my key is a block key some rows do not see
 #pragma unroll
-          for (int q = 0; q < QV; ++q)
-            if (!((visq >> q) & 1u)) x[q] = -INFINITY;
+            for (int q = 0; q < QV; ++q)
+              if (!((visq >> q) & 1u)) x[q] = -INFINITY;
+          }
         }
 
         const bool first = g == 0;
@@ -844,7 +848,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
         // beyond them only produce scores that are masked
         for (int idx = lane; idx < VT_B / 16; idx += 32) reinterpret_cast<uint4*>(v_t)[idx] = make_uint4(0, 0, 0, 0);
         __syncwarp();
-        for (int k0 = 0; k0 < p.Dk; k0 += kMaxBlock) {
+        for (int k0 = 0; k0 < (MASKED ? p.Dk : kMaxBlock); k0 += kMaxBlock) {  // one pass unless masked (Dk <= 8 = D)
           if (k0 > 0) load_rows(k0);
 #pragma unroll
           for (int i = 0; i < NB; ++i) {
@@ -886,7 +890,7 @@ static int attn_fixed_smem(int batch) {
          (HD == 64 ? 8192 : 0);
 }
 
-template <int HD, int NQ>
+template <int HD, int NQ, bool MASKED = false>
 static cudaError_t attn_launch_one(sdlm_ctx* ctx, AttnParams& p, cudaStream_t st, int cta_cap, bool whole_tpcs) {
   const int pair_b = 2 * (2 * kPageSize * HD * 2);
   int n = (kAttnSmemLimit - attn_fixed_smem<HD, NQ>(p.batch)) / (pair_b + 16);
@@ -901,8 +905,8 @@ static cudaError_t attn_launch_one(sdlm_ctx* ctx, AttnParams& p, cudaStream_t st
   if (whole_tpcs && n_cta >= 2) n_cta &= ~1;
   const cudaError_t e =
       whole_tpcs && n_cta >= 2
-          ? launch_overlapped_cluster(block_attn_umma_kernel<HD, NQ>, dim3(n_cta), dim3(attn_threads(NQ)), smem, st, 2, p)
-          : launch_overlapped(block_attn_umma_kernel<HD, NQ>, dim3(n_cta), dim3(attn_threads(NQ)), smem, st, p);
+          ? launch_overlapped_cluster(block_attn_umma_kernel<HD, NQ, MASKED>, dim3(n_cta), dim3(attn_threads(NQ)), smem, st, 2, p)
+          : launch_overlapped(block_attn_umma_kernel<HD, NQ, MASKED>, dim3(n_cta), dim3(attn_threads(NQ)), smem, st, p);
   ctx->launches++;
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -913,10 +917,18 @@ cudaError_t setup_attn(sdlm_ctx* ctx) {
     e = cudaFuncSetAttribute(block_attn_umma_kernel<128, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(block_attn_umma_kernel<128, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(block_attn_umma_kernel<128, 32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(block_attn_umma_kernel<128, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
   } else {
     e = cudaFuncSetAttribute(block_attn_umma_kernel<64, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(block_attn_umma_kernel<64, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(block_attn_umma_kernel<64, 32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(block_attn_umma_kernel<64, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemLimit);
   }
   return e;
 }
@@ -950,6 +962,13 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
   if ((long long)batch * (c.max_pages_per_seq + 1 + ctx->attn_item_cost) * c.n_kv_heads > 13000000ll)
     return cudaErrorInvalidConfiguration;
   const bool wide = ctx->group * D > 32;  // stacked query rows padded to 64, else to 32
+  if (vis != nullptr) {
+    if (c.head_dim == 128)
+      return wide ? attn_launch_one<128, 64, true>(ctx, p, st, cta_cap, whole_tpcs)
+                  : attn_launch_one<128, 32, true>(ctx, p, st, cta_cap, whole_tpcs);
+    return wide ? attn_launch_one<64, 64, true>(ctx, p, st, cta_cap, whole_tpcs)
+                : attn_launch_one<64, 32, true>(ctx, p, st, cta_cap, whole_tpcs);
+  }
   if (c.head_dim == 128)
     return wide ? attn_launch_one<128, 64>(ctx, p, st, cta_cap, whole_tpcs)
                 : attn_launch_one<128, 32>(ctx, p, st, cta_cap, whole_tpcs);
