@@ -328,8 +328,11 @@ sdlm_status sdlm_swiglu(sdlm_ctx* ctx, int32_t rows, int32_t I, const void* gate
  * charges a thread block for every (sequence, KV head) pair it starts (default 12); results do not
  * depend on it.  SDLM_OPT_ATTN_MIN_RANGE: 1..4096, the fewest schedule positions (pages plus item
  * costs) one thread block is given, which bounds how finely a short workload is split.
+ * SDLM_OPT_HOST_TWO_STREAMS: 1 makes sdlm_decode_step_host, when SDLM_OPT_STEP_OVERLAP is set, copy q / k / v
+ * and run attention on a second stream of the context while `hidden` is copied and the LM head runs on the
+ * caller's stream (default 0: everything on the caller's stream, in order of need).
  * Errors: INVALID_ARG. */
-typedef enum sdlm_option { SDLM_OPT_LMHEAD_KERNEL = 0, SDLM_OPT_STEP_OVERLAP = 1, SDLM_OPT_ATTN_ITEM_COST = 2, SDLM_OPT_ATTN_MIN_RANGE = 3 } sdlm_option;
+typedef enum sdlm_option { SDLM_OPT_LMHEAD_KERNEL = 0, SDLM_OPT_STEP_OVERLAP = 1, SDLM_OPT_ATTN_ITEM_COST = 2, SDLM_OPT_ATTN_MIN_RANGE = 3, SDLM_OPT_HOST_TWO_STREAMS = 4 } sdlm_option;
 sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t value);
 
 /* Number of kernels the library has launched through this context since it was created. */

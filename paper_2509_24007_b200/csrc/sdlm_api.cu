@@ -448,6 +448,9 @@ extern "C" sdlm_status sdlm_create(const sdlm_config* cfg, void* kv_pool, size_t
   ctx->launches = 0;
   ctx->lmhead_path = 0;
   ctx->overlap_lmhead = 0;
+  ctx->host_two_streams = 0;
+  ctx->side_stream = nullptr;
+  ctx->ev_fork = ctx->ev_join = nullptr;
   ctx->attn_item_cost = 12;
   ctx->attn_min_range = 8;
   ctx->tmap_w_ptr = nullptr;
@@ -460,7 +463,15 @@ extern "C" sdlm_status sdlm_create(const sdlm_config* cfg, void* kv_pool, size_t
   return SDLM_OK;
 }
 
-extern "C" void sdlm_destroy(sdlm_ctx* ctx) { delete ctx; }
+extern "C" void sdlm_destroy(sdlm_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->side_stream) {
+    cudaStreamDestroy(ctx->side_stream);
+    cudaEventDestroy(ctx->ev_fork);
+    cudaEventDestroy(ctx->ev_join);
+  }
+  delete ctx;
+}
 
 extern "C" sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t value) {
   if (!ctx) return SDLM_ERR_INVALID_ARG;
@@ -468,6 +479,10 @@ extern "C" sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t v
     case SDLM_OPT_LMHEAD_KERNEL:
       if (value < 0 || value > 3) return SDLM_ERR_INVALID_ARG;
       ctx->lmhead_path = value;
+      return SDLM_OK;
+    case SDLM_OPT_HOST_TWO_STREAMS:
+      if (value < 0 || value > 1) return SDLM_ERR_INVALID_ARG;
+      ctx->host_two_streams = value;
       return SDLM_OK;
     case SDLM_OPT_ATTN_ITEM_COST:
       if (value < 0 || value > 64) return SDLM_ERR_INVALID_ARG;
@@ -752,13 +767,32 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
   const size_t q_bytes = rows * c.n_q_heads * c.head_dim * 2, kv_bytes = rows * c.n_kv_heads * c.head_dim * 2;
   char* ws = ctx->ws;
   bool ok = true;
-  ok &= cudaMemcpyAsync(ws + L.st_q, q_host, q_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(ws + L.st_k, k_blk_host, kv_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(ws + L.st_v, v_blk_host, kv_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(ws + L.st_hidden, hidden_host, rows * c.hidden * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  // Side by side (overlap option A > 0): the LM head only needs `hidden`, attention only q / k / v.  The
+  // hidden rows are copied on the caller's stream and the LM head follows at once; q, k, v (and the
+  // sequence ids) are copied on a second stream of the context and attention follows there, on its A
+  // SMs; the commit waits for both.  Otherwise everything is enqueued on the caller's stream in order.
+  const int a_sms = ctx->host_two_streams ? ctx->overlap_lmhead : 0;
+  cudaStream_t qkv_st = st;
+  if (a_sms > 0) {
+    if (!ctx->side_stream) {
+      if (cudaStreamCreateWithFlags(&ctx->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
+          cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess)
+        return SDLM_ERR_CUDA;
+    }
+    qkv_st = ctx->side_stream;
+    ok &= cudaEventRecord(ctx->ev_fork, st) == cudaSuccess;          // whatever the caller enqueued before comes first
+    ok &= cudaStreamWaitEvent(qkv_st, ctx->ev_fork, 0) == cudaSuccess;
+    ok &= cudaMemcpyAsync(ws + L.st_hidden, hidden_host, rows * c.hidden * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  }
+  ok &= cudaMemcpyAsync(ws + L.st_q, q_host, q_bytes, cudaMemcpyHostToDevice, qkv_st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(ws + L.st_k, k_blk_host, kv_bytes, cudaMemcpyHostToDevice, qkv_st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(ws + L.st_v, v_blk_host, kv_bytes, cudaMemcpyHostToDevice, qkv_st) == cudaSuccess;
+  if (a_sms == 0)
+    ok &= cudaMemcpyAsync(ws + L.st_hidden, hidden_host, rows * c.hidden * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
   const int32_t* seq_ids = nullptr;
   if (seq_ids_host) {
-    ok &= cudaMemcpyAsync(ws + L.st_seq_ids, seq_ids_host, (size_t)batch * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(ws + L.st_seq_ids, seq_ids_host, (size_t)batch * 4, cudaMemcpyHostToDevice, qkv_st) == cudaSuccess;
     seq_ids = reinterpret_cast<const int32_t*>(ws + L.st_seq_ids);
   }
   if (!ok) return SDLM_ERR_CUDA;
@@ -787,9 +821,25 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
   copies.token = static_cast<int32_t*>(mapped(token_host));
   copies.p_top1 = static_cast<float*>(mapped(p_top1_host));
   copies.entropy = static_cast<float*>(mapped(entropy_host));
-  s = decode_step_device(ctx, batch, D, seq_ids, tau, mode, ws + L.st_q, ws + L.st_k, ws + L.st_v, ws + L.st_hidden, w_lm,
-                         m_attn ? m_attn : ws + L.st_out, d_token, d_p, d_ent, m_acc ? m_acc : d_acc,
-                         m_out_tokens ? m_out_tokens : d_out_tokens, copies, stream);
+  void* d_attn = m_attn ? m_attn : ws + L.st_out;
+  int32_t* o_acc = m_acc ? m_acc : d_acc;
+  int32_t* o_tok = m_out_tokens ? m_out_tokens : d_out_tokens;
+  if (a_sms > 0) {
+    if (!aligned16(w_lm)) return SDLM_ERR_INVALID_ARG;
+    if (launch_block_attn(ctx, batch, D, seq_ids, ws + L.st_q, ws + L.st_k, ws + L.st_v, d_attn, qkv_st, a_sms,
+                          batch * D > 128) != cudaSuccess)
+      return SDLM_ERR_CUDA;
+    if (cudaEventRecord(ctx->ev_join, qkv_st) != cudaSuccess) return SDLM_ERR_CUDA;
+    s = launch_lmhead(ctx, batch * D, ws + L.st_hidden, w_lm, d_token, d_p, d_ent, nullptr, nullptr, st,
+                      /*independent_of_predecessor=*/false, ctx->sm_count - a_sms);
+    if (s != SDLM_OK) return s;
+    if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return SDLM_ERR_CUDA;
+    s = accept_commit_launch(ctx, batch, D, seq_ids, tau, mode, d_token, d_p, d_ent, ws + L.st_k, ws + L.st_v, o_acc, o_tok,
+                             copies, stream);
+  } else {
+    s = decode_step_device(ctx, batch, D, seq_ids, tau, mode, ws + L.st_q, ws + L.st_k, ws + L.st_v, ws + L.st_hidden, w_lm,
+                           d_attn, d_token, d_p, d_ent, o_acc, o_tok, copies, stream);
+  }
   if (s != SDLM_OK) return s;
   if (attn_out_host && !m_attn)
     ok &= cudaMemcpyAsync(attn_out_host, ws + L.st_out, q_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;

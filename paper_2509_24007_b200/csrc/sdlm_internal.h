@@ -67,6 +67,10 @@ struct sdlm_ctx {
   int attn_min_range;  // shortest range of schedule positions given to one attention thread block
   int attn_item_cost;  // positions the attention schedule charges for starting a (sequence, KV head) pair
   int overlap_lmhead;  // sdlm_decode_step: SMs given to attention while the LM head runs on the rest (0: one after the other)
+  // second stream and fork / join events of the host-buffer step's side-by-side mode (made on first use)
+  int host_two_streams;
+  cudaStream_t side_stream;
+  cudaEvent_t ev_fork, ev_join;
   // cached TMA descriptor of the LM-head weight (keyed by pointer and tile rows)
   const void* tmap_w_ptr;
   int tmap_w_rows;

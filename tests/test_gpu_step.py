@@ -11,7 +11,7 @@ import torch
 
 import paper_2509_24007_b200 as pk
 from paper_2509_24007_b200.harness import DeviceProblem
-from paper_2509_24007_b200.binding import OPT_STEP_OVERLAP
+from paper_2509_24007_b200.binding import OPT_STEP_OVERLAP, OPT_HOST_TWO_STREAMS
 from oracle import sdlm_oracle as orc
 import sdlm_synth as syn
 from oracle_side import (check_attention, check_confidences, check_gamma, check_tokens, oracle_cache)
@@ -194,6 +194,42 @@ def test_decode_step_host_entry_matches_device_calls(results):
     assert torch.equal(out_tok, ref.out_tokens.cpu()) and torch.equal(ent, ref.entropy.cpu())
     t = dp.sd.kv_tables()
     assert np.array_equal(t["page_table"], t_ref["page_table"]) and np.array_equal(t["seq_len"], t_ref["seq_len"])
+
+
+@pytest.mark.parametrize("name,batch,a_sms", [("cfg0", 3, 40), ("cfg2_d4", 6, 42), ("cfg2", 20, 36)])
+def test_decode_step_host_side_by_side_uses_two_streams_and_gives_the_same_step(name, batch, a_sms):
+    """With the overlap option the host-buffer step copies `hidden` and runs the LM head on the caller's
+    stream while q / k / v are copied and attention runs on the context's second stream."""
+    wl = syn.CONFIGS[name].with_(batch=batch, prefix_lo=10, prefix_hi=700)
+    dp = DeviceProblem(wl)
+    B, D, s = wl.batch, wl.block, wl.shape
+    pin = lambda t: t.cpu().pin_memory()
+    attn = torch.empty((B, D, s.n_q_heads, s.head_dim), dtype=torch.bfloat16).pin_memory()
+    tok = torch.empty((B, D), dtype=torch.int32).pin_memory()
+    p = torch.empty((B, D), dtype=torch.float32)                      # pageable on purpose
+    ent = torch.empty((B, D), dtype=torch.float32).pin_memory()
+    acc = torch.empty(B, dtype=torch.int32).pin_memory()
+    out_tok = torch.empty((B, D), dtype=torch.int32).pin_memory()
+    for step in range(3):
+        x = dp.block(step)
+        snap = dp.sd.kv_export()
+        dp.sd.set_option(OPT_STEP_OVERLAP, 0)
+        ref = dp.step(x, wl.tau)
+        torch.cuda.synchronize()
+        t_ref = dp.sd.kv_tables()
+        dp.sd.kv_import(snap)
+        dp.sd.set_option(OPT_STEP_OVERLAP, a_sms)
+        dp.sd.set_option(OPT_HOST_TWO_STREAMS, step % 2 == 0)
+        dp.sd.decode_step_host(wl.tau, pin(x.q), pin(x.k_blk), pin(x.v_blk), pin(x.hidden), dp.w_lm, attn, tok, p, ent,
+                               acc, out_tok)
+        assert dp.sd.device_status()[0] == 0
+        assert (attn.float() - ref.attn.cpu().float()).abs().max().item() <= 2e-2
+        assert (p - ref.p_top1.cpu()).abs().max().item() <= 1e-3 and (ent - ref.entropy.cpu()).abs().max().item() <= 1e-3
+        assert torch.equal(tok, ref.token.cpu()) and torch.equal(acc, ref.accepted_len.cpu())
+        assert torch.equal(out_tok, ref.out_tokens.cpu())
+        t = dp.sd.kv_tables()
+        assert np.array_equal(t["page_table"], t_ref["page_table"]) and np.array_equal(t["seq_len"], t_ref["seq_len"])
+    dp.sd.set_option(OPT_STEP_OVERLAP, 0)
 
 
 @pytest.mark.parametrize("name,batch", [("cfg0", 3), ("cfg2_d4", 6)])
