@@ -335,6 +335,13 @@ sdlm_status sdlm_swiglu(sdlm_ctx* ctx, int32_t rows, int32_t I, const void* gate
 typedef enum sdlm_option { SDLM_OPT_LMHEAD_KERNEL = 0, SDLM_OPT_STEP_OVERLAP = 1, SDLM_OPT_ATTN_ITEM_COST = 2, SDLM_OPT_ATTN_MIN_RANGE = 3, SDLM_OPT_HOST_TWO_STREAMS = 4 } sdlm_option;
 sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t value);
 
+/* Self-test of the bounded waits (the paper has no counterpart): launches one thread block that waits on
+ * a barrier nothing signals.  Every wait inside the library's kernels is bounded the same way (about
+ * 0.2 s of wall time, then a block-wide abort flag); here the wait runs out on purpose, the kernel
+ * records SDLM_ERR_TIMEOUT in the device status (read and clear it with sdlm_device_status) and
+ * returns, and the context stays usable.  Takes about 0.2 s of GPU time.  Errors: INVALID_ARG, CUDA. */
+sdlm_status sdlm_selftest_bounded_wait(sdlm_ctx* ctx, void* stream);
+
 /* Number of kernels the library has launched through this context since it was created. */
 uint64_t sdlm_launch_count(const sdlm_ctx* ctx);
 

@@ -33,7 +33,7 @@ EXPORTED = ["sdlm_pool_bytes", "sdlm_workspace_bytes", "sdlm_create", "sdlm_dest
             "sdlm_kv_pages", "sdlm_block_attn", "sdlm_lmhead_confidence", "sdlm_lmhead_confidence_static", "sdlm_accept_commit",
             "sdlm_device_status", "sdlm_decode_step", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count",
             "sdlm_block_attn_masked", "sdlm_verify_commit", "sdlm_accept_commit_carry",
-            "sdlm_linear", "sdlm_linear3", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu"]
+            "sdlm_linear", "sdlm_linear3", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu", "sdlm_selftest_bounded_wait"]
 
 
 class SdlmError(RuntimeError):
@@ -117,6 +117,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdlm_accept_commit_carry.argtypes = [vp, i32, i32, i32, vp, vp, f32, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_linear.restype = C.c_int
     lib.sdlm_linear.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_selftest_bounded_wait.restype = C.c_int
+    lib.sdlm_selftest_bounded_wait.argtypes = [vp, vp]
     lib.sdlm_linear3.restype = C.c_int
     lib.sdlm_linear3.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_rmsnorm.restype = C.c_int
@@ -507,6 +509,9 @@ class Sdlm:
             self.ctx, batch, D, _ptr(seq_ids), float(tau), int(mode), _ptr(q), _ptr(k_blk), _ptr(v_blk), _ptr(hidden),
             _ptr(w_lm), _ptr(attn_out), _ptr(token), _ptr(p_top1), _ptr(entropy), _ptr(accepted_len),
             _ptr(out_tokens), _stream_ptr(stream)))
+
+    def selftest_bounded_wait(self, stream=None) -> None:
+        self._check("sdlm_selftest_bounded_wait", self.lib.sdlm_selftest_bounded_wait(self.ctx, _stream_ptr(stream)))
 
     def set_option(self, opt: int, value: int) -> None:
         self._check("sdlm_set_option", self.lib.sdlm_set_option(self.ctx, opt, value))

@@ -702,6 +702,36 @@ extern "C" sdlm_status sdlm_block_attn_masked(sdlm_ctx* ctx, int32_t batch, int3
              : SDLM_ERR_CUDA;
 }
 
+// One thread block waits, with the same bounded wait every kernel of the library uses, on a barrier and
+// on a counter that nothing ever signals; each wait gives up after its limit (about 0.2 s), the kernel
+// records SDLM_ERR_TIMEOUT in the device status and returns.  The context stays usable.
+__global__ void selftest_wait_kernel(DevHeader* hdr) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag, counter;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar, 1);
+    ptx::fence_barrier_init();
+    abort_flag = 0;
+    counter = 0;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const bool a = ptx::mbar_wait(&bar, 0, &abort_flag);       // nothing arrives: runs out, sets the abort flag
+    const bool b = ptx::counter_wait(&counter, 0, &abort_flag);  // sees the flag and returns at once
+    if (!a && !b && atomicCAS(&hdr->status[0], 0, (int)SDLM_ERR_TIMEOUT) == 0) {
+      hdr->status[1] = -3;
+      hdr->status[2] = abort_flag;
+    }
+  }
+}
+
+extern "C" sdlm_status sdlm_selftest_bounded_wait(sdlm_ctx* ctx, void* stream) {
+  if (!ctx) return SDLM_ERR_INVALID_ARG;
+  selftest_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->hdr);
+  ctx->launches++;
+  return cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+}
+
 extern "C" sdlm_status sdlm_device_status(sdlm_ctx* ctx, int32_t* host_out, int32_t clear, void* stream) {
   if (!ctx || !host_out) return SDLM_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -131,3 +131,22 @@ def test_out_of_pages_and_capacity_are_reported_not_fatal():
     assert st[0] in (4, 7) and st[3] == 2
     t = sd.kv_tables()
     assert t["seq_len"].tolist() == [64, 126, 0] and t["free_head"] == 3
+
+
+def test_a_wait_that_nothing_signals_runs_out_and_leaves_the_context_usable():
+    """The bounded wait used by every kernel: the self-test kernel waits on a barrier nothing arrives on,
+    gives up after its limit, reports SDLM_ERR_TIMEOUT through the device status; then a normal step works."""
+    import time
+    wl = syn.CONFIGS["cfg0"]
+    dp = DeviceProblem(wl)
+    t0 = time.perf_counter()
+    dp.sd.selftest_bounded_wait()
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    st = dp.sd.device_status(clear=True)
+    assert st[0] == 6 and st[1] == -3 and st[2] == 1          # SDLM_ERR_TIMEOUT, the self-test's mark, abort flag set
+    assert 0.1 < dt < 2.0                                     # about 0.2 s: bounded, not a hang
+    assert dp.sd.device_status()[0] == 0                      # cleared
+    out = dp.step(dp.block(0), wl.tau)                        # the context still works
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0 and int(out.accepted_len[0]) >= 1
