@@ -250,6 +250,18 @@ sdlm_status sdlm_accept_commit_carry(sdlm_ctx* ctx, int32_t batch, int32_t D, in
                                      const float* p_top1, const float* entropy, const void* k_rows,
                                      const void* v_rows, int32_t* accepted_len, int32_t* out_tokens, void* stream);
 
+/* ---- (c) for several caches at once: the layers of a model each keep their own context (KV pool and
+ * tables), and all commit the same accepted lengths, so their tables move in lockstep.  One launch
+ * does what n_layers calls of sdlm_accept_commit would: ctxs [n_layers] contexts of identical
+ * configuration (HOST array), k_blk / v_blk HOST arrays of n_layers DEVICE pointers
+ * [batch, D, Hkv, d] (layer l's block rows); token / p_top1 / entropy / accepted_len / out_tokens
+ * as sdlm_accept_commit (shared by all layers).  n_layers <= 64.  Errors: as sdlm_accept_commit. */
+sdlm_status sdlm_accept_commit_layers(sdlm_ctx* const* ctxs, int32_t n_layers, int32_t batch, int32_t D,
+                                      const int32_t* seq_ids, float tau, sdlm_conf_mode mode, const int32_t* token,
+                                      const float* p_top1, const float* entropy, const void* const* k_blk,
+                                      const void* const* v_blk, int32_t* accepted_len, int32_t* out_tokens,
+                                      void* stream);
+
 /* Synchronises `stream` and copies the sticky device status words to host_out[4]:
  * {sdlm_status (0 = none), sequence slot of the first failure, detail, number of failures}.
  * `clear` != 0 resets them afterwards. */
@@ -302,7 +314,8 @@ sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const
  * sdlm_rope_block: rotary embedding, in place, of x [batch, D, n_heads, head_dim]: the position of row
  *                (b, j) is (length of slot seq_ids[b], or b, as the tables stand on the stream) + j;
  *                x'[i] = x[i] cos a - x[i + d/2] sin a, x'[i + d/2] = x[i + d/2] cos a + x[i] sin a,
- *                a = position * theta^(-2i/d), i < d/2.
+ *                a = position * theta^(-2i/d), i < d/2.  sdlm_rope_block2 does two tensors (a layer's
+ *                query and key rows, n_heads and n_heads2 heads) in one launch.
  * sdlm_swiglu:   out[r, i] = silu(gate_up[r, i]) * gate_up[r, I + i], silu(g) = g / (1 + e^-g);
  *                gate_up [rows, 2I], out [rows, I]; I % 8 == 0.
  * Errors: INVALID_ARG, SHAPE, UNSUPPORTED, CUDA. */
@@ -314,6 +327,8 @@ sdlm_status sdlm_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t H, const void* x, 
                          void* out, void* stream);
 sdlm_status sdlm_rope_block(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, int32_t n_heads, void* x,
                             float theta, void* stream);
+sdlm_status sdlm_rope_block2(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, int32_t n_heads, void* x,
+                             int32_t n_heads2, void* x2, float theta, void* stream);
 sdlm_status sdlm_swiglu(sdlm_ctx* ctx, int32_t rows, int32_t I, const void* gate_up, void* out, void* stream);
 
 /* Tuning / test knobs (the paper has no counterpart).  SDLM_OPT_LMHEAD_KERNEL: which stripe kernel

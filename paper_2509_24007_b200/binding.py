@@ -33,7 +33,23 @@ EXPORTED = ["sdlm_pool_bytes", "sdlm_workspace_bytes", "sdlm_create", "sdlm_dest
             "sdlm_kv_pages", "sdlm_block_attn", "sdlm_lmhead_confidence", "sdlm_lmhead_confidence_static", "sdlm_accept_commit",
             "sdlm_device_status", "sdlm_decode_step", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count",
             "sdlm_block_attn_masked", "sdlm_verify_commit", "sdlm_accept_commit_carry",
-            "sdlm_linear", "sdlm_linear3", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu", "sdlm_selftest_bounded_wait"]
+            "sdlm_linear", "sdlm_linear3", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu", "sdlm_selftest_bounded_wait", "sdlm_rope_block2", "sdlm_accept_commit_layers"]
+
+
+def accept_commit_layers(contexts, tau: float, token, p_top1, entropy, k_blks, v_blks, accepted_len, out_tokens,
+                         mode: int = 0, seq_ids=None, stream=None) -> None:
+    """sdlm_accept_commit_layers: one launch commits the same accepted rows into every layer's cache."""
+    sd0 = contexts[0]
+    n = len(contexts)
+    batch, D = int(k_blks[0].shape[0]), int(k_blks[0].shape[1])
+    ctx_arr = (C.c_void_p * n)(*[c.ctx.value for c in contexts])
+    k_arr = (C.c_void_p * n)(*[_ptr(_dev(t, torch.bfloat16, "k_blk")) for t in k_blks])
+    v_arr = (C.c_void_p * n)(*[_ptr(_dev(t, torch.bfloat16, "v_blk")) for t in v_blks])
+    sd0._check("sdlm_accept_commit_layers", sd0.lib.sdlm_accept_commit_layers(
+        ctx_arr, n, batch, D, _ptr(seq_ids), float(tau), int(mode), _ptr(_dev(token, torch.int32, "token")),
+        _ptr(_dev(p_top1, torch.float32, "p_top1")), _ptr(_dev(entropy, torch.float32, "entropy")), k_arr, v_arr,
+        _ptr(_dev(accepted_len, torch.int32, "accepted_len")), _ptr(_dev(out_tokens, torch.int32, "out_tokens")),
+        _stream_ptr(stream)))
 
 
 class SdlmError(RuntimeError):
@@ -125,6 +141,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdlm_rmsnorm.argtypes = [vp, i32, i32, vp, vp, f32, vp, vp]
     lib.sdlm_rope_block.restype = C.c_int
     lib.sdlm_rope_block.argtypes = [vp, i32, i32, vp, i32, vp, f32, vp]
+    lib.sdlm_accept_commit_layers.restype = C.c_int
+    lib.sdlm_accept_commit_layers.argtypes = [vp, i32, i32, i32, vp, f32, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_rope_block2.restype = C.c_int
+    lib.sdlm_rope_block2.argtypes = [vp, i32, i32, vp, i32, vp, i32, vp, f32, vp]
     lib.sdlm_swiglu.restype = C.c_int
     lib.sdlm_swiglu.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.sdlm_verify_commit.restype = C.c_int
@@ -414,6 +434,15 @@ class Sdlm:
         self._check("sdlm_rope_block", self.lib.sdlm_rope_block(self.ctx, batch, D, _ptr(seq_ids), n_heads, _ptr(x),
                                                                 float(theta), _stream_ptr(stream)))
         return x
+
+    def rope_block2(self, x: torch.Tensor, x2: torch.Tensor, theta: float, seq_ids: Optional[torch.Tensor] = None,
+                    stream=None) -> None:
+        """sdlm_rope_block2, in place: x [batch, D, n_heads, d] and x2 [batch, D, n_heads2, d] in one launch."""
+        _dev(x, torch.bfloat16, "x"); _dev(x2, torch.bfloat16, "x2")
+        batch, D = int(x.shape[0]), int(x.shape[1])
+        self._check("sdlm_rope_block2", self.lib.sdlm_rope_block2(self.ctx, batch, D, _ptr(seq_ids), int(x.shape[2]), _ptr(x),
+                                                                  int(x2.shape[2]), _ptr(x2), float(theta),
+                                                                  _stream_ptr(stream)))
 
     def swiglu(self, gate_up: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
         _dev(gate_up, torch.bfloat16, "gate_up")

@@ -231,7 +231,7 @@ constexpr int kCommitThreads = 256;
 // snapshot of the tables (so the hand-out order is ascending batch row, as one-at-a-time decoding
 // would give), then scatters its own row's K/V.  The tables other CTAs read (seq_len, free_head)
 // are only written by whichever CTA finishes its reads last ("last CTA done" ticket; nobody waits).
-__global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitParams p) {
+__device__ __forceinline__ void accept_commit_body(const CommitParams& p, bool write_outputs) {
   __shared__ int8_t s_gamma[kMaxBatch];
   __shared__ int8_t s_state[kMaxBatch];  // 0 ok, 1 capacity failure, 2 out of pages
   __shared__ int s_warp[kCommitThreads / 32];
@@ -298,17 +298,17 @@ __global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitPar
   // my row
   const int g = s_mine[0], need = s_mine[1], alloc = s_mine[2], len = s_mine[3], state = s_mine[4], na = s_mine[5];
   const int slot = p.seq_ids ? p.seq_ids[b] : b;
-  for (int k = tid; k < p.D; k += kCommitThreads) {
+  for (int k = tid; write_outputs && k < p.D; k += kCommitThreads) {
     if (p.token_copy) p.token_copy[b * p.D + k] = p.token[b * p.D + k];
     if (p.p_top1_copy) p.p_top1_copy[b * p.D + k] = p.p_top1[b * p.D + k];
     if (p.entropy_copy) p.entropy_copy[b * p.D + k] = p.entropy[b * p.D + k];
   }
   if (state != 0) {
     if (tid == 0) {
-      p.accepted_len[b] = -1;
+      if (write_outputs) p.accepted_len[b] = -1;
       report_status(p.hdr, state == 1 ? SDLM_ERR_DEVICE_CHECK : SDLM_ERR_OUT_OF_PAGES, slot, len);
     }
-    for (int k = tid; k < p.D; k += kCommitThreads) p.out_tokens[b * p.D + k] = -1;
+    for (int k = tid; write_outputs && k < p.D; k += kCommitThreads) p.out_tokens[b * p.D + k] = -1;
   } else {
     const int new_idx = (len + kPageSize - 1) / kPageSize;
     int new_page = -1;
@@ -316,8 +316,9 @@ __global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitPar
       new_page = p.free_list[(s_head + (uint32_t)alloc) % (uint32_t)p.num_pages];
       if (tid == 0) p.page_table[(size_t)slot * p.mpps + new_idx] = new_page;
     }
-    if (tid == 0) p.accepted_len[b] = g;
-    for (int k = tid; k < p.D; k += kCommitThreads) p.out_tokens[b * p.D + k] = (k < g) ? p.token[b * p.D + k] : -1;
+    if (tid == 0 && write_outputs) p.accepted_len[b] = g;
+    for (int k = tid; write_outputs && k < p.D; k += kCommitThreads)
+      p.out_tokens[b * p.D + k] = (k < g) ? p.token[b * p.D + k] : -1;
     if (need) {  // a page fresh from the ring may hold anything: clear its V^T tiles first
       const int per_head = kPageSize * p.d / 8;
       for (int idx = tid; idx < p.Hkv * per_head; idx += kCommitThreads)
@@ -364,6 +365,31 @@ __global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitPar
       p.hdr->commit_ticket = 0;
     }
   }
+}
+
+__global__ void __launch_bounds__(kCommitThreads) accept_commit_kernel(CommitParams p) { accept_commit_body(p, true); }
+
+// The same for several caches whose tables move in lockstep (the layers of a model): thread block
+// (b, l) commits sequence b into cache l from that layer's block rows; the acceptance inputs are shared and
+// layer 0 writes the outputs.
+constexpr int kMaxCommitLayers = 64;
+struct CommitLayer {
+  DevHeader* hdr;
+  int32_t* page_table;
+  int32_t* seq_len;
+  const int32_t* free_list;
+  __nv_bfloat16* pool;
+  const __nv_bfloat16* k_blk;
+  const __nv_bfloat16* v_blk;
+};
+struct CommitLayers {
+  CommitLayer layer[kMaxCommitLayers];
+};
+__global__ void __launch_bounds__(kCommitThreads) accept_commit_layers_kernel(CommitParams p, const __grid_constant__ CommitLayers ls) {
+  const CommitLayer& l = ls.layer[blockIdx.y];
+  p.hdr = l.hdr; p.page_table = l.page_table; p.seq_len = l.seq_len; p.free_list = l.free_list;
+  p.pool = l.pool; p.k_blk = l.k_blk; p.v_blk = l.v_blk;
+  accept_commit_body(p, blockIdx.y == 0);
 }
 
 }  // namespace sdlm
@@ -663,6 +689,47 @@ extern "C" sdlm_status sdlm_accept_commit(sdlm_ctx* ctx, int32_t batch, int32_t 
                                           int32_t* accepted_len, int32_t* out_tokens, void* stream) {
   return accept_commit_launch(ctx, batch, D, seq_ids, tau, mode, token, p_top1, entropy, k_blk, v_blk, accepted_len,
                               out_tokens, StatCopies{}, stream);
+}
+
+extern "C" sdlm_status sdlm_accept_commit_layers(sdlm_ctx* const* ctxs, int32_t n_layers, int32_t batch, int32_t D,
+                                                 const int32_t* seq_ids, float tau, sdlm_conf_mode mode,
+                                                 const int32_t* token, const float* p_top1, const float* entropy,
+                                                 const void* const* k_blk, const void* const* v_blk,
+                                                 int32_t* accepted_len, int32_t* out_tokens, void* stream) {
+  if (!ctxs || n_layers < 1 || !k_blk || !v_blk || !token || !p_top1 || !entropy || !accepted_len || !out_tokens)
+    return SDLM_ERR_INVALID_ARG;
+  if (n_layers > kMaxCommitLayers) return SDLM_ERR_SHAPE;
+  if (mode != SDLM_CONF_LOGIT && mode != SDLM_CONF_ENTROPY) return SDLM_ERR_INVALID_ARG;
+  if (!isfinite(tau)) return SDLM_ERR_INVALID_ARG;
+  sdlm_ctx* c0 = ctxs[0];
+  if (!c0) return SDLM_ERR_INVALID_ARG;
+  sdlm_status s = check_batch(c0, batch, D);
+  if (s != SDLM_OK) return s;
+  CommitLayers* L = new (std::nothrow) CommitLayers;
+  if (!L) return SDLM_ERR_CUDA;
+  for (int l = 0; l < n_layers; ++l) {
+    sdlm_ctx* c = ctxs[l];
+    if (!c || !k_blk[l] || !v_blk[l] || !aligned16(k_blk[l]) || !aligned16(v_blk[l]) ||
+        memcmp(&c->cfg, &c0->cfg, sizeof(sdlm_config)) != 0) {
+      delete L;
+      return SDLM_ERR_INVALID_ARG;
+    }
+    L->layer[l] = CommitLayer{c->hdr, c->page_table, c->seq_len, c->free_list, reinterpret_cast<__nv_bfloat16*>(c->pool),
+                              static_cast<const __nv_bfloat16*>(k_blk[l]), static_cast<const __nv_bfloat16*>(v_blk[l])};
+  }
+  const sdlm_config& c = c0->cfg;
+  CommitParams p{};
+  p.seq_ids = seq_ids; p.token = token; p.p_top1 = p_top1; p.entropy = entropy;
+  p.accepted_len = accepted_len; p.out_tokens = out_tokens;
+  p.tau = tau;
+  p.inv_ln_vocab = c.vocab > 1 ? (float)(1.0 / log((double)c.vocab)) : 0.0f;
+  p.mode = (int)mode; p.batch = batch; p.D = D; p.Hkv = c.n_kv_heads; p.d = c.head_dim;
+  p.mpps = c.max_pages_per_seq; p.num_pages = c.num_pages;
+  const cudaError_t e = launch_overlapped(accept_commit_layers_kernel, dim3(batch, n_layers), dim3(kCommitThreads), 0,
+                                          static_cast<cudaStream_t>(stream), p, *L);
+  delete L;
+  c0->launches++;
+  return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
 }
 
 extern "C" sdlm_status sdlm_verify_commit(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids,

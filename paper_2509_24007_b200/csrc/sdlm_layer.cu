@@ -50,23 +50,27 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const __nv_bfloat16* x, co
 // first position after the cached history.  Rotate-half convention: element i < d/2 pairs with i + d/2,
 //   x'[i] = x[i] cos(a_i) - x[i+d/2] sin(a_i),  x'[i+d/2] = x[i+d/2] cos(a_i) + x[i] sin(a_i),
 //   a_i = pos * theta^(-2i/d).   One thread per (row, head, i).
-__global__ void __launch_bounds__(256) rope_block_kernel(__nv_bfloat16* x, const int32_t* seq_len, const int32_t* seq_ids,
-                                                         int batch, int D, int n_heads, int d, float log2_theta) {
+// Two tensors in one launch (a layer's query and key rows): heads 0..n_heads-1 are x's, the next n_heads2 x2's.
+__global__ void __launch_bounds__(256) rope_block_kernel(__nv_bfloat16* x, __nv_bfloat16* x2, const int32_t* seq_len,
+                                                         const int32_t* seq_ids, int batch, int D, int n_heads,
+                                                         int n_heads2, int d, float log2_theta) {
   ptx::grid_dep_launch();
   ptx::grid_dep_wait();
   const int half = d / 2;
-  const size_t total = (size_t)batch * D * n_heads * half;
+  const int heads = n_heads + n_heads2;
+  const size_t total = (size_t)batch * D * heads * half;
   for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
     const int i = (int)(idx % half);
     size_t r = idx / half;
-    const int h = (int)(r % n_heads); r /= n_heads;
+    const int hh = (int)(r % heads); r /= heads;
     const int j = (int)(r % D), b = (int)(r / D);
     const int slot = seq_ids ? seq_ids[b] : b;
     const float pos = (float)(seq_len[slot] + j);
     const float inv_freq = exp2f(-log2_theta * (float)(2 * i) / (float)d);
     float sn, cs;
     sincosf(pos * inv_freq, &sn, &cs);
-    __nv_bfloat16* p = x + (((size_t)b * D + j) * n_heads + h) * d;
+    __nv_bfloat16* p = hh < n_heads ? x + (((size_t)b * D + j) * n_heads + hh) * d
+                                    : x2 + (((size_t)b * D + j) * n_heads2 + (hh - n_heads)) * d;
     const float a = __bfloat162float(p[i]), c = __bfloat162float(p[i + half]);
     p[i] = __float2bfloat16_rn(a * cs - c * sn);
     p[i + half] = __float2bfloat16_rn(c * cs + a * sn);
@@ -134,18 +138,30 @@ extern "C" sdlm_status sdlm_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t H, cons
   return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
 }
 
-extern "C" sdlm_status sdlm_rope_block(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, int32_t n_heads,
-                                       void* x, float theta, void* stream) {
-  if (!ctx || !x || batch < 1 || D < 1 || n_heads < 1 || !(theta > 1.f)) return SDLM_ERR_INVALID_ARG;
+static sdlm_status rope_launch(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, int n_heads, void* x, int n_heads2,
+                               void* x2, float theta, void* stream) {
+  if (!ctx || !x || batch < 1 || D < 1 || n_heads < 1 || n_heads2 < 0 || (n_heads2 > 0 && !x2) || !(theta > 1.f))
+    return SDLM_ERR_INVALID_ARG;
   if (batch > ctx->cfg.max_batch) return SDLM_ERR_SHAPE;
   const int d = ctx->cfg.head_dim;
-  const size_t total = (size_t)batch * D * n_heads * (d / 2);
+  const size_t total = (size_t)batch * D * (n_heads + n_heads2) * (d / 2);
   const int blocks = (int)((total + 255) / 256 < 1184 ? (total + 255) / 256 : 1184);
   const cudaError_t e = launch_overlapped(rope_block_kernel, dim3(blocks), dim3(256), 0, static_cast<cudaStream_t>(stream),
-                                          static_cast<__nv_bfloat16*>(x), (const int32_t*)ctx->seq_len, seq_ids, (int)batch,
-                                          (int)D, (int)n_heads, d, log2f(theta));
+                                          static_cast<__nv_bfloat16*>(x), static_cast<__nv_bfloat16*>(x2),
+                                          (const int32_t*)ctx->seq_len, seq_ids, batch, D, n_heads, n_heads2, d, log2f(theta));
   ctx->launches++;
   return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+}
+
+extern "C" sdlm_status sdlm_rope_block(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, int32_t n_heads,
+                                       void* x, float theta, void* stream) {
+  return rope_launch(ctx, batch, D, seq_ids, n_heads, x, 0, nullptr, theta, stream);
+}
+
+extern "C" sdlm_status sdlm_rope_block2(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, int32_t n_heads,
+                                        void* x, int32_t n_heads2, void* x2, float theta, void* stream) {
+  if (n_heads2 < 1) return SDLM_ERR_INVALID_ARG;
+  return rope_launch(ctx, batch, D, seq_ids, n_heads, x, n_heads2, x2, theta, stream);
 }
 
 extern "C" sdlm_status sdlm_swiglu(sdlm_ctx* ctx, int32_t rows, int32_t I, const void* gate_up, void* out, void* stream) {

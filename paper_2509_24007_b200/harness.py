@@ -13,7 +13,7 @@ import torch
 
 import sdlm_synth as syn
 
-from .binding import CONF_LOGIT, Sdlm, SdlmConfig, bf16_tensor_from_bits
+from .binding import CONF_LOGIT, Sdlm, SdlmConfig, accept_commit_layers, bf16_tensor_from_bits
 
 
 def verification_mask(D: int) -> np.ndarray:
@@ -221,8 +221,7 @@ class DecoderStack:
         for l, (sd, w) in enumerate(zip(self.ctx, self.layers)):
             sd.rmsnorm(self.h, w.ln1, self.EPS, self.x, stream=stream)
             sd.linear3(self.x, self.wqkv[l], self.bqkv[l], self.q, self.k[l], self.v[l], stream=stream)
-            sd.rope_block(self.q, self.THETA, stream=stream)
-            sd.rope_block(self.k[l], self.THETA, stream=stream)
+            sd.rope_block2(self.q, self.k[l], self.THETA, stream=stream)
             sd.block_attn(self.q, self.k[l], self.v[l], self.attn, stream=stream)
             sd.linear(self.attn, w.wo, None, self.h, self.h, stream=stream)
             sd.rmsnorm(self.h, w.ln2, self.EPS, self.x, stream=stream)
@@ -232,8 +231,7 @@ class DecoderStack:
         sd0 = self.ctx[0]
         sd0.rmsnorm(self.h, self.ln_f, self.EPS, self.x, stream=stream)
         sd0.lmhead_confidence(self.x, self.w_lm, out.token, out.p_top1, out.entropy, stream=stream)
-        for l, sd in enumerate(self.ctx):
-            sd.accept_commit(tau, out.token, out.p_top1, out.entropy, self.k[l], self.v[l], 0, out.accepted_len,
+        accept_commit_layers(self.ctx, tau, out.token, out.p_top1, out.entropy, self.k, self.v, out.accepted_len,
                              out.out_tokens, stream=stream)
 
     def launches(self) -> int:

@@ -107,6 +107,14 @@ def test_rope_of_the_block_uses_the_positions_after_the_cached_history(n_heads, 
     got = _f64(x)
     # the angle is formed in fp32 on the GPU: pos * inv_freq carries a relative error of ~2^-23 * pos
     assert np.max(np.abs(got - ref)) <= 2.0 ** -8 * np.max(np.abs(ref)) + 4e-3
+    # query and key rows in one launch: the same values as one launch each
+    _, a64, a = _bf16(rng, (len(lens), 4, n_heads, d))
+    _, b64, b = _bf16(rng, (len(lens), 4, 1, d))
+    a1, b1 = a.clone(), b.clone()
+    dp.sd.rope_block2(a, b, theta)
+    dp.sd.rope_block(a1, theta); dp.sd.rope_block(b1, theta)
+    torch.cuda.synchronize()
+    assert torch.equal(a, a1) and torch.equal(b, b1)
     # with seq_ids the named slots' lengths are used
     _, y64, y = _bf16(rng, (2, 4, n_heads, d))
     ids = torch.tensor([3, 1], dtype=torch.int32).cuda()
