@@ -12,6 +12,13 @@
  *                               K/V appended to the paged cache;
  *   (d) sdlm_kv_pages           bookkeeping of that paged cache (Fig. 2b "cached KV states").
  *
+ * Around them: sdlm_decode_step / sdlm_decode_step_host (the whole step in one call),
+ * sdlm_block_attn_masked, sdlm_verify_commit and sdlm_accept_commit_carry (self-speculative decoding of
+ * Sec. 3.4 and blocks preceded by rows of real tokens), sdlm_linear / sdlm_linear3 / sdlm_rmsnorm /
+ * sdlm_rope_block(2) / sdlm_swiglu / sdlm_accept_commit_layers (the rest of a decoder layer of the
+ * Qwen-2.5 backbone, Sec. 4.1, for whole-model steps), sdlm_lmhead_confidence_static (no workspace
+ * scratch), sdlm_selftest_bounded_wait, options and counters.
+ *
  * Conventions that hold for every call unless stated otherwise
  *   - "device" pointers are CUDA global memory of the current device, owned by the caller; the
  *     library keeps no reference to a per-call pointer once the call's work is enqueued.
