@@ -49,6 +49,8 @@ verified_length on hand-worked cases, against brute force, and where it parts fr
 carry_visibility / accept_and_commit_carry (a block preceded by rows of real tokens): the words equal
 the literal mask A_uv over [history ; carry ; block]; attention under them equals dense attention under
 that mask; a loop of such steps leaves in the cache exactly the real tokens' rows whatever gamma was.
+parallel_training_mask / noise_block_attention (Sec. 3.3 parallel training): the mask has the three parts
+of Fig. 2a and reduces to the single-block A_uv; the noise-block rows equal dense attention under it.
 """
 from __future__ import annotations
 
@@ -157,6 +159,39 @@ def carry_visibility(carry_len: Sequence[int], c_max: int, D: int) -> np.ndarray
             vis[b, r] = (1 << (r + 1)) - 1 if r < c else 1 << r
         vis[b, c_max:] = ((1 << int(c)) - 1) | block_bits
     return vis
+
+
+def parallel_training_mask(n_target: int, starts: Sequence[int], D: int) -> np.ndarray:
+    """The attention mask of parallel block training (Sec. 3.3, "Parallel Training", Fig. 2a) over the
+    reordered input [target sequence (n_target tokens) ; noise block 1 ; noise block 2 ; ...], each noise
+    block Y_T^i = [y^{i-1}, [m] x (D-1)] inserted for start position starts[k] (the block's first token
+    y^{i-1} sits at position starts[k] - 1 of the target sequence; here starts[k] counts the target tokens
+    the block may see, i.e. everything before its own first position).  Three parts:
+      (1) causal attention inside the target sequence (top-left);
+      (2) each noise block sees the target tokens before its start, and nothing after (bottom-left);
+      (3) full attention inside a noise block, none between noise blocks (bottom-right).
+    Returns a boolean [n_target + len(starts) * D] square matrix, True = may attend."""
+    n = n_target + len(starts) * D
+    A = np.zeros((n, n), dtype=bool)
+    for u in range(n_target):
+        A[u, :u + 1] = True
+    for k, s0 in enumerate(starts):
+        lo = n_target + k * D
+        A[lo:lo + D, :int(s0)] = True
+        A[lo:lo + D, lo:lo + D] = True
+    return A
+
+
+def noise_block_attention(q_bits: np.ndarray, k_blk_bits: np.ndarray, v_blk_bits: np.ndarray,
+                          target_k_bits: np.ndarray, target_v_bits: np.ndarray, starts: Sequence[int],
+                          scale: Optional[float] = None) -> np.ndarray:
+    """The noise-block rows of the training forward pass: block k (q, k_blk, v_blk [K, D, heads, d])
+    attends to the first starts[k] tokens of one shared target sequence (target_k / target_v
+    [n_target, Hkv, d]) and to itself, parts (2) and (3) of parallel_training_mask.  This is
+    block_attention with one 'sequence' per noise block whose history is a prefix of the target."""
+    pk = [target_k_bits[:int(s0)] for s0 in starts]
+    pv = [target_v_bits[:int(s0)] for s0 in starts]
+    return block_attention(q_bits, k_blk_bits, v_blk_bits, pk, pv, scale)
 
 
 def verification_visibility(D: int) -> np.ndarray:

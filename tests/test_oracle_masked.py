@@ -239,3 +239,47 @@ def test_a_loop_of_carry_steps_leaves_only_real_token_rows_in_the_cache():
         L = int(cache.seq_len[b])
         k, v = cache.gather_fast(b)
         assert L > start[b] and np.array_equal(k, true_k[b, :L]) and np.array_equal(v, true_v[b, :L])
+
+
+# ---- parallel block training: the noise-block rows (Sec. 3.3, Fig. 2a) ---------------------------
+def test_parallel_training_mask_has_the_three_parts_of_the_figure():
+    n, D, starts = 7, 3, [2, 5, 7]
+    A = orc.parallel_training_mask(n, starts, D)
+    assert np.array_equal(A[:n, :n], np.tril(np.ones((n, n), dtype=bool)))          # (1) causal target sequence
+    assert not A[:n, n:].any()                                                      # targets never see noise blocks
+    for k, s0 in enumerate(starts):
+        lo = n + k * D
+        assert A[lo:lo + D, :s0].all() and not A[lo:lo + D, s0:n].any()             # (2) the prefix before the start
+        assert A[lo:lo + D, lo:lo + D].all()                                        # (3) bidirectional inside the block
+        others = np.ones(len(starts) * D, dtype=bool); others[k * D:(k + 1) * D] = False
+        assert not A[lo:lo + D, n:][:, others].any()                                # no attention between noise blocks
+
+
+def test_one_noise_block_at_the_end_is_the_single_block_mask():
+    """With the block placed after i target tokens the block rows are those of A_uv = 1[v<=u] OR 1[u>=i and v>=i]."""
+    i, D = 6, 4
+    A = orc.parallel_training_mask(i, [i], D)
+    L = _literal_mask(i, D)
+    assert np.array_equal(A[i:, :i], L[i:, :i]) and np.array_equal(A[i:, i:], L[i:, i:])
+    assert np.array_equal(A[:i, :i], L[:i, :i])
+
+
+def test_noise_block_rows_equal_dense_attention_under_the_training_mask():
+    n, D, Hq, Hkv, d = 9, 3, 4, 2, 8
+    starts = [1, 4, 9, 4]
+    rng = np.random.default_rng(31)
+    tk, tv = _rand_bits(rng, (n, Hkv, d)), _rand_bits(rng, (n, Hkv, d))
+    q, kb, vb = _rand_bits(rng, (len(starts), D, Hq, d)), _rand_bits(rng, (len(starts), D, Hkv, d)), _rand_bits(rng, (len(starts), D, Hkv, d))
+    out = orc.noise_block_attention(q, kb, vb, tk, tv, starts)
+    f = lambda bits: torch.from_numpy(syn.bf16_bits_to_f32(bits).astype(np.float64))
+    A = torch.from_numpy(orc.parallel_training_mask(n, starts, D))
+    keys = torch.cat([f(tk), f(kb).reshape(-1, Hkv, d)], 0)
+    vals = torch.cat([f(tv), f(vb).reshape(-1, Hkv, d)], 0)
+    for k in range(len(starts)):
+        for j in range(D):
+            u = n + k * D + j
+            for h in range(Hq):
+                s = (keys[:, h // 2] @ f(q)[k, j, h]) / np.sqrt(d)
+                s = torch.where(A[u], s, torch.tensor(float("-inf"), dtype=torch.float64))
+                ref = torch.softmax(s, 0) @ vals[:, h // 2]
+                assert torch.allclose(torch.from_numpy(out[k, j, h]), ref, rtol=0, atol=1e-13)
