@@ -433,6 +433,38 @@ def time_model_level(torch, pk, wl, lengths, n_layers, intermediate, steps, warm
             "what": "whole-model step (random weights of the 3B shape), every operation a library call, one CUDA graph per step"}
 
 
+def time_noise_blocks(torch, pk, DeviceProblem, shape, n_target=4096, n_blocks=64, D=4, iters=200):
+    """Forward attention of the noise-block rows of parallel block training (Sec. 3.3): one target sequence
+    of n_target tokens in the cache, n_blocks noise blocks with random start positions as batch rows."""
+    wl = syn.Workload("train_noise_blocks", shape, n_blocks, D, 0, 0, (0.9,), seed=4711)
+    lens = np.zeros(n_blocks, dtype=np.int32)
+    lens[0] = n_target
+    dp = DeviceProblem(wl, w_bits=np.zeros((16, shape.hidden), np.uint16), lengths=lens, keep_prefix=False)
+    sd = dp.sd
+    x = syn.block_inputs(wl, np.zeros((shape.vocab, shape.hidden), np.uint16), 0)
+    q, k, v = (pk.bf16_tensor_from_bits(t) for t in (x.q, x.k_blk, x.v_blk))
+    starts = np.sort(np.random.default_rng(wl.seed).integers(1, n_target + 1, size=n_blocks)).astype(np.int32)
+    ids = torch.zeros(n_blocks, dtype=torch.int32, device=sd.device)
+    pl = torch.from_numpy(starts).to(sd.device)
+    out = torch.empty_like(q)
+    for _ in range(5):
+        sd.block_attn_prefix(q, k, v, ids, pl, out)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        sd.block_attn_prefix(q, k, v, ids, pl, out)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) / iters * 1e3
+    assert int(sd.device_status()[0]) == 0
+    key_bytes = int(starts.astype(np.int64).sum()) * 2 * shape.n_kv_heads * shape.head_dim * 2
+    return {"us_per_call": us, "noise_blocks": n_blocks, "target_tokens": n_target, "block_D": D,
+            "keys_read_gbs": key_bytes / (us * 1e-6) / 1e9,
+            "what": "sdlm_block_attn_prefix back to back; the shared target K/V (%.1f MB) stays in L2, so this is not an HBM figure"
+                    % (n_target * 2 * shape.n_kv_heads * shape.head_dim * 2 / 1e6)}
+
+
 def time_e2e(torch, dp, wl, steps, warmup, n_blocks=4):
     """Same metric through sdlm_decode_step_host: pinned host inputs copied in, results copied out, every step."""
     s = wl.shape
@@ -588,6 +620,9 @@ def main():
         if args.workload == "cfg2_d4":      # Qwen2.5-3B: 36 layers, intermediate size 11008
             line["extra"]["model_level_3b_" + wl.name] = time_model_level(torch, pk, wl_run, lengths, 36, 11008,
                                                                           max(4, min(args.steps, 30)))
+            torch.cuda.empty_cache()
+        if args.workload == "cfg2_d4":
+            line["extra"]["training_noise_blocks_3b"] = time_noise_blocks(torch, pk, DeviceProblem, wl.shape)
             torch.cuda.empty_cache()
         n_seqs = min(wl.batch, 32)
         tok, dt = oracle_sample(wl, n_seqs, repeats=2)

@@ -14,7 +14,8 @@
  *
  * Around them: sdlm_decode_step / sdlm_decode_step_host (the whole step in one call),
  * sdlm_block_attn_masked, sdlm_verify_commit and sdlm_accept_commit_carry (self-speculative decoding of
- * Sec. 3.4 and blocks preceded by rows of real tokens), sdlm_linear / sdlm_linear3 / sdlm_rmsnorm /
+ * Sec. 3.4 and blocks preceded by rows of real tokens), sdlm_block_attn_prefix (the noise-block rows of
+ * parallel training, Sec. 3.3), sdlm_linear / sdlm_linear3 / sdlm_rmsnorm /
  * sdlm_rope_block(2) / sdlm_swiglu / sdlm_accept_commit_layers (the rest of a decoder layer of the
  * Qwen-2.5 backbone, Sec. 4.1, for whole-model steps), sdlm_lmhead_confidence_static (no workspace
  * scratch), sdlm_selftest_bounded_wait, options and counters.
@@ -160,6 +161,20 @@ sdlm_status sdlm_kv_pages(sdlm_ctx* ctx, sdlm_kv_op op, const sdlm_kv_args* args
  * Errors: INVALID_ARG, SHAPE (batch > max_batch, D > max_block). */
 sdlm_status sdlm_block_attn(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, const void* q,
                             const void* k_blk, const void* v_blk, void* out, void* stream);
+
+/* ---- (a'') block attention over a prefix of a shared sequence -- Sec. 3.3, parallel training: the
+ * reordered training input is [target sequence ; noise blocks]; each noise block Y_T^i sees the target
+ * tokens before its start position and itself, and no other noise block (the bottom-left and
+ * bottom-right parts of the mask of Fig. 2a).  With the target sequence's K/V in the cache, every noise
+ * block is one batch row: row b attends to the first prefix_len[b] cached tokens of slot seq_ids[b]
+ * (several rows may name the same slot) and, without a mask, to its own D rows.  seq_ids and
+ * prefix_len: device int32 [batch], both required; prefix_len[b] beyond the slot's length is clipped
+ * to it.  Everything else as sdlm_block_attn (batch <= max_batch rows).  The causal top-left part of
+ * that mask (the target sequence attending to itself) is ordinary causal attention and is not
+ * provided.  Errors: INVALID_ARG, SHAPE. */
+sdlm_status sdlm_block_attn_prefix(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids,
+                                   const int32_t* prefix_len, const void* q, const void* k_blk, const void* v_blk,
+                                   void* out, void* stream);
 
 /* ---- (a') block attention with an explicit visibility mask over the block's own keys.
  * Sec. 3.4, self-speculative decoding: the D verification inputs of a block are the sampled tokens

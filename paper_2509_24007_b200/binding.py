@@ -33,7 +33,7 @@ EXPORTED = ["sdlm_pool_bytes", "sdlm_workspace_bytes", "sdlm_create", "sdlm_dest
             "sdlm_kv_pages", "sdlm_block_attn", "sdlm_lmhead_confidence", "sdlm_lmhead_confidence_static", "sdlm_accept_commit",
             "sdlm_device_status", "sdlm_decode_step", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count",
             "sdlm_block_attn_masked", "sdlm_verify_commit", "sdlm_accept_commit_carry",
-            "sdlm_linear", "sdlm_linear3", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu", "sdlm_selftest_bounded_wait", "sdlm_rope_block2", "sdlm_accept_commit_layers"]
+            "sdlm_linear", "sdlm_linear3", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu", "sdlm_selftest_bounded_wait", "sdlm_rope_block2", "sdlm_accept_commit_layers", "sdlm_block_attn_prefix"]
 
 
 def accept_commit_layers(contexts, tau: float, token, p_top1, entropy, k_blks, v_blks, accepted_len, out_tokens,
@@ -127,6 +127,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdlm_lmhead_confidence.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_lmhead_confidence_static.restype = C.c_int
     lib.sdlm_lmhead_confidence_static.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_block_attn_prefix.restype = C.c_int
+    lib.sdlm_block_attn_prefix.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_block_attn_masked.restype = C.c_int
     lib.sdlm_block_attn_masked.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_accept_commit_carry.restype = C.c_int
@@ -328,6 +330,19 @@ class Sdlm:
         self._check("sdlm_block_attn", self.lib.sdlm_block_attn(self.ctx, batch, D, _ptr(seq_ids), _ptr(q), _ptr(k_blk),
                                                                 _ptr(v_blk), _ptr(_dev(out, torch.bfloat16, "out")),
                                                                 _stream_ptr(stream)))
+        return out
+
+    def block_attn_prefix(self, q: torch.Tensor, k_blk: torch.Tensor, v_blk: torch.Tensor, seq_ids: torch.Tensor,
+                          prefix_len: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """sdlm_block_attn_prefix: row b sees the first prefix_len[b] cached tokens of slot seq_ids[b]."""
+        batch, D = int(q.shape[0]), int(q.shape[1])
+        _dev(q, torch.bfloat16, "q"); _dev(k_blk, torch.bfloat16, "k_blk"); _dev(v_blk, torch.bfloat16, "v_blk")
+        _dev(seq_ids, torch.int32, "seq_ids"); _dev(prefix_len, torch.int32, "prefix_len")
+        if out is None:
+            out = torch.empty_like(q)
+        self._check("sdlm_block_attn_prefix", self.lib.sdlm_block_attn_prefix(
+            self.ctx, batch, D, _ptr(seq_ids), _ptr(prefix_len), _ptr(q), _ptr(k_blk), _ptr(v_blk),
+            _ptr(_dev(out, torch.bfloat16, "out")), _stream_ptr(stream)))
         return out
 
     def block_attn_masked(self, q: torch.Tensor, k_blk: torch.Tensor, v_blk: torch.Tensor, vis: torch.Tensor,

@@ -752,6 +752,19 @@ extern "C" sdlm_status sdlm_accept_commit_carry(sdlm_ctx* ctx, int32_t batch, in
                               out_tokens, StatCopies{}, stream, nullptr, carry_len, c_max);
 }
 
+extern "C" sdlm_status sdlm_block_attn_prefix(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids,
+                                              const int32_t* prefix_len, const void* q, const void* k_blk,
+                                              const void* v_blk, void* out, void* stream) {
+  if (!ctx || !seq_ids || !prefix_len || !q || !k_blk || !v_blk || !out) return SDLM_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out)) return SDLM_ERR_INVALID_ARG;
+  const sdlm_status s = check_batch(ctx, batch, D);  // rows may share slots, but the scratch is sized by max_batch rows
+  if (s != SDLM_OK) return s;
+  return launch_block_attn(ctx, batch, D, seq_ids, q, k_blk, v_blk, out, static_cast<cudaStream_t>(stream), 0, false, 0,
+                           nullptr, prefix_len) == cudaSuccess
+             ? SDLM_OK
+             : SDLM_ERR_CUDA;
+}
+
 extern "C" sdlm_status sdlm_block_attn_masked(sdlm_ctx* ctx, int32_t batch, int32_t n_q, int32_t n_k,
                                               const int32_t* seq_ids, const void* q, const void* k_blk,
                                               const void* v_blk, const uint32_t* vis, void* out, void* stream) {

@@ -55,6 +55,9 @@ struct AttnParams {
   // when query position j sees block key t.  The cached history is visible to every position.
   int Dk;
   const uint32_t* vis;
+  // null, or [batch]: row b sees only the first prefix_len[b] cached tokens of its slot (several rows may
+  // name the same slot: the noise blocks of one training sequence)
+  const int32_t* prefix_len;
 };
 
 // 8 warps; 12 when 64 stacked query rows need a second set of softmax warps
@@ -63,7 +66,8 @@ constexpr float kRebaseThreshold = 32.0f;  // log2 units a score may exceed its 
 
 __device__ __forceinline__ int attn_slot(const AttnParams& p, int i) { return p.seq_ids ? p.seq_ids[i] : i; }
 __device__ __forceinline__ int attn_len(const AttnParams& p, int i) {
-  const int len = p.seq_len[attn_slot(p, i)];
+  int len = p.seq_len[attn_slot(p, i)];
+  if (p.prefix_len) len = min(len, p.prefix_len[i]);
   return max(0, min(len, p.mpps * kPageSize));
 }
 
@@ -935,7 +939,7 @@ cudaError_t setup_attn(sdlm_ctx* ctx) {
 
 cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, const void* q,
                               const void* k_blk, const void* v_blk, void* out, cudaStream_t st, int cta_cap,
-                              bool whole_tpcs, int n_blk_keys, const uint32_t* vis) {
+                              bool whole_tpcs, int n_blk_keys, const uint32_t* vis, const int32_t* prefix_len) {
   const sdlm_config& c = ctx->cfg;
   AttnParams p;
   p.pool = reinterpret_cast<const __nv_bfloat16*>(ctx->pool);
@@ -958,6 +962,7 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
   p.release_first = cta_cap > 0 ? 1 : 0;
   p.Dk = n_blk_keys > 0 ? n_blk_keys : D;
   p.vis = vis;
+  p.prefix_len = prefix_len;
   // the kernel's tile arithmetic is 32-bit: (tiles of the launch) x (CTAs) must stay below 2^31
   if ((long long)batch * (c.max_pages_per_seq + 1 + ctx->attn_item_cost) * c.n_kv_heads > 13000000ll)
     return cudaErrorInvalidConfiguration;

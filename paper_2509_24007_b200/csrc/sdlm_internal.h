@@ -143,7 +143,7 @@ inline cudaError_t launch_overlapped_cluster(void (*kernel)(KArgs...), dim3 grid
 cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, const void* q,
                               const void* k_blk, const void* v_blk, void* out, cudaStream_t st,
                               int cta_cap = 0, bool whole_tpcs = false, int n_blk_keys = 0,
-                              const uint32_t* vis = nullptr);
+                              const uint32_t* vis = nullptr, const int32_t* prefix_len = nullptr);
 // `independent_of_predecessor`: the caller guarantees that none of the inputs is written by the
 // kernel enqueued just before on `st` (the stripe kernel then overlaps with it).
 sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,

@@ -275,3 +275,27 @@ def test_carry_commit_reports_a_carry_length_out_of_range():
     assert int(acc[0]) == -1 and int(acc[1]) >= 1
     t = dp.sd.kv_tables()
     assert t["seq_len"][0] == 10 and t["seq_len"][1] == 22
+
+
+# ---- the noise-block rows of parallel block training (Sec. 3.3, Fig. 2a) --------------------------
+@pytest.mark.parametrize("Hq,Hkv,d,D", [(4, 2, 64, 4), (16, 2, 128, 4), (16, 2, 128, 8)])
+def test_noise_blocks_over_a_shared_target_sequence(Hq, Hkv, d, D):
+    """One target sequence in the cache (slot 1 of three), many noise blocks as batch rows, each seeing a
+    prefix of it up to its start position: 0, page boundaries, the whole sequence, and beyond it (clipped)."""
+    shape = syn.Shape(Hq, Hkv, d, 64, 64)
+    n_target = 1500
+    starts = np.array([0, 1, 63, 64, 65, 128, 700, 1499, 1500, 9999, 5, 1024], dtype=np.int32)
+    K = len(starts)
+    wl = syn.Workload("train", shape, K, D, 0, 0, (0.9,), seed=77 + D)
+    lens = np.zeros(K, dtype=np.int32); lens[1] = n_target; lens[2] = 10          # other slots are decoys
+    dp = DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16), lengths=lens)
+    x = dp.block(0)
+    ids = torch.full((K,), 1, dtype=torch.int32).cuda()
+    out = dp.sd.block_attn_prefix(x.q, x.k_blk, x.v_blk, ids, torch.from_numpy(starts).cuda())
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+    tk, tv = dp.prefix[1]
+    ref = orc.noise_block_attention(x.host.q, x.host.k_blk, x.host.v_blk, tk, tv, np.minimum(starts, n_target))
+    check_attention(pk.bits_from_bf16_tensor(out), ref)
+    out2 = dp.sd.block_attn_prefix(x.q, x.k_blk, x.v_blk, ids, torch.from_numpy(starts).cuda())
+    assert torch.equal(out, out2)                                                  # fixed merge order
