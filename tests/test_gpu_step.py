@@ -309,3 +309,39 @@ def test_steps_replayed_from_a_cuda_graph_match_eager_steps():
         t = dp.sd.kv_tables()
         assert np.array_equal(t["seq_len"], t_ref["seq_len"]) and np.array_equal(t["page_table"], t_ref["page_table"])
         assert t["status"][0] == 0
+
+
+@pytest.mark.parametrize("name,batch,a_sms", [("cfg2_d4", 32, 42), ("cfg2", 24, 36)])
+def test_back_to_back_side_by_side_steps_without_host_synchronisation(name, batch, a_sms):
+    """Eight whole steps enqueued back to back: with the overlap option the LM head of step n+1 starts while
+    the commit of step n is still running.  Integer results and tables must equal those of the same steps
+    made as three calls in order; attention and confidences agree to rounding."""
+    wl = syn.CONFIGS[name].with_(batch=batch, steps=10)
+    dp = DeviceProblem(wl)
+    blocks = [dp.block(i) for i in range(8)]
+    snap = dp.sd.kv_export()
+    outs = [dp.alloc_outputs() for _ in range(8)]
+    dp.sd.set_option(OPT_STEP_OVERLAP, 0)
+    for x, o in zip(blocks, outs):
+        dp.step(x, wl.tau, o)
+    torch.cuda.synchronize()
+    t_ref = dp.sd.kv_tables()
+    k_ref = [dp.sd.kv_gather(b, int(t_ref["seq_len"][b])) for b in (0, batch - 1)]
+    dp.sd.kv_import(snap)
+    outs2 = [dp.alloc_outputs() for _ in range(8)]
+    dp.sd.set_option(OPT_STEP_OVERLAP, a_sms)
+    for x, o in zip(blocks, outs2):
+        dp.step(x, wl.tau, o, fused=True)
+    torch.cuda.synchronize()
+    dp.sd.set_option(OPT_STEP_OVERLAP, 0)
+    assert dp.sd.device_status()[0] == 0
+    for o, r in zip(outs2, outs):
+        assert torch.equal(o.token, r.token) and torch.equal(o.accepted_len, r.accepted_len)
+        assert torch.equal(o.out_tokens, r.out_tokens)
+        assert (o.attn.float() - r.attn.float()).abs().max().item() <= 2e-2
+        assert (o.p_top1 - r.p_top1).abs().max().item() <= 1e-3
+    t = dp.sd.kv_tables()
+    assert np.array_equal(t["page_table"], t_ref["page_table"]) and np.array_equal(t["seq_len"], t_ref["seq_len"])
+    for (k, v), b in zip(k_ref, (0, batch - 1)):
+        k2, v2 = dp.sd.kv_gather(b, int(t["seq_len"][b]))
+        assert torch.equal(k, k2) and torch.equal(v, v2)
