@@ -332,6 +332,9 @@ sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const
  * sdlm_linear3:  one product whose N1 + N2 + N3 output columns go to three dense tensors out1 [rows, N1],
  *                out2 [rows, N2], out3 [rows, N3] (the q / k / v projections of a layer from the stacked
  *                weight [N1 + N2 + N3, K] and bias); N1, N2, N3 multiples of 16; no residual.
+ * sdlm_linear_swiglu: the gate / up product and the gating in one call: w_interleaved [2I, K] holds gate row
+ *                i at row 2i and up row i at row 2i + 1; out[r, i] = silu(x . gate_i) * (x . up_i), [rows, I];
+ *                the 2I-wide intermediate is never stored.  I % 8 == 0.
  * sdlm_rmsnorm:  out[r, :] = x[r, :] / sqrt(mean_k x[r, k]^2 + eps) * weight[:]; H % 8 == 0.
  * sdlm_rope_block: rotary embedding, in place, of x [batch, D, n_heads, head_dim]: the position of row
  *                (b, j) is (length of slot seq_ids[b], or b, as the tables stand on the stream) + j;
@@ -345,6 +348,8 @@ sdlm_status sdlm_linear(sdlm_ctx* ctx, int32_t rows, int32_t K, int32_t N, const
                         const void* bias, const void* residual, void* out, void* stream);
 sdlm_status sdlm_linear3(sdlm_ctx* ctx, int32_t rows, int32_t K, int32_t N1, int32_t N2, int32_t N3, const void* x,
                          const void* w, const void* bias, void* out1, void* out2, void* out3, void* stream);
+sdlm_status sdlm_linear_swiglu(sdlm_ctx* ctx, int32_t rows, int32_t K, int32_t I, const void* x, const void* w_interleaved,
+                               void* out, void* stream);
 sdlm_status sdlm_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t H, const void* x, const void* weight, float eps,
                          void* out, void* stream);
 sdlm_status sdlm_rope_block(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, int32_t n_heads, void* x,

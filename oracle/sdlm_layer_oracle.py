@@ -98,7 +98,7 @@ def decoder_stack_hidden(h0: np.ndarray, layers, caches, seq_ids, n_q_heads: int
         attn = round_bf16(block_attention(to_bits(q), to_bits(k), to_bits(v), pk, pv))
         h = round_bf16(linear(attn.reshape(rows, n_q_heads * head_dim), w["wo"], None, h))
         x = round_bf16(rms_norm(h, w["ln2"], eps))
-        act = round_bf16(swiglu(round_bf16(linear(x, w["wgu"]))))
+        act = round_bf16(swiglu(linear(x, w["wgu"])))      # one call: the gate / up product is not stored
         h = round_bf16(linear(act, w["wdown"], None, h))
         k_rows.append(to_bits(k))
         v_rows.append(to_bits(v))

@@ -33,7 +33,7 @@ EXPORTED = ["sdlm_pool_bytes", "sdlm_workspace_bytes", "sdlm_create", "sdlm_dest
             "sdlm_kv_pages", "sdlm_block_attn", "sdlm_lmhead_confidence", "sdlm_lmhead_confidence_static", "sdlm_accept_commit",
             "sdlm_device_status", "sdlm_decode_step", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count",
             "sdlm_block_attn_masked", "sdlm_verify_commit", "sdlm_accept_commit_carry",
-            "sdlm_linear", "sdlm_linear3", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu", "sdlm_selftest_bounded_wait", "sdlm_rope_block2", "sdlm_accept_commit_layers", "sdlm_block_attn_prefix"]
+            "sdlm_linear", "sdlm_linear3", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu", "sdlm_selftest_bounded_wait", "sdlm_rope_block2", "sdlm_accept_commit_layers", "sdlm_block_attn_prefix", "sdlm_linear_swiglu"]
 
 
 def accept_commit_layers(contexts, tau: float, token, p_top1, entropy, k_blks, v_blks, accepted_len, out_tokens,
@@ -137,6 +137,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdlm_linear.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.sdlm_selftest_bounded_wait.restype = C.c_int
     lib.sdlm_selftest_bounded_wait.argtypes = [vp, vp]
+    lib.sdlm_linear_swiglu.restype = C.c_int
+    lib.sdlm_linear_swiglu.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
     lib.sdlm_linear3.restype = C.c_int
     lib.sdlm_linear3.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_rmsnorm.restype = C.c_int
@@ -431,6 +433,19 @@ class Sdlm:
                                                           _ptr(_dev(out1, torch.bfloat16, "out1")),
                                                           _ptr(_dev(out2, torch.bfloat16, "out2")),
                                                           _ptr(_dev(out3, torch.bfloat16, "out3")), _stream_ptr(stream)))
+
+    def linear_swiglu(self, x: torch.Tensor, w_interleaved: torch.Tensor, out: Optional[torch.Tensor] = None,
+                      stream=None) -> torch.Tensor:
+        """sdlm_linear_swiglu: w_interleaved [2I, K] = gate_0, up_0, gate_1, up_1, ...; out [rows, I]."""
+        _dev(x, torch.bfloat16, "x"); _dev(w_interleaved, torch.bfloat16, "w_interleaved")
+        K, I = int(w_interleaved.shape[1]), int(w_interleaved.shape[0]) // 2
+        rows = x.numel() // K
+        if out is None:
+            out = torch.empty((rows, I), dtype=torch.bfloat16, device=self.device)
+        self._check("sdlm_linear_swiglu", self.lib.sdlm_linear_swiglu(self.ctx, rows, K, I, _ptr(x), _ptr(w_interleaved),
+                                                                      _ptr(_dev(out, torch.bfloat16, "out")),
+                                                                      _stream_ptr(stream)))
+        return out
 
     def rmsnorm(self, x: torch.Tensor, weight: torch.Tensor, eps: float, out: Optional[torch.Tensor] = None,
                 stream=None) -> torch.Tensor:

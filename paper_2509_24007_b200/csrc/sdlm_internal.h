@@ -151,7 +151,7 @@ sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const voi
                           bool independent_of_predecessor = false, int cta_cap = 0);
 sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, const void* w, const void* bias,
                           const void* residual, void* out, cudaStream_t st, int seg1 = 0, int seg2 = 0,
-                          void* out2 = nullptr, void* out3 = nullptr);
+                          void* out2 = nullptr, void* out3 = nullptr, int act = 0);
 cudaError_t setup_attn(sdlm_ctx* ctx);
 cudaError_t setup_lmhead(sdlm_ctx* ctx);
 

@@ -126,6 +126,15 @@ extern "C" sdlm_status sdlm_linear3(sdlm_ctx* ctx, int32_t rows, int32_t K, int3
                        N1 + N2, out2, out3);
 }
 
+extern "C" sdlm_status sdlm_linear_swiglu(sdlm_ctx* ctx, int32_t rows, int32_t K, int32_t I, const void* x,
+                                          const void* w_interleaved, void* out, void* stream) {
+  if (!ctx || !x || !w_interleaved || !out || rows < 1 || K < 8 || I < 8) return SDLM_ERR_INVALID_ARG;
+  if (!a16(x) || !a16(w_interleaved) || !a16(out)) return SDLM_ERR_INVALID_ARG;
+  if (K % 8 || I % 8) return SDLM_ERR_UNSUPPORTED;
+  return launch_linear(ctx, rows, K, 2 * I, x, w_interleaved, nullptr, nullptr, out, static_cast<cudaStream_t>(stream), 0, 0,
+                       nullptr, nullptr, 1);
+}
+
 extern "C" sdlm_status sdlm_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t H, const void* x, const void* weight, float eps,
                                     void* out, void* stream) {
   if (!ctx || !x || !weight || !out || rows < 1 || H < 8 || !(eps >= 0.f)) return SDLM_ERR_INVALID_ARG;

@@ -70,6 +70,9 @@ struct LmParams {
   int seg1, seg2;
   __nv_bfloat16* out2;
   __nv_bfloat16* out3;
+  // act = 1: the weight's rows interleave gate and up (row 2i gate_i, row 2i+1 up_i); the epilogue stores
+  // silu(gate_i) * up_i to out[row, i], row pitch V / 2 (no bias, residual, split-K or segments then)
+  int act;
 };
 
 __device__ __forceinline__ __nv_bfloat16* linear_dst(const LmParams& p, int row, int n) {
@@ -202,6 +205,20 @@ __device__ __forceinline__ void store16(const uint32_t (&v)[16], __nv_bfloat16* 
   o1.z = ptx::pack_bf16(z[12], z[13]); o1.w = ptx::pack_bf16(z[14], z[15]);
   *reinterpret_cast<uint4*>(out) = o0;
   *(reinterpret_cast<uint4*>(out) + 1) = o1;
+}
+
+// Eight gated outputs from sixteen accumulators (gate, up, gate, up, ...): silu(g) * u, silu(g) = g / (1 + e^-g).
+__device__ __forceinline__ void store8_swiglu(const uint32_t (&v)[16], __nv_bfloat16* out) {
+  float y[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float g = __uint_as_float(v[2 * i]), u = __uint_as_float(v[2 * i + 1]);
+    y[i] = g / (1.f + __expf(-g)) * u;
+  }
+  uint4 o;
+  o.x = ptx::pack_bf16(y[0], y[1]); o.y = ptx::pack_bf16(y[2], y[3]);
+  o.z = ptx::pack_bf16(y[4], y[5]); o.w = ptx::pack_bf16(y[6], y[7]);
+  *reinterpret_cast<uint4*>(out) = o;
 }
 
 __device__ __forceinline__ void store16_f32(const uint32_t (&v)[16], float* dst) {
@@ -364,7 +381,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
           if (c + 1 < n_chunks) tmem_ld16(taddr + (c + 1) * 16, v1);
           const int row = r * 128 + q * 32 + lane;
           if constexpr (LINEAR) {
-            if (p.ksplit > 1) {
+            if (p.act) {
+              if (n0 + c * 16 < n_end && row < p.rows) store8_swiglu(v0, p.out + (size_t)row * (p.V / 2) + (n0 + c * 16) / 2);
+            } else if (p.ksplit > 1) {
               if (n0 + c * 16 < n_end && row < p.rows) store16_f32(v0, p.part + ((size_t)ks * 128 + row) * p.V + n0 + c * 16);
             } else if (n0 + c * 16 < n_end && row < p.rows)
               store16(v0, linear_dst(p, row, n0 + c * 16),
@@ -377,7 +396,10 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
             ptx::tmem_ld_wait();
             if (c + 2 < n_chunks) tmem_ld16(taddr + (c + 2) * 16, v0);
             if constexpr (LINEAR) {
-              if (p.ksplit > 1) {
+              if (p.act) {
+                if (n0 + (c + 1) * 16 < n_end && row < p.rows)
+                  store8_swiglu(v1, p.out + (size_t)row * (p.V / 2) + (n0 + (c + 1) * 16) / 2);
+              } else if (p.ksplit > 1) {
                 if (n0 + (c + 1) * 16 < n_end && row < p.rows)
                   store16_f32(v1, p.part + ((size_t)ks * 128 + row) * p.V + n0 + (c + 1) * 16);
               } else if (n0 + (c + 1) * 16 < n_end && row < p.rows)
@@ -964,7 +986,8 @@ static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden,
 
 // out[rows, N] = x[rows, K] W[N, K]^T (+ residual), bf16 in and out, fp32 accumulation; row blocks of 128.
 sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, const void* w, const void* bias,
-                          const void* residual, void* out, cudaStream_t st, int seg1, int seg2, void* out2, void* out3) {
+                          const void* residual, void* out, cudaStream_t st, int seg1, int seg2, void* out2, void* out3,
+                          int act) {
   for (int r0 = 0; r0 < rows; r0 += 128) {
     const int nr = rows - r0 < 128 ? rows - r0 : 128;
     LmParams p{};
@@ -976,6 +999,8 @@ sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, 
     p.residual = residual ? static_cast<const __nv_bfloat16*>(residual) + (size_t)r0 * N : nullptr;
     p.bias = static_cast<const __nv_bfloat16*>(bias);
     p.wait_at_end = 0;
+    p.act = act;
+    if (act) p.out = static_cast<__nv_bfloat16*>(out) + (size_t)r0 * (N / 2);
     p.seg1 = seg1; p.seg2 = seg2;
     if (seg1 > 0) {
       p.out = static_cast<__nv_bfloat16*>(out) + (size_t)r0 * seg1;
@@ -1008,7 +1033,7 @@ sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, 
     p.ksplit = 1;
     p.kc_per = KC_all;
     p.part = reinterpret_cast<float*>(ctx->ws + ctx->lay.lin_part);
-    if (N <= kLinSplitMaxN && KC_all >= 64 && seg1 == 0) {  // (with 32 K steps the second launch costs more than it saves)
+    if (N <= kLinSplitMaxN && KC_all >= 64 && seg1 == 0 && act == 0) {  // (with 32 K steps the second launch costs more than it saves)
       const int n_ct = (N + 127) / 128;
       int ks = ctx->sm_count / n_ct;
       if (ks > kLinSplitMax) ks = kLinSplitMax;

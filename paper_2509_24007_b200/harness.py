@@ -193,6 +193,9 @@ class DecoderStack:
         # q, k and v come from one product over the stacked weight
         self.wqkv = [torch.cat([w.wq, w.wk, w.wv], dim=0).contiguous() for w in layers]
         self.bqkv = [torch.cat([w.bq, w.bk, w.bv], dim=0).contiguous() for w in layers]
+        # gate and up rows interleaved, so that the product's epilogue can gate in registers
+        self.wgu_il = [torch.stack([w.wgu[:intermediate], w.wgu[intermediate:]], dim=1).reshape(2 * intermediate, -1).contiguous()
+                       for w in layers]
         for l, sd in enumerate(self.ctx):
             sd.kv_reset(self.free_list)
             for b in range(wl.batch):
@@ -225,8 +228,7 @@ class DecoderStack:
             sd.block_attn(self.q, self.k[l], self.v[l], self.attn, stream=stream)
             sd.linear(self.attn, w.wo, None, self.h, self.h, stream=stream)
             sd.rmsnorm(self.h, w.ln2, self.EPS, self.x, stream=stream)
-            sd.linear(self.x, w.wgu, None, None, self.gu, stream=stream)
-            sd.swiglu(self.gu, self.act, stream=stream)
+            sd.linear_swiglu(self.x, self.wgu_il[l], self.act, stream=stream)
             sd.linear(self.act, w.wdown, None, self.h, self.h, stream=stream)
         sd0 = self.ctx[0]
         sd0.rmsnorm(self.h, self.ln_f, self.EPS, self.x, stream=stream)

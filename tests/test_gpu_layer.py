@@ -71,6 +71,21 @@ def test_linear_with_three_outputs_matches_three_products(rows, K, n):
         c += m
 
 
+@pytest.mark.parametrize("rows,K,I", [(128, 2048, 11008), (9, 256, 40), (200, 512, 1024)])
+def test_gated_product_matches_product_then_swiglu(rows, K, I):
+    """sdlm_linear_swiglu over interleaved gate / up rows against the oracle's swiglu(linear(x, [gate ; up]))."""
+    dp = _ctx()
+    rng = np.random.default_rng(rows + K + I)
+    _, x64, x = _bf16(rng, (rows, K))
+    wb, w64, _ = _bf16(rng, (2 * I, K), std=K ** -0.5)                      # [gate rows ; up rows]
+    il = np.ascontiguousarray(np.stack([wb[:I], wb[I:]], axis=1).reshape(2 * I, K))
+    out = dp.sd.linear_swiglu(x, pk.bf16_tensor_from_bits(il))
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+    ref = lo.swiglu(lo.linear(x64, w64))
+    _check_bf16(_f64(out), ref, "linear_swiglu", rel=2.0 ** -7)
+
+
 def test_linear_in_place_on_the_residual_stream():
     dp = _ctx()
     rng = np.random.default_rng(9)
