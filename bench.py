@@ -523,6 +523,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="enqueue every step from the host instead of replaying a CUDA graph")
     ap.add_argument("--no-overlap", action="store_true", help="attention, then the LM head, each on all SMs (no side-by-side step)")
     ap.add_argument("--no-extra", action="store_true", help="skip the D=8 companion measurement and the CPU baseline")
+    ap.add_argument("--model-level-only", action="store_true",
+                    help="run only the whole-model step of the 3B shape and print its figures (for profiling)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
@@ -539,6 +541,10 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
     torch.cuda.set_device(local_rank)
+    if args.model_level_only:
+        wl_m = wl.with_(steps=RESTORE_EVERY + 2)
+        print(json.dumps(time_model_level(torch, pk, wl_m, syn.prefix_lengths(wl_m), 36, 11008, max(2, min(args.steps, 30)))))
+        return
     dist = None
     if world > 1:
         import torch.distributed as dist
