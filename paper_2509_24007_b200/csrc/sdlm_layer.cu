@@ -9,16 +9,17 @@
 
 namespace sdlm {
 
-// out[r, :] = x[r, :] / sqrt(mean(x[r, :]^2) + eps) * weight[:]; one warp per row, fp32 arithmetic.
-__global__ void __launch_bounds__(256) rmsnorm_kernel(const __nv_bfloat16* x, const __nv_bfloat16* weight,
+// out[r, :] = x[r, :] / sqrt(mean(x[r, :]^2) + eps) * weight[:]; one thread block of four warps per row
+// (a row is a few KB: the kernel is latency, so the rows are spread over as many SMs as there are rows).
+__global__ void __launch_bounds__(128) rmsnorm_kernel(const __nv_bfloat16* x, const __nv_bfloat16* weight,
                                                       __nv_bfloat16* out, int rows, int H, float eps) {
+  __shared__ float s_part[4];
   ptx::grid_dep_launch();
   ptx::grid_dep_wait();
-  const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-  if (row >= rows) return;
+  const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
   const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * H);
   float ss = 0.f;
-  for (int c = lane; c < H / 8; c += 32) {
+  for (int c = tid; c < H / 8; c += 128) {
     const uint4 v = xr[c];
     const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
 #pragma unroll
@@ -29,10 +30,13 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const __nv_bfloat16* x, co
   }
 #pragma unroll
   for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if (lane == 0) s_part[tid >> 5] = ss;
+  __syncthreads();
+  ss = (s_part[0] + s_part[1]) + (s_part[2] + s_part[3]);   // the same order in every thread
   const float inv = rsqrtf(ss / (float)H + eps);
   const uint4* wr = reinterpret_cast<const uint4*>(weight);
   uint4* orow = reinterpret_cast<uint4*>(out + (size_t)row * H);
-  for (int c = lane; c < H / 8; c += 32) {
+  for (int c = tid; c < H / 8; c += 128) {
     const uint4 v = xr[c], w = wr[c];
     const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
     const __nv_bfloat16* g = reinterpret_cast<const __nv_bfloat16*>(&w);
@@ -140,7 +144,7 @@ extern "C" sdlm_status sdlm_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t H, cons
   if (!ctx || !x || !weight || !out || rows < 1 || H < 8 || !(eps >= 0.f)) return SDLM_ERR_INVALID_ARG;
   if (!a16(x) || !a16(weight) || !a16(out)) return SDLM_ERR_INVALID_ARG;
   if (H % 8) return SDLM_ERR_UNSUPPORTED;
-  const cudaError_t e = launch_overlapped(rmsnorm_kernel, dim3((rows + 7) / 8), dim3(256), 0, static_cast<cudaStream_t>(stream),
+  const cudaError_t e = launch_overlapped(rmsnorm_kernel, dim3(rows), dim3(128), 0, static_cast<cudaStream_t>(stream),
                                           static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(weight),
                                           static_cast<__nv_bfloat16*>(out), (int)rows, (int)H, eps);
   ctx->launches++;
