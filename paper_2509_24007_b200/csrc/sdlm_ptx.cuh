@@ -286,8 +286,8 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 // Tiled 2-D copy into this CTA's shared memory whose completion is counted on a barrier given by
-// its shared::cluster address (the first CTA's, for the pair's MMA issuer).  No multicast: every CTA
-// fetches its own box.
+// its shared::cluster address (the first CTA's, for the pair's MMA issuer).  Every CTA fetches
+// its own box: the load is not shared between CTAs.
 __device__ __forceinline__ void tma_load_2d_pair(void* dst_smem, const void* tmap, int x, int y, uint32_t bar_cluster_addr) {
   asm volatile(
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::
@@ -329,7 +329,7 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t* bar, uint16_t cta_mas
                "h"(cta_mask)
                : "memory");
 }
-// The same without multicast: only the issuing CTA's barrier.
+// The same, arriving only on the issuing CTA's barrier.
 __device__ __forceinline__ void umma_commit_pair_local(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
