@@ -769,7 +769,8 @@ __global__ void __launch_bounds__(kMmaThreads) lmhead_mma_kernel(const LmParams 
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) linear_reduce_kernel(const float* part, int ksplit, int rows, int N,
                                                             const __nv_bfloat16* bias, const __nv_bfloat16* residual,
-                                                            __nv_bfloat16* out) {
+                                                            __nv_bfloat16* out, int seg1, int seg2, __nv_bfloat16* out2,
+                                                            __nv_bfloat16* out3) {
   ptx::grid_dep_launch();
   ptx::grid_dep_wait();
   const size_t total = (size_t)rows * (N / 8);
@@ -798,7 +799,12 @@ __global__ void __launch_bounds__(256) linear_reduce_kernel(const float* part, i
     uint4 o;
     o.x = ptx::pack_bf16(z[0], z[1]); o.y = ptx::pack_bf16(z[2], z[3]);
     o.z = ptx::pack_bf16(z[4], z[5]); o.w = ptx::pack_bf16(z[6], z[7]);
-    *(reinterpret_cast<uint4*>(out + row * N) + c) = o;
+    const int n = c * 8;  // segments are multiples of 16 columns: eight columns never straddle one
+    __nv_bfloat16* dst = seg1 == 0   ? out + row * N + n
+                         : n < seg1 ? out + row * seg1 + n
+                         : n < seg2 ? out2 + row * (seg2 - seg1) + (n - seg1)
+                                    : out3 + row * (N - seg2) + (n - seg2);
+    *reinterpret_cast<uint4*>(dst) = o;
   }
 }
 
@@ -1033,15 +1039,27 @@ sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, 
     p.ksplit = 1;
     p.kc_per = KC_all;
     p.part = reinterpret_cast<float*>(ctx->ws + ctx->lay.lin_part);
-    if (N <= kLinSplitMaxN && KC_all >= 64 && seg1 == 0 && act == 0) {  // (with 32 K steps the second launch costs more than it saves)
-      const int n_ct = (N + 127) / 128;
-      int ks = ctx->sm_count / n_ct;
-      if (ks > kLinSplitMax) ks = kLinSplitMax;
-      if (ks > KC_all / 4) ks = KC_all / 4;
-      if (ks >= 2) {
-        p.kc_per = (KC_all + ks - 1) / ks;
+    // Every thread block of a column stripe reads all of x's K columns through its SM's L2 port (about 45 GB/s):
+    // 0.4 us per K step whatever the stripe's width, 13 us for K = 2048.  K ranges divide that too.
+    if (N <= kLinSplitMaxN && KC_all >= 16 && act == 0) {
+      // stripe width and number of K ranges from a small cost model (us): K steps per block at the SM's
+      // L2 port rate, plus the second kernel and its traffic when K is cut
+      double best = 1e30;
+      int best_ct = n_cta, best_ks = 1;
+      for (int bn_try = 64; bn_try <= 256; bn_try *= 2) {
+        const int n_ct = (N + bn_try - 1) / bn_try;
+        if (n_ct > ctx->sm_count) continue;
+        for (int ks = 1; ks <= kLinSplitMax && n_ct * ks <= ctx->sm_count && ks * 2 <= KC_all; ++ks) {
+          const int per = (KC_all + ks - 1) / ks;
+          const double t = per * (16384.0 + bn_try * 128.0) / 45000.0 +
+                           (ks > 1 ? 2.5 + (double)ks * nr * N * 8.0 / 3.0e6 : 0.0);
+          if (t < best) { best = t; best_ct = n_ct; best_ks = ks; }
+        }
+      }
+      if (best_ks > 1) {
+        p.kc_per = (KC_all + best_ks - 1) / best_ks;
         p.ksplit = (KC_all + p.kc_per - 1) / p.kc_per;  // every range non-empty
-        n_cta = n_ct;
+        n_cta = best_ct;
       }
     }
     const int gmax = (groups + n_cta - 1) / n_cta;
@@ -1063,7 +1081,7 @@ sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, 
       const size_t total = (size_t)nr * (N / 8);
       const int blocks = (int)((total + 255) / 256);
       le = launch_overlapped(linear_reduce_kernel, dim3(blocks), dim3(256), 0, st, (const float*)p.part, p.ksplit, nr, N,
-                             p.bias, p.residual, p.out);
+                             p.bias, p.residual, p.out, p.seg1, p.seg2, p.out2, p.out3);
       ctx->launches++;
       if (le != cudaSuccess || cudaGetLastError() != cudaSuccess) return SDLM_ERR_CUDA;
     }
