@@ -14,11 +14,12 @@
  *
  * Around them: sdlm_decode_step / sdlm_decode_step_host (the whole step in one call),
  * sdlm_block_attn_masked, sdlm_verify_commit and sdlm_accept_commit_carry (self-speculative decoding of
- * Sec. 3.4 and blocks preceded by rows of real tokens), sdlm_block_attn_prefix (the noise-block rows of
- * parallel training, Sec. 3.3), sdlm_linear / sdlm_linear3 / sdlm_rmsnorm /
- * sdlm_rope_block(2) / sdlm_swiglu / sdlm_accept_commit_layers (the rest of a decoder layer of the
- * Qwen-2.5 backbone, Sec. 4.1, for whole-model steps), sdlm_lmhead_confidence_static (no workspace
- * scratch), sdlm_selftest_bounded_wait, options and counters.
+ * Sec. 3.4 and blocks preceded by rows of real tokens), sdlm_block_attn_prefix and
+ * sdlm_block_attn_masked_prefix (the noise-block rows and the causal rows of parallel training,
+ * Sec. 3.3), sdlm_linear / sdlm_linear3 / sdlm_rmsnorm / sdlm_rope_block(2) / sdlm_swiglu /
+ * sdlm_accept_commit_layers (the rest of a decoder layer of the Qwen-2.5 backbone, Sec. 4.1, for
+ * whole-model steps), sdlm_lmhead_confidence_static (no workspace scratch),
+ * sdlm_selftest_bounded_wait, options and counters.
  *
  * Conventions that hold for every call unless stated otherwise
  *   - "device" pointers are CUDA global memory of the current device, owned by the caller; the
@@ -170,8 +171,8 @@ sdlm_status sdlm_block_attn(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32
  * (several rows may name the same slot) and, without a mask, to its own D rows.  seq_ids and
  * prefix_len: device int32 [batch], both required; prefix_len[b] beyond the slot's length is clipped
  * to it.  Everything else as sdlm_block_attn (batch <= max_batch rows).  The causal top-left part of
- * that mask (the target sequence attending to itself) is ordinary causal attention and is not
- * provided.  Errors: INVALID_ARG, SHAPE. */
+ * that mask (the target sequence attending to itself) is sdlm_block_attn_masked_prefix below.
+ * Errors: INVALID_ARG, SHAPE. */
 sdlm_status sdlm_block_attn_prefix(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids,
                                    const int32_t* prefix_len, const void* q, const void* k_blk, const void* v_blk,
                                    void* out, void* stream);
@@ -191,6 +192,20 @@ sdlm_status sdlm_block_attn_prefix(sdlm_ctx* ctx, int32_t batch, int32_t D, cons
 sdlm_status sdlm_block_attn_masked(sdlm_ctx* ctx, int32_t batch, int32_t n_q, int32_t n_k, const int32_t* seq_ids,
                                    const void* q, const void* k_blk, const void* v_blk, const uint32_t* vis,
                                    void* out, void* stream);
+
+/* ---- (a''') both at once: row b attends to the first prefix_len[b] cached tokens of slot seq_ids[b]
+ * and to those of its n_k block keys that vis[b,j] names.  Sec. 3.3, parallel training, the causal
+ * top-left part of the mask of Fig. 2a (A_uv = 1[v <= u] inside the target sequence): with the target
+ * sequence's K/V in the cache, cut its query rows into chunks of n <= max_block consecutive positions
+ * u0..u0+n-1; chunk = batch row with prefix_len = u0, block keys = the K/V rows of those n positions,
+ * vis[b,j] = 2^(j+1) - 1 (position u0+j sees block keys 0..j).  Together with sdlm_block_attn_prefix
+ * for the noise blocks this is the whole attention of one parallel-training forward pass.
+ * seq_ids, prefix_len: device int32 [batch], both required; everything else, limits and errors as
+ * sdlm_block_attn_masked. */
+sdlm_status sdlm_block_attn_masked_prefix(sdlm_ctx* ctx, int32_t batch, int32_t n_q, int32_t n_k,
+                                          const int32_t* seq_ids, const int32_t* prefix_len, const void* q,
+                                          const void* k_blk, const void* v_blk, const uint32_t* vis, void* out,
+                                          void* stream);
 
 /* ---- (b) LM head -> softmax statistics -- Sec. 3.2 (Z in R^{D x |V|}), Eq. 8, Eq. 9.
  * For each of `rows` hidden states: z = W h (|V| logits, fp32 accumulate, never stored);

@@ -194,6 +194,32 @@ def noise_block_attention(q_bits: np.ndarray, k_blk_bits: np.ndarray, v_blk_bits
     return block_attention(q_bits, k_blk_bits, v_blk_bits, pk, pv, scale)
 
 
+def training_forward_attention(q_bits: np.ndarray, k_bits: np.ndarray, v_bits: np.ndarray, n_target: int,
+                               starts: Sequence[int], D: int, scale: Optional[float] = None) -> np.ndarray:
+    """Attention of one parallel-training forward pass (Sec. 3.3, Fig. 2a), written as its definition:
+    the reordered input [target sequence ; noise blocks] has n = n_target + len(starts) * D positions,
+    q [n, Hq, d], k / v [n, Hkv, d] (bf16 bits); position u attends to exactly the positions v with
+    parallel_training_mask(n_target, starts, D)[u, v] set:
+        out[u, h, :] = sum_v A_uv exp(q_u,h . k_v * scale) v_v / sum_v A_uv exp(q_u,h . k_v * scale).
+    Dense over the whole n x n mask, no chunking.  Returns float64 [n, Hq, d]."""
+    n, Hq, d = q_bits.shape
+    Hkv = k_bits.shape[1]
+    G = Hq // Hkv
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    A = parallel_training_mask(n_target, starts, D)
+    if A.shape[0] != n:
+        raise ValueError("input length does not match the mask")
+    q, k, v = widen(q_bits), widen(k_bits), widen(v_bits)
+    out = np.zeros((n, Hq, d), dtype=np.float64)
+    for h in range(Hq):
+        s = (q[:, h, :] @ k[:, h // G, :].T) * scale           # [n, n] scores of head h
+        s = np.where(A, s, -np.inf)
+        wgt = np.exp(s - np.max(s, axis=1, keepdims=True))     # every row sees itself: the max is finite
+        out[:, h, :] = (wgt @ v[:, h // G, :]) / np.sum(wgt, axis=1, keepdims=True)
+    return out
+
+
 def verification_visibility(D: int) -> np.ndarray:
     """vis[j] for the D verification inputs of one block (Sec. 3.4, self-speculative decoding), with
     the block's keys listed as T = 2D rows: keys 0..D-1 are the real tokens [x^{i-1}, y^1, ..,

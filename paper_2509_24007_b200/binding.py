@@ -33,7 +33,8 @@ EXPORTED = ["sdlm_pool_bytes", "sdlm_workspace_bytes", "sdlm_create", "sdlm_dest
             "sdlm_kv_pages", "sdlm_block_attn", "sdlm_lmhead_confidence", "sdlm_lmhead_confidence_static", "sdlm_accept_commit",
             "sdlm_device_status", "sdlm_decode_step", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count",
             "sdlm_block_attn_masked", "sdlm_verify_commit", "sdlm_accept_commit_carry",
-            "sdlm_linear", "sdlm_linear3", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu", "sdlm_selftest_bounded_wait", "sdlm_rope_block2", "sdlm_accept_commit_layers", "sdlm_block_attn_prefix", "sdlm_linear_swiglu"]
+            "sdlm_linear", "sdlm_linear3", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu", "sdlm_selftest_bounded_wait", "sdlm_rope_block2", "sdlm_accept_commit_layers", "sdlm_block_attn_prefix", "sdlm_linear_swiglu",
+            "sdlm_block_attn_masked_prefix"]
 
 
 def accept_commit_layers(contexts, tau: float, token, p_top1, entropy, k_blks, v_blks, accepted_len, out_tokens,
@@ -131,6 +132,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdlm_block_attn_prefix.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_block_attn_masked.restype = C.c_int
     lib.sdlm_block_attn_masked.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_block_attn_masked_prefix.restype = C.c_int
+    lib.sdlm_block_attn_masked_prefix.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_accept_commit_carry.restype = C.c_int
     lib.sdlm_accept_commit_carry.argtypes = [vp, i32, i32, i32, vp, vp, f32, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_linear.restype = C.c_int
@@ -362,6 +365,24 @@ class Sdlm:
             _dev(seq_ids, torch.int32, "seq_ids")
         self._check("sdlm_block_attn_masked", self.lib.sdlm_block_attn_masked(
             self.ctx, batch, n_q, n_k, _ptr(seq_ids), _ptr(q), _ptr(k_blk), _ptr(v_blk), _ptr(vis),
+            _ptr(_dev(out, torch.bfloat16, "out")), _stream_ptr(stream)))
+        return out
+
+    def block_attn_masked_prefix(self, q: torch.Tensor, k_blk: torch.Tensor, v_blk: torch.Tensor, vis: torch.Tensor,
+                                 seq_ids: torch.Tensor, prefix_len: torch.Tensor,
+                                 out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """sdlm_block_attn_masked_prefix: vis [batch, n_q] int32 words, seq_ids and prefix_len [batch] int32."""
+        batch, n_q, n_k = int(q.shape[0]), int(q.shape[1]), int(k_blk.shape[1])
+        _dev(q, torch.bfloat16, "q"); _dev(k_blk, torch.bfloat16, "k_blk"); _dev(v_blk, torch.bfloat16, "v_blk")
+        _dev(vis, torch.int32, "vis"); _dev(seq_ids, torch.int32, "seq_ids"); _dev(prefix_len, torch.int32, "prefix_len")
+        if tuple(vis.shape) != (batch, n_q):
+            raise ValueError("vis must be [batch, n_q]")
+        if seq_ids.numel() != batch or prefix_len.numel() != batch:
+            raise ValueError("seq_ids and prefix_len must be [batch]")
+        if out is None:
+            out = torch.empty_like(q)
+        self._check("sdlm_block_attn_masked_prefix", self.lib.sdlm_block_attn_masked_prefix(
+            self.ctx, batch, n_q, n_k, _ptr(seq_ids), _ptr(prefix_len), _ptr(q), _ptr(k_blk), _ptr(v_blk), _ptr(vis),
             _ptr(_dev(out, torch.bfloat16, "out")), _stream_ptr(stream)))
         return out
 

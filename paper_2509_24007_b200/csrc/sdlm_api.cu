@@ -782,6 +782,24 @@ extern "C" sdlm_status sdlm_block_attn_masked(sdlm_ctx* ctx, int32_t batch, int3
              : SDLM_ERR_CUDA;
 }
 
+extern "C" sdlm_status sdlm_block_attn_masked_prefix(sdlm_ctx* ctx, int32_t batch, int32_t n_q, int32_t n_k,
+                                                     const int32_t* seq_ids, const int32_t* prefix_len,
+                                                     const void* q, const void* k_blk, const void* v_blk,
+                                                     const uint32_t* vis, void* out, void* stream) {
+  if (!ctx || !seq_ids || !prefix_len || !q || !k_blk || !v_blk || !vis || !out) return SDLM_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out)) return SDLM_ERR_INVALID_ARG;
+  sdlm_status s = check_batch(ctx, batch, n_q);
+  if (s != SDLM_OK) return s;
+  if (n_k < 1) return SDLM_ERR_INVALID_ARG;
+  if (n_k > kMaxBlockKeys) return SDLM_ERR_SHAPE;
+  if (ctx->group * n_q > kMaxQRows) return SDLM_ERR_SHAPE;
+  if (!(ctx->scale > 0.0f)) return SDLM_ERR_UNSUPPORTED;
+  return launch_block_attn(ctx, batch, n_q, seq_ids, q, k_blk, v_blk, out, static_cast<cudaStream_t>(stream), 0, false,
+                           n_k, vis, prefix_len) == cudaSuccess
+             ? SDLM_OK
+             : SDLM_ERR_CUDA;
+}
+
 // One thread block waits, with the same bounded wait every kernel of the library uses, on a barrier and
 // on a counter that nothing ever signals; each wait gives up after its limit (about 0.2 s), the kernel
 // records SDLM_ERR_TIMEOUT in the device status and returns.  The context stays usable.

@@ -299,3 +299,63 @@ def test_noise_blocks_over_a_shared_target_sequence(Hq, Hkv, d, D):
     check_attention(pk.bits_from_bf16_tensor(out), ref)
     out2 = dp.sd.block_attn_prefix(x.q, x.k_blk, x.v_blk, ids, torch.from_numpy(starts).cuda())
     assert torch.equal(out, out2)                                                  # fixed merge order
+
+
+# ---- the whole attention of a parallel-training forward pass (Sec. 3.3, Fig. 2a) ----------------
+@pytest.mark.parametrize("Hq,Hkv,d,D,n_c,n_target", [(4, 2, 64, 4, 8, 333), (16, 2, 128, 4, 8, 1500), (16, 2, 128, 8, 8, 700),
+                                                    (8, 1, 64, 4, 5, 131), (2, 2, 128, 3, 8, 64)])
+def test_training_forward_attention_from_causal_chunks_and_noise_blocks(Hq, Hkv, d, D, n_c, n_target):
+    """Target sequence in the cache (slot 1).  Its own rows: chunks of n_c positions through
+    sdlm_block_attn_masked_prefix with triangular words; the noise blocks: sdlm_block_attn_prefix.  Both
+    against the oracle's dense attention under the full training mask."""
+    shape = syn.Shape(Hq, Hkv, d, 64, 64)
+    starts = np.array([0, 1, 63, 64, 65, n_target // 2, n_target - 1, n_target, 17, n_target // 3], dtype=np.int32)
+    K = len(starts)
+    n_chunks = (n_target + n_c - 1) // n_c
+    B = max(K, n_chunks, 3)
+    wl = syn.Workload("train_full", shape, B, D, 0, 0, (0.9,), seed=900 + d + D + n_c)
+    lens = np.zeros(B, dtype=np.int32); lens[1] = n_target; lens[2] = 10
+    dp = DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16), lengths=lens, max_block=max(D, n_c))
+    tk, tv = dp.prefix[1]
+    x = syn.block_inputs(wl, np.zeros((shape.vocab, shape.hidden), np.uint16), 0)
+    nq, nk, nv = x.q[:K], x.k_blk[:K], x.v_blk[:K]                                   # the noise blocks
+    rng = np.random.default_rng(wl.seed)
+    tq = syn.f32_to_bf16_bits(rng.normal(size=(n_target, Hq, d)).astype(np.float32))   # queries of the target rows
+
+    # (1) causal rows: chunk c = positions c*n_c .. c*n_c+n_c-1, padded at the end with rows that see key 0
+    pad = n_chunks * n_c - n_target
+    cq = np.concatenate([tq, np.zeros((pad, Hq, d), np.uint16)]).reshape(n_chunks, n_c, Hq, d)
+    ck = np.concatenate([tk, np.zeros((pad, Hkv, d), np.uint16)]).reshape(n_chunks, n_c, Hkv, d)
+    cv = np.concatenate([tv, np.zeros((pad, Hkv, d), np.uint16)]).reshape(n_chunks, n_c, Hkv, d)
+    vis = np.tile(np.array([(1 << (j + 1)) - 1 for j in range(n_c)], dtype=np.uint32), (n_chunks, 1))
+    ids = torch.full((n_chunks,), 1, dtype=torch.int32).cuda()
+    u0 = torch.arange(0, n_chunks * n_c, n_c, dtype=torch.int32).cuda()
+    out_c = dp.sd.block_attn_masked_prefix(_dev_bits(cq), _dev_bits(ck), _dev_bits(cv), _vis_tensor(vis), ids, u0)
+    # (2), (3) noise-block rows
+    out_n = dp.sd.block_attn_prefix(_dev_bits(nq), _dev_bits(nk), _dev_bits(nv), torch.full((K,), 1, dtype=torch.int32).cuda(),
+                                    torch.from_numpy(starts).cuda())
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+
+    ref = orc.training_forward_attention(np.concatenate([tq, nq.reshape(K * D, Hq, d)]),
+                                         np.concatenate([tk, nk.reshape(K * D, Hkv, d)]),
+                                         np.concatenate([tv, nv.reshape(K * D, Hkv, d)]), n_target, starts, D)
+    got_c = pk.bits_from_bf16_tensor(out_c).reshape(n_chunks * n_c, Hq, d)[:n_target]
+    check_attention(got_c, ref[:n_target])
+    check_attention(pk.bits_from_bf16_tensor(out_n).reshape(K * D, Hq, d), ref[n_target:])
+    out_c2 = dp.sd.block_attn_masked_prefix(_dev_bits(cq), _dev_bits(ck), _dev_bits(cv), _vis_tensor(vis), ids, u0)
+    assert torch.equal(out_c, out_c2)
+
+
+def test_masked_prefix_argument_checks():
+    shape = syn.Shape(4, 2, 64, 64, 64)
+    wl, dp = _problem(shape, [100, 5], 4, seed=5)
+    x = dp.block(0)
+    ids = torch.zeros(2, dtype=torch.int32).cuda()
+    vis = torch.full((2, 4), 15, dtype=torch.int32).cuda()
+    with pytest.raises((SdlmError, ValueError)):
+        dp.sd.block_attn_masked_prefix(x.q, x.k_blk, x.v_blk, vis[:, :3], ids, ids)
+    with pytest.raises(SdlmError):
+        dp.sd._check("sdlm_block_attn_masked_prefix", dp.sd.lib.sdlm_block_attn_masked_prefix(
+            dp.sd.ctx, 2, 4, 4, None, None, x.q.data_ptr(), x.k_blk.data_ptr(), x.v_blk.data_ptr(), vis.data_ptr(),
+            x.q.data_ptr(), None))

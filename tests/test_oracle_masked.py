@@ -283,3 +283,70 @@ def test_noise_block_rows_equal_dense_attention_under_the_training_mask():
                 s = torch.where(A[u], s, torch.tensor(float("-inf"), dtype=torch.float64))
                 ref = torch.softmax(s, 0) @ vals[:, h // 2]
                 assert torch.allclose(torch.from_numpy(out[k, j, h]), ref, rtol=0, atol=1e-13)
+
+
+# ---- the whole parallel-training forward attention (Sec. 3.3, Fig. 2a) ---------------------------
+def _training_case(seed, n, starts, D, Hq, Hkv, d):
+    rng = np.random.default_rng(seed)
+    N = n + len(starts) * D
+    return _rand_bits(rng, (N, Hq, d)), _rand_bits(rng, (N, Hkv, d)), _rand_bits(rng, (N, Hkv, d))
+
+
+def test_training_attention_target_rows_are_token_by_token_causal_attention():
+    """Part (1) of the mask by brute force: row u of the target sequence is a softmax over keys 0..u, one
+    exponential at a time, and does not change when the noise blocks are replaced."""
+    import math
+    n, D, Hq, Hkv, d = 11, 3, 4, 2, 8
+    starts = [2, 7, 11]
+    q, k, v = _training_case(5, n, starts, D, Hq, Hkv, d)
+    out = orc.training_forward_attention(q, k, v, n, starts, D)
+    fq, fk, fv = (syn.bf16_bits_to_f32(x).astype(np.float64) for x in (q, k, v))
+    for u in range(n):
+        for h in range(Hq):
+            hk = h // (Hq // Hkv)
+            w = [math.exp(sum(fq[u, h, c] * fk[t, hk, c] for c in range(d)) / math.sqrt(d)) for t in range(u + 1)]
+            ref = [sum(w[t] * fv[t, hk, c] for t in range(u + 1)) / sum(w) for c in range(d)]
+            assert np.allclose(out[u, h], ref, rtol=0, atol=1e-12)
+    q2, k2, v2 = q.copy(), k.copy(), v.copy()
+    rng = np.random.default_rng(6)
+    k2[n:], v2[n:], q2[n:] = _rand_bits(rng, k[n:].shape), _rand_bits(rng, v[n:].shape), _rand_bits(rng, q[n:].shape)
+    assert np.array_equal(orc.training_forward_attention(q2, k2, v2, n, starts, D)[:n], out[:n])
+
+
+def test_training_attention_noise_rows_are_block_attention_over_a_prefix():
+    """Parts (2) and (3): the rows of noise block k equal block attention whose history is the first starts[k]
+    target tokens (the prefix-slicing function, written without any mask matrix)."""
+    n, D, Hq, Hkv, d = 13, 4, 4, 2, 8
+    starts = [1, 5, 13, 5, 8]
+    q, k, v = _training_case(8, n, starts, D, Hq, Hkv, d)
+    out = orc.training_forward_attention(q, k, v, n, starts, D)
+    K = len(starts)
+    ref = orc.noise_block_attention(q[n:].reshape(K, D, Hq, d), k[n:].reshape(K, D, Hkv, d), v[n:].reshape(K, D, Hkv, d),
+                                    k[:n], v[:n], starts)
+    assert np.allclose(out[n:].reshape(K, D, Hq, d), ref, rtol=0, atol=1e-13)
+
+
+def test_training_attention_against_the_library_attention_with_a_boolean_mask():
+    """Hq = Hkv: torch's scaled_dot_product_attention in fp64 with the boolean training mask."""
+    n, D, H, d = 10, 3, 3, 16
+    starts = [3, 10, 6]
+    q, k, v = _training_case(9, n, starts, D, H, H, d)
+    out = orc.training_forward_attention(q, k, v, n, starts, D)
+    f = lambda bits: torch.from_numpy(syn.bf16_bits_to_f32(bits).astype(np.float64)).permute(1, 0, 2)   # [H, N, d]
+    A = torch.from_numpy(orc.parallel_training_mask(n, starts, D))
+    ref = torch.nn.functional.scaled_dot_product_attention(f(q), f(k), f(v), attn_mask=A)
+    assert torch.allclose(torch.from_numpy(out).permute(1, 0, 2), ref, rtol=0, atol=1e-12)
+
+
+def test_training_attention_causal_rows_by_chunks_with_triangular_words():
+    """The decomposition the CUDA path uses for part (1): target rows u0..u0+n_c-1 as one masked block over
+    the first u0 target tokens, block key t visible to row j when t <= j."""
+    n, D, Hq, Hkv, d, n_c = 21, 2, 4, 2, 8, 8
+    starts = [4]
+    q, k, v = _training_case(10, n, starts, D, Hq, Hkv, d)
+    out = orc.training_forward_attention(q, k, v, n, starts, D)
+    for u0 in range(0, n, n_c):
+        m = min(n_c, n - u0)
+        vis = np.array([[(1 << (j + 1)) - 1 for j in range(m)]], dtype=np.int64)
+        ref = orc.block_attention_masked(q[None, u0:u0 + m], k[None, u0:u0 + m], v[None, u0:u0 + m], [k[:u0]], [v[:u0]], vis)
+        assert np.allclose(out[u0:u0 + m], ref[0], rtol=0, atol=1e-13)
