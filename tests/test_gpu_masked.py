@@ -354,8 +354,8 @@ def test_masked_prefix_argument_checks():
     x = dp.block(0)
     ids = torch.zeros(2, dtype=torch.int32).cuda()
     vis = torch.full((2, 4), 15, dtype=torch.int32).cuda()
-    with pytest.raises((SdlmError, ValueError)):
-        dp.sd.block_attn_masked_prefix(x.q, x.k_blk, x.v_blk, vis[:, :3], ids, ids)
+    with pytest.raises(ValueError):
+        dp.sd.block_attn_masked_prefix(x.q, x.k_blk, x.v_blk, vis[:, :3].contiguous(), ids, ids)
     with pytest.raises(SdlmError):
         dp.sd._check("sdlm_block_attn_masked_prefix", dp.sd.lib.sdlm_block_attn_masked_prefix(
             dp.sd.ctx, 2, 4, 4, None, None, x.q.data_ptr(), x.k_blk.data_ptr(), x.v_blk.data_ptr(), vis.data_ptr(),
