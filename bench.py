@@ -433,36 +433,65 @@ def time_model_level(torch, pk, wl, lengths, n_layers, intermediate, steps, warm
             "what": "whole-model step (random weights of the 3B shape), every operation a library call, one CUDA graph per step"}
 
 
-def time_noise_blocks(torch, pk, DeviceProblem, shape, n_target=4096, n_blocks=64, D=4, iters=200):
-    """Forward attention of the noise-block rows of parallel block training (Sec. 3.3): one target sequence
-    of n_target tokens in the cache, n_blocks noise blocks with random start positions as batch rows."""
-    wl = syn.Workload("train_noise_blocks", shape, n_blocks, D, 0, 0, (0.9,), seed=4711)
-    lens = np.zeros(n_blocks, dtype=np.int32)
+def time_noise_blocks(torch, pk, DeviceProblem, shape, n_target=4096, n_blocks=64, D=4, n_c=8, iters=100):
+    """Forward attention of parallel block training (Sec. 3.3, Fig. 2a) over one target sequence of n_target
+    tokens in the cache: the noise-block rows (n_blocks blocks with random start positions as batch rows of
+    sdlm_block_attn_prefix) and the causal rows of the target sequence itself (chunks of n_c positions as
+    batch rows of sdlm_block_attn_masked_prefix with triangular visibility words)."""
+    n_chunks = (n_target + n_c - 1) // n_c
+    B = max(n_blocks, n_chunks)
+    wl = syn.Workload("train_forward", shape, B, D, 0, 0, (0.9,), seed=4711)
+    lens = np.zeros(B, dtype=np.int32)
     lens[0] = n_target
-    dp = DeviceProblem(wl, w_bits=np.zeros((16, shape.hidden), np.uint16), lengths=lens, keep_prefix=False)
+    dp = DeviceProblem(wl, w_bits=np.zeros((16, shape.hidden), np.uint16), lengths=lens, keep_prefix=True,
+                       max_block=max(D, n_c))
     sd = dp.sd
     x = syn.block_inputs(wl, np.zeros((shape.vocab, shape.hidden), np.uint16), 0)
-    q, k, v = (pk.bf16_tensor_from_bits(t) for t in (x.q, x.k_blk, x.v_blk))
+    q, k, v = (pk.bf16_tensor_from_bits(t[:n_blocks]) for t in (x.q, x.k_blk, x.v_blk))
     starts = np.sort(np.random.default_rng(wl.seed).integers(1, n_target + 1, size=n_blocks)).astype(np.int32)
-    ids = torch.zeros(n_blocks, dtype=torch.int32, device=sd.device)
+    ids = torch.zeros(B, dtype=torch.int32, device=sd.device)
     pl = torch.from_numpy(starts).to(sd.device)
     out = torch.empty_like(q)
-    for _ in range(5):
-        sd.block_attn_prefix(q, k, v, ids, pl, out)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(iters):
-        sd.block_attn_prefix(q, k, v, ids, pl, out)
-    e1.record()
-    torch.cuda.synchronize()
-    us = e0.elapsed_time(e1) / iters * 1e3
-    assert int(sd.device_status()[0]) == 0
-    key_bytes = int(starts.astype(np.int64).sum()) * 2 * shape.n_kv_heads * shape.head_dim * 2
+
+    def timed(fn):
+        for _ in range(5):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        assert int(sd.device_status()[0]) == 0
+        return e0.elapsed_time(e1) / iters * 1e3
+
+    us = timed(lambda: sd.block_attn_prefix(q, k, v, ids[:n_blocks], pl, out))
+    row_b = 2 * shape.n_kv_heads * shape.head_dim * 2
+    key_bytes = int(starts.astype(np.int64).sum()) * row_b
+
+    # causal rows: the chunk's own K/V rows are the cached rows of its positions
+    tk, tv = dp.prefix[0]
+    pad = n_chunks * n_c - n_target
+    f = lambda a, h: pk.bf16_tensor_from_bits(np.concatenate([a, np.zeros((pad, h, shape.head_dim), np.uint16)])
+                                              .reshape(n_chunks, n_c, h, shape.head_dim))
+    rng = np.random.default_rng(wl.seed + 1)
+    cq = f(syn.f32_to_bf16_bits(rng.normal(size=(n_target, shape.n_q_heads, shape.head_dim)).astype(np.float32)), shape.n_q_heads)
+    ck, cv = f(tk, shape.n_kv_heads), f(tv, shape.n_kv_heads)
+    vis = torch.from_numpy(np.tile(np.array([(1 << (j + 1)) - 1 for j in range(n_c)], dtype=np.int32), (n_chunks, 1))).to(sd.device)
+    u0 = torch.arange(0, n_chunks * n_c, n_c, dtype=torch.int32, device=sd.device)
+    cout = torch.empty_like(cq)
+    us_c = timed(lambda: sd.block_attn_masked_prefix(cq, ck, cv, vis, ids[:n_chunks], u0, cout))
+    causal_flop = 4.0 * shape.n_q_heads * shape.head_dim * (n_target * (n_target + 1) / 2)
+    causal_key_bytes = int(np.arange(0, n_chunks * n_c, n_c, dtype=np.int64).sum()) * row_b
     return {"us_per_call": us, "noise_blocks": n_blocks, "target_tokens": n_target, "block_D": D,
             "keys_read_gbs": key_bytes / (us * 1e-6) / 1e9,
-            "what": "sdlm_block_attn_prefix back to back; the shared target K/V (%.1f MB) stays in L2, so this is not an HBM figure"
-                    % (n_target * 2 * shape.n_kv_heads * shape.head_dim * 2 / 1e6)}
+            "causal_rows_us_per_call": us_c, "causal_chunk": n_c, "causal_chunks": n_chunks,
+            "causal_tflops": causal_flop / (us_c * 1e-6) / 1e12,
+            "causal_keys_read_gbs": causal_key_bytes / (us_c * 1e-6) / 1e9,
+            "what": "sdlm_block_attn_prefix (noise blocks) and sdlm_block_attn_masked_prefix (causal rows) back to back; "
+                    "the shared target K/V (%.1f MB) stays in L2, so these are not HBM figures; causal_tflops counts the "
+                    "lower triangle only" % (n_target * row_b / 1e6)}
 
 
 def time_e2e(torch, dp, wl, steps, warmup, n_blocks=4):
