@@ -325,7 +325,10 @@ sdlm_status sdlm_decode_step(sdlm_ctx* ctx, int32_t batch, int32_t D, const int3
  * accepted_len [batch] and out_tokens [batch,D] back to HOST (any may be NULL to skip) and
  * synchronises `stream` before returning.  A result buffer that is page-locked host memory the GPU
  * can address (cudaHostAlloc / cudaHostRegister) is written by the kernels directly, without a
- * copy after the step; its contents are defined once the call has returned.  w_lm stays a DEVICE
+ * copy after the step; its contents are defined once the call has returned.  Likewise q, k_blk and
+ * v_blk in such memory (16-byte aligned) are not staged: attention and the commit read those rows,
+ * once each, straight from the host buffer, which must stay unchanged until the call returns;
+ * hidden is always copied (every thread block of the LM head re-reads it).  w_lm stays a DEVICE
  * pointer (model state).
  * Errors: as the three calls, plus CUDA. */
 sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids_host,

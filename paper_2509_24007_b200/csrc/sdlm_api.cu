@@ -899,6 +899,27 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
   // hidden rows are copied on the caller's stream and the LM head follows at once; q, k, v (and the
   // sequence ids) are copied on a second stream of the context and attention follows there, on its A
   // SMs; the commit waits for both.  Otherwise everything is enqueued on the caller's stream in order.
+  // Page-locked host memory that the GPU can address is used in place: result buffers are written by the
+  // kernels themselves (attention's output rows during the step, the small per-row results by the commit
+  // kernel), and the block's q / k / v rows, which attention and the commit read once, are read by those
+  // kernels straight from the host buffer.  That saves a copy each; any other host buffer goes through a
+  // copy.  (`hidden` is always copied: every thread block of the LM head re-reads it.)
+  auto mapped = [](const void* host_ptr) -> void* {
+    if (!host_ptr) return nullptr;
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, host_ptr) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    return a.type == cudaMemoryTypeHost ? a.devicePointer : nullptr;
+  };
+  auto mapped16 = [&](const void* host_ptr) -> const void* {
+    const void* d = mapped(host_ptr);
+    return d && aligned16(d) ? d : nullptr;
+  };
+  const void* in_q = mapped16(q_host);
+  const void* in_k = mapped16(k_blk_host);
+  const void* in_v = mapped16(v_blk_host);
   const int a_sms = ctx->host_two_streams ? ctx->overlap_lmhead : 0;
   cudaStream_t qkv_st = st;
   if (a_sms > 0) {
@@ -913,9 +934,18 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
     ok &= cudaStreamWaitEvent(qkv_st, ctx->ev_fork, 0) == cudaSuccess;
     ok &= cudaMemcpyAsync(ws + L.st_hidden, hidden_host, rows * c.hidden * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
   }
-  ok &= cudaMemcpyAsync(ws + L.st_q, q_host, q_bytes, cudaMemcpyHostToDevice, qkv_st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(ws + L.st_k, k_blk_host, kv_bytes, cudaMemcpyHostToDevice, qkv_st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(ws + L.st_v, v_blk_host, kv_bytes, cudaMemcpyHostToDevice, qkv_st) == cudaSuccess;
+  if (!in_q) {
+    ok &= cudaMemcpyAsync(ws + L.st_q, q_host, q_bytes, cudaMemcpyHostToDevice, qkv_st) == cudaSuccess;
+    in_q = ws + L.st_q;
+  }
+  if (!in_k) {
+    ok &= cudaMemcpyAsync(ws + L.st_k, k_blk_host, kv_bytes, cudaMemcpyHostToDevice, qkv_st) == cudaSuccess;
+    in_k = ws + L.st_k;
+  }
+  if (!in_v) {
+    ok &= cudaMemcpyAsync(ws + L.st_v, v_blk_host, kv_bytes, cudaMemcpyHostToDevice, qkv_st) == cudaSuccess;
+    in_v = ws + L.st_v;
+  }
   if (a_sms == 0)
     ok &= cudaMemcpyAsync(ws + L.st_hidden, hidden_host, rows * c.hidden * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
   const int32_t* seq_ids = nullptr;
@@ -929,18 +959,6 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
   float* d_ent = reinterpret_cast<float*>(ws + L.st_ent);
   int32_t* d_acc = reinterpret_cast<int32_t*>(ws + L.st_acc);
   int32_t* d_out_tokens = reinterpret_cast<int32_t*>(ws + L.st_out_tokens);
-  // A result buffer in page-locked host memory that the GPU can address is written by the kernels
-  // themselves (attention's output rows during the step, the small per-row results by the commit
-  // kernel), which saves a copy after the step; any other host buffer is filled by a copy.
-  auto mapped = [](void* host_ptr) -> void* {
-    if (!host_ptr) return nullptr;
-    cudaPointerAttributes a;
-    if (cudaPointerGetAttributes(&a, host_ptr) != cudaSuccess) {
-      cudaGetLastError();
-      return nullptr;
-    }
-    return a.type == cudaMemoryTypeHost ? a.devicePointer : nullptr;
-  };
   void* m_attn = mapped(attn_out_host);
   if (m_attn && !aligned16(m_attn)) m_attn = nullptr;
   int32_t* m_acc = static_cast<int32_t*>(mapped(accepted_len_host));
@@ -954,18 +972,17 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
   int32_t* o_tok = m_out_tokens ? m_out_tokens : d_out_tokens;
   if (a_sms > 0) {
     if (!aligned16(w_lm)) return SDLM_ERR_INVALID_ARG;
-    if (launch_block_attn(ctx, batch, D, seq_ids, ws + L.st_q, ws + L.st_k, ws + L.st_v, d_attn, qkv_st, a_sms,
-                          batch * D > 128) != cudaSuccess)
+    if (launch_block_attn(ctx, batch, D, seq_ids, in_q, in_k, in_v, d_attn, qkv_st, a_sms, batch * D > 128) != cudaSuccess)
       return SDLM_ERR_CUDA;
     if (cudaEventRecord(ctx->ev_join, qkv_st) != cudaSuccess) return SDLM_ERR_CUDA;
     s = launch_lmhead(ctx, batch * D, ws + L.st_hidden, w_lm, d_token, d_p, d_ent, nullptr, nullptr, st,
                       /*independent_of_predecessor=*/false, ctx->sm_count - a_sms);
     if (s != SDLM_OK) return s;
     if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return SDLM_ERR_CUDA;
-    s = accept_commit_launch(ctx, batch, D, seq_ids, tau, mode, d_token, d_p, d_ent, ws + L.st_k, ws + L.st_v, o_acc, o_tok,
-                             copies, stream);
+    s = accept_commit_launch(ctx, batch, D, seq_ids, tau, mode, d_token, d_p, d_ent, in_k, in_v, o_acc, o_tok, copies,
+                             stream);
   } else {
-    s = decode_step_device(ctx, batch, D, seq_ids, tau, mode, ws + L.st_q, ws + L.st_k, ws + L.st_v, ws + L.st_hidden, w_lm,
+    s = decode_step_device(ctx, batch, D, seq_ids, tau, mode, in_q, in_k, in_v, ws + L.st_hidden, w_lm,
                            d_attn, d_token, d_p, d_ent, o_acc, o_tok, copies, stream);
   }
   if (s != SDLM_OK) return s;

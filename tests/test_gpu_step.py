@@ -164,10 +164,12 @@ def test_cfg4_long_prefix_multi_step_loop():
     print("cfg4 committed", total_ref, "tokens in", wl.steps, "steps; flagged", flagged)
 
 
+@pytest.mark.parametrize("inputs", ["page-locked", "pageable"])
 @pytest.mark.parametrize("results", ["page-locked", "pageable", "mixed"])
-def test_decode_step_host_entry_matches_device_calls(results):
+def test_decode_step_host_entry_matches_device_calls(results, inputs):
     """Page-locked result buffers are written by the kernels themselves, pageable ones by copies after
-    the step: the host sees the same values either way, and entropy too."""
+    the step; page-locked q / k / v rows are read in place by the kernels, pageable ones are copied in:
+    the host sees the same values either way, and entropy too."""
     wl = syn.CONFIGS["cfg0"].with_(batch=3, prefix_lo=10, prefix_hi=200)
     dp = DeviceProblem(wl)
     x = dp.block(0)
@@ -175,7 +177,7 @@ def test_decode_step_host_entry_matches_device_calls(results):
     torch.cuda.synchronize()
     t_ref = dp.sd.kv_tables()
     dp.reset_cache()
-    pin = lambda t: t.cpu().pin_memory()
+    pin = (lambda t: t.cpu().pin_memory()) if inputs == "page-locked" else (lambda t: t.cpu())
     B, D, s = wl.batch, wl.block, wl.shape
     def buf(shape, dtype, i):
         t = torch.full(shape, -7, dtype=dtype)
