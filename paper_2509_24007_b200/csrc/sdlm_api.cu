@@ -895,10 +895,6 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
   const size_t q_bytes = rows * c.n_q_heads * c.head_dim * 2, kv_bytes = rows * c.n_kv_heads * c.head_dim * 2;
   char* ws = ctx->ws;
   bool ok = true;
-  // Side by side (overlap option A > 0): the LM head only needs `hidden`, attention only q / k / v.  The
-  // hidden rows are copied on the caller's stream and the LM head follows at once; q, k, v (and the
-  // sequence ids) are copied on a second stream of the context and attention follows there, on its A
-  // SMs; the commit waits for both.  Otherwise everything is enqueued on the caller's stream in order.
   // Page-locked host memory that the GPU can address is used in place: result buffers are written by the
   // kernels themselves (attention's output rows during the step, the small per-row results by the commit
   // kernel), and the block's q / k / v rows, which attention and the commit read once, are read by those
@@ -913,13 +909,16 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
     }
     return a.type == cudaMemoryTypeHost ? a.devicePointer : nullptr;
   };
-  auto mapped16 = [&](const void* host_ptr) -> const void* {
-    const void* d = mapped(host_ptr);
+  auto mapped16 = [&](const void* host_ptr) -> void* {
+    void* d = mapped(host_ptr);
     return d && aligned16(d) ? d : nullptr;
   };
-  const void* in_q = mapped16(q_host);
-  const void* in_k = mapped16(k_blk_host);
-  const void* in_v = mapped16(v_blk_host);
+  // Two streams (option; only with the overlap option A > 0): `hidden` is copied and the LM head runs on
+  // the caller's stream while q, k, v (and the sequence ids) are copied and attention runs, on its A SMs,
+  // on a second stream of the context; the commit waits for both.  Otherwise everything is enqueued on
+  // the caller's stream.  Either way the copy of `hidden` goes first, so that the GPU is busy while the
+  // host looks up the other buffers, and the result buffers are looked up after the long kernels are
+  // under way.
   const int a_sms = ctx->host_two_streams ? ctx->overlap_lmhead : 0;
   cudaStream_t qkv_st = st;
   if (a_sms > 0) {
@@ -932,8 +931,11 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
     qkv_st = ctx->side_stream;
     ok &= cudaEventRecord(ctx->ev_fork, st) == cudaSuccess;          // whatever the caller enqueued before comes first
     ok &= cudaStreamWaitEvent(qkv_st, ctx->ev_fork, 0) == cudaSuccess;
-    ok &= cudaMemcpyAsync(ws + L.st_hidden, hidden_host, rows * c.hidden * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
   }
+  ok &= cudaMemcpyAsync(ws + L.st_hidden, hidden_host, rows * c.hidden * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  const void* in_q = mapped16(q_host);
+  const void* in_k = mapped16(k_blk_host);
+  const void* in_v = mapped16(v_blk_host);
   if (!in_q) {
     ok &= cudaMemcpyAsync(ws + L.st_q, q_host, q_bytes, cudaMemcpyHostToDevice, qkv_st) == cudaSuccess;
     in_q = ws + L.st_q;
@@ -946,45 +948,41 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
     ok &= cudaMemcpyAsync(ws + L.st_v, v_blk_host, kv_bytes, cudaMemcpyHostToDevice, qkv_st) == cudaSuccess;
     in_v = ws + L.st_v;
   }
-  if (a_sms == 0)
-    ok &= cudaMemcpyAsync(ws + L.st_hidden, hidden_host, rows * c.hidden * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
   const int32_t* seq_ids = nullptr;
   if (seq_ids_host) {
     ok &= cudaMemcpyAsync(ws + L.st_seq_ids, seq_ids_host, (size_t)batch * 4, cudaMemcpyHostToDevice, qkv_st) == cudaSuccess;
     seq_ids = reinterpret_cast<const int32_t*>(ws + L.st_seq_ids);
   }
   if (!ok) return SDLM_ERR_CUDA;
+  if (!aligned16(w_lm)) return SDLM_ERR_INVALID_ARG;
   int32_t* d_token = reinterpret_cast<int32_t*>(ws + L.st_token);
   float* d_p = reinterpret_cast<float*>(ws + L.st_p);
   float* d_ent = reinterpret_cast<float*>(ws + L.st_ent);
   int32_t* d_acc = reinterpret_cast<int32_t*>(ws + L.st_acc);
   int32_t* d_out_tokens = reinterpret_cast<int32_t*>(ws + L.st_out_tokens);
-  void* m_attn = mapped(attn_out_host);
-  if (m_attn && !aligned16(m_attn)) m_attn = nullptr;
+  void* m_attn = mapped16(attn_out_host);
+  void* d_attn = m_attn ? m_attn : ws + L.st_out;
+  const int overlap = ctx->overlap_lmhead;  // A: attention's SMs in the side-by-side step (0: in order)
+  if (launch_block_attn(ctx, batch, D, seq_ids, in_q, in_k, in_v, d_attn, qkv_st, overlap, overlap > 0 && batch * D > 128) !=
+      cudaSuccess)
+    return SDLM_ERR_CUDA;
+  if (a_sms > 0 && cudaEventRecord(ctx->ev_join, qkv_st) != cudaSuccess) return SDLM_ERR_CUDA;
+  // on one stream the LM head follows attention, which lets it go at once when the two run side by side;
+  // on two streams it follows the copy of `hidden` and takes its wait as a full dependency
+  s = launch_lmhead(ctx, batch * D, ws + L.st_hidden, w_lm, d_token, d_p, d_ent, nullptr, nullptr, st,
+                    /*independent_of_predecessor=*/a_sms == 0 && overlap > 0, overlap > 0 ? ctx->sm_count - overlap : 0);
+  if (s != SDLM_OK) return s;
+  if (a_sms > 0 && cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return SDLM_ERR_CUDA;
   int32_t* m_acc = static_cast<int32_t*>(mapped(accepted_len_host));
   int32_t* m_out_tokens = static_cast<int32_t*>(mapped(out_tokens_host));
   StatCopies copies;
   copies.token = static_cast<int32_t*>(mapped(token_host));
   copies.p_top1 = static_cast<float*>(mapped(p_top1_host));
   copies.entropy = static_cast<float*>(mapped(entropy_host));
-  void* d_attn = m_attn ? m_attn : ws + L.st_out;
   int32_t* o_acc = m_acc ? m_acc : d_acc;
   int32_t* o_tok = m_out_tokens ? m_out_tokens : d_out_tokens;
-  if (a_sms > 0) {
-    if (!aligned16(w_lm)) return SDLM_ERR_INVALID_ARG;
-    if (launch_block_attn(ctx, batch, D, seq_ids, in_q, in_k, in_v, d_attn, qkv_st, a_sms, batch * D > 128) != cudaSuccess)
-      return SDLM_ERR_CUDA;
-    if (cudaEventRecord(ctx->ev_join, qkv_st) != cudaSuccess) return SDLM_ERR_CUDA;
-    s = launch_lmhead(ctx, batch * D, ws + L.st_hidden, w_lm, d_token, d_p, d_ent, nullptr, nullptr, st,
-                      /*independent_of_predecessor=*/false, ctx->sm_count - a_sms);
-    if (s != SDLM_OK) return s;
-    if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return SDLM_ERR_CUDA;
-    s = accept_commit_launch(ctx, batch, D, seq_ids, tau, mode, d_token, d_p, d_ent, in_k, in_v, o_acc, o_tok, copies,
-                             stream);
-  } else {
-    s = decode_step_device(ctx, batch, D, seq_ids, tau, mode, in_q, in_k, in_v, ws + L.st_hidden, w_lm,
-                           d_attn, d_token, d_p, d_ent, o_acc, o_tok, copies, stream);
-  }
+  s = accept_commit_launch(ctx, batch, D, seq_ids, tau, mode, d_token, d_p, d_ent, in_k, in_v, o_acc, o_tok, copies,
+                           stream);
   if (s != SDLM_OK) return s;
   if (attn_out_host && !m_attn)
     ok &= cudaMemcpyAsync(attn_out_host, ws + L.st_out, q_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
