@@ -16,7 +16,7 @@
  * sdlm_block_attn_masked, sdlm_verify_commit and sdlm_accept_commit_carry (self-speculative decoding of
  * Sec. 3.4 and blocks preceded by rows of real tokens), sdlm_block_attn_prefix and
  * sdlm_block_attn_masked_prefix (the noise-block rows and the causal rows of parallel training,
- * Sec. 3.3), sdlm_linear / sdlm_linear3 / sdlm_rmsnorm / sdlm_rope_block(2) / sdlm_swiglu /
+ * Sec. 3.3), sdlm_linear / sdlm_linear3 / sdlm_linear_rmsnorm / sdlm_rmsnorm / sdlm_rope_block(2) / sdlm_swiglu /
  * sdlm_accept_commit_layers (the rest of a decoder layer of the Qwen-2.5 backbone, Sec. 4.1, for
  * whole-model steps), sdlm_lmhead_confidence_static (no workspace scratch),
  * sdlm_selftest_bounded_wait, options and counters.
@@ -370,6 +370,16 @@ sdlm_status sdlm_linear_swiglu(sdlm_ctx* ctx, int32_t rows, int32_t K, int32_t I
                                void* out, void* stream);
 sdlm_status sdlm_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t H, const void* x, const void* weight, float eps,
                          void* out, void* stream);
+
+/* sdlm_linear followed by sdlm_rmsnorm of its output rows, for a product whose result is normalised
+ * next (the output and down projections of a pre-norm decoder layer, Sec. 4.1):
+ *   out = x w^T (+ bias) (+ residual),  norm_out[r,:] = out[r,:] / sqrt(mean(out[r,:]^2) + eps) * norm_weight.
+ * norm_weight [N], norm_out [rows, N]: device bf16, 16-byte aligned; the rest as sdlm_linear (residual
+ * may be out).  Same values, bit for bit, as the two calls; where the product is cut along K the sum
+ * of the K ranges and the norm share one kernel.  Errors: as sdlm_linear and sdlm_rmsnorm. */
+sdlm_status sdlm_linear_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t K, int32_t N, const void* x, const void* w,
+                                const void* bias, const void* residual, void* out, const void* norm_weight,
+                                float eps, void* norm_out, void* stream);
 sdlm_status sdlm_rope_block(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, int32_t n_heads, void* x,
                             float theta, void* stream);
 sdlm_status sdlm_rope_block2(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, int32_t n_heads, void* x,

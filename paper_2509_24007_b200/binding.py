@@ -34,7 +34,7 @@ EXPORTED = ["sdlm_pool_bytes", "sdlm_workspace_bytes", "sdlm_create", "sdlm_dest
             "sdlm_device_status", "sdlm_decode_step", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count",
             "sdlm_block_attn_masked", "sdlm_verify_commit", "sdlm_accept_commit_carry",
             "sdlm_linear", "sdlm_linear3", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu", "sdlm_selftest_bounded_wait", "sdlm_rope_block2", "sdlm_accept_commit_layers", "sdlm_block_attn_prefix", "sdlm_linear_swiglu",
-            "sdlm_block_attn_masked_prefix"]
+            "sdlm_block_attn_masked_prefix", "sdlm_linear_rmsnorm"]
 
 
 def accept_commit_layers(contexts, tau: float, token, p_top1, entropy, k_blks, v_blks, accepted_len, out_tokens,
@@ -136,6 +136,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdlm_block_attn_masked_prefix.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_accept_commit_carry.restype = C.c_int
     lib.sdlm_accept_commit_carry.argtypes = [vp, i32, i32, i32, vp, vp, f32, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_linear_rmsnorm.restype = C.c_int
+    lib.sdlm_linear_rmsnorm.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, f32, vp, vp]
     lib.sdlm_linear.restype = C.c_int
     lib.sdlm_linear.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.sdlm_selftest_bounded_wait.restype = C.c_int
@@ -440,6 +442,22 @@ class Sdlm:
         self._check("sdlm_linear", self.lib.sdlm_linear(self.ctx, rows, K, N, _ptr(x), _ptr(w), _ptr(bias), _ptr(residual),
                                                         _ptr(_dev(out, torch.bfloat16, "out")), _stream_ptr(stream)))
         return out
+
+    def linear_rmsnorm(self, x: torch.Tensor, w: torch.Tensor, norm_weight: torch.Tensor, eps: float,
+                       bias: Optional[torch.Tensor] = None, residual: Optional[torch.Tensor] = None,
+                       out: Optional[torch.Tensor] = None, norm_out: Optional[torch.Tensor] = None, stream=None):
+        """sdlm_linear_rmsnorm: out = x w^T (+ bias) (+ residual) and norm_out = RMSNorm(out) * norm_weight."""
+        _dev(x, torch.bfloat16, "x"); _dev(w, torch.bfloat16, "w"); _dev(norm_weight, torch.bfloat16, "norm_weight")
+        K, N = int(w.shape[1]), int(w.shape[0])
+        rows = x.numel() // K
+        if out is None:
+            out = torch.empty((rows, N), dtype=torch.bfloat16, device=self.device)
+        if norm_out is None:
+            norm_out = torch.empty((rows, N), dtype=torch.bfloat16, device=self.device)
+        self._check("sdlm_linear_rmsnorm", self.lib.sdlm_linear_rmsnorm(
+            self.ctx, rows, K, N, _ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(_dev(out, torch.bfloat16, "out")),
+            _ptr(norm_weight), float(eps), _ptr(_dev(norm_out, torch.bfloat16, "norm_out")), _stream_ptr(stream)))
+        return out, norm_out
 
     def linear3(self, x: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor], out1: torch.Tensor,
                 out2: torch.Tensor, out3: torch.Tensor, stream=None) -> None:

@@ -149,9 +149,17 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
 sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
                           float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st,
                           bool independent_of_predecessor = false, int cta_cap = 0);
+// RMSNorm of a linear product's output rows, written beside them (norm_out = out / rms(out) * weight)
+struct LinNorm {
+  const void* weight;
+  float eps;
+  void* out;
+};
 sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, const void* w, const void* bias,
                           const void* residual, void* out, cudaStream_t st, int seg1 = 0, int seg2 = 0,
-                          void* out2 = nullptr, void* out3 = nullptr, int act = 0);
+                          void* out2 = nullptr, void* out3 = nullptr, int act = 0, const LinNorm* norm = nullptr);
+cudaError_t launch_rmsnorm(sdlm_ctx* ctx, int rows, int H, const void* x, const void* weight, float eps, void* out,
+                           cudaStream_t st);
 cudaError_t setup_attn(sdlm_ctx* ctx);
 cudaError_t setup_lmhead(sdlm_ctx* ctx);
 

@@ -107,6 +107,15 @@ __global__ void __launch_bounds__(256) swiglu_kernel(const __nv_bfloat16* gate_u
 
 static inline bool a16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+cudaError_t launch_rmsnorm(sdlm_ctx* ctx, int rows, int H, const void* x, const void* weight, float eps, void* out,
+                           cudaStream_t st) {
+  const cudaError_t e = launch_overlapped(rmsnorm_kernel, dim3(rows), dim3(128), 0, st, static_cast<const __nv_bfloat16*>(x),
+                                          static_cast<const __nv_bfloat16*>(weight), static_cast<__nv_bfloat16*>(out), rows, H,
+                                          eps);
+  ctx->launches++;
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
 }  // namespace sdlm
 
 using namespace sdlm;
@@ -144,11 +153,22 @@ extern "C" sdlm_status sdlm_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t H, cons
   if (!ctx || !x || !weight || !out || rows < 1 || H < 8 || !(eps >= 0.f)) return SDLM_ERR_INVALID_ARG;
   if (!a16(x) || !a16(weight) || !a16(out)) return SDLM_ERR_INVALID_ARG;
   if (H % 8) return SDLM_ERR_UNSUPPORTED;
-  const cudaError_t e = launch_overlapped(rmsnorm_kernel, dim3(rows), dim3(128), 0, static_cast<cudaStream_t>(stream),
-                                          static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(weight),
-                                          static_cast<__nv_bfloat16*>(out), (int)rows, (int)H, eps);
-  ctx->launches++;
-  return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
+  return launch_rmsnorm(ctx, rows, H, x, weight, eps, out, static_cast<cudaStream_t>(stream)) == cudaSuccess ? SDLM_OK
+                                                                                                             : SDLM_ERR_CUDA;
+}
+
+extern "C" sdlm_status sdlm_linear_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t K, int32_t N, const void* x, const void* w,
+                                           const void* bias, const void* residual, void* out, const void* norm_weight,
+                                           float eps, void* norm_out, void* stream) {
+  if (!ctx || !x || !w || !out || !norm_weight || !norm_out || rows < 1 || K < 8 || N < 16 || !(eps >= 0.f))
+    return SDLM_ERR_INVALID_ARG;
+  if (!a16(x) || !a16(w) || !a16(out) || !a16(norm_weight) || !a16(norm_out) || (bias && !a16(bias)) ||
+      (residual && !a16(residual)))
+    return SDLM_ERR_INVALID_ARG;
+  if (K % 8 || N % 16) return SDLM_ERR_UNSUPPORTED;
+  const LinNorm norm{norm_weight, eps, norm_out};
+  return launch_linear(ctx, rows, K, N, x, w, bias, residual, out, static_cast<cudaStream_t>(stream), 0, 0, nullptr, nullptr,
+                       0, &norm);
 }
 
 static sdlm_status rope_launch(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, int n_heads, void* x, int n_heads2,

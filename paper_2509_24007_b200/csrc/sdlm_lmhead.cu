@@ -808,6 +808,83 @@ __global__ void __launch_bounds__(256) linear_reduce_kernel(const float* part, i
   }
 }
 
+// The same sums for a product whose rows are normalised next: one thread block per row adds the K ranges,
+// bias and residual, rounds and stores the row, and writes RMSNorm(row) * weight beside it.  The sums, the
+// rounding and the order of the squares are those of linear_reduce_kernel followed by the row-wise norm
+// kernel, so the two ways give the same bits.  N / 8 <= 128 * kNormChunks.
+constexpr int kNormChunks = 4;
+__global__ void __launch_bounds__(128) linear_reduce_norm_kernel(const float* part, int ksplit, int N,
+                                                                 const __nv_bfloat16* bias,
+                                                                 const __nv_bfloat16* residual, __nv_bfloat16* out,
+                                                                 const __nv_bfloat16* norm_w, float eps,
+                                                                 __nv_bfloat16* norm_out) {
+  __shared__ float s_part[4];
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
+  const size_t row = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, nc = N / 8;
+  uint4 hv[kNormChunks];
+  float ss = 0.f;
+#pragma unroll
+  for (int k = 0; k < kNormChunks; ++k) {
+    const int c = tid + 128 * k;
+    if (c < nc) {
+      float z[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      for (int sp = 0; sp < ksplit; ++sp) {
+        const float4* src = reinterpret_cast<const float4*>(part + ((size_t)sp * 128 + row) * N) + 2 * c;
+        const float4 a = __ldcg(src), b = __ldcg(src + 1);
+        z[0] += a.x; z[1] += a.y; z[2] += a.z; z[3] += a.w;
+        z[4] += b.x; z[5] += b.y; z[6] += b.z; z[7] += b.w;
+      }
+      if (bias) {
+        const uint4 v = *(reinterpret_cast<const uint4*>(bias) + c);
+        const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) z[i] += __bfloat162float(e[i]);
+      }
+      if (residual) {
+        const uint4 v = *(reinterpret_cast<const uint4*>(residual + row * N) + c);
+        const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) z[i] += __bfloat162float(e[i]);
+      }
+      uint4 o;
+      o.x = ptx::pack_bf16(z[0], z[1]); o.y = ptx::pack_bf16(z[2], z[3]);
+      o.z = ptx::pack_bf16(z[4], z[5]); o.w = ptx::pack_bf16(z[6], z[7]);
+      *(reinterpret_cast<uint4*>(out + row * N) + c) = o;
+      hv[k] = o;
+      const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&o);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float f = __bfloat162float(e[i]);
+        ss = fmaf(f, f, ss);
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if (lane == 0) s_part[tid >> 5] = ss;
+  __syncthreads();
+  ss = (s_part[0] + s_part[1]) + (s_part[2] + s_part[3]);
+  const float inv = rsqrtf(ss / (float)N + eps);
+#pragma unroll
+  for (int k = 0; k < kNormChunks; ++k) {
+    const int c = tid + 128 * k;
+    if (c < nc) {
+      const uint4 w = *(reinterpret_cast<const uint4*>(norm_w) + c);
+      const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&hv[k]);
+      const __nv_bfloat16* g = reinterpret_cast<const __nv_bfloat16*>(&w);
+      uint4 o;
+      uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        ow[i] = ptx::pack_bf16(__bfloat162float(e[2 * i]) * inv * __bfloat162float(g[2 * i]),
+                               __bfloat162float(e[2 * i + 1]) * inv * __bfloat162float(g[2 * i + 1]));
+      *(reinterpret_cast<uint4*>(norm_out + row * N) + c) = o;
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // merge of the per-stripe partials: one warp per row, fixed order
 // ---------------------------------------------------------------------------------------------
@@ -993,7 +1070,7 @@ static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden,
 // out[rows, N] = x[rows, K] W[N, K]^T (+ residual), bf16 in and out, fp32 accumulation; row blocks of 128.
 sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, const void* w, const void* bias,
                           const void* residual, void* out, cudaStream_t st, int seg1, int seg2, void* out2, void* out3,
-                          int act) {
+                          int act, const LinNorm* norm) {
   for (int r0 = 0; r0 < rows; r0 += 128) {
     const int nr = rows - r0 < 128 ? rows - r0 : 128;
     LmParams p{};
@@ -1077,6 +1154,14 @@ sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, 
                                        tm_x, tm_w, p, n_stages);
     ctx->launches++;
     if (le != cudaSuccess || cudaGetLastError() != cudaSuccess) return SDLM_ERR_CUDA;
+    __nv_bfloat16* norm_out = norm ? static_cast<__nv_bfloat16*>(norm->out) + (size_t)r0 * N : nullptr;
+    if (p.ksplit > 1 && norm && N / 8 <= 128 * kNormChunks) {
+      le = launch_overlapped(linear_reduce_norm_kernel, dim3(nr), dim3(128), 0, st, (const float*)p.part, p.ksplit, N,
+                             p.bias, p.residual, p.out, static_cast<const __nv_bfloat16*>(norm->weight), norm->eps, norm_out);
+      ctx->launches++;
+      if (le != cudaSuccess || cudaGetLastError() != cudaSuccess) return SDLM_ERR_CUDA;
+      continue;
+    }
     if (p.ksplit > 1) {
       const size_t total = (size_t)nr * (N / 8);
       const int blocks = (int)((total + 255) / 256);
@@ -1085,6 +1170,7 @@ sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, 
       ctx->launches++;
       if (le != cudaSuccess || cudaGetLastError() != cudaSuccess) return SDLM_ERR_CUDA;
     }
+    if (norm && launch_rmsnorm(ctx, nr, N, p.out, norm->weight, norm->eps, norm_out, st) != cudaSuccess) return SDLM_ERR_CUDA;
   }
   return SDLM_OK;
 }

@@ -221,17 +221,17 @@ class DecoderStack:
         """h0 [B, D, H]: the block's input embeddings.  out.attn is not used (attention is per layer)."""
         wl, s = self.wl, self.wl.shape
         self.h.copy_(h0.reshape(self.h.shape))
+        self.ctx[0].rmsnorm(self.h, self.layers[0].ln1, self.EPS, self.x, stream=stream)
         for l, (sd, w) in enumerate(zip(self.ctx, self.layers)):
-            sd.rmsnorm(self.h, w.ln1, self.EPS, self.x, stream=stream)
             sd.linear3(self.x, self.wqkv[l], self.bqkv[l], self.q, self.k[l], self.v[l], stream=stream)
             sd.rope_block2(self.q, self.k[l], self.THETA, stream=stream)
             sd.block_attn(self.q, self.k[l], self.v[l], self.attn, stream=stream)
-            sd.linear(self.attn, w.wo, None, self.h, self.h, stream=stream)
-            sd.rmsnorm(self.h, w.ln2, self.EPS, self.x, stream=stream)
+            # the residual stream is updated in place and its norm for the next product comes with it
+            sd.linear_rmsnorm(self.attn, w.wo, w.ln2, self.EPS, None, self.h, self.h, self.x, stream=stream)
             sd.linear_swiglu(self.x, self.wgu_il[l], self.act, stream=stream)
-            sd.linear(self.act, w.wdown, None, self.h, self.h, stream=stream)
+            nxt = self.layers[l + 1].ln1 if l + 1 < self.L else self.ln_f
+            sd.linear_rmsnorm(self.act, w.wdown, nxt, self.EPS, None, self.h, self.h, self.x, stream=stream)
         sd0 = self.ctx[0]
-        sd0.rmsnorm(self.h, self.ln_f, self.EPS, self.x, stream=stream)
         sd0.lmhead_confidence(self.x, self.w_lm, out.token, out.p_top1, out.entropy, stream=stream)
         accept_commit_layers(self.ctx, tau, out.token, out.p_top1, out.entropy, self.k, self.v, out.accepted_len,
                              out.out_tokens, stream=stream)

@@ -97,6 +97,37 @@ def test_linear_in_place_on_the_residual_stream():
     _check_bf16(_f64(r), lo.linear(x64, w64, None, r64), "linear in place")
 
 
+@pytest.mark.parametrize("rows,K,N", [(128, 2048, 2048), (128, 11008, 2048), (37, 2048, 2048), (200, 4096, 4096),
+                                      (128, 2048, 4112), (9, 72, 48), (128, 256, 1024)])
+@pytest.mark.parametrize("extras", ["plain", "both", "in place"])
+def test_product_with_the_norm_of_its_rows_equals_the_two_calls(rows, K, N, extras):
+    """sdlm_linear_rmsnorm against sdlm_linear followed by sdlm_rmsnorm, bit for bit (products that are cut
+    along K, where the sum of the ranges and the norm share a kernel, and products that are not), and
+    against the oracle's two functions."""
+    dp = _ctx()
+    rng = np.random.default_rng(rows + K + N + 1)
+    _, x64, x = _bf16(rng, (rows, K))
+    _, w64, w = _bf16(rng, (N, K), std=K ** -0.5)
+    _, b64, b = _bf16(rng, (N,))
+    _, r64, r = _bf16(rng, (rows, N))
+    _, g64, g = _bf16(rng, (N,))
+    eps = 1e-6
+    use = extras != "plain"
+    ref_out = dp.sd.linear(x, w, b if use else None, r if use else None)
+    ref_norm = dp.sd.rmsnorm(ref_out, g, eps)
+    if extras == "in place":
+        res = r.clone()
+        out, norm = dp.sd.linear_rmsnorm(x, w, g, eps, b, res, out=res)
+    else:
+        out, norm = dp.sd.linear_rmsnorm(x, w, g, eps, b if use else None, r if use else None)
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+    assert torch.equal(out, ref_out) and torch.equal(norm, ref_norm)
+    o64 = lo.linear(x64, w64, b64 if use else None, r64 if use else None)
+    _check_bf16(_f64(out), o64, "linear")
+    _check_bf16(_f64(norm), lo.rms_norm(_f64(out), g64, eps), "norm of the stored rows")
+
+
 @pytest.mark.parametrize("rows,H", [(1, 8), (7, 256), (128, 2048), (130, 5120), (3, 1000)])
 def test_rmsnorm_matches_the_oracle(rows, H):
     dp = _ctx()
