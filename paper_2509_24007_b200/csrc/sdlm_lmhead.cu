@@ -284,16 +284,38 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  if (!p.wait_at_end) ptx::grid_dep_wait();  // the hidden states may come from the kernel before this one
+  // The rows of x (and the residual, and the partial sums' buffer) may belong to the kernel before this
+  // one; the weights do not.  In a chain of products with small kernels between them, the producer
+  // therefore sends for the first ring of weight tiles before it waits, and for their x tiles after.
+  if (LINEAR ? warp != 0 : !p.wait_at_end) ptx::grid_dep_wait();
 
   if (warp == 0) {
     if (lane == 0) {  // ---- TMA producer
       uint32_t it = 0;
       bool ok = true;
       const uint64_t w_policy = ptx::l2_evict_first_policy();  // W is read once per call
+      uint32_t pre = 0;
+      if constexpr (LINEAR) {
+        const uint32_t total = (uint32_t)n_tiles * (uint32_t)KC;
+        pre = KC > 0 ? min(total, (uint32_t)n_stages) : 0u;
+        for (uint32_t j = 0; j < pre; ++j) {
+          const int t = (int)j / KC, kc = (int)j % KC;
+          ptx::mbar_arrive_expect_tx(&full[j], (uint32_t)(R * p.a_box_rows * kBK * 2 + w_tile_bytes));
+          ptx::tma_load_2d_hint(smem + (size_t)j * stage_bytes + R * kATileBytes, &tmap_w, (kc0 + kc) * kBK,
+                                n_begin + t * p.bn, &full[j], w_policy);
+        }
+        ptx::grid_dep_wait();
+        for (uint32_t j = 0; j < pre; ++j) {
+          const int kc = (int)j % KC;
+#pragma unroll
+          for (int r = 0; r < R; ++r)
+            ptx::tma_load_2d(smem + (size_t)j * stage_bytes + r * kATileBytes, &tmap_h, (kc0 + kc) * kBK, r * 128, &full[j]);
+        }
+      }
       for (int t = 0; t < n_tiles && ok; ++t) {
         const int n0 = n_begin + t * p.bn;
         for (int kc = 0; kc < KC; ++kc, ++it) {
+          if (it < pre) continue;  // sent for above
           const int s = it % n_stages;
           if (it >= (uint32_t)n_stages && !ptx::mbar_wait(&empty[s], ((it / n_stages) & 1) ^ 1, abort)) {
             ok = false;
