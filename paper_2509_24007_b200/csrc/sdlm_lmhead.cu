@@ -786,6 +786,35 @@ __global__ void __launch_bounds__(kMmaThreads) lmhead_mma_kernel(const LmParams 
   }
 }
 
+// Eight adjacent output columns of one row: the K ranges' partial sums in range order, then bias, then
+// residual, rounded to bf16 once.
+__device__ __forceinline__ uint4 reduce_chunk(const float* part, int ksplit, size_t row, int N, int c,
+                                              const __nv_bfloat16* bias, const __nv_bfloat16* residual) {
+  float z[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  for (int s = 0; s < ksplit; ++s) {
+    const float4* src = reinterpret_cast<const float4*>(part + ((size_t)s * 128 + row) * N) + 2 * c;
+    const float4 a = __ldcg(src), b = __ldcg(src + 1);
+    z[0] += a.x; z[1] += a.y; z[2] += a.z; z[3] += a.w;
+    z[4] += b.x; z[5] += b.y; z[6] += b.z; z[7] += b.w;
+  }
+  if (bias) {
+    const uint4 v = *(reinterpret_cast<const uint4*>(bias) + c);
+    const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) z[i] += __bfloat162float(e[i]);
+  }
+  if (residual) {
+    const uint4 v = *(reinterpret_cast<const uint4*>(residual + row * N) + c);
+    const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) z[i] += __bfloat162float(e[i]);
+  }
+  uint4 o;
+  o.x = ptx::pack_bf16(z[0], z[1]); o.y = ptx::pack_bf16(z[2], z[3]);
+  o.z = ptx::pack_bf16(z[4], z[5]); o.w = ptx::pack_bf16(z[6], z[7]);
+  return o;
+}
+
 // ---------------------------------------------------------------------------------------------
 // split-K linear: out = bf16(sum_s part[s] + bias + residual), splits added in index order
 // ---------------------------------------------------------------------------------------------
@@ -799,28 +828,7 @@ __global__ void __launch_bounds__(256) linear_reduce_kernel(const float* part, i
   for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
     const int c = (int)(idx % (N / 8));
     const size_t row = idx / (N / 8);
-    float z[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    for (int s = 0; s < ksplit; ++s) {
-      const float4* src = reinterpret_cast<const float4*>(part + ((size_t)s * 128 + row) * N) + 2 * c;
-      const float4 a = __ldcg(src), b = __ldcg(src + 1);
-      z[0] += a.x; z[1] += a.y; z[2] += a.z; z[3] += a.w;
-      z[4] += b.x; z[5] += b.y; z[6] += b.z; z[7] += b.w;
-    }
-    if (bias) {
-      const uint4 v = *(reinterpret_cast<const uint4*>(bias) + c);
-      const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) z[i] += __bfloat162float(e[i]);
-    }
-    if (residual) {
-      const uint4 v = *(reinterpret_cast<const uint4*>(residual + row * N) + c);
-      const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) z[i] += __bfloat162float(e[i]);
-    }
-    uint4 o;
-    o.x = ptx::pack_bf16(z[0], z[1]); o.y = ptx::pack_bf16(z[2], z[3]);
-    o.z = ptx::pack_bf16(z[4], z[5]); o.w = ptx::pack_bf16(z[6], z[7]);
+    const uint4 o = reduce_chunk(part, ksplit, row, N, c, bias, residual);
     const int n = c * 8;  // segments are multiples of 16 columns: eight columns never straddle one
     __nv_bfloat16* dst = seg1 == 0   ? out + row * N + n
                          : n < seg1 ? out + row * seg1 + n
@@ -851,28 +859,7 @@ __global__ void __launch_bounds__(128) linear_reduce_norm_kernel(const float* pa
   for (int k = 0; k < kNormChunks; ++k) {
     const int c = tid + 128 * k;
     if (c < nc) {
-      float z[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-      for (int sp = 0; sp < ksplit; ++sp) {
-        const float4* src = reinterpret_cast<const float4*>(part + ((size_t)sp * 128 + row) * N) + 2 * c;
-        const float4 a = __ldcg(src), b = __ldcg(src + 1);
-        z[0] += a.x; z[1] += a.y; z[2] += a.z; z[3] += a.w;
-        z[4] += b.x; z[5] += b.y; z[6] += b.z; z[7] += b.w;
-      }
-      if (bias) {
-        const uint4 v = *(reinterpret_cast<const uint4*>(bias) + c);
-        const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) z[i] += __bfloat162float(e[i]);
-      }
-      if (residual) {
-        const uint4 v = *(reinterpret_cast<const uint4*>(residual + row * N) + c);
-        const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) z[i] += __bfloat162float(e[i]);
-      }
-      uint4 o;
-      o.x = ptx::pack_bf16(z[0], z[1]); o.y = ptx::pack_bf16(z[2], z[3]);
-      o.z = ptx::pack_bf16(z[4], z[5]); o.w = ptx::pack_bf16(z[6], z[7]);
+      const uint4 o = reduce_chunk(part, ksplit, row, N, c, bias, residual);
       *(reinterpret_cast<uint4*>(out + row * N) + c) = o;
       hv[k] = o;
       const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&o);
