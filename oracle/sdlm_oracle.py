@@ -51,6 +51,10 @@ the literal mask A_uv over [history ; carry ; block]; attention under them equal
 that mask; a loop of such steps leaves in the cache exactly the real tokens' rows whatever gamma was.
 parallel_training_mask / noise_block_attention (Sec. 3.3 parallel training): the mask has the three parts
 of Fig. 2a and reduces to the single-block A_uv; the noise-block rows equal dense attention under it.
+training_forward_attention (the whole forward attention under that mask, dense): target rows equal
+token-by-token causal softmax in plain loops and ignore the noise blocks; noise rows equal
+noise_block_attention; with Hq = Hkv the whole equals torch's fp64 scaled_dot_product_attention under
+the boolean mask; chunks of target rows equal block_attention_masked with triangular words.
 """
 from __future__ import annotations
 
