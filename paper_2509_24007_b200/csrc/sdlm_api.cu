@@ -861,8 +861,12 @@ static sdlm_status decode_step_device(sdlm_ctx* ctx, int32_t batch, int32_t D, c
     return SDLM_ERR_CUDA;
   if (!hidden || !w_lm || !token || !p_top1 || !entropy) return SDLM_ERR_INVALID_ARG;
   if (!aligned16(hidden) || !aligned16(w_lm)) return SDLM_ERR_INVALID_ARG;
+  // Attention writes none of the LM head's inputs, so the LM head never waits for it before it starts:
+  // side by side it runs from the beginning, in order its thread blocks stream weights from the moment
+  // attention's leave their SMs, not from the moment the slowest of them is done.  (In order, attention
+  // lets it go only after its own wait, so whatever was enqueued before the step is complete by then.)
   s = launch_lmhead(ctx, batch * D, hidden, w_lm, token, p_top1, entropy, nullptr, nullptr,
-                    static_cast<cudaStream_t>(stream), /*independent_of_predecessor=*/a_sms > 0,
+                    static_cast<cudaStream_t>(stream), /*independent_of_predecessor=*/true,
                     a_sms > 0 ? ctx->sm_count - a_sms : 0);
   if (s != SDLM_OK) return s;
   return accept_commit_launch(ctx, batch, D, seq_ids, tau, mode, token, p_top1, entropy, k_blk, v_blk, accepted_len,
@@ -967,10 +971,11 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
       cudaSuccess)
     return SDLM_ERR_CUDA;
   if (a_sms > 0 && cudaEventRecord(ctx->ev_join, qkv_st) != cudaSuccess) return SDLM_ERR_CUDA;
-  // on one stream the LM head follows attention, which lets it go at once when the two run side by side;
-  // on two streams it follows the copy of `hidden` and takes its wait as a full dependency
+  // on one stream the LM head follows attention and does not wait for it (attention has waited for the
+  // copy of `hidden` before it lets the LM head go); on two streams it follows the copy of `hidden`
+  // and takes its wait as a full dependency
   s = launch_lmhead(ctx, batch * D, ws + L.st_hidden, w_lm, d_token, d_p, d_ent, nullptr, nullptr, st,
-                    /*independent_of_predecessor=*/a_sms == 0 && overlap > 0, overlap > 0 ? ctx->sm_count - overlap : 0);
+                    /*independent_of_predecessor=*/a_sms == 0, overlap > 0 ? ctx->sm_count - overlap : 0);
   if (s != SDLM_OK) return s;
   if (a_sms > 0 && cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return SDLM_ERR_CUDA;
   int32_t* m_acc = static_cast<int32_t*>(mapped(accepted_len_host));
