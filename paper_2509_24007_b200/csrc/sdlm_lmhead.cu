@@ -285,9 +285,11 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   // The rows of x (and the residual, and the partial sums' buffer) may belong to the kernel before this
-  // one; the weights do not.  In a chain of products with small kernels between them, the producer
-  // therefore sends for the first ring of weight tiles before it waits, and for their x tiles after.
-  if (LINEAR ? warp != 0 : !p.wait_at_end) ptx::grid_dep_wait();
+  // one; the weights do not.  Where the kernel has to wait for that kernel at all, the producer therefore
+  // sends for the first ring of weight tiles before it waits, and for their x tiles after: in a chain
+  // of calls with small kernels between them the weight stream starts while those finish.
+  const bool waits_at_start = LINEAR || !p.wait_at_end;
+  if (waits_at_start && warp != 0) ptx::grid_dep_wait();
 
   if (warp == 0) {
     if (lane == 0) {  // ---- TMA producer
@@ -295,7 +297,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
       bool ok = true;
       const uint64_t w_policy = ptx::l2_evict_first_policy();  // W is read once per call
       uint32_t pre = 0;
-      if constexpr (LINEAR) {
+      if (waits_at_start) {
         const uint32_t total = (uint32_t)n_tiles * (uint32_t)KC;
         pre = KC > 0 ? min(total, (uint32_t)n_stages) : 0u;
         for (uint32_t j = 0; j < pre; ++j) {
