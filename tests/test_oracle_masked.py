@@ -350,3 +350,25 @@ def test_training_attention_causal_rows_by_chunks_with_triangular_words():
         vis = np.array([[(1 << (j + 1)) - 1 for j in range(m)]], dtype=np.int64)
         ref = orc.block_attention_masked(q[None, u0:u0 + m], k[None, u0:u0 + m], v[None, u0:u0 + m], [k[:u0]], [v[:u0]], vis)
         assert np.allclose(out[u0:u0 + m], ref[0], rtol=0, atol=1e-13)
+
+
+def test_parallel_training_mask_against_the_hand_written_matrices():
+    """tests/golden/training_mask_worked_example.txt: 0/1 matrices typed from the figure's description."""
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "training_mask_worked_example.txt")
+    cases, cur = [], None
+    for line in open(path):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        if line.startswith("mask training"):
+            kv = dict(t.split("=") for t in line.split()[2:])
+            cur = (int(kv["n_target"]), int(kv["D"]), [int(x) for x in kv["starts"].split(",")], [])
+            cases.append(cur)
+        else:
+            cur[3].append([int(x) for x in line.split()])
+    assert len(cases) == 2
+    for n, D, starts, rows in cases:
+        want = np.array(rows, dtype=bool)
+        assert want.shape == (n + len(starts) * D,) * 2
+        assert np.array_equal(orc.parallel_training_mask(n, starts, D), want)
