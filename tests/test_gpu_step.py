@@ -347,3 +347,41 @@ def test_back_to_back_side_by_side_steps_without_host_synchronisation(name, batc
     for (k, v), b in zip(k_ref, (0, batch - 1)):
         k2, v2 = dp.sd.kv_gather(b, int(t["seq_len"][b]))
         assert torch.equal(k, k2) and torch.equal(v, v2)
+
+
+def test_in_order_step_takes_hidden_from_the_library_kernel_enqueued_just_before():
+    """In order the LM head does not wait for attention before it starts, but attention lets it go only after
+    its own wait: `hidden` may therefore be the pending output of the call enqueued just before the step
+    (here a row-wise norm, a kernel that lets its successor start early), also right behind a long kernel."""
+    wl = syn.CONFIGS["cfg2_d4"].with_(batch=6, prefix_lo=10, prefix_hi=700)
+    dp = DeviceProblem(wl)
+    sd = dp.sd
+    sd.set_option(OPT_STEP_OVERLAP, 0)
+    x = dp.block(0)
+    H = wl.shape.hidden
+    g = torch.ones(H, dtype=torch.bfloat16, device="cuda")
+    raw = (x.hidden.float() * 3.0).to(torch.bfloat16)
+    hidden = sd.rmsnorm(raw, g, 1e-6)
+    torch.cuda.synchronize()
+    snap = sd.kv_export()
+    ref = dp.alloc_outputs()
+    sd.decode_step(wl.tau, x.q, x.k_blk, x.v_blk, hidden, dp.w_lm, ref.attn, ref.token, ref.p_top1, ref.entropy,
+                   ref.accepted_len, ref.out_tokens)
+    torch.cuda.synchronize()
+    big = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    pending = torch.empty_like(hidden)
+    out = dp.alloc_outputs()
+    for rep in range(8):
+        sd.kv_import(snap)
+        pending.zero_()
+        torch.cuda.synchronize()
+        big.fill_(rep)                                   # something long in front
+        sd.rmsnorm(raw, g, 1e-6, pending)                # writes `hidden` ...
+        sd.decode_step(wl.tau, x.q, x.k_blk, x.v_blk, pending, dp.w_lm, out.attn, out.token, out.p_top1, out.entropy,
+                       out.accepted_len, out.out_tokens)  # ... which the step reads
+        torch.cuda.synchronize()
+        assert sd.device_status()[0] == 0
+        assert torch.equal(pending, hidden)
+        assert torch.equal(out.token, ref.token) and torch.equal(out.p_top1, ref.p_top1)
+        assert torch.equal(out.entropy, ref.entropy) and torch.equal(out.accepted_len, ref.accepted_len)
+        assert torch.equal(out.attn, ref.attn)
