@@ -352,11 +352,11 @@ def test_training_attention_causal_rows_by_chunks_with_triangular_words():
         assert np.allclose(out[u0:u0 + m], ref[0], rtol=0, atol=1e-13)
 
 
-def test_parallel_training_mask_against_the_hand_written_matrices():
+def test_masks_against_the_hand_written_matrices():
     """tests/golden/training_mask_worked_example.txt: 0/1 matrices typed from the figure's description."""
     import os
     path = os.path.join(os.path.dirname(__file__), "golden", "training_mask_worked_example.txt")
-    cases, cur = [], None
+    cases, verif, cur = [], [], None
     for line in open(path):
         line = line.strip()
         if not line or line.startswith("#"):
@@ -365,10 +365,16 @@ def test_parallel_training_mask_against_the_hand_written_matrices():
             kv = dict(t.split("=") for t in line.split()[2:])
             cur = (int(kv["n_target"]), int(kv["D"]), [int(x) for x in kv["starts"].split(",")], [])
             cases.append(cur)
+        elif line.startswith("mask verification"):
+            cur = (int(line.split("D=")[1]), None, None, [])
+            verif.append(cur)
         else:
             cur[3].append([int(x) for x in line.split()])
-    assert len(cases) == 2
+    assert len(cases) == 2 and len(verif) == 1
     for n, D, starts, rows in cases:
         want = np.array(rows, dtype=bool)
         assert want.shape == (n + len(starts) * D,) * 2
         assert np.array_equal(orc.parallel_training_mask(n, starts, D), want)
+    for D, _, _, rows in verif:
+        words = [sum(bit << t for t, bit in enumerate(r)) for r in rows]
+        assert np.array_equal(orc.verification_visibility(D), np.array(words, dtype=np.int64))
