@@ -793,11 +793,23 @@ __global__ void __launch_bounds__(kMmaThreads) lmhead_mma_kernel(const LmParams 
 __device__ __forceinline__ uint4 reduce_chunk(const float* part, int ksplit, size_t row, int N, int c,
                                               const __nv_bfloat16* bias, const __nv_bfloat16* residual) {
   float z[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-  for (int s = 0; s < ksplit; ++s) {
-    const float4* src = reinterpret_cast<const float4*>(part + ((size_t)s * 128 + row) * N) + 2 * c;
-    const float4 a = __ldcg(src), b = __ldcg(src + 1);
-    z[0] += a.x; z[1] += a.y; z[2] += a.z; z[3] += a.w;
-    z[4] += b.x; z[5] += b.y; z[6] += b.z; z[7] += b.w;
+  for (int s0 = 0; s0 < ksplit; s0 += 4) {  // four ranges' loads in flight; added in range order
+    float4 a[4], b[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (s0 + u < ksplit) {
+        const float4* src = reinterpret_cast<const float4*>(part + ((size_t)(s0 + u) * 128 + row) * N) + 2 * c;
+        a[u] = __ldcg(src);
+        b[u] = __ldcg(src + 1);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (s0 + u < ksplit) {
+        z[0] += a[u].x; z[1] += a[u].y; z[2] += a[u].z; z[3] += a[u].w;
+        z[4] += b[u].x; z[5] += b[u].y; z[6] += b[u].z; z[7] += b[u].w;
+      }
+    }
   }
   if (bias) {
     const uint4 v = *(reinterpret_cast<const uint4*>(bias) + c);
