@@ -4,9 +4,15 @@
 
 A step is one pass of the whole hot path over one batch of synthetic block inputs.  The default
 workload is the batch-32, D=4, Qwen2.5-3B-shaped ragged step; the metric is committed tokens per
-second.  One JSON line is printed by rank 0.  With N > 1 (torchrun) every rank runs an independent
-replica of the workload on its own GPU (the path shards by sequence; there is no collective in the
-data path), so scaling is "weak" and `value` sums the tokens of all ranks over the slowest rank's time.
+second of the step run IN ORDER (attention, then the LM head, then acceptance and commit, each on all
+SMs: the order a model needs, whose LM head reads the last layer's output).  The region of exactly
+`--steps` steps is timed repeatedly until at least half a second has been timed; `ms_per_step` is the
+median over those regions.  The side-by-side mode of the library (attention beside the LM head, only
+valid for two independent micro-batches) is reported in a field of its own.  One JSON line is printed
+by rank 0.  With N > 1 every rank runs an independent replica of the workload on its own GPU (the path
+shards by sequence; there is no collective in the data path), so scaling is "weak" and `value` sums the
+tokens of all ranks over the slowest rank's time; `python bench.py --gpus N` without torchrun starts the
+N ranks itself.
 """
 from __future__ import annotations
 
@@ -30,11 +36,12 @@ METRIC, UNIT = "committed_tokens_per_s", "tokens/s"
 
 
 def _peaks():
+    """(HBM GB/s, sustained bf16 TFLOP/s, where they come from)."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         d = json.load(open(path))
-        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
-    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+        return float(d["hbm_gbs"]), float(d.get("bf16_tflops_sustained", 1400.0)), "measured (MEASURED_PEAKS.json)"
+    return 6650.0, 1400.0, "fallback (6.65 TB/s and 1.4 PFLOP/s sustained, earlier measurements on this pool)"
 
 
 class ClockSampler:
@@ -164,19 +171,29 @@ LMHEAD_NCU_TRAFFIC = 634216704   # bytes per launch of lmhead_umma_kernel<1> at 
 RESTORE_EVERY = 8   # steps between restores of the cache tables, so that prefix lengths stay the workload's
 
 
-def time_workload(torch, dp, wl, steps, warmup, n_blocks=4, use_graph=True, overlap=True):
-    """Device-timed region of `steps` whole steps (one sdlm_decode_step call each, nothing else on the
-    stream but a table restore every RESTORE_EVERY steps).  Before it, un-timed: warm-up steps, the
-    three calls timed one by one (attention and the LM-head call bracketed by events: the latter is the
-    dominant kernel's launch duration for the roofline), and the choice of how many SMs attention gets
-    when the step runs attention and the LM head side by side."""
+MIN_TIMED_S = 0.5     # the region of `steps` steps is repeated until this much has been timed
+MAX_REGIONS = 2000
+
+
+def time_workload(torch, dp, wl, steps, warmup, n_blocks=4, use_graph=True, overlap=True, min_timed_s=MIN_TIMED_S,
+                  reduce_max=None, barrier=None, sampler=None):
+    """Device-timed regions of exactly `steps` whole steps (one sdlm_decode_step call each, nothing else on
+    the stream but a table restore every RESTORE_EVERY steps), repeated until min_timed_s has been timed.
+    First the step in order (attention, LM head, commit, each on all SMs): that is the primary figure.  Then,
+    un-timed, the three calls one by one (attention and the LM-head call bracketed by events: the latter is
+    the dominant kernel's launch duration for the roofline) and, with `overlap`, the library's side-by-side
+    mode (attention on A SMs beside the LM head), A chosen by a short sweep, timed the same way.
+    reduce_max / barrier: the whole-job maximum of a per-rank time and the barrier between ranks (None on
+    one GPU); sampler: started around the in-order regions only."""
     from paper_2509_24007_b200.binding import OPT_STEP_OVERLAP
     blocks = [dp.block(i) for i in range(n_blocks)]
     out = dp.alloc_outputs()
     stream = torch.cuda.current_stream()
     sd = dp.sd
-    acc_buf = torch.zeros((steps, wl.batch), dtype=torch.int32, device=sd.device)   # gamma of every timed step
+    acc_buf = torch.zeros((max(steps, 1), wl.batch), dtype=torch.int32, device=sd.device)   # gamma of every step of a region
     saved = sd.kv_save()
+    reduce_max = reduce_max or (lambda x: x)
+    barrier = barrier or torch.cuda.synchronize
 
     def one_step(x, acc, st=None):
         sd.decode_step(wl.tau, x.q, x.k_blk, x.v_blk, x.hidden, dp.w_lm, out.attn, out.token, out.p_top1, out.entropy,
@@ -211,82 +228,107 @@ def time_workload(torch, dp, wl, steps, warmup, n_blocks=4, use_graph=True, over
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) / n
 
+    def regions(a_sms, min_s, clock_sampler=None):
+        """Timed regions of `steps` steps in the launch mode a_sms (0: in order); returns their figures."""
+        sd.set_option(OPT_STEP_OVERLAP, a_sms)
+        run(max(warmup, RESTORE_EVERY), 0)
+        torch.cuda.synchronize()
+        graph, per_graph, acc_g = None, 0, None
+        if use_graph and steps >= RESTORE_EVERY:
+            # RESTORE_EVERY steps (with their table restore) captured once and replayed: the library never
+            # synchronises with the host, so the whole loop can live in a CUDA graph
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            graph = torch.cuda.CUDAGraph()
+            acc_g = torch.zeros((RESTORE_EVERY, wl.batch), dtype=torch.int32, device=sd.device)
+            with torch.cuda.stream(side):
+                n0 = sd.launch_count()
+                with torch.cuda.graph(graph, stream=side):
+                    sd.kv_restore(saved, stream=side)
+                    for i in range(RESTORE_EVERY):
+                        one_step(blocks[(warmup + i) % n_blocks], acc_g[i], side)
+                per_graph = sd.launch_count() - n0
+            stream.wait_stream(side)
+            for _ in range(2):
+                graph.replay()
+            torch.cuda.synchronize()
+        replays = steps // RESTORE_EVERY if graph is not None else 0
+        rest = steps - replays * RESTORE_EVERY
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        times, tokens, launches, total = [], 0, 0, 0.0
+        if clock_sampler is not None:
+            clock_sampler.start()
+        while total < min_s * 1e3 and len(times) < MAX_REGIONS:
+            barrier()
+            launches0 = sd.launch_count()
+            ev0.record(stream)
+            for _ in range(replays):
+                graph.replay()
+            run(rest, warmup, acc_buf)
+            ev1.record(stream)
+            torch.cuda.synchronize()
+            ms = reduce_max(ev0.elapsed_time(ev1))
+            if not times:      # every region commits the same tokens: the inputs and the restores repeat
+                launches = sd.launch_count() - launches0 + replays * per_graph
+                tokens = int(acc_buf[:rest].clamp(min=0).sum().item())
+                if graph is not None:
+                    tokens += replays * int(acc_g.clamp(min=0).sum().item())
+            times.append(ms)
+            total += ms
+        clocks = clock_sampler.stop() if clock_sampler is not None else None
+        # the sticky status is read before anything else touches the context
+        assert int(sd.device_status()[0]) == 0, "device status set during the timed region"
+        sd.kv_restore(saved)
+        torch.cuda.synchronize()
+        t = np.asarray(times)
+        return {"ms_total": float(np.median(t)), "ms_per_step": float(np.median(t)) / steps, "regions": len(times),
+                "ms_timed": float(t.sum()), "spread": [float(t.min()) / steps, float(t.max()) / steps],
+                "tokens": tokens, "launches": launches, "graph": graph is not None, "clocks": clocks}
+
+    # ---- primary: the step in order
     sd.set_option(OPT_STEP_OVERLAP, 0)
     run(warmup, 0)
-    # per-call device times, each call on all SMs
+    res = regions(0, min_timed_s, sampler)
+    # ---- per-call device times, each call on all SMs
     n2 = min(max(steps, 8), 200)
     mk = lambda: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n2)]
     lm_ev, at_ev = mk(), mk()
     run_three_calls(n2, warmup, lm_ev, at_ev)
     torch.cuda.synchronize()
-    lm_ms = float(np.mean([a.elapsed_time(b) for a, b in lm_ev]))
-    at_ms = float(np.mean([a.elapsed_time(b) for a, b in at_ev]))
-    # side by side: attention's share of the SMs starts from its share of the two calls' SM-time and
-    # is settled by timing a few neighbours (and the in-order step) on RESTORE_EVERY * 3 steps each
-    a_sms, sweep = 0, {}
+    assert int(sd.device_status()[0]) == 0, "device status set during the three-call steps"
+    res["lm_ms"] = float(np.mean([a.elapsed_time(b) for a, b in lm_ev]))
+    res["attn_ms"] = float(np.mean([a.elapsed_time(b) for a, b in at_ev]))
+    # ---- side by side: attention's share of the SMs starts from its share of the two calls' SM-time and
+    # is settled by timing a few neighbours on RESTORE_EVERY * 3 steps each
+    res["side_by_side"] = None
     if overlap:
+        sweep = {}
         sms = torch.cuda.get_device_properties(sd.device).multi_processor_count
-        a0 = 2 * int(round(sms * at_ms / (at_ms + lm_ms) / 2))   # even: with more than 128 rows both kernels take whole SM pairs
+        a0 = 2 * int(round(sms * res["attn_ms"] / (res["attn_ms"] + res["lm_ms"]) / 2))   # even: with more than 128 rows both kernels take whole SM pairs
         def try_sms(a):
-            if a not in sweep and (a == 0 or 1 <= a < sms):
+            if a not in sweep and 1 <= a < sms:
                 sd.set_option(OPT_STEP_OVERLAP, a)
                 run(RESTORE_EVERY, warmup)
                 sweep[a] = min(timed(RESTORE_EVERY * 3, warmup) for _ in range(2))
-        for a in [0] + [a0 + d for d in (-8, -6, -4, -2, 0, 2, 4, 6, 8)]:
+        for a in [a0 + d for d in (-8, -4, 0, 4, 8)]:
             try_sms(a)
         for _ in range(4):   # the best at an end of the range tried: look further that way
-            split = {a: t for a, t in sweep.items() if a > 0}
-            best = min(split, key=split.get)
-            if best == min(split):
-                for d in (2, 4, 6): try_sms(best - d)
-            elif best == max(split):
-                for d in (2, 4, 6): try_sms(best + d)
+            best = min(sweep, key=sweep.get)
+            if best == min(sweep):
+                for d in (4, 8): try_sms(best - d)
+            elif best == max(sweep):
+                for d in (4, 8): try_sms(best + d)
             else:
                 break
+        for d in (-2, 2):
+            try_sms(min(sweep, key=sweep.get) + d)
         a_sms = min(sweep, key=sweep.get)
-    sd.set_option(OPT_STEP_OVERLAP, a_sms)
-    run(max(warmup, RESTORE_EVERY), 0)
-    torch.cuda.synchronize()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    graph, per_graph = None, 0
-    if use_graph and steps >= RESTORE_EVERY:
-        # RESTORE_EVERY steps (with their table restore) captured once and replayed: the library never
-        # synchronises with the host, so the whole loop can live in a CUDA graph
-        side = torch.cuda.Stream()
-        side.wait_stream(stream)
-        graph = torch.cuda.CUDAGraph()
-        acc_g = torch.zeros((RESTORE_EVERY, wl.batch), dtype=torch.int32, device=sd.device)
-        with torch.cuda.stream(side):
-            n0 = sd.launch_count()
-            with torch.cuda.graph(graph, stream=side):
-                sd.kv_restore(saved, stream=side)
-                for i in range(RESTORE_EVERY):
-                    one_step(blocks[(warmup + i) % n_blocks], acc_g[i], side)
-            per_graph = sd.launch_count() - n0
-        stream.wait_stream(side)
-        for _ in range(2):
-            graph.replay()
-        torch.cuda.synchronize()
-    launches0 = sd.launch_count()
-    replays = steps // RESTORE_EVERY if graph is not None else 0
-    rest = steps - replays * RESTORE_EVERY
-    ev0.record(stream)
-    for _ in range(replays):
-        graph.replay()
-    run(rest, warmup, acc_buf)
-    ev1.record(stream)
-    torch.cuda.synchronize()
-    launches = sd.launch_count() - launches0 + replays * per_graph
-    ms = ev0.elapsed_time(ev1)
-    tokens = int(acc_buf[:rest].clamp(min=0).sum().item())
-    if graph is not None:
-        tokens += replays * int(acc_g.clamp(min=0).sum().item())
-    sd.kv_restore(saved)
-    torch.cuda.synchronize()
-    assert int(sd.device_status()[0]) == 0, "device status set during the timed region"
-    return {"ms_total": ms, "ms_per_step": ms / steps, "tokens": tokens, "lm_ms": lm_ms,
-            "attn_ms": at_ms, "launches": launches, "graph": graph is not None, "attn_sms": a_sms,
-            "sweep_us": {str(k): round(v * 1e3, 1) for k, v in sorted(sweep.items())}}
+        side = regions(a_sms, min_timed_s / 2)
+        side["attn_sms"] = a_sms
+        side["sweep_us"] = {str(k): round(v * 1e3, 1) for k, v in sorted(sweep.items())}
+        res["side_by_side"] = side
+        sd.set_option(OPT_STEP_OVERLAP, 0)
+    return res
 
 
 def time_speculative(torch, dp, wl, steps, warmup, n_blocks=4, p_agree=0.8):
@@ -328,13 +370,12 @@ def time_speculative(torch, dp, wl, steps, warmup, n_blocks=4, p_agree=0.8):
 
 def time_carry(torch, pk, DeviceProblem, wl, steps, warmup, n_blocks=4):
     """Steps whose block is preceded by up to D-1 carry rows of real tokens (Sec. 3.3 causal rows):
-    masked attention over c_max + D rows / block keys, LM head on the D block positions, Eq. 7, commit
-    of the real-token rows only.  Three library calls per step.  The carry lengths are those a first
-    step's acceptance gives and are held fixed, so that every timed step does the same work."""
-    from paper_2509_24007_b200.harness import carry_mask
+    attention over c_max + D rows / block keys (visibility built in the kernel from the carry lengths on
+    the device), LM head on the D block positions, Eq. 7, commit of the real-token rows only, and the next
+    step's carry lengths written on the device.  Three library calls per step, no host round trip."""
     D, c_max = wl.block, wl.block - 1
     R = c_max + D
-    dp = DeviceProblem(wl, keep_prefix=False, max_block=R)
+    dp = DeviceProblem(wl.with_(steps=2 * (RESTORE_EVERY + 2)), keep_prefix=False, max_block=min(8, R))
     sd = dp.sd
     wide = wl.with_(block=R)
     rows = [syn.block_inputs(wide, dp.w_bits, 300 + i) for i in range(n_blocks)]
@@ -343,13 +384,9 @@ def time_carry(torch, pk, DeviceProblem, wl, steps, warmup, n_blocks=4):
     out = dp.alloc_outputs()
     attn = torch.empty((wl.batch, R, wl.shape.n_q_heads, wl.shape.head_dim), dtype=torch.bfloat16, device=sd.device)
     saved = sd.kv_save()
-    first = dp.step(dp.block(0), wl.tau)                      # a plain step: its gamma - 1 are the carry lengths
-    torch.cuda.synchronize()
-    carry_host = (first.accepted_len.cpu().numpy() - 1).clip(0, c_max).astype(np.int32)
-    carry = torch.from_numpy(carry_host).to(sd.device)
-    vis = torch.from_numpy(carry_mask(carry_host, c_max, D).view(np.int32)).to(sd.device)
-    sd.kv_restore(saved)
+    carry = torch.zeros(wl.batch, dtype=torch.int32, device=sd.device)
     acc = torch.zeros((steps, wl.batch), dtype=torch.int32, device=sd.device)
+    appended = torch.zeros((), dtype=torch.int64, device=sd.device)
     stream = torch.cuda.current_stream()
 
     def run(n, first_i, keep):
@@ -357,13 +394,16 @@ def time_carry(torch, pk, DeviceProblem, wl, steps, warmup, n_blocks=4):
             if i % RESTORE_EVERY == 0:
                 sd.kv_restore(saved)
             q, k, v, hidden = blocks[(first_i + i) % n_blocks]
-            sd.block_attn_masked(q, k, v, vis, attn)
+            if keep:
+                appended.add_(carry.sum() + wl.batch)
+            sd.block_attn_carry(q, k, v, carry, c_max, attn)
             sd.lmhead_confidence(hidden, dp.w_lm, out.token, out.p_top1, out.entropy)
             sd.accept_commit_carry(wl.tau, carry, c_max, out.token, out.p_top1, out.entropy, k, v, 0,
-                                   acc[i] if keep else out.accepted_len, out.out_tokens)
+                                   acc[i] if keep else out.accepted_len, out.out_tokens, next_carry_len=carry)
 
     run(warmup, 0, False)
     torch.cuda.synchronize()
+    n0 = sd.launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     run(steps, warmup, True)
@@ -371,10 +411,13 @@ def time_carry(torch, pk, DeviceProblem, wl, steps, warmup, n_blocks=4):
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
     assert int(sd.device_status()[0]) == 0, "device status set during the carry steps"
-    tokens = int(acc.clamp(min=0).sum().item())
+    # a token is committed once its K/V are cached: the carry rows and position 0 of every step
+    tokens = int(appended.item())
     return {"value": tokens / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / steps, "tokens_per_step": tokens / steps,
-            "rows_appended_per_step": int(carry_host.sum()) + wl.batch, "query_positions": R,
-            "what": "block preceded by gamma_prev - 1 carry rows of real tokens; only real-token K/V are cached"}
+            "accepted_per_step": int(acc.clamp(min=0).sum().item()) / steps, "query_positions": R,
+            "launches_per_step": (sd.launch_count() - n0) / steps,
+            "what": "block preceded by gamma_prev - 1 carry rows of real tokens, carry lengths kept on the device; "
+                    "only real-token K/V are cached (tokens counted when their K/V enter the cache)"}
 
 
 def time_model_level(torch, pk, wl, lengths, n_layers, intermediate, steps, warmup=2):
@@ -542,16 +585,63 @@ def aggregate_over_ranks(dist, torch, ms_total, tokens, e2e_value, device):
     return float(t.item()), int(n.item()), float(e.item())
 
 
+def _roofline(wl, lengths, lm_ms, attn_ms, peak_hbm, peak_tf, peak_src, traffic=None):
+    """Roofline objects of one workload's two kernels.  The LM head with up to 128 rows streams the weight
+    once and is bound by HBM; with 129..256 rows (the CTA-pair kernel) its 2 * rows * H * V flops take longer
+    than its bytes at the measured rates, so it is reported against the sustained bf16 tensor rate."""
+    s = wl.shape
+    lm_bytes = syn.lm_head_bytes(wl) + wl.rows * s.hidden * 2           # weight once + hidden rows once
+    kv_bytes = syn.kv_read_bytes(wl, lengths)
+    lm_gbs = lm_bytes / (lm_ms * 1e-3) / 1e9
+    attn = {"bound": "hbm", "kernel": "block_attn_umma_kernel (sdlm_block_attn)", "achieved": kv_bytes / (attn_ms * 1e-3) / 1e9,
+            "peak": peak_hbm, "unit": "GB/s", "frac": kv_bytes / (attn_ms * 1e-3) / 1e9 / peak_hbm,
+            "algorithmic_bytes": kv_bytes, "launch_ms": attn_ms}
+    timing = ("CUDA events around the call on its stream (the call alone on all SMs), mean over the same steps run as "
+              "three calls")
+    if wl.rows > 128:
+        flops = 2.0 * wl.rows * s.hidden * s.vocab
+        tf = flops / (lm_ms * 1e-3) / 1e12
+        lm = {"bound": "tensor", "kernel": "lmhead_pair_kernel (sdlm_lmhead_confidence: CTA-pair stripe kernel + merge of the stripes)",
+              "timing": timing, "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": tf / peak_tf,
+              "peak_source": peak_src + ", bf16_tflops_sustained", "traffic": None, "algorithmic_flops": flops,
+              "algorithmic_bytes": lm_bytes, "hbm_gbs": lm_gbs, "hbm_frac": lm_gbs / peak_hbm, "launch_ms": lm_ms}
+    else:
+        lm = {"bound": "hbm", "kernel": "lmhead_umma_kernel (sdlm_lmhead_confidence: stripe kernel + merge of the stripes)",
+              "timing": timing, "achieved": lm_gbs, "peak": peak_hbm, "unit": "GB/s", "frac": lm_gbs / peak_hbm,
+              "peak_source": peak_src, "traffic": traffic,
+              "traffic_source": ("dram__bytes_read.sum + dram__bytes_write.sum of one launch, "
+                                 "profiles/lmhead_umma_and_block_attn_umma__cfg2_d4.md") if traffic else None,
+              "algorithmic_bytes": lm_bytes, "launch_ms": lm_ms}
+    step_bytes = lm_bytes + kv_bytes + 2 * wl.rows * s.n_q_heads * s.head_dim * 2
+    return lm, attn, step_bytes
+
+
+def _spawn_ranks(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start the N ranks with torch.distributed.run."""
+    import socket
+    import torch
+    have = torch.cuda.device_count() if torch.cuda.is_available() else 0
+    if have < n:
+        sys.stderr.write(f"bench.py --gpus {n}: {have} CUDA device(s) visible; every rank needs a GPU of its own\n")
+        return 2
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg2_d4", choices=syn.workloads())
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="enqueue every step from the host instead of replaying a CUDA graph")
-    ap.add_argument("--no-overlap", action="store_true", help="attention, then the LM head, each on all SMs (no side-by-side step)")
-    ap.add_argument("--no-extra", action="store_true", help="skip the D=8 companion measurement and the CPU baseline")
+    ap.add_argument("--no-overlap", action="store_true", help="skip the side-by-side mode (the primary figure is the in-order step either way)")
+    ap.add_argument("--no-extra", action="store_true", help="skip the other workloads, the widening measurements and the CPU baseline")
     ap.add_argument("--model-level-only", action="store_true",
                     help="run only the whole-model step of the 3B shape and print its figures (for profiling)")
     args = ap.parse_args()
@@ -560,6 +650,12 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     wl = syn.CONFIGS[args.workload]
+    if args.gpus < 1:
+        raise SystemExit("--gpus must be at least 1")
+    if args.gpus > 1 and world == 1 and args.impl == "native":
+        raise SystemExit(_spawn_ranks(args.gpus))
+    if world > 1 and world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but the launcher started {world} ranks")
     if args.impl == "reference":
         run_reference(args, wl)
         return
@@ -587,85 +683,113 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local_rank)
+    def reduce_max(x):
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
     barrier()
-    if rank == 0:
-        sampler.start()
-    res = time_workload(torch, dp, wl_run, args.steps, args.warmup, use_graph=not args.no_graph, overlap=not args.no_overlap)
+    res = time_workload(torch, dp, wl_run, args.steps, args.warmup, use_graph=not args.no_graph, overlap=not args.no_overlap,
+                        reduce_max=reduce_max, barrier=barrier, sampler=sampler)
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
     e2e = time_e2e(torch, dp, wl_run, max(3, min(args.steps, 100)), 3)
-    ms_total, tokens, e2e["value"] = aggregate_over_ranks(dist, torch, res["ms_total"], res["tokens"], e2e["value"], "cuda")
+    side = res["side_by_side"]
+    _, tokens, e2e["value"] = aggregate_over_ranks(dist, torch, res["ms_total"], res["tokens"], e2e["value"], "cuda")
+    side_tokens = aggregate_over_ranks(dist, torch, 0.0, side["tokens"], 0.0, "cuda")[1] if side else 0
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
-    peak, peak_src = _peaks()
-    s = wl.shape
-    lm_bytes = syn.lm_head_bytes(wl) + wl.rows * s.hidden * 2           # weight once + hidden rows once
-    kv_bytes = syn.kv_read_bytes(wl, lengths)
-    step_bytes = lm_bytes + kv_bytes + 2 * wl.rows * s.n_q_heads * s.head_dim * 2
-    lm_gbs = lm_bytes / (res["lm_ms"] * 1e-3) / 1e9
+    peak, peak_tf, peak_src = _peaks()
+    lm_roof, attn_roof, step_bytes = _roofline(wl, lengths, res["lm_ms"], res["attn_ms"], peak, peak_tf, peak_src,
+                                               LMHEAD_NCU_TRAFFIC if wl.name == "cfg2_3b_b32_d4" else None)
+    ms_step = res["ms_per_step"]            # whole-job: every region's time is the slowest rank's
+    gbs = step_bytes / (ms_step * 1e-3) / 1e9
     line = {
-        "metric": METRIC, "value": tokens / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "metric": METRIC, "value": tokens / (res["ms_total"] * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "ms_per_step_spread": res["spread"],
+        "timed_regions": res["regions"], "ms_timed": res["ms_timed"],
+        "timing": (f"the region of {args.steps} steps timed {res['regions']} times with CUDA events ({res['ms_timed']:.0f} ms in all); "
+                   "ms_per_step is the median region's, ms_per_step_spread the fastest and slowest region's"),
+        "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": _config(wl, lengths),
         "tokens_per_step": tokens / args.steps / world,
         "gpu_launches": res["launches"],
         "launch_mode": (f"CUDA graph of {RESTORE_EVERY} steps replayed" if res["graph"] else "one host call per library call"),
-        "step_mode": ({"side_by_side": True, "attention_sms": res["attn_sms"], "lm_head_sms": "the rest",
-                       "chosen": "un-timed sweep before the timed region (us/step by attention SMs; 0 = in order)",
-                       "sweep_us": res["sweep_us"]} if res["attn_sms"] else
-                      {"side_by_side": False, "sweep_us": res["sweep_us"]}),
-        "clocks": clocks,
+        "step_mode": "in order: attention, then the LM head, then acceptance and commit, each on all SMs",
+        "clocks": res["clocks"],
         "e2e": e2e,
-        "roofline": {"bound": "hbm", "kernel": "lmhead_umma_kernel (sdlm_lmhead_confidence: stripe kernel + merge of the stripes)",
-                     "timing": "CUDA events around the call on its stream (the call alone on all SMs), mean over the same steps run as three calls just before the timed region",
-                     "achieved": lm_gbs, "peak": peak, "unit": "GB/s", "frac": lm_gbs / peak,
-                     "peak_source": peak_src, "traffic": LMHEAD_NCU_TRAFFIC if wl.name == "cfg2_3b_b32_d4" else None,
-                     "traffic_source": "dram__bytes_read.sum + dram__bytes_write.sum of one launch, profiles/lmhead_umma_and_block_attn_umma__cfg2_d4.md",
-                     "algorithmic_bytes": lm_bytes,
-                     "launch_ms": res["lm_ms"]},
-        "step": {"algorithmic_bytes": step_bytes, "achieved_gbs": step_bytes / (ms_total / args.steps * 1e-3) / 1e9,
-                 "frac_of_peak": step_bytes / (ms_total / args.steps * 1e-3) / 1e9 / peak,
-                 "frac_of_8tbs": step_bytes / (ms_total / args.steps * 1e-3) / 1e9 / 8000.0,
-                 "attn_ms": res["attn_ms"], "attn_gbs": kv_bytes / (res["attn_ms"] * 1e-3) / 1e9, "lm_ms": res["lm_ms"]},
+        "roofline": lm_roof,
+        "roofline_attention": attn_roof,
+        "step": {"algorithmic_bytes": step_bytes, "in_order_ms": ms_step, "in_order_gbs": gbs,
+                 "in_order_frac_of_peak": gbs / peak, "in_order_frac_of_8tbs": gbs / 8000.0,
+                 "target": "0.70 of 8 TB/s over attention plus LM head", "target_met_in_order": bool(gbs / 8000.0 >= 0.70),
+                 "attn_ms": res["attn_ms"], "lm_ms": res["lm_ms"]},
     }
-    if not args.no_extra and world == 1:
-        if args.workload == "cfg2_d4":      # committed tokens/s is asked for at D=4 and D=8
-            wl8 = syn.CONFIGS["cfg2"].with_(steps=RESTORE_EVERY + 2)
-            del dp
-            torch.cuda.empty_cache()
-            dp8 = DeviceProblem(wl8, keep_prefix=False)
-            r8 = time_workload(torch, dp8, wl8, max(8, min(args.steps, 200)), 3, use_graph=not args.no_graph,
-                               overlap=not args.no_overlap)
-            line["extra"] = {wl8.name: {"value": r8["tokens"] / (r8["ms_total"] * 1e-3), "unit": UNIT,
-                                        "ms_per_step": r8["ms_per_step"], "lm_ms": r8["lm_ms"], "attn_ms": r8["attn_ms"],
-                                        "attention_sms": r8["attn_sms"]}}
-            del dp8
-        if args.workload == "cfg2_d4":
+    if side:
+        sgbs = step_bytes / (side["ms_per_step"] * 1e-3) / 1e9
+        line["side_by_side"] = {
+            "ms_per_step": side["ms_per_step"], "ms_per_step_spread": side["spread"], "timed_regions": side["regions"],
+            "value": side_tokens / (side["ms_total"] * 1e-3), "unit": UNIT, "attention_sms": side["attn_sms"],
+            "achieved_gbs": sgbs, "frac_of_8tbs": sgbs / 8000.0, "sweep_us": side["sweep_us"],
+            "caveat": ("attention on some SMs beside the LM head on the rest (SDLM_OPT_STEP_OVERLAP): valid only where the LM head's "
+                       "input does not depend on that attention, i.e. for two independent micro-batches; one batch of a model "
+                       "must run in order, which is what `value` times")}
+    if not args.no_extra:
+        extra = {}
+        steps_x = max(RESTORE_EVERY, min(args.steps, 200))
+        del dp
+        torch.cuda.empty_cache()
+        if args.workload == "cfg2_d4":      # the other configurations, each with its own rooflines
+            for name in ("cfg1", "cfg2", "cfg3", "cfg4"):
+                wx = syn.CONFIGS[name]
+                wx_run = wx.with_(steps=RESTORE_EVERY + 2)
+                dpx = DeviceProblem(wx_run, keep_prefix=False)
+                rx = time_workload(torch, dpx, wx_run, steps_x, 3, use_graph=not args.no_graph, overlap=not args.no_overlap,
+                                   min_timed_s=0.2)
+                lm_x, attn_x, bytes_x = _roofline(wx, dpx.lengths, rx["lm_ms"], rx["attn_ms"], peak, peak_tf, peak_src)
+                gx = bytes_x / (rx["ms_per_step"] * 1e-3) / 1e9
+                extra[wx.name] = {"value": rx["tokens"] / (rx["ms_total"] * 1e-3), "unit": UNIT, "ms_per_step": rx["ms_per_step"],
+                                  "ms_per_step_spread": rx["spread"], "timed_regions": rx["regions"], "steps": steps_x,
+                                  "tokens_per_step": rx["tokens"] / steps_x, "config": _config(wx, dpx.lengths),
+                                  "step": {"algorithmic_bytes": bytes_x, "in_order_gbs": gx, "in_order_frac_of_peak": gx / peak,
+                                           "in_order_frac_of_8tbs": gx / 8000.0},
+                                  "roofline": lm_x, "roofline_attention": attn_x}
+                if rx["side_by_side"]:
+                    sx = rx["side_by_side"]
+                    extra[wx.name]["side_by_side"] = {"ms_per_step": sx["ms_per_step"], "attention_sms": sx["attn_sms"],
+                                                      "value": sx["tokens"] / (sx["ms_total"] * 1e-3)}
+                del dpx
+                torch.cuda.empty_cache()
             dps = DeviceProblem(wl_run, keep_prefix=False)
-            line["extra"]["self_speculative_" + wl.name] = time_speculative(torch, dps, wl_run, max(8, min(args.steps, 200)), 3)
+            extra["self_speculative_" + wl.name] = time_speculative(torch, dps, wl_run, steps_x, 3)
             del dps
             torch.cuda.empty_cache()
-        if args.workload == "cfg2_d4":
-            line["extra"]["carry_over_" + wl.name] = time_carry(torch, pk, DeviceProblem, wl_run, max(8, min(args.steps, 200)), 3)
+            extra["carry_over_" + wl.name] = time_carry(torch, pk, DeviceProblem, wl_run, steps_x, 3)
             torch.cuda.empty_cache()
-        if args.workload == "cfg2_d4":      # Qwen2.5-3B: 36 layers, intermediate size 11008
-            line["extra"]["model_level_3b_" + wl.name] = time_model_level(torch, pk, wl_run, lengths, 36, 11008,
-                                                                          max(4, min(args.steps, 30)))
+            wl8 = syn.CONFIGS["cfg2"]
+            extra["carry_over_" + wl8.name] = time_carry(torch, pk, DeviceProblem, wl8.with_(seed=wl8.seed + 1000 * rank), steps_x, 3)
             torch.cuda.empty_cache()
-        if args.workload == "cfg2_d4":
-            line["extra"]["training_noise_blocks_3b"] = time_noise_blocks(torch, pk, DeviceProblem, wl.shape)
+            # Qwen2.5-3B: 36 layers, intermediate size 11008
+            extra["model_level_3b_" + wl.name] = time_model_level(torch, pk, wl_run, lengths, 36, 11008, max(4, min(args.steps, 30)))
             torch.cuda.empty_cache()
+            extra["training_noise_blocks_3b"] = time_noise_blocks(torch, pk, DeviceProblem, wl.shape)
+            torch.cuda.empty_cache()
+        line["extra"] = extra
         n_seqs = min(wl.batch, 32)
         tok, dt = oracle_sample(wl, n_seqs, repeats=2)
         line["cpu_baseline"] = {"value": tok / dt, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
                                 "sample": f"oracle decode_step on the first {n_seqs} of {wl.batch} sequences "
-                                          f"({n_seqs * wl.block} rows; best of 2 runs, {dt:.1f} s each), fp64 numpy"}
+                                          f"({n_seqs * wl.block} rows; best of 2 runs, {dt:.1f} s each), fp64 numpy; "
+                                          "timed on rank 0 only"}
     print(json.dumps(line))
+    sys.stdout.flush()
     if dist is not None:
+        dist.barrier()
         dist.destroy_process_group()
 
 

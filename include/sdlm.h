@@ -13,8 +13,9 @@
  *   (d) sdlm_kv_pages           bookkeeping of that paged cache (Fig. 2b "cached KV states").
  *
  * Around them: sdlm_decode_step / sdlm_decode_step_host (the whole step in one call),
- * sdlm_block_attn_masked, sdlm_verify_commit and sdlm_accept_commit_carry (self-speculative decoding of
- * Sec. 3.4 and blocks preceded by rows of real tokens), sdlm_block_attn_prefix and
+ * sdlm_block_attn_masked, sdlm_block_attn_verify, sdlm_verify_commit (self-speculative decoding of
+ * Sec. 3.4), sdlm_block_attn_carry and sdlm_accept_commit_carry (blocks preceded by rows of real tokens,
+ * Sec. 3.3), sdlm_block_attn_prefix and
  * sdlm_block_attn_masked_prefix (the noise-block rows and the causal rows of parallel training,
  * Sec. 3.3), sdlm_linear / sdlm_linear3 / sdlm_linear_rmsnorm / sdlm_rmsnorm / sdlm_rope_block(2) / sdlm_swiglu /
  * sdlm_accept_commit_layers (the rest of a decoder layer of the Qwen-2.5 backbone, Sec. 4.1, for
@@ -93,9 +94,9 @@ sdlm_status sdlm_create(const sdlm_config* cfg, void* kv_pool, size_t kv_pool_by
 void sdlm_destroy(sdlm_ctx* ctx);
 const char* sdlm_status_str(sdlm_status s);
 
-/* ---- (d) page bookkeeping -- the paper only says that cached KV states are reused (Fig. 2b,
- * Sec. 3.2 "predictions are repeated starting from the previous step's end position"); paging,
- * the free list and its order are this library's.
+/* ---- (d) page bookkeeping -- the paper only says that cached KV states are reused (Fig. 2b) and that
+ * the next step starts where the previous one stopped (Sec. 3.2); paging, the free list and its order
+ * are this library's.
  *
  * The cache is a pool of pages of 64 tokens shared by all sequence slots.  Pages are handed out
  * from a ring `free_list[num_pages]` at position free_head (mod num_pages); released pages are
@@ -113,11 +114,16 @@ typedef enum sdlm_kv_op {
                               DEVICE bf16 [args.length, Hkv, d]; rows at or beyond the slot's current
                               length are left untouched                                             */
   SDLM_KV_EXPORT = 5,      /* synchronise `stream`, copy all tables to HOST args.host_buf            */
-  SDLM_KV_IMPORT = 6,      /* restore tables from a HOST buffer written by EXPORT (same config)      */
+  SDLM_KV_IMPORT = 6,      /* restore tables from a HOST buffer written by EXPORT (same config); the buffer
+                              is checked on the host first (lengths within max_pages_per_seq * 64, every
+                              page a sequence or the live part of the ring refers to inside the pool and
+                              referred to once): INVALID_ARG and nothing copied otherwise                */
   SDLM_KV_SAVE = 7,        /* copy all tables to DEVICE args.dev_buf (>= table_bytes), enqueued on `stream`,
                               no host synchronisation                                                */
   SDLM_KV_RESTORE = 8      /* the reverse of SAVE: lengths, page tables and the free ring go back to the
-                              saved state (cache rows written since stay in the pool, unreferenced)   */
+                              saved state (cache rows written since stay in the pool, unreferenced).
+                              RESTORE and IMPORT leave the sticky device status as it is: a failure
+                              recorded since the SAVE / EXPORT stays visible                          */
 } sdlm_kv_op;
 
 typedef struct sdlm_kv_args {
@@ -147,7 +153,10 @@ typedef struct sdlm_kv_result {
 /* `args` may be NULL for QUERY; `result` may be NULL except for QUERY.  ADD_SEQ / RELEASE_SEQ /
  * GATHER / RESET are enqueued on `stream` (RESET copies args.free_list before returning).  A pool
  * that runs dry during ADD_SEQ sets the device status OUT_OF_PAGES and leaves the slot empty.
- * Errors: INVALID_ARG (null / slot or length out of range / short host buffer), CUDA. */
+ * RESET checks on the host that args.free_list is a permutation of 0..num_pages-1 (INVALID_ARG, nothing
+ * enqueued, otherwise).
+ * Errors: INVALID_ARG (null / slot or length out of range / short host buffer / tables or free list that
+ * fail the checks above), CUDA. */
 sdlm_status sdlm_kv_pages(sdlm_ctx* ctx, sdlm_kv_op op, const sdlm_kv_args* args, sdlm_kv_result* result,
                           void* stream);
 
@@ -192,6 +201,32 @@ sdlm_status sdlm_block_attn_prefix(sdlm_ctx* ctx, int32_t batch, int32_t D, cons
 sdlm_status sdlm_block_attn_masked(sdlm_ctx* ctx, int32_t batch, int32_t n_q, int32_t n_k, const int32_t* seq_ids,
                                    const void* q, const void* k_blk, const void* v_blk, const uint32_t* vis,
                                    void* out, void* stream);
+
+/* ---- (a') with the verification inputs' visibility built by the library -- Sec. 3.4, self-speculative
+ * decoding: verification input j of a block is the sampled tokens before position j plus one [m] at
+ * position j.  k_blk / v_blk [batch, 2D, Hkv, d] list the block's keys as D rows of real tokens
+ * [x^{i-1}, y^1 .. y^{D-1}] followed by the D rows of the [m] inputs; q, out [batch, D, Hq, d].  Query
+ * position j sees the whole cached history, the real keys t < j and the [m] key D + j (position 0 is
+ * x^{i-1} itself, whose own key is key D).  Same values as sdlm_block_attn_masked with those words.
+ * 2D <= 16.  Errors: as sdlm_block_attn_masked. */
+sdlm_status sdlm_block_attn_verify(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, const void* q,
+                                   const void* k_blk, const void* v_blk, void* out, void* stream);
+
+/* ---- (a') for a block preceded by carry rows -- Sec. 3.3: with i the block's first position,
+ * A_uv = 1[v <= u] for the rows u < i in front of the block and full attention inside it.  The tokens a
+ * step accepts beyond position 0 were predicted at [m] inputs; the next step feeds them as c = carry_len[b]
+ * rows of real tokens in front of its block.  q, out [batch, c_max + D, Hq, d]; k_rows / v_rows
+ * [batch, c_max + D, Hkv, d]: rows 0..c-1 the carry rows (rows c..c_max-1 are padding), rows c_max.. the D
+ * block positions.  carry_len: DEVICE int32 [batch], read by the kernel (values outside 0..c_max are
+ * clipped), so a decode loop needs no host round trip: sdlm_accept_commit_carry writes the next step's.
+ * Carry row r sees the history and carry keys 0..r; a padding row the history and its own key (its output
+ * is not a result); a block position the history, carry keys 0..c-1 and every block key.
+ * c_max + D <= 16 query positions, computed (Hq/Hkv) * positions <= 64 stacked rows and at most max_block
+ * positions per launch (15 positions at Hq/Hkv = 8 take two launches over the same keys).
+ * Errors: as sdlm_block_attn_masked. */
+sdlm_status sdlm_block_attn_carry(sdlm_ctx* ctx, int32_t batch, int32_t D, int32_t c_max, const int32_t* seq_ids,
+                                  const int32_t* carry_len, const void* q, const void* k_rows, const void* v_rows,
+                                  void* out, void* stream);
 
 /* ---- (a''') both at once: row b attends to the first prefix_len[b] cached tokens of slot seq_ids[b]
  * and to those of its n_k block keys that vis[b,j] names.  Sec. 3.3, parallel training, the causal
@@ -279,13 +314,16 @@ sdlm_status sdlm_verify_commit(sdlm_ctx* ctx, int32_t batch, int32_t D, const in
  * (device int32 carry_len [batch], each in 0..c_max; the rows up to c_max are padding), row c_max the
  * block's position 0 (x^{i-1}).  accepted_len / out_tokens: exactly as sdlm_accept_commit (Eq. 7 over
  * the D block positions); the cache grows by the carry_len[b] + 1 real rows, appended as single
- * tokens in order.  accepted_len[b] - 1 is the next step's carry_len[b].  c_max + D <= 16.
+ * tokens in order.  next_carry_len (DEVICE int32 [batch], or NULL) receives the next step's carry
+ * lengths, min(accepted_len[b] - 1, c_max), 0 for a sequence that failed; it may be the same array as
+ * carry_len (it is written after every thread block has read this step's lengths).  c_max + D <= 16.
  * Errors and device-side checks: as sdlm_accept_commit; a carry_len outside 0..c_max is reported as
  * SDLM_ERR_DEVICE_CHECK and that sequence is left unchanged. */
 sdlm_status sdlm_accept_commit_carry(sdlm_ctx* ctx, int32_t batch, int32_t D, int32_t c_max, const int32_t* seq_ids,
                                      const int32_t* carry_len, float tau, sdlm_conf_mode mode, const int32_t* token,
                                      const float* p_top1, const float* entropy, const void* k_rows,
-                                     const void* v_rows, int32_t* accepted_len, int32_t* out_tokens, void* stream);
+                                     const void* v_rows, int32_t* accepted_len, int32_t* out_tokens,
+                                     int32_t* next_carry_len, void* stream);
 
 /* ---- (c) for several caches at once: the layers of a model each keep their own context (KV pool and
  * tables), and all commit the same accepted lengths, so their tables move in lockstep.  One launch
@@ -301,7 +339,9 @@ sdlm_status sdlm_accept_commit_layers(sdlm_ctx* const* ctxs, int32_t n_layers, i
 
 /* Synchronises `stream` and copies the sticky device status words to host_out[4]:
  * {sdlm_status (0 = none), sequence slot of the first failure, detail, number of failures}.
- * `clear` != 0 resets them afterwards. */
+ * `clear` != 0 resets them afterwards, together with the kernels' arrival counters and tickets (which a
+ * kernel that gave up on a bounded wait may have left half counted): after SDLM_ERR_TIMEOUT, read the
+ * status with `clear` set before the context is used again. */
 sdlm_status sdlm_device_status(sdlm_ctx* ctx, int32_t* host_out, int32_t clear, void* stream);
 
 /* ---- whole step on device memory: (a) + (b) + (c) in one call, same arguments and results as the

@@ -14,7 +14,10 @@ Pins (tests/test_oracle_layer.py): linear against torch.matmul in fp64 and on id
 rms_norm against torch.nn.functional.rms_norm, on constant rows and under rescaling of the input;
 rope as multiplication by e^{i a} of the complex pairs, norm preservation, position 0 = identity,
 and the relative-position property <rope(q, m), rope(k, n)> = f(m - n); swiglu against torch's
-silu, at 0 and for large |gate|.
+silu, at 0 and for large |gate|; block_attention_values against sdlm_oracle.block_attention on
+bf16-representable inputs; decoder_stack_hidden (the composition, float64 throughout, nothing rounded
+between operations) against a layer written a second time from torch's float64 routines and on the
+special cases listed in its docstring.
 """
 from __future__ import annotations
 
@@ -72,34 +75,60 @@ def to_bits(x: np.ndarray) -> np.ndarray:
     return (((u + 0x7FFF + ((u >> 16) & 1)) >> 16) & 0xFFFF).astype(np.uint16)
 
 
+def block_attention_values(q: np.ndarray, k_blk: np.ndarray, v_blk: np.ndarray, prefix_k, prefix_v) -> np.ndarray:
+    """The single-block attention of Sec. 3.3 (rows u >= i: all cached tokens and all D block positions are
+    visible) on float64 values: q [B, D, Hq, d], k_blk / v_blk [B, D, Hkv, d], prefix_k[b] / prefix_v[b]
+    [P_b, Hkv, d].  out[b, j, h] = softmax_t(q[b, j, h] . K_t / sqrt(d)) V_t over t in [history ; block],
+    query head h reading KV head h // (Hq / Hkv).  The same definition as sdlm_oracle.block_attention,
+    which takes bf16 bit patterns; a layer's q / k / v are products in float64 and are not rounded here."""
+    B, D, Hq, d = q.shape
+    Hkv = k_blk.shape[2]
+    G = Hq // Hkv
+    out = np.zeros((B, D, Hq, d))
+    for b in range(B):
+        for hk in range(Hkv):
+            keys = np.concatenate([prefix_k[b][:, hk, :], k_blk[b, :, hk, :]], axis=0)
+            vals = np.concatenate([prefix_v[b][:, hk, :], v_blk[b, :, hk, :]], axis=0)
+            for h in range(hk * G, (hk + 1) * G):
+                for j in range(D):
+                    s = (keys @ q[b, j, h]) / np.sqrt(d)
+                    w = np.exp(s - np.max(s))
+                    out[b, j, h] = (w @ vals) / np.sum(w)
+    return out
+
+
 def decoder_stack_hidden(h0: np.ndarray, layers, caches, seq_ids, n_q_heads: int, n_kv_heads: int, head_dim: int,
                          eps: float, theta: float):
     """The residual stream of one whole-model block step, [B, D, H] -> [B*D, H], through pre-norm decoder
-    layers: h += Wo attn(rope(Wq x + bq), rope(Wk x + bk), Wv x + bv | that layer's cache), x = rms_norm(h);
-    h += Wdown swiglu(Wgu rms_norm(h)).  `layers` is a list of dicts of float64 arrays (ln1, wq, bq, wk,
-    bk, wv, bv, wo, ln2, wgu, wdown); `caches` one PagedKVCache per layer.  Every operation's result is
-    rounded to bf16, as each is a tensor of that type between two library calls.  Returns the final
-    stream (float64 of bf16 values) and the per-layer K / V rows of the block as bf16 bits
-    [B, D, Hkv, d] (what a commit appends).  The composition has no published worked example to pin it
-    to: "parity unpinned" as a whole; every part is pinned on its own."""
-    from .sdlm_oracle import block_attention
+    layers of the Qwen-2.5 kind (Sec. 4.1 names the backbone; the layer is its textbook definition):
+        x = rms_norm(h, ln1);  q, k, v = Wq x + bq, Wk x + bk, Wv x + bv;  q, k = rope(q), rope(k) at the
+        positions (cached length of the sequence) + j;  h = h + Wo attention(q, k, v | that layer's cache);
+        h = h + Wdown swiglu(Wgu rms_norm(h, ln2)).
+    Everything is float64 from the inputs on: no intermediate is rounded (the cached history is bf16 by
+    definition and is widened exactly).  `layers` is a list of dicts of float64 arrays (ln1, wq, bq, wk, bk,
+    wv, bv, wo, ln2, wgu, wdown); `caches` one PagedKVCache per layer.  Returns the final stream and the
+    per-layer K / V rows of the block, float64 [B, D, Hkv, d].
+    Pins (tests/test_oracle_layer.py): one layer written a second time from torch's float64 rms_norm /
+    linear / silu / scaled_dot_product_attention and a complex-number rotary embedding; identity
+    projections with a zero MLP reduce a layer to h + attention(rope(x), rope(x), x); a zero output
+    projection and a zero down projection leave the stream unchanged; two layers are one layer applied
+    twice."""
+    from .sdlm_oracle import widen
     B, D, H = h0.shape
     rows = B * D
-    h = round_bf16(h0.reshape(rows, H))
+    h = np.asarray(h0, dtype=np.float64).reshape(rows, H)
     k_rows, v_rows = [], []
     for w, cache in zip(layers, caches):
-        x = round_bf16(rms_norm(h, w["ln1"], eps))
-        q = round_bf16(linear(x, w["wq"], w["bq"])).reshape(B, D, n_q_heads, head_dim)
-        k = round_bf16(linear(x, w["wk"], w["bk"])).reshape(B, D, n_kv_heads, head_dim)
-        v = round_bf16(linear(x, w["wv"], w["bv"])).reshape(B, D, n_kv_heads, head_dim)
+        x = rms_norm(h, w["ln1"], eps)
+        q = linear(x, w["wq"], w["bq"]).reshape(B, D, n_q_heads, head_dim)
+        k = linear(x, w["wk"], w["bk"]).reshape(B, D, n_kv_heads, head_dim)
+        v = linear(x, w["wv"], w["bv"]).reshape(B, D, n_kv_heads, head_dim)
         pos = np.array([int(cache.seq_len[int(s)]) for s in seq_ids])[:, None] + np.arange(D)[None, :]
-        q, k = round_bf16(rope(q, pos, theta)), round_bf16(rope(k, pos, theta))
-        pk, pv = zip(*[cache.gather_fast(int(s)) for s in seq_ids])
-        attn = round_bf16(block_attention(to_bits(q), to_bits(k), to_bits(v), pk, pv))
-        h = round_bf16(linear(attn.reshape(rows, n_q_heads * head_dim), w["wo"], None, h))
-        x = round_bf16(rms_norm(h, w["ln2"], eps))
-        act = round_bf16(swiglu(linear(x, w["wgu"])))      # one call: the gate / up product is not stored
-        h = round_bf16(linear(act, w["wdown"], None, h))
-        k_rows.append(to_bits(k))
-        v_rows.append(to_bits(v))
+        q, k = rope(q, pos, theta), rope(k, pos, theta)
+        hist = [cache.gather_fast(int(s)) for s in seq_ids]
+        attn = block_attention_values(q, k, v, [widen(a) for a, _ in hist], [widen(b) for _, b in hist])
+        h = linear(attn.reshape(rows, n_q_heads * head_dim), w["wo"], None, h)
+        h = linear(swiglu(linear(rms_norm(h, w["ln2"], eps), w["wgu"])), w["wdown"], None, h)
+        k_rows.append(k)
+        v_rows.append(v)
     return h, k_rows, v_rows

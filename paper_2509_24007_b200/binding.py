@@ -33,6 +33,7 @@ EXPORTED = ["sdlm_pool_bytes", "sdlm_workspace_bytes", "sdlm_create", "sdlm_dest
             "sdlm_kv_pages", "sdlm_block_attn", "sdlm_lmhead_confidence", "sdlm_lmhead_confidence_static", "sdlm_accept_commit",
             "sdlm_device_status", "sdlm_decode_step", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count",
             "sdlm_block_attn_masked", "sdlm_verify_commit", "sdlm_accept_commit_carry",
+            "sdlm_block_attn_verify", "sdlm_block_attn_carry",
             "sdlm_linear", "sdlm_linear3", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu", "sdlm_selftest_bounded_wait", "sdlm_rope_block2", "sdlm_accept_commit_layers", "sdlm_block_attn_prefix", "sdlm_linear_swiglu",
             "sdlm_block_attn_masked_prefix", "sdlm_linear_rmsnorm"]
 
@@ -135,7 +136,11 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdlm_block_attn_masked_prefix.restype = C.c_int
     lib.sdlm_block_attn_masked_prefix.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_accept_commit_carry.restype = C.c_int
-    lib.sdlm_accept_commit_carry.argtypes = [vp, i32, i32, i32, vp, vp, f32, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_accept_commit_carry.argtypes = [vp, i32, i32, i32, vp, vp, f32, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_block_attn_verify.restype = C.c_int
+    lib.sdlm_block_attn_verify.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_block_attn_carry.restype = C.c_int
+    lib.sdlm_block_attn_carry.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_linear_rmsnorm.restype = C.c_int
     lib.sdlm_linear_rmsnorm.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, f32, vp, vp]
     lib.sdlm_linear.restype = C.c_int
@@ -312,6 +317,16 @@ class Sdlm:
         self.kv_pages(KV_EXPORT, host_buf=buf)
         return buf
 
+    def copy_pool_from(self, other: "Sdlm", stream=None) -> None:
+        """Raw copy of another context's KV pool (same configuration) into this one's, for resuming from
+        exported tables."""
+        if other.pool_bytes != self.pool_bytes:
+            raise ValueError("pools differ in size")
+        a = (self._pool.data_ptr() + 1023) // 1024 * 1024 - self._pool.data_ptr()
+        b = (other._pool.data_ptr() + 1023) // 1024 * 1024 - other._pool.data_ptr()
+        with torch.cuda.stream(stream or torch.cuda.current_stream()):
+            self._pool[a:a + self.pool_bytes].copy_(other._pool[b:b + other.pool_bytes])
+
     def kv_save(self, dev_buf: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
         """Device-side snapshot of the tables (no host synchronisation); returns the buffer."""
         if dev_buf is None:
@@ -370,6 +385,42 @@ class Sdlm:
             _ptr(_dev(out, torch.bfloat16, "out")), _stream_ptr(stream)))
         return out
 
+    def block_attn_verify(self, q: torch.Tensor, k_blk: torch.Tensor, v_blk: torch.Tensor,
+                          out: Optional[torch.Tensor] = None, seq_ids: Optional[torch.Tensor] = None,
+                          stream=None) -> torch.Tensor:
+        """sdlm_block_attn_verify: q [batch, D, Hq, d], k_blk / v_blk [batch, 2D, Hkv, d] (real tokens, then masks)."""
+        batch, D = int(q.shape[0]), int(q.shape[1])
+        _dev(q, torch.bfloat16, "q"); _dev(k_blk, torch.bfloat16, "k_blk"); _dev(v_blk, torch.bfloat16, "v_blk")
+        if int(k_blk.shape[1]) != 2 * D or int(v_blk.shape[1]) != 2 * D:
+            raise ValueError("k_blk / v_blk must hold 2D rows per sequence")
+        if out is None:
+            out = torch.empty_like(q)
+        if seq_ids is not None:
+            _dev(seq_ids, torch.int32, "seq_ids")
+        self._check("sdlm_block_attn_verify", self.lib.sdlm_block_attn_verify(
+            self.ctx, batch, D, _ptr(seq_ids), _ptr(q), _ptr(k_blk), _ptr(v_blk),
+            _ptr(_dev(out, torch.bfloat16, "out")), _stream_ptr(stream)))
+        return out
+
+    def block_attn_carry(self, q: torch.Tensor, k_rows: torch.Tensor, v_rows: torch.Tensor, carry_len: torch.Tensor,
+                         c_max: int, out: Optional[torch.Tensor] = None, seq_ids: Optional[torch.Tensor] = None,
+                         stream=None) -> torch.Tensor:
+        """sdlm_block_attn_carry: q [batch, c_max + D, Hq, d], k_rows / v_rows [batch, c_max + D, Hkv, d],
+        carry_len [batch] int32 on the device."""
+        batch, R = int(q.shape[0]), int(q.shape[1])
+        _dev(q, torch.bfloat16, "q"); _dev(k_rows, torch.bfloat16, "k_rows"); _dev(v_rows, torch.bfloat16, "v_rows")
+        _dev(carry_len, torch.int32, "carry_len")
+        if int(k_rows.shape[1]) != R or int(v_rows.shape[1]) != R or carry_len.numel() != batch or not 0 <= c_max < R:
+            raise ValueError("q, k_rows, v_rows must hold c_max + D rows per sequence and carry_len one entry each")
+        if out is None:
+            out = torch.empty_like(q)
+        if seq_ids is not None:
+            _dev(seq_ids, torch.int32, "seq_ids")
+        self._check("sdlm_block_attn_carry", self.lib.sdlm_block_attn_carry(
+            self.ctx, batch, R - int(c_max), int(c_max), _ptr(seq_ids), _ptr(carry_len), _ptr(q), _ptr(k_rows),
+            _ptr(v_rows), _ptr(_dev(out, torch.bfloat16, "out")), _stream_ptr(stream)))
+        return out
+
     def block_attn_masked_prefix(self, q: torch.Tensor, k_blk: torch.Tensor, v_blk: torch.Tensor, vis: torch.Tensor,
                                  seq_ids: torch.Tensor, prefix_len: torch.Tensor,
                                  out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
@@ -410,8 +461,9 @@ class Sdlm:
                             p_top1: torch.Tensor, entropy: torch.Tensor, k_rows: torch.Tensor, v_rows: torch.Tensor,
                             mode: int = CONF_LOGIT, accepted_len: Optional[torch.Tensor] = None,
                             out_tokens: Optional[torch.Tensor] = None, seq_ids: Optional[torch.Tensor] = None,
-                            stream=None):
-        """sdlm_accept_commit_carry: k_rows / v_rows are [batch, c_max + D, Hkv, d]."""
+                            next_carry_len: Optional[torch.Tensor] = None, stream=None):
+        """sdlm_accept_commit_carry: k_rows / v_rows are [batch, c_max + D, Hkv, d]; next_carry_len (int32
+        [batch] on the device, may be carry_len itself) receives the next step's carry lengths."""
         batch, D = int(token.shape[0]), int(token.shape[1])
         _dev(carry_len, torch.int32, "carry_len"); _dev(token, torch.int32, "token")
         _dev(p_top1, torch.float32, "p_top1"); _dev(entropy, torch.float32, "entropy")
@@ -428,6 +480,7 @@ class Sdlm:
             self.ctx, batch, D, int(c_max), _ptr(seq_ids), _ptr(carry_len), float(tau), int(mode), _ptr(token),
             _ptr(p_top1), _ptr(entropy), _ptr(k_rows), _ptr(v_rows),
             _ptr(_dev(accepted_len, torch.int32, "accepted_len")), _ptr(_dev(out_tokens, torch.int32, "out_tokens")),
+            _ptr(_dev(next_carry_len, torch.int32, "next_carry_len")) if next_carry_len is not None else None,
             _stream_ptr(stream)))
         return accepted_len, out_tokens
 

@@ -6,6 +6,7 @@
 #include <math.h>
 #include <new>
 #include <string.h>
+#include <vector>
 
 namespace sdlm {
 
@@ -201,6 +202,7 @@ struct CommitParams {
   // carry_len[b] of them real tokens accepted in the step before, row c_max the block's position 0.
   // Those carry_len[b] + 1 rows are appended instead of block rows 0..gamma-1; gamma is still output.
   const int32_t* carry_len;
+  int32_t* next_carry_len;  // null, or [batch]: min(gamma - 1, c_max), 0 for a row that failed; may be carry_len itself
   int c_max;
   float tau, inv_ln_vocab;
   int mode, batch, D, Hkv, d, mpps, num_pages;
@@ -232,7 +234,8 @@ constexpr int kCommitThreads = 256;
 // would give), then scatters its own row's K/V.  The tables other CTAs read (seq_len, free_head)
 // are only written by whichever CTA finishes its reads last ("last CTA done" ticket; nobody waits).
 __device__ __forceinline__ void accept_commit_body(const CommitParams& p, bool write_outputs) {
-  __shared__ int8_t s_gamma[kMaxBatch];
+  __shared__ int8_t s_gamma[kMaxBatch];  // rows the sequence grows by
+  __shared__ int8_t s_acc[kMaxBatch];    // gamma
   __shared__ int8_t s_state[kMaxBatch];  // 0 ok, 1 capacity failure, 2 out of pages
   __shared__ int s_warp[kCommitThreads / 32];
   __shared__ int s_carry, s_mine[6];     // my row: gamma, need, alloc index, len, state, rows to append
@@ -278,6 +281,7 @@ __device__ __forceinline__ void accept_commit_body(const CommitParams& p, bool w
     if (need && (uint32_t)alloc >= avail) { state = 2; }
     if (i < p.batch) {
       s_gamma[i] = (int8_t)na;   // what the sequence grows by
+      s_acc[i] = (int8_t)g;
       s_state[i] = (int8_t)state;
       if (i == b) { s_mine[0] = g; s_mine[1] = need; s_mine[2] = alloc; s_mine[3] = len; s_mine[4] = state; s_mine[5] = na; }
     }
@@ -359,6 +363,9 @@ __device__ __forceinline__ void accept_commit_body(const CommitParams& p, bool w
         const int sl = p.seq_ids ? p.seq_ids[i] : i;
         p.seq_len[sl] += s_gamma[i];
       }
+      // the next step's carry rows are the tokens accepted beyond position 0; written here, after every
+      // thread block has read this step's carry lengths, so the two arrays may be one
+      if (p.next_carry_len && write_outputs) p.next_carry_len[i] = s_state[i] == 0 ? min((int)s_acc[i] - 1, p.c_max) : 0;
     }
     if (tid == 0) {
       p.hdr->free_head = s_head + min((uint32_t)total_need, avail);
@@ -400,6 +407,10 @@ using namespace sdlm;
 // C ABI
 // ---------------------------------------------------------------------------------------------
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+// RESTORE and IMPORT write the exported region from here on: free_head, free_tail (and the two tickets,
+// zero between launches), then the tables.  The status words in front of them stay as they are.
+constexpr size_t kStateOffset = offsetof(DevHeader, free_head);
+static_assert(kStateOffset == 16, "restores keep 16-byte alignment");
 
 extern "C" size_t sdlm_pool_bytes(const sdlm_config* cfg) {
   if (!cfg || !config_valid(*cfg)) return 0;
@@ -426,9 +437,50 @@ extern "C" const char* sdlm_status_str(sdlm_status s) {
   return "unknown status";
 }
 
+// true when list[0..n) holds every page id 0..n-1 exactly once
+static bool is_permutation(const int32_t* list, int n) {
+  std::vector<bool> seen((size_t)n, false);
+  for (int i = 0; i < n; ++i) {
+    const int32_t v = list[i];
+    if (v < 0 || v >= n || seen[(size_t)v]) return false;
+    seen[(size_t)v] = true;
+  }
+  return true;
+}
+
+// Checks tables a caller hands in (IMPORT) before anything is copied: lengths within the page table's
+// reach, every page a sequence or the live part of the free ring refers to inside the pool, and no page
+// referred to twice.  `buf` has the layout EXPORT writes.
+static bool tables_valid(const sdlm_ctx* ctx, const char* buf) {
+  const sdlm_config& c = ctx->cfg;
+  const WorkspaceLayout& L = ctx->lay;
+  const DevHeader* hdr = reinterpret_cast<const DevHeader*>(buf + (L.hdr - L.hdr));
+  const int32_t* table = reinterpret_cast<const int32_t*>(buf + (L.page_table - L.hdr));
+  const int32_t* len = reinterpret_cast<const int32_t*>(buf + (L.seq_len - L.hdr));
+  const int32_t* ring = reinterpret_cast<const int32_t*>(buf + (L.free_list - L.hdr));
+  const uint32_t live = hdr->free_tail - hdr->free_head;
+  if (live > (uint32_t)c.num_pages) return false;
+  std::vector<bool> used((size_t)c.num_pages, false);
+  auto take = [&](int32_t page) {
+    if (page < 0 || page >= c.num_pages || used[(size_t)page]) return false;
+    used[(size_t)page] = true;
+    return true;
+  };
+  for (int b = 0; b < c.max_batch; ++b) {
+    if (len[b] < 0 || len[b] > c.max_pages_per_seq * kPageSize) return false;
+    const int n = (len[b] + kPageSize - 1) / kPageSize;
+    for (int i = 0; i < n; ++i)
+      if (!take(table[(size_t)b * c.max_pages_per_seq + i])) return false;
+  }
+  for (uint32_t i = 0; i < live; ++i)
+    if (!take(ring[(hdr->free_head + i) % (uint32_t)c.num_pages])) return false;
+  return true;
+}
+
 static sdlm_status reset_tables(sdlm_ctx* ctx, const int32_t* host_free_list, cudaStream_t st) {
   const sdlm_config& c = ctx->cfg;
   if (host_free_list) {
+    if (!is_permutation(host_free_list, c.num_pages)) return SDLM_ERR_INVALID_ARG;
     if (cudaMemcpyAsync(ctx->free_list, host_free_list, (size_t)c.num_pages * 4, cudaMemcpyHostToDevice, st) !=
         cudaSuccess)
       return SDLM_ERR_CUDA;
@@ -481,6 +533,8 @@ extern "C" sdlm_status sdlm_create(const sdlm_config* cfg, void* kv_pool, size_t
   ctx->attn_min_range = 8;
   ctx->tmap_w_ptr = nullptr;
   ctx->tmap_w_rows = 0;
+  ctx->tmap_h_ptr = nullptr;
+  ctx->tmap_h_rows = ctx->tmap_h_box = 0;
   if (setup_attn(ctx) != cudaSuccess || setup_lmhead(ctx) != cudaSuccess) { delete ctx; return SDLM_ERR_CUDA; }
   sdlm_status s = reset_tables(ctx, nullptr, 0);
   if (s == SDLM_OK && cudaStreamSynchronize(0) != cudaSuccess) s = SDLM_ERR_CUDA;
@@ -595,18 +649,26 @@ extern "C" sdlm_status sdlm_kv_pages(sdlm_ctx* ctx, sdlm_kv_op op, const sdlm_kv
     case SDLM_KV_SAVE:
     case SDLM_KV_RESTORE: {
       if (!a || !a->dev_buf || a->dev_bytes < table_bytes || !aligned16(a->dev_buf)) return SDLM_ERR_INVALID_ARG;
-      void* tables = ctx->ws + ctx->lay.hdr;
-      const cudaError_t e = op == SDLM_KV_SAVE
-                                ? cudaMemcpyAsync(a->dev_buf, tables, table_bytes, cudaMemcpyDeviceToDevice, st)
-                                : cudaMemcpyAsync(tables, a->dev_buf, table_bytes, cudaMemcpyDeviceToDevice, st);
+      // The sticky status words and the kernels' tickets at the head of the header are not table
+      // state: a restore starts at the ring cursors and leaves them as they are.
+      char* tables = ctx->ws + ctx->lay.hdr;
+      const cudaError_t e =
+          op == SDLM_KV_SAVE
+              ? cudaMemcpyAsync(a->dev_buf, tables, table_bytes, cudaMemcpyDeviceToDevice, st)
+              : cudaMemcpyAsync(tables + kStateOffset, static_cast<const char*>(a->dev_buf) + kStateOffset,
+                                table_bytes - kStateOffset, cudaMemcpyDeviceToDevice, st);
       if (r) r->table_bytes = table_bytes;
       return e == cudaSuccess ? SDLM_OK : SDLM_ERR_CUDA;
     }
     case SDLM_KV_IMPORT: {
       if (!a || !a->host_buf || a->host_bytes < table_bytes) return SDLM_ERR_INVALID_ARG;
+      if (!tables_valid(ctx, static_cast<const char*>(a->host_buf))) return SDLM_ERR_INVALID_ARG;
       if (cudaStreamSynchronize(st) != cudaSuccess) return SDLM_ERR_CUDA;
-      if (cudaMemcpy(ctx->ws + ctx->lay.hdr, a->host_buf, table_bytes, cudaMemcpyHostToDevice) != cudaSuccess)
+      if (cudaMemcpy(ctx->ws + ctx->lay.hdr + kStateOffset, static_cast<const char*>(a->host_buf) + kStateOffset,
+                     table_bytes - kStateOffset, cudaMemcpyHostToDevice) != cudaSuccess)
         return SDLM_ERR_CUDA;
+      // the ring cursors share a 16-byte group with two tickets, which are zero whenever no kernel runs
+      if (cudaMemset(&ctx->hdr->commit_ticket, 0, 8) != cudaSuccess) return SDLM_ERR_CUDA;
       return SDLM_OK;
     }
   }
@@ -654,7 +716,8 @@ static sdlm_status accept_commit_launch(sdlm_ctx* ctx, int32_t batch, int32_t D,
                                         const float* entropy, const void* k_blk, const void* v_blk,
                                         int32_t* accepted_len, int32_t* out_tokens, const StatCopies& copies,
                                         void* stream, const int32_t* verify_token = nullptr,
-                                        const int32_t* carry_len = nullptr, int c_max = 0) {
+                                        const int32_t* carry_len = nullptr, int c_max = 0,
+                                        int32_t* next_carry_len = nullptr) {
   if (!ctx || !token || !k_blk || !v_blk || !accepted_len || !out_tokens) return SDLM_ERR_INVALID_ARG;
   if (!verify_token && (!p_top1 || !entropy)) return SDLM_ERR_INVALID_ARG;
   if (!aligned16(k_blk) || !aligned16(v_blk)) return SDLM_ERR_INVALID_ARG;
@@ -672,6 +735,7 @@ static sdlm_status accept_commit_launch(sdlm_ctx* ctx, int32_t batch, int32_t D,
   p.token_copy = copies.token; p.p_top1_copy = copies.p_top1; p.entropy_copy = copies.entropy;
   p.verify_token = verify_token;
   p.carry_len = carry_len;
+  p.next_carry_len = next_carry_len;
   p.c_max = c_max;
   p.tau = tau;
   p.inv_ln_vocab = c.vocab > 1 ? (float)(1.0 / log((double)c.vocab)) : 0.0f;
@@ -745,11 +809,12 @@ extern "C" sdlm_status sdlm_accept_commit_carry(sdlm_ctx* ctx, int32_t batch, in
                                                 const int32_t* seq_ids, const int32_t* carry_len, float tau,
                                                 sdlm_conf_mode mode, const int32_t* token, const float* p_top1,
                                                 const float* entropy, const void* k_rows, const void* v_rows,
-                                                int32_t* accepted_len, int32_t* out_tokens, void* stream) {
+                                                int32_t* accepted_len, int32_t* out_tokens, int32_t* next_carry_len,
+                                                void* stream) {
   if (!carry_len || c_max < 0) return SDLM_ERR_INVALID_ARG;
   if (c_max + D > kMaxBlockKeys) return SDLM_ERR_SHAPE;
   return accept_commit_launch(ctx, batch, D, seq_ids, tau, mode, token, p_top1, entropy, k_rows, v_rows, accepted_len,
-                              out_tokens, StatCopies{}, stream, nullptr, carry_len, c_max);
+                              out_tokens, StatCopies{}, stream, nullptr, carry_len, c_max, next_carry_len);
 }
 
 extern "C" sdlm_status sdlm_block_attn_prefix(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids,
@@ -800,6 +865,47 @@ extern "C" sdlm_status sdlm_block_attn_masked_prefix(sdlm_ctx* ctx, int32_t batc
              : SDLM_ERR_CUDA;
 }
 
+// Masked attention whose visibility words the kernel derives itself.  n_q query positions per sequence are
+// computed in as few launches as fit the (Hq/Hkv) * positions <= 64 stacked rows and max_block positions of
+// one launch, every launch over all n_k block keys.
+static sdlm_status attn_derived_mask(sdlm_ctx* ctx, int32_t batch, int32_t n_q, int32_t n_k, const int32_t* seq_ids,
+                                     const void* q, const void* k_blk, const void* v_blk, void* out, int kind,
+                                     const int32_t* carry_len, int c_max, void* stream) {
+  if (!ctx || !q || !k_blk || !v_blk || !out) return SDLM_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out)) return SDLM_ERR_INVALID_ARG;
+  if (batch < 1 || n_q < 1 || n_k < 1) return SDLM_ERR_INVALID_ARG;
+  if (batch > ctx->cfg.max_batch || n_k > kMaxBlockKeys || n_q > kMaxBlockKeys) return SDLM_ERR_SHAPE;
+  if (!(ctx->scale > 0.0f)) return SDLM_ERR_UNSUPPORTED;  // masking is by -inf scores: needs a positive scale
+  const int per_launch = ctx->cfg.max_block < kMaxQRows / ctx->group ? ctx->cfg.max_block : kMaxQRows / ctx->group;
+  if (per_launch < 1) return SDLM_ERR_SHAPE;
+  const int launches = (n_q + per_launch - 1) / per_launch, each = (n_q + launches - 1) / launches;
+  for (int first = 0; first < n_q; first += each) {
+    const AttnMask m{kind, carry_len, c_max, n_q, first};
+    const int n = n_q - first < each ? n_q - first : each;
+    if (launch_block_attn(ctx, batch, n, seq_ids, q, k_blk, v_blk, out, static_cast<cudaStream_t>(stream), 0, false, n_k,
+                          nullptr, nullptr, &m) != cudaSuccess)
+      return SDLM_ERR_CUDA;
+  }
+  return SDLM_OK;
+}
+
+extern "C" sdlm_status sdlm_block_attn_verify(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids,
+                                              const void* q, const void* k_blk, const void* v_blk, void* out,
+                                              void* stream) {
+  if (D < 1) return SDLM_ERR_INVALID_ARG;
+  if (2 * D > kMaxBlockKeys) return SDLM_ERR_SHAPE;
+  return attn_derived_mask(ctx, batch, D, 2 * D, seq_ids, q, k_blk, v_blk, out, 1, nullptr, 0, stream);
+}
+
+extern "C" sdlm_status sdlm_block_attn_carry(sdlm_ctx* ctx, int32_t batch, int32_t D, int32_t c_max,
+                                             const int32_t* seq_ids, const int32_t* carry_len, const void* q,
+                                             const void* k_rows, const void* v_rows, void* out, void* stream) {
+  if (!carry_len || D < 1 || c_max < 0) return SDLM_ERR_INVALID_ARG;
+  if (c_max + D > kMaxBlockKeys) return SDLM_ERR_SHAPE;
+  return attn_derived_mask(ctx, batch, c_max + D, c_max + D, seq_ids, q, k_rows, v_rows, out, 2, carry_len, c_max,
+                           stream);
+}
+
 // One thread block waits, with the same bounded wait every kernel of the library uses, on a barrier and
 // on a counter that nothing ever signals; each wait gives up after its limit (about 0.2 s), the kernel
 // records SDLM_ERR_TIMEOUT in the device status and returns.  The context stays usable.
@@ -834,7 +940,15 @@ extern "C" sdlm_status sdlm_device_status(sdlm_ctx* ctx, int32_t* host_out, int3
   if (!ctx || !host_out) return SDLM_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaMemcpyAsync(host_out, ctx->hdr->status, 16, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SDLM_ERR_CUDA;
-  if (clear && cudaMemsetAsync(ctx->hdr->status, 0, 16, st) != cudaSuccess) return SDLM_ERR_CUDA;
+  if (clear) {
+    // A kernel that gave up on a bounded wait may have left its arrival counters and tickets half
+    // counted; clearing the status puts them back to zero as well, so the next call starts clean.
+    const sdlm_config& c = ctx->cfg;
+    if (cudaMemsetAsync(ctx->hdr->status, 0, 16, st) != cudaSuccess ||
+        cudaMemsetAsync(&ctx->hdr->commit_ticket, 0, 8, st) != cudaSuccess ||
+        cudaMemsetAsync(ctx->ws + ctx->lay.attn_cnt, 0, (size_t)c.max_batch * c.n_kv_heads * 4, st) != cudaSuccess)
+      return SDLM_ERR_CUDA;
+  }
   if (cudaStreamSynchronize(st) != cudaSuccess) return SDLM_ERR_CUDA;
   return SDLM_OK;
 }
@@ -850,17 +964,22 @@ static sdlm_status decode_step_device(sdlm_ctx* ctx, int32_t batch, int32_t D, c
                                       const void* hidden, const void* w_lm, void* attn_out, int32_t* token,
                                       float* p_top1, float* entropy, int32_t* accepted_len, int32_t* out_tokens,
                                       const StatCopies& copies, void* stream) {
+  // every argument of the three calls is checked before the first of them is enqueued
   if (!ctx || !q || !k_blk || !v_blk || !attn_out) return SDLM_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(attn_out)) return SDLM_ERR_INVALID_ARG;
+  if (!hidden || !w_lm || !token || !p_top1 || !entropy || !accepted_len || !out_tokens) return SDLM_ERR_INVALID_ARG;
+  if (!aligned16(hidden) || !aligned16(w_lm)) return SDLM_ERR_INVALID_ARG;
+  if (mode != SDLM_CONF_LOGIT && mode != SDLM_CONF_ENTROPY) return SDLM_ERR_INVALID_ARG;
+  if (!isfinite(tau)) return SDLM_ERR_INVALID_ARG;
   sdlm_status s = check_batch(ctx, batch, D);
+  if (s != SDLM_OK) return s;
+  s = lmhead_supported(ctx, batch * D);
   if (s != SDLM_OK) return s;
   const int a_sms = ctx->overlap_lmhead;
   // with more than 128 rows the LM head runs as CTA pairs: attention then takes whole pairs of SMs
   if (launch_block_attn(ctx, batch, D, seq_ids, q, k_blk, v_blk, attn_out, static_cast<cudaStream_t>(stream), a_sms,
                         a_sms > 0 && batch * D > 128) != cudaSuccess)
     return SDLM_ERR_CUDA;
-  if (!hidden || !w_lm || !token || !p_top1 || !entropy) return SDLM_ERR_INVALID_ARG;
-  if (!aligned16(hidden) || !aligned16(w_lm)) return SDLM_ERR_INVALID_ARG;
   // Attention writes none of the LM head's inputs, so the LM head never waits for it before it starts:
   // side by side it runs from the beginning, in order its thread blocks stream weights from the moment
   // attention's leave their SMs, not from the moment the slowest of them is done.  (In order, attention
@@ -890,7 +1009,12 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
                                              int32_t* token_host, float* p_top1_host, float* entropy_host,
                                              int32_t* accepted_len_host, int32_t* out_tokens_host, void* stream) {
   if (!ctx || !q_host || !k_blk_host || !v_blk_host || !hidden_host || !w_lm) return SDLM_ERR_INVALID_ARG;
+  if (!aligned16(w_lm)) return SDLM_ERR_INVALID_ARG;
+  if (mode != SDLM_CONF_LOGIT && mode != SDLM_CONF_ENTROPY) return SDLM_ERR_INVALID_ARG;
+  if (!isfinite(tau)) return SDLM_ERR_INVALID_ARG;
   sdlm_status s = check_batch(ctx, batch, D);
+  if (s != SDLM_OK) return s;
+  s = lmhead_supported(ctx, batch * D);
   if (s != SDLM_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const sdlm_config& c = ctx->cfg;
@@ -958,7 +1082,6 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
     seq_ids = reinterpret_cast<const int32_t*>(ws + L.st_seq_ids);
   }
   if (!ok) return SDLM_ERR_CUDA;
-  if (!aligned16(w_lm)) return SDLM_ERR_INVALID_ARG;
   int32_t* d_token = reinterpret_cast<int32_t*>(ws + L.st_token);
   float* d_p = reinterpret_cast<float*>(ws + L.st_p);
   float* d_ent = reinterpret_cast<float*>(ws + L.st_ent);

@@ -55,10 +55,37 @@ struct AttnParams {
   // when query position j sees block key t.  The cached history is visible to every position.
   int Dk;
   const uint32_t* vis;
+  // Where the visibility words come from (MASKED kernels only): kVisWords = the array `vis`
+  // [batch][q_stride]; kVisVerify = the verification inputs of Sec. 3.4 (q_stride = D positions, 2D block
+  // keys: D real tokens, then D masks); kVisCarry = c_max carry rows in front of a block of
+  // q_stride - c_max positions (Sec. 3.3: causal rows of real tokens, then the bidirectional block), the
+  // number of real carry rows of sequence b read from carry_len[b].
+  int vis_kind;
+  const int32_t* carry_len;
+  int c_max;
+  // q and out hold q_stride positions per sequence; this launch computes positions q_first .. q_first + D - 1
+  // (a block of more positions than one launch stacks is computed in several launches over the same keys)
+  int q_stride, q_first;
   // null, or [batch]: row b sees only the first prefix_len[b] cached tokens of its slot (several rows may
   // name the same slot: the noise blocks of one training sequence)
   const int32_t* prefix_len;
 };
+
+enum { kVisNone = 0, kVisWords = 1, kVisVerify = 2, kVisCarry = 3 };
+
+// Visibility word of query position j (of this launch) of batch row b: bit t set when it sees block key t.
+//   verification (Sec. 3.4): position jj sees the real tokens before it and the mask at its own position;
+//   carry (Sec. 3.3, A_uv = 1[v <= u] for rows in front of the block, full attention inside it): a carry row
+//   sees the carry keys up to itself (a padding row only itself), a block position every real carry key of
+//   its sequence and every block key.
+__device__ __forceinline__ uint32_t vis_word(const AttnParams& p, int b, int j) {
+  const int jj = p.q_first + j;
+  if (p.vis_kind == kVisWords) return p.vis[(size_t)b * p.q_stride + jj];
+  if (p.vis_kind == kVisVerify) return ((1u << jj) - 1u) | (1u << (p.q_stride + jj));
+  const int c = min(max(p.carry_len[b], 0), p.c_max);
+  if (jj < p.c_max) return jj < c ? (2u << jj) - 1u : 1u << jj;
+  return ((1u << c) - 1u) | (((1u << (p.q_stride - p.c_max)) - 1u) << p.c_max);
+}
 
 // 8 warps; 12 when 64 stacked query rows need a second set of softmax warps
 constexpr int attn_threads(int nq) { return nq == 64 ? 384 : 256; }
@@ -277,7 +304,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     // with seq_ids the rows of the first `batch` slots may not be the ones used: harmless, they exist
     const size_t lim_len = ((size_t)p.batch * 4 + line - 1) / line;
     const size_t n_tab = ((size_t)p.batch * p.mpps * 4 + line - 1) / line;
-    const size_t n_q = ((size_t)p.batch * p.D * p.Hq * HD * 2 + line - 1) / line;
+    const size_t n_q = ((size_t)p.batch * p.q_stride * p.Hq * HD * 2 + line - 1) / line;
     const size_t n_kv = ((size_t)p.batch * p.Dk * p.Hkv * HD * 2 + line - 1) / line;
     const size_t total = lim_len + n_tab + n_q + 2 * n_kv;  // (the lengths too: one line, for the other thread blocks)
     for (size_t i = (size_t)blockIdx.x * blockDim.x + tid; i < total; i += (size_t)gridDim.x * blockDim.x) {
@@ -508,10 +535,10 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       const int n = it.t1 - it.t0, ng = (n + 1) / 2;
       // which of my 32 query rows see my key if it turns out to be a block key (bit q: row qb + q)
       [[maybe_unused]] uint32_t visq = 0xffffffffu;
-      if (MASKED && p.vis != nullptr && it.t1 > it.pages) {
+      if (MASKED && p.vis_kind != kVisNone && it.t1 > it.pages) {
         visq = 0;
         int j = qb / p.G, rem = qb % p.G;
-        uint32_t vj = j < p.D ? p.vis[(size_t)it.b * p.D + j] : 0u;
+        uint32_t vj = j < p.D ? vis_word(p, it.b, j) : 0u;
 #pragma unroll
         for (int q = 0; q < QV; ++q) {
           const uint32_t bit = qb + q < GD ? (kt < 32 ? (vj >> kt) & 1u : 0u) : 1u;  // padding rows: no mask
@@ -519,7 +546,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
           if (++rem == p.G) {
             rem = 0;
             ++j;
-            vj = j < p.D ? p.vis[(size_t)it.b * p.D + j] : 0u;
+            vj = j < p.D ? vis_word(p, it.b, j) : 0u;
           }
         }
       }
@@ -668,7 +695,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
 
       const int d = kg;
       // row q = j*G + g  <->  out[b, j, h*G + g, :]
-      __nv_bfloat16* out_base = p.out + ((size_t)it.b * p.D * p.Hq + it.h * p.G) * HD + d;
+      __nv_bfloat16* out_base = p.out + (((size_t)it.b * p.q_stride + p.q_first) * p.Hq + it.h * p.G) * HD + d;
       if (it.n_splits == 1) {
         if (d < HD) {
 #pragma unroll
@@ -756,7 +783,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
           if (row_thread) fbuf[mrow] = 1.0f / L;
           if (!meet()) { ok = false; break; }
           if (4 * dq < HD) {
-            __nv_bfloat16* ob = p.out + ((size_t)it.b * p.D * p.Hq + it.h * p.G) * HD + 4 * dq;
+            __nv_bfloat16* ob = p.out + (((size_t)it.b * p.q_stride + p.q_first) * p.Hq + it.h * p.G) * HD + 4 * dq;
 #pragma unroll
             for (int i = 0; i < NQ / NSW; ++i) {
               const int q = qg + NSW * i;
@@ -794,7 +821,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
         const int idx = (first + i) * 32 + lane, r = idx / (HD / 8), c = idx % (HD / 8);
         qreg[i] = make_uint4(0, 0, 0, 0);
         if (r < GD)
-          qreg[i] = __ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)x.b * p.D * p.Hq + x.h * p.G) * HD + row_off[r]) + c);
+          qreg[i] = __ldg(reinterpret_cast<const uint4*>(p.q + (((size_t)x.b * p.q_stride + p.q_first) * p.Hq + x.h * p.G) * HD + row_off[r]) + c);
       }
     };
     auto store_q = [&](int first) {
@@ -939,7 +966,8 @@ cudaError_t setup_attn(sdlm_ctx* ctx) {
 
 cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, const void* q,
                               const void* k_blk, const void* v_blk, void* out, cudaStream_t st, int cta_cap,
-                              bool whole_tpcs, int n_blk_keys, const uint32_t* vis, const int32_t* prefix_len) {
+                              bool whole_tpcs, int n_blk_keys, const uint32_t* vis, const int32_t* prefix_len,
+                              const AttnMask* mask) {
   const sdlm_config& c = ctx->cfg;
   AttnParams p;
   p.pool = reinterpret_cast<const __nv_bfloat16*>(ctx->pool);
@@ -962,12 +990,24 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
   p.release_first = cta_cap > 0 ? 1 : 0;
   p.Dk = n_blk_keys > 0 ? n_blk_keys : D;
   p.vis = vis;
+  p.vis_kind = vis ? kVisWords : kVisNone;
+  p.carry_len = nullptr;
+  p.c_max = 0;
+  p.q_stride = D;
+  p.q_first = 0;
+  if (mask) {
+    p.vis_kind = mask->kind == 1 ? kVisVerify : mask->kind == 2 ? kVisCarry : p.vis_kind;
+    p.carry_len = mask->carry_len;
+    p.c_max = mask->c_max;
+    p.q_stride = mask->q_stride;
+    p.q_first = mask->q_first;
+  }
   p.prefix_len = prefix_len;
   // the kernel's tile arithmetic is 32-bit: (tiles of the launch) x (CTAs) must stay below 2^31
   if ((long long)batch * (c.max_pages_per_seq + 1 + ctx->attn_item_cost) * c.n_kv_heads > 13000000ll)
     return cudaErrorInvalidConfiguration;
   const bool wide = ctx->group * D > 32;  // stacked query rows padded to 64, else to 32
-  if (vis != nullptr) {
+  if (p.vis_kind != kVisNone) {
     if (c.head_dim == 128)
       return wide ? attn_launch_one<128, 64, true>(ctx, p, st, cta_cap, whole_tpcs)
                   : attn_launch_one<128, 32, true>(ctx, p, st, cta_cap, whole_tpcs);

@@ -75,6 +75,10 @@ struct sdlm_ctx {
   const void* tmap_w_ptr;
   int tmap_w_rows;
   alignas(64) unsigned char tmap_w[128];
+  // and of the LM head's hidden-state rows (keyed by pointer, rows and box rows)
+  const void* tmap_h_ptr;
+  int tmap_h_rows, tmap_h_box;
+  alignas(64) unsigned char tmap_h[128];
 };
 
 namespace sdlm {
@@ -140,15 +144,25 @@ inline cudaError_t launch_overlapped_cluster(void (*kernel)(KArgs...), dim3 grid
 }
 
 // ---- launchers implemented in the kernel translation units ---------------------------------
+// Visibility of the block's own keys built inside the kernel (kind 1: verification inputs, 2: carry rows in
+// front of the block), and which of the q_stride positions per sequence one launch computes.
+struct AttnMask {
+  int kind;
+  const int32_t* carry_len;
+  int c_max;
+  int q_stride, q_first;
+};
 cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, const void* q,
                               const void* k_blk, const void* v_blk, void* out, cudaStream_t st,
                               int cta_cap = 0, bool whole_tpcs = false, int n_blk_keys = 0,
-                              const uint32_t* vis = nullptr, const int32_t* prefix_len = nullptr);
+                              const uint32_t* vis = nullptr, const int32_t* prefix_len = nullptr,
+                              const AttnMask* mask = nullptr);
 // `independent_of_predecessor`: the caller guarantees that none of the inputs is written by the
 // kernel enqueued just before on `st` (the stripe kernel then overlaps with it).
 sdlm_status launch_lmhead(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
                           float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st,
                           bool independent_of_predecessor = false, int cta_cap = 0);
+sdlm_status lmhead_supported(const sdlm_ctx* ctx, int rows);
 // RMSNorm of a linear product's output rows, written beside them (norm_out = out / rms(out) * weight)
 struct LinNorm {
   const void* weight;

@@ -996,6 +996,28 @@ cudaError_t setup_lmhead(sdlm_ctx* ctx) {
                               kMmaStages * kMmaStageBytes + 128);
 }
 
+// The hidden-state tensor map of the LM head, kept by (pointer, rows, box rows): a decode loop hands in
+// the same buffer every step, and encoding a map costs the host a few microseconds per call.
+static const CUtensorMap* hidden_tmap(sdlm_ctx* ctx, const void* hidden, int rows, int box_rows) {
+  if (ctx->tmap_h_ptr != hidden || ctx->tmap_h_rows != rows || ctx->tmap_h_box != box_rows) {
+    ctx->tmap_h_ptr = nullptr;
+    if (!make_tmap(reinterpret_cast<CUtensorMap*>(ctx->tmap_h), hidden, rows, ctx->cfg.hidden, box_rows)) return nullptr;
+    ctx->tmap_h_ptr = hidden;
+    ctx->tmap_h_rows = rows;
+    ctx->tmap_h_box = box_rows;
+  }
+  return reinterpret_cast<const CUtensorMap*>(ctx->tmap_h);
+}
+
+// What launch_lmhead would refuse for this many rows, found out without enqueuing anything.
+sdlm_status lmhead_supported(const sdlm_ctx* ctx, int rows) {
+  if (rows < 1) return SDLM_ERR_INVALID_ARG;
+  if (rows > ctx->cfg.max_batch * ctx->cfg.max_block) return SDLM_ERR_SHAPE;
+  const bool use_umma = ctx->lmhead_path != 1 && rows <= 256 && ctx->cfg.vocab >= 16;
+  if (ctx->lmhead_path >= 2 && !use_umma) return SDLM_ERR_UNSUPPORTED;
+  return SDLM_OK;
+}
+
 // `partials` holds one float4 per (stripe, row): [max_stripes][rows_pad].
 static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden, const void* w_lm, int32_t* token,
                                     float* p_top1, float* entropy, float* max_logit, float* lse, cudaStream_t st,
@@ -1032,8 +1054,9 @@ static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden,
     const int stage_bytes = kATileBytes + p.bn * kBK * 2;
     int n_stages = kUmmaSmemBudget / stage_bytes;
     if (n_stages > 8) n_stages = 8;
-    CUtensorMap tm_h;
-    if (!make_tmap(&tm_h, hidden, rows, c.hidden, 128)) return SDLM_ERR_CUDA;
+    const CUtensorMap* tm_hp = hidden_tmap(ctx, hidden, rows, 128);
+    if (!tm_hp) return SDLM_ERR_CUDA;
+    const CUtensorMap& tm_h = *tm_hp;
     if (ctx->tmap_w_ptr != w_lm || ctx->tmap_w_rows != p.bn / 2) {
       if (!make_tmap(reinterpret_cast<CUtensorMap*>(ctx->tmap_w), w_lm, c.vocab, c.hidden, p.bn / 2)) return SDLM_ERR_CUDA;
       ctx->tmap_w_ptr = w_lm;
@@ -1057,11 +1080,12 @@ static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden,
     int n_stages = kUmmaSmemBudget / stage_bytes;
     if (n_stages > 8) n_stages = 8;
     if (n_stages < 2) return SDLM_ERR_UNSUPPORTED;
-    CUtensorMap tm_h;
     // With few rows the box only covers them (rounded up to the 8-row swizzle group): the other
     // accumulator lanes then compute on whatever the stage held before, and are never read back.
     p.a_box_rows = R == 1 ? ((rows + 7) / 8 * 8 < 128 ? (rows + 7) / 8 * 8 : 128) : 128;
-    if (!make_tmap(&tm_h, hidden, rows, c.hidden, p.a_box_rows)) return SDLM_ERR_CUDA;
+    const CUtensorMap* tm_hp = hidden_tmap(ctx, hidden, rows, p.a_box_rows);
+    if (!tm_hp) return SDLM_ERR_CUDA;
+    const CUtensorMap& tm_h = *tm_hp;
     if (ctx->tmap_w_ptr != w_lm || ctx->tmap_w_rows != p.bn) {
       if (!make_tmap(reinterpret_cast<CUtensorMap*>(ctx->tmap_w), w_lm, c.vocab, c.hidden, p.bn)) return SDLM_ERR_CUDA;
       ctx->tmap_w_ptr = w_lm;

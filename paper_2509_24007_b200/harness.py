@@ -16,13 +16,6 @@ import sdlm_synth as syn
 from .binding import CONF_LOGIT, Sdlm, SdlmConfig, accept_commit_layers, bf16_tensor_from_bits
 
 
-def verification_mask(D: int) -> np.ndarray:
-    """Visibility words for sdlm_block_attn_masked in the verification pass of a self-speculative step
-    (Sec. 3.4), with the block's 2D keys laid out as [real tokens 0..D-1, [m] of positions 0..D-1]:
-    position j sees the real tokens before it and the [m] at its own position."""
-    return np.array([((1 << j) - 1) + (1 << (D + j)) for j in range(D)], dtype=np.uint32)
-
-
 @dataclass
 class DeviceBlock:
     q: torch.Tensor
@@ -32,30 +25,14 @@ class DeviceBlock:
     host: syn.BlockInputs
 
 
-def carry_mask(carry_len, c_max: int, D: int) -> np.ndarray:
-    """Visibility words [batch, c_max + D] for sdlm_block_attn_masked when each block is preceded by
-    carry_len[b] <= c_max rows of real tokens (rows / keys 0..c_max-1, padded; then the D block positions):
-    a carry row sees the carry keys up to itself, a padding row only itself, a block position every
-    carry key of its sequence and every block key (Sec. 3.3)."""
-    carry_len = np.asarray(carry_len, dtype=np.int64)
-    out = np.empty((len(carry_len), c_max + D), dtype=np.uint32)
-    r = np.arange(c_max, dtype=np.int64)
-    for b, c in enumerate(carry_len):
-        out[b, :c_max] = np.where(r < c, (np.int64(2) << r) - 1, np.int64(1) << r)
-        out[b, c_max:] = ((1 << int(c)) - 1) + (((1 << D) - 1) << c_max)
-    return out
-
-
 @dataclass
 class DeviceVerify:
     q: torch.Tensor        # [B, D, Hq, d]
     k_blk: torch.Tensor    # [B, 2D, Hkv, d]: real tokens' keys, then the [m] keys
     v_blk: torch.Tensor
     hidden: torch.Tensor   # [B, D, H]
-    vis: torch.Tensor      # [B, D] int32 (uint32 visibility words)
     host: "syn.VerifyInputs"
     host_hidden: np.ndarray
-    host_vis: np.ndarray
 
 
 @dataclass
@@ -70,7 +47,9 @@ class StepOutputs:
 
 class DeviceProblem:
     def __init__(self, wl: syn.Workload, w_bits: Optional[np.ndarray] = None, lengths: Optional[np.ndarray] = None,
-                 max_block: Optional[int] = None, keep_prefix: bool = True):
+                 max_block: Optional[int] = None, keep_prefix: bool = True, prefix=None, fill: bool = True):
+        """prefix: the per-sequence (k, v) bit arrays to use instead of drawing them again; fill=False
+        leaves the cache empty (tables reset, no sequence added)."""
         self.wl = wl
         s = wl.shape
         self.lengths = syn.prefix_lengths(wl) if lengths is None else np.asarray(lengths, dtype=np.int32)
@@ -81,8 +60,11 @@ class DeviceProblem:
         self.sd = Sdlm(self.cfg)
         self.w_bits = syn.lm_head_weight(wl) if w_bits is None else w_bits
         self.w_lm = bf16_tensor_from_bits(self.w_bits)
-        self.prefix = []
-        self.reset_cache(keep_prefix)
+        self.prefix = list(prefix) if prefix is not None else []
+        if fill:
+            self.reset_cache(keep_prefix)
+        else:
+            self.sd.kv_reset(self.free_list)
 
     def reset_cache(self, keep_prefix: bool = True) -> None:
         """Free list := the seeded permutation, then every sequence's prefix is added in slot order."""
@@ -109,20 +91,19 @@ class DeviceProblem:
         wl = self.wl
         v = syn.verify_inputs(wl, self.w_bits, step)
         h = syn.verify_hidden(wl, self.w_bits, step, p_agree)
-        vis = np.tile(verification_mask(wl.block), (wl.batch, 1))
         return DeviceVerify(bf16_tensor_from_bits(v.q), bf16_tensor_from_bits(v.k_blk), bf16_tensor_from_bits(v.v_blk),
-                            bf16_tensor_from_bits(h), torch.from_numpy(vis.view(np.int32)).to(self.sd.device), v, h, vis)
+                            bf16_tensor_from_bits(h), v, h)
 
     def speculative_step(self, x: DeviceBlock, xv: "DeviceVerify", out: StepOutputs, out_v: StepOutputs,
                          stream=None) -> None:
         """One self-speculative step (Sec. 3.4) on device-resident inputs, five library calls: first pass
-        (attention, LM head -> speculative tokens), verification pass (masked attention over the real
-        tokens' and the [m] keys, LM head -> verification tokens), then gamma_verify and the commit of
+        (attention, LM head -> speculative tokens), verification pass (attention over the real
+        tokens' and the [m] keys under the verification inputs' visibility, LM head -> verification tokens), then gamma_verify and the commit of
         the kept real-token rows.  No host synchronisation."""
         sd = self.sd
         sd.block_attn(x.q, x.k_blk, x.v_blk, out.attn, stream=stream)
         sd.lmhead_confidence(x.hidden, self.w_lm, out.token, out.p_top1, out.entropy, stream=stream)
-        sd.block_attn_masked(xv.q, xv.k_blk, xv.v_blk, xv.vis, out_v.attn, stream=stream)
+        sd.block_attn_verify(xv.q, xv.k_blk, xv.v_blk, out_v.attn, stream=stream)
         sd.lmhead_confidence(xv.hidden, self.w_lm, out_v.token, out_v.p_top1, out_v.entropy, stream=stream)
         sd.verify_commit(out.token, out_v.token, x.k_blk, x.v_blk, out.accepted_len, out.out_tokens, stream=stream)
 

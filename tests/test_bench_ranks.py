@@ -40,3 +40,15 @@ def test_two_ranks_take_the_slowest_time_and_sum_the_tokens():
 def test_single_rank_passes_values_through():
     import bench
     assert bench.aggregate_over_ranks(None, torch, 5.0, 7, 9.0, "cpu") == (5.0, 7, 9.0)
+
+
+def test_asking_for_more_gpus_than_there_are_fails_loudly():
+    """`python bench.py --gpus 2` outside a launcher starts the ranks itself; without two GPUs it must exit
+    non-zero and print no result line (never a line that says n_gpus: 1)."""
+    import subprocess
+    if torch.cuda.is_available() and torch.cuda.device_count() >= 2:
+        return
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "8"], capture_output=True,
+                       text=True, timeout=300)
+    assert r.returncode != 0
+    assert "n_gpus" not in r.stdout and "GPU" in r.stderr

@@ -150,3 +150,99 @@ def test_a_wait_that_nothing_signals_runs_out_and_leaves_the_context_usable():
     out = dp.step(dp.block(0), wl.tau)                        # the context still works
     torch.cuda.synchronize()
     assert dp.sd.device_status()[0] == 0 and int(out.accepted_len[0]) >= 1
+
+
+def test_restore_and_import_leave_a_recorded_failure_visible():
+    """The sticky status is not table state: a time-out recorded after a SAVE / EXPORT is still there after
+    RESTORE / IMPORT, while lengths, page tables and ring cursors go back."""
+    wl = syn.CONFIGS["cfg0"]
+    dp = DeviceProblem(wl)
+    saved, exported = dp.sd.kv_save(), dp.sd.kv_export()
+    before = dp.sd.kv_tables()
+    dp.step(dp.block(0), wl.tau)                              # the tables move
+    dp.sd.selftest_bounded_wait()                             # and a failure is recorded
+    torch.cuda.synchronize()
+    assert dp.sd.kv_tables()["seq_len"][0] > before["seq_len"][0]
+    dp.sd.kv_restore(saved)
+    st = dp.sd.device_status()
+    assert st[0] == 6 and st[1] == -3                         # SDLM_ERR_TIMEOUT survived the restore
+    t = dp.sd.kv_tables()
+    assert np.array_equal(t["seq_len"], before["seq_len"]) and t["free_head"] == before["free_head"]
+    dp.step(dp.block(0), wl.tau)
+    dp.sd.kv_import(exported)
+    assert dp.sd.device_status(clear=True)[0] == 6            # and the import
+    t = dp.sd.kv_tables()
+    assert np.array_equal(t["seq_len"], before["seq_len"]) and np.array_equal(t["page_table"], before["page_table"])
+    assert t["status"][0] == 0
+    out = dp.step(dp.block(0), wl.tau)                        # the context works on
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0 and int(out.accepted_len[0]) >= 1
+
+
+def test_tables_handed_in_by_the_caller_are_checked_on_the_host_before_anything_is_copied():
+    """IMPORT with a page id outside the pool, a length beyond the table's reach, a page referred to twice
+    or a ring that overlaps a sequence, and RESET with a free list that is no permutation: INVALID_ARG,
+    the live tables untouched, nothing launched."""
+    wl = syn.CONFIGS["cfg0"].with_(batch=2, prefix_lo=70, prefix_hi=150)
+    dp = DeviceProblem(wl)
+    sd = dp.sd
+    good = sd.kv_export()
+    live = sd.kv_tables()
+    cfg = sd.cfg
+    al = lambda x: (x + 255) // 256 * 256
+    off_pt = al(64)
+    off_len = off_pt + al(cfg.max_batch * cfg.max_pages_per_seq * 4)
+    off_ring = off_len + al(cfg.max_batch * 4)
+
+    def broken(edit):
+        buf = good.copy()
+        edit(buf[:64].view(np.uint32), buf[off_pt:off_pt + cfg.max_batch * cfg.max_pages_per_seq * 4].view(np.int32),
+             buf[off_len:off_len + cfg.max_batch * 4].view(np.int32), buf[off_ring:off_ring + cfg.num_pages * 4].view(np.int32))
+        return buf
+
+    def page_out_of_pool(h, pt, ln, ring): pt[0] = cfg.num_pages
+    def negative_page(h, pt, ln, ring): pt[0] = -1
+    def length_beyond_reach(h, pt, ln, ring): ln[0] = cfg.max_pages_per_seq * 64 + 1
+    def negative_length(h, pt, ln, ring): ln[1] = -5
+    def page_twice(h, pt, ln, ring): pt[cfg.max_pages_per_seq] = pt[0]
+    def ring_overlaps_a_sequence(h, pt, ln, ring): ring[h[4] % cfg.num_pages] = pt[0]
+    def ring_too_long(h, pt, ln, ring): h[5] = h[4] + cfg.num_pages + 1
+    n0 = sd.launch_count()
+    for edit in (page_out_of_pool, negative_page, length_beyond_reach, negative_length, page_twice, ring_overlaps_a_sequence,
+                 ring_too_long):
+        with pytest.raises(pk.SdlmError) as e:
+            sd.kv_import(broken(edit))
+        assert e.value.code == 1, edit.__name__
+    for bad in (np.zeros(cfg.num_pages, np.int32), np.arange(1, cfg.num_pages + 1, dtype=np.int32),
+                np.concatenate([[-1], np.arange(1, cfg.num_pages)]).astype(np.int32)):
+        with pytest.raises(pk.SdlmError) as e:
+            sd.kv_reset(bad)
+        assert e.value.code == 1
+    assert sd.launch_count() == n0
+    now = sd.kv_tables()
+    for key in ("page_table", "seq_len", "free_list"):
+        assert np.array_equal(now[key], live[key])
+    sd.kv_import(good)                                        # the untouched export still goes in
+    assert np.array_equal(sd.kv_tables()["seq_len"], live["seq_len"])
+
+
+def test_decode_step_checks_every_argument_before_it_enqueues_anything():
+    wl = syn.CONFIGS["cfg0"]
+    dp = DeviceProblem(wl)
+    x, out = dp.block(0), dp.alloc_outputs()
+    out.attn.fill_(7.0)
+    torch.cuda.synchronize()
+    n0 = dp.sd.launch_count()
+    args = [dp.sd.ctx, wl.batch, wl.block, None, 0.9, 0, x.q.data_ptr(), x.k_blk.data_ptr(), x.v_blk.data_ptr(),
+            x.hidden.data_ptr(), dp.w_lm.data_ptr(), out.attn.data_ptr(), out.token.data_ptr(), out.p_top1.data_ptr(),
+            out.entropy.data_ptr(), out.accepted_len.data_ptr(), out.out_tokens.data_ptr(), None]
+    for missing in (9, 10, 12, 15, 16):                       # hidden, w_lm, token, accepted_len, out_tokens
+        a = list(args)
+        a[missing] = None
+        assert dp.sd.lib.sdlm_decode_step(*a) == 1            # SDLM_ERR_INVALID_ARG
+    a = list(args); a[5] = 9                                  # no such confidence mode
+    assert dp.sd.lib.sdlm_decode_step(*a) == 1
+    a = list(args); a[10] = dp.w_lm.data_ptr() + 2            # misaligned weight
+    assert dp.sd.lib.sdlm_decode_step(*a) == 1
+    torch.cuda.synchronize()
+    assert dp.sd.launch_count() == n0 and bool((out.attn == 7.0).all())

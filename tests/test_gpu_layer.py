@@ -193,7 +193,8 @@ def test_layer_pieces_reject_bad_arguments():
 
 
 def test_two_layer_stack_step_matches_the_oracle_composition():
-    """A tiny whole-model step: the residual stream after two layers, then LM head and acceptance on the
+    """A tiny whole-model step: the residual stream after two layers against the oracle's float64
+    composition (tolerance from the number of bf16 tensors on the way), then LM head and acceptance on the
     GPU's own final hidden state (so that the integer results are compared without accumulated drift),
     and every layer's cache grown by the same accepted rows."""
     from paper_2509_24007_b200.harness import DecoderStack, LayerWeights
@@ -232,13 +233,19 @@ def test_two_layer_stack_step_matches_the_oracle_composition():
         assert all(sd.device_status()[0] == 0 for sd in stack.ctx)
         h_ref, k_ref, v_ref = lo.decoder_stack_hidden(syn.bf16_bits_to_f32(h0_bits).astype(np.float64), host_layers, caches,
                                                      range(B), Hq, Hkv, d, stack.EPS, stack.THETA)
+        # The oracle is float64 throughout; the library keeps a bf16 tensor between two calls.  Along the
+        # longest chain of a layer there are 8 such roundings (norm, q/k/v, rotary, attention output,
+        # stream after the output projection, norm, gated activation, stream after the down projection),
+        # each at most 2^-9 of the largest magnitude and adding up linearly at worst; one more unit stands
+        # for fp32 accumulation order and the approximate exponentials.
+        unit = 2.0 ** -9
         h_gpu = _f64(stack.h)
         scale = np.max(np.abs(h_ref))
-        assert np.max(np.abs(h_gpu - h_ref)) <= 0.03 * scale, (np.max(np.abs(h_gpu - h_ref)), scale)
+        assert np.max(np.abs(h_gpu - h_ref)) <= (8 * L + 1) * unit * scale, (np.max(np.abs(h_gpu - h_ref)), scale)
         for l in range(L):                                   # the rows each layer is about to commit
-            for got, ref in ((stack.k[l], k_ref[l]), (stack.v[l], v_ref[l])):
-                r64 = syn.bf16_bits_to_f32(ref).astype(np.float64)
-                assert np.max(np.abs(_f64(got) - r64)) <= 0.03 * np.max(np.abs(r64))
+            for got, ref, n_round in ((stack.k[l], k_ref[l], 8 * l + 3), (stack.v[l], v_ref[l], 8 * l + 2)):
+                err = np.max(np.abs(_f64(got) - ref))
+                assert err <= (n_round + 1) * unit * np.max(np.abs(ref)), (l, err, np.max(np.abs(ref)))
         # head and acceptance: from the GPU's own final normalised hidden state
         x_bits = pk.bits_from_bf16_tensor(stack.x).reshape(B, D, H)
         stats = orc.lm_head_statistics(x_bits, w_bits)

@@ -6,7 +6,7 @@ import torch
 
 import paper_2509_24007_b200 as pk
 from paper_2509_24007_b200.binding import SdlmError
-from paper_2509_24007_b200.harness import DeviceProblem, verification_mask
+from paper_2509_24007_b200.harness import DeviceProblem
 from oracle import sdlm_oracle as orc
 import sdlm_synth as syn
 from oracle_side import check_attention, oracle_cache
@@ -80,9 +80,22 @@ def test_masked_attention_long_prefix_split_over_many_thread_blocks():
     check_attention(pk.bits_from_bf16_tensor(out), orc.block_attention_masked(q, k, v, pk_, pv_, vis.astype(np.int64)))
 
 
-def test_the_library_side_verification_mask_is_the_oracles():
-    for D in range(1, 9):
-        assert np.array_equal(verification_mask(D).astype(np.int64), orc.verification_visibility(D))
+@pytest.mark.parametrize("Hq,Hkv,d,D", [(4, 2, 64, 4), (16, 2, 128, 4), (16, 2, 128, 8), (8, 1, 64, 1), (40, 8, 128, 5)])
+def test_verification_attention_builds_the_words_of_sec_3_4_itself(Hq, Hkv, d, D):
+    """sdlm_block_attn_verify takes no mask: against the oracle under verification_visibility, and bit for
+    bit what the explicit-mask call gives when it is handed the oracle's words."""
+    shape = syn.Shape(Hq, Hkv, d, 64, 64)
+    lens = [0, 1, 64, 200, 1500]
+    wl, dp = _problem(shape, lens, D, seed=810 + Hq + D)
+    q = _rows(wl, D, 0, "q"); k = _rows(wl, 2 * D, 1, "k"); v = _rows(wl, 2 * D, 2, "v")
+    vis = np.tile(orc.verification_visibility(D), (len(lens), 1))
+    out = dp.sd.block_attn_verify(_dev_bits(q), _dev_bits(k), _dev_bits(v))
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+    pk_, pv_ = zip(*dp.prefix)
+    check_attention(pk.bits_from_bf16_tensor(out), orc.block_attention_masked(q, k, v, pk_, pv_, vis))
+    explicit = dp.sd.block_attn_masked(_dev_bits(q), _dev_bits(k), _dev_bits(v), _vis_tensor(vis))
+    assert torch.equal(out, explicit)
 
 
 @pytest.mark.parametrize("name", ["cfg2_d4", "cfg2"])
@@ -91,15 +104,14 @@ def test_verification_pass_attention_at_full_size(name):
     wl = syn.CONFIGS[name]
     dp = DeviceProblem(wl, keep_prefix=True)
     ver = syn.verify_inputs(wl, dp.w_bits, 0)
-    vis = np.tile(verification_mask(wl.block), (wl.batch, 1))
-    out = dp.sd.block_attn_masked(_dev_bits(ver.q), _dev_bits(ver.k_blk), _dev_bits(ver.v_blk), _vis_tensor(vis))
+    vis = np.tile(orc.verification_visibility(wl.block), (wl.batch, 1))
+    out = dp.sd.block_attn_verify(_dev_bits(ver.q), _dev_bits(ver.k_blk), _dev_bits(ver.v_blk))
     torch.cuda.synchronize()
     assert dp.sd.device_status()[0] == 0
     order = np.argsort(dp.lengths)
     sample = sorted({int(order[0]), int(order[-1]), 0, wl.batch - 1, 13})
     pk_, pv_ = zip(*[dp.prefix[b] for b in sample])
-    ref = orc.block_attention_masked(ver.q[sample], ver.k_blk[sample], ver.v_blk[sample], pk_, pv_,
-                                     vis[sample].astype(np.int64))
+    ref = orc.block_attention_masked(ver.q[sample], ver.k_blk[sample], ver.v_blk[sample], pk_, pv_, vis[sample])
     check_attention(pk.bits_from_bf16_tensor(out)[sample], ref)
 
 
@@ -150,7 +162,7 @@ def test_self_speculative_step_matches_the_oracle(name, batch):
         check_attention(pk.bits_from_bf16_tensor(out.attn), orc.block_attention(x.host.q, x.host.k_blk, x.host.v_blk, pk_, pv_))
         check_attention(pk.bits_from_bf16_tensor(out_v.attn),
                         orc.block_attention_masked(xv.host.q, xv.host.k_blk, xv.host.v_blk, pk_, pv_,
-                                                   xv.host_vis.astype(np.int64)))
+                                                   np.tile(orc.verification_visibility(wl.block), (batch, 1))))
         flagged = []
         st1 = orc.lm_head_statistics(x.host.hidden, dp.w_bits, w64)
         st2 = orc.lm_head_statistics(xv.host_hidden, dp.w_bits, w64)
@@ -189,36 +201,61 @@ def test_masked_attention_rejects_bad_arguments():
 
 
 # ---- a block preceded by carry rows of real tokens ----------------------------------------------
-def test_the_library_side_carry_mask_is_the_oracles():
-    from paper_2509_24007_b200.harness import carry_mask
-    for c_max, D in ((0, 4), (3, 4), (7, 8), (2, 1)):
-        lens = list(range(c_max + 1)) * 2
-        assert np.array_equal(carry_mask(lens, c_max, D).astype(np.int64), orc.carry_visibility(lens, c_max, D))
+@pytest.mark.parametrize("Hq,Hkv,d,D,c_max", [(4, 2, 64, 4, 3), (16, 2, 128, 4, 3), (16, 2, 128, 8, 7), (40, 8, 128, 8, 7),
+                                               (8, 1, 64, 5, 2), (4, 2, 64, 1, 0)])
+def test_carry_attention_builds_the_words_of_sec_3_3_from_device_carry_lengths(Hq, Hkv, d, D, c_max):
+    """sdlm_block_attn_carry reads carry_len on the device and takes no mask: against the oracle under
+    carry_visibility (every carry length 0..c_max occurs), with more query positions than one launch
+    stacks (15 positions at Hq/Hkv = 8) included."""
+    shape = syn.Shape(Hq, Hkv, d, 64, 64)
+    carry = np.array(list(range(c_max + 1)) + [c_max, 0], dtype=np.int32)
+    B, R = len(carry), c_max + D
+    lens = ([0, 1, 63, 64, 65, 200, 1000, 130, 5, 700] * 2)[:B]
+    wl = syn.Workload("masked", shape, B, D, 0, 0, (0.9,), seed=1500 + Hq + D)
+    dp = DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16), lengths=np.asarray(lens, np.int32),
+                       max_block=min(8, R))
+    q = _rows(wl, R, 0, "q"); k = _rows(wl, R, 1, "k"); v = _rows(wl, R, 2, "v")
+    out = dp.sd.block_attn_carry(_dev_bits(q), _dev_bits(k), _dev_bits(v), torch.from_numpy(carry).cuda(), c_max)
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+    pk_, pv_ = zip(*dp.prefix)
+    vis = orc.carry_visibility(carry, c_max, D)
+    ref = orc.block_attention_masked(q, k, v, pk_, pv_, vis)
+    real = [(b, r) for b in range(B) for r in list(range(int(carry[b]))) + list(range(c_max, R))]
+    idx = tuple(np.array(real).T)
+    check_attention(pk.bits_from_bf16_tensor(out)[idx], ref[idx])          # padding rows are not outputs
+    if R <= 8 and (Hq // Hkv) * R <= 64:                                   # one launch: the explicit-mask call, bit for bit
+        explicit = dp.sd.block_attn_masked(_dev_bits(q), _dev_bits(k), _dev_bits(v), _vis_tensor(vis))
+        assert torch.equal(out, explicit)
 
 
-@pytest.mark.parametrize("shape_name,D,c_max", [("tiny", 4, 3), ("3b", 4, 3), ("tiny", 3, 2), ("tiny", 1, 0)])
-def test_carry_step_loop_matches_the_oracle_and_caches_only_real_rows(shape_name, D, c_max):
-    """Several steps of: masked attention over [carry rows ; block], LM head on the block positions,
-    Eq. 7, commit of the real-token rows.  Against the oracle step by step; and at the end the cache
-    holds exactly the true rows of the positions it covers (the junk [m] rows never enter it)."""
-    from paper_2509_24007_b200.harness import carry_mask
+@pytest.mark.parametrize("shape_name,D,c_max", [("tiny", 4, 3), ("3b", 4, 3), ("3b", 8, 7), ("32b", 8, 7), ("tiny", 3, 2),
+                                                ("tiny", 1, 0)])
+def test_carry_loop_runs_on_the_device_and_caches_only_real_rows(shape_name, D, c_max):
+    """Eight steps of: attention over [carry rows ; block] (carry lengths read on the device), LM head on the
+    block positions, Eq. 7, commit of the real-token rows, next carry lengths written on the device -- all
+    enqueued back to back with no copy to the host in between.  The oracle loop runs first (it also fixes
+    which true rows each step's inputs carry); every step's outputs, the final tables and the cache
+    contents must agree, and the cache must hold exactly the true rows (junk [m] rows never enter it)."""
     from oracle_side import check_tokens, check_confidences, check_gamma
-    shape = syn.SHAPE_TINY if shape_name == "tiny" else syn.Shape(16, 2, 128, 256, 1024)
-    B = 4
+    shape = {"tiny": syn.SHAPE_TINY, "3b": syn.Shape(16, 2, 128, 256, 1024), "32b": syn.Shape(40, 8, 128, 256, 1024)}[shape_name]
+    B, steps = 4, 8
     lens = np.array([0, 62, 64, 300], dtype=np.int32)
-    wl = syn.Workload("carry", shape, B, D, 0, 0, (0.9,), steps=8, seed=1200 + D)
-    dp = DeviceProblem(wl, lengths=lens, max_block=c_max + D)
+    wl = syn.Workload("carry", shape, B, D, 0, 0, (0.9,), steps=steps + 2, seed=1200 + D)
+    dp = DeviceProblem(wl, lengths=lens, max_block=min(8, c_max + D))
     cache = oracle_cache(wl, dp.lengths, dp.num_pages, dp.mpps, dp.prefix)
     rng = np.random.default_rng(D)
     Hkv, d = shape.n_kv_heads, shape.head_dim
-    true_k = syn.f32_to_bf16_bits(rng.normal(size=(B, 600, Hkv, d)).astype(np.float32))
-    true_v = syn.f32_to_bf16_bits(rng.normal(size=(B, 600, Hkv, d)).astype(np.float32))
+    true_k = syn.f32_to_bf16_bits(rng.normal(size=(B, 700, Hkv, d)).astype(np.float32))
+    true_v = syn.f32_to_bf16_bits(rng.normal(size=(B, 700, Hkv, d)).astype(np.float32))
     for b in range(B):                                   # the prefixes the problem was built with are "true" rows too
         true_k[b, :lens[b]], true_v[b, :lens[b]] = dp.prefix[b]
     w64 = orc.widen(dp.w_bits)
-    carry = np.zeros(B, dtype=np.int32)
     R = c_max + D
-    for step in range(5):
+    # ---- the oracle loop, which also decides what each step is fed
+    carry = np.zeros(B, dtype=np.int32)
+    fed, refs = [], []
+    for step in range(steps):
         x = syn.block_inputs(wl, dp.w_bits, step)
         q = syn.f32_to_bf16_bits(rng.normal(size=(B, R, shape.n_q_heads, d)).astype(np.float32))
         k_rows = syn.f32_to_bf16_bits(rng.normal(size=(B, R, Hkv, d)).astype(np.float32))     # junk unless overwritten
@@ -228,31 +265,47 @@ def test_carry_step_loop_matches_the_oracle_and_caches_only_real_rows(shape_name
             for r in range(int(carry[b])):
                 k_rows[b, r], v_rows[b, r] = true_k[b, L + r], true_v[b, L + r]
             k_rows[b, c_max], v_rows[b, c_max] = true_k[b, L + carry[b]], true_v[b, L + carry[b]]
-        vis = carry_mask(carry, c_max, D)
+        vis = orc.carry_visibility(carry, c_max, D)
         pk_, pv_ = zip(*[cache.gather_fast(b) for b in range(B)])
-        dk, dv = _dev_bits(k_rows), _dev_bits(v_rows)
-        attn = dp.sd.block_attn_masked(_dev_bits(q), dk, dv, _vis_tensor(vis))
-        tok, p, ent = dp.sd.lmhead_confidence(_dev_bits(x.hidden), dp.w_lm)[:3]
-        acc, out_tok = dp.sd.accept_commit_carry(wl.tau, torch.from_numpy(carry).cuda(), c_max, tok.view(B, D),
-                                                 p.view(B, D), ent.view(B, D), dk, dv)
-        torch.cuda.synchronize()
-        assert dp.sd.device_status()[0] == 0
-        ref = orc.block_attention_masked(q, k_rows, v_rows, pk_, pv_, vis.astype(np.int64))
-        real = [(b, r) for b in range(B) for r in list(range(int(carry[b]))) + list(range(c_max, R))]
-        got = pk.bits_from_bf16_tensor(attn)
-        idx = tuple(np.array(real).T)
-        check_attention(got[idx], ref[idx])                # padding rows are not outputs
+        attn = orc.block_attention_masked(q, k_rows, v_rows, pk_, pv_, vis)
         stats = orc.lm_head_statistics(x.hidden, dp.w_bits, w64)
+        res = orc.accept_and_commit_carry(cache, range(B), stats.token.reshape(B, D), stats.p_top1.reshape(B, D), wl.tau,
+                                          carry, c_max, k_rows, v_rows)
+        fed.append((q, k_rows, v_rows, x.hidden))
+        refs.append((attn, stats, res, carry.copy(), cache.seq_len.copy(), cache.page_table.copy()))
+        carry = np.minimum(res.accepted_len - 1, c_max).astype(np.int32)
+    # ---- the device loop: everything enqueued, nothing read back until the end
+    dev = [tuple(_dev_bits(t) for t in f) for f in fed]
+    carry_dev = torch.zeros(B, dtype=torch.int32, device="cuda")
+    carries = torch.zeros((steps + 1, B), dtype=torch.int32, device="cuda")
+    outs = []
+    torch.cuda.synchronize()
+    for step in range(steps):
+        q, k_rows, v_rows, hidden = dev[step]
+        attn = dp.sd.block_attn_carry(q, k_rows, v_rows, carry_dev, c_max)
+        tok, p, ent = dp.sd.lmhead_confidence(hidden, dp.w_lm)[:3]
+        acc, out_tok = dp.sd.accept_commit_carry(wl.tau, carry_dev, c_max, tok.view(B, D), p.view(B, D), ent.view(B, D),
+                                                 k_rows, v_rows, next_carry_len=carry_dev)       # in place
+        carries[step + 1].copy_(carry_dev)
+        outs.append((attn, tok, p, ent, acc, out_tok))
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+    got_carries = carries.cpu().numpy()
+    for step in range(steps):
+        attn_ref, stats, res, carry_in, _, _ = refs[step]
+        attn, tok, p, ent, acc, out_tok = outs[step]
+        assert np.array_equal(got_carries[step], carry_in)
+        real = [(b, r) for b in range(B) for r in list(range(int(carry_in[b]))) + list(range(c_max, R))]
+        idx = tuple(np.array(real).T)
+        check_attention(pk.bits_from_bf16_tensor(attn)[idx], attn_ref[idx])
         flagged = []
         check_tokens(tok.cpu().numpy(), stats, flagged)
         check_confidences(p.cpu().numpy(), ent.cpu().numpy(), stats)
-        res = orc.accept_and_commit_carry(cache, range(B), stats.token.reshape(B, D), stats.p_top1.reshape(B, D), wl.tau,
-                                          carry, c_max, k_rows, v_rows)
         assert check_gamma(acc.cpu().numpy(), res, flagged) == 0 and not flagged, flagged
         assert np.array_equal(out_tok.cpu().numpy(), res.out_tokens)
-        t = dp.sd.kv_tables()
-        assert np.array_equal(t["page_table"], cache.page_table) and np.array_equal(t["seq_len"], cache.seq_len)
-        carry = (res.accepted_len - 1).astype(np.int32)
+    t = dp.sd.kv_tables()
+    assert np.array_equal(t["page_table"], cache.page_table) and np.array_equal(t["seq_len"], cache.seq_len)
+    assert max(int(r[3].max()) for r in refs) > 0 or D == 1          # some step did carry rows over
     for b in range(B):
         L = int(cache.seq_len[b])
         k, v = dp.sd.kv_gather(b, L)
