@@ -87,8 +87,9 @@ __device__ __forceinline__ uint32_t vis_word(const AttnParams& p, int b, int j) 
   return ((1u << c) - 1u) | (((1u << (p.q_stride - p.c_max)) - 1u) << p.c_max);
 }
 
-// 8 warps; 12 when 64 stacked query rows need a second set of softmax warps
-constexpr int attn_threads(int nq) { return nq == 64 ? 384 : 256; }
+// 12 warps (loader, two MMA issuers, stager; four softmax; four epilogue); 16 when 64 stacked query rows
+// need a second set of softmax warps
+constexpr int attn_threads(int nq) { return nq == 64 ? 512 : 384; }
 constexpr float kRebaseThreshold = 32.0f;  // log2 units a score may exceed its row reference by
 
 __device__ __forceinline__ int attn_slot(const AttnParams& p, int i) { return p.seq_ids ? p.seq_ids[i] : i; }
@@ -222,7 +223,10 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
   constexpr int P_BUF_B = 2 * P_PANEL_B;
   // two P^T buffers, except where a third two-tile ring stage is worth more than the second buffer
   constexpr int PB = (HD == 128 && NQ == 64) ? 1 : 2;
-  constexpr uint32_t O_COL = 128, TMEM_COLS = 256;  // S^T buffers at columns 0 and NQ
+  // tensor memory: S^T buffers at columns 0 and NQ, O^T buffers (one per item in flight) at 128 and 128 + NQ
+  constexpr uint32_t O_COL = 128, TMEM_COLS = 256;
+  constexpr int NSW = NQ / 8;        // softmax warps (one set of four per 32 stacked rows)
+  constexpr int W_EPI = 4 + NSW;     // first of the four epilogue warps
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -236,26 +240,32 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
   uint64_t* s_free = s_full + 2;        // [2]
   uint64_t* p_full = s_free + 2;        // [2]
   uint64_t* p_free = p_full + 2;        // [2]
-  uint64_t* q_full = p_free + 2;
+  uint64_t* o_done = p_free + 2;        // [2] the item's last O^T instruction has completed
+  uint64_t* o_free = o_done + 2;        // [2] the epilogue has read the item's O^T out of tensor memory
+  uint64_t* q_full = o_free + 2;
   uint64_t* q_free = q_full + 1;
-  uint64_t* o_done = q_free + 1;
-  uint64_t* o_free = o_done + 1;
-  uint64_t* ep_bar = o_free + 1;
-  uint64_t* drain = ep_bar + 1;         // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 3);  // one spare slot keeps the floats below 16-byte aligned
+  uint64_t* ep_bar = q_free + 1;        // meeting point of the softmax warps
+  uint64_t* ep2_bar = ep_bar + 1;       // meeting point of the epilogue warps
+  uint64_t* l_ready = ep2_bar + 1;      // softmax -> epilogue: the item's row sums and references are in shared memory
+  uint64_t* l_read = l_ready + 1;       // epilogue -> softmax: they have been read
+  uint64_t* drain = l_read + 1;         // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 2);
   volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* s_last = abort + 1;
-  volatile int* blk_go = abort + 2;     // warp 0 -> warp 6: block-tile ring slots that are free so far
+  volatile int* blk_go = abort + 2;     // warp 0 -> warp 3: block-tile ring slots that are free so far
   volatile int* flag = abort + 3;       // [3] "some score outgrew its reference", by group mod 3
   float* mref = reinterpret_cast<float*>(const_cast<int*>(abort) + 7);  // [64] row references (log2 units); 16-byte aligned
-  float* fbuf = mref + 64;              // [64] rescale factors of a reference move; 1 / row sum in a merge
-  int* row_off = reinterpret_cast<int*>(fbuf + 64);  // [64] element offset of stacked row r inside a (b, KV head) slab
-  // Scratch that is only needed while no O^T instruction can be reading P^T (a reference move waits
-  // for the previous one, the end of an item for the last one) lives in the P^T buffers:
+  float* fbuf = mref + 64;              // [64] rescale factors of a reference move
+  float* ltot = fbuf + 64;              // [2][64] row sums over all keys of an item, by item parity
+  uint16_t* row_hd = reinterpret_cast<uint16_t*>(ltot + 128);  // [64] stacked row r sits row_hd[r] * d elements into a (b, KV head) slab
+  int* s_first = reinterpret_cast<int*>(row_hd + 64);          // [batch + 1], then lengths [batch], then slots [batch]
+  // Scratch inside the P^T buffers.  mnew / mx (a reference move) are only touched while no O^T instruction
+  // can be reading P^T (the move waits for the previous one).  The hand-off of an item's row sums and final
+  // references to the epilogue warps lies further in, in the buffer of the item's last group, once that
+  // group's O^T instruction is done; the next P^T column written there waits until they have been read.
   float* mnew = reinterpret_cast<float*>(p_s);   // [64] references after a move
   int* mx = reinterpret_cast<int*>(p_s) + 64;    // [4][64] per-warp row maxima
-  float* lsum = reinterpret_cast<float*>(p_s) + 320;  // [4][64] per-warp row sums
-  int* s_first = row_off + 64;                         // [batch + 1], then lengths [batch], then slots [batch]
+  constexpr int SCR_LSUM = 1280;                 // [4][64] per-warp row sums, then [64] final references (byte offset in a buffer)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int GD = p.G * p.D;
@@ -267,15 +277,18 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     }
     for (int s = 0; s < 2; ++s) {
       ptx::mbar_init(&s_full[s], 1);
-      ptx::mbar_init(&s_free[s], NQ / 8);  // one arrival per softmax warp
-      ptx::mbar_init(&p_full[s], NQ / 8);
+      ptx::mbar_init(&s_free[s], NSW);  // one arrival per softmax warp
+      ptx::mbar_init(&p_full[s], NSW);
       ptx::mbar_init(&p_free[s], 1);
+      ptx::mbar_init(&o_done[s], 1);
+      ptx::mbar_init(&o_free[s], 4);    // one arrival per epilogue warp
     }
     ptx::mbar_init(q_full, 1);
     ptx::mbar_init(q_free, 1);
-    ptx::mbar_init(o_done, 1);
-    ptx::mbar_init(o_free, NQ / 8);
-    ptx::mbar_init(ep_bar, NQ / 8);
+    ptx::mbar_init(ep_bar, NSW);
+    ptx::mbar_init(ep2_bar, 4);
+    ptx::mbar_init(l_ready, NSW);
+    ptx::mbar_init(l_read, 4);
     ptx::mbar_init(&drain[0], 1);
     ptx::mbar_init(&drain[1], 1);
     *abort = 0;
@@ -341,8 +354,8 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     }
     if (lane == 0) s_first[p.batch] = carry;
   }
-  // stacked row r = j*G + g is q[b, j, h*G + g, :] (and the same row of out)
-  if (tid >= 64 && tid < 128) row_off[tid - 64] = tid - 64 < GD ? (((tid - 64) / p.G) * p.Hq + (tid - 64) % p.G) * HD : -1;
+  // stacked row r = j*G + g is q[b, j, h*G + g, :] (and the same row of out): (j*Hq + g) * d elements into the slab
+  if (tid >= 64 && tid < 128) row_hd[tid - 64] = tid - 64 < GD ? (uint16_t)(((tid - 64) / p.G) * p.Hq + (tid - 64) % p.G) : (uint16_t)0xffff;
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
@@ -356,7 +369,6 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     }
   }
   const uint32_t tmem_base = *tmem_slot;
-
   if (warp == 0) {
     // ---------------------------------------------------------------- cached tiles: bulk copies
     ItemWalk w;
@@ -396,7 +408,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
               ptx::bulk_g2s_hint(st + K_REGION_B + j * VT_B, src + KH * K_PANEL_B, VT_B, &full[ring.stage], kv_policy);
             }
             if (has_blk) {
-              // The block's own tile is written by warp 6, which then gives the group's second
+              // The block's own tile is written by warp 3, which then gives the group's second
               // arrival.  This warp does the waiting for the ring slot, because it reaches the slot
               // in ring order, and passes it on through a counter.
               __threadfence_block();
@@ -461,7 +473,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       }
     }
     __syncwarp();
-  } else if (warp == 7) {
+  } else if (warp == 2) {
     // ---------------------------------------------------------------- O^T += V^T P^T issuer
     if (lane == 0) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NQ >> 3) << 17) | ((128u >> 4) << 24);
@@ -474,18 +486,19 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       bool ok = true;
       while (ok && walk_next(w, p, it)) {
         const int n = it.t1 - it.t0, ng = (n + 1) / 2;
+        const uint32_t ob = item_idx & 1u, use = item_idx >> 1;  // O^T buffer of this item and how often it was used before
         for (int g = 0; g < ng; ++g) {
           const uint32_t pb = gc % PB;
           if (!ptx::mbar_wait(&p_full[pb], (gc / PB) & 1u, abort)) { ok = false; break; }
-          // the first instruction of an item overwrites O^T: the previous item's must have been read out
-          if (g == 0 && item_idx > 0 && !ptx::mbar_wait(o_free, (item_idx - 1) & 1u, abort)) { ok = false; break; }
+          // the first instruction of an item overwrites its O^T buffer: the item before last must have been read out
+          if (g == 0 && use > 0 && !ptx::mbar_wait(&o_free[ob], (use - 1) & 1u, abort)) { ok = false; break; }
           ptx::tc_fence_after();
           const int tiles = min(2, n - 2 * g);
           const uint32_t av = st_addr + (uint32_t)ring.stage * PAIR_B + K_REGION_B, bp = p_addr + pb * P_BUF_B;
           for (int j = 0; j < tiles; ++j)
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-              ptx::umma_bf16_ss(tmem_base + O_COL, attn_smem_desc(av + j * VT_B + k * 32),
+              ptx::umma_bf16_ss(tmem_base + O_COL + ob * NQ, attn_smem_desc(av + j * VT_B + k * 32),
                                 attn_smem_desc(bp + j * P_PANEL_B + k * 32), idesc, (g == 0 && j == 0 && k == 0) ? 0u : 1u);
           // P^T is only written after S^T of the same group was read, so K of this stage is done as well
           ptx::umma_commit(&stage_free[ring.stage]);
@@ -494,7 +507,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
           ++gc;
         }
         if (!ok) break;
-        ptx::umma_commit(o_done);
+        ptx::umma_commit(&o_done[ob]);
         ++item_idx;
       }
       if (!ok) {
@@ -504,21 +517,22 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       }
     }
     __syncwarp();
-  } else if (warp < 6 || warp >= 8) {
+  } else if (warp >= 4 && warp < W_EPI) {
     // ---------------------------------------------------------------- softmax: thread = key of the group
-    // Four warps cover the 128 keys of a group; with 64 stacked query rows a second set of four
-    // (warps 8..11) takes the upper 32 rows, so that no thread handles more than 32 values per group.
+    // Four warps cover the 128 keys of a group; with 64 stacked query rows a second set of four takes the
+    // upper 32 rows, so that no thread handles more than 32 values per group.  These warps never wait
+    // for global memory: an item's results are handed to the epilogue warps and the next item starts.
     constexpr int QV = 32;                          // query rows (columns of S^T) per thread
     const int qd = warp & 3;                        // TMEM lane quarter of this warp
-    const int qb = warp >= 8 ? 32 : 0;              // first query row of this warp's set
-    const int sw = (warp >= 8 ? 4 : 0) + qd;        // index among the softmax warps
-    const int kg = qd * 32 + lane;       // key within the group = accumulator lane; also the d index at the end
+    const int qb = ((warp - 4) >> 2) * 32;          // first query row of this warp's set
+    const int kg = qd * 32 + lane;       // key within the group = accumulator lane
     const int tj = kg >> 6, kt = kg & 63;  // tile of the group, key within that tile
     const uint32_t lane_addr = tmem_base + ((uint32_t)(qd * 32) << 16);
     ItemWalk w;
     walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
     Item it;
     uint32_t gc = 0, item_idx = 0, ep_uses = 0;
+    int lread_buf = -1;  // the P^T buffer that still holds the previous item's hand-off (-1: none, or read)
     bool ok = true;
     // all softmax warps meet; false when a wait ran out
     auto meet = [&]() -> bool {
@@ -533,6 +547,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
 #pragma unroll
       for (int q = 0; q < QV; ++q) l[q] = 0.f;
       const int n = it.t1 - it.t0, ng = (n + 1) / 2;
+      const uint32_t o_addr = lane_addr + O_COL + (item_idx & 1u) * NQ + qb;  // this item's O^T columns of my rows
       // which of my 32 query rows see my key if it turns out to be a block key (bit q: row qb + q)
       [[maybe_unused]] uint32_t visq = 0xffffffffu;
       if (MASKED && p.vis_kind != kVisNone && it.t1 > it.pages) {
@@ -555,104 +570,133 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
         const bool mine = kt < tile_valid(it, it.t0 + 2 * g + tj, p.Dk);  // does my key exist?
         if (!__all_sync(0xffffffffu, ptx::mbar_wait(&s_full[sb], (gc >> 1) & 1u, abort))) { ok = false; break; }
         ptx::tc_fence_after();
-        float x[QV];  // my key's score for every row, then its exponent relative to the row reference
+        // My key's scores for 16 of my rows (c = 0, 1), straight from tensor memory; they are read again
+        // wherever they are needed rather than kept, which leaves the registers to the row sums.
+        [[maybe_unused]] const bool blk_key = MASKED && visq != 0xffffffffu && it.t0 + 2 * g + tj == it.pages;
+        auto scores = [&](int c, float (&x)[16]) {
+          ptx::tmem_ld16(lane_addr + sb * NQ + qb + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&x[0]));
+          ptx::tmem_ld_wait();
+          if constexpr (MASKED) {
+            if (blk_key) {  // my key is a block key some rows do not see
 #pragma unroll
-        for (int c = 0; c < QV / 16; ++c)
-          ptx::tmem_ld16(lane_addr + sb * NQ + qb + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&x[c * 16]));
-        ptx::tmem_ld_wait();
-        ptx::tc_fence_before();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&s_free[sb]);
-        if constexpr (MASKED) {
-          if (visq != 0xffffffffu && it.t0 + 2 * g + tj == it.pages) {  // my key is a block key some rows do not see
-#pragma unroll
-            for (int q = 0; q < QV; ++q)
-              if (!((visq >> q) & 1u)) x[q] = -INFINITY;
+              for (int i = 0; i < 16; ++i)
+                if (!((visq >> (c * 16 + i)) & 1u)) x[i] = -INFINITY;
+            }
           }
-        }
+        };
 
         const bool first = g == 0;
-        bool moved = first;  // the first group of an item always sets the references
-        const uint32_t fi = gc % 3u;
-        if (warp == 2 && lane == 0) flag[(fi + 1u) % 3u] = 0;  // last read two groups ago
-        float e[QV];  // exponents of my key relative to the row references
-        if (!first) {
-          float xm = -INFINITY;
+        if (first) {
+          // The item's references start at the scores of its first key (which always exists): one thread
+          // per set of rows publishes them, no reduction over keys.  A row that does not see that key
+          // (masked) starts at 0.  Whatever is too low for a later score is moved below, as in any group.
+          if (qd == 0) {  // the warp that holds key 0 (tensor-memory loads are warp-wide); its lane 0 writes
 #pragma unroll
-          for (int q4 = 0; q4 < QV; q4 += 4) {
-            const float4 mr = *reinterpret_cast<const float4*>(mref + qb + q4);
-            e[q4] = fmaf(x[q4], p.scale_log2, -mr.x);
-            e[q4 + 1] = fmaf(x[q4 + 1], p.scale_log2, -mr.y);
-            e[q4 + 2] = fmaf(x[q4 + 2], p.scale_log2, -mr.z);
-            e[q4 + 3] = fmaf(x[q4 + 3], p.scale_log2, -mr.w);
-            xm = fmaxf(fmaxf(xm, fmaxf(e[q4], e[q4 + 1])), fmaxf(e[q4 + 2], e[q4 + 3]));
+            for (int c = 0; c < 2; ++c) {
+              float x[16];
+              scores(c, x);
+              if (lane == 0) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                  const float v = x[i] * p.scale_log2;
+                  mref[qb + c * 16 + i] = v > -INFINITY ? v : 0.f;
+                }
+              }
+            }
           }
-          const bool need = mine && xm > kRebaseThreshold;
-          if (__any_sync(0xffffffffu, need) && lane == 0) flag[fi] = 1;
           if (!meet()) { ok = false; break; }
-          moved = flag[fi] != 0;
         }
-        if (moved) {
+        const uint32_t fi = gc % 3u;
+        if (warp == 4 && lane == 0) flag[(fi + 1u) % 3u] = 0;  // last read two groups ago
+        float xm = -INFINITY;  // my key's largest exponent relative to the row references
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          float x[16];
+          scores(c, x);
+#pragma unroll
+          for (int i4 = 0; i4 < 16; i4 += 4) {
+            const float4 mr = *reinterpret_cast<const float4*>(mref + qb + c * 16 + i4);
+            xm = fmaxf(fmaxf(xm, fmaxf(fmaf(x[i4], p.scale_log2, -mr.x), fmaf(x[i4 + 1], p.scale_log2, -mr.y))),
+                       fmaxf(fmaf(x[i4 + 2], p.scale_log2, -mr.z), fmaf(x[i4 + 3], p.scale_log2, -mr.w)));
+          }
+        }
+        const bool need = mine && xm > kRebaseThreshold;
+        if (__any_sync(0xffffffffu, need) && lane == 0) flag[fi] = 1;
+        if (!meet()) { ok = false; break; }
+        if (flag[fi] != 0) {
           // ---- move the row references to max(old reference, this group's row maxima).  The scratch
           // for this sits in the P^T buffers and O^T is about to be rescaled: the previous O^T
-          // instruction must be done (for the first group of an item the previous item's end saw to it).
+          // instruction must be done (before the first group of an item the previous item's end saw to it).
           if (!first) {
             const uint32_t prev = gc - 1;
             if (!__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[prev % PB], (prev / PB) & 1u, abort))) { ok = false; break; }
           }
 #pragma unroll
-          for (int q = 0; q < QV; ++q) {
-            const int v = __reduce_max_sync(0xffffffffu, mine ? ordered_int(x[q] * p.scale_log2) : kIntMin);
-            if (lane == q) mx[qd * 64 + qb + q] = v;
+          for (int c = 0; c < 2; ++c) {
+            float x[16];
+            scores(c, x);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const int v = __reduce_max_sync(0xffffffffu, mine ? ordered_int(x[i] * p.scale_log2) : kIntMin);
+              if (lane == c * 16 + i) mx[qd * 64 + qb + lane] = v;
+            }
           }
           if (!meet()) { ok = false; break; }
 #pragma unroll
           for (int q = 0; q < QV; ++q) {
             const int gi = max(max(mx[qb + q], mx[64 + qb + q]), max(mx[128 + qb + q], mx[192 + qb + q]));
-            const float m_old = first ? -INFINITY : mref[qb + q];
-            float m_new = gi == kIntMin ? m_old : fmaxf(m_old, ordered_float(gi));
-            if (m_new == -INFINITY) m_new = 0.f;  // no key at all (cannot happen: every group has one)
-            const float f = first ? 0.f : ptx::ex2(m_old - m_new);
+            const float m_old = mref[qb + q];
+            const float m_new = gi == kIntMin ? m_old : fmaxf(m_old, ordered_float(gi));
+            const float f = ptx::ex2(m_old - m_new);
             l[q] *= f;
             if (kg == q) { mnew[qb + q] = m_new; fbuf[qb + q] = f; }
           }
           if (!meet()) { ok = false; break; }  // everybody has read the old references
           if (kg < QV) mref[qb + kg] = mnew[qb + kg];
           if (!first) {  // O^T holds sums relative to the old references
-            ptx::tc_fence_after();
 #pragma unroll
             for (int c = 0; c < QV / 16; ++c) {
               uint32_t o[16];
-              ptx::tmem_ld16(lane_addr + O_COL + qb + c * 16, o);
+              ptx::tmem_ld16(o_addr + c * 16, o);
               ptx::tmem_ld_wait();
 #pragma unroll
               for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * fbuf[qb + c * 16 + i]);
-              ptx::tmem_st16(lane_addr + O_COL + qb + c * 16, o);
+              ptx::tmem_st16(o_addr + c * 16, o);
             }
             ptx::tmem_st_wait();
           }
           if (!meet()) { ok = false; break; }  // the new references are visible
-#pragma unroll
-          for (int q4 = 0; q4 < QV; q4 += 4) {
-            const float4 mr = *reinterpret_cast<const float4*>(mref + qb + q4);
-            e[q4] = fmaf(x[q4], p.scale_log2, -mr.x);
-            e[q4 + 1] = fmaf(x[q4 + 1], p.scale_log2, -mr.y);
-            e[q4 + 2] = fmaf(x[q4 + 2], p.scale_log2, -mr.z);
-            e[q4 + 3] = fmaf(x[q4 + 3], p.scale_log2, -mr.w);
-          }
         }
         // P^T column of my key: 2^(s*scale - reference), rounded to bf16; absent keys give 0
         const uint32_t pbuf = gc % PB;
+        if (lread_buf == (int)pbuf) {  // the buffer still holds the previous item's hand-off: it must have been read
+          if (!__all_sync(0xffffffffu, ptx::mbar_wait(l_read, (item_idx - 1) & 1u, abort))) { ok = false; break; }
+          lread_buf = -1;
+        }
         if (gc >= (uint32_t)PB && !__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[pbuf], ((gc / PB) & 1u) ^ 1u, abort))) { ok = false; break; }
         uint8_t* pcol = p_s + pbuf * P_BUF_B + tj * P_PANEL_B + (kt & 7) * 2;
 #pragma unroll
-        for (int q = 0; q < QV; ++q) {
-          e[q] = mine ? ptx::ex2(e[q]) : 0.f;
-          l[q] += e[q];
-        }
+        for (int c = 0; c < 2; ++c) {
+          float x[16];
+          scores(c, x);
+          if (c == 1) {  // the last read of this S^T buffer
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&s_free[sb]);
+          }
 #pragma unroll
-        for (int q = 0; q < QV; ++q)
-          *reinterpret_cast<__nv_bfloat16*>(pcol + (qb + q) * 128 + (((kt >> 3) ^ (q & 7)) << 4)) = __float2bfloat16_rn(e[q]);
+          for (int i4 = 0; i4 < 16; i4 += 4) {
+            const float4 mr = *reinterpret_cast<const float4*>(mref + qb + c * 16 + i4);
+            const float m4[4] = {mr.x, mr.y, mr.z, mr.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int q = c * 16 + i4 + i;
+              const float e = mine ? ptx::ex2(fmaf(x[i4 + i], p.scale_log2, -m4[i])) : 0.f;
+              l[q] += e;
+              *reinterpret_cast<__nv_bfloat16*>(pcol + (qb + q) * 128 + (((kt >> 3) ^ (q & 7)) << 4)) = __float2bfloat16_rn(e);
+            }
+          }
+        }
         ptx::fence_proxy_async();
         ptx::tc_fence_before();
         __syncwarp();
@@ -660,12 +704,9 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       }
       if (!ok) break;
 
-      // ---- end of item: row sums over all keys (lane q of each warp ends up with the warp's sum of row q)
-      float* ls = lsum;
-      float lwarp[QV / 32];
-#pragma unroll
-      for (int half = 0; half < QV / 32; ++half) {
-        float* v = &l[half * 32];
+      // ---- end of item: row sums over this warp's keys (lane q ends up with the warp's sum of row qb + q)
+      {
+        float* v = l;
 #pragma unroll
         for (int off = 16; off >= 1; off >>= 1) {
 #pragma unroll
@@ -675,134 +716,160 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
             v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
           }
         }
-        lwarp[half] = v[0];
       }
-      // the last O^T instruction of the item is done: O^T is complete and the P^T buffers are idle
-      if (!__all_sync(0xffffffffu, ptx::mbar_wait(o_done, item_idx & 1u, abort))) { ok = false; break; }
-      ptx::tc_fence_after();
-#pragma unroll
-      for (int half = 0; half < QV / 32; ++half) ls[qd * 64 + qb + half * 32 + lane] = lwarp[half];
-      if (!meet()) { ok = false; break; }
-      float o[QV];  // O^T row d = kg: one value per query row of this warp's set
-#pragma unroll
-      for (int c = 0; c < QV / 16; ++c)
-        ptx::tmem_ld16(lane_addr + O_COL + qb + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&o[c * 16]));
-      ptx::tmem_ld_wait();
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(o_free);
+      // They go, with the final references, into the P^T buffer of the item's last group once that group's
+      // O^T instruction is done (and the hand-off before this one has been read).
+      const uint32_t last = gc - 1, b_last = last % PB;
+      if (lread_buf >= 0) {
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(l_read, (item_idx - 1) & 1u, abort))) { ok = false; break; }
+        lread_buf = -1;
+      }
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[b_last], (last / PB) & 1u, abort))) { ok = false; break; }
+      float* hand = reinterpret_cast<float*>(p_s + b_last * P_BUF_B + SCR_LSUM);
+      hand[qd * 64 + qb + lane] = l[0];
+      if (kg < QV) hand[256 + qb + kg] = mref[qb + kg];
+      if (!meet()) { ok = false; break; }  // the references are copied before the next item's first key replaces them
+      if (lane == 0) ptx::mbar_arrive(l_ready);
+      lread_buf = (int)b_last;
       ++item_idx;
-
-      const int d = kg;
-      // row q = j*G + g  <->  out[b, j, h*G + g, :]
-      __nv_bfloat16* out_base = p.out + (((size_t)it.b * p.q_stride + p.q_first) * p.Hq + it.h * p.G) * HD + d;
-      if (it.n_splits == 1) {
-        if (d < HD) {
+    }
+    if (!ok && lane == 0) attn_timeout(p, 3);
+  } else if (warp >= W_EPI) {
+    // ---------------------------------------------------------------- epilogue: thread = output column d
+    // Takes an item's O^T out of tensor memory, divides by the row sums and writes the output rows, or, for
+    // a (sequence, KV head) pair cut by a range boundary, leaves fp32 partials and merges them if this was
+    // the last of the pair's thread blocks to arrive.  Runs beside the next item's scores and sums.
+    const int ew = warp - W_EPI;
+    const int t = ew * 32 + lane;  // accumulator lane = output column
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(ew * 32) << 16);
+    ItemWalk w;
+    walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
+    Item it;
+    uint32_t gc = 0, item_idx = 0, ep2_uses = 0;
+    bool ok = true;
+    auto meet2 = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ep2_bar);
+      const bool r = __all_sync(0xffffffffu, ptx::mbar_wait(ep2_bar, ep2_uses & 1u, abort));
+      ++ep2_uses;
+      return r;
+    };
+    while (ok && walk_next(w, p, it)) {
+      const uint32_t ob = item_idx & 1u, use = item_idx >> 1;
+      gc += (uint32_t)((it.t1 - it.t0 + 1) / 2);
+      const uint32_t b_last = (gc - 1) % PB;  // where the softmax warps left this item's sums
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(l_ready, item_idx & 1u, abort))) { ok = false; break; }
+      const float* hand = reinterpret_cast<const float*>(p_s + b_last * P_BUF_B + SCR_LSUM);
+      float m_row = 0.f, l_row = 0.f;
+      if (t < NQ) {
+        l_row = hand[t] + hand[64 + t] + hand[128 + t] + hand[192 + t];
+        m_row = hand[256 + t];
+        ltot[ob * 64 + t] = l_row;
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(l_read);
+      if (!meet2()) { ok = false; break; }  // the row sums are visible to all four warps
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&o_done[ob], use & 1u, abort))) { ok = false; break; }
+      ptx::tc_fence_after();
+      const float* lt = ltot + ob * 64;
+      // row q = j*G + g  <->  out[b, q_first + j, h*G + g, :]
+      __nv_bfloat16* out_slab = p.out + (((size_t)it.b * p.q_stride + p.q_first) * p.Hq + it.h * p.G) * HD;
+      const size_t slot_row = (size_t)(blockIdx.x + it.pair) * NQ;
+      // O^T row d = t, 32 stacked query rows at a time: divided by the row sums into the output, or as it is
+      // into this split's partial result
 #pragma unroll
-          for (int q = 0; q < QV; ++q) {
-            if (qb + q < GD) {
-              const float lt = ls[qb + q] + ls[64 + qb + q] + ls[128 + qb + q] + ls[192 + qb + q];
-              out_base[row_off[qb + q]] = __float2bfloat16_rn(o[q] / lt);
-            }
+      for (int q0 = 0; q0 < NQ; q0 += 32) {
+        float o[32];
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+          ptx::tmem_ld16(lane_addr + O_COL + ob * NQ + q0 + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&o[c * 16]));
+        ptx::tmem_ld_wait();
+        if (q0 + 32 == NQ) {  // everything is in registers: the buffer may take the item after next
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&o_free[ob]);
+        }
+        if (t < HD) {
+          if (it.n_splits == 1) {
+#pragma unroll
+            for (int q = 0; q < 32; ++q)
+              if (q0 + q < GD) out_slab[(size_t)row_hd[q0 + q] * HD + t] = __float2bfloat16_rn(o[q] / lt[q0 + q]);
+          } else {
+#pragma unroll
+            for (int q = 0; q < 32; ++q) p.part_o[(slot_row + q0 + q) * HD + t] = o[q];
           }
         }
-      } else {
-        const size_t slot_row = (size_t)(blockIdx.x + it.pair) * NQ;
-        if (d < HD) {
-#pragma unroll
-          for (int q = 0; q < QV; ++q) p.part_o[(slot_row + qb + q) * HD + d] = o[q];
-        }
-        const int mrow = qb + kg;  // the query row this thread looks after where one thread per row is needed
-        if (kg < QV) {
-          // a row that saw no key in this split (all of them masked) takes no part in the merge
-          const float lrow = ls[mrow] + ls[64 + mrow] + ls[128 + mrow] + ls[192 + mrow];
-          *reinterpret_cast<float2*>(p.part_ml + (slot_row + mrow) * 2) =
-              make_float2(lrow > 0.f ? mref[mrow] : -INFINITY, lrow);
-        }
+      }
+      ++item_idx;
+      if (it.n_splits > 1) {
+        // a row that saw no key in this split (all of them masked) takes no part in the merge
+        if (t < NQ) *reinterpret_cast<float2*>(p.part_ml + (slot_row + t) * 2) = make_float2(l_row > 0.f ? m_row : -INFINITY, l_row);
         __threadfence();
-        if (!meet()) { ok = false; break; }
-        if (warp == 2 && lane == 0) {  // every split of the pair counts once; the last one merges
+        if (!meet2()) { ok = false; break; }
+        if (t == 0) {  // every split of the pair counts once; the last one merges
           const int arrived = atomicAdd(&p.pair_cnt[it.pair], 1);
           const int last = arrived == it.n_splits - 1;
           if (last) p.pair_cnt[it.pair] = 0;
           *s_last = last;
         }
-        if (!meet()) { ok = false; break; }
+        if (!meet2()) { ok = false; break; }
         if (*s_last) {
-          // ---- merge the splits of this pair (fixed order: run-to-run identical).  Row q's weight of
-          // split s is 2^(m_s - m) with m = max_s m_s; the weights go through the (now idle) P^T
-          // buffers, every thread sums four output columns, and the row sum L divides at the end.
+          // ---- merge the splits of this pair (fixed order: run-to-run identical).  Row q's weight of split
+          // s is 2^(m_s - m) with m = max_s m_s.  A thread owns (row, four columns) units, consecutive threads
+          // consecutive columns of one row; it reads its rows' (m_s, l_s) itself, so nothing is shared.
           __threadfence();
-          constexpr int kCap = PB * P_BUF_B / 4 / NQ;  // splits whose weights fit into the P^T buffers at once
-          float* wbuf = reinterpret_cast<float*>(p_s);
+          constexpr int C4 = HD / 4, UPT = 8;
           const size_t first_row = (size_t)(it.c_first + it.pair) * NQ;
-          float m = -INFINITY, L = 0.f;
-          const bool row_thread = kg < QV && mrow < GD;
-          if (row_thread) {
-#pragma unroll 8
-            for (int s = 0; s < it.n_splits; ++s) m = fmaxf(m, __ldcg(p.part_ml + (first_row + (size_t)s * NQ + mrow) * 2));
-          }
-          constexpr int NSW = NQ / 8;           // softmax warps
-          const int dq = lane, qg = sw;         // four columns 4*dq.. of the rows q = qg mod NSW
-          float acc[NQ / NSW][4];
+          for (int u0 = 0; u0 < GD * C4; u0 += 128 * UPT) {
+            float m[UPT], L[UPT], a0[UPT], a1[UPT], a2[UPT], a3[UPT];
+            int uq[UPT];
 #pragma unroll
-          for (int i = 0; i < NQ / NSW; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
-          for (int c0 = 0; c0 < it.n_splits; c0 += kCap) {
-            const int cn = min(kCap, it.n_splits - c0);
-            if (c0 > 0 && !meet()) { ok = false; break; }  // the previous chunk's weights are no longer read
-            if (row_thread) {
-#pragma unroll 8
-              for (int s = 0; s < cn; ++s) {
-                const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (first_row + (size_t)(c0 + s) * NQ + mrow) * 2));
-                const float a = ptx::ex2(ml.x - m);
-                L = fmaf(a, ml.y, L);
-                wbuf[s * NQ + mrow] = a;
-              }
+            for (int i = 0; i < UPT; ++i) {
+              const int u = u0 + i * 128 + t;
+              uq[i] = u < GD * C4 ? u / C4 : -1;
+              m[i] = -INFINITY;
+              L[i] = a0[i] = a1[i] = a2[i] = a3[i] = 0.f;
             }
-            if (!meet()) { ok = false; break; }
-            if (4 * dq < HD) {
-#pragma unroll 4
-              for (int s = 0; s < cn; ++s) {
-                const float* src = p.part_o + (first_row + (size_t)(c0 + s) * NQ) * HD + 4 * dq;
+            for (int s = 0; s < it.n_splits; ++s) {
+              const float* ml = p.part_ml + (first_row + (size_t)s * NQ) * 2;
 #pragma unroll
-                for (int i = 0; i < NQ / NSW; ++i) {
-                  const int q = qg + NSW * i;
-                  if (q < GD) {
-                    const float wq = wbuf[s * NQ + q];
-                    const float4 v = __ldcg(reinterpret_cast<const float4*>(src + (size_t)q * HD));
-                    acc[i][0] = fmaf(wq, v.x, acc[i][0]);
-                    acc[i][1] = fmaf(wq, v.y, acc[i][1]);
-                    acc[i][2] = fmaf(wq, v.z, acc[i][2]);
-                    acc[i][3] = fmaf(wq, v.w, acc[i][3]);
-                  }
+              for (int i = 0; i < UPT; ++i)
+                if (uq[i] >= 0) m[i] = fmaxf(m[i], __ldcg(ml + uq[i] * 2));
+            }
+            for (int s = 0; s < it.n_splits; ++s) {
+              const float* ml = p.part_ml + (first_row + (size_t)s * NQ) * 2;
+              const float* po = p.part_o + (first_row + (size_t)s * NQ) * HD + 4 * (t % C4);
+#pragma unroll
+              for (int i = 0; i < UPT; ++i) {
+                if (uq[i] >= 0) {
+                  const float2 r = __ldcg(reinterpret_cast<const float2*>(ml + uq[i] * 2));
+                  const float4 v = __ldcg(reinterpret_cast<const float4*>(po + (size_t)uq[i] * HD));
+                  const float a = ptx::ex2(r.x - m[i]);
+                  L[i] = fmaf(a, r.y, L[i]);
+                  a0[i] = fmaf(a, v.x, a0[i]);
+                  a1[i] = fmaf(a, v.y, a1[i]);
+                  a2[i] = fmaf(a, v.z, a2[i]);
+                  a3[i] = fmaf(a, v.w, a3[i]);
                 }
               }
             }
-          }
-          if (!ok) break;
-          if (row_thread) fbuf[mrow] = 1.0f / L;
-          if (!meet()) { ok = false; break; }
-          if (4 * dq < HD) {
-            __nv_bfloat16* ob = p.out + (((size_t)it.b * p.q_stride + p.q_first) * p.Hq + it.h * p.G) * HD + 4 * dq;
 #pragma unroll
-            for (int i = 0; i < NQ / NSW; ++i) {
-              const int q = qg + NSW * i;
-              if (q < GD) {
-                const float inv = fbuf[q];
+            for (int i = 0; i < UPT; ++i) {
+              if (uq[i] >= 0) {
+                const float inv = 1.0f / L[i];
                 uint2 v;
-                v.x = ptx::pack_bf16(acc[i][0] * inv, acc[i][1] * inv);
-                v.y = ptx::pack_bf16(acc[i][2] * inv, acc[i][3] * inv);
-                *reinterpret_cast<uint2*>(ob + row_off[q]) = v;
+                v.x = ptx::pack_bf16(a0[i] * inv, a1[i] * inv);
+                v.y = ptx::pack_bf16(a2[i] * inv, a3[i] * inv);
+                *reinterpret_cast<uint2*>(out_slab + (size_t)row_hd[uq[i]] * HD + 4 * (t % C4)) = v;
               }
             }
           }
-          if (!meet()) { ok = false; break; }  // the P^T buffers and fbuf go back to the softmax
         }
       }
     }
-    if (!ok && lane == 0) attn_timeout(p, 3);
+    if (!ok && lane == 0) attn_timeout(p, 6);
   } else {
-    // ---------------------------------------------------------------- warp 6: Q rows and the block's own tile
+    // ---------------------------------------------------------------- warp 3: Q rows and the block's own tile
     constexpr int NQC = NQ * (HD / 8) / 32;  // 16-byte chunks of the stacked query rows per lane
     ItemWalk w;
     walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
@@ -814,14 +881,14 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     // loads): those are fetched one item ahead, the rest (only with 64 stacked rows) when the item starts.
     constexpr int NQR = NQC < 16 ? NQC : 16;
     uint4 qreg[NQR];
-    // stacked query rows: row r = j*G + g  <->  q[b, j, h*G + g, :]; rows beyond G*D are zero
+    // stacked query rows: row r = j*G + g  <->  q[b, q_first + j, h*G + g, :]; rows beyond G*D are zero
     auto fetch_q = [&](const Item& x, int first) {
 #pragma unroll
       for (int i = 0; i < NQR; ++i) {
         const int idx = (first + i) * 32 + lane, r = idx / (HD / 8), c = idx % (HD / 8);
         qreg[i] = make_uint4(0, 0, 0, 0);
         if (r < GD)
-          qreg[i] = __ldg(reinterpret_cast<const uint4*>(p.q + (((size_t)x.b * p.q_stride + p.q_first) * p.Hq + x.h * p.G) * HD + row_off[r]) + c);
+          qreg[i] = __ldg(reinterpret_cast<const uint4*>(p.q + (((size_t)x.b * p.q_stride + p.q_first) * p.Hq + x.h * p.G + row_hd[r]) * HD) + c);
       }
     };
     auto store_q = [&](int first) {
@@ -914,10 +981,11 @@ constexpr int kAttnSmemLimit = 232448;  // largest dynamic shared memory of one 
 
 template <int HD, int NQ>
 static int attn_fixed_smem(int batch) {
-  // alignment slack, Q, the P^T buffers, 16 barrier slots, flags, row scratch, prefix sums; for d = 64 the
-  // M = 128 O^T instruction reads 64 rows past the last V^T tile, which must still be shared memory
+  // alignment slack, Q, the P^T buffers, 20 barrier slots, flags, row scratch (references, factors, two sets
+  // of row sums, row offsets), prefix sums; for d = 64 the M = 128 O^T instruction reads 64 rows past the
+  // last V^T tile, which must still be shared memory
   const int p_buffers = (HD == 128 && NQ == 64) ? 1 : 2;
-  return 1024 + (HD / 64) * NQ * 128 + p_buffers * 2 * NQ * 128 + 16 * 8 + 32 + 3 * 64 * 4 + (batch + 1) * 12 + 64 +
+  return 1024 + (HD / 64) * NQ * 128 + p_buffers * 2 * NQ * 128 + 20 * 8 + 32 + 4 * 64 * 4 + 64 * 2 + (batch + 1) * 12 + 16 +
          (HD == 64 ? 8192 : 0);
 }
 
