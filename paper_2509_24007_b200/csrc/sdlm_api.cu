@@ -43,7 +43,7 @@ WorkspaceLayout workspace_layout(const sdlm_config& c) {
   L.attn_max_items = kAttnMaxCtas + c.max_batch * c.n_kv_heads;
   L.attn_ml = take((size_t)L.attn_max_items * L.q_rows_pad * 2 * 4);
   L.attn_o = take((size_t)L.attn_max_items * L.q_rows_pad * c.head_dim * 4);
-  L.attn_cnt = take((size_t)c.max_batch * c.n_kv_heads * 4);
+  L.attn_cnt = take((size_t)c.max_batch * c.n_kv_heads * 8);
   L.st_q = take(rows * c.n_q_heads * c.head_dim * 2);
   L.st_k = take(rows * c.n_kv_heads * c.head_dim * 2);
   L.st_v = take(rows * c.n_kv_heads * c.head_dim * 2);
@@ -485,7 +485,7 @@ static sdlm_status reset_tables(sdlm_ctx* ctx, const int32_t* host_free_list, cu
         cudaSuccess)
       return SDLM_ERR_CUDA;
   }
-  if (cudaMemsetAsync(ctx->ws + ctx->lay.attn_cnt, 0, (size_t)c.max_batch * c.n_kv_heads * 4, st) != cudaSuccess)
+  if (cudaMemsetAsync(ctx->ws + ctx->lay.attn_cnt, 0, (size_t)c.max_batch * c.n_kv_heads * 8, st) != cudaSuccess)
     return SDLM_ERR_CUDA;
   reset_tables_kernel<<<64, 256, 0, st>>>(ctx->hdr, ctx->page_table, ctx->seq_len, ctx->free_list,
                                          c.max_batch * c.max_pages_per_seq, c.max_batch, c.num_pages,
@@ -946,7 +946,7 @@ extern "C" sdlm_status sdlm_device_status(sdlm_ctx* ctx, int32_t* host_out, int3
     const sdlm_config& c = ctx->cfg;
     if (cudaMemsetAsync(ctx->hdr->status, 0, 16, st) != cudaSuccess ||
         cudaMemsetAsync(&ctx->hdr->commit_ticket, 0, 8, st) != cudaSuccess ||
-        cudaMemsetAsync(ctx->ws + ctx->lay.attn_cnt, 0, (size_t)c.max_batch * c.n_kv_heads * 4, st) != cudaSuccess)
+        cudaMemsetAsync(ctx->ws + ctx->lay.attn_cnt, 0, (size_t)c.max_batch * c.n_kv_heads * 8, st) != cudaSuccess)
       return SDLM_ERR_CUDA;
   }
   if (cudaStreamSynchronize(st) != cudaSuccess) return SDLM_ERR_CUDA;

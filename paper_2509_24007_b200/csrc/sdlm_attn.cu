@@ -43,7 +43,7 @@ struct AttnParams {
   __nv_bfloat16* out;
   float* part_ml;  // [slot][row][2]  (reference max in log2 units, sum)
   float* part_o;   // [slot][row][d]
-  int* pair_cnt;   // [batch * Hkv] arrivals of finished splits; zero between launches
+  int2* pair_info; // [batch * Hkv] (first thread block, number of thread blocks) of every pair, for the merge kernel
   DevHeader* hdr;
   float scale_log2;  // softmax scale * log2(e)
   int batch, D, Hq, Hkv, G, mpps, num_pages, n_stages;
@@ -251,7 +251,6 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
   uint64_t* drain = l_read + 1;         // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 2);
   volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  volatile int* s_last = abort + 1;
   volatile int* blk_go = abort + 2;     // warp 0 -> warp 3: block-tile ring slots that are free so far
   volatile int* flag = abort + 3;       // [3] "some score outgrew its reference", by group mod 3
   float* mref = reinterpret_cast<float*>(const_cast<int*>(abort) + 7);  // [64] row references (log2 units); 16-byte aligned
@@ -369,6 +368,11 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     }
   }
   const uint32_t tmem_base = *tmem_slot;
+  // Registers follow the work (384 threads start at 168 registers each, 512 at 128): the group of four
+  // copy / issue / staging warps and the epilogue warps give some up, the softmax warps, which hold a key's
+  // scores and sums for 32 rows, take them.  Each group's code sits inside the branch that sets its count.
+  if (warp < 4) {
+    ptx::reg_dealloc<NQ == 64 ? 104 : 144>();
   if (warp == 0) {
     // ---------------------------------------------------------------- cached tiles: bulk copies
     ItemWalk w;
@@ -387,7 +391,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
         int page0 = __shfl_sync(0xffffffffu, my_page, (2 * g) & 31);
         int page1 = __shfl_sync(0xffffffffu, my_page, (2 * g + 1) & 31);
         if (lane == 0) {
-          if (issued >= (uint32_t)NS && !ptx::mbar_wait(&stage_free[ring.stage], ring.phase ^ 1u, abort)) ok = false;
+          if (issued >= (uint32_t)NS && !ptx::mbar_wait_paced(&stage_free[ring.stage], ring.phase ^ 1u, abort)) ok = false;
           if (ok) {
             const int cached = max(0, min(2, n_cached - 2 * g));   // cached tiles of this group
             const bool has_blk = n > n_cached && (n - 1) / 2 == g;  // the block's own tile is in it
@@ -517,357 +521,6 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       }
     }
     __syncwarp();
-  } else if (warp >= 4 && warp < W_EPI) {
-    // ---------------------------------------------------------------- softmax: thread = key of the group
-    // Four warps cover the 128 keys of a group; with 64 stacked query rows a second set of four takes the
-    // upper 32 rows, so that no thread handles more than 32 values per group.  These warps never wait
-    // for global memory: an item's results are handed to the epilogue warps and the next item starts.
-    constexpr int QV = 32;                          // query rows (columns of S^T) per thread
-    const int qd = warp & 3;                        // TMEM lane quarter of this warp
-    const int qb = ((warp - 4) >> 2) * 32;          // first query row of this warp's set
-    const int kg = qd * 32 + lane;       // key within the group = accumulator lane
-    const int tj = kg >> 6, kt = kg & 63;  // tile of the group, key within that tile
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(qd * 32) << 16);
-    ItemWalk w;
-    walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
-    Item it;
-    uint32_t gc = 0, item_idx = 0, ep_uses = 0;
-    int lread_buf = -1;  // the P^T buffer that still holds the previous item's hand-off (-1: none, or read)
-    bool ok = true;
-    // all softmax warps meet; false when a wait ran out
-    auto meet = [&]() -> bool {
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(ep_bar);
-      const bool r = __all_sync(0xffffffffu, ptx::mbar_wait(ep_bar, ep_uses & 1u, abort));
-      ++ep_uses;
-      return r;
-    };
-    while (ok && walk_next(w, p, it)) {
-      float l[QV];  // this key subset's share of every row sum
-#pragma unroll
-      for (int q = 0; q < QV; ++q) l[q] = 0.f;
-      const int n = it.t1 - it.t0, ng = (n + 1) / 2;
-      const uint32_t o_addr = lane_addr + O_COL + (item_idx & 1u) * NQ + qb;  // this item's O^T columns of my rows
-      // which of my 32 query rows see my key if it turns out to be a block key (bit q: row qb + q)
-      [[maybe_unused]] uint32_t visq = 0xffffffffu;
-      if (MASKED && p.vis_kind != kVisNone && it.t1 > it.pages) {
-        visq = 0;
-        int j = qb / p.G, rem = qb % p.G;
-        uint32_t vj = j < p.D ? vis_word(p, it.b, j) : 0u;
-#pragma unroll
-        for (int q = 0; q < QV; ++q) {
-          const uint32_t bit = qb + q < GD ? (kt < 32 ? (vj >> kt) & 1u : 0u) : 1u;  // padding rows: no mask
-          visq |= bit << q;
-          if (++rem == p.G) {
-            rem = 0;
-            ++j;
-            vj = j < p.D ? vis_word(p, it.b, j) : 0u;
-          }
-        }
-      }
-      for (int g = 0; g < ng; ++g, ++gc) {
-        const uint32_t sb = gc & 1u;
-        const bool mine = kt < tile_valid(it, it.t0 + 2 * g + tj, p.Dk);  // does my key exist?
-        if (!__all_sync(0xffffffffu, ptx::mbar_wait(&s_full[sb], (gc >> 1) & 1u, abort))) { ok = false; break; }
-        ptx::tc_fence_after();
-        // My key's scores for 16 of my rows (c = 0, 1), straight from tensor memory; they are read again
-        // wherever they are needed rather than kept, which leaves the registers to the row sums.
-        [[maybe_unused]] const bool blk_key = MASKED && visq != 0xffffffffu && it.t0 + 2 * g + tj == it.pages;
-        auto scores = [&](int c, float (&x)[16]) {
-          ptx::tmem_ld16(lane_addr + sb * NQ + qb + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&x[0]));
-          ptx::tmem_ld_wait();
-          if constexpr (MASKED) {
-            if (blk_key) {  // my key is a block key some rows do not see
-#pragma unroll
-              for (int i = 0; i < 16; ++i)
-                if (!((visq >> (c * 16 + i)) & 1u)) x[i] = -INFINITY;
-            }
-          }
-        };
-
-        const bool first = g == 0;
-        if (first) {
-          // The item's references start at the scores of its first key (which always exists): one thread
-          // per set of rows publishes them, no reduction over keys.  A row that does not see that key
-          // (masked) starts at 0.  Whatever is too low for a later score is moved below, as in any group.
-          if (qd == 0) {  // the warp that holds key 0 (tensor-memory loads are warp-wide); its lane 0 writes
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-              float x[16];
-              scores(c, x);
-              if (lane == 0) {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                  const float v = x[i] * p.scale_log2;
-                  mref[qb + c * 16 + i] = v > -INFINITY ? v : 0.f;
-                }
-              }
-            }
-          }
-          if (!meet()) { ok = false; break; }
-        }
-        const uint32_t fi = gc % 3u;
-        if (warp == 4 && lane == 0) flag[(fi + 1u) % 3u] = 0;  // last read two groups ago
-        float xm = -INFINITY;  // my key's largest exponent relative to the row references
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          float x[16];
-          scores(c, x);
-#pragma unroll
-          for (int i4 = 0; i4 < 16; i4 += 4) {
-            const float4 mr = *reinterpret_cast<const float4*>(mref + qb + c * 16 + i4);
-            xm = fmaxf(fmaxf(xm, fmaxf(fmaf(x[i4], p.scale_log2, -mr.x), fmaf(x[i4 + 1], p.scale_log2, -mr.y))),
-                       fmaxf(fmaf(x[i4 + 2], p.scale_log2, -mr.z), fmaf(x[i4 + 3], p.scale_log2, -mr.w)));
-          }
-        }
-        const bool need = mine && xm > kRebaseThreshold;
-        if (__any_sync(0xffffffffu, need) && lane == 0) flag[fi] = 1;
-        if (!meet()) { ok = false; break; }
-        if (flag[fi] != 0) {
-          // ---- move the row references to max(old reference, this group's row maxima).  The scratch
-          // for this sits in the P^T buffers and O^T is about to be rescaled: the previous O^T
-          // instruction must be done (before the first group of an item the previous item's end saw to it).
-          if (!first) {
-            const uint32_t prev = gc - 1;
-            if (!__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[prev % PB], (prev / PB) & 1u, abort))) { ok = false; break; }
-          }
-#pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            float x[16];
-            scores(c, x);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const int v = __reduce_max_sync(0xffffffffu, mine ? ordered_int(x[i] * p.scale_log2) : kIntMin);
-              if (lane == c * 16 + i) mx[qd * 64 + qb + lane] = v;
-            }
-          }
-          if (!meet()) { ok = false; break; }
-#pragma unroll
-          for (int q = 0; q < QV; ++q) {
-            const int gi = max(max(mx[qb + q], mx[64 + qb + q]), max(mx[128 + qb + q], mx[192 + qb + q]));
-            const float m_old = mref[qb + q];
-            const float m_new = gi == kIntMin ? m_old : fmaxf(m_old, ordered_float(gi));
-            const float f = ptx::ex2(m_old - m_new);
-            l[q] *= f;
-            if (kg == q) { mnew[qb + q] = m_new; fbuf[qb + q] = f; }
-          }
-          if (!meet()) { ok = false; break; }  // everybody has read the old references
-          if (kg < QV) mref[qb + kg] = mnew[qb + kg];
-          if (!first) {  // O^T holds sums relative to the old references
-#pragma unroll
-            for (int c = 0; c < QV / 16; ++c) {
-              uint32_t o[16];
-              ptx::tmem_ld16(o_addr + c * 16, o);
-              ptx::tmem_ld_wait();
-#pragma unroll
-              for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * fbuf[qb + c * 16 + i]);
-              ptx::tmem_st16(o_addr + c * 16, o);
-            }
-            ptx::tmem_st_wait();
-          }
-          if (!meet()) { ok = false; break; }  // the new references are visible
-        }
-        // P^T column of my key: 2^(s*scale - reference), rounded to bf16; absent keys give 0
-        const uint32_t pbuf = gc % PB;
-        if (lread_buf == (int)pbuf) {  // the buffer still holds the previous item's hand-off: it must have been read
-          if (!__all_sync(0xffffffffu, ptx::mbar_wait(l_read, (item_idx - 1) & 1u, abort))) { ok = false; break; }
-          lread_buf = -1;
-        }
-        if (gc >= (uint32_t)PB && !__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[pbuf], ((gc / PB) & 1u) ^ 1u, abort))) { ok = false; break; }
-        uint8_t* pcol = p_s + pbuf * P_BUF_B + tj * P_PANEL_B + (kt & 7) * 2;
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          float x[16];
-          scores(c, x);
-          if (c == 1) {  // the last read of this S^T buffer
-            ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&s_free[sb]);
-          }
-#pragma unroll
-          for (int i4 = 0; i4 < 16; i4 += 4) {
-            const float4 mr = *reinterpret_cast<const float4*>(mref + qb + c * 16 + i4);
-            const float m4[4] = {mr.x, mr.y, mr.z, mr.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const int q = c * 16 + i4 + i;
-              const float e = mine ? ptx::ex2(fmaf(x[i4 + i], p.scale_log2, -m4[i])) : 0.f;
-              l[q] += e;
-              *reinterpret_cast<__nv_bfloat16*>(pcol + (qb + q) * 128 + (((kt >> 3) ^ (q & 7)) << 4)) = __float2bfloat16_rn(e);
-            }
-          }
-        }
-        ptx::fence_proxy_async();
-        ptx::tc_fence_before();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&p_full[pbuf]);
-      }
-      if (!ok) break;
-
-      // ---- end of item: row sums over this warp's keys (lane q ends up with the warp's sum of row qb + q)
-      {
-        float* v = l;
-#pragma unroll
-        for (int off = 16; off >= 1; off >>= 1) {
-#pragma unroll
-          for (int i = 0; i < off; ++i) {
-            const bool up = (lane & off) != 0;
-            const float send = up ? v[i] : v[i + off], keep = up ? v[i + off] : v[i];
-            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-          }
-        }
-      }
-      // They go, with the final references, into the P^T buffer of the item's last group once that group's
-      // O^T instruction is done (and the hand-off before this one has been read).
-      const uint32_t last = gc - 1, b_last = last % PB;
-      if (lread_buf >= 0) {
-        if (!__all_sync(0xffffffffu, ptx::mbar_wait(l_read, (item_idx - 1) & 1u, abort))) { ok = false; break; }
-        lread_buf = -1;
-      }
-      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[b_last], (last / PB) & 1u, abort))) { ok = false; break; }
-      float* hand = reinterpret_cast<float*>(p_s + b_last * P_BUF_B + SCR_LSUM);
-      hand[qd * 64 + qb + lane] = l[0];
-      if (kg < QV) hand[256 + qb + kg] = mref[qb + kg];
-      if (!meet()) { ok = false; break; }  // the references are copied before the next item's first key replaces them
-      if (lane == 0) ptx::mbar_arrive(l_ready);
-      lread_buf = (int)b_last;
-      ++item_idx;
-    }
-    if (!ok && lane == 0) attn_timeout(p, 3);
-  } else if (warp >= W_EPI) {
-    // ---------------------------------------------------------------- epilogue: thread = output column d
-    // Takes an item's O^T out of tensor memory, divides by the row sums and writes the output rows, or, for
-    // a (sequence, KV head) pair cut by a range boundary, leaves fp32 partials and merges them if this was
-    // the last of the pair's thread blocks to arrive.  Runs beside the next item's scores and sums.
-    const int ew = warp - W_EPI;
-    const int t = ew * 32 + lane;  // accumulator lane = output column
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(ew * 32) << 16);
-    ItemWalk w;
-    walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
-    Item it;
-    uint32_t gc = 0, item_idx = 0, ep2_uses = 0;
-    bool ok = true;
-    auto meet2 = [&]() -> bool {
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(ep2_bar);
-      const bool r = __all_sync(0xffffffffu, ptx::mbar_wait(ep2_bar, ep2_uses & 1u, abort));
-      ++ep2_uses;
-      return r;
-    };
-    while (ok && walk_next(w, p, it)) {
-      const uint32_t ob = item_idx & 1u, use = item_idx >> 1;
-      gc += (uint32_t)((it.t1 - it.t0 + 1) / 2);
-      const uint32_t b_last = (gc - 1) % PB;  // where the softmax warps left this item's sums
-      if (!__all_sync(0xffffffffu, ptx::mbar_wait(l_ready, item_idx & 1u, abort))) { ok = false; break; }
-      const float* hand = reinterpret_cast<const float*>(p_s + b_last * P_BUF_B + SCR_LSUM);
-      float m_row = 0.f, l_row = 0.f;
-      if (t < NQ) {
-        l_row = hand[t] + hand[64 + t] + hand[128 + t] + hand[192 + t];
-        m_row = hand[256 + t];
-        ltot[ob * 64 + t] = l_row;
-      }
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(l_read);
-      if (!meet2()) { ok = false; break; }  // the row sums are visible to all four warps
-      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&o_done[ob], use & 1u, abort))) { ok = false; break; }
-      ptx::tc_fence_after();
-      const float* lt = ltot + ob * 64;
-      // row q = j*G + g  <->  out[b, q_first + j, h*G + g, :]
-      __nv_bfloat16* out_slab = p.out + (((size_t)it.b * p.q_stride + p.q_first) * p.Hq + it.h * p.G) * HD;
-      const size_t slot_row = (size_t)(blockIdx.x + it.pair) * NQ;
-      // O^T row d = t, 32 stacked query rows at a time: divided by the row sums into the output, or as it is
-      // into this split's partial result
-#pragma unroll
-      for (int q0 = 0; q0 < NQ; q0 += 32) {
-        float o[32];
-#pragma unroll
-        for (int c = 0; c < 2; ++c)
-          ptx::tmem_ld16(lane_addr + O_COL + ob * NQ + q0 + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&o[c * 16]));
-        ptx::tmem_ld_wait();
-        if (q0 + 32 == NQ) {  // everything is in registers: the buffer may take the item after next
-          ptx::tc_fence_before();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(&o_free[ob]);
-        }
-        if (t < HD) {
-          if (it.n_splits == 1) {
-#pragma unroll
-            for (int q = 0; q < 32; ++q)
-              if (q0 + q < GD) out_slab[(size_t)row_hd[q0 + q] * HD + t] = __float2bfloat16_rn(o[q] / lt[q0 + q]);
-          } else {
-#pragma unroll
-            for (int q = 0; q < 32; ++q) p.part_o[(slot_row + q0 + q) * HD + t] = o[q];
-          }
-        }
-      }
-      ++item_idx;
-      if (it.n_splits > 1) {
-        // a row that saw no key in this split (all of them masked) takes no part in the merge
-        if (t < NQ) *reinterpret_cast<float2*>(p.part_ml + (slot_row + t) * 2) = make_float2(l_row > 0.f ? m_row : -INFINITY, l_row);
-        __threadfence();
-        if (!meet2()) { ok = false; break; }
-        if (t == 0) {  // every split of the pair counts once; the last one merges
-          const int arrived = atomicAdd(&p.pair_cnt[it.pair], 1);
-          const int last = arrived == it.n_splits - 1;
-          if (last) p.pair_cnt[it.pair] = 0;
-          *s_last = last;
-        }
-        if (!meet2()) { ok = false; break; }
-        if (*s_last) {
-          // ---- merge the splits of this pair (fixed order: run-to-run identical).  Row q's weight of split
-          // s is 2^(m_s - m) with m = max_s m_s.  A thread owns (row, four columns) units, consecutive threads
-          // consecutive columns of one row; it reads its rows' (m_s, l_s) itself, so nothing is shared.
-          __threadfence();
-          constexpr int C4 = HD / 4, UPT = 8;
-          const size_t first_row = (size_t)(it.c_first + it.pair) * NQ;
-          for (int u0 = 0; u0 < GD * C4; u0 += 128 * UPT) {
-            float m[UPT], L[UPT], a0[UPT], a1[UPT], a2[UPT], a3[UPT];
-            int uq[UPT];
-#pragma unroll
-            for (int i = 0; i < UPT; ++i) {
-              const int u = u0 + i * 128 + t;
-              uq[i] = u < GD * C4 ? u / C4 : -1;
-              m[i] = -INFINITY;
-              L[i] = a0[i] = a1[i] = a2[i] = a3[i] = 0.f;
-            }
-            for (int s = 0; s < it.n_splits; ++s) {
-              const float* ml = p.part_ml + (first_row + (size_t)s * NQ) * 2;
-#pragma unroll
-              for (int i = 0; i < UPT; ++i)
-                if (uq[i] >= 0) m[i] = fmaxf(m[i], __ldcg(ml + uq[i] * 2));
-            }
-            for (int s = 0; s < it.n_splits; ++s) {
-              const float* ml = p.part_ml + (first_row + (size_t)s * NQ) * 2;
-              const float* po = p.part_o + (first_row + (size_t)s * NQ) * HD + 4 * (t % C4);
-#pragma unroll
-              for (int i = 0; i < UPT; ++i) {
-                if (uq[i] >= 0) {
-                  const float2 r = __ldcg(reinterpret_cast<const float2*>(ml + uq[i] * 2));
-                  const float4 v = __ldcg(reinterpret_cast<const float4*>(po + (size_t)uq[i] * HD));
-                  const float a = ptx::ex2(r.x - m[i]);
-                  L[i] = fmaf(a, r.y, L[i]);
-                  a0[i] = fmaf(a, v.x, a0[i]);
-                  a1[i] = fmaf(a, v.y, a1[i]);
-                  a2[i] = fmaf(a, v.z, a2[i]);
-                  a3[i] = fmaf(a, v.w, a3[i]);
-                }
-              }
-            }
-#pragma unroll
-            for (int i = 0; i < UPT; ++i) {
-              if (uq[i] >= 0) {
-                const float inv = 1.0f / L[i];
-                uint2 v;
-                v.x = ptx::pack_bf16(a0[i] * inv, a1[i] * inv);
-                v.y = ptx::pack_bf16(a2[i] * inv, a3[i] * inv);
-                *reinterpret_cast<uint2*>(out_slab + (size_t)row_hd[uq[i]] * HD + 4 * (t % C4)) = v;
-              }
-            }
-          }
-        }
-      }
-    }
-    if (!ok && lane == 0) attn_timeout(p, 6);
   } else {
     // ---------------------------------------------------------------- warp 3: Q rows and the block's own tile
     constexpr int NQC = NQ * (HD / 8) / 32;  // 16-byte chunks of the stacked query rows per lane
@@ -877,9 +530,9 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     Ring ring{0, 0};
     uint32_t blk_idx = 0, item_idx = 0;
     bool ok = true;
-    // At most 16 chunks per lane are kept in registers at a time (more would spill and serialise the
-    // loads): those are fetched one item ahead, the rest (only with 64 stacked rows) when the item starts.
-    constexpr int NQR = NQC < 16 ? NQC : 16;
+    // At most 16 chunks per lane (8 with 64 stacked rows, where this warp has fewer registers) are kept in
+    // registers at a time: those are fetched one item ahead, the rest when the item starts.
+    constexpr int NQR = NQC < 16 ? NQC : (NQ == 64 ? 8 : 16);
     uint4 qreg[NQR];
     // stacked query rows: row r = j*G + g  <->  q[b, q_first + j, h*G + g, :]; rows beyond G*D are zero
     auto fetch_q = [&](const Item& x, int first) {
@@ -901,7 +554,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     bool have = walk_next(w, p, it);
     if (have) fetch_q(it, 0);
     while (ok && have) {
-      if (item_idx > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait(q_free, (item_idx - 1) & 1u, abort))) { ok = false; break; }
+      if (item_idx > 0 && !ptx::mbar_wait_warp_relaxed(q_free, (item_idx - 1) & 1u, abort)) { ok = false; break; }
       store_q(0);
       for (int first = NQR; first < NQC; first += NQR) {
         fetch_q(it, first);
@@ -968,12 +621,334 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     }
     if (!ok && lane == 0) attn_timeout(p, 4);
   }
+  } else if (warp < W_EPI) {
+    ptx::reg_alloc<NQ == 64 ? 160 : 232>();
+    // ---------------------------------------------------------------- softmax: thread = key of the group
+    // Four warps cover the 128 keys of a group; with 64 stacked query rows a second set of four takes the
+    // upper 32 rows, so that no thread handles more than 32 values per group.  These warps never wait
+    // for global memory: an item's results are handed to the epilogue warps and the next item starts.
+    constexpr int QV = 32;                          // query rows (columns of S^T) per thread
+    const int qd = warp & 3;                        // TMEM lane quarter of this warp
+    const int qb = ((warp - 4) >> 2) * 32;          // first query row of this warp's set
+    const int kg = qd * 32 + lane;       // key within the group = accumulator lane
+    const int tj = kg >> 6, kt = kg & 63;  // tile of the group, key within that tile
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(qd * 32) << 16);
+    ItemWalk w;
+    walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
+    Item it;
+    uint32_t gc = 0, item_idx = 0, ep_uses = 0;
+    int lread_buf = -1;  // the P^T buffer that still holds the previous item's hand-off (-1: none, or read)
+    bool ok = true;
+    // all softmax warps meet; false when a wait ran out
+    auto meet = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ep_bar);
+      const bool r = __all_sync(0xffffffffu, ptx::mbar_wait(ep_bar, ep_uses & 1u, abort));
+      ++ep_uses;
+      return r;
+    };
+    while (ok && walk_next(w, p, it)) {
+      float l[QV];  // this key subset's share of every row sum
+#pragma unroll
+      for (int q = 0; q < QV; ++q) l[q] = 0.f;
+      const int n = it.t1 - it.t0, ng = (n + 1) / 2;
+      const uint32_t o_addr = lane_addr + O_COL + (item_idx & 1u) * NQ + qb;  // this item's O^T columns of my rows
+      // which of my 32 query rows see my key if it turns out to be a block key (bit q: row qb + q)
+      [[maybe_unused]] uint32_t visq = 0xffffffffu;
+      if (MASKED && p.vis_kind != kVisNone && it.t1 > it.pages) {
+        visq = 0;
+        int j = qb / p.G, rem = qb % p.G;
+        uint32_t vj = j < p.D ? vis_word(p, it.b, j) : 0u;
+#pragma unroll
+        for (int q = 0; q < QV; ++q) {
+          const uint32_t bit = qb + q < GD ? (kt < 32 ? (vj >> kt) & 1u : 0u) : 1u;  // padding rows: no mask
+          visq |= bit << q;
+          if (++rem == p.G) {
+            rem = 0;
+            ++j;
+            vj = j < p.D ? vis_word(p, it.b, j) : 0u;
+          }
+        }
+      }
+      for (int g = 0; g < ng; ++g, ++gc) {
+        const uint32_t sb = gc & 1u;
+        const bool mine = kt < tile_valid(it, it.t0 + 2 * g + tj, p.Dk);  // does my key exist?
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(&s_full[sb], (gc >> 1) & 1u, abort))) { ok = false; break; }
+        ptx::tc_fence_after();
+        float x[QV];  // my key's score for every one of my rows
+#pragma unroll
+        for (int c = 0; c < QV / 16; ++c)
+          ptx::tmem_ld16(lane_addr + sb * NQ + qb + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&x[c * 16]));
+        ptx::tmem_ld_wait();
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&s_free[sb]);
+        if constexpr (MASKED) {
+          if (visq != 0xffffffffu && it.t0 + 2 * g + tj == it.pages) {  // my key is a block key some rows do not see
+#pragma unroll
+            for (int q = 0; q < QV; ++q)
+              if (!((visq >> q) & 1u)) x[q] = -INFINITY;
+          }
+        }
+
+        const bool first = g == 0;
+        if (first) {
+          // The item's references start at the scores of its first key (which always exists): one thread
+          // per set of rows publishes them, no reduction over keys.  A row that does not see that key
+          // (masked) starts at 0.  Whatever is too low for a later score is moved below, as in any group.
+          if (kg == 0) {
+#pragma unroll
+            for (int q = 0; q < QV; ++q) {
+              const float v = x[q] * p.scale_log2;
+              mref[qb + q] = v > -INFINITY ? v : 0.f;
+            }
+          }
+          if (!meet()) { ok = false; break; }
+        }
+        const uint32_t fi = gc % 3u;
+        if (warp == 4 && lane == 0) flag[(fi + 1u) % 3u] = 0;  // last read two groups ago
+        // Exponents of my key relative to the row references, formed before the warps meet (whoever arrives
+        // early waits anyway) so that only the exponentials and the stores are left after it.
+        float e[QV];
+        float xm = -INFINITY;
+#pragma unroll
+        for (int q4 = 0; q4 < QV; q4 += 4) {
+          const float4 mr = *reinterpret_cast<const float4*>(mref + qb + q4);
+          e[q4] = fmaf(x[q4], p.scale_log2, -mr.x);
+          e[q4 + 1] = fmaf(x[q4 + 1], p.scale_log2, -mr.y);
+          e[q4 + 2] = fmaf(x[q4 + 2], p.scale_log2, -mr.z);
+          e[q4 + 3] = fmaf(x[q4 + 3], p.scale_log2, -mr.w);
+          xm = fmaxf(fmaxf(xm, fmaxf(e[q4], e[q4 + 1])), fmaxf(e[q4 + 2], e[q4 + 3]));
+        }
+        const bool need = mine && xm > kRebaseThreshold;
+        if (__any_sync(0xffffffffu, need) && lane == 0) flag[fi] = 1;
+        if (!meet()) { ok = false; break; }
+        if (flag[fi] != 0) {
+          // ---- move the row references to max(old reference, this group's row maxima).  The scratch
+          // for this sits in the P^T buffers and O^T is about to be rescaled: the previous O^T
+          // instruction must be done (before the first group of an item the previous item's end saw to it).
+          if (!first) {
+            const uint32_t prev = gc - 1;
+            if (!__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[prev % PB], (prev / PB) & 1u, abort))) { ok = false; break; }
+          }
+#pragma unroll
+          for (int q = 0; q < QV; ++q) {
+            const int v = __reduce_max_sync(0xffffffffu, mine ? ordered_int(x[q] * p.scale_log2) : kIntMin);
+            if (lane == q) mx[qd * 64 + qb + q] = v;
+          }
+          if (!meet()) { ok = false; break; }
+#pragma unroll
+          for (int q = 0; q < QV; ++q) {
+            const int gi = max(max(mx[qb + q], mx[64 + qb + q]), max(mx[128 + qb + q], mx[192 + qb + q]));
+            const float m_old = mref[qb + q];
+            const float m_new = gi == kIntMin ? m_old : fmaxf(m_old, ordered_float(gi));
+            const float f = ptx::ex2(m_old - m_new);
+            l[q] *= f;
+            if (kg == q) { mnew[qb + q] = m_new; fbuf[qb + q] = f; }
+          }
+          if (!meet()) { ok = false; break; }  // everybody has read the old references
+          if (kg < QV) mref[qb + kg] = mnew[qb + kg];
+          if (!first) {  // O^T holds sums relative to the old references
+            ptx::tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < QV / 16; ++c) {
+              uint32_t o[16];
+              ptx::tmem_ld16(o_addr + c * 16, o);
+              ptx::tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * fbuf[qb + c * 16 + i]);
+              ptx::tmem_st16(o_addr + c * 16, o);
+            }
+            ptx::tmem_st_wait();
+          }
+          if (!meet()) { ok = false; break; }  // the new references are visible
+#pragma unroll
+          for (int q4 = 0; q4 < QV; q4 += 4) {
+            const float4 mr = *reinterpret_cast<const float4*>(mref + qb + q4);
+            e[q4] = fmaf(x[q4], p.scale_log2, -mr.x);
+            e[q4 + 1] = fmaf(x[q4 + 1], p.scale_log2, -mr.y);
+            e[q4 + 2] = fmaf(x[q4 + 2], p.scale_log2, -mr.z);
+            e[q4 + 3] = fmaf(x[q4 + 3], p.scale_log2, -mr.w);
+          }
+        }
+        // P^T column of my key: 2^(s*scale - reference), rounded to bf16; absent keys give 0
+        const uint32_t pbuf = gc % PB;
+        if (lread_buf == (int)pbuf) {  // the buffer still holds the previous item's hand-off: it must have been read
+          if (!__all_sync(0xffffffffu, ptx::mbar_wait(l_read, (item_idx - 1) & 1u, abort))) { ok = false; break; }
+          lread_buf = -1;
+        }
+        if (gc >= (uint32_t)PB && !__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[pbuf], ((gc / PB) & 1u) ^ 1u, abort))) { ok = false; break; }
+        uint8_t* pcol = p_s + pbuf * P_BUF_B + tj * P_PANEL_B + (kt & 7) * 2;
+        // The weight as the tensor core will see it (bf16), and that same value into the row sum: numerator
+        // and denominator then carry the same rounding, and a lone key weighs exactly 1.
+#pragma unroll
+        for (int q = 0; q < QV; ++q) {
+          const __nv_bfloat16 w = __float2bfloat16_rn(mine ? ptx::ex2(e[q]) : 0.f);
+          l[q] += __bfloat162float(w);
+          *reinterpret_cast<__nv_bfloat16*>(pcol + (qb + q) * 128 + (((kt >> 3) ^ (q & 7)) << 4)) = w;
+        }
+        ptx::fence_proxy_async();
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&p_full[pbuf]);
+      }
+      if (!ok) break;
+
+      // ---- end of item: row sums over this warp's keys (lane q ends up with the warp's sum of row qb + q)
+      {
+        float* v = l;
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+#pragma unroll
+          for (int i = 0; i < off; ++i) {
+            const bool up = (lane & off) != 0;
+            const float send = up ? v[i] : v[i + off], keep = up ? v[i + off] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+          }
+        }
+      }
+      // They go, with the final references, into the P^T buffer of the item's last group once that group's
+      // O^T instruction is done (and the hand-off before this one has been read).
+      const uint32_t last = gc - 1, b_last = last % PB;
+      if (lread_buf >= 0) {
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(l_read, (item_idx - 1) & 1u, abort))) { ok = false; break; }
+        lread_buf = -1;
+      }
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[b_last], (last / PB) & 1u, abort))) { ok = false; break; }
+      float* hand = reinterpret_cast<float*>(p_s + b_last * P_BUF_B + SCR_LSUM);
+      hand[qd * 64 + qb + lane] = l[0];
+      if (kg < QV) hand[256 + qb + kg] = mref[qb + kg];
+      if (!meet()) { ok = false; break; }  // the references are copied before the next item's first key replaces them
+      if (lane == 0) ptx::mbar_arrive(l_ready);
+      lread_buf = (int)b_last;
+      ++item_idx;
+    }
+    if (!ok && lane == 0) attn_timeout(p, 3);
+  } else {
+    ptx::reg_dealloc<NQ == 64 ? 88 : 128>();
+    // ---------------------------------------------------------------- epilogue: thread = output column d
+    // Takes an item's O^T out of tensor memory, divides by the row sums and writes the output rows, or, for
+    // a (sequence, KV head) pair cut by a range boundary, leaves fp32 partials and merges them if this was
+    // the last of the pair's thread blocks to arrive.  Runs beside the next item's scores and sums.
+    const int ew = warp - W_EPI;
+    const int t = ew * 32 + lane;  // accumulator lane = output column
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(ew * 32) << 16);
+    ItemWalk w;
+    walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
+    Item it;
+    uint32_t gc = 0, item_idx = 0, ep2_uses = 0;
+    bool ok = true;
+    auto meet2 = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ep2_bar);
+      const bool r = __all_sync(0xffffffffu, ptx::mbar_wait(ep2_bar, ep2_uses & 1u, abort));
+      ++ep2_uses;
+      return r;
+    };
+    while (ok && walk_next(w, p, it)) {
+      const uint32_t ob = item_idx & 1u, use = item_idx >> 1;
+      gc += (uint32_t)((it.t1 - it.t0 + 1) / 2);
+      const uint32_t b_last = (gc - 1) % PB;  // where the softmax warps left this item's sums
+      if (!ptx::mbar_wait_warp_relaxed(l_ready, item_idx & 1u, abort)) { ok = false; break; }
+      const float* hand = reinterpret_cast<const float*>(p_s + b_last * P_BUF_B + SCR_LSUM);
+      float m_row = 0.f, l_row = 0.f;
+      if (t < NQ) {
+        l_row = hand[t] + hand[64 + t] + hand[128 + t] + hand[192 + t];
+        m_row = hand[256 + t];
+        ltot[ob * 64 + t] = l_row;
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(l_read);
+      if (!meet2()) { ok = false; break; }  // the row sums are visible to all four warps
+      if (!ptx::mbar_wait_warp_relaxed(&o_done[ob], use & 1u, abort)) { ok = false; break; }
+      ptx::tc_fence_after();
+      const float* lt = ltot + ob * 64;
+      // row q = j*G + g  <->  out[b, q_first + j, h*G + g, :]
+      __nv_bfloat16* out_slab = p.out + (((size_t)it.b * p.q_stride + p.q_first) * p.Hq + it.h * p.G) * HD;
+      const size_t slot_row = (size_t)(blockIdx.x + it.pair) * NQ;
+      // O^T row d = t, 32 stacked query rows at a time: divided by the row sums into the output, or as it is
+      // into this split's partial result
+#pragma unroll
+      for (int q0 = 0; q0 < NQ; q0 += 32) {
+        float o[32];
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+          ptx::tmem_ld16(lane_addr + O_COL + ob * NQ + q0 + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&o[c * 16]));
+        ptx::tmem_ld_wait();
+        if (q0 + 32 == NQ) {  // everything is in registers: the buffer may take the item after next
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&o_free[ob]);
+        }
+        if (t < HD) {
+          if (it.n_splits == 1) {
+#pragma unroll
+            for (int q = 0; q < 32; ++q)
+              if (q0 + q < GD) out_slab[(size_t)row_hd[q0 + q] * HD + t] = __float2bfloat16_rn(o[q] / lt[q0 + q]);
+          } else {
+#pragma unroll
+            for (int q = 0; q < 32; ++q) p.part_o[(slot_row + q0 + q) * HD + t] = o[q];
+          }
+        }
+      }
+      ++item_idx;
+      // a row that saw no key in this split (all of them masked) takes no part in the merge
+      if (it.n_splits > 1 && t < NQ)
+        *reinterpret_cast<float2*>(p.part_ml + (slot_row + t) * 2) = make_float2(l_row > 0.f ? m_row : -INFINITY, l_row);
+      // the thread block that holds a pair's first tiles tells the merge kernel where the pair's partials are
+      if (t == 0 && (int)blockIdx.x == it.c_first) p.pair_info[it.pair] = make_int2(it.c_first, it.n_splits);
+    }
+    if (!ok && lane == 0) attn_timeout(p, 6);
+  }
   ptx::tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, TMEM_COLS);
   }
+}
+
+// Merges the partial results of the (sequence, KV head) pairs that a range boundary cut (fixed order:
+// run-to-run identical).  Split s of a pair left, for every stacked query row, its reference m_s, its sum
+// l_s and its unnormalised output row O_s; the row's result is sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s
+// with m = max_s m_s.  One thread block per (pair, eight rows), one thread per (row, four columns): the
+// work of a long sequence's many splits is spread over the whole GPU instead of falling to one thread block.
+constexpr int kMergeRows = 8;
+template <int HD, int NQ>
+__global__ void __launch_bounds__(kMergeRows * (HD / 4)) block_attn_merge_kernel(const AttnParams p) {
+  constexpr int C4 = HD / 4;
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();  // the partials and the pair records come from the attention kernel
+  const int pair = blockIdx.x, b = pair / p.Hkv, h = pair % p.Hkv;
+  const int q = blockIdx.y * kMergeRows + threadIdx.x / C4, c = threadIdx.x % C4;
+  const int2 info = __ldcg(&p.pair_info[pair]);
+  const int n_splits = info.y;
+  if (n_splits <= 1 || q >= p.G * p.D) return;  // written in full by the one thread block that had the pair
+  const size_t first_row = (size_t)(info.x + pair) * NQ + q;
+  const float* ml = p.part_ml + first_row * 2;
+  const float* po = p.part_o + first_row * HD + 4 * c;
+  float m = -INFINITY;
+#pragma unroll 8
+  for (int s = 0; s < n_splits; ++s) m = fmaxf(m, __ldcg(ml + (size_t)s * NQ * 2));
+  float L = 0.f, a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 8
+  for (int s = 0; s < n_splits; ++s) {
+    const float2 r = __ldcg(reinterpret_cast<const float2*>(ml + (size_t)s * NQ * 2));
+    const float4 v = __ldcg(reinterpret_cast<const float4*>(po + (size_t)s * NQ * HD));
+    const float a = ptx::ex2(r.x - m);
+    L = fmaf(a, r.y, L);
+    a0 = fmaf(a, v.x, a0);
+    a1 = fmaf(a, v.y, a1);
+    a2 = fmaf(a, v.z, a2);
+    a3 = fmaf(a, v.w, a3);
+  }
+  const float inv = 1.0f / L;
+  uint2 v;
+  v.x = ptx::pack_bf16(a0 * inv, a1 * inv);
+  v.y = ptx::pack_bf16(a2 * inv, a3 * inv);
+  // row q = j*G + g  <->  out[b, q_first + j, h*G + g, :]
+  __nv_bfloat16* out_row = p.out + (((size_t)b * p.q_stride + p.q_first + q / p.G) * p.Hq + h * p.G + q % p.G) * HD;
+  *reinterpret_cast<uint2*>(out_row + 4 * c) = v;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1002,10 +977,15 @@ static cudaError_t attn_launch_one(sdlm_ctx* ctx, AttnParams& p, cudaStream_t st
   // Beside a kernel that runs as CTA pairs, attention is launched as clusters of two as well (it uses
   // nothing of the cluster): its thread blocks then fill whole pairs of SMs instead of one SM of many pairs.
   if (whole_tpcs && n_cta >= 2) n_cta &= ~1;
-  const cudaError_t e =
+  cudaError_t e =
       whole_tpcs && n_cta >= 2
           ? launch_overlapped_cluster(block_attn_umma_kernel<HD, NQ, MASKED>, dim3(n_cta), dim3(attn_threads(NQ)), smem, st, 2, p)
           : launch_overlapped(block_attn_umma_kernel<HD, NQ, MASKED>, dim3(n_cta), dim3(attn_threads(NQ)), smem, st, p);
+  ctx->launches++;
+  if (e != cudaSuccess) return e;
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  const int row_blocks = (p.G * p.D + kMergeRows - 1) / kMergeRows;
+  e = launch_overlapped(block_attn_merge_kernel<HD, NQ>, dim3(p.batch * p.Hkv, row_blocks), dim3(kMergeRows * (HD / 4)), 0, st, p);
   ctx->launches++;
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -1048,7 +1028,7 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
   p.out = static_cast<__nv_bfloat16*>(out);
   p.part_ml = reinterpret_cast<float*>(ctx->ws + ctx->lay.attn_ml);
   p.part_o = reinterpret_cast<float*>(ctx->ws + ctx->lay.attn_o);
-  p.pair_cnt = reinterpret_cast<int*>(ctx->ws + ctx->lay.attn_cnt);
+  p.pair_info = reinterpret_cast<int2*>(ctx->ws + ctx->lay.attn_cnt);
   p.hdr = ctx->hdr;
   p.scale_log2 = ctx->scale * 1.4426950408889634f;
   p.batch = batch; p.D = D; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.G = ctx->group;

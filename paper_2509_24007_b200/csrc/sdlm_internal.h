@@ -37,7 +37,7 @@ struct WorkspaceLayout {
   size_t lin_part;                                         // float [kLinSplitMax][128][kLinSplitMaxN]
   size_t lm_partials;                                      // float4 [kLmMaxStripes][max_rows]
   size_t attn_ml, attn_o;                                  // split-KV partial (m, l) and O
-  size_t attn_cnt;                                         // per (batch row, KV head) arrival counters
+  size_t attn_cnt;                                         // per (batch row, KV head): first thread block and number of splits
   size_t st_q, st_k, st_v, st_hidden, st_out, st_seq_ids, st_token, st_p, st_ent, st_acc, st_out_tokens;
   size_t total;
   int attn_max_items;

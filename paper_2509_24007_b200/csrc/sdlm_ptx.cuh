@@ -20,6 +20,18 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// ---- register reallocation between warp groups ------------------------------------------------------
+// All four warps of a group (warps 4k .. 4k+3) raise or lower their per-thread register count together;
+// a raise waits until other groups have released enough.  The count is a multiple of 8 in 24..256.
+template <int N>
+__device__ __forceinline__ void reg_alloc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void reg_dealloc() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+
 // ---- mbarrier -------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
@@ -70,6 +82,29 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     }
   }
 }
+// The same for a whole warp whose wait is long and whose wake-up need not be prompt (a warp that takes an
+// item's results at the item's end, a stage that is refilled a group later): only lane 0 polls, with a
+// pause between polls, so that the waiting warp leaves the issue slots of its scheduler to the warps that
+// are working; every lane gets the outcome.  Must be called by the whole warp.
+__device__ __forceinline__ bool mbar_wait_warp_relaxed(uint64_t* bar, uint32_t parity, volatile int* abort) {
+  int ok = 1;
+  if ((threadIdx.x & 31) == 0 && !mbar_try_wait(bar, parity)) {
+    const uint64_t t0 = global_ns();
+    for (uint32_t i = 1;; ++i) {
+      __nanosleep(96);
+      if (mbar_try_wait(bar, parity)) break;
+      if ((i & 15u) == 0) {
+        if (*abort) { ok = 0; break; }
+        if (global_ns() - t0 > kWaitLimitNs) {
+          *abort = 1;
+          ok = 0;
+          break;
+        }
+      }
+    }
+  }
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
 // Same bounds for a plain shared-memory counter that another warp of the CTA increments: returns
 // once *counter > seen.  Unlike an mbarrier parity, a counter cannot be misread by a waiter that is
 // several steps behind or ahead of the signaller.
@@ -77,14 +112,31 @@ __device__ __forceinline__ bool counter_wait(volatile int* counter, int seen, vo
   if (*counter > seen) { __threadfence_block(); return true; }
   const uint64_t t0 = global_ns();
   for (uint32_t i = 1;; ++i) {
+    __nanosleep(96);  // the counter moves once per item: poll at leisure
     if (*counter > seen) { __threadfence_block(); return true; }
-    if ((i & 63u) == 0) {
+    if ((i & 15u) == 0) {
       if (*abort) return false;
       if (global_ns() - t0 > kWaitLimitNs) {
         *abort = 1;
         return false;
       }
-      __nanosleep(32);
+    }
+  }
+}
+// mbar_wait for one thread whose wait is usually long (a ring stage that frees a group later): pauses
+// between polls instead of polling back to back.
+__device__ __forceinline__ bool mbar_wait_paced(uint64_t* bar, uint32_t parity, volatile int* abort) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_ns();
+  for (uint32_t i = 1;; ++i) {
+    __nanosleep(64);
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 15u) == 0) {
+      if (*abort) return false;
+      if (global_ns() - t0 > kWaitLimitNs) {
+        *abort = 1;
+        return false;
+      }
     }
   }
 }
