@@ -72,7 +72,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         self.t.join(timeout=2)
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in self.lines:
             f = [x.strip() for x in ln.split(",")]
@@ -82,11 +82,15 @@ class ClockSampler:
                 sm.append(float(f[0])); mx.append(float(f[1]))
             except ValueError:
                 continue
+            try:
+                pw.append(float(f[2]))
+            except ValueError:
+                pass
             for n, v in zip(names, f[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "power_w": float(np.median(pw)) if pw else None, "reasons": sorted(reasons), "samples": len(sm)}
 
 
 def _blas_threads() -> int:
@@ -258,7 +262,7 @@ def time_workload(torch, dp, wl, steps, warmup, n_blocks=4, use_graph=True, over
         times, tokens, launches, total = [], 0, 0, 0.0
         if clock_sampler is not None:
             clock_sampler.start()
-        while total < min_s * 1e3 and len(times) < MAX_REGIONS:
+        while (total < min_s * 1e3 or not times) and len(times) < MAX_REGIONS:
             barrier()
             launches0 = sd.launch_count()
             ev0.record(stream)
@@ -642,6 +646,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="enqueue every step from the host instead of replaying a CUDA graph")
     ap.add_argument("--no-overlap", action="store_true", help="skip the side-by-side mode (the primary figure is the in-order step either way)")
     ap.add_argument("--no-extra", action="store_true", help="skip the other workloads, the widening measurements and the CPU baseline")
+    ap.add_argument("--min-timed-s", type=float, default=MIN_TIMED_S,
+                    help="repeat the region of --steps steps until this much has been timed (0: one region, for profiling runs)")
     ap.add_argument("--model-level-only", action="store_true",
                     help="run only the whole-model step of the 3B shape and print its figures (for profiling)")
     args = ap.parse_args()
@@ -693,7 +699,7 @@ def main():
     sampler = ClockSampler(local_rank) if rank == 0 else None
     barrier()
     res = time_workload(torch, dp, wl_run, args.steps, args.warmup, use_graph=not args.no_graph, overlap=not args.no_overlap,
-                        reduce_max=reduce_max, barrier=barrier, sampler=sampler)
+                        min_timed_s=args.min_timed_s, reduce_max=reduce_max, barrier=barrier, sampler=sampler)
     barrier()
     e2e = time_e2e(torch, dp, wl_run, max(3, min(args.steps, 100)), 3)
     side = res["side_by_side"]

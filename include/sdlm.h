@@ -435,14 +435,20 @@ sdlm_status sdlm_swiglu(sdlm_ctx* ctx, int32_t rows, int32_t I, const void* gate
  * other SMs (the work is split over fewer thread blocks each, so results agree to rounding, not
  * bit for bit; default 0: one after the other on all SMs).
  * SDLM_OPT_ATTN_ITEM_COST: 0..64, how many cache pages' worth of work the attention schedule
- * charges a thread block for every (sequence, KV head) pair it starts (default 12); results do not
+ * charges a thread block for every (sequence, KV head) pair it starts (default 8); results do not
  * depend on it.  SDLM_OPT_ATTN_MIN_RANGE: 1..4096, the fewest schedule positions (pages plus item
  * costs) one thread block is given, which bounds how finely a short workload is split.
  * SDLM_OPT_HOST_TWO_STREAMS: 1 makes sdlm_decode_step_host, when SDLM_OPT_STEP_OVERLAP is set, copy q / k / v
  * and run attention on a second stream of the context while `hidden` is copied and the LM head runs on the
  * caller's stream (default 0: everything on the caller's stream, in order of need).
+ * SDLM_OPT_ATTN_EARLY_PREFETCH: 0..4096, how many cached K/V tiles (one page of one KV head each) a thread
+ * block of the attention kernel asks the memory system to bring into L2 while it is still waiting for the
+ * kernel before it on the stream (default 0: off; in the decode step measured here it changed nothing, the
+ * step being bound elsewhere).  The cached history is not produced by that
+ * kernel; the tables are read as they stand at that moment and only steer the prefetch: results do not depend
+ * on the option.
  * Errors: INVALID_ARG. */
-typedef enum sdlm_option { SDLM_OPT_LMHEAD_KERNEL = 0, SDLM_OPT_STEP_OVERLAP = 1, SDLM_OPT_ATTN_ITEM_COST = 2, SDLM_OPT_ATTN_MIN_RANGE = 3, SDLM_OPT_HOST_TWO_STREAMS = 4 } sdlm_option;
+typedef enum sdlm_option { SDLM_OPT_LMHEAD_KERNEL = 0, SDLM_OPT_STEP_OVERLAP = 1, SDLM_OPT_ATTN_ITEM_COST = 2, SDLM_OPT_ATTN_MIN_RANGE = 3, SDLM_OPT_HOST_TWO_STREAMS = 4, SDLM_OPT_ATTN_EARLY_PREFETCH = 5 } sdlm_option;
 sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t value);
 
 /* Self-test of the bounded waits (the paper has no counterpart): launches one thread block that waits on

@@ -43,7 +43,7 @@ WorkspaceLayout workspace_layout(const sdlm_config& c) {
   L.attn_max_items = kAttnMaxCtas + c.max_batch * c.n_kv_heads;
   L.attn_ml = take((size_t)L.attn_max_items * L.q_rows_pad * 2 * 4);
   L.attn_o = take((size_t)L.attn_max_items * L.q_rows_pad * c.head_dim * 4);
-  L.attn_cnt = take((size_t)c.max_batch * c.n_kv_heads * 8);
+  L.attn_cnt = take((size_t)c.max_batch * c.n_kv_heads * 12);  // per pair: a record for the merge kernel, an arrival count
   L.st_q = take(rows * c.n_q_heads * c.head_dim * 2);
   L.st_k = take(rows * c.n_kv_heads * c.head_dim * 2);
   L.st_v = take(rows * c.n_kv_heads * c.head_dim * 2);
@@ -485,7 +485,7 @@ static sdlm_status reset_tables(sdlm_ctx* ctx, const int32_t* host_free_list, cu
         cudaSuccess)
       return SDLM_ERR_CUDA;
   }
-  if (cudaMemsetAsync(ctx->ws + ctx->lay.attn_cnt, 0, (size_t)c.max_batch * c.n_kv_heads * 8, st) != cudaSuccess)
+  if (cudaMemsetAsync(ctx->ws + ctx->lay.attn_cnt, 0, (size_t)c.max_batch * c.n_kv_heads * 12, st) != cudaSuccess)
     return SDLM_ERR_CUDA;
   reset_tables_kernel<<<64, 256, 0, st>>>(ctx->hdr, ctx->page_table, ctx->seq_len, ctx->free_list,
                                          c.max_batch * c.max_pages_per_seq, c.max_batch, c.num_pages,
@@ -529,11 +529,14 @@ extern "C" sdlm_status sdlm_create(const sdlm_config* cfg, void* kv_pool, size_t
   ctx->host_two_streams = 0;
   ctx->side_stream = nullptr;
   ctx->ev_fork = ctx->ev_join = nullptr;
-  ctx->attn_item_cost = 12;
+  ctx->attn_item_cost = 8;
   ctx->attn_min_range = 8;
+  ctx->attn_early_prefetch = 0;
   ctx->tmap_w_ptr = nullptr;
   ctx->tmap_w_rows = 0;
   ctx->tmap_h_ptr = nullptr;
+  ctx->defer_merge = 0;
+  ctx->pending_merge_fn = nullptr;
   ctx->tmap_h_rows = ctx->tmap_h_box = 0;
   if (setup_attn(ctx) != cudaSuccess || setup_lmhead(ctx) != cudaSuccess) { delete ctx; return SDLM_ERR_CUDA; }
   sdlm_status s = reset_tables(ctx, nullptr, 0);
@@ -571,6 +574,10 @@ extern "C" sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t v
     case SDLM_OPT_ATTN_MIN_RANGE:
       if (value < 1 || value > 4096) return SDLM_ERR_INVALID_ARG;
       ctx->attn_min_range = value;
+      return SDLM_OK;
+    case SDLM_OPT_ATTN_EARLY_PREFETCH:
+      if (value < 0 || value > 4096) return SDLM_ERR_INVALID_ARG;
+      ctx->attn_early_prefetch = value;
       return SDLM_OK;
     case SDLM_OPT_STEP_OVERLAP:
       if (value < 0 || value >= ctx->sm_count) return SDLM_ERR_INVALID_ARG;
@@ -946,7 +953,7 @@ extern "C" sdlm_status sdlm_device_status(sdlm_ctx* ctx, int32_t* host_out, int3
     const sdlm_config& c = ctx->cfg;
     if (cudaMemsetAsync(ctx->hdr->status, 0, 16, st) != cudaSuccess ||
         cudaMemsetAsync(&ctx->hdr->commit_ticket, 0, 8, st) != cudaSuccess ||
-        cudaMemsetAsync(ctx->ws + ctx->lay.attn_cnt, 0, (size_t)c.max_batch * c.n_kv_heads * 8, st) != cudaSuccess)
+        cudaMemsetAsync(ctx->ws + ctx->lay.attn_cnt, 0, (size_t)c.max_batch * c.n_kv_heads * 12, st) != cudaSuccess)
       return SDLM_ERR_CUDA;
   }
   if (cudaStreamSynchronize(st) != cudaSuccess) return SDLM_ERR_CUDA;
@@ -977,9 +984,13 @@ static sdlm_status decode_step_device(sdlm_ctx* ctx, int32_t batch, int32_t D, c
   if (s != SDLM_OK) return s;
   const int a_sms = ctx->overlap_lmhead;
   // with more than 128 rows the LM head runs as CTA pairs: attention then takes whole pairs of SMs
-  if (launch_block_attn(ctx, batch, D, seq_ids, q, k_blk, v_blk, attn_out, static_cast<cudaStream_t>(stream), a_sms,
-                        a_sms > 0 && batch * D > 128) != cudaSuccess)
-    return SDLM_ERR_CUDA;
+  // side by side, the LM-head kernel has to be the launch right after attention: the merge of attention's
+  // split partials (which nothing in this step reads) then follows the LM head
+  ctx->defer_merge = a_sms > 0;
+  const cudaError_t ae = launch_block_attn(ctx, batch, D, seq_ids, q, k_blk, v_blk, attn_out, static_cast<cudaStream_t>(stream),
+                                           a_sms, a_sms > 0 && batch * D > 128);
+  ctx->defer_merge = 0;
+  if (ae != cudaSuccess) return SDLM_ERR_CUDA;
   // Attention writes none of the LM head's inputs, so the LM head never waits for it before it starts:
   // side by side it runs from the beginning, in order its thread blocks stream weights from the moment
   // attention's leave their SMs, not from the moment the slowest of them is done.  (In order, attention
@@ -987,6 +998,7 @@ static sdlm_status decode_step_device(sdlm_ctx* ctx, int32_t batch, int32_t D, c
   s = launch_lmhead(ctx, batch * D, hidden, w_lm, token, p_top1, entropy, nullptr, nullptr,
                     static_cast<cudaStream_t>(stream), /*independent_of_predecessor=*/true,
                     a_sms > 0 ? ctx->sm_count - a_sms : 0);
+  if (launch_pending_merge(ctx, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SDLM_ERR_CUDA;
   if (s != SDLM_OK) return s;
   return accept_commit_launch(ctx, batch, D, seq_ids, tau, mode, token, p_top1, entropy, k_blk, v_blk, accepted_len,
                               out_tokens, copies, stream);
@@ -1090,15 +1102,18 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
   void* m_attn = mapped16(attn_out_host);
   void* d_attn = m_attn ? m_attn : ws + L.st_out;
   const int overlap = ctx->overlap_lmhead;  // A: attention's SMs in the side-by-side step (0: in order)
-  if (launch_block_attn(ctx, batch, D, seq_ids, in_q, in_k, in_v, d_attn, qkv_st, overlap, overlap > 0 && batch * D > 128) !=
-      cudaSuccess)
-    return SDLM_ERR_CUDA;
+  ctx->defer_merge = overlap > 0 && a_sms == 0;  // side by side on one stream: the merge follows the LM head
+  const cudaError_t ae =
+      launch_block_attn(ctx, batch, D, seq_ids, in_q, in_k, in_v, d_attn, qkv_st, overlap, overlap > 0 && batch * D > 128);
+  ctx->defer_merge = 0;
+  if (ae != cudaSuccess) return SDLM_ERR_CUDA;
   if (a_sms > 0 && cudaEventRecord(ctx->ev_join, qkv_st) != cudaSuccess) return SDLM_ERR_CUDA;
   // on one stream the LM head follows attention and does not wait for it (attention has waited for the
   // copy of `hidden` before it lets the LM head go); on two streams it follows the copy of `hidden`
   // and takes its wait as a full dependency
   s = launch_lmhead(ctx, batch * D, ws + L.st_hidden, w_lm, d_token, d_p, d_ent, nullptr, nullptr, st,
                     /*independent_of_predecessor=*/a_sms == 0, overlap > 0 ? ctx->sm_count - overlap : 0);
+  if (launch_pending_merge(ctx, st) != cudaSuccess) return SDLM_ERR_CUDA;
   if (s != SDLM_OK) return s;
   if (a_sms > 0 && cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return SDLM_ERR_CUDA;
   int32_t* m_acc = static_cast<int32_t*>(mapped(accepted_len_host));

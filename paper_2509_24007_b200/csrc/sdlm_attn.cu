@@ -30,6 +30,8 @@
 #include "sdlm_internal.h"
 #include "sdlm_ptx.cuh"
 
+#include <string.h>
+
 namespace sdlm {
 
 struct AttnParams {
@@ -43,10 +45,17 @@ struct AttnParams {
   __nv_bfloat16* out;
   float* part_ml;  // [slot][row][2]  (reference max in log2 units, sum)
   float* part_o;   // [slot][row][d]
-  int2* pair_info; // [batch * Hkv] (first thread block, number of thread blocks) of every pair, for the merge kernel
+  // [batch * Hkv] per (sequence, KV head) pair: for kernels that merge their splits themselves, how many of
+  // the pair's splits have arrived (zero between launches); for the others, (first thread block, number of
+  // thread blocks), left for the merge kernel.
+  int* pair_cnt;
+  int2* pair_info;
   DevHeader* hdr;
   float scale_log2;  // softmax scale * log2(e)
   int batch, D, Hq, Hkv, G, mpps, num_pages, n_stages;
+  int max_slots;  // sequence slots of the context
+  // cached tiles (per thread block) to pull towards L2 while the kernel still waits for its predecessor (0: none)
+  int early_prefetch;
   int min_range;  // shortest range of positions worth a CTA of its own
   int item_cost;  // what starting a (sequence, KV head) pair costs a CTA, in tiles (see ItemWalk)
   int release_first;  // let the next kernel on the stream start before this one has waited for the one before it
@@ -72,6 +81,14 @@ struct AttnParams {
 };
 
 enum { kVisNone = 0, kVisWords = 1, kVisVerify = 2, kVisCarry = 3 };
+
+// Who merges the partial results of a pair cut by a range boundary.  With 32 stacked rows the last of the
+// pair's thread blocks to arrive does it in its epilogue warps: few bytes, no further launch, and the next
+// kernel on the stream is not held up by one.  With 64 rows (and the long sequences that come with large
+// blocks) the partials of one pair run to hundreds of KB, too much for four warps of one thread block: a
+// merge kernel spreads them over the GPU.
+template <int NQ>
+constexpr bool kMergeInKernel = NQ == 32;
 
 // Visibility word of query position j (of this launch) of batch row b: bit t set when it sees block key t.
 //   verification (Sec. 3.4): position jj sees the real tokens before it and the mask at its own position;
@@ -177,6 +194,43 @@ __device__ __forceinline__ bool walk_next(ItemWalk& w, const AttnParams& p, Item
   return false;
 }
 
+// Warp-wide: exclusive prefix sum over the batch of (item cost + pages + 1), the lengths and the slots, into
+// shared memory (layout of ItemWalk).  EARLY: called before the kernel has waited for its predecessor, with
+// loads that bypass L1, on tables that the predecessor may still be changing; whatever it reads then is
+// only used to choose what to prefetch.
+template <bool EARLY>
+__device__ __forceinline__ void build_schedule(const AttnParams& p, int* s_first, int lane) {
+  int carry = 0;
+  for (int base = 0; base < p.batch; base += 32) {
+    const int i = base + lane;
+    int n = 0;
+    if (i < p.batch) {
+      int slot, len;
+      if (EARLY) {
+        slot = p.seq_ids ? __ldcg(p.seq_ids + i) : i;
+        slot = min(max(slot, 0), p.max_slots - 1);
+        len = __ldcg(p.seq_len + slot);
+        if (p.prefix_len) len = min(len, __ldcg(p.prefix_len + i));
+        len = max(0, min(len, p.mpps * kPageSize));
+      } else {
+        slot = attn_slot(p, i);
+        len = attn_len(p, i);
+      }
+      s_first[p.batch + 1 + i] = len;
+      s_first[2 * p.batch + 1 + i] = slot;
+      n = (len + kPageSize - 1) / kPageSize + 1 + p.item_cost;
+    }
+    int incl = n;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (i < p.batch) s_first[i] = carry + incl - n;
+    carry += __shfl_sync(0xffffffffu, incl, 31);
+  }
+  if (lane == 0) s_first[p.batch] = carry;
+}
+
 // Ring position of the n-th tile this CTA pushes through its stages.
 struct Ring {
   int stage;
@@ -251,6 +305,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
   uint64_t* drain = l_read + 1;         // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 2);
   volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* s_last = abort + 1;    // epilogue: this thread block arrived last at the pair it just finished
   volatile int* blk_go = abort + 2;     // warp 0 -> warp 3: block-tile ring slots that are free so far
   volatile int* flag = abort + 3;       // [3] "some score outgrew its reference", by group mod 3
   float* mref = reinterpret_cast<float*>(const_cast<int*>(abort) + 7);  // [64] row references (log2 units); 16-byte aligned
@@ -304,6 +359,33 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
   // side-by-side step lets its LM-head kernel go first: that kernel reads nothing a predecessor wrote
   // and takes its own wait before it writes.
   if (p.release_first) ptx::grid_dep_launch();
+  // A thread block of this kernel is often resident long before its predecessor on the stream is done (the
+  // kernels in front of it in a decode step finish SM by SM), with the memory system idle.  The cached K/V of
+  // the history is not something that predecessor produces, so the time is used to pull this thread block's
+  // share of it towards L2: the tables are read as they stand (possibly about to change: lengths only grow,
+  // by a few tokens), the schedule is worked out from them exactly as it will be after the wait, and every
+  // tile it names is prefetched (page ids checked against the pool; a prefetch changes nothing but timing).
+  if (p.early_prefetch > 0) {
+    if (warp == 0) build_schedule<true>(p, s_first, lane);
+    __syncthreads();
+    ItemWalk w;
+    walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
+    Item it;
+    const int n_warps = blockDim.x >> 5;
+    int idx = 0;
+    while (idx < p.early_prefetch && walk_next(w, p, it)) {
+      const int n_cached = min(min(it.t1, it.pages) - it.t0, p.early_prefetch - idx);
+      for (int k = warp - idx % n_warps + (warp < idx % n_warps ? n_warps : 0); k < n_cached; k += n_warps) {
+        if (lane == 0) {
+          const int page = __ldcg(p.page_table + (size_t)it.slot * p.mpps + it.t0 + k);
+          if (page >= 0 && page < p.num_pages)
+            ptx::bulk_prefetch_l2(p.pool + kv_tile_offset(page, it.h, 0, p.Hkv, HD), (uint32_t)TILE_B);
+        }
+      }
+      idx += max(n_cached, 0);
+    }
+    __syncthreads();  // the schedule in shared memory is rebuilt after the wait
+  }
   ptx::grid_dep_wait();
   if (!p.release_first) ptx::grid_dep_launch();
   // The start-up chain is lengths -> page table -> first tiles (and query rows), each a trip to DRAM
@@ -332,27 +414,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
   }
 
   // exclusive prefix sum of (pages + 1) per batch row
-  if (warp == 0) {
-    int carry = 0;
-    for (int base = 0; base < p.batch; base += 32) {
-      const int i = base + lane;
-      int n = 0;
-      if (i < p.batch) {
-        const int len = attn_len(p, i);
-        s_first[p.batch + 1 + i] = len;
-        s_first[2 * p.batch + 1 + i] = attn_slot(p, i);
-        n = (len + kPageSize - 1) / kPageSize + 1 + p.item_cost;
-      }
-      int incl = n;
-      for (int o = 1; o < 32; o <<= 1) {
-        const int v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-      }
-      if (i < p.batch) s_first[i] = carry + incl - n;
-      carry += __shfl_sync(0xffffffffu, incl, 31);
-    }
-    if (lane == 0) s_first[p.batch] = carry;
-  }
+  if (warp == 0) build_schedule<false>(p, s_first, lane);
   // stacked row r = j*G + g is q[b, j, h*G + g, :] (and the same row of out): (j*Hq + g) * d elements into the slab
   if (tid >= 64 && tid < 128) row_hd[tid - 64] = tid - 64 < GD ? (uint16_t)(((tid - 64) / p.G) * p.Hq + (tid - 64) % p.G) : (uint16_t)0xffff;
   ptx::tc_fence_before();
@@ -895,8 +957,78 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       // a row that saw no key in this split (all of them masked) takes no part in the merge
       if (it.n_splits > 1 && t < NQ)
         *reinterpret_cast<float2*>(p.part_ml + (slot_row + t) * 2) = make_float2(l_row > 0.f ? m_row : -INFINITY, l_row);
-      // the thread block that holds a pair's first tiles tells the merge kernel where the pair's partials are
-      if (t == 0 && (int)blockIdx.x == it.c_first) p.pair_info[it.pair] = make_int2(it.c_first, it.n_splits);
+      if constexpr (kMergeInKernel<NQ>) {
+        if (it.n_splits > 1) {
+          // ---- 32 stacked rows: the last of the pair's thread blocks to arrive merges the splits here (fixed
+          // order: run-to-run identical; nobody waits).  Row q's weight of split s is 2^(m_s - m) with
+          // m = max_s m_s.  A thread owns eight (row, four columns) units, consecutive threads consecutive
+          // columns of one row; it reads its rows' (m_s, l_s) itself, so nothing is shared.
+          __threadfence();
+          if (!meet2()) { ok = false; break; }
+          if (t == 0) {  // every split of the pair counts once
+            const int arrived = atomicAdd(&p.pair_cnt[it.pair], 1);
+            const int last = arrived == it.n_splits - 1;
+            if (last) p.pair_cnt[it.pair] = 0;  // zero between launches
+            *s_last = last;
+          }
+          if (!meet2()) { ok = false; break; }
+          if (*s_last) {
+            __threadfence();
+            constexpr int C4 = HD / 4, UPT = 8;
+            const size_t first_row = (size_t)(it.c_first + it.pair) * NQ;
+            for (int u0 = 0; u0 < GD * C4; u0 += 128 * UPT) {
+              float m[UPT], L[UPT], a0[UPT], a1[UPT], a2[UPT], a3[UPT];
+              int uq[UPT];
+#pragma unroll
+              for (int i = 0; i < UPT; ++i) {
+                const int u = u0 + i * 128 + t;
+                uq[i] = u < GD * C4 ? u / C4 : -1;
+                m[i] = -INFINITY;
+                L[i] = a0[i] = a1[i] = a2[i] = a3[i] = 0.f;
+              }
+#pragma unroll 4
+              for (int s = 0; s < it.n_splits; ++s) {
+                const float* ml = p.part_ml + (first_row + (size_t)s * NQ) * 2;
+#pragma unroll
+                for (int i = 0; i < UPT; ++i)
+                  if (uq[i] >= 0) m[i] = fmaxf(m[i], __ldcg(ml + uq[i] * 2));
+              }
+#pragma unroll 2
+              for (int s = 0; s < it.n_splits; ++s) {
+                const float* ml = p.part_ml + (first_row + (size_t)s * NQ) * 2;
+                const float* po = p.part_o + (first_row + (size_t)s * NQ) * HD + 4 * (t % C4);
+#pragma unroll
+                for (int i = 0; i < UPT; ++i) {
+                  if (uq[i] >= 0) {
+                    const float2 r = __ldcg(reinterpret_cast<const float2*>(ml + uq[i] * 2));
+                    const float4 v = __ldcg(reinterpret_cast<const float4*>(po + (size_t)uq[i] * HD));
+                    const float a = ptx::ex2(r.x - m[i]);
+                    L[i] = fmaf(a, r.y, L[i]);
+                    a0[i] = fmaf(a, v.x, a0[i]);
+                    a1[i] = fmaf(a, v.y, a1[i]);
+                    a2[i] = fmaf(a, v.z, a2[i]);
+                    a3[i] = fmaf(a, v.w, a3[i]);
+                  }
+                }
+              }
+#pragma unroll
+              for (int i = 0; i < UPT; ++i) {
+                if (uq[i] >= 0) {
+                  const float inv = 1.0f / L[i];
+                  uint2 v;
+                  v.x = ptx::pack_bf16(a0[i] * inv, a1[i] * inv);
+                  v.y = ptx::pack_bf16(a2[i] * inv, a3[i] * inv);
+                  *reinterpret_cast<uint2*>(out_slab + (size_t)row_hd[uq[i]] * HD + 4 * (t % C4)) = v;
+                }
+              }
+            }
+          }
+        }
+      } else {
+        // 64 stacked rows: the merge kernel does it; the thread block that holds a pair's first tiles tells it
+        // where the pair's partials are
+        if (t == 0 && (int)blockIdx.x == it.c_first) p.pair_info[it.pair] = make_int2(it.c_first, it.n_splits);
+      }
     }
     if (!ok && lane == 0) attn_timeout(p, 6);
   }
@@ -911,44 +1043,69 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
 // Merges the partial results of the (sequence, KV head) pairs that a range boundary cut (fixed order:
 // run-to-run identical).  Split s of a pair left, for every stacked query row, its reference m_s, its sum
 // l_s and its unnormalised output row O_s; the row's result is sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s
-// with m = max_s m_s.  One thread block per (pair, eight rows), one thread per (row, four columns): the
-// work of a long sequence's many splits is spread over the whole GPU instead of falling to one thread block.
-constexpr int kMergeRows = 8;
+// with m = max_s m_s.  The work of a long sequence's many splits is spread over the whole GPU instead of
+// falling to one thread block.  Thread blocks are single warps with few registers: launched as a programmatic
+// dependent they sit waiting on SMs that the attention kernel has left, and at most 32 of them fit on an SM,
+// which leaves the threads, registers and all the shared memory that the kernel after this one needs to
+// start there too.  A thread owns two (row, four columns) units.
+constexpr int kMergeUnits = 2;
 template <int HD, int NQ>
-__global__ void __launch_bounds__(kMergeRows * (HD / 4)) block_attn_merge_kernel(const AttnParams p) {
-  constexpr int C4 = HD / 4;
+__global__ void __maxnreg__(40) block_attn_merge_kernel(const AttnParams p) {
+  constexpr int C4 = HD / 4, ROWS = 32 * kMergeUnits / C4;  // rows per warp: 2 (d = 128) or 4 (d = 64)
   ptx::grid_dep_launch();
   ptx::grid_dep_wait();  // the partials and the pair records come from the attention kernel
   const int pair = blockIdx.x, b = pair / p.Hkv, h = pair % p.Hkv;
-  const int q = blockIdx.y * kMergeRows + threadIdx.x / C4, c = threadIdx.x % C4;
   const int2 info = __ldcg(&p.pair_info[pair]);
   const int n_splits = info.y;
-  if (n_splits <= 1 || q >= p.G * p.D) return;  // written in full by the one thread block that had the pair
-  const size_t first_row = (size_t)(info.x + pair) * NQ + q;
-  const float* ml = p.part_ml + first_row * 2;
-  const float* po = p.part_o + first_row * HD + 4 * c;
-  float m = -INFINITY;
-#pragma unroll 8
-  for (int s = 0; s < n_splits; ++s) m = fmaxf(m, __ldcg(ml + (size_t)s * NQ * 2));
-  float L = 0.f, a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+  if (n_splits <= 1) return;  // written in full by the one thread block that had the pair
+  const int GD = p.G * p.D;
+  int q[kMergeUnits], c[kMergeUnits];
+  float m[kMergeUnits], L[kMergeUnits], a0[kMergeUnits], a1[kMergeUnits], a2[kMergeUnits], a3[kMergeUnits];
+#pragma unroll
+  for (int i = 0; i < kMergeUnits; ++i) {
+    const int u = i * 32 + threadIdx.x;
+    q[i] = blockIdx.y * ROWS + u / C4;
+    c[i] = u % C4;
+    if (q[i] >= GD) q[i] = -1;
+    m[i] = -INFINITY;
+    L[i] = a0[i] = a1[i] = a2[i] = a3[i] = 0.f;
+  }
+  const size_t first_row = (size_t)(info.x + pair) * NQ;
 #pragma unroll 8
   for (int s = 0; s < n_splits; ++s) {
-    const float2 r = __ldcg(reinterpret_cast<const float2*>(ml + (size_t)s * NQ * 2));
-    const float4 v = __ldcg(reinterpret_cast<const float4*>(po + (size_t)s * NQ * HD));
-    const float a = ptx::ex2(r.x - m);
-    L = fmaf(a, r.y, L);
-    a0 = fmaf(a, v.x, a0);
-    a1 = fmaf(a, v.y, a1);
-    a2 = fmaf(a, v.z, a2);
-    a3 = fmaf(a, v.w, a3);
+#pragma unroll
+    for (int i = 0; i < kMergeUnits; ++i)
+      if (q[i] >= 0) m[i] = fmaxf(m[i], __ldcg(p.part_ml + (first_row + (size_t)s * NQ + q[i]) * 2));
   }
-  const float inv = 1.0f / L;
-  uint2 v;
-  v.x = ptx::pack_bf16(a0 * inv, a1 * inv);
-  v.y = ptx::pack_bf16(a2 * inv, a3 * inv);
-  // row q = j*G + g  <->  out[b, q_first + j, h*G + g, :]
-  __nv_bfloat16* out_row = p.out + (((size_t)b * p.q_stride + p.q_first + q / p.G) * p.Hq + h * p.G + q % p.G) * HD;
-  *reinterpret_cast<uint2*>(out_row + 4 * c) = v;
+#pragma unroll 4
+  for (int s = 0; s < n_splits; ++s) {
+#pragma unroll
+    for (int i = 0; i < kMergeUnits; ++i) {
+      if (q[i] >= 0) {
+        const size_t row = first_row + (size_t)s * NQ + q[i];
+        const float2 r = __ldcg(reinterpret_cast<const float2*>(p.part_ml + row * 2));
+        const float4 v = __ldcg(reinterpret_cast<const float4*>(p.part_o + row * HD + 4 * c[i]));
+        const float a = ptx::ex2(r.x - m[i]);
+        L[i] = fmaf(a, r.y, L[i]);
+        a0[i] = fmaf(a, v.x, a0[i]);
+        a1[i] = fmaf(a, v.y, a1[i]);
+        a2[i] = fmaf(a, v.z, a2[i]);
+        a3[i] = fmaf(a, v.w, a3[i]);
+      }
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kMergeUnits; ++i) {
+    if (q[i] >= 0) {
+      const float inv = 1.0f / L[i];
+      uint2 v;
+      v.x = ptx::pack_bf16(a0[i] * inv, a1[i] * inv);
+      v.y = ptx::pack_bf16(a2[i] * inv, a3[i] * inv);
+      // row q = j*G + g  <->  out[b, q_first + j, h*G + g, :]
+      __nv_bfloat16* out_row = p.out + (((size_t)b * p.q_stride + p.q_first + q[i] / p.G) * p.Hq + h * p.G + q[i] % p.G) * HD;
+      *reinterpret_cast<uint2*>(out_row + 4 * c[i]) = v;
+    }
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -962,6 +1119,21 @@ static int attn_fixed_smem(int batch) {
   const int p_buffers = (HD == 128 && NQ == 64) ? 1 : 2;
   return 1024 + (HD / 64) * NQ * 128 + p_buffers * 2 * NQ * 128 + 20 * 8 + 32 + 4 * 64 * 4 + 64 * 2 + (batch + 1) * 12 + 16 +
          (HD == 64 ? 8192 : 0);
+}
+
+template <int HD, int NQ>
+static cudaError_t merge_launch_params(sdlm_ctx* ctx, const AttnParams& p, cudaStream_t st) {
+  const int rows_per_warp = 32 * kMergeUnits / (HD / 4);
+  const cudaError_t e = launch_overlapped(block_attn_merge_kernel<HD, NQ>,
+                                          dim3(p.batch * p.Hkv, (p.G * p.D + rows_per_warp - 1) / rows_per_warp), dim3(32), 0, st, p);
+  ctx->launches++;
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+template <int HD, int NQ>
+static cudaError_t merge_launch(sdlm_ctx* ctx, cudaStream_t st) {
+  AttnParams p;
+  memcpy(&p, ctx->pending_merge, sizeof(AttnParams));
+  return merge_launch_params<HD, NQ>(ctx, p, st);
 }
 
 template <int HD, int NQ, bool MASKED = false>
@@ -984,10 +1156,21 @@ static cudaError_t attn_launch_one(sdlm_ctx* ctx, AttnParams& p, cudaStream_t st
   ctx->launches++;
   if (e != cudaSuccess) return e;
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  const int row_blocks = (p.G * p.D + kMergeRows - 1) / kMergeRows;
-  e = launch_overlapped(block_attn_merge_kernel<HD, NQ>, dim3(p.batch * p.Hkv, row_blocks), dim3(kMergeRows * (HD / 4)), 0, st, p);
-  ctx->launches++;
-  return e != cudaSuccess ? e : cudaGetLastError();
+  if (kMergeInKernel<NQ>) return cudaSuccess;
+  if (ctx->defer_merge) {  // the caller launches it after the kernel that runs beside attention
+    static_assert(sizeof(AttnParams) <= sizeof(ctx->pending_merge), "room for the held-back merge's parameters");
+    memcpy(ctx->pending_merge, &p, sizeof(AttnParams));
+    ctx->pending_merge_fn = &merge_launch<HD, NQ>;
+    return cudaSuccess;
+  }
+  return merge_launch_params<HD, NQ>(ctx, p, st);
+}
+
+cudaError_t launch_pending_merge(sdlm_ctx* ctx, cudaStream_t st) {
+  if (!ctx->pending_merge_fn) return cudaSuccess;
+  cudaError_t (*fn)(sdlm_ctx*, cudaStream_t) = ctx->pending_merge_fn;
+  ctx->pending_merge_fn = nullptr;
+  return fn(ctx, st);
 }
 
 cudaError_t setup_attn(sdlm_ctx* ctx) {
@@ -1029,12 +1212,15 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
   p.part_ml = reinterpret_cast<float*>(ctx->ws + ctx->lay.attn_ml);
   p.part_o = reinterpret_cast<float*>(ctx->ws + ctx->lay.attn_o);
   p.pair_info = reinterpret_cast<int2*>(ctx->ws + ctx->lay.attn_cnt);
+  p.pair_cnt = reinterpret_cast<int*>(ctx->ws + ctx->lay.attn_cnt + (size_t)c.max_batch * c.n_kv_heads * 8);
   p.hdr = ctx->hdr;
   p.scale_log2 = ctx->scale * 1.4426950408889634f;
   p.batch = batch; p.D = D; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.G = ctx->group;
   p.mpps = c.max_pages_per_seq; p.num_pages = c.num_pages; p.n_stages = 0;
   p.item_cost = ctx->attn_item_cost;
   p.min_range = ctx->attn_min_range;
+  p.max_slots = c.max_batch;
+  p.early_prefetch = ctx->attn_early_prefetch;
   p.release_first = cta_cap > 0 ? 1 : 0;
   p.Dk = n_blk_keys > 0 ? n_blk_keys : D;
   p.vis = vis;

@@ -37,7 +37,7 @@ struct WorkspaceLayout {
   size_t lin_part;                                         // float [kLinSplitMax][128][kLinSplitMaxN]
   size_t lm_partials;                                      // float4 [kLmMaxStripes][max_rows]
   size_t attn_ml, attn_o;                                  // split-KV partial (m, l) and O
-  size_t attn_cnt;                                         // per (batch row, KV head): first thread block and number of splits
+  size_t attn_cnt;                                         // per (batch row, KV head): record for the merge kernel, arrival count
   size_t st_q, st_k, st_v, st_hidden, st_out, st_seq_ids, st_token, st_p, st_ent, st_acc, st_out_tokens;
   size_t total;
   int attn_max_items;
@@ -66,6 +66,7 @@ struct sdlm_ctx {
   int lmhead_path;  // 0 = pick by shape, 1 = force the mma.sync kernel, 2 = force the tcgen05 kernel
   int attn_min_range;  // shortest range of schedule positions given to one attention thread block
   int attn_item_cost;  // positions the attention schedule charges for starting a (sequence, KV head) pair
+  int attn_early_prefetch;  // cached tiles per thread block that attention prefetches before its dependency wait (0: off)
   int overlap_lmhead;  // sdlm_decode_step: SMs given to attention while the LM head runs on the rest (0: one after the other)
   // second stream and fork / join events of the host-buffer step's side-by-side mode (made on first use)
   int host_two_streams;
@@ -75,6 +76,12 @@ struct sdlm_ctx {
   const void* tmap_w_ptr;
   int tmap_w_rows;
   alignas(64) unsigned char tmap_w[128];
+  // Attention's merge of split partials, held back (side-by-side step: the kernel that runs beside attention
+  // has to be the very next launch, so the merge follows it): set defer_merge before the attention launch,
+  // call launch_pending_merge after the launch in between.
+  int defer_merge;
+  cudaError_t (*pending_merge_fn)(sdlm_ctx*, cudaStream_t);
+  alignas(16) unsigned char pending_merge[256];
   // and of the LM head's hidden-state rows (keyed by pointer, rows and box rows)
   const void* tmap_h_ptr;
   int tmap_h_rows, tmap_h_box;
@@ -174,6 +181,7 @@ sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, 
                           void* out2 = nullptr, void* out3 = nullptr, int act = 0, const LinNorm* norm = nullptr);
 cudaError_t launch_rmsnorm(sdlm_ctx* ctx, int rows, int H, const void* x, const void* weight, float eps, void* out,
                            cudaStream_t st);
+cudaError_t launch_pending_merge(sdlm_ctx* ctx, cudaStream_t st);
 cudaError_t setup_attn(sdlm_ctx* ctx);
 cudaError_t setup_lmhead(sdlm_ctx* ctx);
 
