@@ -541,6 +541,74 @@ def time_noise_blocks(torch, pk, DeviceProblem, shape, n_target=4096, n_blocks=6
                     "lower triangle only" % (n_target * row_b / 1e6)}
 
 
+def attention_timeline(torch, wl, flush_l2=False, reps=6):
+    """Wall-clock marks inside the attention kernel of the in-order step, from the library built with
+    `python paper_2509_24007_b200/build.py --timeline`.  Steps are enqueued back to back (one sdlm_decode_step
+    call each, no events between them); the marks are those of the last step's attention launch, in
+    microseconds after the moment its dependency wait returned (the commit of the step before is complete),
+    as the median and the maximum over the thread blocks.  flush_l2: attention calls alone, back to back,
+    with a buffer larger than L2 written between them (cold) or not (warm), to separate cold-cache start-up
+    from the rest."""
+    import ctypes
+    import paper_2509_24007_b200.binding as b
+    from paper_2509_24007_b200 import build
+    from paper_2509_24007_b200.harness import DeviceProblem
+    if not os.path.exists(build.LIB_TIMELINE):
+        build.build(timeline=True)
+    b.LIB_PATH, b._lib = build.LIB_TIMELINE, None
+    dp = DeviceProblem(wl, keep_prefix=False)
+    sd = dp.sd
+    sd.lib.sdlm_timeline_read.argtypes = [ctypes.c_void_p]
+    blocks = [dp.block(i) for i in range(4)]
+    out = dp.alloc_outputs()
+    saved = sd.kv_save()
+    buf = np.zeros((160, 16), dtype=np.uint64)
+    names = {0: "resident", 2: "roles_start", 9: "first_copies_issued", 8: "query_rows_staged", 3: "first_tiles_and_q",
+             4: "first_p", 5: "last_p", 6: "epilogue_done", 7: "block_done"}
+
+    def step(i):
+        x = blocks[i % 4]
+        sd.decode_step(wl.tau, x.q, x.k_blk, x.v_blk, x.hidden, dp.w_lm, out.attn, out.token, out.p_top1, out.entropy,
+                       out.accepted_len, out.out_tokens)
+
+    def read():
+        assert sd.lib.sdlm_timeline_read(buf.ctypes.data) == 0
+        t = buf.astype(np.int64)
+        act = t[:, 7] > 0
+        t0 = t[act, 1].min()
+        return {n: [round(float(np.median((t[act, c] - t0) / 1e3)), 1), round(float(((t[act, c] - t0) / 1e3).max()), 1)]
+                for c, n in names.items()} | {"thread_blocks": int(act.sum()),
+                                              "resident_before_release_us": [round(float(((t0 - t[act, 0]) / 1e3).min()), 1),
+                                                                             round(float(np.median((t0 - t[act, 0]) / 1e3)), 1),
+                                                                             round(float(((t0 - t[act, 0]) / 1e3).max()), 1)]}
+
+    rows = {"in_step": [], "alone_warm": [], "alone_l2_flushed": []}
+    for i in range(40):
+        if i % RESTORE_EVERY == 0:
+            sd.kv_restore(saved)
+        step(i)
+    for _ in range(reps):
+        sd.kv_restore(saved)
+        for i in range(7):
+            step(i)
+        rows["in_step"].append(read())
+    if flush_l2:
+        big = torch.empty(300 << 20, dtype=torch.uint8, device=sd.device)
+        for mode in ("alone_warm", "alone_l2_flushed"):
+            for _ in range(reps):
+                for i in range(6):
+                    if mode == "alone_l2_flushed":
+                        big.fill_(1)
+                    x = blocks[i % 4]
+                    sd.block_attn(x.q, x.k_blk, x.v_blk, out.attn)
+                rows[mode].append(read())
+    assert int(sd.device_status()[0]) == 0
+    med = lambda rs: {k: [float(np.median([r[k][j] for r in rs])) for j in range(len(rs[0][k]))] if isinstance(rs[0][k], list)
+                      else rs[0][k] for k in rs[0]} if rs else None
+    return {"workload": wl.name, "unit": "us after the dependency wait returned: [median, max] over thread blocks, median over repetitions",
+            **{k: med(v) for k, v in rows.items() if v}}
+
+
 def time_e2e(torch, dp, wl, steps, warmup, n_blocks=4):
     """Same metric through sdlm_decode_step_host: pinned host inputs copied in, results copied out, every step."""
     s = wl.shape
@@ -648,6 +716,8 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the other workloads, the widening measurements and the CPU baseline")
     ap.add_argument("--min-timed-s", type=float, default=MIN_TIMED_S,
                     help="repeat the region of --steps steps until this much has been timed (0: one region, for profiling runs)")
+    ap.add_argument("--timeline", action="store_true",
+                    help="print in-kernel wall-clock marks of the attention kernel (library built with build.py --timeline) and exit")
     ap.add_argument("--model-level-only", action="store_true",
                     help="run only the whole-model step of the 3B shape and print its figures (for profiling)")
     args = ap.parse_args()
@@ -672,6 +742,9 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
     torch.cuda.set_device(local_rank)
+    if args.timeline:
+        print(json.dumps(attention_timeline(torch, wl.with_(steps=RESTORE_EVERY + 2), flush_l2=True)))
+        return
     if args.model_level_only:
         wl_m = wl.with_(steps=RESTORE_EVERY + 2)
         print(json.dumps(time_model_level(torch, pk, wl_m, syn.prefix_lengths(wl_m), 36, 11008, max(2, min(args.steps, 30)))))

@@ -9,6 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsdlm.so")
+LIB_TIMELINE = os.path.join(HERE, "libsdlm_timeline.so")   # the same library with in-kernel wall-clock marks (--timeline)
 SOURCES = ["sdlm_api.cu", "sdlm_attn.cu", "sdlm_lmhead.cu", "sdlm_layer.cu"]
 HEADERS = ["sdlm_internal.h", "sdlm_ptx.cuh", os.path.join("..", "..", "include", "sdlm.h")]
 
@@ -28,12 +29,19 @@ def needs_build() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every CUDA source for sm_100a into one shared library; returns its path."""
-    if not force and not needs_build():
-        return LIB
+def build(force: bool = False, verbose: bool = False, timeline: bool = False) -> str:
+    """Compile every CUDA source for sm_100a into one shared library; returns its path.  timeline=True
+    builds a second library, libsdlm_timeline.so, whose attention kernel leaves wall-clock marks that
+    bench.py --timeline reads (a measuring aid; the product library is unchanged)."""
+    if timeline:
+        out = LIB_TIMELINE
+    else:
+        out = LIB
+        if not force and not needs_build():
+            return LIB
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-Xcompiler", "-fPIC", "-shared", "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
+           "-Xcompiler", "-fPIC", "-shared", "-o", out] + (["-DSDLM_TIMELINE"] if timeline else []) + \
+          [os.path.join(CSRC, s) for s in SOURCES]
     if verbose:
         cmd.insert(1, "-Xptxas"); cmd.insert(2, "-v")
     res = subprocess.run(cmd, capture_output=True, text=True)
@@ -41,8 +49,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
     if verbose:
         sys.stderr.write(res.stderr)
-    return LIB
+    return out
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, timeline="--timeline" in sys.argv))

@@ -5,32 +5,51 @@
 // one per (sequence, KV head) for the D block tokens -- form one sequence that is cut into equal
 // contiguous ranges, one per CTA, so every SM streams the same number of bytes.  The part of a
 // (sequence, KV head) pair that falls into one CTA's range is an "item"; a pair cut by a range
-// boundary leaves partial (reference, sum, O) results, which the last of its CTAs to finish merges
-// (arrival counter per pair; nobody waits).
+// boundary leaves partial (reference, sum, O) results that are merged in fixed order: with 32 stacked
+// query rows by the last of the pair's CTAs to finish (arrival counter per pair; nobody waits), with
+// 64 by a merge kernel that spreads the larger partials over the GPU.
 //
 // Inside a CTA the tiles of an item are taken two at a time (a "group" of up to 128 keys) and the
 // two contractions run on the 5th-generation tensor cores with the KEYS, not the few query rows,
 // on the 128 accumulator lanes:
 //     S^T = K Q^T      M = 128 keys,  N = the G*D stacked query rows (padded to 32 or 64), K = d
 //     O^T += V^T P^T   M = d,         N = query rows,                                     K = keys
-// so no lane computes padding and the operands re-read per instruction are small.  Roles:
+// so no lane computes padding and the operands re-read per instruction are small.  Roles (warp groups of
+// four; registers are moved from the first and the last group to the softmax warps):
 //   warp 0      bulk copies of cached tiles (K panels and V^T tile, stored in the pool in the
 //               tensor-core shared-memory layout) into a ring of two-tile buffers;
 //   warp 1      one thread issues the S^T instructions (S^T double-buffered in tensor memory);
-//   warp 7      one thread issues the O^T instructions;
-//   warps 2..5  softmax: thread = accumulator lane = one key; it holds that key's score for 32
-//               query rows, exponentiates against per-row references kept in shared memory, adds to
-//               its private row sums and writes its column of P^T (bf16) into the B-operand buffer
-//               (with 64 stacked rows warps 8..11 do the same for rows 32..63);
-//   warp 6      stages the stacked query rows (fetched one item ahead) and the block's own K/V rows.
-// The reference of a row is not the running maximum: it is only moved (and O^T, sums rescaled)
-// when some score exceeds it by more than 2^32, which the softmax warps agree on once per group;
-// the first group of an item always sets it to that group's exact row maxima.  Probabilities are
-// therefore exact up to rounding, and rescaling O^T in tensor memory is rare.
+//   warp 2      one thread issues the O^T instructions (O^T double-buffered: one buffer per item in flight);
+//   warp 3      stages the stacked query rows (fetched one item ahead) and the block's own K/V rows;
+//   warps 4..7  softmax: thread = accumulator lane = one key; it holds that key's score for 32
+//               query rows, exponentiates against per-row references kept in shared memory, adds the
+//               bf16-rounded weights to its private row sums and writes its column of P^T into the
+//               B-operand buffer (with 64 stacked rows warps 8..11 do the same for rows 32..63);
+//   last four   epilogue: take an item's O^T out of tensor memory, divide by the row sums and write the
+//               output rows (or the partial result of a split, and merge), while the softmax warps are
+//               already at the next item.
+// The reference of a row is not the running maximum: an item starts from the scores of its first key and
+// the reference is only moved (and O^T, sums rescaled) when some score exceeds it by more than 2^32,
+// which the softmax warps agree on once per group.  Probabilities are therefore exact up to rounding, and
+// rescaling O^T in tensor memory is rare.
 #include "sdlm_internal.h"
 #include "sdlm_ptx.cuh"
 
 #include <string.h>
+
+// Build with -DSDLM_TIMELINE (build.py --timeline) to have every thread block of the attention kernel leave
+// wall-clock marks of its last launch in a device array that sdlm_timeline_read copies out: a measuring aid,
+// not part of the library proper (the marks cost a store each).
+#ifdef SDLM_TIMELINE
+__device__ unsigned long long g_sdlm_timeline[160][16];
+extern "C" int sdlm_timeline_read(void* host_out) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return 1;
+  return cudaMemcpyFromSymbol(host_out, g_sdlm_timeline, sizeof(g_sdlm_timeline)) == cudaSuccess ? 0 : 1;
+}
+#define SDLM_MARK(i) (g_sdlm_timeline[blockIdx.x][i] = sdlm::ptx::global_ns())
+#else
+#define SDLM_MARK(i) ((void)0)
+#endif
 
 namespace sdlm {
 
@@ -323,6 +342,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int GD = p.G * p.D;
+  if (tid == 0) SDLM_MARK(0);  // thread block resident
   // set-up that touches no global memory runs while the kernel before this one drains
   if (tid == 32) {
     for (int s = 0; s < NS; ++s) {
@@ -388,6 +408,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
   }
   ptx::grid_dep_wait();
   if (!p.release_first) ptx::grid_dep_launch();
+  if (tid == 0) SDLM_MARK(1);  // the kernel before this one is complete
   // The start-up chain is lengths -> page table -> first tiles (and query rows), each a trip to DRAM
   // that costs several microseconds under a concurrent weight stream.  Pulling the page table and the
   // block's query / key / value rows towards L2 now, alongside the load of the lengths, takes the
@@ -430,6 +451,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     }
   }
   const uint32_t tmem_base = *tmem_slot;
+  if (tid == 0) SDLM_MARK(2);  // schedule built, roles start
   // Registers follow the work (384 threads start at 168 registers each, 512 at 128): the group of four
   // copy / issue / staging warps and the epilogue warps give some up, the softmax warps, which hold a key's
   // scores and sums for 32 rows, take them.  Each group's code sits inside the branch that sets its count.
@@ -487,6 +509,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
         ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
         if (!ok) break;
         ring.advance(NS);
+        if (issued == 0 && lane == 0) SDLM_MARK(9);  // first group's copies issued
         ++issued;
       }
     }
@@ -516,6 +539,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
         for (int g = 0; g < ng; ++g) {
           const uint32_t sb = gc & 1u;
           if (!ptx::mbar_wait(&full[ring.stage], ring.phase, abort)) { ok = false; break; }
+          if (gc == 0) SDLM_MARK(3);  // query rows staged and first tiles landed
           if (gc >= 2 && !ptx::mbar_wait(&s_free[sb], ((gc >> 1) & 1u) ^ 1u, abort)) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t bk = st_addr + (uint32_t)ring.stage * PAIR_B;
@@ -625,6 +649,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       ptx::fence_proxy_async();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(q_full);
+      if (lane == 0 && item_idx == 0) SDLM_MARK(8);  // first item's query rows staged
       ++item_idx;
 
       // the next item's query rows travel while this item is being processed
@@ -853,6 +878,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&p_full[pbuf]);
+        if (gc == 0 && warp == 4 && lane == 0) SDLM_MARK(4);  // first P^T written
       }
       if (!ok) break;
 
@@ -885,6 +911,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       lread_buf = (int)b_last;
       ++item_idx;
     }
+    if (warp == 4 && lane == 0) SDLM_MARK(5);  // last P^T written
     if (!ok && lane == 0) attn_timeout(p, 3);
   } else {
     ptx::reg_dealloc<NQ == 64 ? 88 : 128>();
@@ -1030,6 +1057,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
         if (t == 0 && (int)blockIdx.x == it.c_first) p.pair_info[it.pair] = make_int2(it.c_first, it.n_splits);
       }
     }
+    if (t == 0) SDLM_MARK(6);  // last item written out (and merged)
     if (!ok && lane == 0) attn_timeout(p, 6);
   }
   ptx::tc_fence_before();
@@ -1038,6 +1066,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, TMEM_COLS);
   }
+  if (tid == 0) SDLM_MARK(7);  // thread block done
 }
 
 // Merges the partial results of the (sequence, KV head) pairs that a range boundary cut (fixed order:
