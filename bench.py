@@ -529,14 +529,19 @@ def time_noise_blocks(torch, pk, DeviceProblem, shape, n_target=4096, n_blocks=6
     u0 = torch.arange(0, n_chunks * n_c, n_c, dtype=torch.int32, device=sd.device)
     cout = torch.empty_like(cq)
     us_c = timed(lambda: sd.block_attn_masked_prefix(cq, ck, cv, vis, ids[:n_chunks], u0, cout))
+    # the same rows as one call of the causal kernel with 128-row query tiles
+    tq = pk.bf16_tensor_from_bits(syn.f32_to_bf16_bits(rng.normal(size=(n_target, shape.n_q_heads, shape.head_dim)).astype(np.float32)))
+    tout = torch.empty_like(tq)
+    us_k = timed(lambda: sd.causal_attn(0, tq, 0, tout))
     causal_flop = 4.0 * shape.n_q_heads * shape.head_dim * (n_target * (n_target + 1) / 2)
     causal_key_bytes = int(np.arange(0, n_chunks * n_c, n_c, dtype=np.int64).sum()) * row_b
     return {"us_per_call": us, "noise_blocks": n_blocks, "target_tokens": n_target, "block_D": D,
             "keys_read_gbs": key_bytes / (us * 1e-6) / 1e9,
             "causal_rows_us_per_call": us_c, "causal_chunk": n_c, "causal_chunks": n_chunks,
             "causal_tflops": causal_flop / (us_c * 1e-6) / 1e12,
+            "causal_kernel_us_per_call": us_k, "causal_kernel_tflops": causal_flop / (us_k * 1e-6) / 1e12,
             "causal_keys_read_gbs": causal_key_bytes / (us_c * 1e-6) / 1e9,
-            "what": "sdlm_block_attn_prefix (noise blocks) and sdlm_block_attn_masked_prefix (causal rows) back to back; "
+            "what": "sdlm_block_attn_prefix (noise blocks), sdlm_block_attn_masked_prefix (causal rows in chunks of 8) and sdlm_causal_attn (the same causal rows, 128-row query tiles), each back to back; "
                     "the shared target K/V (%.1f MB) stays in L2, so these are not HBM figures; causal_tflops counts the "
                     "lower triangle only" % (n_target * row_b / 1e6)}
 

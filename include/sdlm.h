@@ -17,7 +17,7 @@
  * Sec. 3.4), sdlm_block_attn_carry and sdlm_accept_commit_carry (blocks preceded by rows of real tokens,
  * Sec. 3.3), sdlm_block_attn_prefix and
  * sdlm_block_attn_masked_prefix (the noise-block rows and the causal rows of parallel training,
- * Sec. 3.3), sdlm_linear / sdlm_linear3 / sdlm_linear_rmsnorm / sdlm_rmsnorm / sdlm_rope_block(2) / sdlm_swiglu /
+ * Sec. 3.3), sdlm_causal_attn (those causal rows as one call with 128-row query tiles), sdlm_linear / sdlm_linear3 / sdlm_linear_rmsnorm / sdlm_rmsnorm / sdlm_rope_block(2) / sdlm_swiglu /
  * sdlm_accept_commit_layers (the rest of a decoder layer of the Qwen-2.5 backbone, Sec. 4.1, for
  * whole-model steps), sdlm_lmhead_confidence_static (no workspace scratch),
  * sdlm_selftest_bounded_wait, options and counters.
@@ -241,6 +241,22 @@ sdlm_status sdlm_block_attn_masked_prefix(sdlm_ctx* ctx, int32_t batch, int32_t 
                                           const int32_t* seq_ids, const int32_t* prefix_len, const void* q,
                                           const void* k_blk, const void* v_blk, const uint32_t* vis, void* out,
                                           void* stream);
+
+/* ---- causal attention of a cached sequence with itself -- Sec. 3.3, parallel training, the top-left part
+ * of the mask of Fig. 2a (A_uv = 1[v <= u] inside the target sequence), as one call with query tiles of 128
+ * rows on the tensor cores.  With the target sequence's K/V in the cache of slot `seq`, query row r is the
+ * token at position first_pos + r and attends to the cached tokens 0 .. first_pos + r (its own included):
+ *   out[r,h,:] = softmax_{t <= first_pos + r}( q[r,h,:] . K_t * scale ) V_t,   KV head h / (Hq/Hkv).
+ * q, out [n_rows, Hq, d]: device bf16.  The slot must hold at least first_pos + n_rows tokens (a row whose
+ * position lies beyond the cached length sees the whole cached sequence; the result for an empty slot is
+ * undefined).  Same arithmetic as sdlm_block_attn (fp32 scores, sums and accumulation, weights rounded to
+ * bf16 before they meet V, bf16 output); the cache is not modified; no workspace scratch.  Together with
+ * sdlm_block_attn_prefix for the noise blocks this is the whole attention of one parallel-training forward
+ * pass (sdlm_block_attn_masked_prefix computes the same rows in chunks of up to 8 positions).
+ * Errors: INVALID_ARG (null, misaligned, seq / first_pos / n_rows out of range), SHAPE (first_pos + n_rows
+ * beyond max_pages_per_seq * 64), UNSUPPORTED (softmax_scale not positive). */
+sdlm_status sdlm_causal_attn(sdlm_ctx* ctx, int32_t seq, int32_t first_pos, int32_t n_rows, const void* q, void* out,
+                             void* stream);
 
 /* ---- (b) LM head -> softmax statistics -- Sec. 3.2 (Z in R^{D x |V|}), Eq. 8, Eq. 9.
  * For each of `rows` hidden states: z = W h (|V| logits, fp32 accumulate, never stored);

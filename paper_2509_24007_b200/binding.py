@@ -34,7 +34,7 @@ EXPORTED = ["sdlm_pool_bytes", "sdlm_workspace_bytes", "sdlm_create", "sdlm_dest
             "sdlm_kv_pages", "sdlm_block_attn", "sdlm_lmhead_confidence", "sdlm_lmhead_confidence_static", "sdlm_accept_commit",
             "sdlm_device_status", "sdlm_decode_step", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count",
             "sdlm_block_attn_masked", "sdlm_verify_commit", "sdlm_accept_commit_carry",
-            "sdlm_block_attn_verify", "sdlm_block_attn_carry",
+            "sdlm_block_attn_verify", "sdlm_block_attn_carry", "sdlm_causal_attn",
             "sdlm_linear", "sdlm_linear3", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu", "sdlm_selftest_bounded_wait", "sdlm_rope_block2", "sdlm_accept_commit_layers", "sdlm_block_attn_prefix", "sdlm_linear_swiglu",
             "sdlm_block_attn_masked_prefix", "sdlm_linear_rmsnorm"]
 
@@ -138,6 +138,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdlm_block_attn_masked_prefix.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sdlm_accept_commit_carry.restype = C.c_int
     lib.sdlm_accept_commit_carry.argtypes = [vp, i32, i32, i32, vp, vp, f32, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_causal_attn.restype = C.c_int
+    lib.sdlm_causal_attn.argtypes = [vp, i32, i32, i32, vp, vp, vp]
     lib.sdlm_block_attn_verify.restype = C.c_int
     lib.sdlm_block_attn_verify.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.sdlm_block_attn_carry.restype = C.c_int
@@ -384,6 +386,17 @@ class Sdlm:
         self._check("sdlm_block_attn_masked", self.lib.sdlm_block_attn_masked(
             self.ctx, batch, n_q, n_k, _ptr(seq_ids), _ptr(q), _ptr(k_blk), _ptr(v_blk), _ptr(vis),
             _ptr(_dev(out, torch.bfloat16, "out")), _stream_ptr(stream)))
+        return out
+
+    def causal_attn(self, seq: int, q: torch.Tensor, first_pos: int = 0, out: Optional[torch.Tensor] = None,
+                    stream=None) -> torch.Tensor:
+        """sdlm_causal_attn: q [n_rows, Hq, d]; row r attends to the cached tokens 0 .. first_pos + r of slot seq."""
+        _dev(q, torch.bfloat16, "q")
+        if out is None:
+            out = torch.empty_like(q)
+        self._check("sdlm_causal_attn", self.lib.sdlm_causal_attn(
+            self.ctx, int(seq), int(first_pos), int(q.shape[0]), _ptr(q), _ptr(_dev(out, torch.bfloat16, "out")),
+            _stream_ptr(stream)))
         return out
 
     def block_attn_verify(self, q: torch.Tensor, k_blk: torch.Tensor, v_blk: torch.Tensor,

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsdlm.so")
 LIB_TIMELINE = os.path.join(HERE, "libsdlm_timeline.so")   # the same library with in-kernel wall-clock marks (--timeline)
-SOURCES = ["sdlm_api.cu", "sdlm_attn.cu", "sdlm_lmhead.cu", "sdlm_layer.cu"]
+SOURCES = ["sdlm_api.cu", "sdlm_attn.cu", "sdlm_causal.cu", "sdlm_lmhead.cu", "sdlm_layer.cu"]
 HEADERS = ["sdlm_internal.h", "sdlm_ptx.cuh", os.path.join("..", "..", "include", "sdlm.h")]
 
 

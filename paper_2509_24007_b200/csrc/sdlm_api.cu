@@ -538,7 +538,7 @@ extern "C" sdlm_status sdlm_create(const sdlm_config* cfg, void* kv_pool, size_t
   ctx->defer_merge = 0;
   ctx->pending_merge_fn = nullptr;
   ctx->tmap_h_rows = ctx->tmap_h_box = 0;
-  if (setup_attn(ctx) != cudaSuccess || setup_lmhead(ctx) != cudaSuccess) { delete ctx; return SDLM_ERR_CUDA; }
+  if (setup_attn(ctx) != cudaSuccess || setup_causal(ctx) != cudaSuccess || setup_lmhead(ctx) != cudaSuccess) { delete ctx; return SDLM_ERR_CUDA; }
   sdlm_status s = reset_tables(ctx, nullptr, 0);
   if (s == SDLM_OK && cudaStreamSynchronize(0) != cudaSuccess) s = SDLM_ERR_CUDA;
   if (s != SDLM_OK) { delete ctx; return s; }
@@ -911,6 +911,18 @@ extern "C" sdlm_status sdlm_block_attn_carry(sdlm_ctx* ctx, int32_t batch, int32
   if (c_max + D > kMaxBlockKeys) return SDLM_ERR_SHAPE;
   return attn_derived_mask(ctx, batch, c_max + D, c_max + D, seq_ids, q, k_rows, v_rows, out, 2, carry_len, c_max,
                            stream);
+}
+
+extern "C" sdlm_status sdlm_causal_attn(sdlm_ctx* ctx, int32_t seq, int32_t first_pos, int32_t n_rows, const void* q,
+                                        void* out, void* stream) {
+  if (!ctx || !q || !out) return SDLM_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out)) return SDLM_ERR_INVALID_ARG;
+  if (seq < 0 || seq >= ctx->cfg.max_batch || first_pos < 0 || n_rows < 1) return SDLM_ERR_INVALID_ARG;
+  if ((long long)first_pos + n_rows > (long long)ctx->cfg.max_pages_per_seq * kPageSize) return SDLM_ERR_SHAPE;
+  if (!(ctx->scale > 0.0f)) return SDLM_ERR_UNSUPPORTED;
+  return launch_causal_attn(ctx, seq, first_pos, n_rows, q, out, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? SDLM_OK
+             : SDLM_ERR_CUDA;
 }
 
 // One thread block waits, with the same bounded wait every kernel of the library uses, on a barrier and

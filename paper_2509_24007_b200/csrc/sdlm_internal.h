@@ -182,6 +182,8 @@ sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, 
 cudaError_t launch_rmsnorm(sdlm_ctx* ctx, int rows, int H, const void* x, const void* weight, float eps, void* out,
                            cudaStream_t st);
 cudaError_t launch_pending_merge(sdlm_ctx* ctx, cudaStream_t st);
+cudaError_t launch_causal_attn(sdlm_ctx* ctx, int slot, int first_pos, int n_rows, const void* q, void* out, cudaStream_t st);
+cudaError_t setup_causal(sdlm_ctx* ctx);
 cudaError_t setup_attn(sdlm_ctx* ctx);
 cudaError_t setup_lmhead(sdlm_ctx* ctx);
 

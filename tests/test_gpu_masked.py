@@ -401,6 +401,33 @@ def test_training_forward_attention_from_causal_chunks_and_noise_blocks(Hq, Hkv,
     assert torch.equal(out_c, out_c2)
 
 
+@pytest.mark.parametrize("Hq,Hkv,d,n_target", [(4, 2, 64, 333), (16, 2, 128, 1500), (16, 2, 128, 129), (8, 1, 64, 131), (2, 2, 128, 64),
+                                               (40, 8, 128, 700), (4, 4, 128, 1)])
+def test_causal_kernel_over_the_cached_target_sequence(Hq, Hkv, d, n_target):
+    """sdlm_causal_attn (128-row query tiles) on the target sequence in the cache: the target rows of the
+    oracle's dense attention under the full training mask; the whole sequence in one call, and the same rows
+    in three calls that start in the middle of a tile and of a page; twice for run-to-run identity."""
+    shape = syn.Shape(Hq, Hkv, d, 64, 64)
+    wl = syn.Workload("causal", shape, 3, 4, 0, 0, (0.9,), seed=1700 + d + n_target)
+    lens = np.array([10, n_target, 0], dtype=np.int32)                        # the target sequence sits in slot 1
+    dp = DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16), lengths=lens)
+    tk, tv = dp.prefix[1]
+    rng = np.random.default_rng(wl.seed)
+    tq = syn.f32_to_bf16_bits(rng.normal(size=(n_target, Hq, d)).astype(np.float32))
+    ref = orc.training_forward_attention(tq, tk, tv, n_target, [], 4)          # no noise blocks: the causal part alone
+    out = dp.sd.causal_attn(1, _dev_bits(tq))
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+    check_attention(pk.bits_from_bf16_tensor(out), ref)
+    assert torch.equal(out, dp.sd.causal_attn(1, _dev_bits(tq)))
+    cuts = sorted({0, min(n_target, 70), min(n_target, 70 + 193), n_target})
+    parts = [dp.sd.causal_attn(1, _dev_bits(tq[a:b]), first_pos=a) for a, b in zip(cuts[:-1], cuts[1:]) if b > a]
+    torch.cuda.synchronize()
+    check_attention(pk.bits_from_bf16_tensor(torch.cat(parts)), ref)
+    with pytest.raises(SdlmError):
+        dp.sd.causal_attn(7, _dev_bits(tq))                                    # no such slot
+
+
 def test_masked_prefix_argument_checks():
     shape = syn.Shape(4, 2, 64, 64, 64)
     wl, dp = _problem(shape, [100, 5], 4, seed=5)
