@@ -56,21 +56,26 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
   constexpr int PAIR_B = K_REGION_B + 2 * VT_B;
   constexpr int Q_PANEL_B = 128 * 128;            // 128 rows x 64 dims
   constexpr int P_PANEL_B = 128 * 128;            // 128 rows x 64 keys
+  constexpr int P_BUF_B = 2 * P_PANEL_B;          // the weights of one group of 128 keys
   constexpr uint32_t O_COL = 256, TMEM_COLS = 512;  // S buffers at columns 0 and 128, O at 256
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* q_s = smem;
   uint8_t* p_s = q_s + KH * Q_PANEL_B;
-  uint8_t* stages = p_s + 2 * P_PANEL_B;
+  uint8_t* stages = p_s + 2 * P_BUF_B;  // two P buffers: the weights of the next 128 keys are written while O += P V runs
   const int NS = p.n_stages;
-  uint64_t* full = reinterpret_cast<uint64_t*>(stages + (size_t)NS * PAIR_B);
-  uint64_t* stage_free = full + NS;
-  uint64_t* s_full = stage_free + NS;  // [2]
+  // a stage's K panels and its V^T tiles are loaded, and given back, separately: K is free again as soon as the
+  // scores of its group are computed, long before the group's weights meet V
+  uint64_t* full_k = reinterpret_cast<uint64_t*>(stages + (size_t)NS * PAIR_B);
+  uint64_t* full_v = full_k + NS;
+  uint64_t* k_free = full_v + NS;
+  uint64_t* v_free = k_free + NS;
+  uint64_t* s_full = v_free + NS;  // [2]
   uint64_t* s_free = s_full + 2;       // [2]
-  uint64_t* p_full = s_free + 2;
-  uint64_t* p_free = p_full + 1;
-  uint64_t* o_done = p_free + 1;
+  uint64_t* p_full = s_free + 2;       // [2]
+  uint64_t* p_free = p_full + 2;       // [2]
+  uint64_t* o_done = p_free + 2;
   uint64_t* drain = o_done + 1;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
   volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -83,15 +88,19 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
 
   if (tid == 32) {
     for (int s = 0; s < NS; ++s) {
-      ptx::mbar_init(&full[s], 1);
-      ptx::mbar_init(&stage_free[s], 1);
+      ptx::mbar_init(&full_k[s], 1);
+      ptx::mbar_init(&full_v[s], 1);
+      ptx::mbar_init(&k_free[s], 1);
+      ptx::mbar_init(&v_free[s], 1);
     }
     for (int s = 0; s < 2; ++s) {
       ptx::mbar_init(&s_full[s], 1);
       ptx::mbar_init(&s_free[s], 4);  // one arrival per softmax warp
     }
-    ptx::mbar_init(p_full, 4);
-    ptx::mbar_init(p_free, 1);
+    for (int s = 0; s < 2; ++s) {
+      ptx::mbar_init(&p_full[s], 4);
+      ptx::mbar_init(&p_free[s], 1);
+    }
     ptx::mbar_init(o_done, 1);
     ptx::mbar_init(drain, 1);
     *abort = 0;
@@ -129,18 +138,28 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
       const int32_t* ptab = p.page_table + (size_t)p.slot * p.mpps;
       const uint64_t kv_policy = ptx::l2_evict_first_policy();
       bool ok = true;
-      int my_page = 0, stage = 0;
-      uint32_t phase = 0;
-      for (int g = 0; g < n_groups && ok; ++g) {
-        if ((2 * g) % 32 == 0 && 2 * g + lane < n_tiles) my_page = ptab[2 * g + lane];  // one latency per 32 tiles
-        const int page0 = __shfl_sync(0xffffffffu, my_page, (2 * g) & 31);
-        const int page1 = __shfl_sync(0xffffffffu, my_page, (2 * g + 1) & 31);
+      // Order of the copies: K of the first NS groups, then for every group its V^T and the K of the group NS
+      // further on, which is the order in which the issuer gives the buffers back.  Page ids are read 32 tiles
+      // at a time (lane i holds tile base + i), one window for the K copies and one for the V^T copies.
+      int win_base[2] = {-1, -1}, win_page[2] = {0, 0};
+      auto copy_part = [&](int g, bool v_part) {  // warp-wide; lane 0 issues
+        const int stage = g % NS;
+        const uint32_t use = (uint32_t)(g / NS);
+        const int w = v_part ? 1 : 0, base = (2 * g) & ~31;
+        if (win_base[w] != base) {
+          win_base[w] = base;
+          win_page[w] = base + lane < n_tiles ? ptab[base + lane] : 0;
+        }
+        const int page0 = __shfl_sync(0xffffffffu, win_page[w], (2 * g) & 31);
+        const int page1 = __shfl_sync(0xffffffffu, win_page[w], (2 * g + 1) & 31);
         if (lane == 0) {
-          if (g >= NS && !ptx::mbar_wait_paced(&stage_free[stage], phase ^ 1u, abort)) ok = false;
+          uint64_t* freed = v_part ? &v_free[stage] : &k_free[stage];
+          if (use > 0 && !ptx::mbar_wait_paced(freed, (use - 1) & 1u, abort)) ok = false;
           if (ok) {
             const int tiles = min(2, n_tiles - 2 * g);
             uint8_t* st = stages + (size_t)stage * PAIR_B;
-            ptx::mbar_arrive_expect_tx(&full[stage], (uint32_t)(tiles * TILE_B));
+            uint64_t* bar = v_part ? &full_v[stage] : &full_k[stage];
+            ptx::mbar_arrive_expect_tx(bar, (uint32_t)(tiles * (v_part ? VT_B : KH * K_PANEL_B)));
             for (int j = 0; j < tiles; ++j) {
               int page = j ? page1 : page0;
               if (page < 0 || page >= p.num_pages) {  // never follow a bad table entry out of the pool
@@ -148,20 +167,26 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
                 page = 0;
               }
               const uint8_t* src = reinterpret_cast<const uint8_t*>(p.pool + kv_tile_offset(page, hk, 0, p.Hkv, HD));
+              if (v_part) {
+                ptx::bulk_g2s_hint(st + K_REGION_B + j * VT_B, src + KH * K_PANEL_B, VT_B, bar, kv_policy);
+              } else {
 #pragma unroll
-              for (int kh = 0; kh < KH; ++kh)
-                ptx::bulk_g2s_hint(st + kh * 2 * K_PANEL_B + j * K_PANEL_B, src + kh * K_PANEL_B, K_PANEL_B, &full[stage],
-                                   kv_policy);
-              ptx::bulk_g2s_hint(st + K_REGION_B + j * VT_B, src + KH * K_PANEL_B, VT_B, &full[stage], kv_policy);
+                for (int kh = 0; kh < KH; ++kh)
+                  ptx::bulk_g2s_hint(st + kh * 2 * K_PANEL_B + j * K_PANEL_B, src + kh * K_PANEL_B, K_PANEL_B, bar, kv_policy);
+              }
             }
           }
         }
         ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-        if (++stage == NS) { stage = 0; phase ^= 1u; }
+      };
+      for (int g = 0; g < min(NS, n_groups) && ok; ++g) copy_part(g, false);
+      for (int g = 0; g < n_groups && ok; ++g) {
+        copy_part(g, true);
+        if (ok && g + NS < n_groups) copy_part(g + NS, false);
       }
       if (lane == 0 && (!ok || *abort)) {  // winding down: let the copies already issued land
         causal_timeout(p, 1);
-        for (int s = 0; s < NS; ++s) ptx::mbar_wait_brief(&full[s], 0);
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
       }
       __syncwarp();
     } else if (warp == 1) {
@@ -174,7 +199,7 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
         auto issue_s = [&](int g) -> bool {
           const int stage = g % NS;
           const uint32_t sb = (uint32_t)g & 1u;
-          if (!ptx::mbar_wait(&full[stage], (uint32_t)(g / NS) & 1u, abort)) return false;
+          if (!ptx::mbar_wait(&full_k[stage], (uint32_t)(g / NS) & 1u, abort)) return false;
           if (g >= 2 && !ptx::mbar_wait(&s_free[sb], (((uint32_t)g >> 1) & 1u) ^ 1u, abort)) return false;
           ptx::tc_fence_after();
           const uint32_t bk = st_addr + (uint32_t)stage * PAIR_B;
@@ -185,22 +210,25 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
               ptx::umma_bf16_ss(tmem_base + sb * 128, causal_smem_desc(q_addr + kh * Q_PANEL_B + k * 32),
                                 causal_smem_desc(bk + kh * 2 * K_PANEL_B + k * 32), idesc_s, (kh | k) ? 1u : 0u);
           ptx::umma_commit(&s_full[sb]);
+          ptx::umma_commit(&k_free[stage]);  // the K panels of this stage may be replaced
           return true;
         };
         ok = issue_s(0);
         for (int g = 0; g < n_groups && ok; ++g) {
           if (g + 1 < n_groups && !issue_s(g + 1)) { ok = false; break; }
-          if (!ptx::mbar_wait(p_full, (uint32_t)g & 1u, abort)) { ok = false; break; }
-          ptx::tc_fence_after();
+          const uint32_t pb = (uint32_t)g & 1u;
+          if (!ptx::mbar_wait(&p_full[pb], ((uint32_t)g >> 1) & 1u, abort)) { ok = false; break; }
           const int stage = g % NS, tiles = min(2, n_tiles - 2 * g);
+          if (!ptx::mbar_wait(&full_v[stage], (uint32_t)(g / NS) & 1u, abort)) { ok = false; break; }
+          ptx::tc_fence_after();
           const uint32_t bv = st_addr + (uint32_t)stage * PAIR_B + K_REGION_B;
           for (int j = 0; j < tiles; ++j)
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-              ptx::umma_bf16_ss(tmem_base + O_COL, causal_smem_desc(p_addr + j * P_PANEL_B + k * 32),
+              ptx::umma_bf16_ss(tmem_base + O_COL, causal_smem_desc(p_addr + pb * P_BUF_B + j * P_PANEL_B + k * 32),
                                 causal_smem_desc(bv + j * VT_B + k * 32), idesc_o, (g | j | k) ? 1u : 0u);
-          ptx::umma_commit(&stage_free[stage]);  // K of this stage was read before P was written
-          ptx::umma_commit(p_free);
+          ptx::umma_commit(&v_free[stage]);
+          ptx::umma_commit(&p_free[pb]);
         }
         if (ok) {
           ptx::umma_commit(o_done);
@@ -225,27 +253,29 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
         ptx::tc_fence_after();
         const int k0 = g * 128;
         const bool edge = k0 + 128 > min(len, pos0 + 1);  // some row of the tile does not see some key of this group
-        // pass 1: the row's largest score in this group
+        // this row's 128 scores, out of tensor memory once; the buffer goes back to the issuer at once
+        uint32_t x[128];
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          ptx::tmem_ld_32x32b_x32(lane_addr + sb * 128 + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&x[c * 32]));
+        ptx::tmem_ld_wait();
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&s_free[sb]);
         float mx = -INFINITY;
+        if (edge) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t x[32];
-          ptx::tmem_ld_32x32b_x32(lane_addr + sb * 128 + c * 32, x);
-          ptx::tmem_ld_wait();
-          if (edge) {
+          for (int i = 0; i < 128; ++i)
+            if (k0 + i < my_keys) mx = fmaxf(mx, __uint_as_float(x[i]));
+        } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (k0 + c * 32 + i < my_keys) mx = fmaxf(mx, __uint_as_float(x[i]));
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(x[i]));
-          }
+          for (int i = 0; i < 128; i += 2) mx = ptx::max3(mx, __uint_as_float(x[i]), __uint_as_float(x[i + 1]));
         }
         mx *= p.scale_log2;  // the scale is positive
-        // the previous O += P V must be done before P is overwritten (and before O is rescaled)
-        if (g > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait(p_free, (uint32_t)(g - 1) & 1u, abort))) { ok = false; break; }
         const bool move = mx > m_ref + kCausalRebase || (m_ref == -INFINITY && mx > -INFINITY);
         if (__any_sync(0xffffffffu, move)) {
+          // O is about to be rescaled: the previous O += P V must be done
+          if (g > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[(g - 1) & 1], ((uint32_t)(g - 1) >> 1) & 1u, abort))) { ok = false; break; }
           float alpha = 1.0f;
           if (move) {
             alpha = m_ref == -INFINITY ? 0.f : ptx::ex2(m_ref - mx);
@@ -264,26 +294,22 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
               ptx::tmem_st16(lane_addr + O_COL + c * 16, o);
             }
             ptx::tmem_st_wait();
+            ptx::tc_fence_before();
           }
         }
-        // pass 2: weights 2^(s * scale - reference), rounded to bf16, into the A operand of O += P V; the same
-        // rounded values into the row sum.  A row that sees no key of the group writes zeros.
+        // this P buffer was read by the O += P V of two groups ago
+        const uint32_t pb = (uint32_t)g & 1u;
+        if (g >= 2 && !__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[pb], (((uint32_t)g >> 1) & 1u) ^ 1u, abort))) { ok = false; break; }
+        // weights 2^(s * scale - reference), rounded to bf16, into the A operand of O += P V; the same rounded
+        // values into the row sum.  A row that sees no key of the group writes zeros.
         const float neg_ref = m_ref == -INFINITY ? 0.f : -m_ref;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          uint32_t x[32];
-          ptx::tmem_ld_32x32b_x32(lane_addr + sb * 128 + c * 32, x);
-          ptx::tmem_ld_wait();
-          if (c == 3) {  // the last read of this S buffer
-            ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&s_free[sb]);
-          }
           uint32_t packed[16];
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
-            float w0 = ptx::ex2(fmaf(__uint_as_float(x[i]), p.scale_log2, neg_ref));
-            float w1 = ptx::ex2(fmaf(__uint_as_float(x[i + 1]), p.scale_log2, neg_ref));
+            float w0 = ptx::ex2(fmaf(__uint_as_float(x[c * 32 + i]), p.scale_log2, neg_ref));
+            float w1 = ptx::ex2(fmaf(__uint_as_float(x[c * 32 + i + 1]), p.scale_log2, neg_ref));
             if (edge) {
               if (k0 + c * 32 + i >= my_keys) w0 = 0.f;
               if (k0 + c * 32 + i + 1 >= my_keys) w1 = 0.f;
@@ -293,7 +319,7 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
             packed[i >> 1] = *reinterpret_cast<const uint32_t*>(&w);
           }
           // keys c*32 .. c*32+31 of the group: panel c >> 1, 16-byte chunks (c & 1) * 4 .. + 3 of this row
-          uint8_t* prow = p_s + (c >> 1) * P_PANEL_B + row * 128;
+          uint8_t* prow = p_s + pb * P_BUF_B + (c >> 1) * P_PANEL_B + row * 128;
 #pragma unroll
           for (int cc = 0; cc < 4; ++cc)
             *reinterpret_cast<uint4*>(prow + ((((c & 1) * 4 + cc) ^ (row & 7)) << 4)) =
@@ -302,7 +328,7 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
         ptx::fence_proxy_async();
         ptx::tc_fence_before();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(p_full);
+        if (lane == 0) ptx::mbar_arrive(&p_full[pb]);
       }
       if (ok && !__all_sync(0xffffffffu, ptx::mbar_wait(o_done, 0, abort))) ok = false;
       if (ok) {
@@ -348,12 +374,13 @@ constexpr int kCausalSmemLimit = 232448;
 template <int HD>
 static cudaError_t causal_launch(sdlm_ctx* ctx, CausalParams& p, cudaStream_t st) {
   const int pair_b = 2 * (2 * kPageSize * HD * 2);
-  const int fixed = 1024 + (HD / 64) * 128 * 128 + 2 * 128 * 128 + 16 * 8 + 64;
-  int n = (kCausalSmemLimit - fixed) / (pair_b + 16);
+  const int fixed = 1024 + (HD / 64) * 128 * 128 + 2 * (2 * 128 * 128) + 16 * 8 + 64;  // slack, Q, two P buffers, barriers, flags
+  // (every ring stage has four barriers)
+  int n = (kCausalSmemLimit - fixed) / (pair_b + 32);
   if (n > 4) n = 4;
   if (n < 2) return cudaErrorLaunchOutOfResources;
   p.n_stages = n;
-  const size_t smem = (size_t)fixed + (size_t)n * (pair_b + 16);
+  const size_t smem = (size_t)fixed + (size_t)n * (pair_b + 32);
   const cudaError_t e = launch_overlapped(causal_attn_umma_kernel<HD>, dim3((p.n_rows + 127) / 128, p.Hq),
                                           dim3(kCausalThreads), smem, st, p);
   ctx->launches++;
