@@ -14,8 +14,10 @@
 // half of the head's S columns, so it never passes through shared memory; the next S of the head is issued
 // behind the product that reads P (MMAs of one thread run in issue order).  Cached tiles arrive by bulk
 // copies in the layout the tensor cores read (see sdlm_internal.h); K and V^T have rings of their own.
-// Warp 0 copies, warp 1 issues all MMAs (the loop is warp-uniform, one elected lane issues), warps 2..5 /
-// 6..9 are the softmax of the first / second head (thread = query row) and, at the end, write the rows out.
+// Warp 0 copies, warp 1 issues all MMAs (the loop is warp-uniform, one elected lane issues; warps 2 and 3 only
+// fill the warp group, which gives most of its registers to the others), warps 4..11 / 12..19 are the softmax
+// of the first / second head: two threads per query row, one for each cached tile of
+// the group, which agree on the row's reference through shared memory; at the end they write the rows out.
 // The reference of a row is moved (and its O row and sum rescaled) only when a score exceeds it by more
 // than 2^8; only the groups that touch the diagonal look at key indices.
 #include "sdlm_internal.h"
@@ -59,7 +61,7 @@ struct CausalParams {
   int slot, first_pos, n_rows, Hq, Hkv, G, mpps, num_pages, n_k, n_v;
 };
 
-constexpr int kCausalThreads = 320;
+constexpr int kCausalThreads = 640;
 constexpr float kCausalRebase = 8.0f;  // log2 units a score may exceed its row reference by
 
 __device__ __forceinline__ uint64_t causal_smem_desc(uint32_t saddr) {
@@ -76,6 +78,96 @@ __device__ __forceinline__ void causal_umma_ts(uint32_t d_tmem, uint32_t a_tmem,
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
       "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
+}
+
+// Two fp32 lanes per instruction (fma.rn.f32x2 / add.rn.f32x2): half the issue slots of the scalar forms.
+__device__ __forceinline__ float2 causal_fma2(float2 a, float2 b, float2 c) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+  return d;
+}
+__device__ __forceinline__ float2 causal_add2(float2 a, float2 b) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "add.rn.f32x2 rd, ra, rb;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return d;
+}
+// 2^t for two arguments t <= 2^7 on the FMA and integer pipes instead of the special-function unit, which is
+// the narrowest pipe of the softmax: t = n + f with n = round(t), |f| <= 1/2; 2^f from a cubic fitted for the
+// smallest largest relative error on that interval (7.5e-5, a twenty-fifth of the bf16 rounding that follows);
+// n goes into the exponent field.  Arguments below -125 give 2^-125 times the cubic (weights that small add nothing).
+__device__ __forceinline__ float2 causal_exp2_poly2(float2 t) {
+  const float kMagic = 12582912.f;  // 1.5 * 2^23: adding it leaves round(t) in the low mantissa bits
+  t.x = fmaxf(t.x, -125.f);
+  t.y = fmaxf(t.y, -125.f);
+  const float2 r = causal_add2(t, make_float2(kMagic, kMagic));
+  const float2 n = causal_add2(r, make_float2(-kMagic, -kMagic));
+  const float2 f = causal_fma2(n, make_float2(-1.f, -1.f), t);
+  float2 q = causal_fma2(f, make_float2(0.0551716648f, 0.0551716648f), make_float2(0.2426111251f, 0.2426111251f));
+  q = causal_fma2(q, f, make_float2(0.6932609677f, 0.6932609677f));
+  q = causal_fma2(q, f, make_float2(0.9999280572f, 0.9999280572f));
+  return make_float2(__int_as_float(__float_as_int(q.x) + (__float_as_int(r.x) << 23)),
+                     __int_as_float(__float_as_int(q.y) + (__float_as_int(r.y) << 23)));
+}
+
+// Largest of a thread's 64 scores; with EDGE only over the keys k0 + i < my_keys the row sees.
+template <bool EDGE>
+__device__ __forceinline__ float causal_row_max(const uint32_t (&x)[64], int k0, int my_keys) {
+  float mx = -INFINITY;
+  if (EDGE) {
+#pragma unroll
+    for (int i = 0; i < 64; ++i)
+      if (k0 + i < my_keys) mx = fmaxf(mx, __uint_as_float(x[i]));
+  } else {
+#pragma unroll
+    for (int i = 0; i < 64; i += 2) mx = ptx::max3(mx, __uint_as_float(x[i]), __uint_as_float(x[i + 1]));
+  }
+  return mx;
+}
+// A thread's 64 weights 2^(x * scale + neg_ref) as bf16 pairs into 32 tensor-memory columns at taddr; returns the
+// sum of the rounded weights.  Three pairs of every eight take the power of two from the cubic, the
+// others from the special-function unit.
+template <bool EDGE>
+__device__ __forceinline__ float causal_weights(const uint32_t (&x)[64], uint32_t taddr, float scale, float neg_ref, int k0,
+                                                int my_keys) {
+  const float2 scale2 = make_float2(scale, scale), neg_ref2 = make_float2(neg_ref, neg_ref);
+  float2 l2 = make_float2(0.f, 0.f);
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    uint32_t packed[16];
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+      const float2 t = causal_fma2(make_float2(__uint_as_float(x[c * 32 + i]), __uint_as_float(x[c * 32 + i + 1])), scale2, neg_ref2);
+      float2 wf;
+      if (((i >> 1) & 7) < 3) {
+        wf = causal_exp2_poly2(t);
+      } else {
+        wf.x = ptx::ex2(t.x);
+        wf.y = ptx::ex2(t.y);
+      }
+      if (EDGE) {
+        if (k0 + c * 32 + i >= my_keys) wf.x = 0.f;
+        if (k0 + c * 32 + i + 1 >= my_keys) wf.y = 0.f;
+      }
+      const __nv_bfloat162 w = __floats2bfloat162_rn(wf.x, wf.y);
+      const uint32_t wb = *reinterpret_cast<const uint32_t*>(&w);
+      // the sum takes the rounded weights, the ones O is formed from: a row that one key dominates then comes out
+      // as that key's V row exactly, whatever the rounding of its weight
+      l2 = causal_add2(l2, make_float2(__uint_as_float(wb << 16), __uint_as_float(wb & 0xffff0000u)));
+      packed[i >> 1] = wb;
+    }
+    ptx::tmem_st16(taddr + c * 16, packed);
+  }
+  return l2.x + l2.y;
 }
 
 __device__ __forceinline__ void causal_timeout(const CausalParams& p, int where) {
@@ -95,7 +187,8 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
   constexpr int Q_PANEL_B = 128 * 128;           // 128 rows x 64 dims
   constexpr int Q_B = KH * Q_PANEL_B;            // one head's query tile
   constexpr int GK = 2 * kPageSize;              // keys per group
-  // tensor memory: S of head X at columns X*128 (its P over the first 64 of them); O of head X at 256 + X*128
+  // tensor memory: S of head X at columns X*128 (P of the group's tile j over columns X*128 + 64j .. + 31);
+  // O of head X at 256 + X*128
   constexpr uint32_t O_COL = 256, TMEM_COLS = 512;
 
   extern __shared__ uint8_t smem_raw[];
@@ -110,10 +203,13 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
   uint64_t* v_free = full_v + NV;
   uint64_t* s_full = v_free + NV;      // [head]
   uint64_t* p_full = s_full + 2;       // [head]
-  uint64_t* o_done = p_full + 2;
+  uint64_t* m_bar = p_full + 2;        // [head]: both halves of a row have written their maximum
+  uint64_t* l_bar = m_bar + 2;         // [head]: ... their sum
+  uint64_t* o_done = l_bar + 2;
   uint64_t* drain = o_done + 1;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
   volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  __nv_bfloat16* m_s = reinterpret_cast<__nv_bfloat16*>(tmem_slot + 4);  // [head][half][128 rows]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n_qt = (p.n_rows + 127) / 128;
@@ -134,7 +230,9 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
     }
     for (int s = 0; s < 2; ++s) {
       ptx::mbar_init(&s_full[s], 1);
-      ptx::mbar_init(&p_full[s], 4);  // one arrival per softmax warp of the head
+      ptx::mbar_init(&p_full[s], 8);  // one arrival per softmax warp of the head
+      ptx::mbar_init(&m_bar[s], 8);
+      ptx::mbar_init(&l_bar[s], 8);
     }
     ptx::mbar_init(o_done, 1);
     ptx::mbar_init(drain, 1);
@@ -167,8 +265,12 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (n_groups > 0) {
-    if (warp == 0) {
+  // Registers move between warp groups inside the thread block's own allocation (640 threads x 96 at launch):
+  // 128 x 56 + 512 x 104 stays below it, so the raise below never waits for registers that nobody gives back.
+  static_assert(128 * 56 + 512 * 104 <= kCausalThreads * 96, "register budget of the warp groups");
+  if (warp < 4) {
+    ptx::reg_dealloc<56>();
+    if (n_groups > 0 && warp == 0) {
       // ---------------------------------------------------------------- cached tiles: bulk copies
       const int32_t* ptab = p.page_table + (size_t)p.slot * p.mpps;
       bool ok = true;
@@ -221,7 +323,7 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
       }
       __syncwarp();
-    } else if (warp == 1) {
+    } else if (n_groups > 0 && warp == 1) {
       // ---------------------------------------------------------------- MMA issuer
       // Per group g and head x: O_x += P_x(g-1) V(g-1), then S_x(g) = Q_x K(g)^T over the columns that P_x(g-1)
       // was read from.  The whole warp runs the loop and the waits; one elected lane issues (see ptx::elect_one).
@@ -237,10 +339,10 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
           if (g > 0) {  // O_x += P_x(g-1) V(g-1)
             const int gv = g - 1, vs = gv % NV, tiles = min(2, n_tiles - 2 * gv);
             CAUSAL_T(c0);
-            if (x == 0 && !__all_sync(0xffffffffu, ptx::mbar_wait(&full_v[vs], (uint32_t)(gv / NV) & 1u, abort))) { ok = false; break; }
+            if (x == 0 && !__all_sync(0xffffffffu, ptx::mbar_wait_parked(&full_v[vs], (uint32_t)(gv / NV) & 1u, abort))) { ok = false; break; }
             CAUSAL_T(c1);
             CAUSAL_ACC(2, c0, c1);
-            if (!__all_sync(0xffffffffu, ptx::mbar_wait(&p_full[x], (uint32_t)gv & 1u, abort))) { ok = false; break; }
+            if (!__all_sync(0xffffffffu, ptx::mbar_wait_parked(&p_full[x], (uint32_t)gv & 1u, abort))) { ok = false; break; }
             CAUSAL_T(d1);
             CAUSAL_ACC(3 + x, c1, d1);
             ptx::tc_fence_after();
@@ -249,7 +351,7 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
               for (int j = 0; j < tiles; ++j)
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
-                  causal_umma_ts(tmem_base + O_COL + x * 128, tmem_base + x * 128 + j * 32 + k * 8,
+                  causal_umma_ts(tmem_base + O_COL + x * 128, tmem_base + x * 128 + j * 64 + k * 8,
                                  d_v + (uint64_t)((j * VT_B + k * 32) >> 4), idesc_o, (gv | j | k) ? 1u : 0u);
               if (x == n_heads - 1) ptx::umma_commit(&v_free[vs]);
             }
@@ -260,7 +362,7 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
           if (g < n_groups) {  // S_x(g) = Q_x K(g)^T
             const int ks = g % NK;
             CAUSAL_T(a0);
-            if (x == 0 && !__all_sync(0xffffffffu, ptx::mbar_wait(&full_k[ks], (uint32_t)(g / NK) & 1u, abort))) { ok = false; break; }
+            if (x == 0 && !__all_sync(0xffffffffu, ptx::mbar_wait_parked(&full_k[ks], (uint32_t)(g / NK) & 1u, abort))) { ok = false; break; }
             CAUSAL_T(a1);
             CAUSAL_ACC(0, a0, a1);
             ptx::tc_fence_after();
@@ -292,11 +394,17 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
         ptx::mbar_wait_brief(drain, 0);
       }
       __syncwarp();
-    } else if ((warp - 2) / 4 < n_heads) {
-      // ---------------------------------------------------------------- softmax and output: thread = query row of head X
-      const int X = (warp - 2) / 4, qd = warp & 3, row = qd * 32 + lane;
+    }
+  } else {
+    ptx::reg_alloc<104>();
+    if (n_groups > 0 && (warp - 4) / 8 < n_heads) {
+      // ---------------------------------------------------------------- softmax and output
+      // Thread = (query row of head X, half h): the keys of the group's cached tile h, the columns h*d/2 .. of O.
+      const int X = (warp - 4) >> 3, h = ((warp - 4) >> 2) & 1, qd = warp & 3, row = qd * 32 + lane;
       const uint32_t lane_addr = tmem_base + ((uint32_t)(qd * 32) << 16);
-      const uint32_t s_col = (uint32_t)X * 128, o_col = O_COL + (uint32_t)X * 128;
+      const uint32_t s_col = (uint32_t)X * 128 + (uint32_t)h * 64, o_col = O_COL + (uint32_t)X * 128 + (uint32_t)h * (HD / 2);
+      __nv_bfloat16* m_mine = m_s + (X * 2 + h) * 128 + row;
+      const __nv_bfloat16* m_other = m_s + (X * 2 + (h ^ 1)) * 128 + row;
       const int pos = pos0 + row;               // this row's position: it sees keys 0 .. pos (below the cache length)
       const int my_keys = min(len, pos + 1);
       float m_ref = -INFINITY, l = 0.f;
@@ -305,37 +413,28 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
       for (int g = 0; g < n_groups; ++g) {
         CAUSAL_T(t0);
         // S_x(g) complete; so is O_x += P_x(g-1) V(g-1), which was issued before it
-        if (!__all_sync(0xffffffffu, ptx::mbar_wait(&s_full[X], (uint32_t)g & 1u, abort))) { ok = false; break; }
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait_parked(&s_full[X], (uint32_t)g & 1u, abort))) { ok = false; break; }
         CAUSAL_T(t1);
         CAUSAL_ACC(0, t0, t1);
         ptx::tc_fence_after();
-        const int k0 = g * GK;
-        const bool edge = k0 + GK > min(len, pos0 + 1);  // some row of the tile does not see some key of this group
-        // pass 1: the row's maximum over the group
-        float mx = -INFINITY;
-        {
-          uint32_t xa[32], xb[32];
-          ptx::tmem_ld_32x32b_x32(lane_addr + s_col, xa);
-          ptx::tmem_ld_wait();
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t(&cur)[32] = (c & 1) ? xb : xa;
-            uint32_t(&nxt)[32] = (c & 1) ? xa : xb;
-            if (c < 3) ptx::tmem_ld_32x32b_x32(lane_addr + s_col + (c + 1) * 32, nxt);  // in flight while this chunk is reduced
-            if (edge) {
-#pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (k0 + c * 32 + i < my_keys) mx = fmaxf(mx, __uint_as_float(cur[i]));
-            } else {
-#pragma unroll
-              for (int i = 0; i < 32; i += 2) mx = ptx::max3(mx, __uint_as_float(cur[i]), __uint_as_float(cur[i + 1]));
-            }
-            if (c < 3) ptx::tmem_ld_wait();
-          }
-        }
-        mx *= p.scale_log2;  // the scale is positive
+        const int k0 = g * GK + h * kPageSize;              // first key of this thread's columns
+        const bool edge = g * GK + GK > min(len, pos0 + 1);  // some row of the tile does not see some key of this group
+        uint32_t x[64];
+        ptx::tmem_ld64(lane_addr + s_col, x);
+        ptx::tmem_ld_wait();
+        float mx = edge ? causal_row_max<true>(x, k0, my_keys) : causal_row_max<false>(x, k0, my_keys);
+        // The row's two threads must use one reference: each leaves its maximum, rounded to bf16, in shared
+        // memory and takes the larger of the two rounded values (any common value near the maximum serves).
+        const __nv_bfloat16 mine = __float2bfloat16_rn(mx * p.scale_log2);  // the scale is positive
+        *m_mine = mine;
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&m_bar[X]);
         CAUSAL_T(t2);
         CAUSAL_ACC(1, t1, t2);
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait_parked(&m_bar[X], (uint32_t)g & 1u, abort))) { ok = false; break; }
+        mx = fmaxf(__bfloat162float(mine), __bfloat162float(*m_other));
+        CAUSAL_T(t3);
+        CAUSAL_ACC(2, t2, t3);
         const bool move = mx > m_ref + kCausalRebase || (m_ref == -INFINITY && mx > -INFINITY);
         if (__any_sync(0xffffffffu, move)) {
           float alpha = 1.0f;
@@ -346,7 +445,7 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
           }
           if (g > 0) {  // O holds sums relative to the old references (nothing before the first group)
 #pragma unroll
-            for (int c = 0; c < HD / 16; ++c) {
+            for (int c = 0; c < HD / 32; ++c) {
               uint32_t o[16];
               ptx::tmem_ld16(lane_addr + o_col + c * 16, o);
               ptx::tmem_ld_wait();
@@ -357,36 +456,12 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
           }
         }
         CAUSAL_T(t4);
-        CAUSAL_ACC(3, t2, t4);
-        // pass 2: weights 2^(s * scale - reference), rounded to bf16, two per column over the S columns already
-        // read; the same rounded values into the row sum.  A key the row does not see gets weight zero.
+        CAUSAL_ACC(3, t3, t4);
+        // weights 2^(s * scale - reference), rounded to bf16, two per column over the first half of this
+        // thread's S columns.  A key the row does not see gets weight zero.
         const float neg_ref = m_ref == -INFINITY ? 0.f : -m_ref;
-        {
-          uint32_t xa[32], xb[32];
-          ptx::tmem_ld_32x32b_x32(lane_addr + s_col, xa);
-          ptx::tmem_ld_wait();
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t(&cur)[32] = (c & 1) ? xb : xa;
-            uint32_t(&nxt)[32] = (c & 1) ? xa : xb;
-            if (c < 3) ptx::tmem_ld_32x32b_x32(lane_addr + s_col + (c + 1) * 32, nxt);
-            uint32_t packed[16];
-#pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              float w0 = ptx::ex2(fmaf(__uint_as_float(cur[i]), p.scale_log2, neg_ref));
-              float w1 = ptx::ex2(fmaf(__uint_as_float(cur[i + 1]), p.scale_log2, neg_ref));
-              if (edge) {
-                if (k0 + c * 32 + i >= my_keys) w0 = 0.f;
-                if (k0 + c * 32 + i + 1 >= my_keys) w1 = 0.f;
-              }
-              const __nv_bfloat162 w = __floats2bfloat162_rn(w0, w1);
-              l += __low2float(w) + __high2float(w);
-              packed[i >> 1] = *reinterpret_cast<const uint32_t*>(&w);
-            }
-            if (c < 3) ptx::tmem_ld_wait();  // the next chunk is in registers before columns it came from are overwritten
-            ptx::tmem_st16(lane_addr + s_col + c * 16, packed);
-          }
-        }
+        l += edge ? causal_weights<true>(x, lane_addr + s_col, p.scale_log2, neg_ref, k0, my_keys)
+                  : causal_weights<false>(x, lane_addr + s_col, p.scale_log2, neg_ref, k0, my_keys);
         ptx::tmem_st_wait();
         ptx::tc_fence_before();
         __syncwarp();
@@ -394,14 +469,23 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
         CAUSAL_T(t5);
         CAUSAL_ACC(4, t4, t5);
       }
-      if (warp == 2 && lane == 0) CAUSAL_PH_OUT(8, 6);
+      if (warp == 4 && lane == 0) CAUSAL_PH_OUT(8, 6);
       if (ok && !__all_sync(0xffffffffu, ptx::mbar_wait(o_done, 0, abort))) ok = false;
+      if (ok) {
+        // every MMA is complete, so the query tiles in shared memory are free: the row's two sums meet there
+        float* l_s = reinterpret_cast<float*>(q_s);
+        l_s[(X * 2 + h) * 128 + row] = l;
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&l_bar[X]);
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(&l_bar[X], 0, abort))) ok = false;
+        if (ok) l += l_s[(X * 2 + (h ^ 1)) * 128 + row];
+      }
       if (ok) {
         ptx::tc_fence_after();
         const float inv = 1.0f / l;
-        __nv_bfloat16* out_row = p.out + ((size_t)(r0 + row) * p.Hq + head_a + X) * HD;
+        __nv_bfloat16* out_row = p.out + ((size_t)(r0 + row) * p.Hq + head_a + X) * HD + h * (HD / 2);
 #pragma unroll
-        for (int c = 0; c < HD / 16; ++c) {
+        for (int c = 0; c < HD / 32; ++c) {
           uint32_t o[16];
           ptx::tmem_ld16(lane_addr + o_col + c * 16, o);
           ptx::tmem_ld_wait();
@@ -439,8 +523,8 @@ constexpr int kCausalSmemLimit = 232448;
 template <int HD>
 static cudaError_t causal_launch(sdlm_ctx* ctx, CausalParams& p, cudaStream_t st) {
   const int part_b = 2 * kPageSize * HD * 2;  // K (or V^T) of one group of two cached tiles
-  // alignment slack, two heads' query tiles, 6 barriers, flags; two barriers per ring slot
-  const int fixed = 1024 + 2 * (HD / 64) * 128 * 128 + 6 * 8 + 64;
+  // alignment slack, two heads' query tiles, 10 barriers, flags, the row maxima; two barriers per ring slot
+  const int fixed = 1024 + 2 * (HD / 64) * 128 * 128 + 10 * 8 + 16 + 2 * 2 * 128 * 2;
   const int slots = (kCausalSmemLimit - fixed) / (part_b + 16);  // ring slots of either kind that fit
   if (slots < 4) return cudaErrorLaunchOutOfResources;
   p.n_v = slots / 2 > 6 ? 6 : slots / 2;  // K is asked for a product earlier than V^T: the odd slot goes to its ring
