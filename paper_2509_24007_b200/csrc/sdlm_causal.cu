@@ -3,8 +3,8 @@
 // sequence's K/V in the cache, query row r (position first_pos + r) attends to cached tokens
 // 0 .. first_pos + r.
 //
-// One CTA per (tile of 128 consecutive query positions, pair of query heads of one KV head); the longest
-// tiles are launched first.  The two heads share every cached K / V^T tile the CTA loads and take turns on
+// One CTA per (tile of 128 consecutive query positions, pair of query heads of one KV head); the tiles with
+// the most keys are launched first, across all head pairs.  The two heads share every cached K / V^T tile the CTA loads and take turns on
 // the tensor core: while the softmax threads of one work on its scores, the other's products run.  Query
 // rows sit on the 128 accumulator lanes, so a row's maximum and sum are private to one thread.  Per group of
 // 128 keys (two cached tiles) and head:
@@ -32,6 +32,11 @@ extern "C" int sdlm_causal_phase_read(void* host_out) {
   if (cudaDeviceSynchronize() != cudaSuccess) return 1;
   return cudaMemcpyFromSymbol(host_out, g_sdlm_causal_phase, sizeof(g_sdlm_causal_phase)) == cudaSuccess ? 0 : 1;
 }
+#define CAUSAL_STAMP(i)                                                                  \
+  do {                                                                                   \
+    const int blk_ = blockIdx.y * gridDim.x + blockIdx.x;                                \
+    if (blk_ < 1024 && threadIdx.x == 0) g_sdlm_causal_phase[blk_][i] = (long long)sdlm::ptx::global_ns(); \
+  } while (0)
 #define CAUSAL_T(var) const long long var = clock64()
 #define CAUSAL_ACC(i, a, b) (ph[i] += (b) - (a))
 #define CAUSAL_PH_DECL long long ph[8] = {0, 0, 0, 0, 0, 0, 0, 0}
@@ -42,6 +47,7 @@ extern "C" int sdlm_causal_phase_read(void* host_out) {
       for (int i_ = 0; i_ < (n); ++i_) g_sdlm_causal_phase[blk_][(base) + i_] = ph[i_]; \
   } while (0)
 #else
+#define CAUSAL_STAMP(i) ((void)0)
 #define CAUSAL_T(var) ((void)0)
 #define CAUSAL_ACC(i, a, b) ((void)0)
 #define CAUSAL_PH_DECL ((void)0)
@@ -213,10 +219,12 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n_qt = (p.n_rows + 127) / 128;
-  const int qt = n_qt - 1 - (int)blockIdx.x;  // the tiles with the most keys first
   const int HP = (p.G + 1) / 2;               // head pairs per KV head
-  const int hk = (int)blockIdx.y / HP, head_a = hk * p.G + 2 * ((int)blockIdx.y % HP);
-  const int n_heads = 2 * ((int)blockIdx.y % HP) + 1 < p.G ? 2 : 1;  // an odd group leaves its last head alone
+  // Thread blocks are handed out in the order of their index: all head pairs of the tile with the most keys first,
+  // then those of the next tile, so that the long ones start together and the short ones fill in behind them.
+  const int pair = (int)blockIdx.x % (p.Hkv * HP), qt = n_qt - 1 - (int)blockIdx.x / (p.Hkv * HP);
+  const int hk = pair / HP, head_a = hk * p.G + 2 * (pair % HP);
+  const int n_heads = 2 * (pair % HP) + 1 < p.G ? 2 : 1;  // an odd group leaves its last head alone
   const int r0 = qt * 128, rows = min(128, p.n_rows - r0);
 
   if (tid == 32) {
@@ -245,6 +253,7 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
   }
   ptx::grid_dep_launch();
   ptx::grid_dep_wait();  // the query rows and the cache may come from the kernels before this one
+  CAUSAL_STAMP(14);
 
   const int len = max(0, min(p.seq_len[p.slot], p.mpps * kPageSize));
   const int pos0 = p.first_pos + r0;                        // position of the tile's first row
@@ -511,6 +520,7 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
   }
   ptx::tc_fence_before();
   __syncthreads();
+  CAUSAL_STAMP(15);
   if (warp == 1) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, TMEM_COLS);
@@ -531,7 +541,7 @@ static cudaError_t causal_launch(sdlm_ctx* ctx, CausalParams& p, cudaStream_t st
   p.n_k = slots - p.n_v > 6 ? 6 : slots - p.n_v;
   const size_t smem = (size_t)fixed + (size_t)(p.n_k + p.n_v) * (part_b + 16);
   const int head_pairs = p.Hkv * ((p.G + 1) / 2);
-  const cudaError_t e = launch_overlapped(causal_attn_umma_kernel<HD>, dim3((p.n_rows + 127) / 128, head_pairs),
+  const cudaError_t e = launch_overlapped(causal_attn_umma_kernel<HD>, dim3(((p.n_rows + 127) / 128) * head_pairs),
                                           dim3(kCausalThreads), smem, st, p);
   ctx->launches++;
   return e != cudaSuccess ? e : cudaGetLastError();
