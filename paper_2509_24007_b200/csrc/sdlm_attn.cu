@@ -524,9 +524,10 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     __syncwarp();
   } else if (warp == 1) {
     // ---------------------------------------------------------------- S^T = K Q^T issuer
-    if (lane == 0) {
+    // The whole warp walks the items and waits; one elected lane issues (see ptx::elect_one).
+    {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NQ >> 3) << 17) | ((128u >> 4) << 24);
-      const uint32_t q_addr = ptx::smem_u32(q_s), st_addr = ptx::smem_u32(stages);
+      const uint64_t d_q = attn_smem_desc(ptx::smem_u32(q_s)), d_st = attn_smem_desc(ptx::smem_u32(stages));
       ItemWalk w;
       walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
       Item it;
@@ -534,29 +535,32 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       uint32_t gc = 0, item_idx = 0;
       bool ok = true;
       while (ok && walk_next(w, p, it)) {
-        if (!ptx::mbar_wait(q_full, item_idx & 1u, abort)) { ok = false; break; }
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(q_full, item_idx & 1u, abort))) { ok = false; break; }
         const int ng = (it.t1 - it.t0 + 1) / 2;
         for (int g = 0; g < ng; ++g) {
           const uint32_t sb = gc & 1u;
-          if (!ptx::mbar_wait(&full[ring.stage], ring.phase, abort)) { ok = false; break; }
-          if (gc == 0) SDLM_MARK(3);  // query rows staged and first tiles landed
-          if (gc >= 2 && !ptx::mbar_wait(&s_free[sb], ((gc >> 1) & 1u) ^ 1u, abort)) { ok = false; break; }
+          if (!__all_sync(0xffffffffu, ptx::mbar_wait(&full[ring.stage], ring.phase, abort))) { ok = false; break; }
+          if (gc == 0 && lane == 0) SDLM_MARK(3);  // query rows staged and first tiles landed
+          if (gc >= 2 && !__all_sync(0xffffffffu, ptx::mbar_wait(&s_free[sb], ((gc >> 1) & 1u) ^ 1u, abort))) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint32_t bk = st_addr + (uint32_t)ring.stage * PAIR_B;
+          const uint64_t d_k = d_st + (uint64_t)((ring.stage * PAIR_B) >> 4);
+          if (ptx::elect_one()) {
 #pragma unroll
-          for (int kh = 0; kh < KH; ++kh)
+            for (int kh = 0; kh < KH; ++kh)
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              ptx::umma_bf16_ss(tmem_base + sb * NQ, attn_smem_desc(bk + kh * 2 * K_PANEL_B + k * 32),
-                                attn_smem_desc(q_addr + kh * Q_PANEL_B + k * 32), idesc, (kh | k) ? 1u : 0u);
-          ptx::umma_commit(&s_full[sb]);
-          if (g == ng - 1) ptx::umma_commit(q_free);  // every S^T of this item is computed: Q may be replaced
+              for (int k = 0; k < 4; ++k)
+                ptx::umma_bf16_ss(tmem_base + sb * NQ, d_k + (uint64_t)((kh * 2 * K_PANEL_B + k * 32) >> 4),
+                                  d_q + (uint64_t)((kh * Q_PANEL_B + k * 32) >> 4), idesc, (kh | k) ? 1u : 0u);
+            ptx::umma_commit(&s_full[sb]);
+            if (g == ng - 1) ptx::umma_commit(q_free);  // every S^T of this item is computed: Q may be replaced
+          }
+          __syncwarp();
           ring.advance(NS);
           ++gc;
         }
         ++item_idx;
       }
-      if (!ok) {  // winding down: the MMAs already issued must finish before TMEM and smem are released
+      if (!ok && lane == 0) {  // winding down: the MMAs already issued must finish before TMEM and smem are released
         attn_timeout(p, 2);
         ptx::umma_commit(&drain[0]);
         ptx::mbar_wait_brief(&drain[0], 0);
@@ -565,9 +569,9 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     __syncwarp();
   } else if (warp == 2) {
     // ---------------------------------------------------------------- O^T += V^T P^T issuer
-    if (lane == 0) {
+    {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NQ >> 3) << 17) | ((128u >> 4) << 24);
-      const uint32_t p_addr = ptx::smem_u32(p_s), st_addr = ptx::smem_u32(stages);
+      const uint64_t d_p = attn_smem_desc(ptx::smem_u32(p_s)), d_st = attn_smem_desc(ptx::smem_u32(stages));
       ItemWalk w;
       walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
       Item it;
@@ -579,28 +583,35 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
         const uint32_t ob = item_idx & 1u, use = item_idx >> 1;  // O^T buffer of this item and how often it was used before
         for (int g = 0; g < ng; ++g) {
           const uint32_t pb = gc % PB;
-          if (!ptx::mbar_wait(&p_full[pb], (gc / PB) & 1u, abort)) { ok = false; break; }
+          if (!__all_sync(0xffffffffu, ptx::mbar_wait(&p_full[pb], (gc / PB) & 1u, abort))) { ok = false; break; }
           // the first instruction of an item overwrites its O^T buffer: the item before last must have been read out
-          if (g == 0 && use > 0 && !ptx::mbar_wait(&o_free[ob], (use - 1) & 1u, abort)) { ok = false; break; }
+          if (g == 0 && use > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait(&o_free[ob], (use - 1) & 1u, abort))) { ok = false; break; }
           ptx::tc_fence_after();
           const int tiles = min(2, n - 2 * g);
-          const uint32_t av = st_addr + (uint32_t)ring.stage * PAIR_B + K_REGION_B, bp = p_addr + pb * P_BUF_B;
-          for (int j = 0; j < tiles; ++j)
+          const uint64_t d_v = d_st + (uint64_t)((ring.stage * PAIR_B + K_REGION_B) >> 4), d_pb = d_p + (uint64_t)((pb * P_BUF_B) >> 4);
+          if (ptx::elect_one()) {
+            for (int j = 0; j < tiles; ++j)
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              ptx::umma_bf16_ss(tmem_base + O_COL + ob * NQ, attn_smem_desc(av + j * VT_B + k * 32),
-                                attn_smem_desc(bp + j * P_PANEL_B + k * 32), idesc, (g == 0 && j == 0 && k == 0) ? 0u : 1u);
-          // P^T is only written after S^T of the same group was read, so K of this stage is done as well
-          ptx::umma_commit(&stage_free[ring.stage]);
-          ptx::umma_commit(&p_free[pb]);
+              for (int k = 0; k < 4; ++k)
+                ptx::umma_bf16_ss(tmem_base + O_COL + ob * NQ, d_v + (uint64_t)((j * VT_B + k * 32) >> 4),
+                                  d_pb + (uint64_t)((j * P_PANEL_B + k * 32) >> 4), idesc, (g == 0 && j == 0 && k == 0) ? 0u : 1u);
+            // P^T is only written after S^T of the same group was read, so K of this stage is done as well
+            ptx::umma_commit(&stage_free[ring.stage]);
+            ptx::umma_commit(&p_free[pb]);
+            if (g == ng - 1) ptx::umma_commit(&o_done[ob]);
+          }
+          __syncwarp();
           ring.advance(NS);
           ++gc;
         }
         if (!ok) break;
-        ptx::umma_commit(&o_done[ob]);
+        if (ng == 0) {  // an item without tiles still reports its (untouched) O^T buffer
+          if (ptx::elect_one()) ptx::umma_commit(&o_done[ob]);
+          __syncwarp();
+        }
         ++item_idx;
       }
-      if (!ok) {
+      if (!ok && lane == 0) {
         attn_timeout(p, 5);
         ptx::umma_commit(&drain[1]);
         ptx::mbar_wait_brief(&drain[1], 0);

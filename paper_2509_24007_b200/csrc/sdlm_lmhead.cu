@@ -338,41 +338,46 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
     }
     __syncwarp();  // the warp arrives at the closing barrier as a whole
   } else if (warp == 1) {
-    if (lane == 0) {  // ---- MMA issuer
+    // ---- MMA issuer: the whole warp runs the loop and the waits, one elected lane issues (see ptx::elect_one)
+    {
       // instruction descriptor: D fp32, A and B bf16, both K-major, N = bn, M = 128
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.bn >> 3) << 17) | ((128u >> 4) << 24);
+      const uint64_t d_smem = umma_smem_desc(ptx::smem_u32(smem));  // byte offsets / 16 are added to its address field
       uint32_t it = 0;
       bool ok = true;
       for (int t = 0; t < n_tiles && ok; ++t) {
         const int as = t % NACC;
         const uint32_t use = (uint32_t)t / NACC;
-        if (use > 0 && !ptx::mbar_wait(&acc_empty[as], (use & 1) ^ 1, abort)) {
+        if (use > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait(&acc_empty[as], (use & 1) ^ 1, abort))) {
           ok = false;
           break;
         }
         ptx::tc_fence_after();
         for (int kc = 0; kc < KC; ++kc, ++it) {
           const int s = it % n_stages;
-          if (!ptx::mbar_wait(&full[s], (it / n_stages) & 1, abort)) {
+          if (!__all_sync(0xffffffffu, ptx::mbar_wait(&full[s], (it / n_stages) & 1, abort))) {
             ok = false;
             break;
           }
           ptx::tc_fence_after();
-          const uint32_t a_addr = ptx::smem_u32(smem + (size_t)s * stage_bytes);
-          const uint32_t b_addr = a_addr + R * kATileBytes;
+          const uint64_t d_a = d_smem + (uint64_t)(((size_t)s * stage_bytes) >> 4);
+          const uint64_t d_b = d_a + (uint64_t)((R * kATileBytes) >> 4);
+          if (ptx::elect_one()) {
 #pragma unroll
-          for (int r = 0; r < R; ++r) {
-            const uint32_t d_tmem = tmem_base + (uint32_t)((R == 1 ? as : r) * 256);
+            for (int r = 0; r < R; ++r) {
+              const uint32_t d_tmem = tmem_base + (uint32_t)((R == 1 ? as : r) * 256);
 #pragma unroll
-            for (int k = 0; k < kBK / 16; ++k)
-              ptx::umma_bf16_ss(d_tmem, umma_smem_desc(a_addr + r * kATileBytes + k * 32),
-                                umma_smem_desc(b_addr + k * 32), idesc, (kc | k) ? 1u : 0u);
+              for (int k = 0; k < kBK / 16; ++k)
+                ptx::umma_bf16_ss(d_tmem, d_a + (uint64_t)((r * kATileBytes + k * 32) >> 4), d_b + (uint64_t)((k * 32) >> 4), idesc,
+                                  (kc | k) ? 1u : 0u);
+            }
+            ptx::umma_commit(&empty[s]);  // stage reusable once these MMAs have read it
+            if (kc == KC - 1) ptx::umma_commit(&acc_full[as]);  // accumulator complete
           }
-          ptx::umma_commit(&empty[s]);  // stage reusable once these MMAs have read it
+          __syncwarp();
         }
-        if (ok) ptx::umma_commit(&acc_full[as]);  // accumulator complete
       }
-      if (!ok) {  // winding down: the MMAs already issued must finish before TMEM and smem are released
+      if (!ok && lane == 0) {  // winding down: the MMAs already issued must finish before TMEM and smem are released
         lm_timeout(p.hdr, 2);
         ptx::umma_commit(drain);
         ptx::mbar_wait_brief(drain, 0);
@@ -566,39 +571,43 @@ __global__ void __launch_bounds__(kPairThreads, 1)
     }
     __syncwarp();  // the warp arrives at the closing barrier as a whole
   } else if (warp == 1) {
-    if (lane == 0 && cta == 0) {  // ---- MMA issuer of the pair
+    if (cta == 0) {  // ---- MMA issuer of the pair: the whole warp runs the loop and the waits, one elected lane issues
       // instruction descriptor: D fp32, A and B bf16, both K-major, N, M = 256 over the two CTAs
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((256u >> 4) << 24);
+      const uint64_t d_smem = umma_smem_desc(ptx::smem_u32(smem));  // byte offsets / 16 are added to its address field
       uint32_t it = 0;
       bool ok = true;
       for (int t = 0; t < n_tiles && ok; ++t) {
         // one accumulator set: both CTAs' epilogues must have read tile t-1
-        if (t > 0 && !ptx::mbar_wait_cluster(acc_empty, (uint32_t)(t - 1) & 1u, abort)) {
+        if (t > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait_cluster(acc_empty, (uint32_t)(t - 1) & 1u, abort))) {
           ok = false;
           break;
         }
         ptx::tc_fence_after();
         for (int kc = 0; kc < KC; ++kc, ++it) {
           const int s = it % n_stages;
-          if (!ptx::mbar_wait_cluster(&full[s], (it / n_stages) & 1, abort)) {
+          if (!__all_sync(0xffffffffu, ptx::mbar_wait_cluster(&full[s], (it / n_stages) & 1, abort))) {
             ok = false;
             break;
           }
           ptx::tc_fence_after();
-          const uint32_t a_addr = ptx::smem_u32(smem + (size_t)s * stage_bytes);
-          const uint32_t b_addr = a_addr + kATileBytes;
+          const uint64_t d_a = d_smem + (uint64_t)(((size_t)s * stage_bytes) >> 4);
+          const uint64_t d_b = d_a + (uint64_t)(kATileBytes >> 4);
+          if (ptx::elect_one()) {
 #pragma unroll
-          for (int j = 0; j < 2; ++j) {
+            for (int j = 0; j < 2; ++j) {
 #pragma unroll
-            for (int k = 0; k < kBK / 16; ++k)
-              ptx::umma_bf16_ss_pair(tmem_base + (uint32_t)(j * 256), umma_smem_desc(a_addr + k * 32),
-                                     umma_smem_desc(b_addr + j * w_half_bytes + k * 32), idesc, (kc | k) ? 1u : 0u);
+              for (int k = 0; k < kBK / 16; ++k)
+                ptx::umma_bf16_ss_pair(tmem_base + (uint32_t)(j * 256), d_a + (uint64_t)((k * 32) >> 4),
+                                       d_b + (uint64_t)((j * w_half_bytes + k * 32) >> 4), idesc, (kc | k) ? 1u : 0u);
+            }
+            ptx::umma_commit_pair(&empty[s], 3);  // the stage is reusable in both CTAs once these MMAs have read it
+            if (kc == KC - 1) ptx::umma_commit_pair(acc_full, 3);  // both CTAs' accumulators complete
           }
-          ptx::umma_commit_pair(&empty[s], 3);  // the stage is reusable in both CTAs once these MMAs have read it
+          __syncwarp();
         }
-        if (ok) ptx::umma_commit_pair(acc_full, 3);  // both CTAs' accumulators complete
       }
-      if (!ok) {  // winding down: the MMAs already issued must finish before TMEM and smem are released
+      if (!ok && lane == 0) {  // winding down: the MMAs already issued must finish before TMEM and smem are released
         lm_timeout(p.hdr, 7);
         ptx::umma_commit_pair_local(drain);
         ptx::mbar_wait_brief(drain, 0);
