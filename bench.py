@@ -546,6 +546,40 @@ def time_noise_blocks(torch, pk, DeviceProblem, shape, n_target=4096, n_blocks=6
                     "lower triangle only" % (n_target * row_b / 1e6)}
 
 
+def time_causal_kernel(torch, pk, DeviceProblem, shape, n_target, iters=30):
+    """sdlm_causal_attn (Sec. 3.3 "Parallel Training", the causal part of Fig. 2a) over one cached target
+    sequence: calls back to back, CUDA events around them.  Flops are counted over the lower triangle only
+    (4 * Hq * d * n(n+1)/2); the roofline is the tensor one, against the burst bf16 rate (the kernel is timed
+    alone, for milliseconds)."""
+    wl = syn.Workload("causal", shape, 1, 4, 0, 0, (0.9,), seed=4712)
+    dp = DeviceProblem(wl, w_bits=np.zeros((16, shape.hidden), np.uint16), lengths=np.array([n_target], np.int32), keep_prefix=False)
+    sd = dp.sd
+    rng = np.random.default_rng(wl.seed)
+    tq = pk.bf16_tensor_from_bits(syn.f32_to_bf16_bits(rng.normal(size=(n_target, shape.n_q_heads, shape.head_dim)).astype(np.float32)))
+    tout = torch.empty_like(tq)
+    for _ in range(5):
+        sd.causal_attn(0, tq, 0, tout)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        sd.causal_attn(0, tq, 0, tout)
+    e1.record()
+    torch.cuda.synchronize()
+    assert int(sd.device_status()[0]) == 0
+    us = e0.elapsed_time(e1) / iters * 1e3
+    flop = 4.0 * shape.n_q_heads * shape.head_dim * (n_target * (n_target + 1) / 2)
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak = float(json.load(open(path))["bf16_tflops"]) if os.path.exists(path) else 1590.0
+    return {"shape": {"q_heads": shape.n_q_heads, "kv_heads": shape.n_kv_heads, "head_dim": shape.head_dim}, "target_tokens": n_target,
+            "us_per_call": us,
+            "roofline": {"bound": "tensor", "kernel": "causal_attn_umma_kernel (sdlm_causal_attn)", "achieved": flop / (us * 1e-6) / 1e12,
+                         "peak": peak, "unit": "TFLOP/s", "frac": flop / (us * 1e-6) / 1e12 / peak,
+                         "peak_source": "measured (MEASURED_PEAKS.json), bf16_tflops (burst)" if os.path.exists(path)
+                         else "fallback (1.59 PFLOP/s, an earlier measurement on this pool)",
+                         "algorithmic_flops": flop, "traffic": None}}
+
+
 def attention_timeline(torch, wl, flush_l2=False, reps=6):
     """Wall-clock marks inside the attention kernel of the in-order step, from the library built with
     `python paper_2509_24007_b200/build.py --timeline`.  Steps are enqueued back to back (one sdlm_decode_step
@@ -568,7 +602,8 @@ def attention_timeline(torch, wl, flush_l2=False, reps=6):
     out = dp.alloc_outputs()
     saved = sd.kv_save()
     buf = np.zeros((160, 16), dtype=np.uint64)
-    names = {0: "resident", 2: "roles_start", 9: "first_copies_issued", 8: "query_rows_staged", 3: "first_tiles_and_q",
+    names = {0: "resident", 2: "roles_start", 10: "stager_in_role", 11: "stager_first_item", 12: "stager_first_chunks_stored",
+             9: "first_copies_issued", 8: "query_rows_staged", 3: "first_tiles_and_q",
              4: "first_p", 5: "last_p", 6: "epilogue_done", 7: "block_done"}
 
     def step(i):
@@ -723,6 +758,9 @@ def main():
                     help="repeat the region of --steps steps until this much has been timed (0: one region, for profiling runs)")
     ap.add_argument("--timeline", action="store_true",
                     help="print in-kernel wall-clock marks of the attention kernel (library built with build.py --timeline) and exit")
+    ap.add_argument("--causal-only", type=int, default=0, metavar="TOKENS",
+                    help="run only the causal forward-attention kernel over a cached target sequence of this many tokens "
+                         "(shape of --workload) and print its figures (for profiling)")
     ap.add_argument("--model-level-only", action="store_true",
                     help="run only the whole-model step of the 3B shape and print its figures (for profiling)")
     args = ap.parse_args()
@@ -749,6 +787,9 @@ def main():
     torch.cuda.set_device(local_rank)
     if args.timeline:
         print(json.dumps(attention_timeline(torch, wl.with_(steps=RESTORE_EVERY + 2), flush_l2=True)))
+        return
+    if args.causal_only:
+        print(json.dumps(time_causal_kernel(torch, pk, DeviceProblem, wl.shape, args.causal_only, iters=max(2, min(args.steps, 30)))))
         return
     if args.model_level_only:
         wl_m = wl.with_(steps=RESTORE_EVERY + 2)
@@ -862,6 +903,10 @@ def main():
             extra["model_level_3b_" + wl.name] = time_model_level(torch, pk, wl_run, lengths, 36, 11008, max(4, min(args.steps, 30)))
             torch.cuda.empty_cache()
             extra["training_noise_blocks_3b"] = time_noise_blocks(torch, pk, DeviceProblem, wl.shape)
+            torch.cuda.empty_cache()
+            # the causal part of the training mask with the kernel of its own: 3B shape at 4096 and 16384 tokens, 32B shape at 4096
+            extra["training_causal_kernel"] = [time_causal_kernel(torch, pk, DeviceProblem, sh, n)
+                                               for sh, n in ((wl.shape, 4096), (wl.shape, 16384), (syn.CONFIGS["cfg3"].shape, 4096))]
             torch.cuda.empty_cache()
         line["extra"] = extra
         n_seqs = min(wl.batch, 32)

@@ -648,11 +648,14 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
         *reinterpret_cast<uint4*>(q_s + (c >> 3) * Q_PANEL_B + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = qreg[i];
       }
     };
+    if (lane == 0) SDLM_MARK(10);  // stager warp in its role
     bool have = walk_next(w, p, it);
+    if (lane == 0) SDLM_MARK(11);  // first item known
     if (have) fetch_q(it, 0);
     while (ok && have) {
       if (item_idx > 0 && !ptx::mbar_wait_warp_relaxed(q_free, (item_idx - 1) & 1u, abort)) { ok = false; break; }
       store_q(0);
+      if (lane == 0 && item_idx == 0) SDLM_MARK(12);  // first chunks of the query rows arrived and stored
       for (int first = NQR; first < NQC; first += NQR) {
         fetch_q(it, first);
         store_q(first);

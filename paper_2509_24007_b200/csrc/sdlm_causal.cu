@@ -261,22 +261,35 @@ __global__ void __launch_bounds__(kCausalThreads, 1) causal_attn_umma_kernel(con
   const int n_tiles = (n_keys + kPageSize - 1) / kPageSize;
   const int n_groups = (n_tiles + 1) / 2;
 
-  // query rows of both heads into shared memory, swizzled as an MMA operand; rows beyond the end are zero
-  for (int idx = tid; idx < n_heads * 128 * (HD / 8); idx += kCausalThreads) {
-    const int x = idx / (128 * (HD / 8)), r = (idx / (HD / 8)) % 128, c = idx % (HD / 8);
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (r < rows) v = __ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)(r0 + r) * p.Hq + head_a + x) * HD) + c);
-    *reinterpret_cast<uint4*>(q_s + x * Q_B + (c >> 3) * Q_PANEL_B + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = v;
-  }
-  ptx::fence_proxy_async();
   ptx::tc_fence_before();
-  __syncthreads();
+  __syncthreads();  // barriers initialised, tensor memory allocated
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   // Registers move between warp groups inside the thread block's own allocation (640 threads x 96 at launch):
   // 128 x 56 + 512 x 104 stays below it, so the raise below never waits for registers that nobody gives back.
   static_assert(128 * 56 + 512 * 104 <= kCausalThreads * 96, "register budget of the warp groups");
+  if (warp != 0) {
+    // Query rows of both heads into shared memory, swizzled as an MMA operand; rows beyond the end are zero.
+    // Every warp but the first, which is already sending for the first cached tiles: all loads first, then the stores.
+    constexpr int kStagers = kCausalThreads - 32, kIters = (2 * 128 * (HD / 8) + kStagers - 1) / kStagers;
+    uint4 v[kIters];
+#pragma unroll
+    for (int i = 0; i < kIters; ++i) {
+      const int idx = tid - 32 + i * kStagers;
+      const int x = idx / (128 * (HD / 8)), r = (idx / (HD / 8)) % 128, c = idx % (HD / 8);
+      v[i] = make_uint4(0, 0, 0, 0);
+      if (x < n_heads && r < rows) v[i] = __ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)(r0 + r) * p.Hq + head_a + x) * HD) + c);
+    }
+#pragma unroll
+    for (int i = 0; i < kIters; ++i) {
+      const int idx = tid - 32 + i * kStagers;
+      const int x = idx / (128 * (HD / 8)), r = (idx / (HD / 8)) % 128, c = idx % (HD / 8);
+      if (x < n_heads) *reinterpret_cast<uint4*>(q_s + x * Q_B + (c >> 3) * Q_PANEL_B + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = v[i];
+    }
+    ptx::fence_proxy_async();
+    asm volatile("bar.sync 1, %0;" ::"n"(kStagers) : "memory");  // the issuer may read the query tiles
+  }
   if (warp < 4) {
     ptx::reg_dealloc<56>();
     if (n_groups > 0 && warp == 0) {
