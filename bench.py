@@ -171,7 +171,7 @@ def _config(wl: syn.Workload, lengths=None):
     return c
 
 
-LMHEAD_NCU_TRAFFIC = 634216704   # bytes per launch of lmhead_umma_kernel<1> at cfg2_d4 (ncu, see profiles/)
+LMHEAD_NCU_TRAFFIC = 634481920   # bytes per launch of lmhead_umma_kernel<1> at cfg2_d4 (ncu, see profiles/)
 RESTORE_EVERY = 8   # steps between restores of the cache tables, so that prefix lengths stay the workload's
 
 
