@@ -424,7 +424,7 @@ def time_carry(torch, pk, DeviceProblem, wl, steps, warmup, n_blocks=4):
                     "only real-token K/V are cached (tokens counted when their K/V enter the cache)"}
 
 
-def time_model_level(torch, pk, wl, lengths, n_layers, intermediate, steps, warmup=2):
+def time_model_level(torch, pk, wl, lengths, n_layers, intermediate, steps, warmup=2, label="3B"):
     """Whole-model NSP decode steps: n_layers decoder layers of the Qwen-2.5 shape (random weights made
     on the device) around the block attention, final norm, LM head, acceptance and one commit per layer.
     One CUDA graph holds a table restore of every layer and one step; it is replayed `steps` times."""
@@ -441,7 +441,7 @@ def time_model_level(torch, pk, wl, lengths, n_layers, intermediate, steps, warm
                            rnd((H, I), I ** -0.5)) for _ in range(n_layers)]
     w_lm = pk.bf16_tensor_from_bits(syn.lm_head_weight(wl))
     stack = DecoderStack(wl, n_layers, I, lengths, layers, rnd((H,), 0.05, 1.0), w_lm,
-                         lambda l, b, n: (rnd((n, Hkv, d), 1.0), rnd((n, Hkv, d), 1.0)))
+                         lambda l, b, n: (rnd((n, Hkv, d), 1.0), rnd((n, Hkv, d), 1.0)), drop_split_weights=True)
     B, D = wl.batch, wl.block
     out = StepOutputs(torch.empty((B, D, Hq, d), dtype=torch.bfloat16, device=dev), torch.empty((B, D), dtype=torch.int32, device=dev),
                       torch.empty((B, D), dtype=torch.float32, device=dev), torch.empty((B, D), dtype=torch.float32, device=dev),
@@ -477,7 +477,8 @@ def time_model_level(torch, pk, wl, lengths, n_layers, intermediate, steps, warm
             "layers": n_layers, "intermediate": I, "library_launches_per_step": per_step,
             "weight_bytes": stack.weight_bytes(), "kv_bytes": kv,
             "achieved_gbs": (stack.weight_bytes() + kv) / (ms * 1e-3) / 1e9,
-            "what": "whole-model step (random weights of the 3B shape), every operation a library call, one CUDA graph per step"}
+            "batch": wl.batch, "block_D": wl.block,
+            "what": f"whole-model step (random weights of the {label} shape), every operation a library call, one CUDA graph per step"}
 
 
 def time_noise_blocks(torch, pk, DeviceProblem, shape, n_target=4096, n_blocks=64, D=4, n_c=8, iters=100):
@@ -762,7 +763,8 @@ def main():
                     help="run only the causal forward-attention kernel over a cached target sequence of this many tokens "
                          "(shape of --workload) and print its figures (for profiling)")
     ap.add_argument("--model-level-only", action="store_true",
-                    help="run only the whole-model step of the 3B shape and print its figures (for profiling)")
+                    help="run only the whole-model step and print its figures (for profiling): the 3B shape, 36 layers; "
+                         "with --workload cfg3 the 32B shape, 64 layers, batch 32")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
@@ -792,8 +794,12 @@ def main():
         print(json.dumps(time_causal_kernel(torch, pk, DeviceProblem, wl.shape, args.causal_only, iters=max(2, min(args.steps, 30)))))
         return
     if args.model_level_only:
-        wl_m = wl.with_(steps=RESTORE_EVERY + 2)
-        print(json.dumps(time_model_level(torch, pk, wl_m, syn.prefix_lengths(wl_m), 36, 11008, max(2, min(args.steps, 30)))))
+        if wl.shape.hidden == 5120:
+            wl_m = wl.with_(batch=32, steps=RESTORE_EVERY + 2)
+            print(json.dumps(time_model_level(torch, pk, wl_m, syn.prefix_lengths(wl_m), 64, 27648, max(2, min(args.steps, 8)), label="32B")))
+        else:
+            wl_m = wl.with_(steps=RESTORE_EVERY + 2)
+            print(json.dumps(time_model_level(torch, pk, wl_m, syn.prefix_lengths(wl_m), 36, 11008, max(2, min(args.steps, 30)))))
         return
     dist = None
     if world > 1:
@@ -901,6 +907,13 @@ def main():
             torch.cuda.empty_cache()
             # Qwen2.5-3B: 36 layers, intermediate size 11008
             extra["model_level_3b_" + wl.name] = time_model_level(torch, pk, wl_run, lengths, 36, 11008, max(4, min(args.steps, 30)))
+            torch.cuda.empty_cache()
+            # Qwen2.5-32B: 64 layers, intermediate size 27648; batch 32 of cfg3's 64 so that 62 GB of weights and 64 caches fit
+            wl32 = syn.CONFIGS["cfg3"].with_(batch=32, steps=RESTORE_EVERY + 2, name="cfg3_32b_b32_d4")
+            try:
+                extra["model_level_32b_" + wl32.name] = time_model_level(torch, pk, wl32, syn.prefix_lengths(wl32), 64, 27648, 4, label="32B")
+            except torch.OutOfMemoryError as e:   # a smaller GPU or a shared one: the figure is left out, the line stands
+                extra["model_level_32b_" + wl32.name] = {"skipped": "out of device memory: " + str(e)[:120]}
             torch.cuda.empty_cache()
             extra["training_noise_blocks_3b"] = time_noise_blocks(torch, pk, DeviceProblem, wl.shape)
             torch.cuda.empty_cache()

@@ -160,8 +160,10 @@ class DecoderStack:
     THETA = 1.0e6
 
     def __init__(self, wl: syn.Workload, n_layers: int, intermediate: int, lengths: np.ndarray, layers, ln_f, w_lm,
-                 prefix_fn):
-        """layers: list of LayerWeights; prefix_fn(layer, b, length) -> (k, v) device tensors [length, Hkv, d]."""
+                 prefix_fn, drop_split_weights: bool = False):
+        """layers: list of LayerWeights; prefix_fn(layer, b, length) -> (k, v) device tensors [length, Hkv, d].
+        drop_split_weights: forget every layer's wq / wk / wv / wgu once the stacked and interleaved copies that
+        the step reads exist (a 32B-shaped stack does not fit twice)."""
         s = wl.shape
         self.wl, self.L, self.I = wl, n_layers, intermediate
         self.lengths = np.asarray(lengths, dtype=np.int32)
@@ -171,12 +173,17 @@ class DecoderStack:
                          max_block=wl.block, page_size=s.page_size)
         self.ctx = [Sdlm(cfg) for _ in range(n_layers)]
         self.layers, self.ln_f, self.w_lm = layers, ln_f, w_lm
-        # q, k and v come from one product over the stacked weight
-        self.wqkv = [torch.cat([w.wq, w.wk, w.wv], dim=0).contiguous() for w in layers]
-        self.bqkv = [torch.cat([w.bq, w.bk, w.bv], dim=0).contiguous() for w in layers]
-        # gate and up rows interleaved, so that the product's epilogue can gate in registers
-        self.wgu_il = [torch.stack([w.wgu[:intermediate], w.wgu[intermediate:]], dim=1).reshape(2 * intermediate, -1).contiguous()
-                       for w in layers]
+        w0 = layers[0]
+        self._weight_bytes = n_layers * sum(t.numel() * 2 for t in (w0.wq, w0.wk, w0.wv, w0.wo, w0.wgu, w0.wdown)) + w_lm.numel() * 2
+        self.wqkv, self.bqkv, self.wgu_il = [], [], []
+        for w in layers:
+            # q, k and v come from one product over the stacked weight
+            self.wqkv.append(torch.cat([w.wq, w.wk, w.wv], dim=0).contiguous())
+            self.bqkv.append(torch.cat([w.bq, w.bk, w.bv], dim=0).contiguous())
+            # gate and up rows interleaved, so that the product's epilogue can gate in registers
+            self.wgu_il.append(torch.stack([w.wgu[:intermediate], w.wgu[intermediate:]], dim=1).reshape(2 * intermediate, -1).contiguous())
+            if drop_split_weights:
+                w.wq = w.wk = w.wv = w.wgu = None
         for l, sd in enumerate(self.ctx):
             sd.kv_reset(self.free_list)
             for b in range(wl.batch):
@@ -221,6 +228,4 @@ class DecoderStack:
         return sum(sd.launch_count() for sd in self.ctx)
 
     def weight_bytes(self) -> int:
-        per = sum(t.numel() * 2 for t in (self.layers[0].wq, self.layers[0].wk, self.layers[0].wv, self.layers[0].wo,
-                                          self.layers[0].wgu, self.layers[0].wdown))
-        return per * self.L + self.w_lm.numel() * 2
+        return self._weight_bytes

@@ -428,6 +428,33 @@ def test_causal_kernel_over_the_cached_target_sequence(Hq, Hkv, d, n_target):
         dp.sd.causal_attn(7, _dev_bits(tq))                                    # no such slot
 
 
+@pytest.mark.parametrize("Hq,Hkv,d,n_target,dense", [(16, 2, 128, 4096, True), (16, 2, 128, 16384, False), (40, 8, 128, 4096, False)])
+def test_causal_kernel_at_the_sizes_the_bench_times(Hq, Hkv, d, n_target, dense):
+    """sdlm_causal_attn in the launch configuration bench.py times (whole target sequence in one call): at 4096
+    tokens of the 3B shape every output against the oracle's dense attention under the training mask; at
+    16384 tokens and at the 32B shape sampled rows (first and last rows of tiles and pages, the ends, random
+    ones) against the oracle's block attention with D = 1, whose single row sees the tokens before it and
+    itself, i.e. the causal row of Sec. 3.3."""
+    shape = syn.Shape(Hq, Hkv, d, 64, 64)
+    wl = syn.Workload("causal_full", shape, 1, 4, 0, 0, (0.9,), seed=2900 + Hq + n_target)
+    dp = DeviceProblem(wl, w_bits=np.zeros((shape.vocab, shape.hidden), np.uint16), lengths=np.array([n_target], dtype=np.int32))
+    tk, tv = dp.prefix[0]
+    rng = np.random.default_rng(wl.seed)
+    tq = syn.f32_to_bf16_bits(rng.normal(size=(n_target, Hq, d)).astype(np.float32))
+    out = dp.sd.causal_attn(0, _dev_bits(tq))
+    torch.cuda.synchronize()
+    assert dp.sd.device_status()[0] == 0
+    got = pk.bits_from_bf16_tensor(out)
+    if dense:
+        check_attention(got, orc.training_forward_attention(tq, tk, tv, n_target, [], 4))
+    else:
+        rows = sorted({0, 1, 63, 64, 127, 128, 129, n_target // 2 - 1, n_target // 2, n_target - 129, n_target - 128, n_target - 1}
+                      | set(int(r) for r in rng.integers(0, n_target, size=12)))
+        for u in rows:
+            ref = orc.block_attention(tq[u][None, None], tk[u][None, None], tv[u][None, None], [tk[:u]], [tv[:u]])
+            check_attention(got[u][None, None], ref)
+
+
 def test_masked_prefix_argument_checks():
     shape = syn.Shape(4, 2, 64, 64, 64)
     wl, dp = _problem(shape, [100, 5], 4, seed=5)
