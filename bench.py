@@ -605,7 +605,8 @@ def attention_timeline(torch, wl, flush_l2=False, reps=6):
     buf = np.zeros((160, 16), dtype=np.uint64)
     names = {0: "resident", 2: "roles_start", 10: "stager_in_role", 11: "stager_first_item", 12: "stager_first_chunks_stored",
              9: "first_copies_issued", 8: "query_rows_staged", 3: "first_tiles_and_q",
-             4: "first_p", 5: "last_p", 6: "epilogue_done", 7: "block_done"}
+             4: "first_p", 5: "last_p", 13: "last_item_o_complete", 14: "last_split_partial_fenced", 15: "last_split_arrival_count_known",
+             6: "epilogue_done", 7: "block_done"}
 
     def step(i):
         x = blocks[i % 4]
@@ -617,8 +618,11 @@ def attention_timeline(torch, wl, flush_l2=False, reps=6):
         t = buf.astype(np.int64)
         act = t[:, 7] > 0
         t0 = t[act, 1].min()
-        return {n: [round(float(np.median((t[act, c] - t0) / 1e3)), 1), round(float(((t[act, c] - t0) / 1e3).max()), 1)]
-                for c, n in names.items()} | {"thread_blocks": int(act.sum()),
+        # a mark that a thread block did not pass in this launch still holds an older launch's time: left out
+        # (mark 0 is taken before the wait, so it is the one that may lie before the launch's own wait mark)
+        cur = lambda c: act & ((t[:, c] >= t[:, 1]) | (c == 0))
+        return {n: [round(float(np.median((t[cur(c), c] - t0) / 1e3)), 1), round(float(((t[cur(c), c] - t0) / 1e3).max()), 1)]
+                for c, n in names.items() if cur(c).any()} | {"thread_blocks": int(act.sum()),
                                               "resident_before_release_us": [round(float(((t0 - t[act, 0]) / 1e3).min()), 1),
                                                                              round(float(np.median((t0 - t[act, 0]) / 1e3)), 1),
                                                                              round(float(((t0 - t[act, 0]) / 1e3).max()), 1)]}

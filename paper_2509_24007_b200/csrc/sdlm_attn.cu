@@ -965,6 +965,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       if (!meet2()) { ok = false; break; }  // the row sums are visible to all four warps
       if (!ptx::mbar_wait_warp_relaxed(&o_done[ob], use & 1u, abort)) { ok = false; break; }
       ptx::tc_fence_after();
+      if (t == 0) SDLM_MARK(13);  // the (last) item's O^T is complete
       const float* lt = ltot + ob * 64;
       // row q = j*G + g  <->  out[b, q_first + j, h*G + g, :]
       __nv_bfloat16* out_slab = p.out + (((size_t)it.b * p.q_stride + p.q_first) * p.Hq + it.h * p.G) * HD;
@@ -1005,6 +1006,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
           // m = max_s m_s.  A thread owns eight (row, four columns) units, consecutive threads consecutive
           // columns of one row; it reads its rows' (m_s, l_s) itself, so nothing is shared.
           __threadfence();
+          if (t == 0) SDLM_MARK(14);  // the split's partial is written and fenced
           if (!meet2()) { ok = false; break; }
           if (t == 0) {  // every split of the pair counts once
             const int arrived = atomicAdd(&p.pair_cnt[it.pair], 1);
@@ -1013,6 +1015,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
             *s_last = last;
           }
           if (!meet2()) { ok = false; break; }
+          if (t == 0) SDLM_MARK(15);  // the arrival count is known
           if (*s_last) {
             __threadfence();
             constexpr int C4 = HD / 4, UPT = 8;
