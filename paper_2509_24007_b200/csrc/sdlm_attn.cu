@@ -441,9 +441,9 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
+  Item i0;
   {
     ItemWalk w0;
-    Item i0;
     walk_begin(w0, s_first, p.batch, p.Hkv, p.min_range);
     if (!walk_next(w0, p, i0)) {  // no tile falls into this CTA's range (uniform for the CTA)
       if (warp == 1) ptx::tmem_dealloc(*tmem_slot, TMEM_COLS);
@@ -452,6 +452,25 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
   }
   const uint32_t tmem_base = *tmem_slot;
   if (tid == 0) SDLM_MARK(2);  // schedule built, roles start
+  // The first item's stacked query rows (row r = j*G + g  <->  q[b, q_first + j, h*G + g, :]; rows beyond G*D are
+  // zero) are staged by the softmax and epilogue warps, which have nothing else to do yet: a few 16-byte chunks
+  // per thread instead of sixteen per lane of the staging warp, which takes over from the second item on.
+  if (warp >= 4) {
+    const int n_st = (int)blockDim.x - 128;
+    for (int idx = tid - 128; idx < NQ * (HD / 8); idx += n_st) {
+      const int r = idx / (HD / 8), c = idx % (HD / 8);
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (r < GD)
+        v = __ldg(reinterpret_cast<const uint4*>(p.q + (((size_t)i0.b * p.q_stride + p.q_first) * p.Hq + i0.h * p.G + row_hd[r]) * HD) + c);
+      *reinterpret_cast<uint4*>(q_s + (c >> 3) * Q_PANEL_B + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = v;
+    }
+    ptx::fence_proxy_async();
+    asm volatile("bar.sync 2, %0;" ::"r"(n_st) : "memory");
+    if (tid == 128) {
+      ptx::mbar_arrive(q_full);
+      SDLM_MARK(8);  // first item's query rows staged
+    }
+  }
   // Registers follow the work (384 threads start at 168 registers each, 512 at 128): the group of four
   // copy / issue / staging warps and the epilogue warps give some up, the softmax warps, which hold a key's
   // scores and sums for 32 rows, take them.  Each group's code sits inside the branch that sets its count.
@@ -651,19 +670,18 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     if (lane == 0) SDLM_MARK(10);  // stager warp in its role
     bool have = walk_next(w, p, it);
     if (lane == 0) SDLM_MARK(11);  // first item known
-    if (have) fetch_q(it, 0);
     while (ok && have) {
-      if (item_idx > 0 && !ptx::mbar_wait_warp_relaxed(q_free, (item_idx - 1) & 1u, abort)) { ok = false; break; }
-      store_q(0);
-      if (lane == 0 && item_idx == 0) SDLM_MARK(12);  // first chunks of the query rows arrived and stored
-      for (int first = NQR; first < NQC; first += NQR) {
-        fetch_q(it, first);
-        store_q(first);
+      if (item_idx > 0) {  // the first item's rows were staged by the other warps
+        if (!ptx::mbar_wait_warp_relaxed(q_free, (item_idx - 1) & 1u, abort)) { ok = false; break; }
+        store_q(0);
+        for (int first = NQR; first < NQC; first += NQR) {
+          fetch_q(it, first);
+          store_q(first);
+        }
+        ptx::fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(q_full);
       }
-      ptx::fence_proxy_async();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(q_full);
-      if (lane == 0 && item_idx == 0) SDLM_MARK(8);  // first item's query rows staged
       ++item_idx;
 
       // the next item's query rows travel while this item is being processed
