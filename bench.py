@@ -603,7 +603,7 @@ def attention_timeline(torch, wl, flush_l2=False, reps=6):
     out = dp.alloc_outputs()
     saved = sd.kv_save()
     buf = np.zeros((160, 16), dtype=np.uint64)
-    names = {0: "resident", 2: "roles_start", 10: "stager_in_role", 11: "stager_first_item",
+    names = {0: "resident", 2: "roles_start", 10: "stager_in_role", 11: "stager_first_item", 12: "copy_warp_first_item",
              9: "first_copies_issued", 8: "query_rows_staged", 3: "first_tiles_and_q",
              4: "first_p", 5: "last_p", 13: "last_item_o_complete", 14: "last_split_partial_fenced", 15: "last_split_arrival_count_known",
              6: "epilogue_done", 7: "block_done"}

@@ -441,14 +441,13 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
+  // the thread block's first item, and the walk as it stands behind it: the copy warp starts from these
   Item i0;
-  {
-    ItemWalk w0;
-    walk_begin(w0, s_first, p.batch, p.Hkv, p.min_range);
-    if (!walk_next(w0, p, i0)) {  // no tile falls into this CTA's range (uniform for the CTA)
-      if (warp == 1) ptx::tmem_dealloc(*tmem_slot, TMEM_COLS);
-      return;
-    }
+  ItemWalk w0;
+  walk_begin(w0, s_first, p.batch, p.Hkv, p.min_range);
+  if (!walk_next(w0, p, i0)) {  // no tile falls into this CTA's range (uniform for the CTA)
+    if (warp == 1) ptx::tmem_dealloc(*tmem_slot, TMEM_COLS);
+    return;
   }
   const uint32_t tmem_base = *tmem_slot;
   if (tid == 0) SDLM_MARK(2);  // schedule built, roles start
@@ -478,14 +477,14 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     ptx::reg_dealloc<NQ == 64 ? 104 : 144>();
   if (warp == 0) {
     // ---------------------------------------------------------------- cached tiles: bulk copies
-    ItemWalk w;
-    walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
-    Item it;
+    ItemWalk w = w0;
+    Item it = i0;
     Ring ring{0, 0};
     uint32_t issued = 0;  // groups so far
     const uint64_t kv_policy = ptx::l2_evict_first_policy();  // cached tiles are read once per call
     bool ok = true;
-    while (ok && walk_next(w, p, it)) {
+    for (bool have = true; ok && have; have = walk_next(w, p, it)) {
+      if (issued == 0 && lane == 0) SDLM_MARK(12);  // the copy warp is in its loop
       const int32_t* ptab = p.page_table + (size_t)it.slot * p.mpps;
       const int n = it.t1 - it.t0, n_cached = min(it.t1, it.pages) - it.t0;
       int my_page = 0;
