@@ -546,13 +546,12 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NQ >> 3) << 17) | ((128u >> 4) << 24);
       const uint64_t d_q = attn_smem_desc(ptx::smem_u32(q_s)), d_st = attn_smem_desc(ptx::smem_u32(stages));
-      ItemWalk w;
-      walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
-      Item it;
+      ItemWalk w = w0;  // the walk behind the first item, which every thread has worked out already
+      Item it = i0;
       Ring ring{0, 0};
       uint32_t gc = 0, item_idx = 0;
       bool ok = true;
-      while (ok && walk_next(w, p, it)) {
+      for (bool have = true; ok && have; have = walk_next(w, p, it)) {
         if (!__all_sync(0xffffffffu, ptx::mbar_wait(q_full, item_idx & 1u, abort))) { ok = false; break; }
         const int ng = (it.t1 - it.t0 + 1) / 2;
         for (int g = 0; g < ng; ++g) {
@@ -590,13 +589,12 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NQ >> 3) << 17) | ((128u >> 4) << 24);
       const uint64_t d_p = attn_smem_desc(ptx::smem_u32(p_s)), d_st = attn_smem_desc(ptx::smem_u32(stages));
-      ItemWalk w;
-      walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
-      Item it;
+      ItemWalk w = w0;  // the walk behind the first item, which every thread has worked out already
+      Item it = i0;
       Ring ring{0, 0};
       uint32_t gc = 0, item_idx = 0;
       bool ok = true;
-      while (ok && walk_next(w, p, it)) {
+      for (bool have = true; ok && have; have = walk_next(w, p, it)) {
         const int n = it.t1 - it.t0, ng = (n + 1) / 2;
         const uint32_t ob = item_idx & 1u, use = item_idx >> 1;  // O^T buffer of this item and how often it was used before
         for (int g = 0; g < ng; ++g) {
@@ -639,9 +637,8 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
   } else {
     // ---------------------------------------------------------------- warp 3: Q rows and the block's own tile
     constexpr int NQC = NQ * (HD / 8) / 32;  // 16-byte chunks of the stacked query rows per lane
-    ItemWalk w;
-    walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
-    Item it, nxt;
+    ItemWalk w = w0;  // the walk behind the first item, which every thread has worked out already
+    Item it = i0, nxt;
     Ring ring{0, 0};
     uint32_t blk_idx = 0, item_idx = 0;
     bool ok = true;
@@ -667,7 +664,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       }
     };
     if (lane == 0) SDLM_MARK(10);  // stager warp in its role
-    bool have = walk_next(w, p, it);
+    bool have = true;
     if (lane == 0) SDLM_MARK(11);  // first item known
     while (ok && have) {
       if (item_idx > 0) {  // the first item's rows were staged by the other warps
@@ -751,9 +748,8 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     const int kg = qd * 32 + lane;       // key within the group = accumulator lane
     const int tj = kg >> 6, kt = kg & 63;  // tile of the group, key within that tile
     const uint32_t lane_addr = tmem_base + ((uint32_t)(qd * 32) << 16);
-    ItemWalk w;
-    walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
-    Item it;
+    ItemWalk w = w0;  // the walk behind the first item, which every thread has worked out already
+    Item it = i0;
     uint32_t gc = 0, item_idx = 0, ep_uses = 0;
     int lread_buf = -1;  // the P^T buffer that still holds the previous item's hand-off (-1: none, or read)
     bool ok = true;
@@ -765,7 +761,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       ++ep_uses;
       return r;
     };
-    while (ok && walk_next(w, p, it)) {
+    for (bool have = true; ok && have; have = walk_next(w, p, it)) {
       float l[QV];  // this key subset's share of every row sum
 #pragma unroll
       for (int q = 0; q < QV; ++q) l[q] = 0.f;
@@ -953,9 +949,8 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     const int ew = warp - W_EPI;
     const int t = ew * 32 + lane;  // accumulator lane = output column
     const uint32_t lane_addr = tmem_base + ((uint32_t)(ew * 32) << 16);
-    ItemWalk w;
-    walk_begin(w, s_first, p.batch, p.Hkv, p.min_range);
-    Item it;
+    ItemWalk w = w0;  // the walk behind the first item, which every thread has worked out already
+    Item it = i0;
     uint32_t gc = 0, item_idx = 0, ep2_uses = 0;
     bool ok = true;
     auto meet2 = [&]() -> bool {
@@ -965,7 +960,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       ++ep2_uses;
       return r;
     };
-    while (ok && walk_next(w, p, it)) {
+    for (bool have = true; ok && have; have = walk_next(w, p, it)) {
       const uint32_t ob = item_idx & 1u, use = item_idx >> 1;
       gc += (uint32_t)((it.t1 - it.t0 + 1) / 2);
       const uint32_t b_last = (gc - 1) % PB;  // where the softmax warps left this item's sums
