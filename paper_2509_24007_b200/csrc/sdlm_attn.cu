@@ -159,6 +159,7 @@ struct ItemWalk {
   uint32_t total;      // positions in the whole launch (the host keeps total * gridDim below 2^31)
   uint32_t cur, hi;
   uint32_t nc;
+  int row;             // batch row of the last item handed out (-1: none yet)
 };
 
 __device__ __forceinline__ int pos_owner(uint32_t x, uint32_t total, uint32_t nc) {
@@ -170,6 +171,7 @@ __device__ __forceinline__ void walk_begin(ItemWalk& w, const int* s_first, int 
   w.s_len = s_first + batch + 1;
   w.s_slot = w.s_len + batch;
   w.total = (uint32_t)s_first[batch] * (uint32_t)Hkv;
+  w.row = -1;
   // Never more ranges than positions (every range is then non-empty), and no range shorter than a
   // few tiles: below that the fixed cost of a CTA and of merging its partial result outweighs
   // the parallelism.
@@ -182,17 +184,30 @@ __device__ __forceinline__ void walk_begin(ItemWalk& w, const int* s_first, int 
   w.hi = (blockIdx.x + 1) * w.total / w.nc;
 }
 
+// SPLITS: also work out which thread blocks share the item's pair (two integer divisions that only the epilogue
+// needs).  The batch row is looked for from the previous item's row onwards, by bisection only the first time,
+// and the head within the row by counting: an item switch costs a few dozen instructions.
+template <bool SPLITS = true>
 __device__ __forceinline__ bool walk_next(ItemWalk& w, const AttnParams& p, Item& it) {
   const uint32_t cost = (uint32_t)p.item_cost;
   while (w.cur < w.hi) {
-    int lo = 0, hi = p.batch - 1;
-    while (lo < hi) {
-      const int mid = (lo + hi + 1) >> 1;
-      if ((uint32_t)w.s_first[mid] * (uint32_t)p.Hkv <= w.cur) lo = mid; else hi = mid - 1;
+    int lo;
+    if (w.row < 0) {
+      lo = 0;
+      int hi = p.batch - 1;
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if ((uint32_t)w.s_first[mid] * (uint32_t)p.Hkv <= w.cur) lo = mid; else hi = mid - 1;
+      }
+    } else {
+      lo = w.row;
+      while (lo + 1 < p.batch && (uint32_t)w.s_first[lo + 1] * (uint32_t)p.Hkv <= w.cur) ++lo;
     }
+    w.row = lo;
     const uint32_t span = (uint32_t)(w.s_first[lo + 1] - w.s_first[lo]);  // cost + tiles of one pair
     const uint32_t row_start = (uint32_t)w.s_first[lo] * (uint32_t)p.Hkv;
-    const uint32_t h = (w.cur - row_start) / span;
+    uint32_t h = 0;
+    for (uint32_t off = w.cur - row_start; off >= span; off -= span) ++h;  // (cur - row_start) / span, at most Hkv - 1
     const uint32_t pair_start = row_start + h * span;
     const uint32_t a0 = w.cur - pair_start, a1 = min(w.hi, pair_start + span) - pair_start;
     w.cur = pair_start + a1;
@@ -205,9 +220,10 @@ __device__ __forceinline__ bool walk_next(ItemWalk& w, const AttnParams& p, Item
     it.slot = w.s_slot[lo];
     it.len = w.s_len[lo];
     it.pair = lo * p.Hkv + it.h;
-    // the CTAs that hold real tiles of this pair are consecutive
-    it.c_first = pos_owner(pair_start + cost, w.total, w.nc);
-    it.n_splits = pos_owner(pair_start + span - 1, w.total, w.nc) - it.c_first + 1;
+    if (SPLITS) {  // the CTAs that hold real tiles of this pair are consecutive
+      it.c_first = pos_owner(pair_start + cost, w.total, w.nc);
+      it.n_splits = pos_owner(pair_start + span - 1, w.total, w.nc) - it.c_first + 1;
+    }
     return true;
   }
   return false;
@@ -393,7 +409,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     Item it;
     const int n_warps = blockDim.x >> 5;
     int idx = 0;
-    while (idx < p.early_prefetch && walk_next(w, p, it)) {
+    while (idx < p.early_prefetch && walk_next<false>(w, p, it)) {
       const int n_cached = min(min(it.t1, it.pages) - it.t0, p.early_prefetch - idx);
       for (int k = warp - idx % n_warps + (warp < idx % n_warps ? n_warps : 0); k < n_cached; k += n_warps) {
         if (lane == 0) {
@@ -483,7 +499,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     uint32_t issued = 0;  // groups so far
     const uint64_t kv_policy = ptx::l2_evict_first_policy();  // cached tiles are read once per call
     bool ok = true;
-    for (bool have = true; ok && have; have = walk_next(w, p, it)) {
+    for (bool have = true; ok && have; have = walk_next<false>(w, p, it)) {
       if (issued == 0 && lane == 0) SDLM_MARK(12);  // the copy warp is in its loop
       const int32_t* ptab = p.page_table + (size_t)it.slot * p.mpps;
       const int n = it.t1 - it.t0, n_cached = min(it.t1, it.pages) - it.t0;
@@ -551,7 +567,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       Ring ring{0, 0};
       uint32_t gc = 0, item_idx = 0;
       bool ok = true;
-      for (bool have = true; ok && have; have = walk_next(w, p, it)) {
+      for (bool have = true; ok && have; have = walk_next<false>(w, p, it)) {
         if (!__all_sync(0xffffffffu, ptx::mbar_wait(q_full, item_idx & 1u, abort))) { ok = false; break; }
         const int ng = (it.t1 - it.t0 + 1) / 2;
         for (int g = 0; g < ng; ++g) {
@@ -594,7 +610,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       Ring ring{0, 0};
       uint32_t gc = 0, item_idx = 0;
       bool ok = true;
-      for (bool have = true; ok && have; have = walk_next(w, p, it)) {
+      for (bool have = true; ok && have; have = walk_next<false>(w, p, it)) {
         const int n = it.t1 - it.t0, ng = (n + 1) / 2;
         const uint32_t ob = item_idx & 1u, use = item_idx >> 1;  // O^T buffer of this item and how often it was used before
         for (int g = 0; g < ng; ++g) {
@@ -681,7 +697,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       ++item_idx;
 
       // the next item's query rows travel while this item is being processed
-      have = walk_next(w, p, nxt);
+      have = walk_next<false>(w, p, nxt);
       if (have) fetch_q(nxt, 0);
 
       const int n = it.t1 - it.t0, ng = (n + 1) / 2;
@@ -761,7 +777,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
       ++ep_uses;
       return r;
     };
-    for (bool have = true; ok && have; have = walk_next(w, p, it)) {
+    for (bool have = true; ok && have; have = walk_next<false>(w, p, it)) {
       float l[QV];  // this key subset's share of every row sum
 #pragma unroll
       for (int q = 0; q < QV; ++q) l[q] = 0.f;
