@@ -910,12 +910,28 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
         if (gc >= (uint32_t)PB && !__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[pbuf], ((gc / PB) & 1u) ^ 1u, abort))) { ok = false; break; }
         uint8_t* pcol = p_s + pbuf * P_BUF_B + tj * P_PANEL_B + (kt & 7) * 2;
         // The weight as the tensor core will see it (bf16), and that same value into the row sum: numerator
-        // and denominator then carry the same rounding, and a lone key weighs exactly 1.
+        // and denominator then carry the same rounding, and a lone key weighs exactly 1.  Two rows at a time:
+        // one conversion for both, and for three pairs of every eight the power of two from the cubic on the FMA
+        // pipe instead of the special-function unit, which the exponentials and the conversions share and
+        // which is what the softmax warps wait for with 64 stacked rows.
 #pragma unroll
-        for (int q = 0; q < QV; ++q) {
-          const __nv_bfloat16 w = __float2bfloat16_rn(mine ? ptx::ex2(e[q]) : 0.f);
-          l[q] += __bfloat162float(w);
-          *reinterpret_cast<__nv_bfloat16*>(pcol + (qb + q) * 128 + (((kt >> 3) ^ (q & 7)) << 4)) = w;
+        for (int q = 0; q < QV; q += 2) {
+          float2 wf;
+          if (((q >> 1) & 7) < 3) {
+            wf = ptx::exp2_poly2(make_float2(e[q], e[q + 1]));
+            if constexpr (MASKED) {  // a masked key (score -inf) weighs exactly 0, as 2^-inf does
+              if (e[q] == -INFINITY) wf.x = 0.f;
+              if (e[q + 1] == -INFINITY) wf.y = 0.f;
+            }
+          } else {
+            wf.x = ptx::ex2(e[q]);
+            wf.y = ptx::ex2(e[q + 1]);
+          }
+          const uint32_t wb = mine ? ptx::pack_bf16(wf.x, wf.y) : 0u;
+          l[q] += __uint_as_float(wb << 16);
+          l[q + 1] += __uint_as_float(wb & 0xffff0000u);
+          *reinterpret_cast<uint16_t*>(pcol + (qb + q) * 128 + (((kt >> 3) ^ (q & 7)) << 4)) = (uint16_t)wb;
+          *reinterpret_cast<uint16_t*>(pcol + (qb + q + 1) * 128 + (((kt >> 3) ^ ((q + 1) & 7)) << 4)) = (uint16_t)(wb >> 16);
         }
         ptx::fence_proxy_async();
         ptx::tc_fence_before();

@@ -86,45 +86,6 @@ __device__ __forceinline__ void causal_umma_ts(uint32_t d_tmem, uint32_t a_tmem,
       : "memory");
 }
 
-// Two fp32 lanes per instruction (fma.rn.f32x2 / add.rn.f32x2): half the issue slots of the scalar forms.
-__device__ __forceinline__ float2 causal_fma2(float2 a, float2 b, float2 c) {
-  float2 d;
-  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
-      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
-      "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
-      "mov.b64 {%0, %1}, rd;\n\t}"
-      : "=f"(d.x), "=f"(d.y)
-      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
-  return d;
-}
-__device__ __forceinline__ float2 causal_add2(float2 a, float2 b) {
-  float2 d;
-  asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
-      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
-      "add.rn.f32x2 rd, ra, rb;\n\t"
-      "mov.b64 {%0, %1}, rd;\n\t}"
-      : "=f"(d.x), "=f"(d.y)
-      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
-  return d;
-}
-// 2^t for two arguments t <= 2^7 on the FMA and integer pipes instead of the special-function unit, which is
-// the narrowest pipe of the softmax: t = n + f with n = round(t), |f| <= 1/2; 2^f from a cubic fitted for the
-// smallest largest relative error on that interval (7.5e-5, a twenty-fifth of the bf16 rounding that follows);
-// n goes into the exponent field.  Arguments below -125 give 2^-125 times the cubic (weights that small add nothing).
-__device__ __forceinline__ float2 causal_exp2_poly2(float2 t) {
-  const float kMagic = 12582912.f;  // 1.5 * 2^23: adding it leaves round(t) in the low mantissa bits
-  t.x = fmaxf(t.x, -125.f);
-  t.y = fmaxf(t.y, -125.f);
-  const float2 r = causal_add2(t, make_float2(kMagic, kMagic));
-  const float2 n = causal_add2(r, make_float2(-kMagic, -kMagic));
-  const float2 f = causal_fma2(n, make_float2(-1.f, -1.f), t);
-  float2 q = causal_fma2(f, make_float2(0.0551716648f, 0.0551716648f), make_float2(0.2426111251f, 0.2426111251f));
-  q = causal_fma2(q, f, make_float2(0.6932609677f, 0.6932609677f));
-  q = causal_fma2(q, f, make_float2(0.9999280572f, 0.9999280572f));
-  return make_float2(__int_as_float(__float_as_int(q.x) + (__float_as_int(r.x) << 23)),
-                     __int_as_float(__float_as_int(q.y) + (__float_as_int(r.y) << 23)));
-}
-
 // Largest of a thread's 64 scores; with EDGE only over the keys k0 + i < my_keys the row sees.
 template <bool EDGE>
 __device__ __forceinline__ float causal_row_max(const uint32_t (&x)[64], int k0, int my_keys) {
@@ -152,10 +113,10 @@ __device__ __forceinline__ float causal_weights(const uint32_t (&x)[64], uint32_
     uint32_t packed[16];
 #pragma unroll
     for (int i = 0; i < 32; i += 2) {
-      const float2 t = causal_fma2(make_float2(__uint_as_float(x[c * 32 + i]), __uint_as_float(x[c * 32 + i + 1])), scale2, neg_ref2);
+      const float2 t = ptx::fma2_f2(make_float2(__uint_as_float(x[c * 32 + i]), __uint_as_float(x[c * 32 + i + 1])), scale2, neg_ref2);
       float2 wf;
       if (((i >> 1) & 7) < 3) {
-        wf = causal_exp2_poly2(t);
+        wf = ptx::exp2_poly2(t);
       } else {
         wf.x = ptx::ex2(t.x);
         wf.y = ptx::ex2(t.y);
@@ -168,7 +129,7 @@ __device__ __forceinline__ float causal_weights(const uint32_t (&x)[64], uint32_
       const uint32_t wb = *reinterpret_cast<const uint32_t*>(&w);
       // the sum takes the rounded weights, the ones O is formed from: a row that one key dominates then comes out
       // as that key's V row exactly, whatever the rounding of its weight
-      l2 = causal_add2(l2, make_float2(__uint_as_float(wb << 16), __uint_as_float(wb & 0xffff0000u)));
+      l2 = ptx::add2_f2(l2, make_float2(__uint_as_float(wb << 16), __uint_as_float(wb & 0xffff0000u)));
       packed[i >> 1] = wb;
     }
     ptx::tmem_st16(taddr + c * 16, packed);

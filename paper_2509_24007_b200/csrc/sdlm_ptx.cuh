@@ -480,5 +480,44 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// Two fp32 lanes per instruction (fma.rn.f32x2 / add.rn.f32x2): half the issue slots of the scalar forms.
+__device__ __forceinline__ float2 fma2_f2(float2 a, float2 b, float2 c) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+  return d;
+}
+__device__ __forceinline__ float2 add2_f2(float2 a, float2 b) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "add.rn.f32x2 rd, ra, rb;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return d;
+}
+// 2^t for two arguments t <= 2^7 on the FMA and integer pipes instead of the special-function unit, which is
+// the narrowest pipe of the softmax: t = n + f with n = round(t), |f| <= 1/2; 2^f from a cubic fitted for the
+// smallest largest relative error on that interval (7.5e-5, a twenty-fifth of the bf16 rounding that follows);
+// n goes into the exponent field.  Arguments below -125 give 2^-125 times the cubic (weights that small add nothing).
+__device__ __forceinline__ float2 exp2_poly2(float2 t) {
+  const float kMagic = 12582912.f;  // 1.5 * 2^23: adding it leaves round(t) in the low mantissa bits
+  t.x = fmaxf(t.x, -125.f);
+  t.y = fmaxf(t.y, -125.f);
+  const float2 r = add2_f2(t, make_float2(kMagic, kMagic));
+  const float2 n = add2_f2(r, make_float2(-kMagic, -kMagic));
+  const float2 f = fma2_f2(n, make_float2(-1.f, -1.f), t);
+  float2 q = fma2_f2(f, make_float2(0.0551716648f, 0.0551716648f), make_float2(0.2426111251f, 0.2426111251f));
+  q = fma2_f2(q, f, make_float2(0.6932609677f, 0.6932609677f));
+  q = fma2_f2(q, f, make_float2(0.9999280572f, 0.9999280572f));
+  return make_float2(__int_as_float(__float_as_int(q.x) + (__float_as_int(r.x) << 23)),
+                     __int_as_float(__float_as_int(q.y) + (__float_as_int(r.y) << 23)));
+}
+
 }  // namespace ptx
 }  // namespace sdlm
