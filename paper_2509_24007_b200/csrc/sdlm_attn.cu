@@ -901,19 +901,14 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
             e[q4 + 3] = fmaf(x[q4 + 3], p.scale_log2, -mr.w);
           }
         }
-        // P^T column of my key: 2^(s*scale - reference), rounded to bf16; absent keys give 0
-        const uint32_t pbuf = gc % PB;
-        if (lread_buf == (int)pbuf) {  // the buffer still holds the previous item's hand-off: it must have been read
-          if (!__all_sync(0xffffffffu, ptx::mbar_wait(l_read, (item_idx - 1) & 1u, abort))) { ok = false; break; }
-          lread_buf = -1;
-        }
-        if (gc >= (uint32_t)PB && !__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[pbuf], ((gc / PB) & 1u) ^ 1u, abort))) { ok = false; break; }
-        uint8_t* pcol = p_s + pbuf * P_BUF_B + tj * P_PANEL_B + (kt & 7) * 2;
+        // P^T column of my key: 2^(s*scale - reference), rounded to bf16; absent keys give 0.
         // The weight as the tensor core will see it (bf16), and that same value into the row sum: numerator
         // and denominator then carry the same rounding, and a lone key weighs exactly 1.  Two rows at a time:
         // one conversion for both, and for three pairs of every eight the power of two from the cubic on the FMA
         // pipe instead of the special-function unit, which the exponentials and the conversions share and
-        // which is what the softmax warps wait for with 64 stacked rows.
+        // which is what the softmax warps wait for with 64 stacked rows.  The weights are formed before the
+        // buffer they go to is waited for: the O^T instruction that still reads it runs meanwhile.
+        uint32_t wbuf[QV / 2];
 #pragma unroll
         for (int q = 0; q < QV; q += 2) {
           float2 wf;
@@ -930,8 +925,19 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
           const uint32_t wb = mine ? ptx::pack_bf16(wf.x, wf.y) : 0u;
           l[q] += __uint_as_float(wb << 16);
           l[q + 1] += __uint_as_float(wb & 0xffff0000u);
-          *reinterpret_cast<uint16_t*>(pcol + (qb + q) * 128 + (((kt >> 3) ^ (q & 7)) << 4)) = (uint16_t)wb;
-          *reinterpret_cast<uint16_t*>(pcol + (qb + q + 1) * 128 + (((kt >> 3) ^ ((q + 1) & 7)) << 4)) = (uint16_t)(wb >> 16);
+          wbuf[q >> 1] = wb;
+        }
+        const uint32_t pbuf = gc % PB;
+        if (lread_buf == (int)pbuf) {  // the buffer still holds the previous item's hand-off: it must have been read
+          if (!__all_sync(0xffffffffu, ptx::mbar_wait(l_read, (item_idx - 1) & 1u, abort))) { ok = false; break; }
+          lread_buf = -1;
+        }
+        if (gc >= (uint32_t)PB && !__all_sync(0xffffffffu, ptx::mbar_wait(&p_free[pbuf], ((gc / PB) & 1u) ^ 1u, abort))) { ok = false; break; }
+        uint8_t* pcol = p_s + pbuf * P_BUF_B + tj * P_PANEL_B + (kt & 7) * 2;
+#pragma unroll
+        for (int q = 0; q < QV; q += 2) {
+          *reinterpret_cast<uint16_t*>(pcol + (qb + q) * 128 + (((kt >> 3) ^ (q & 7)) << 4)) = (uint16_t)wbuf[q >> 1];
+          *reinterpret_cast<uint16_t*>(pcol + (qb + q + 1) * 128 + (((kt >> 3) ^ ((q + 1) & 7)) << 4)) = (uint16_t)(wbuf[q >> 1] >> 16);
         }
         ptx::fence_proxy_async();
         ptx::tc_fence_before();
