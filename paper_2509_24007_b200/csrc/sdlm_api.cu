@@ -531,7 +531,8 @@ extern "C" sdlm_status sdlm_create(const sdlm_config* cfg, void* kv_pool, size_t
   ctx->ev_fork = ctx->ev_join = nullptr;
   ctx->attn_item_cost = 8;
   ctx->attn_min_range = 8;
-  ctx->attn_early_prefetch = 0;
+  ctx->attn_early_prefetch = -1;
+  ctx->in_decode_step = 0;
   ctx->tmap_w_ptr = nullptr;
   ctx->tmap_w_rows = 0;
   ctx->tmap_h_ptr = nullptr;
@@ -576,7 +577,7 @@ extern "C" sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t v
       ctx->attn_min_range = value;
       return SDLM_OK;
     case SDLM_OPT_ATTN_EARLY_PREFETCH:
-      if (value < 0 || value > 4096) return SDLM_ERR_INVALID_ARG;
+      if (value < -1 || value > 4096) return SDLM_ERR_INVALID_ARG;
       ctx->attn_early_prefetch = value;
       return SDLM_OK;
     case SDLM_OPT_STEP_OVERLAP:
@@ -999,8 +1000,10 @@ static sdlm_status decode_step_device(sdlm_ctx* ctx, int32_t batch, int32_t D, c
   // side by side, the LM-head kernel has to be the launch right after attention: the merge of attention's
   // split partials (which nothing in this step reads) then follows the LM head
   ctx->defer_merge = a_sms > 0;
+  ctx->in_decode_step = a_sms == 0;
   const cudaError_t ae = launch_block_attn(ctx, batch, D, seq_ids, q, k_blk, v_blk, attn_out, static_cast<cudaStream_t>(stream),
                                            a_sms, a_sms > 0 && batch * D > 128);
+  ctx->in_decode_step = 0;
   ctx->defer_merge = 0;
   if (ae != cudaSuccess) return SDLM_ERR_CUDA;
   // Attention writes none of the LM head's inputs, so the LM head never waits for it before it starts:
@@ -1115,8 +1118,10 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
   void* d_attn = m_attn ? m_attn : ws + L.st_out;
   const int overlap = ctx->overlap_lmhead;  // A: attention's SMs in the side-by-side step (0: in order)
   ctx->defer_merge = overlap > 0 && a_sms == 0;  // side by side on one stream: the merge follows the LM head
+  ctx->in_decode_step = overlap == 0;
   const cudaError_t ae =
       launch_block_attn(ctx, batch, D, seq_ids, in_q, in_k, in_v, d_attn, qkv_st, overlap, overlap > 0 && batch * D > 128);
+  ctx->in_decode_step = 0;
   ctx->defer_merge = 0;
   if (ae != cudaSuccess) return SDLM_ERR_CUDA;
   if (a_sms > 0 && cudaEventRecord(ctx->ev_join, qkv_st) != cudaSuccess) return SDLM_ERR_CUDA;

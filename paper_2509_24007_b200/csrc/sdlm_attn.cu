@@ -1316,7 +1316,8 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
   p.item_cost = ctx->attn_item_cost;
   p.min_range = ctx->attn_min_range;
   p.max_slots = c.max_batch;
-  p.early_prefetch = ctx->attn_early_prefetch;
+  // unless the caller has chosen: twelve tiles ahead inside an in-order decode step (measured best on the 3B step), none elsewhere
+  p.early_prefetch = ctx->attn_early_prefetch >= 0 ? ctx->attn_early_prefetch : (ctx->in_decode_step ? 12 : 0);
   p.release_first = cta_cap > 0 ? 1 : 0;
   p.Dk = n_blk_keys > 0 ? n_blk_keys : D;
   p.vis = vis;

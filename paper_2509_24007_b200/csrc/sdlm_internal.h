@@ -66,7 +66,8 @@ struct sdlm_ctx {
   int lmhead_path;  // 0 = pick by shape, 1 = force the mma.sync kernel, 2 = force the tcgen05 kernel
   int attn_min_range;  // shortest range of schedule positions given to one attention thread block
   int attn_item_cost;  // positions the attention schedule charges for starting a (sequence, KV head) pair
-  int attn_early_prefetch;  // cached tiles per thread block that attention prefetches before its dependency wait (0: off)
+  int attn_early_prefetch;  // cached tiles per thread block that attention prefetches before its dependency wait (0: off; -1: 12 inside a decode step, where the kernels before it leave the memory system idle, 0 elsewhere)
+  int in_decode_step;       // set around the attention launch of sdlm_decode_step / sdlm_decode_step_host
   int overlap_lmhead;  // sdlm_decode_step: SMs given to attention while the LM head runs on the rest (0: one after the other)
   // second stream and fork / join events of the host-buffer step's side-by-side mode (made on first use)
   int host_two_streams;

@@ -11,7 +11,7 @@ import torch
 
 import paper_2509_24007_b200 as pk
 from paper_2509_24007_b200.harness import DeviceProblem
-from paper_2509_24007_b200.binding import OPT_STEP_OVERLAP, OPT_HOST_TWO_STREAMS
+from paper_2509_24007_b200.binding import OPT_STEP_OVERLAP, OPT_HOST_TWO_STREAMS, OPT_ATTN_EARLY_PREFETCH
 from oracle import sdlm_oracle as orc
 import sdlm_synth as syn
 from oracle_side import (check_attention, check_confidences, check_gamma, check_tokens, oracle_cache)
@@ -315,6 +315,35 @@ def test_block_size_one_is_next_token_decode_on_the_gpu():
         out, stats, res, n_bad = _one_step(dp, cache, tau, step)
         assert n_bad == 0 and out.accepted_len.cpu().tolist() == [1] * wl.batch
         _compare_tables(dp, cache)
+
+
+@pytest.mark.parametrize("name,batch", [("cfg0", 4), ("cfg2_d4", 12)])
+def test_early_prefetch_of_cached_tiles_changes_no_result(name, batch):
+    """SDLM_OPT_ATTN_EARLY_PREFETCH only steers what the attention kernel asks the memory system for before its
+    dependency wait (from tables that the step before may still be changing): five fused steps enqueued back to
+    back give the same attention rows, tokens, accepted lengths and tables with the prefetch off, at the library's
+    own choice (-1: on inside a decode step) and far beyond what a thread block has (4096 tiles)."""
+    wl = syn.CONFIGS[name].with_(batch=batch)
+    dp = DeviceProblem(wl)
+    blocks = [dp.block(i) for i in range(5)]
+    saved = dp.sd.kv_save()
+    results = []
+    for value in (0, -1, 4096):
+        dp.sd.set_option(OPT_ATTN_EARLY_PREFETCH, value)
+        dp.sd.kv_restore(saved)
+        outs = [dp.alloc_outputs() for _ in blocks]
+        for x, o in zip(blocks, outs):
+            dp.step(x, wl.tau, o, fused=True)
+        torch.cuda.synchronize()
+        t = dp.sd.kv_tables()
+        assert t["status"][0] == 0
+        results.append(([(o.attn.clone(), o.token.clone(), o.accepted_len.clone(), o.out_tokens.clone()) for o in outs], t))
+    for other, t in results[1:]:
+        for a, b in zip(results[0][0], other):
+            assert all(torch.equal(u, v) for u, v in zip(a, b))
+        assert np.array_equal(t["seq_len"], results[0][1]["seq_len"]) and np.array_equal(t["page_table"], results[0][1]["page_table"])
+    with pytest.raises(Exception):
+        dp.sd.set_option(OPT_ATTN_EARLY_PREFETCH, -2)
 
 
 def test_steps_replayed_from_a_cuda_graph_match_eager_steps():
