@@ -436,6 +436,18 @@ sdlm_status sdlm_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t H, const void* x, 
 sdlm_status sdlm_linear_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t K, int32_t N, const void* x, const void* w,
                                 const void* bias, const void* residual, void* out, const void* norm_weight,
                                 float eps, void* norm_out, void* stream);
+/* sdlm_linear3 of a layer's stacked q / k / v weight followed by sdlm_rope_block2 of the query and key rows
+ * (Sec. 4.1, the Qwen-2.5 attention input), as one call:
+ *   [q | k | v] = x w^T (+ bias),  q [batch, D, n_heads, head_dim] and k [batch, D, n_heads2, head_dim] rotated
+ *   at positions (length of slot seq_ids[b], or b) + j, v [batch, D, n_heads2, head_dim] as it is.
+ * x [batch * D, K], w [(n_heads + 2 n_heads2) * head_dim, K], bias of that many entries or NULL: device bf16,
+ * 16-byte aligned; seq_ids DEVICE int32 [batch] or NULL; K % 8 == 0, head_dim % 16 == 0 (else UNSUPPORTED).
+ * Same values, bit for bit, as the two calls: where the product is cut along K and has at most 128 rows, the
+ * kernel that adds the K ranges rotates the rows it has just rounded; otherwise the rotary kernel follows the product.
+ * Errors: INVALID_ARG, SHAPE (batch above max_batch), UNSUPPORTED, CUDA. */
+sdlm_status sdlm_linear3_rope(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, int32_t K, int32_t n_heads,
+                              int32_t n_heads2, const void* x, const void* w, const void* bias, void* q, void* k, void* v,
+                              float theta, void* stream);
 sdlm_status sdlm_rope_block(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, int32_t n_heads, void* x,
                             float theta, void* stream);
 sdlm_status sdlm_rope_block2(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, int32_t n_heads, void* x,

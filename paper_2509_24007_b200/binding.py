@@ -35,7 +35,7 @@ EXPORTED = ["sdlm_pool_bytes", "sdlm_workspace_bytes", "sdlm_create", "sdlm_dest
             "sdlm_device_status", "sdlm_decode_step", "sdlm_decode_step_host", "sdlm_set_option", "sdlm_launch_count",
             "sdlm_block_attn_masked", "sdlm_verify_commit", "sdlm_accept_commit_carry",
             "sdlm_block_attn_verify", "sdlm_block_attn_carry", "sdlm_causal_attn",
-            "sdlm_linear", "sdlm_linear3", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu", "sdlm_selftest_bounded_wait", "sdlm_rope_block2", "sdlm_accept_commit_layers", "sdlm_block_attn_prefix", "sdlm_linear_swiglu",
+            "sdlm_linear", "sdlm_linear3", "sdlm_linear3_rope", "sdlm_rmsnorm", "sdlm_rope_block", "sdlm_swiglu", "sdlm_selftest_bounded_wait", "sdlm_rope_block2", "sdlm_accept_commit_layers", "sdlm_block_attn_prefix", "sdlm_linear_swiglu",
             "sdlm_block_attn_masked_prefix", "sdlm_linear_rmsnorm"]
 
 
@@ -154,6 +154,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdlm_linear_swiglu.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
     lib.sdlm_linear3.restype = C.c_int
     lib.sdlm_linear3.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+    lib.sdlm_linear3_rope.restype = C.c_int
+    lib.sdlm_linear3_rope.argtypes = [vp, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, f32, vp]
     lib.sdlm_rmsnorm.restype = C.c_int
     lib.sdlm_rmsnorm.argtypes = [vp, i32, i32, vp, vp, f32, vp, vp]
     lib.sdlm_rope_block.restype = C.c_int
@@ -539,6 +541,21 @@ class Sdlm:
                                                           _ptr(_dev(out1, torch.bfloat16, "out1")),
                                                           _ptr(_dev(out2, torch.bfloat16, "out2")),
                                                           _ptr(_dev(out3, torch.bfloat16, "out3")), _stream_ptr(stream)))
+
+    def linear3_rope(self, x: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor], q: torch.Tensor, k: torch.Tensor,
+                     v: torch.Tensor, theta: float, seq_ids: Optional[torch.Tensor] = None, stream=None) -> None:
+        """sdlm_linear3_rope: q [batch, D, n_heads, d], k and v [batch, D, n_heads2, d] from x [batch * D, K] and the
+        stacked weight; q and k come out rotated."""
+        _dev(x, torch.bfloat16, "x"); _dev(w, torch.bfloat16, "w")
+        batch, D, K = int(q.shape[0]), int(q.shape[1]), int(w.shape[1])
+        if x.numel() != batch * D * K or k.shape != v.shape or tuple(k.shape[:2]) != (batch, D):
+            raise ValueError("x must be [batch * D, K]; k and v [batch, D, n_heads2, d]")
+        if (int(q.shape[2]) + 2 * int(k.shape[2])) * int(q.shape[3]) != int(w.shape[0]):
+            raise ValueError("the three outputs must take all of w's rows")
+        self._check("sdlm_linear3_rope", self.lib.sdlm_linear3_rope(
+            self.ctx, batch, D, _ptr(seq_ids), K, int(q.shape[2]), int(k.shape[2]), _ptr(x), _ptr(w), _ptr(bias),
+            _ptr(_dev(q, torch.bfloat16, "q")), _ptr(_dev(k, torch.bfloat16, "k")), _ptr(_dev(v, torch.bfloat16, "v")),
+            float(theta), _stream_ptr(stream)))
 
     def linear_swiglu(self, x: torch.Tensor, w_interleaved: torch.Tensor, out: Optional[torch.Tensor] = None,
                       stream=None) -> torch.Tensor:

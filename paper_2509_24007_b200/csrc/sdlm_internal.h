@@ -177,9 +177,34 @@ struct LinNorm {
   float eps;
   void* out;
 };
+// One pair of the rotary embedding (rotate-half convention): elements i and i + d/2 of a head at position `pos`,
+//   lo' = lo cos(a) - hi sin(a),  hi' = hi cos(a) + lo sin(a),  a = pos * theta^(-2i/d).
+// Every kernel that rotates goes through this function, so that they agree bit for bit.
+#ifdef __CUDACC__
+__device__ __forceinline__ void rope_pair(float lo, float hi, float pos, int i, int d, float log2_theta, float& out_lo,
+                                          float& out_hi) {
+  const float inv_freq = exp2f(-log2_theta * (float)(2 * i) / (float)d);
+  float sn, cs;
+  sincosf(pos * inv_freq, &sn, &cs);
+  out_lo = lo * cs - hi * sn;
+  out_hi = hi * cs + lo * sn;
+}
+#endif
+// Rotary embedding of the first two outputs of a three-output product (a layer's query and key rows), applied
+// where the product's rows are rounded: row r of the product is block row (r / D, r % D).
+struct LinRope {
+  const int32_t* seq_len;
+  const int32_t* seq_ids;  // or null
+  int D, d;
+  float log2_theta;
+};
 sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, const void* w, const void* bias,
                           const void* residual, void* out, cudaStream_t st, int seg1 = 0, int seg2 = 0,
-                          void* out2 = nullptr, void* out3 = nullptr, int act = 0, const LinNorm* norm = nullptr);
+                          void* out2 = nullptr, void* out3 = nullptr, int act = 0, const LinNorm* norm = nullptr,
+                          const LinRope* rope = nullptr);
+// x / x2: the rows [row0, row0 + n_rows) of the two tensors, i.e. already offset to row0.
+cudaError_t launch_rope_rows(sdlm_ctx* ctx, void* x, void* x2, const LinRope& r, int row0, int n_rows, int n_heads, int n_heads2,
+                             cudaStream_t st);
 cudaError_t launch_rmsnorm(sdlm_ctx* ctx, int rows, int H, const void* x, const void* weight, float eps, void* out,
                            cudaStream_t st);
 cudaError_t launch_pending_merge(sdlm_ctx* ctx, cudaStream_t st);

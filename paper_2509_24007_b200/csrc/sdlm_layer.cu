@@ -70,14 +70,12 @@ __global__ void __launch_bounds__(256) rope_block_kernel(__nv_bfloat16* x, __nv_
     const int j = (int)(r % D), b = (int)(r / D);
     const int slot = seq_ids ? seq_ids[b] : b;
     const float pos = (float)(seq_len[slot] + j);
-    const float inv_freq = exp2f(-log2_theta * (float)(2 * i) / (float)d);
-    float sn, cs;
-    sincosf(pos * inv_freq, &sn, &cs);
     __nv_bfloat16* p = hh < n_heads ? x + (((size_t)b * D + j) * n_heads + hh) * d
                                     : x2 + (((size_t)b * D + j) * n_heads2 + (hh - n_heads)) * d;
-    const float a = __bfloat162float(p[i]), c = __bfloat162float(p[i + half]);
-    p[i] = __float2bfloat16_rn(a * cs - c * sn);
-    p[i + half] = __float2bfloat16_rn(c * cs + a * sn);
+    float lo, hi;
+    rope_pair(__bfloat162float(p[i]), __bfloat162float(p[i + half]), pos, i, d, log2_theta, lo, hi);
+    p[i] = __float2bfloat16_rn(lo);
+    p[i + half] = __float2bfloat16_rn(hi);
   }
 }
 
@@ -171,6 +169,45 @@ extern "C" sdlm_status sdlm_linear_rmsnorm(sdlm_ctx* ctx, int32_t rows, int32_t 
                        0, &norm);
 }
 
+namespace sdlm {
+// Rows [row0, row0 + n_rows) of the block tensors (row = b * D + j), for a product that rotates its own q / k rows
+// but was not cut along K, so that no second kernel rounds them.
+__global__ void __launch_bounds__(256) rope_rows_kernel(__nv_bfloat16* x, __nv_bfloat16* x2, const int32_t* seq_len,
+                                                        const int32_t* seq_ids, int row0, int n_rows, int D, int n_heads,
+                                                        int n_heads2, int d, float log2_theta) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
+  const int half = d / 2;
+  const int heads = n_heads + n_heads2;
+  const size_t total = (size_t)n_rows * heads * half;
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
+    const int i = (int)(idx % half);
+    size_t r = idx / half;
+    const int hh = (int)(r % heads);
+    const size_t row = r / heads;  // x and x2 start at row0
+    const int grow = row0 + (int)row;
+    const int b = grow / D, j = grow % D;
+    const int slot = seq_ids ? seq_ids[b] : b;
+    const float pos = (float)(seq_len[slot] + j);
+    __nv_bfloat16* p = hh < n_heads ? x + (row * n_heads + hh) * d : x2 + (row * n_heads2 + (hh - n_heads)) * d;
+    float lo, hi;
+    rope_pair(__bfloat162float(p[i]), __bfloat162float(p[i + half]), pos, i, d, log2_theta, lo, hi);
+    p[i] = __float2bfloat16_rn(lo);
+    p[i + half] = __float2bfloat16_rn(hi);
+  }
+}
+cudaError_t launch_rope_rows(sdlm_ctx* ctx, void* x, void* x2, const LinRope& r, int row0, int n_rows, int n_heads, int n_heads2,
+                             cudaStream_t st) {
+  const size_t total = (size_t)n_rows * (n_heads + n_heads2) * (r.d / 2);
+  const int blocks = (int)((total + 255) / 256 < 1184 ? (total + 255) / 256 : 1184);
+  const cudaError_t e = launch_overlapped(rope_rows_kernel, dim3(blocks), dim3(256), 0, st, static_cast<__nv_bfloat16*>(x),
+                                          static_cast<__nv_bfloat16*>(x2), r.seq_len, r.seq_ids, row0, n_rows, r.D, n_heads,
+                                          n_heads2, r.d, r.log2_theta);
+  ctx->launches++;
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+}  // namespace sdlm
+
 static sdlm_status rope_launch(sdlm_ctx* ctx, int batch, int D, const int32_t* seq_ids, int n_heads, void* x, int n_heads2,
                                void* x2, float theta, void* stream) {
   if (!ctx || !x || batch < 1 || D < 1 || n_heads < 1 || n_heads2 < 0 || (n_heads2 > 0 && !x2) || !(theta > 1.f))
@@ -195,6 +232,21 @@ extern "C" sdlm_status sdlm_rope_block2(sdlm_ctx* ctx, int32_t batch, int32_t D,
                                         void* x, int32_t n_heads2, void* x2, float theta, void* stream) {
   if (n_heads2 < 1) return SDLM_ERR_INVALID_ARG;
   return rope_launch(ctx, batch, D, seq_ids, n_heads, x, n_heads2, x2, theta, stream);
+}
+
+extern "C" sdlm_status sdlm_linear3_rope(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids, int32_t K,
+                                         int32_t n_heads, int32_t n_heads2, const void* x, const void* w, const void* bias,
+                                         void* q, void* k, void* v, float theta, void* stream) {
+  if (!ctx || !x || !w || !q || !k || !v || batch < 1 || D < 1 || K < 8 || n_heads < 1 || n_heads2 < 1 || !(theta > 1.f))
+    return SDLM_ERR_INVALID_ARG;
+  if (!a16(x) || !a16(w) || !a16(q) || !a16(k) || !a16(v) || (bias && !a16(bias))) return SDLM_ERR_INVALID_ARG;
+  if (batch > ctx->cfg.max_batch) return SDLM_ERR_SHAPE;
+  const int d = ctx->cfg.head_dim;
+  if (K % 8 || d % 16) return SDLM_ERR_UNSUPPORTED;
+  const LinRope rope{(const int32_t*)ctx->seq_len, seq_ids, D, d, log2f(theta)};
+  const int N1 = n_heads * d, N2 = n_heads2 * d;
+  return launch_linear(ctx, batch * D, K, N1 + 2 * N2, x, w, bias, nullptr, q, static_cast<cudaStream_t>(stream), N1, N1 + N2,
+                       k, v, 0, nullptr, &rope);
 }
 
 extern "C" sdlm_status sdlm_swiglu(sdlm_ctx* ctx, int32_t rows, int32_t I, const void* gate_up, void* out, void* stream) {

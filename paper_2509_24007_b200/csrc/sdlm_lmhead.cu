@@ -861,6 +861,52 @@ __global__ void __launch_bounds__(256) linear_reduce_kernel(const float* part, i
   }
 }
 
+// The same sums for a three-output product whose first two outputs are a layer's query and key rows: a thread
+// adds the K ranges for the two eight-column chunks that hold elements i and i + d/2 of one head, rounds them as
+// linear_reduce_kernel does, rotates the pairs (rope_pair) and rounds again, so the result equals that kernel
+// followed by the rotary kernel bit for bit.  The third output's chunks are summed and stored as they are.
+// Row `row` of this block of rows is block row (row0 + row) / D, position (row0 + row) % D.
+__global__ void __launch_bounds__(256) linear_reduce_rope_kernel(const float* part, int ksplit, int rows, int N,
+                                                                 const __nv_bfloat16* bias, __nv_bfloat16* out, int seg1,
+                                                                 int seg2, __nv_bfloat16* out2, __nv_bfloat16* out3,
+                                                                 LinRope rp, int row0) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
+  const int units_qk = seg2 / 16, units = units_qk + (N - seg2) / 8;
+  const int cpd = rp.d / 16;  // pairs of chunks per head
+  const size_t total = (size_t)rows * units;
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
+    const int u = (int)(idx % units);
+    const size_t row = idx / units;
+    if (u >= units_qk) {
+      const int c = seg2 / 8 + (u - units_qk);
+      *reinterpret_cast<uint4*>(out3 + row * (N - seg2) + (c * 8 - seg2)) = reduce_chunk(part, ksplit, row, N, c, bias, nullptr);
+      continue;
+    }
+    const int head = u / cpd, ci = u % cpd;
+    const int c_lo = head * (rp.d / 8) + ci;
+    uint4 o_lo = reduce_chunk(part, ksplit, row, N, c_lo, bias, nullptr);
+    uint4 o_hi = reduce_chunk(part, ksplit, row, N, c_lo + cpd, bias, nullptr);
+    const int grow = row0 + (int)row;
+    const int b = grow / rp.D, j = grow % rp.D;
+    const int slot = rp.seq_ids ? rp.seq_ids[b] : b;
+    const float pos = (float)(rp.seq_len[slot] + j);
+    __nv_bfloat16* lo = reinterpret_cast<__nv_bfloat16*>(&o_lo);
+    __nv_bfloat16* hi = reinterpret_cast<__nv_bfloat16*>(&o_hi);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      float a, c;
+      rope_pair(__bfloat162float(lo[e]), __bfloat162float(hi[e]), pos, ci * 8 + e, rp.d, rp.log2_theta, a, c);
+      lo[e] = __float2bfloat16_rn(a);
+      hi[e] = __float2bfloat16_rn(c);
+    }
+    const int n = c_lo * 8;  // a head never straddles a segment
+    __nv_bfloat16* dst = n < seg1 ? out + row * seg1 + n : out2 + row * (seg2 - seg1) + (n - seg1);
+    *reinterpret_cast<uint4*>(dst) = o_lo;
+    *reinterpret_cast<uint4*>(dst + rp.d / 2) = o_hi;
+  }
+}
+
 // The same sums for a product whose rows are normalised next: one thread block per row adds the K ranges,
 // bias and residual, rounds and stores the row, and writes RMSNorm(row) * weight beside it.  The sums, the
 // rounding and the order of the squares are those of linear_reduce_kernel followed by the row-wise norm
@@ -1126,7 +1172,10 @@ static sdlm_status launch_lmhead_on(sdlm_ctx* ctx, int rows, const void* hidden,
 // out[rows, N] = x[rows, K] W[N, K]^T (+ residual), bf16 in and out, fp32 accumulation; row blocks of 128.
 sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, const void* w, const void* bias,
                           const void* residual, void* out, cudaStream_t st, int seg1, int seg2, void* out2, void* out3,
-                          int act, const LinNorm* norm) {
+                          int act, const LinNorm* norm, const LinRope* rope) {
+  // With one block of rows the rotation rides on the sum of the K ranges; with several, each block's sum must end
+  // before the next block's product reuses the partial sums, so a longer sum delays the chain: rotate once at the end.
+  bool rotated = false;
   for (int r0 = 0; r0 < rows; r0 += 128) {
     const int nr = rows - r0 < 128 ? rows - r0 : 128;
     LmParams p{};
@@ -1218,6 +1267,16 @@ sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, 
       if (le != cudaSuccess || cudaGetLastError() != cudaSuccess) return SDLM_ERR_CUDA;
       continue;
     }
+    if (p.ksplit > 1 && rope && rows <= 128) {
+      rotated = true;
+      const size_t total = (size_t)nr * (seg2 / 16 + (N - seg2) / 8);
+      const int blocks = (int)((total + 255) / 256);
+      le = launch_overlapped(linear_reduce_rope_kernel, dim3(blocks), dim3(256), 0, st, (const float*)p.part, p.ksplit, nr, N,
+                             p.bias, p.out, p.seg1, p.seg2, p.out2, p.out3, *rope, r0);
+      ctx->launches++;
+      if (le != cudaSuccess || cudaGetLastError() != cudaSuccess) return SDLM_ERR_CUDA;
+      continue;
+    }
     if (p.ksplit > 1) {
       const size_t total = (size_t)nr * (N / 8);
       const int blocks = (int)((total + 255) / 256);
@@ -1228,6 +1287,9 @@ sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, 
     }
     if (norm && launch_rmsnorm(ctx, nr, N, p.out, norm->weight, norm->eps, norm_out, st) != cudaSuccess) return SDLM_ERR_CUDA;
   }
+  if (rope && !rotated &&
+      launch_rope_rows(ctx, out, out2, *rope, 0, rows, seg1 / rope->d, (seg2 - seg1) / rope->d, st) != cudaSuccess)
+    return SDLM_ERR_CUDA;
   return SDLM_OK;
 }
 

@@ -211,8 +211,7 @@ class DecoderStack:
         self.h.copy_(h0.reshape(self.h.shape))
         self.ctx[0].rmsnorm(self.h, self.layers[0].ln1, self.EPS, self.x, stream=stream)
         for l, (sd, w) in enumerate(zip(self.ctx, self.layers)):
-            sd.linear3(self.x, self.wqkv[l], self.bqkv[l], self.q, self.k[l], self.v[l], stream=stream)
-            sd.rope_block2(self.q, self.k[l], self.THETA, stream=stream)
+            sd.linear3_rope(self.x, self.wqkv[l], self.bqkv[l], self.q, self.k[l], self.v[l], self.THETA, stream=stream)
             sd.block_attn(self.q, self.k[l], self.v[l], self.attn, stream=stream)
             # the residual stream is updated in place and its norm for the next product comes with it
             sd.linear_rmsnorm(self.attn, w.wo, w.ln2, self.EPS, None, self.h, self.h, self.x, stream=stream)

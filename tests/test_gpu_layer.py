@@ -170,6 +170,42 @@ def test_rope_of_the_block_uses_the_positions_after_the_cached_history(n_heads, 
     assert np.max(np.abs(_f64(y) - ref2)) <= 2.0 ** -8 * np.max(np.abs(ref2)) + 4e-3
 
 
+@pytest.mark.parametrize("batch,D,K,heads", [(3, 4, 256, (4, 1)), (40, 4, 2048, (4, 2)), (32, 4, 2048, (4, 2)), (5, 3, 2048, (16, 2)), (33, 8, 1024, (2, 2))])
+def test_qkv_product_with_rotary_equals_the_two_calls_and_the_oracle(batch, D, K, heads):
+    """One call for a layer's q / k / v rows: the same bits as the product followed by the rotary call, whether
+    the product is cut along K (the rotation rides on the sum of the K ranges) or not, over several row blocks,
+    with and without seq_ids."""
+    lens = tuple(int(v) for v in np.random.default_rng(batch).integers(0, 500, size=batch))
+    dp = _ctx(lens, D=D)
+    d, theta = dp.wl.shape.head_dim, 1.0e6
+    hq, hk = heads
+    rng = np.random.default_rng(batch + K)
+    _, x64, x = _bf16(rng, (batch * D, K))
+    _, w64, w = _bf16(rng, ((hq + 2 * hk) * d, K), std=K ** -0.5)
+    _, b64, b = _bf16(rng, ((hq + 2 * hk) * d,))
+    new = lambda h: torch.full((batch, D, h, d), 7.0, dtype=torch.bfloat16, device="cuda")
+    for ids in (None, torch.tensor(np.random.default_rng(1).permutation(batch).astype(np.int32)).cuda()):
+        q, k, v = new(hq), new(hk), new(hk)
+        q1, k1, v1 = new(hq), new(hk), new(hk)
+        dp.sd.linear3_rope(x, w, b, q, k, v, theta, seq_ids=ids)
+        dp.sd.linear3(x, w, b, q1, k1, v1)
+        dp.sd.rope_block2(q1, k1, theta, seq_ids=ids)
+        torch.cuda.synchronize()
+        assert dp.sd.device_status()[0] == 0
+        assert torch.equal(q, q1) and torch.equal(k, k1) and torch.equal(v, v1)
+    # against the oracle: product rounded to bf16, then the rotation (slots in the last order used)
+    prod = lo.linear(x64, w64, b64)
+    rb = lambda a: syn.bf16_bits_to_f32(syn.f32_to_bf16_bits(a.astype(np.float32))).astype(np.float64)
+    order = ids.cpu().numpy()
+    pos = np.asarray(lens)[order][:, None] + np.arange(D)[None, :]
+    ref_q = lo.rope(rb(prod[:, :hq * d]).reshape(batch, D, hq, d), pos, theta)
+    ref_k = lo.rope(rb(prod[:, hq * d:(hq + hk) * d]).reshape(batch, D, hk, d), pos, theta)
+    for got, ref in ((q, ref_q), (k, ref_k)):
+        assert np.max(np.abs(_f64(got) - ref)) <= 2.0 ** -7 * np.max(np.abs(ref)) + 4e-3
+    _check_bf16(_f64(v).reshape(batch * D, -1), prod[:, (hq + hk) * d:], "v of linear3_rope")
+    assert dp.sd.linear3_rope.__doc__
+
+
 @pytest.mark.parametrize("rows,I", [(1, 8), (9, 1000), (128, 11008)])
 def test_swiglu_matches_the_oracle(rows, I):
     dp = _ctx()
