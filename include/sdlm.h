@@ -383,9 +383,12 @@ sdlm_status sdlm_decode_step(sdlm_ctx* ctx, int32_t batch, int32_t D, const int3
  * can address (cudaHostAlloc / cudaHostRegister) is written by the kernels directly, without a
  * copy after the step; its contents are defined once the call has returned.  Likewise q, k_blk and
  * v_blk in such memory (16-byte aligned) are not staged: attention and the commit read those rows,
- * once each, straight from the host buffer, which must stay unchanged until the call returns;
- * hidden is always copied (every thread block of the LM head re-reads it).  w_lm stays a DEVICE
- * pointer (model state).
+ * once each, straight from the host buffer, which must stay unchanged until the call returns (q only while
+ * few thread blocks share its rows: see SDLM_OPT_HOST_INPLACE_MAX_KB);
+ * hidden always ends up in device memory (every thread block of the LM head re-reads it): by a copy in front of
+ * the kernels, or, when it lies in such memory and the step runs in order on one stream, fetched by otherwise
+ * idle warps of the attention kernel, the LM head then waiting for that kernel (SDLM_OPT_HOST_HIDDEN_BY_ATTN).
+ * w_lm stays a DEVICE pointer (model state).
  * Errors: as the three calls, plus CUDA. */
 sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32_t D, const int32_t* seq_ids_host,
                                   float tau, sdlm_conf_mode mode, const void* q_host, const void* k_blk_host,
@@ -477,8 +480,16 @@ sdlm_status sdlm_swiglu(sdlm_ctx* ctx, int32_t rows, int32_t I, const void* gate
  * way).  The cached history is not produced by that
  * kernel; the tables are read as they stand at that moment and only steer the prefetch: results do not depend
  * on the option.
+ * SDLM_OPT_HOST_HIDDEN_BY_ATTN: 0..2.  sdlm_decode_step_host, in order on one stream, has the attention kernel
+ * fetch a page-locked, GPU-addressable `hidden` instead of copying it first: 2 always, 1 (default) when `hidden`
+ * holds at least 384 KB (below that the copy is as cheap as the LM head's wait for attention), 0 never.
+ * SDLM_OPT_HOST_INPLACE_MAX_KB: 0..2^20 (default 2^20).  sdlm_decode_step_host uses a page-locked, GPU-addressable
+ * q, k_blk, v_blk or attn_out buffer in place only up to this size; larger ones go through a copy (0: all are
+ * copied).  Within the limit q is still copied when the (sequence, KV head) pairs are cut over several thread
+ * blocks often enough that its rows would cross the bus more than about a megabyte more than once.
+ * Results depend on neither option.
  * Errors: INVALID_ARG. */
-typedef enum sdlm_option { SDLM_OPT_LMHEAD_KERNEL = 0, SDLM_OPT_STEP_OVERLAP = 1, SDLM_OPT_ATTN_ITEM_COST = 2, SDLM_OPT_ATTN_MIN_RANGE = 3, SDLM_OPT_HOST_TWO_STREAMS = 4, SDLM_OPT_ATTN_EARLY_PREFETCH = 5 } sdlm_option;
+typedef enum sdlm_option { SDLM_OPT_LMHEAD_KERNEL = 0, SDLM_OPT_STEP_OVERLAP = 1, SDLM_OPT_ATTN_ITEM_COST = 2, SDLM_OPT_ATTN_MIN_RANGE = 3, SDLM_OPT_HOST_TWO_STREAMS = 4, SDLM_OPT_ATTN_EARLY_PREFETCH = 5, SDLM_OPT_HOST_HIDDEN_BY_ATTN = 6, SDLM_OPT_HOST_INPLACE_MAX_KB = 7 } sdlm_option;
 sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t value);
 
 /* Self-test of the bounded waits (the paper has no counterpart): launches one thread block that waits on

@@ -26,6 +26,8 @@ OPT_ATTN_ITEM_COST = 2
 OPT_ATTN_MIN_RANGE = 3
 OPT_HOST_TWO_STREAMS = 4
 OPT_ATTN_EARLY_PREFETCH = 5
+OPT_HOST_HIDDEN_BY_ATTN = 6
+OPT_HOST_INPLACE_MAX_KB = 7
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "UNSUPPORTED", 4: "OUT_OF_PAGES", 5: "CUDA",
                 6: "TIMEOUT", 7: "DEVICE_CHECK", 8: "WORKSPACE"}

@@ -527,12 +527,17 @@ extern "C" sdlm_status sdlm_create(const sdlm_config* cfg, void* kv_pool, size_t
   ctx->lmhead_path = 0;
   ctx->overlap_lmhead = 0;
   ctx->host_two_streams = 0;
+  ctx->host_hidden_by_attn = 1;
+  ctx->host_inplace_max_kb = 1 << 20;
   ctx->side_stream = nullptr;
   ctx->ev_fork = ctx->ev_join = nullptr;
   ctx->attn_item_cost = 8;
   ctx->attn_min_range = 8;
   ctx->attn_early_prefetch = -1;
   ctx->in_decode_step = 0;
+  ctx->attn_side_src = nullptr;
+  ctx->attn_side_dst = nullptr;
+  ctx->attn_side_chunks = 0;
   ctx->tmap_w_ptr = nullptr;
   ctx->tmap_w_rows = 0;
   ctx->tmap_h_ptr = nullptr;
@@ -567,6 +572,14 @@ extern "C" sdlm_status sdlm_set_option(sdlm_ctx* ctx, sdlm_option opt, int32_t v
     case SDLM_OPT_HOST_TWO_STREAMS:
       if (value < 0 || value > 1) return SDLM_ERR_INVALID_ARG;
       ctx->host_two_streams = value;
+      return SDLM_OK;
+    case SDLM_OPT_HOST_HIDDEN_BY_ATTN:
+      if (value < 0 || value > 2) return SDLM_ERR_INVALID_ARG;
+      ctx->host_hidden_by_attn = value;
+      return SDLM_OK;
+    case SDLM_OPT_HOST_INPLACE_MAX_KB:
+      if (value < 0 || value > (1 << 20)) return SDLM_ERR_INVALID_ARG;
+      ctx->host_inplace_max_kb = value;
       return SDLM_OK;
     case SDLM_OPT_ATTN_ITEM_COST:
       if (value < 0 || value > 64) return SDLM_ERR_INVALID_ARG;
@@ -1087,10 +1100,24 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
     ok &= cudaEventRecord(ctx->ev_fork, st) == cudaSuccess;          // whatever the caller enqueued before comes first
     ok &= cudaStreamWaitEvent(qkv_st, ctx->ev_fork, 0) == cudaSuccess;
   }
-  ok &= cudaMemcpyAsync(ws + L.st_hidden, hidden_host, rows * c.hidden * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  const void* in_q = mapped16(q_host);
-  const void* in_k = mapped16(k_blk_host);
-  const void* in_v = mapped16(v_blk_host);
+  // `hidden` in page-locked memory that the GPU can address (in-order step on one stream): no copy in front of the
+  // kernels; the attention kernel's epilogue warps, idle until their first item ends, fetch it, and the LM head,
+  // which streams its first weight tiles before it waits, takes attention's completion as a full dependency.
+  // (Below 384 KB the copy is short and the LM head's wait for the end of attention costs as much: measured.)
+  const bool fetch_hidden = ctx->host_hidden_by_attn == 2 || (ctx->host_hidden_by_attn == 1 && rows * c.hidden * 2 >= 384u * 1024u);
+  const void* m_hidden = a_sms == 0 && ctx->overlap_lmhead == 0 && fetch_hidden ? mapped16(hidden_host) : nullptr;
+  if (!m_hidden)
+    ok &= cudaMemcpyAsync(ws + L.st_hidden, hidden_host, rows * c.hidden * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  const size_t inplace_max = (size_t)ctx->host_inplace_max_kb << 10;
+  // The query rows are read by every thread block that has a share of their (sequence, KV head) pair: with few
+  // pairs for the SMs each row crosses the bus several times, and beyond about a megabyte of such re-reads a copy
+  // in front of the kernel is cheaper (measured on the 3B-shaped steps: batch 32 D = 4 in place, D = 8 and the
+  // batch-8 32k-token step copied; the 32B-shaped batch-64 step, whose pairs are not cut, in place).
+  const double cuts = (double)ctx->sm_count / ((double)batch * c.n_kv_heads) - 1.0;
+  const bool q_inplace = q_bytes <= inplace_max && (cuts <= 0.0 || (double)q_bytes * cuts <= 1048576.0);
+  const void* in_q = q_inplace ? mapped16(q_host) : nullptr;
+  const void* in_k = kv_bytes <= inplace_max ? mapped16(k_blk_host) : nullptr;
+  const void* in_v = kv_bytes <= inplace_max ? mapped16(v_blk_host) : nullptr;
   if (!in_q) {
     ok &= cudaMemcpyAsync(ws + L.st_q, q_host, q_bytes, cudaMemcpyHostToDevice, qkv_st) == cudaSuccess;
     in_q = ws + L.st_q;
@@ -1114,14 +1141,20 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
   float* d_ent = reinterpret_cast<float*>(ws + L.st_ent);
   int32_t* d_acc = reinterpret_cast<int32_t*>(ws + L.st_acc);
   int32_t* d_out_tokens = reinterpret_cast<int32_t*>(ws + L.st_out_tokens);
-  void* m_attn = mapped16(attn_out_host);
+  void* m_attn = q_bytes <= inplace_max ? mapped16(attn_out_host) : nullptr;
   void* d_attn = m_attn ? m_attn : ws + L.st_out;
   const int overlap = ctx->overlap_lmhead;  // A: attention's SMs in the side-by-side step (0: in order)
   ctx->defer_merge = overlap > 0 && a_sms == 0;  // side by side on one stream: the merge follows the LM head
   ctx->in_decode_step = overlap == 0;
+  if (m_hidden) {
+    ctx->attn_side_src = m_hidden;
+    ctx->attn_side_dst = ws + L.st_hidden;
+    ctx->attn_side_chunks = (uint32_t)(rows * c.hidden * 2 / 16);
+  }
   const cudaError_t ae =
       launch_block_attn(ctx, batch, D, seq_ids, in_q, in_k, in_v, d_attn, qkv_st, overlap, overlap > 0 && batch * D > 128);
   ctx->in_decode_step = 0;
+  ctx->attn_side_src = nullptr;
   ctx->defer_merge = 0;
   if (ae != cudaSuccess) return SDLM_ERR_CUDA;
   if (a_sms > 0 && cudaEventRecord(ctx->ev_join, qkv_st) != cudaSuccess) return SDLM_ERR_CUDA;
@@ -1129,7 +1162,7 @@ extern "C" sdlm_status sdlm_decode_step_host(sdlm_ctx* ctx, int32_t batch, int32
   // copy of `hidden` before it lets the LM head go); on two streams it follows the copy of `hidden`
   // and takes its wait as a full dependency
   s = launch_lmhead(ctx, batch * D, ws + L.st_hidden, w_lm, d_token, d_p, d_ent, nullptr, nullptr, st,
-                    /*independent_of_predecessor=*/a_sms == 0, overlap > 0 ? ctx->sm_count - overlap : 0);
+                    /*independent_of_predecessor=*/a_sms == 0 && !m_hidden, overlap > 0 ? ctx->sm_count - overlap : 0);
   if (launch_pending_merge(ctx, st) != cudaSuccess) return SDLM_ERR_CUDA;
   if (s != SDLM_OK) return s;
   if (a_sms > 0 && cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return SDLM_ERR_CUDA;

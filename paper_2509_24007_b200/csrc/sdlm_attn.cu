@@ -97,7 +97,28 @@ struct AttnParams {
   // null, or [batch]: row b sees only the first prefix_len[b] cached tokens of its slot (several rows may
   // name the same slot: the noise blocks of one training sequence)
   const int32_t* prefix_len;
+  // An unrelated copy that rides on this kernel (null / 0: none): side_chunks 16-byte chunks from side_src, which
+  // the GPU can address but which may lie in host memory, to side_dst in device memory, done by the epilogue
+  // warps of every thread block before their first item is ready.  The host-buffer step uses it to bring the
+  // LM head's hidden rows in without a copy in front of the kernels.
+  const uint4* side_src;
+  uint4* side_dst;
+  uint32_t side_chunks;
 };
+
+// The thread block's share of the side copy: `n_thr` threads, thread `t`; loads first, then stores.
+__device__ __forceinline__ void attn_side_copy(const AttnParams& p, int t, int n_thr) {
+  const uint32_t stride = gridDim.x * (uint32_t)n_thr;
+  for (uint32_t i = blockIdx.x * (uint32_t)n_thr + (uint32_t)t; i < p.side_chunks; i += 4 * stride) {
+    uint4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (i + u * stride < p.side_chunks) v[u] = __ldcv(p.side_src + i + u * stride);
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (i + u * stride < p.side_chunks) p.side_dst[i + u * stride] = v[u];
+  }
+}
 
 enum { kVisNone = 0, kVisWords = 1, kVisVerify = 2, kVisCarry = 3 };
 
@@ -462,6 +483,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
   ItemWalk w0;
   walk_begin(w0, s_first, p.batch, p.Hkv, p.min_range);
   if (!walk_next(w0, p, i0)) {  // no tile falls into this CTA's range (uniform for the CTA)
+    if (p.side_chunks && warp >= W_EPI) attn_side_copy(p, tid - W_EPI * 32, 128);
     if (warp == 1) ptx::tmem_dealloc(*tmem_slot, TMEM_COLS);
     return;
   }
@@ -986,6 +1008,7 @@ __global__ void __launch_bounds__(attn_threads(NQ), 1) block_attn_umma_kernel(co
     // the last of the pair's thread blocks to arrive.  Runs beside the next item's scores and sums.
     const int ew = warp - W_EPI;
     const int t = ew * 32 + lane;  // accumulator lane = output column
+    if (p.side_chunks) attn_side_copy(p, t, 128);  // these warps have nothing to do until the first item ends
     const uint32_t lane_addr = tmem_base + ((uint32_t)(ew * 32) << 16);
     ItemWalk w = w0;  // the walk behind the first item, which every thread has worked out already
     Item it = i0;
@@ -1334,6 +1357,9 @@ cudaError_t launch_block_attn(sdlm_ctx* ctx, int batch, int D, const int32_t* se
     p.q_first = mask->q_first;
   }
   p.prefix_len = prefix_len;
+  p.side_src = static_cast<const uint4*>(ctx->attn_side_src);
+  p.side_dst = static_cast<uint4*>(ctx->attn_side_dst);
+  p.side_chunks = ctx->attn_side_src ? ctx->attn_side_chunks : 0u;
   // the kernel's tile arithmetic is 32-bit: (tiles of the launch) x (CTAs) must stay below 2^31
   if ((long long)batch * (c.max_pages_per_seq + 1 + ctx->attn_item_cost) * c.n_kv_heads > 13000000ll)
     return cudaErrorInvalidConfiguration;

@@ -67,10 +67,15 @@ struct sdlm_ctx {
   int attn_min_range;  // shortest range of schedule positions given to one attention thread block
   int attn_item_cost;  // positions the attention schedule charges for starting a (sequence, KV head) pair
   int attn_early_prefetch;  // cached tiles per thread block that attention prefetches before its dependency wait (0: off; -1: 12 inside a decode step, where the kernels before it leave the memory system idle, 0 elsewhere)
+  const void* attn_side_src;  // set around one attention launch: a copy that the kernel carries (see AttnParams)
+  void* attn_side_dst;
+  uint32_t attn_side_chunks;
   int in_decode_step;       // set around the attention launch of sdlm_decode_step / sdlm_decode_step_host
   int overlap_lmhead;  // sdlm_decode_step: SMs given to attention while the LM head runs on the rest (0: one after the other)
   // second stream and fork / join events of the host-buffer step's side-by-side mode (made on first use)
   int host_two_streams;
+  int host_inplace_max_kb;  // sdlm_decode_step_host: larger q / k / v / attn_out buffers are copied, not used in place
+  int host_hidden_by_attn;  // sdlm_decode_step_host: addressable page-locked `hidden` is fetched by the attention kernel (2: always, 1: from 384 KB) or copied first (0)
   cudaStream_t side_stream;
   cudaEvent_t ev_fork, ev_join;
   // cached TMA descriptor of the LM-head weight (keyed by pointer and tile rows)

@@ -237,6 +237,40 @@ def test_decode_step_host_entry_matches_device_calls(results, inputs):
     assert np.array_equal(t["page_table"], t_ref["page_table"]) and np.array_equal(t["seq_len"], t_ref["seq_len"])
 
 
+@pytest.mark.parametrize("name,batch", [("cfg0", 3), ("cfg2_d4", 32), ("cfg2", 20)])
+def test_decode_step_host_hidden_fetched_by_attention_equals_the_copy(name, batch):
+    """Page-locked `hidden` fetched by the attention kernel's idle warps, or copied in front of the kernels, and
+    q / k / v / attn_out used in place or through copies: the same step, bit for bit, over several steps that reuse one host buffer with new contents each time (a stale
+    cached line of host memory would show as the step before's tokens)."""
+    from paper_2509_24007_b200 import binding
+    wl = syn.CONFIGS[name].with_(batch=batch)
+    B, D, s = wl.batch, wl.block, wl.shape
+    runs = []
+    for by_attn, inplace_kb in ((2, 1 << 20), (0, 1 << 20), (2, 0), (1, 16)):
+        dp = DeviceProblem(wl)
+        dp.sd.set_option(binding.OPT_HOST_HIDDEN_BY_ATTN, by_attn)
+        dp.sd.set_option(binding.OPT_HOST_INPLACE_MAX_KB, inplace_kb)
+        q, k, v, h = (t.cpu().pin_memory() for t in (lambda x: (x.q, x.k_blk, x.v_blk, x.hidden))(dp.block(0)))
+        attn = torch.empty((B, D, s.n_q_heads, s.head_dim), dtype=torch.bfloat16).pin_memory()
+        tok, p = torch.empty((B, D), dtype=torch.int32).pin_memory(), torch.empty((B, D), dtype=torch.float32).pin_memory()
+        acc, out_tok = torch.empty(B, dtype=torch.int32).pin_memory(), torch.empty((B, D), dtype=torch.int32).pin_memory()
+        steps = []
+        for i in range(4):
+            x = dp.block(i)
+            for dst, src in ((q, x.q), (k, x.k_blk), (v, x.v_blk), (h, x.hidden)):
+                dst.copy_(src.cpu())
+            dp.sd.decode_step_host(wl.tau, q, k, v, h, dp.w_lm, attn, tok, p, None, acc, out_tok)
+            steps.append([t.clone() for t in (attn, tok, p, acc, out_tok)])
+        assert dp.sd.device_status()[0] == 0
+        runs.append((steps, dp.sd.kv_tables()))
+    a, ta = runs[0]
+    assert len({tuple(st[1].flatten().tolist()) for st in a}) > 1  # the steps differ: a stale buffer would not
+    for b, tb in runs[1:]:  # copies of everything, and of the larger buffers only: the same step
+        for sa, sb in zip(a, b):
+            assert all(torch.equal(u, w) for u, w in zip(sa, sb))
+        assert np.array_equal(ta["page_table"], tb["page_table"]) and np.array_equal(ta["seq_len"], tb["seq_len"])
+
+
 @pytest.mark.parametrize("name,batch,a_sms", [("cfg0", 3, 40), ("cfg2_d4", 6, 42), ("cfg2", 20, 36)])
 def test_decode_step_host_side_by_side_uses_two_streams_and_gives_the_same_step(name, batch, a_sms):
     """With the overlap option the host-buffer step copies `hidden` and runs the LM head on the caller's
