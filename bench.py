@@ -472,12 +472,47 @@ def time_model_level(torch, pk, wl, lengths, n_layers, intermediate, steps, warm
     ms = e0.elapsed_time(e1) / steps
     assert all(int(sd.device_status()[0]) == 0 for sd in stack.ctx), "device status set during the model-level steps"
     tokens = int(out.accepted_len.clamp(min=0).sum().item())
+
+    def per_layer_us(fn, replays=10):
+        """One of the layer's calls alone: a graph of n_layers launches, layer l on layer l's weights and cache."""
+        for l in range(n_layers):
+            fn(l, None)
+        torch.cuda.synchronize()
+        side.wait_stream(torch.cuda.current_stream())
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(gr, stream=side):
+                for l in range(n_layers):
+                    fn(l, side)
+        torch.cuda.current_stream().wait_stream(side)
+        gr.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(replays):
+            gr.replay()
+        b.record()
+        torch.cuda.synchronize()
+        return round(a.elapsed_time(b) / replays / n_layers * 1e3, 2)
+
+    st_, ly = stack, stack.layers
+    stack.restore()
+    pieces = {
+        "qkv_product_with_rotary": per_layer_us(lambda l, sm: st_.ctx[l].linear3_rope(st_.x, st_.wqkv[l], st_.bqkv[l], st_.q, st_.k[l], st_.v[l], st_.THETA, stream=sm)),
+        "block_attention": per_layer_us(lambda l, sm: st_.ctx[l].block_attn(st_.q, st_.k[l], st_.v[l], st_.attn, stream=sm)),
+        "output_projection_with_norm": per_layer_us(lambda l, sm: st_.ctx[l].linear_rmsnorm(st_.attn, ly[l].wo, ly[l].ln2, st_.EPS, None, st_.h, st_.h, st_.x, stream=sm)),
+        "gate_up_with_swiglu": per_layer_us(lambda l, sm: st_.ctx[l].linear_swiglu(st_.x, st_.wgu_il[l], st_.act, stream=sm)),
+        "down_projection_with_norm": per_layer_us(lambda l, sm: st_.ctx[l].linear_rmsnorm(st_.act, ly[l].wdown, ly[l].ln2, st_.EPS, None, st_.h, st_.h, st_.x, stream=sm)),
+    }
+    assert all(int(sd.device_status()[0]) == 0 for sd in stack.ctx), "device status set while timing the layer's calls"
     kv = syn.kv_read_bytes(wl, lengths) * n_layers
     return {"value": tokens / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "tokens_per_step": tokens,
             "layers": n_layers, "intermediate": I, "library_launches_per_step": per_step,
             "weight_bytes": stack.weight_bytes(), "kv_bytes": kv,
             "achieved_gbs": (stack.weight_bytes() + kv) / (ms * 1e-3) / 1e9,
             "batch": wl.batch, "block_D": wl.block,
+            "per_layer_call_us": pieces,
+            "per_layer_call_us_note": "each call of a layer timed alone as one CUDA graph of n_layers launches over the layers' own weights and caches",
             "what": f"whole-model step (random weights of the {label} shape), every operation a library call, one CUDA graph per step"}
 
 
