@@ -797,29 +797,43 @@ __global__ void __launch_bounds__(kMmaThreads) lmhead_mma_kernel(const LmParams 
   }
 }
 
-// Eight adjacent output columns of one row: the K ranges' partial sums in range order, then bias, then
-// residual, rounded to bf16 once.
-__device__ __forceinline__ uint4 reduce_chunk(const float* part, int ksplit, size_t row, int N, int c,
-                                              const __nv_bfloat16* bias, const __nv_bfloat16* residual) {
-  float z[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-  for (int s0 = 0; s0 < ksplit; s0 += 4) {  // four ranges' loads in flight; added in range order
-    float4 a[4], b[4];
+// Eight adjacent output columns of one row, for up to two column chunks at once: the K ranges' partial sums added
+// in range order, eight ranges' loads of both chunks in flight (the kernels that call this are bound by the
+// number of dependent trips to L2, not by bytes).
+__device__ __forceinline__ void reduce_sums(const float* part, int ksplit, size_t row, int N, int c0, int c1, bool two,
+                                            float (&z0)[8], float (&z1)[8]) {
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+  for (int i = 0; i < 8; ++i) z0[i] = z1[i] = 0.f;
+  for (int s0 = 0; s0 < ksplit; s0 += 8) {
+    float4 a0[8], b0[8], a1[8], b1[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
       if (s0 + u < ksplit) {
-        const float4* src = reinterpret_cast<const float4*>(part + ((size_t)(s0 + u) * 128 + row) * N) + 2 * c;
-        a[u] = __ldcg(src);
-        b[u] = __ldcg(src + 1);
+        const float4* base = reinterpret_cast<const float4*>(part + ((size_t)(s0 + u) * 128 + row) * N);
+        a0[u] = __ldcg(base + 2 * c0);
+        b0[u] = __ldcg(base + 2 * c0 + 1);
+        if (two) {
+          a1[u] = __ldcg(base + 2 * c1);
+          b1[u] = __ldcg(base + 2 * c1 + 1);
+        }
       }
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < 8; ++u) {
       if (s0 + u < ksplit) {
-        z[0] += a[u].x; z[1] += a[u].y; z[2] += a[u].z; z[3] += a[u].w;
-        z[4] += b[u].x; z[5] += b[u].y; z[6] += b[u].z; z[7] += b[u].w;
+        z0[0] += a0[u].x; z0[1] += a0[u].y; z0[2] += a0[u].z; z0[3] += a0[u].w;
+        z0[4] += b0[u].x; z0[5] += b0[u].y; z0[6] += b0[u].z; z0[7] += b0[u].w;
+        if (two) {
+          z1[0] += a1[u].x; z1[1] += a1[u].y; z1[2] += a1[u].z; z1[3] += a1[u].w;
+          z1[4] += b1[u].x; z1[5] += b1[u].y; z1[6] += b1[u].z; z1[7] += b1[u].w;
+        }
       }
     }
   }
+}
+// ... then bias, then residual, rounded to bf16 once.
+__device__ __forceinline__ uint4 reduce_finish(float (&z)[8], size_t row, int N, int c, const __nv_bfloat16* bias,
+                                               const __nv_bfloat16* residual) {
   if (bias) {
     const uint4 v = *(reinterpret_cast<const uint4*>(bias) + c);
     const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
@@ -836,6 +850,12 @@ __device__ __forceinline__ uint4 reduce_chunk(const float* part, int ksplit, siz
   o.x = ptx::pack_bf16(z[0], z[1]); o.y = ptx::pack_bf16(z[2], z[3]);
   o.z = ptx::pack_bf16(z[4], z[5]); o.w = ptx::pack_bf16(z[6], z[7]);
   return o;
+}
+__device__ __forceinline__ uint4 reduce_chunk(const float* part, int ksplit, size_t row, int N, int c,
+                                              const __nv_bfloat16* bias, const __nv_bfloat16* residual) {
+  float z[8], unused[8];
+  reduce_sums(part, ksplit, row, N, c, c, false, z, unused);
+  return reduce_finish(z, row, N, c, bias, residual);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -885,8 +905,10 @@ __global__ void __launch_bounds__(256) linear_reduce_rope_kernel(const float* pa
     }
     const int head = u / cpd, ci = u % cpd;
     const int c_lo = head * (rp.d / 8) + ci;
-    uint4 o_lo = reduce_chunk(part, ksplit, row, N, c_lo, bias, nullptr);
-    uint4 o_hi = reduce_chunk(part, ksplit, row, N, c_lo + cpd, bias, nullptr);
+    float z_lo[8], z_hi[8];
+    reduce_sums(part, ksplit, row, N, c_lo, c_lo + cpd, true, z_lo, z_hi);
+    uint4 o_lo = reduce_finish(z_lo, row, N, c_lo, bias, nullptr);
+    uint4 o_hi = reduce_finish(z_hi, row, N, c_lo + cpd, bias, nullptr);
     const int grow = row0 + (int)row;
     const int b = grow / rp.D, j = grow % rp.D;
     const int slot = rp.seq_ids ? rp.seq_ids[b] : b;
@@ -925,17 +947,25 @@ __global__ void __launch_bounds__(128) linear_reduce_norm_kernel(const float* pa
   uint4 hv[kNormChunks];
   float ss = 0.f;
 #pragma unroll
-  for (int k = 0; k < kNormChunks; ++k) {
-    const int c = tid + 128 * k;
-    if (c < nc) {
-      const uint4 o = reduce_chunk(part, ksplit, row, N, c, bias, residual);
-      *(reinterpret_cast<uint4*>(out + row * N) + c) = o;
-      hv[k] = o;
-      const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&o);
+  for (int k = 0; k < kNormChunks; k += 2) {
+    const int c0 = tid + 128 * k, c1 = c0 + 128;
+    if (c0 < nc) {
+      float z0[8], z1[8];
+      reduce_sums(part, ksplit, row, N, c0, c1, c1 < nc, z0, z1);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const float f = __bfloat162float(e[i]);
-        ss = fmaf(f, f, ss);
+      for (int h = 0; h < 2; ++h) {  // the squares in chunk order, as the row-wise norm kernel takes them
+        const int c = h ? c1 : c0;
+        if (c < nc) {
+          const uint4 o = reduce_finish(h ? z1 : z0, row, N, c, bias, residual);
+          *(reinterpret_cast<uint4*>(out + row * N) + c) = o;
+          hv[k + h] = o;
+          const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&o);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float f = __bfloat162float(e[i]);
+            ss = fmaf(f, f, ss);
+          }
+        }
       }
     }
   }
