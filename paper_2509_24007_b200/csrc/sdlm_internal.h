@@ -16,7 +16,8 @@ constexpr int kMaxBlockKeys = 16;    // rows of k_blk / v_blk per sequence in th
 constexpr int kMaxQRows = 64;        // (Hq/Hkv) * D stacked query rows per KV head
 constexpr int kMaxBatch = 4096;
 constexpr int kLinSplitMax = 12;      // most K ranges of a split-K linear
-constexpr int kLinSplitMaxN = 4096;   // widest output a split-K linear takes
+constexpr int kLinSplitMaxN = 4096;   // widest output that may be cut into kLinSplitMax K ranges (sizes the partial sums)
+constexpr int kLinSplitWideN = 8192;  // widest output a split-K linear takes: fewer ranges, the same partial-sum buffer
 constexpr int kLmMaxStripes = 1024;  // upper bound on vocab stripes (one partial per stripe per row)
 constexpr int kAttnMaxCtas = 160;    // upper bound on the attention grid (one CTA per SM)
 

@@ -932,8 +932,8 @@ __global__ void __launch_bounds__(256) linear_reduce_rope_kernel(const float* pa
 // The same sums for a product whose rows are normalised next: one thread block per row adds the K ranges,
 // bias and residual, rounds and stores the row, and writes RMSNorm(row) * weight beside it.  The sums, the
 // rounding and the order of the squares are those of linear_reduce_kernel followed by the row-wise norm
-// kernel, so the two ways give the same bits.  N / 8 <= 128 * kNormChunks.
-constexpr int kNormChunks = 4;
+// kernel, so the two ways give the same bits.  N / 8 <= 128 * kNormChunks (N <= 6144).
+constexpr int kNormChunks = 6;
 __global__ void __launch_bounds__(128) linear_reduce_norm_kernel(const float* part, int ksplit, int N,
                                                                  const __nv_bfloat16* bias,
                                                                  const __nv_bfloat16* residual, __nv_bfloat16* out,
@@ -1253,7 +1253,9 @@ sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, 
     p.part = reinterpret_cast<float*>(ctx->ws + ctx->lay.lin_part);
     // Every thread block of a column stripe reads all of x's K columns through its SM's L2 port (about 45 GB/s):
     // 0.4 us per K step whatever the stripe's width, 13 us for K = 2048.  K ranges divide that too.
-    if (N <= kLinSplitMaxN && KC_all >= 16 && act == 0) {
+    if (N <= kLinSplitWideN && KC_all >= 16 && act == 0) {
+      // as many ranges as the partial-sum buffer holds for this width
+      const int ks_cap = N <= kLinSplitMaxN ? kLinSplitMax : kLinSplitMax * kLinSplitMaxN / N;
       // stripe width and number of K ranges from a small cost model (us): K steps per block at the SM's
       // L2 port rate, plus the second kernel and its traffic when K is cut
       double best = 1e30;
@@ -1261,7 +1263,7 @@ sdlm_status launch_linear(sdlm_ctx* ctx, int rows, int K, int N, const void* x, 
       for (int bn_try = 64; bn_try <= 256; bn_try *= 2) {
         const int n_ct = (N + bn_try - 1) / bn_try;
         if (n_ct > ctx->sm_count) continue;
-        for (int ks = 1; ks <= kLinSplitMax && n_ct * ks <= ctx->sm_count && ks * 2 <= KC_all; ++ks) {
+        for (int ks = 1; ks <= ks_cap && n_ct * ks <= ctx->sm_count && ks * 2 <= KC_all; ++ks) {
           const int per = (KC_all + ks - 1) / ks;
           const double t = per * (16384.0 + bn_try * 128.0) / 45000.0 +
                            (ks > 1 ? 2.5 + (double)ks * nr * N * 8.0 / 3.0e6 : 0.0);

@@ -33,11 +33,13 @@ def _check_bf16(got, ref, what, rel=2.0 ** -8):
 
 
 @pytest.mark.parametrize("rows,K,N", [(1, 64, 16), (5, 72, 48), (128, 256, 1024), (129, 128, 256), (256, 2048, 512),
-                                      (33, 1000, 2512), (128, 2048, 22016)])
+                                      (33, 1000, 2512), (128, 2048, 22016), (128, 6912, 5120), (70, 2048, 8192)])
 @pytest.mark.parametrize("extras", ["plain", "bias", "residual", "both"])
 def test_linear_matches_the_oracle(rows, K, N, extras):
     if N == 22016 and extras != "both":
         pytest.skip("the large shape once")
+    if K == 6912 and extras in ("bias", "residual"):
+        pytest.skip("the long shape twice")
     dp = _ctx()
     rng = np.random.default_rng(rows + K + N)
     _, x64, x = _bf16(rng, (rows, K))
@@ -98,7 +100,9 @@ def test_linear_in_place_on_the_residual_stream():
 
 
 @pytest.mark.parametrize("rows,K,N", [(128, 2048, 2048), (128, 11008, 2048), (37, 2048, 2048), (200, 4096, 4096),
-                                      (128, 2048, 4112), (9, 72, 48), (128, 256, 1024)])
+                                      (128, 2048, 4112), (9, 72, 48), (128, 256, 1024), (128, 5120, 5120),
+                                      (150, 6912, 5120), (128, 2048, 6144), (64, 2048, 7168), (128, 1024, 8192),
+                                      (16, 1024, 8208)])
 @pytest.mark.parametrize("extras", ["plain", "both", "in place"])
 def test_product_with_the_norm_of_its_rows_equals_the_two_calls(rows, K, N, extras):
     """sdlm_linear_rmsnorm against sdlm_linear followed by sdlm_rmsnorm, bit for bit (products that are cut
@@ -170,7 +174,8 @@ def test_rope_of_the_block_uses_the_positions_after_the_cached_history(n_heads, 
     assert np.max(np.abs(_f64(y) - ref2)) <= 2.0 ** -8 * np.max(np.abs(ref2)) + 4e-3
 
 
-@pytest.mark.parametrize("batch,D,K,heads", [(3, 4, 256, (4, 1)), (40, 4, 2048, (4, 2)), (32, 4, 2048, (4, 2)), (5, 3, 2048, (16, 2)), (33, 8, 1024, (2, 2))])
+@pytest.mark.parametrize("batch,D,K,heads", [(3, 4, 256, (4, 1)), (40, 4, 2048, (4, 2)), (32, 4, 2048, (4, 2)), (5, 3, 2048, (16, 2)), (33, 8, 1024, (2, 2)),
+                                             (32, 4, 2048, (80, 16))])
 def test_qkv_product_with_rotary_equals_the_two_calls_and_the_oracle(batch, D, K, heads):
     """One call for a layer's q / k / v rows: the same bits as the product followed by the rotary call, whether
     the product is cut along K (the rotation rides on the sum of the K ranges) or not, over several row blocks,
