@@ -265,6 +265,13 @@ def test_decode_step_host_hidden_fetched_by_attention_equals_the_copy(name, batc
         runs.append((steps, dp.sd.kv_tables()))
     a, ta = runs[0]
     assert len({tuple(st[1].flatten().tolist()) for st in a}) > 1  # the steps differ: a stale buffer would not
+    # ... and the same as the three calls on device-resident inputs (which the oracle checks at these sizes)
+    dev = DeviceProblem(wl)
+    for i, sa in enumerate(a):
+        ref = dev.step(dev.block(i), wl.tau)
+        torch.cuda.synchronize()
+        for got, want in zip(sa, (ref.attn, ref.token, ref.p_top1, ref.accepted_len, ref.out_tokens)):
+            assert torch.equal(got, want.cpu())
     for b, tb in runs[1:]:  # copies of everything, and of the larger buffers only: the same step
         for sa, sb in zip(a, b):
             assert all(torch.equal(u, w) for u, w in zip(sa, sb))
