@@ -709,16 +709,17 @@ def time_e2e(torch, dp, wl, steps, warmup, n_blocks=4):
     for i in range(warmup):
         dp.sd.decode_step_host(wl.tau, *host[i % n_blocks], dp.w_lm, attn, tok, p, None, acc, out_tok)
     torch.cuda.synchronize()
-    tokens = 0
     acc_np = acc.numpy()
+    acc_hist = np.empty((steps, B), dtype=np.int32)  # every step's accepted lengths, read from the result buffer
     t0 = time.perf_counter()
     for i in range(steps):
         if i % RESTORE_EVERY == 0:
             dp.sd.kv_restore(saved)
         dp.sd.decode_step_host(wl.tau, *host[(warmup + i) % n_blocks], dp.w_lm, attn, tok, p, None, acc, out_tok)
-        tokens += int(acc_np.clip(min=0).sum())
+        acc_hist[i] = acc_np  # the call has synchronised: the step's result is in host memory
     torch.cuda.synchronize()
     dt = time.perf_counter() - t0
+    tokens = int(acc_hist.clip(min=0).sum())
     return {"value": tokens / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
             "ms_per_step": 1e3 * dt / steps}
 
