@@ -232,6 +232,17 @@ def test_layer_pieces_reject_bad_arguments():
     with pytest.raises(pk.SdlmError):
         dp.sd.linear(torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda"),
                      torch.zeros((8, 64), dtype=torch.bfloat16, device="cuda"))   # N < 16
+    # the q / k / v product with rotary: more block rows than the context's batch, a base that is no base; nothing runs
+    d = dp.wl.shape.head_dim
+    n0 = dp.sd.launch_count()
+    z = lambda *shape: torch.zeros(shape, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(pk.SdlmError) as e:
+        dp.sd.linear3_rope(z(16, 64), z(4 * d, 64), None, z(4, 4, 2, d), z(4, 4, 1, d), z(4, 4, 1, d), 1.0e6)
+    assert e.value.code == 2                                              # SDLM_ERR_SHAPE: the context holds three sequences
+    with pytest.raises(pk.SdlmError) as e:
+        dp.sd.linear3_rope(z(12, 64), z(4 * d, 64), None, z(3, 4, 2, d), z(3, 4, 1, d), z(3, 4, 1, d), 1.0)
+    assert e.value.code == 1                                              # SDLM_ERR_INVALID_ARG
+    assert dp.sd.launch_count() == n0
 
 
 def test_two_layer_stack_step_matches_the_oracle_composition():
